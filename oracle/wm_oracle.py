@@ -1,0 +1,193 @@
+"""ctypes front end of ``wm_oracle.c`` (test infrastructure only; see the C file's header).
+
+Every function takes and returns numpy arrays on the host.  The shared object is built on
+first use into ``oracle/_build/`` with gcc; ``build()`` may be called ahead of time.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from dataclasses import dataclass
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "wm_oracle.c")
+_OUT_DIR = os.path.join(_HERE, "_build")
+_SO = os.path.join(_OUT_DIR, "libwm_oracle.so")
+_lib = None
+
+POLY_CRC32C = 0x82F63B78
+POLY_ZLIB = 0xEDB88320
+
+STATUS = {
+    0: "OK", -1: "ERR_ARG", -2: "ERR_CAPACITY", -3: "ERR_FORMAT", -4: "ERR_META_CRC",
+    -5: "ERR_STRUCT", -6: "ERR_DESC", -7: "ERR_CHUNK_CRC", -8: "ERR_STALE", -9: "ERR_CACHE_CRC",
+}
+
+
+class _CResult(ctypes.Structure):
+    _fields_ = [
+        ("status", ctypes.c_int32), ("first_bad_chunk", ctypes.c_uint32),
+        ("n_bad_chunks", ctypes.c_uint32), ("n_present", ctypes.c_uint32),
+        ("wire_len", ctypes.c_uint64), ("payload_bytes", ctypes.c_uint64),
+        ("cache_crc", ctypes.c_uint32), ("reserved", ctypes.c_uint32),
+    ]
+
+
+@dataclass
+class Result:
+    status: int
+    first_bad_chunk: int
+    n_bad_chunks: int
+    n_present: int
+    wire_len: int
+    payload_bytes: int
+    cache_crc: int
+
+    @property
+    def status_name(self) -> str:
+        return STATUS.get(self.status, str(self.status))
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc (-O2, no intrinsics) and return the path of the library."""
+    if force or not os.path.exists(_SO) or os.path.getmtime(_SO) < os.path.getmtime(_SRC):
+        os.makedirs(_OUT_DIR, exist_ok=True)
+        tmp = _SO + f".{os.getpid()}.tmp"
+        subprocess.check_call(["gcc", "-O2", "-std=c99", "-shared", "-fPIC", "-o", tmp, _SRC])
+        os.replace(tmp, _SO)
+    return _SO
+
+
+def _load():
+    global _lib
+    if _lib is not None:
+        return _lib
+    lib = ctypes.CDLL(build())
+    u8p, u32p = ctypes.c_void_p, ctypes.c_void_p
+    u64, u32 = ctypes.c_uint64, ctypes.c_uint32
+    lib.wmo_crc_bitwise.restype = u32
+    lib.wmo_crc_bitwise.argtypes = [u8p, u64, u32]
+    lib.wmo_crc32c.restype = u32
+    lib.wmo_crc32c.argtypes = [u8p, u64]
+    lib.wmo_crc_combine.restype = u32
+    lib.wmo_crc_combine.argtypes = [u32, u32, u64]
+    for name in ("wmo_num_chunks", "wmo_meta_end", "wmo_wire_bound"):
+        getattr(lib, name).restype = u64
+        getattr(lib, name).argtypes = [u64, u32]
+    lib.wmo_num_tiles.restype = u64
+    lib.wmo_num_tiles.argtypes = [u64]
+    lib.wmo_checksum.restype = ctypes.c_int
+    lib.wmo_checksum.argtypes = [u8p, u64, u32, u32p]
+    lib.wmo_dirty_diff.restype = ctypes.c_int
+    lib.wmo_dirty_diff.argtypes = [u8p, u8p, u64, u32, u8p, u32p, u32p]
+    lib.wmo_encode.restype = ctypes.c_int
+    lib.wmo_encode.argtypes = [u8p, u64, u32, u8p, u32p, u8p, u64, ctypes.POINTER(_CResult)]
+    lib.wmo_decode_verify.restype = ctypes.c_int
+    lib.wmo_decode_verify.argtypes = [u8p, u64, u8p, u64, u32, u32p, ctypes.POINTER(_CResult)]
+    _lib = lib
+    return lib
+
+
+def _bytes_view(a) -> np.ndarray:
+    a = np.ascontiguousarray(a)
+    return a.view(np.uint8).reshape(-1)
+
+
+def _ptr(a: np.ndarray) -> int:
+    return a.ctypes.data
+
+
+def _result(r: _CResult) -> Result:
+    return Result(r.status, r.first_bad_chunk, r.n_bad_chunks, r.n_present, r.wire_len,
+                  r.payload_bytes, r.cache_crc)
+
+
+def crc_bitwise(data, poly: int = POLY_CRC32C) -> int:
+    b = _bytes_view(np.frombuffer(data, dtype=np.uint8) if isinstance(data, (bytes, bytearray)) else data)
+    return int(_load().wmo_crc_bitwise(_ptr(b), b.size, poly))
+
+
+def crc32c(data) -> int:
+    b = _bytes_view(np.frombuffer(data, dtype=np.uint8) if isinstance(data, (bytes, bytearray)) else data)
+    return int(_load().wmo_crc32c(_ptr(b), b.size))
+
+
+def crc_combine(crc_a: int, crc_b: int, len_b: int) -> int:
+    return int(_load().wmo_crc_combine(crc_a, crc_b, len_b))
+
+
+def num_chunks(nbytes: int, chunk_bytes: int) -> int:
+    return int(_load().wmo_num_chunks(nbytes, chunk_bytes))
+
+
+def num_tiles(nbytes: int) -> int:
+    return int(_load().wmo_num_tiles(nbytes))
+
+
+def meta_end(nbytes: int, chunk_bytes: int) -> int:
+    return int(_load().wmo_meta_end(nbytes, chunk_bytes))
+
+
+def wire_bound(nbytes: int, chunk_bytes: int) -> int:
+    return int(_load().wmo_wire_bound(nbytes, chunk_bytes))
+
+
+def _check(status: int, what: str) -> None:
+    if status == -1:
+        raise ValueError(f"oracle {what}: bad argument")
+
+
+def checksum(cache, chunk_bytes: int) -> np.ndarray:
+    b = _bytes_view(cache)
+    out = np.zeros(num_chunks(b.size, chunk_bytes), dtype=np.uint32)
+    _check(_load().wmo_checksum(_ptr(b), b.size, chunk_bytes, _ptr(out)), "checksum")
+    return out
+
+
+def dirty_diff(cache, prev, chunk_bytes: int):
+    """Return (dirty u8[n_chunks], dirty_idx u32[n_dirty])."""
+    a, p = _bytes_view(cache), _bytes_view(prev)
+    if a.size != p.size:
+        raise ValueError("snapshots differ in size")
+    nc = num_chunks(a.size, chunk_bytes)
+    dirty = np.zeros(nc, dtype=np.uint8)
+    idx = np.zeros(nc, dtype=np.uint32)
+    n = np.zeros(1, dtype=np.uint32)
+    _check(_load().wmo_dirty_diff(_ptr(a), _ptr(p), a.size, chunk_bytes, _ptr(dirty), _ptr(idx), _ptr(n)),
+           "dirty_diff")
+    return dirty, idx[: int(n[0])].copy()
+
+
+def encode(cache, chunk_bytes: int, dirty=None, crc_in=None, wire_cap: int | None = None):
+    """Return (wire u8[wire_len or wire_cap], crc u32[n_chunks], Result)."""
+    b = _bytes_view(cache)
+    nc = num_chunks(b.size, chunk_bytes)
+    cap = wire_bound(b.size, chunk_bytes) if wire_cap is None else int(wire_cap)
+    wire = np.zeros(cap, dtype=np.uint8)
+    crc = np.zeros(nc, dtype=np.uint32) if crc_in is None else np.array(crc_in, dtype=np.uint32).copy()
+    d = None if dirty is None else np.ascontiguousarray(dirty, dtype=np.uint8)
+    res = _CResult()
+    st = _load().wmo_encode(_ptr(b), b.size, chunk_bytes, None if d is None else _ptr(d), _ptr(crc),
+                            _ptr(wire), cap, ctypes.byref(res))
+    _check(st, "encode")
+    r = _result(res)
+    if r.status == 0:
+        wire = wire[: r.wire_len].copy()
+    return wire, crc, r
+
+
+def decode_verify(wire, nbytes: int, chunk_bytes: int, dst=None, dst_crc=None, wire_len: int | None = None):
+    """Return (dst u8[nbytes], dst_crc u32[n_chunks], Result).  ``dst`` and ``dst_crc`` are
+    copied first, so the caller's arrays play the part of the live state and stay untouched."""
+    w = _bytes_view(wire)
+    nc = num_chunks(nbytes, chunk_bytes)
+    out = np.zeros(nbytes, dtype=np.uint8) if dst is None else _bytes_view(dst).copy()
+    crc = np.zeros(nc, dtype=np.uint32) if dst_crc is None else np.array(dst_crc, dtype=np.uint32).copy()
+    res = _CResult()
+    st = _load().wmo_decode_verify(_ptr(w), w.size if wire_len is None else int(wire_len), _ptr(out),
+                                   nbytes, chunk_bytes, _ptr(crc), ctypes.byref(res))
+    _check(st, "decode_verify")
+    return out, crc, _result(res)
