@@ -1,0 +1,164 @@
+/*
+ * wm.h - C ABI of the B200 data path of an exact-state session mover.
+ *
+ * The library turns a GPU-resident bf16 attention cache into a verified wire image and
+ * back: per-chunk checksums, a dirty-chunk diff against the previous snapshot, a lossless
+ * encode into one contiguous buffer, and a decode that re-fingerprints the decoded bytes
+ * so that the destination is bit-identical to the source or is not installed.
+ *
+ * Conventions for every call
+ *   - Pointers marked [dev] are device memory owned by the caller; the library allocates
+ *     nothing per call and keeps no per-session state.  Constant tables are uploaded once
+ *     per device on first use (that first call may synchronise the device).
+ *   - `stream` is a cudaStream_t passed as void*.  All work is enqueued on it; no call
+ *     synchronises.  Data-dependent outcomes arrive in `*result` [dev] on the stream.
+ *   - The return value is host-side and synchronous: WM_ERR_ARG for a bad argument
+ *     (null pointer, nbytes == 0, chunk_bytes not a multiple of 16384 or above 2^30, a
+ *     cache / wire / dst pointer that is not 16-byte aligned, a workspace that is too
+ *     small or not 16-byte aligned, wire_cap below the metadata size), WM_ERR_CUDA for
+ *     a launch failure, else WM_OK.
+ *   - Calls that share a workspace must be ordered on one stream (or by events).
+ *   - All integers in the wire image are little-endian.  Tile = 16384 bytes, group = 256
+ *     bf16 elements; n_chunks = ceil(nbytes / chunk_bytes), n_tiles = ceil(nbytes / 16384).
+ */
+#ifndef WM_H
+#define WM_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define WM_TILE_BYTES 16384u
+
+typedef enum {
+    WM_OK = 0,
+    WM_ERR_ARG = -1,        /* host-side argument check                                  */
+    WM_ERR_CAPACITY = -2,   /* encode: wire image does not fit wire_cap                  */
+    WM_ERR_FORMAT = -3,     /* decode: header does not match the call                    */
+    WM_ERR_META_CRC = -4,   /* decode: header / directory / tile table damaged           */
+    WM_ERR_STRUCT = -5,     /* decode: directory and tile table disagree                 */
+    WM_ERR_DESC = -6,       /* decode: a group descriptor is invalid                     */
+    WM_ERR_CHUNK_CRC = -7,  /* decode: a decoded chunk does not have the source's CRC    */
+    WM_ERR_STALE = -8,      /* decode: a chunk not shipped differs at the destination    */
+    WM_ERR_CACHE_CRC = -9,  /* decode: directory CRCs do not combine to the cache CRC    */
+    WM_ERR_TIMEOUT = -10,   /* a bounded device-side wait ran out                        */
+    WM_ERR_CUDA = -11       /* CUDA runtime error on launch                              */
+} wm_status;
+
+/* Outcome of wm_encode / wm_decode_verify, written on the stream.  40 bytes. */
+typedef struct {
+    int32_t  status;           /* wm_status                                              */
+    uint32_t first_bad_chunk;  /* lowest chunk failing the failing check (decode)        */
+    uint32_t n_bad_chunks;     /* chunks failing that check (decode)                     */
+    uint32_t n_present;        /* chunks carried by the wire image                       */
+    uint64_t wire_len;         /* bytes of the wire image (encode: needed size)          */
+    uint64_t payload_bytes;    /* wire_len minus metadata                                */
+    uint32_t cache_crc;        /* CRC32C of the whole cache                              */
+    uint32_t reserved;
+} wm_result;
+
+/* Geometry helpers (pure host arithmetic). */
+uint64_t wm_num_chunks(uint64_t nbytes, uint32_t chunk_bytes);
+uint64_t wm_num_tiles(uint64_t nbytes);
+/* Size of header + chunk directory + tile table, rounded up to 32 bytes. */
+uint64_t wm_meta_bytes(uint64_t nbytes, uint32_t chunk_bytes);
+/* Worst-case wire size (every tile stored raw): wm_meta_bytes + nbytes. */
+uint64_t wm_wire_bound(uint64_t nbytes, uint32_t chunk_bytes);
+/* Scratch the calls below need for this geometry (one size fits all four). */
+uint64_t wm_workspace_bytes(uint64_t nbytes, uint32_t chunk_bytes);
+
+/*
+ * wm_checksum - CRC32C of every chunk of the flat cache.
+ * Paper: the verification plane (Section 6.5: per-chunk CRC, GF(2)-combined) and the
+ * transfer / CRC-verify / rehydrate primitive (Section 4.1).  The polynomial is CRC32C
+ * (reflected 0x82F63B78, init and final xor all ones; "123456789" -> 0xE3069283).
+ *   cache     [dev] nbytes bytes, 16-byte aligned, read only
+ *   crc_out   [dev] u32[n_chunks]; crc_out[c] = CRC32C(cache[c*chunk_bytes, min((c+1)*chunk_bytes, nbytes)))
+ *   workspace [dev] wm_workspace_bytes() bytes, 16-byte aligned
+ */
+wm_status wm_checksum(const void* cache, uint64_t nbytes, uint32_t chunk_bytes,
+                      uint32_t* crc_out, void* workspace, uint64_t workspace_bytes, void* stream);
+
+/*
+ * wm_dirty_diff - which chunks changed since the previous snapshot.
+ * Paper: live pre-copy (Appendix G: round 0 ships every chunk, each later round the dirty
+ * ones) and the measured dirty fraction per generation step (Section 3.3).  The compare is
+ * exact (byte for byte), not a comparison of checksums.
+ *   cache, prev   [dev] nbytes bytes each, 16-byte aligned, read only
+ *   dirty_out     [dev] u8[n_chunks]: 1 iff any byte of the chunk differs, else 0
+ *   dirty_idx_out [dev] u32[n_chunks] or NULL: ascending indices of dirty chunks in the
+ *                 first *n_dirty_out entries (the rest is left untouched)
+ *   n_dirty_out   [dev] u32: number of dirty chunks
+ */
+wm_status wm_dirty_diff(const void* cache, const void* prev, uint64_t nbytes, uint32_t chunk_bytes,
+                        uint8_t* dirty_out, uint32_t* dirty_idx_out, uint32_t* n_dirty_out,
+                        void* workspace, uint64_t workspace_bytes, void* stream);
+
+/*
+ * wm_encode - checksum + lossless encode into one contiguous wire image (format WM1).
+ * Paper: the lossless codec inside the verified envelope (Section 6.4: bf16 plane split, the
+ * exponent plane carries the redundancy, every round trip bit-exact, receipts bind to the
+ * decoded bytes).  The paper fixes those properties, not a layout; WM1 is this library's:
+ *
+ *   header[64] | chunk_dir[16*n_chunks] | tile_tab[2*n_tiles] | zero pad to 32 | payload
+ *   header: 0 "WMV1" | 4 u16 version=1 | 6 u16 flags (bit0: a dirty mask was given) |
+ *           8 u64 nbytes | 16 u32 chunk_bytes | 20 u32 tile_bytes=16384 | 24 u32 n_chunks |
+ *           28 u32 n_present | 32 u64 payload_bytes | 40 u64 wire_len | 48 u32 cache_crc |
+ *           52 u32 meta_crc (CRC32C of the metadata with this field as zero) | 56 zero[8]
+ *   chunk_dir[c]: u64 payload_off | u32 enc_len | u32 crc
+ *   tile_tab[t] (u16): 0 tile of an absent chunk | 258..511 PACK tile of 32*value bytes |
+ *           512 RAW full tile | 0xFFFF RAW partial tail tile (nbytes mod 16384 bytes)
+ *   payload: encoded tiles of present chunks in ascending order, no padding
+ *   PACK tile (32 groups of 256 elements): desc[32] u16 (base | w<<8 | chk<<12,
+ *           chk = (base&15) ^ (base>>4) ^ w ^ 5) | SM[8192] | Epack_0 .. Epack_31.
+ *           Element v (u16): E = (v>>7)&0xFF, SM = ((v&0x7F)<<1) | (v>>15).  Per group
+ *           base = min E, w = bit length of (max E - base); a tile packs iff sum w <= 253
+ *           (length 8256 + 32*sum w), else it is stored raw.  Inside a group, element e
+ *           (memory order) has coded position k = 8*((e%64)/2) + 2*(e/64) + (e%2); SM[256 g + k]
+ *           is its SM byte and bits [k w, (k+1) w) of Epack_g (LSB-first) hold E - base.
+ *
+ *   dirty     [dev] u8[n_chunks] or NULL (NULL = every chunk present: the fused
+ *             checksum+encode of a full move)
+ *   crc_inout [dev] u32[n_chunks]: written for present chunks, read (trusted) for absent ones
+ *   wire      [dev] wire_cap bytes, 16-byte aligned; bytes beyond result->wire_len are unspecified
+ *   result    [dev] status WM_OK, WM_ERR_CAPACITY (nothing is written past wire_cap;
+ *             wire_len still reports the needed size) or WM_ERR_TIMEOUT
+ * The image is canonical: equal inputs give equal bytes in [0, wire_len).
+ */
+wm_status wm_encode(const void* cache, uint64_t nbytes, uint32_t chunk_bytes, const uint8_t* dirty,
+                    uint32_t* crc_inout, void* wire, uint64_t wire_cap,
+                    void* workspace, uint64_t workspace_bytes, wm_result* result, void* stream);
+
+/*
+ * wm_decode_verify - decode a wire image into the shadow buffer and verify it.
+ * Paper: commit only on a matching fingerprint (Section 4.1, Sufficiency: a torn state can
+ * never be installed; Table 1: migrate stages into a shadow slot, commit re-verifies).
+ * Checks, in this order; the first failing step gives result->status:
+ *   1 header fields equal the call's arguments and wire_len        WM_ERR_FORMAT
+ *   2 meta_crc                                                     WM_ERR_META_CRC
+ *   3 directory and tile table are consistent                      WM_ERR_STRUCT
+ *   4 PACK tiles in tile order: descriptors valid (WM_ERR_DESC), then 258 + sum w equals the
+ *     tile entry (WM_ERR_STRUCT); the status is that of the lowest failing tile
+ *   5 CRC32C of every decoded chunk equals its directory CRC       WM_ERR_CHUNK_CRC
+ *   6 absent chunk: dst_crc_inout[c] equals its directory CRC      WM_ERR_STALE
+ *   7 the directory CRCs combine to header.cache_crc               WM_ERR_CACHE_CRC
+ *   8 only then dst_crc_inout[c] <- crc for present chunks, status WM_OK
+ *   dst           [dev] nbytes bytes, 16-byte aligned: the SHADOW slot.  Present chunks are
+ *                 written, absent chunks are left as they are.  On any failure its content is
+ *                 unspecified (never written outside [dst, dst+nbytes)) and dst_crc_inout is
+ *                 unchanged: the caller installs (swaps in) dst only on WM_OK.
+ *   dst_crc_inout [dev] u32[n_chunks]: the receiver's CRC vector for the content of dst
+ */
+wm_status wm_decode_verify(const void* wire, uint64_t wire_len, void* dst, uint64_t nbytes,
+                           uint32_t chunk_bytes, uint32_t* dst_crc_inout,
+                           void* workspace, uint64_t workspace_bytes, wm_result* result, void* stream);
+
+/* Number of kernels the last call of each kind enqueued (for launch accounting). */
+uint32_t wm_last_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* WM_H */

@@ -1,0 +1,188 @@
+"""Thin Python binding of the C ABI in ``include/wm.h`` (argument marshalling only).
+
+Every step of the path runs in the CUDA library; torch is used for device memory and
+streams.  There is no CPU fallback: importing this module without the built library, or
+calling it without a CUDA device, raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SO = os.path.join(_HERE, "libwm.so")
+
+STATUS = {
+    0: "OK", -1: "ERR_ARG", -2: "ERR_CAPACITY", -3: "ERR_FORMAT", -4: "ERR_META_CRC", -5: "ERR_STRUCT",
+    -6: "ERR_DESC", -7: "ERR_CHUNK_CRC", -8: "ERR_STALE", -9: "ERR_CACHE_CRC", -10: "ERR_TIMEOUT",
+    -11: "ERR_CUDA",
+}
+RESULT_BYTES = 40
+EXPORTS = ("wm_num_chunks", "wm_num_tiles", "wm_meta_bytes", "wm_wire_bound", "wm_workspace_bytes",
+           "wm_checksum", "wm_dirty_diff", "wm_encode", "wm_decode_verify", "wm_last_launch_count")
+
+
+class WmError(RuntimeError):
+    pass
+
+
+def load_library() -> ctypes.CDLL:
+    if not os.path.exists(_SO):
+        raise WmError(f"{_SO} is missing: build it with `python -m paper_2607_10389_b200.build` "
+                      "(there is no CPU fallback)")
+    lib = ctypes.CDLL(_SO)
+    u64, u32, vp = ctypes.c_uint64, ctypes.c_uint32, ctypes.c_void_p
+    lib.wm_num_chunks.restype = u64
+    lib.wm_num_chunks.argtypes = [u64, u32]
+    lib.wm_num_tiles.restype = u64
+    lib.wm_num_tiles.argtypes = [u64]
+    for n in ("wm_meta_bytes", "wm_wire_bound", "wm_workspace_bytes"):
+        getattr(lib, n).restype = u64
+        getattr(lib, n).argtypes = [u64, u32]
+    lib.wm_last_launch_count.restype = u32
+    lib.wm_last_launch_count.argtypes = []
+    lib.wm_checksum.restype = ctypes.c_int
+    lib.wm_checksum.argtypes = [vp, u64, u32, vp, vp, u64, vp]
+    lib.wm_dirty_diff.restype = ctypes.c_int
+    lib.wm_dirty_diff.argtypes = [vp, vp, u64, u32, vp, vp, vp, vp, u64, vp]
+    lib.wm_encode.restype = ctypes.c_int
+    lib.wm_encode.argtypes = [vp, u64, u32, vp, vp, vp, u64, vp, u64, vp, vp]
+    lib.wm_decode_verify.restype = ctypes.c_int
+    lib.wm_decode_verify.argtypes = [vp, u64, vp, u64, u32, vp, vp, u64, vp, vp]
+    return lib
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    global _lib
+    if _lib is None:
+        _lib = load_library()
+    return _lib
+
+
+@dataclass
+class Result:
+    status: int
+    first_bad_chunk: int
+    n_bad_chunks: int
+    n_present: int
+    wire_len: int
+    payload_bytes: int
+    cache_crc: int
+
+    @property
+    def status_name(self) -> str:
+        return STATUS.get(self.status, str(self.status))
+
+    @property
+    def ok(self) -> bool:
+        return self.status == 0
+
+
+def read_result(result_dev: torch.Tensor) -> Result:
+    """Copy a 40-byte device result record to the host (synchronises the current stream)."""
+    raw = result_dev.cpu().numpy().tobytes()
+    import struct
+    st, fb, nb, npres, wl, pb, cc, _ = struct.unpack("<iIIIQQII", raw)
+    return Result(st, fb, nb, npres, wl, pb, cc)
+
+
+def num_chunks(nbytes: int, chunk_bytes: int) -> int:
+    return int(lib().wm_num_chunks(nbytes, chunk_bytes))
+
+
+def num_tiles(nbytes: int) -> int:
+    return int(lib().wm_num_tiles(nbytes))
+
+
+def meta_bytes(nbytes: int, chunk_bytes: int) -> int:
+    return int(lib().wm_meta_bytes(nbytes, chunk_bytes))
+
+
+def wire_bound(nbytes: int, chunk_bytes: int) -> int:
+    return int(lib().wm_wire_bound(nbytes, chunk_bytes))
+
+
+def workspace_bytes(nbytes: int, chunk_bytes: int) -> int:
+    return int(lib().wm_workspace_bytes(nbytes, chunk_bytes))
+
+
+def last_launch_count() -> int:
+    return int(lib().wm_last_launch_count())
+
+
+def _dev_u8(t: torch.Tensor, what: str) -> torch.Tensor:
+    if not t.is_cuda:
+        raise WmError(f"{what} must be a CUDA tensor (there is no CPU path)")
+    if not t.is_contiguous():
+        raise WmError(f"{what} must be contiguous")
+    return t
+
+
+def _stream(stream) -> int:
+    s = torch.cuda.current_stream() if stream is None else stream
+    return s.cuda_stream
+
+
+def _check(rc: int, what: str) -> None:
+    if rc != 0:
+        raise WmError(f"{what}: {STATUS.get(rc, rc)}")
+
+
+def new_workspace(nbytes: int, chunk_bytes: int, device="cuda") -> torch.Tensor:
+    n = workspace_bytes(nbytes, chunk_bytes)
+    if n == 0:
+        raise WmError("bad geometry")
+    return torch.empty(n, dtype=torch.uint8, device=device)
+
+
+def new_result(device="cuda") -> torch.Tensor:
+    return torch.zeros(RESULT_BYTES, dtype=torch.uint8, device=device)
+
+
+def wm_checksum(cache: torch.Tensor, chunk_bytes: int, crc_out: torch.Tensor, workspace: torch.Tensor,
+                stream=None) -> None:
+    _dev_u8(cache, "cache")
+    nbytes = cache.numel() * cache.element_size()
+    _check(lib().wm_checksum(cache.data_ptr(), nbytes, chunk_bytes, crc_out.data_ptr(), workspace.data_ptr(),
+                             workspace.numel(), _stream(stream)), "wm_checksum")
+
+
+def wm_dirty_diff(cache: torch.Tensor, prev: torch.Tensor, chunk_bytes: int, dirty_out: torch.Tensor,
+                  dirty_idx_out, n_dirty_out: torch.Tensor, workspace: torch.Tensor, stream=None) -> None:
+    _dev_u8(cache, "cache")
+    _dev_u8(prev, "prev")
+    nbytes = cache.numel() * cache.element_size()
+    if prev.numel() * prev.element_size() != nbytes:
+        raise WmError("snapshots differ in size")
+    _check(lib().wm_dirty_diff(cache.data_ptr(), prev.data_ptr(), nbytes, chunk_bytes, dirty_out.data_ptr(),
+                               None if dirty_idx_out is None else dirty_idx_out.data_ptr(),
+                               n_dirty_out.data_ptr(), workspace.data_ptr(), workspace.numel(),
+                               _stream(stream)), "wm_dirty_diff")
+
+
+def wm_encode(cache: torch.Tensor, chunk_bytes: int, dirty, crc_inout: torch.Tensor, wire: torch.Tensor,
+              workspace: torch.Tensor, result: torch.Tensor, stream=None, wire_cap=None) -> None:
+    _dev_u8(cache, "cache")
+    _dev_u8(wire, "wire")
+    nbytes = cache.numel() * cache.element_size()
+    cap = wire.numel() if wire_cap is None else int(wire_cap)
+    _check(lib().wm_encode(cache.data_ptr(), nbytes, chunk_bytes, None if dirty is None else dirty.data_ptr(),
+                           crc_inout.data_ptr(), wire.data_ptr(), cap, workspace.data_ptr(), workspace.numel(),
+                           result.data_ptr(), _stream(stream)), "wm_encode")
+
+
+def wm_decode_verify(wire: torch.Tensor, wire_len: int, dst: torch.Tensor, chunk_bytes: int,
+                     dst_crc_inout: torch.Tensor, workspace: torch.Tensor, result: torch.Tensor,
+                     stream=None) -> None:
+    _dev_u8(wire, "wire")
+    _dev_u8(dst, "dst")
+    nbytes = dst.numel() * dst.element_size()
+    _check(lib().wm_decode_verify(wire.data_ptr(), int(wire_len), dst.data_ptr(), nbytes, chunk_bytes,
+                                  dst_crc_inout.data_ptr(), workspace.data_ptr(), workspace.numel(),
+                                  result.data_ptr(), _stream(stream)), "wm_decode_verify")

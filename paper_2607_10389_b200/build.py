@@ -1,0 +1,37 @@
+"""Build the CUDA library (libwm.so) in-tree for sm_100a with nvcc."""
+from __future__ import annotations
+
+import os
+import subprocess
+import sys
+
+HERE = os.path.dirname(os.path.abspath(__file__))
+SRC = [os.path.join(HERE, "csrc", "wm_kernels.cu")]
+DEPS = [os.path.join(HERE, "csrc", f) for f in ("wm_kernels.cu", "wm_device.cuh", "wm_tables.h")] + [
+    os.path.join(os.path.dirname(HERE), "include", "wm.h")]
+OUT = os.path.join(HERE, "libwm.so")
+
+
+def needs_build() -> bool:
+    if not os.path.exists(OUT):
+        return True
+    t = os.path.getmtime(OUT)
+    return any(os.path.getmtime(d) > t for d in DEPS)
+
+
+def build(force: bool = False, verbose: bool = False) -> str:
+    if not force and not needs_build():
+        return OUT
+    nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
+    cmd = [nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
+           "-diag-suppress", "177", "-shared", "-Xcompiler", "-fPIC", "-o", OUT + ".tmp"] + SRC
+    if verbose:
+        cmd.insert(1, "-Xptxas")
+        cmd.insert(2, "-v")
+    subprocess.check_call(cmd)
+    os.replace(OUT + ".tmp", OUT)
+    return OUT
+
+
+if __name__ == "__main__":
+    print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))

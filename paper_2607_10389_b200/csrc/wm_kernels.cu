@@ -1,0 +1,1235 @@
+// CUDA kernels (sm_100a) and C ABI of the session mover's data path.
+//
+// Kernel map (every call enqueues a short chain on the caller's stream, no host sync):
+//   wm_checksum      : k_tile_digests -> k_checksum_finish
+//   wm_dirty_diff    : k_diff_init -> k_diff -> k_diff_compact
+//   wm_encode        : k_encode_init -> k_encode (single pass, decoupled look-back over tile
+//                      lengths) -> k_encode_finish (directory, cache CRC, header)
+//                      -> k_meta_crc (metadata CRC, result)
+//   wm_decode_verify : k_decode_init -> k_meta_crc (header + metadata CRC gate)
+//                      -> k_decode_struct_chunks -> k_decode_struct_scan (structure gate)
+//                      -> k_decode (unpack + CRC of decoded bytes) -> k_decode_finish
+#include <cstdint>
+#include <cstdio>
+#include <cstring>
+#include <mutex>
+
+#include <cuda_runtime.h>
+
+#include "../../include/wm.h"
+#include "wm_device.cuh"
+
+namespace wm {
+
+// ------------------------------------------------------------------ geometry / workspace
+
+struct Geo {
+    uint64_t nbytes;
+    uint64_t meta_end;
+    uint32_t chunk_bytes;
+    uint32_t tiles_per_chunk;
+    uint32_t n_chunks;
+    uint32_t n_tiles;
+    uint32_t tail_len;        // nbytes mod 16384 (0: the last tile is full)
+    uint32_t last_chunk_len;  // bytes of the last chunk
+    uint32_t k_tail;          // x^(8 tail_len)
+    uint32_t k_chunk;         // x^(8 chunk_bytes)
+    uint32_t k_last_chunk;    // x^(8 last_chunk_len)
+    uint32_t n_meta_slices;   // ceil(meta_end / 16384)
+};
+
+struct Ctrl {                 // first 256 bytes of the workspace
+    uint32_t ticket;
+    uint32_t poison;
+    uint32_t err;             // bit0 capacity, bit1 timeout
+    uint32_t done_a;
+    uint32_t done_b;
+    uint32_t n_present;
+    uint32_t gate;            // decode: status of an earlier failing step (0 = none)
+    uint32_t bad3_first, bad3_count;
+    uint32_t bad4_first, bad4_count;
+    uint32_t bad5_first, bad5_count;
+    uint32_t bad6_first, bad6_count;
+    uint32_t pad0;
+    unsigned long long bad4_key;   // lowest failing tile * 2 + (1 if STRUCT)
+    unsigned long long payload_total;
+    uint32_t hdr_n_present, hdr_cache_crc;
+    uint32_t pad[42];
+};
+static_assert(sizeof(Ctrl) == 256, "control block is 256 bytes");
+
+struct Ws {
+    Ctrl* ctrl;
+    unsigned long long* state;   // [n_tiles] look-back words
+    uint32_t* dig;               // [n_tiles] tile digests
+    uint32_t* rel;               // [n_tiles] decode: tile offset inside its chunk's payload
+    uint32_t* cflag;             // [n_chunks] bit0 present, bit1..: failed step 3/4/5/6
+    uint32_t* ccrc;              // [n_chunks]
+    uint32_t* mdig;              // [n_meta_slices]
+};
+
+constexpr uint32_t CF_PRESENT = 1, CF_BAD3 = 2, CF_BAD4 = 4, CF_BAD5 = 8, CF_BAD6 = 16;
+
+static inline uint64_t align16(uint64_t v) { return (v + 15) & ~(uint64_t)15; }
+
+struct WsLayout {
+    uint64_t state, dig, rel, cflag, ccrc, mdig, total;
+};
+
+static WsLayout ws_layout(const Geo& g)
+{
+    WsLayout L;
+    uint64_t o = sizeof(Ctrl);
+    L.state = o; o = align16(o + 8ull * g.n_tiles);
+    L.dig = o;   o = align16(o + 4ull * g.n_tiles);
+    L.rel = o;   o = align16(o + 4ull * g.n_tiles);
+    L.cflag = o; o = align16(o + 4ull * g.n_chunks);
+    L.ccrc = o;  o = align16(o + 4ull * g.n_chunks);
+    L.mdig = o;  o = align16(o + 4ull * g.n_meta_slices);
+    L.total = o;
+    return L;
+}
+
+static Ws ws_carve(void* base, const Geo& g)
+{
+    WsLayout L = ws_layout(g);
+    unsigned char* b = static_cast<unsigned char*>(base);
+    Ws w;
+    w.ctrl = reinterpret_cast<Ctrl*>(b);
+    w.state = reinterpret_cast<unsigned long long*>(b + L.state);
+    w.dig = reinterpret_cast<uint32_t*>(b + L.dig);
+    w.rel = reinterpret_cast<uint32_t*>(b + L.rel);
+    w.cflag = reinterpret_cast<uint32_t*>(b + L.cflag);
+    w.ccrc = reinterpret_cast<uint32_t*>(b + L.ccrc);
+    w.mdig = reinterpret_cast<uint32_t*>(b + L.mdig);
+    return w;
+}
+
+static bool make_geo(uint64_t nbytes, uint32_t chunk_bytes, Geo& g)
+{
+    if (nbytes == 0 || chunk_bytes == 0 || chunk_bytes % kTile != 0 || chunk_bytes > (1u << 30)) return false;
+    uint64_t nt = (nbytes + kTile - 1) / kTile;
+    if (nt > 0xFFFFFFFFull) return false;
+    g.nbytes = nbytes;
+    g.chunk_bytes = chunk_bytes;
+    g.tiles_per_chunk = chunk_bytes / kTile;
+    g.n_chunks = (uint32_t)((nbytes + chunk_bytes - 1) / chunk_bytes);
+    g.n_tiles = (uint32_t)nt;
+    g.meta_end = (64ull + 16ull * g.n_chunks + 2ull * g.n_tiles + 31ull) & ~31ull;
+    g.tail_len = (uint32_t)(nbytes % kTile);
+    g.last_chunk_len = (uint32_t)(nbytes - (uint64_t)(g.n_chunks - 1) * chunk_bytes);
+    g.k_tail = x_pow_bytes(g.tail_len);
+    g.k_chunk = x_pow_bytes(chunk_bytes);
+    g.k_last_chunk = x_pow_bytes(g.last_chunk_len);
+    g.n_meta_slices = (uint32_t)((g.meta_end + kTile - 1) / kTile);
+    return true;
+}
+
+__device__ __forceinline__ uint64_t chunk_len_dev(const Geo& g, uint32_t c)
+{
+    return (c + 1 == g.n_chunks) ? g.last_chunk_len : g.chunk_bytes;
+}
+
+// ------------------------------------------------------------------ per-team shared state
+
+struct TeamCtl {
+    uint32_t wtab[32];     // per group: base | w << 8
+    uint32_t wdig[8];      // per warp: its contribution to the tile digest
+    uint32_t next;         // next tile ticket (0xFFFFFFFF: stop)
+    uint32_t status;
+    unsigned long long excl;
+};
+constexpr uint32_t kTeamSmemEncode = kTile + sizeof(TeamCtl);
+constexpr uint32_t kTeamSmemPlain = sizeof(TeamCtl);
+
+// Digest of the team's current tile from the words each lane holds; result in wdig[] (valid
+// for thread 0 after the next team barrier).  `init_fold`: complement the tile's first word.
+__device__ __forceinline__ void tile_digest_to_smem(const SmemTables& T, uint32_t (&w)[kWordsPerLane], bool init_fold,
+                                                    uint32_t warp, uint32_t lane, TeamCtl* tc)
+{
+    const uint32_t m = (init_fold && warp == 0 && lane == 0) ? 0xFFFFFFFFu : 0u;
+    w[0] ^= m;
+    uint32_t d = warp_block_digest(T, w, lane);
+    w[0] ^= m;
+    uint32_t v = warp_place(T, d, warp, lane);
+    if (lane == 0) tc->wdig[warp] = v;
+}
+
+__device__ __forceinline__ uint32_t team_digest(const TeamCtl* tc)
+{
+    uint32_t d = 0;
+#pragma unroll
+    for (int i = 0; i < 8; i++) d ^= tc->wdig[i];
+    return d;
+}
+
+// CRC32C of chunk c from its tiles' digests (Horner over tiles; the all-ones init was folded
+// into the first tile's digest, the final complement is applied here).
+__device__ uint32_t chunk_crc_from_digests(const Geo& g, const uint32_t* HT, const uint32_t* T0,
+                                           const uint32_t* dig, const unsigned char* bytes, uint32_t c)
+{
+    const uint64_t clen = chunk_len_dev(g, c);
+    if (clen < 4) return crc_bytewise(T0, bytes + (uint64_t)c * g.chunk_bytes, (uint32_t)clen);
+    const uint32_t t0 = c * g.tiles_per_chunk;
+    const uint32_t ntc = (uint32_t)((clen + kTile - 1) / kTile);
+    const bool ragged = (clen % kTile) != 0;
+    uint32_t st = 0;
+    for (uint32_t i = 0; i < ntc; i++) {
+        if (i + 1 == ntc && ragged) st = mulmod_dev(st, g.k_tail);
+        else st = advance_tile(HT, st);
+        st ^= dig[t0 + i];
+    }
+    return ~st;
+}
+
+__device__ __forceinline__ void load_ht_t0(uint32_t* sHT, uint32_t* sT0, const Tables* tab)
+{
+    for (uint32_t i = threadIdx.x; i < 1024; i += blockDim.x) sHT[i] = (&tab->HT[0][0])[i];
+    for (uint32_t i = threadIdx.x; i < 256; i += blockDim.x) sT0[i] = tab->T0[i];
+    __syncthreads();
+}
+
+// CRC32C of the concatenation of all chunks from their finished CRCs (block-wide; every
+// thread of a 1024-thread block must call).  crc(A||B) = crc(A) x^(8 len B) + crc(B).
+__device__ uint32_t combine_chunk_crcs(const Geo& g, const uint32_t* crc, uint32_t stride_words, uint32_t* sbuf)
+{
+    const uint32_t n = g.n_chunks;
+    if (n == 1) return __ldcg(&crc[0]);
+    const uint32_t m = n - 1;                       // chunks of full length
+    const uint32_t T = blockDim.x;                  // 1024
+    const uint32_t R = (m + T - 1) / T;             // run per thread
+    const uint64_t pad = (uint64_t)T * R - m;       // leading empty slots
+    uint32_t acc = 0;
+    for (uint32_t s = 0; s < R; s++) {
+        uint64_t slot = (uint64_t)threadIdx.x * R + s;
+        uint32_t v = slot >= pad ? __ldcg(&crc[(slot - pad) * stride_words]) : 0u;
+        acc = (acc ? mulmod_dev(acc, g.k_chunk) : 0u) ^ v;
+    }
+    // multiplier of one run: k_chunk^R
+    uint32_t M = 0x80000000u, b = g.k_chunk;
+    for (uint32_t e = R; e; e >>= 1) {
+        if (e & 1u) M = mulmod_dev(M, b);
+        if (e > 1) b = mulmod_dev(b, b);
+    }
+    sbuf[threadIdx.x] = acc;
+    __syncthreads();
+    for (uint32_t width = T / 2; width >= 1; width >>= 1) {
+        uint32_t v = 0;
+        if (threadIdx.x < width) {
+            uint32_t a = sbuf[2 * threadIdx.x], c2 = sbuf[2 * threadIdx.x + 1];
+            v = (a ? mulmod_dev(a, M) : 0u) ^ c2;
+        }
+        __syncthreads();
+        if (threadIdx.x < width) sbuf[threadIdx.x] = v;
+        __syncthreads();
+        M = mulmod_dev(M, M);
+    }
+    uint32_t fold = sbuf[0];
+    __syncthreads();
+    return mulmod_dev(fold, g.k_last_chunk) ^ __ldcg(&crc[(uint64_t)m * stride_words]);
+}
+
+// ------------------------------------------------------------------ wm_checksum
+
+template <int TEAMS>
+__global__ void __launch_bounds__(TEAMS * 256, 1)
+k_tile_digests(const unsigned char* __restrict__ cache, Geo g, Ws ws, const Tables* __restrict__ tab)
+{
+    extern __shared__ __align__(16) unsigned char smem[];
+    SmemTables T = load_tables(smem, tab);
+    const uint32_t team = threadIdx.x / kTeamThreads, tt = threadIdx.x % kTeamThreads;
+    const uint32_t warp = tt / 32, lane = tt % 32;
+    TeamCtl* tc = reinterpret_cast<TeamCtl*>(smem + kSmemTables + team * kTeamSmemPlain);
+    const uint32_t stride = gridDim.x * TEAMS;
+    for (uint32_t t = blockIdx.x * TEAMS + team; t < g.n_tiles; t += stride) {
+        const uint64_t off = (uint64_t)t * kTile;
+        const uint64_t left = g.nbytes - off;
+        const bool first = (t % g.tiles_per_chunk) == 0;
+        uint32_t w[kWordsPerLane];
+        bool fold;
+        if (left >= kTile) { load_tile_words(cache + off, warp, lane, w); fold = first; }
+        else { load_tile_words_guarded(cache + off, (uint32_t)left, first, -8, warp, lane, w); fold = false; }
+        tile_digest_to_smem(T, w, fold, warp, lane, tc);
+        team_bar(team);
+        if (tt == 0) ws.dig[t] = team_digest(tc);
+        team_bar(team);
+    }
+}
+
+__global__ void k_checksum_finish(const unsigned char* __restrict__ cache, Geo g, Ws ws,
+                                  const Tables* __restrict__ tab, uint32_t* __restrict__ crc_out)
+{
+    __shared__ uint32_t sHT[1024];
+    __shared__ uint32_t sT0[256];
+    load_ht_t0(sHT, sT0, tab);
+    uint32_t c = blockIdx.x * blockDim.x + threadIdx.x;
+    if (c < g.n_chunks) crc_out[c] = chunk_crc_from_digests(g, sHT, sT0, ws.dig, cache, c);
+}
+
+// ------------------------------------------------------------------ wm_dirty_diff
+
+__global__ void k_diff_init(Ws ws)
+{
+    if (threadIdx.x == 0 && blockIdx.x == 0) { ws.ctrl->ticket = 0; ws.ctrl->n_present = 0; }
+}
+
+// One block per chunk at a time (ticketed); the chunk is scanned in 32 KiB steps and dropped
+// at the first step that shows a difference.
+__global__ void __launch_bounds__(256)
+k_diff(const unsigned char* __restrict__ cache, const unsigned char* __restrict__ prev, Geo g, Ws ws,
+       uint8_t* __restrict__ dirty_out)
+{
+    __shared__ uint32_t s_chunk;
+    constexpr uint32_t kStep = 256 * 16 * 8;      // bytes per block step
+    while (true) {
+        __syncthreads();
+        if (threadIdx.x == 0) s_chunk = atomicAdd(&ws.ctrl->ticket, 1u);
+        __syncthreads();
+        const uint32_t c = s_chunk;
+        if (c >= g.n_chunks) break;
+        const uint64_t base = (uint64_t)c * g.chunk_bytes;
+        const uint64_t clen = chunk_len_dev(g, c);
+        const uint64_t vec_len = clen & ~(uint64_t)15;
+        int any = 0;
+        for (uint64_t o = 0; o < vec_len; o += kStep) {
+            uint4 a[8], b[8];
+#pragma unroll
+            for (int k = 0; k < 8; k++) {
+                uint64_t p = o + ((uint64_t)k * 256 + threadIdx.x) * 16;
+                if (p < vec_len) {
+                    a[k] = __ldcs(reinterpret_cast<const uint4*>(cache + base + p));
+                    b[k] = __ldcs(reinterpret_cast<const uint4*>(prev + base + p));
+                } else {
+                    a[k] = make_uint4(0, 0, 0, 0); b[k] = a[k];
+                }
+            }
+            uint32_t d = 0;
+#pragma unroll
+            for (int k = 0; k < 8; k++)
+                d |= (a[k].x ^ b[k].x) | (a[k].y ^ b[k].y) | (a[k].z ^ b[k].z) | (a[k].w ^ b[k].w);
+            any = __syncthreads_or(d != 0);
+            if (any) break;
+        }
+        if (!any && vec_len < clen) {             // ragged tail of the last chunk, < 16 bytes
+            uint32_t d = 0;
+            if (threadIdx.x < clen - vec_len)
+                d = cache[base + vec_len + threadIdx.x] != prev[base + vec_len + threadIdx.x];
+            any = __syncthreads_or(d);
+        }
+        if (threadIdx.x == 0) dirty_out[c] = any ? 1 : 0;
+    }
+}
+
+// Ascending index list of dirty chunks and their count (one block, ballot + popc scan).
+__global__ void __launch_bounds__(1024)
+k_diff_compact(Geo g, const uint8_t* __restrict__ dirty, uint32_t* __restrict__ idx_out, uint32_t* __restrict__ n_out)
+{
+    __shared__ uint32_t s_warp[32];
+    __shared__ uint32_t s_carry;
+    const uint32_t lane = threadIdx.x % 32, warp = threadIdx.x / 32;
+    if (threadIdx.x == 0) s_carry = 0;
+    __syncthreads();
+    for (uint32_t base = 0; base < g.n_chunks; base += 1024) {
+        const uint32_t c = base + threadIdx.x;
+        const bool d = c < g.n_chunks && dirty[c] != 0;
+        const uint32_t bal = __ballot_sync(0xFFFFFFFFu, d);
+        if (lane == 0) s_warp[warp] = __popc(bal);
+        __syncthreads();
+        uint32_t before = s_carry;
+        for (uint32_t w2 = 0; w2 < warp; w2++) before += s_warp[w2];
+        if (d && idx_out) idx_out[before + __popc(bal & ((1u << lane) - 1u))] = c;
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            uint32_t tot = 0;
+            for (int w2 = 0; w2 < 32; w2++) tot += s_warp[w2];
+            s_carry += tot;
+        }
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) *n_out = s_carry;
+}
+
+// ------------------------------------------------------------------ wm_encode
+
+__global__ void k_encode_init(Geo g, Ws ws, unsigned char* wire)
+{
+    const uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
+    for (uint64_t t = i; t < g.n_tiles; t += stride) ws.state[t] = 0ull;
+    if (i < sizeof(Ctrl) / 4) reinterpret_cast<uint32_t*>(ws.ctrl)[i] = 0u;
+    // zero padding between the tile table and the payload
+    const uint64_t tab_end = 64ull + 16ull * g.n_chunks + 2ull * g.n_tiles;
+    if (i < g.meta_end - tab_end) wire[tab_end + i] = 0;
+}
+
+constexpr unsigned long long kFlagA = 1ull << 62, kFlagP = 2ull << 62, kValMask = (1ull << 62) - 1;
+constexpr uint32_t kSpinLimit = 1u << 20;
+
+// Exclusive prefix of tile lengths for tile t (warp-wide decoupled look-back; every lane of
+// one warp calls).  Tiles are claimed in ticket order, so every predecessor belongs to a
+// team that is already running and publishes its own length before it waits for anything:
+// the wait below cannot deadlock.  It is bounded all the same; when the bound is hit the
+// call is poisoned and reports WM_ERR_TIMEOUT.
+__device__ unsigned long long lookback(unsigned long long* state, uint32_t t, uint32_t len, uint32_t lane, Ctrl* ctrl)
+{
+    if (t == 0) {
+        if (lane == 0) st_volatile_u64(reinterpret_cast<uint64_t*>(&state[0]), kFlagP | len);
+        return 0;
+    }
+    if (lane == 0) st_volatile_u64(reinterpret_cast<uint64_t*>(&state[t]), kFlagA | len);
+    unsigned long long excl = 0;
+    long long hi = (long long)t - 1;
+    uint32_t polls = 0;
+    bool failed = false;
+    while (true) {
+        const long long idx = hi - (long long)lane;
+        unsigned long long v;
+        while (true) {
+            v = idx >= 0 ? ld_volatile_u64(reinterpret_cast<const uint64_t*>(&state[idx])) : kFlagP;
+            if (__all_sync(0xFFFFFFFFu, (v >> 62) != 0)) break;
+            if (++polls > kSpinLimit) { failed = true; break; }
+        }
+        if (failed) break;
+        const uint32_t pm = __ballot_sync(0xFFFFFFFFu, (v >> 62) == 2);
+        if (pm) {
+            const uint32_t first = __ffs(pm) - 1;
+            const uint32_t part = __reduce_add_sync(0xFFFFFFFFu, lane < first ? (uint32_t)(v & kValMask) : 0u);
+            const unsigned long long pv = __shfl_sync(0xFFFFFFFFu, v, first) & kValMask;
+            excl += part + pv;
+            break;
+        }
+        excl += __reduce_add_sync(0xFFFFFFFFu, (uint32_t)(v & kValMask));
+        hi -= 32;
+    }
+    if (failed) {
+        if (lane == 0) { atomicOr(&ctrl->err, 2u); atomicExch(&ctrl->poison, 1u); }
+        excl = 0;
+    }
+    if (lane == 0) st_volatile_u64(reinterpret_cast<uint64_t*>(&state[t]), kFlagP | (excl + len));
+    return excl;
+}
+
+__device__ __forceinline__ uint32_t next_ticket(Ctrl* ctrl)
+{
+    if (ld_volatile_u32(&ctrl->poison)) return 0xFFFFFFFFu;
+    return atomicAdd(&ctrl->ticket, 1u);
+}
+
+__device__ __forceinline__ uint32_t desc_of(uint32_t base, uint32_t w)
+{
+    return base | (w << 8) | ((((base & 15u) ^ (base >> 4) ^ w ^ 5u) & 15u) << 12);
+}
+
+template <int TEAMS>
+__global__ void __launch_bounds__(TEAMS * 256, 1)
+k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restrict__ dirty,
+         unsigned char* __restrict__ wire, uint64_t wire_cap, Ws ws, const Tables* __restrict__ tab)
+{
+    extern __shared__ __align__(16) unsigned char smem[];
+    SmemTables T = load_tables(smem, tab);
+    const uint32_t team = threadIdx.x / kTeamThreads, tt = threadIdx.x % kTeamThreads;
+    const uint32_t warp = tt / 32, lane = tt % 32;
+    unsigned char* out = smem + kSmemTables + team * kTeamSmemEncode;
+    TeamCtl* tc = reinterpret_cast<TeamCtl*>(out + kTile);
+    unsigned char* dir = wire + 64;
+    uint16_t* tile_tab = reinterpret_cast<uint16_t*>(wire + 64 + 16ull * g.n_chunks);
+
+    if (tt == 0) tc->next = next_ticket(ws.ctrl);
+    team_bar(team);
+    uint32_t t = tc->next;
+    uint32_t nxt[kWordsPerLane];
+    {
+        const bool ok = t < g.n_tiles && (g.nbytes - (uint64_t)t * kTile) >= kTile &&
+                        (!dirty || dirty[t / g.tiles_per_chunk]);
+        if (ok) load_tile_words(cache + (uint64_t)t * kTile, warp, lane, nxt);
+    }
+
+    while (t < g.n_tiles) {
+        uint32_t cur[kWordsPerLane];
+#pragma unroll
+        for (int i = 0; i < 16; i++) cur[i] = nxt[i];
+        const uint32_t c = t / g.tiles_per_chunk;
+        const bool first = (t % g.tiles_per_chunk) == 0;
+        const bool present = !dirty || dirty[c] != 0;
+        const uint64_t off = (uint64_t)t * kTile;
+        const uint64_t left = g.nbytes - off;
+        const bool full = left >= kTile;
+
+        team_bar(team);                                               // bar0
+        if (tt == 0) tc->next = next_ticket(ws.ctrl);
+
+        // ---- phase A: checksum digest, per-group exponent range
+        if (present) {
+            if (!full) load_tile_words_guarded(cache + off, (uint32_t)left, first, -8, warp, lane, cur);
+            tile_digest_to_smem(T, cur, first && full, warp, lane, tc);
+            if (full) {
+#pragma unroll
+                for (int j = 0; j < 4; j++) {
+                    const uint32_t a0 = cur[4 * j] & 0x7FFF7FFFu, a1 = cur[4 * j + 1] & 0x7FFF7FFFu;
+                    const uint32_t a2 = cur[4 * j + 2] & 0x7FFF7FFFu, a3 = cur[4 * j + 3] & 0x7FFF7FFFu;
+                    uint32_t mn = min_u16x2(min_u16x2(a0, a1), min_u16x2(a2, a3));
+                    uint32_t mx = max_u16x2(max_u16x2(a0, a1), max_u16x2(a2, a3));
+                    mn = min(mn & 0xFFFFu, mn >> 16);
+                    mx = max(mx & 0xFFFFu, mx >> 16);
+                    const uint32_t emin = __reduce_min_sync(0xFFFFFFFFu, mn) >> 7;
+                    const uint32_t emax = __reduce_max_sync(0xFFFFFFFFu, mx) >> 7;
+                    const uint32_t range = emax - emin;
+                    const uint32_t wd = 32u - __clz(range);
+                    if (lane == 0) tc->wtab[4 * warp + j] = emin | (wd << 8);
+                }
+            }
+        }
+        team_bar(team);                                               // bar1
+
+        // ---- prefetch the next tile while this one is packed
+        const uint32_t tn = tc->next;
+        {
+            const bool ok = tn < g.n_tiles && (g.nbytes - (uint64_t)tn * kTile) >= kTile &&
+                            (!dirty || dirty[tn / g.tiles_per_chunk]);
+            if (ok) load_tile_words(cache + (uint64_t)tn * kTile, warp, lane, nxt);
+        }
+
+        // ---- phase B: pack into shared memory (or decide RAW), look-back for the offset
+        uint32_t enc_len = 0, entry = 0;
+        bool packed = false;
+        if (present && full) {
+            const uint32_t wt = tc->wtab[lane];
+            const uint32_t wv = (wt >> 8) & 15u;
+            uint32_t incl = wv;
+#pragma unroll
+            for (int d = 1; d < 32; d <<= 1) {
+                uint32_t o = __shfl_up_sync(0xFFFFFFFFu, incl, d);
+                if (lane >= (uint32_t)d) incl += o;
+            }
+            const uint32_t S = __shfl_sync(0xFFFFFFFFu, incl, 31);
+            if (S <= 253u) {
+                packed = true;
+                enc_len = 8256u + 32u * S;
+                entry = 258u + S;
+                if (warp == 0) reinterpret_cast<uint16_t*>(out)[lane] = (uint16_t)desc_of(wt & 0xFFu, wv);
+#pragma unroll
+                for (int j = 0; j < 4; j++) {
+                    const uint32_t gi = 4 * warp + j;
+                    const uint32_t wtg = __shfl_sync(0xFFFFFFFFu, wt, gi);
+                    const uint32_t exg = __shfl_sync(0xFFFFFFFFu, incl - wv, gi);
+                    const uint32_t base = wtg & 0xFFu, wd = (wtg >> 8) & 15u;
+                    uint32_t Tr[4];
+#pragma unroll
+                    for (int r = 0; r < 4; r++) {
+                        const uint32_t W = cur[4 * j + r];
+                        Tr[r] = ((W << 1) & 0xFFFEFFFEu) | ((W >> 15) & 0x00010001u);
+                    }
+                    const uint32_t sma = __byte_perm(Tr[0], Tr[1], 0x6420), smb = __byte_perm(Tr[2], Tr[3], 0x6420);
+                    *reinterpret_cast<uint2*>(out + 64 + 256 * gi + 8 * lane) = make_uint2(sma, smb);
+                    if (wd) {
+                        const uint32_t b4 = base * 0x01010101u;
+                        const uint32_t da = __byte_perm(Tr[0], Tr[1], 0x7531) - b4;
+                        const uint32_t db = __byte_perm(Tr[2], Tr[3], 0x7531) - b4;
+                        const uint32_t sh = 8u - wd;
+                        const uint32_t ya = (da & 0x00FF00FFu) | ((da & 0xFF00FF00u) >> sh);
+                        const uint32_t yb = (db & 0x00FF00FFu) | ((db & 0xFF00FF00u) >> sh);
+                        const uint32_t za = (ya & 0xFFFFu) | ((ya >> 16) << (2 * wd));
+                        const uint32_t zb = (yb & 0xFFFFu) | ((yb >> 16) << (2 * wd));
+                        const unsigned long long P = (unsigned long long)za | ((unsigned long long)zb << (4 * wd));
+                        unsigned char* ep = out + 8256 + 32 * exg + lane * wd;
+                        if (wd == 4) *reinterpret_cast<uint32_t*>(ep) = (uint32_t)P;
+                        else if (wd == 8) *reinterpret_cast<uint2*>(ep) = make_uint2((uint32_t)P, (uint32_t)(P >> 32));
+                        else if ((wd & 1u) == 0) {
+                            for (uint32_t k = 0; k < wd; k += 2) *reinterpret_cast<uint16_t*>(ep + k) = (uint16_t)(P >> (8 * k));
+                        } else {
+                            for (uint32_t k = 0; k < wd; k++) ep[k] = (unsigned char)(P >> (8 * k));
+                        }
+                    }
+                }
+            } else {
+                enc_len = kTile;
+                entry = 512u;
+            }
+        } else if (present) {
+            enc_len = (uint32_t)left;
+            entry = 0xFFFFu;
+        }
+        if (warp == 0) {
+            const unsigned long long e = lookback(ws.state, t, enc_len, lane, ws.ctrl);
+            if (lane == 0) tc->excl = e;
+        }
+        team_bar(team);                                               // bar2
+
+        // ---- phase C: move the encoded tile to its place in the wire image
+        const unsigned long long excl = tc->excl;
+        if (present) {
+            const uint64_t dst = g.meta_end + excl;
+            if (dst + enc_len > wire_cap) {
+                if (tt == 0) atomicOr(&ws.ctrl->err, 1u);
+            } else if (packed) {
+                for (uint32_t i = tt * 16; i < enc_len; i += kTeamThreads * 16)
+                    *reinterpret_cast<uint4*>(wire + dst + i) = *reinterpret_cast<const uint4*>(out + i);
+            } else if (full) {
+                unsigned char* p = wire + dst + warp * 2048u + lane * 4u;
+#pragma unroll
+                for (int i = 0; i < 16; i++) st_stream_u32(p + i * 128, cur[i]);
+            } else {
+                for (uint32_t i = tt; i < enc_len; i += kTeamThreads) wire[dst + i] = cache[off + i];
+            }
+        }
+        if (tt == 0) {
+            tile_tab[t] = (uint16_t)entry;
+            if (present) ws.dig[t] = team_digest(tc);
+            if (first) *reinterpret_cast<unsigned long long*>(dir + 16ull * c) = excl;
+        }
+        t = tn;
+    }
+}
+
+// Directory (enc_len, crc), chunk CRCs, present count; the last block to finish combines the
+// chunk CRCs into the cache CRC and writes the header (meta_crc left zero).
+__global__ void __launch_bounds__(1024)
+k_encode_finish(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restrict__ dirty,
+                uint32_t* __restrict__ crc_inout, unsigned char* __restrict__ wire, Ws ws,
+                const Tables* __restrict__ tab)
+{
+    __shared__ uint32_t sHT[1024];
+    __shared__ uint32_t sT0[256];
+    __shared__ uint32_t sbuf[1024];
+    __shared__ bool s_last;
+    load_ht_t0(sHT, sT0, tab);
+    unsigned char* dir = wire + 64;
+    const unsigned long long total = ws.state[g.n_tiles - 1] & kValMask;
+    const uint32_t c = blockIdx.x * blockDim.x + threadIdx.x;
+    uint32_t present = 0;
+    if (c < g.n_chunks) {
+        present = (!dirty || dirty[c]) ? 1u : 0u;
+        uint32_t crc;
+        if (present) {
+            crc = chunk_crc_from_digests(g, sHT, sT0, ws.dig, cache, c);
+            crc_inout[c] = crc;
+        } else {
+            crc = crc_inout[c];
+        }
+        const unsigned long long po = *reinterpret_cast<const unsigned long long*>(dir + 16ull * c);
+        const unsigned long long nx = (c + 1 < g.n_chunks)
+                                          ? *reinterpret_cast<const unsigned long long*>(dir + 16ull * (c + 1)) : total;
+        *reinterpret_cast<uint32_t*>(dir + 16ull * c + 8) = (uint32_t)(nx - po);
+        *reinterpret_cast<uint32_t*>(dir + 16ull * c + 12) = crc;
+    }
+    __threadfence();
+    const uint32_t cnt = __syncthreads_count(present);
+    if (threadIdx.x == 0) {
+        if (cnt) atomicAdd(&ws.ctrl->n_present, cnt);
+        __threadfence();
+        s_last = atomicAdd(&ws.ctrl->done_a, 1u) == gridDim.x - 1;
+    }
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+    const uint32_t cache_crc = combine_chunk_crcs(g, reinterpret_cast<const uint32_t*>(dir + 12), 4, sbuf);
+    if (threadIdx.x == 0) {
+        const uint32_t n_present = ld_volatile_u32(&ws.ctrl->n_present);
+        uint32_t* h = reinterpret_cast<uint32_t*>(wire);
+        h[0] = 0x31564D57u;                                  // "WMV1"
+        h[1] = 1u | ((dirty ? 1u : 0u) << 16);               // version, flags
+        h[2] = (uint32_t)g.nbytes; h[3] = (uint32_t)(g.nbytes >> 32);
+        h[4] = g.chunk_bytes; h[5] = kTile; h[6] = g.n_chunks; h[7] = n_present;
+        h[8] = (uint32_t)total; h[9] = (uint32_t)(total >> 32);
+        const unsigned long long wl = g.meta_end + total;
+        h[10] = (uint32_t)wl; h[11] = (uint32_t)(wl >> 32);
+        h[12] = cache_crc; h[13] = 0u; h[14] = 0u; h[15] = 0u;
+        ws.ctrl->hdr_cache_crc = cache_crc;
+        ws.ctrl->hdr_n_present = n_present;
+        ws.ctrl->payload_total = total;
+    }
+}
+
+// CRC32C of the metadata region wire[0, meta_end) with the meta_crc field read as zero.
+// The region is right-aligned in a whole number of virtual 16 KiB slices (leading zeros),
+// one block (one team) per slice; the last block to finish folds the slice digests.
+//   mode 0 (encode): store the CRC into the header and write the result record.
+//   mode 1 (decode): check the header against the call (FORMAT), then the CRC (META_CRC);
+//                    on failure set the gate and write the result record.
+__global__ void __launch_bounds__(256, 1)
+k_meta_crc(unsigned char* wire, uint64_t wire_len, Geo g, Ws ws, const Tables* __restrict__ tab,
+           wm_result* result, int mode)
+{
+    extern __shared__ __align__(16) unsigned char smem[];
+    __shared__ bool s_last;
+    __shared__ int s_format_bad;
+    SmemTables T = load_tables(smem, tab);
+    const uint32_t warp = threadIdx.x / 32, lane = threadIdx.x % 32;
+    TeamCtl* tc = reinterpret_cast<TeamCtl*>(smem + kSmemTables);
+
+    if (mode == 1) {
+        // FORMAT check by every block (cheap, keeps the gate decision local)
+        if (threadIdx.x == 0) {
+            int bad = 0;
+            if (wire_len < 64) bad = 1;
+            else {
+                const uint32_t* h = reinterpret_cast<const uint32_t*>(wire);
+                const unsigned long long nb = h[2] | ((unsigned long long)h[3] << 32);
+                const unsigned long long pb = h[8] | ((unsigned long long)h[9] << 32);
+                const unsigned long long wl = h[10] | ((unsigned long long)h[11] << 32);
+                if (h[0] != 0x31564D57u || (h[1] & 0xFFFFu) != 1u || (h[1] >> 16) > 1u || nb != g.nbytes ||
+                    h[4] != g.chunk_bytes || h[5] != kTile || h[6] != g.n_chunks || wl != wire_len ||
+                    wire_len < g.meta_end || pb != wire_len - g.meta_end)
+                    bad = 1;
+            }
+            s_format_bad = bad;
+        }
+        __syncthreads();
+        if (s_format_bad) {
+            if (blockIdx.x == 0 && threadIdx.x == 0) {
+                ws.ctrl->gate = (uint32_t)WM_ERR_FORMAT;
+                wm_result r;
+                memset(&r, 0, sizeof r);
+                r.status = WM_ERR_FORMAT;
+                *result = r;
+            }
+            return;
+        }
+    }
+
+    const uint64_t pad = (uint64_t)g.n_meta_slices * kTile - g.meta_end;    // multiple of 4
+    const uint32_t s = blockIdx.x;
+    uint32_t w[kWordsPerLane];
+#pragma unroll
+    for (int i = 0; i < 16; i++) {
+        const uint64_t vb = (uint64_t)s * kTile + (warp * 16 + i) * 128 + lane * 4;
+        uint32_t v = 0;
+        if (vb >= pad) {
+            const uint64_t rb = vb - pad;
+            v = *reinterpret_cast<const uint32_t*>(wire + rb);
+            if (rb == 52) v = 0;
+            if (rb == 0) v ^= 0xFFFFFFFFu;
+        }
+        w[i] = v;
+    }
+    tile_digest_to_smem(T, w, false, warp, lane, tc);
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        ws.mdig[s] = team_digest(tc);
+        __threadfence();
+        s_last = atomicAdd(&ws.ctrl->done_b, 1u) == gridDim.x - 1;
+    }
+    __syncthreads();
+    if (!s_last || threadIdx.x != 0) return;
+    __threadfence();
+    uint32_t st = 0;
+    for (uint32_t i = 0; i < g.n_meta_slices; i++) {
+        st = advance_tile(&tab->HT[0][0], st);
+        st ^= ld_volatile_u32(&ws.mdig[i]);
+    }
+    const uint32_t crc = ~st;
+    if (mode == 0) {
+        reinterpret_cast<uint32_t*>(wire)[13] = crc;
+        wm_result r;
+        memset(&r, 0, sizeof r);
+        const uint32_t err = ld_volatile_u32(&ws.ctrl->err);
+        r.status = (err & 2u) ? WM_ERR_TIMEOUT : (err & 1u) ? WM_ERR_CAPACITY : WM_OK;
+        r.n_present = ws.ctrl->hdr_n_present;
+        r.payload_bytes = ws.ctrl->payload_total;
+        r.wire_len = g.meta_end + ws.ctrl->payload_total;
+        r.cache_crc = ws.ctrl->hdr_cache_crc;
+        *result = r;
+    } else {
+        const uint32_t* h = reinterpret_cast<const uint32_t*>(wire);
+        ws.ctrl->hdr_n_present = h[7];
+        ws.ctrl->hdr_cache_crc = h[12];
+        ws.ctrl->payload_total = h[8] | ((unsigned long long)h[9] << 32);
+        if (crc != h[13]) {
+            ws.ctrl->gate = (uint32_t)WM_ERR_META_CRC;
+            wm_result r;
+            memset(&r, 0, sizeof r);
+            r.status = WM_ERR_META_CRC;
+            r.n_present = h[7];
+            r.payload_bytes = ws.ctrl->payload_total;
+            r.wire_len = wire_len;
+            r.cache_crc = h[12];
+            *result = r;
+        }
+    }
+}
+
+// ------------------------------------------------------------------ wm_decode_verify
+
+__global__ void k_decode_init(Ws ws)
+{
+    if (blockIdx.x == 0 && threadIdx.x < sizeof(Ctrl) / 4) {
+        uint32_t v = 0;
+        const uint32_t i = threadIdx.x;
+        if (i == offsetof(Ctrl, bad3_first) / 4 || i == offsetof(Ctrl, bad4_first) / 4 ||
+            i == offsetof(Ctrl, bad5_first) / 4 || i == offsetof(Ctrl, bad6_first) / 4 ||
+            i == offsetof(Ctrl, bad4_key) / 4 || i == offsetof(Ctrl, bad4_key) / 4 + 1)
+            v = 0xFFFFFFFFu;
+        reinterpret_cast<uint32_t*>(ws.ctrl)[i] = v;
+    }
+}
+
+__device__ __forceinline__ void fill_result(wm_result* result, const Ctrl* ctrl, uint64_t wire_len, int status,
+                                            uint32_t first, uint32_t count)
+{
+    wm_result r;
+    memset(&r, 0, sizeof r);
+    r.status = status;
+    r.first_bad_chunk = first;
+    r.n_bad_chunks = count;
+    r.n_present = ctrl->hdr_n_present;
+    r.payload_bytes = ctrl->payload_total;
+    r.wire_len = wire_len;
+    r.cache_crc = ctrl->hdr_cache_crc;
+    *result = r;
+}
+
+// Step 3, per chunk (one warp each): tile entries against the chunk's length and enc_len;
+// also produces each tile's offset inside its chunk's payload.
+__global__ void __launch_bounds__(256)
+k_decode_struct_chunks(const unsigned char* __restrict__ wire, Geo g, Ws ws)
+{
+    if (ld_volatile_u32(&ws.ctrl->gate)) return;
+    const uint32_t lane = threadIdx.x % 32;
+    const uint32_t c = blockIdx.x * (blockDim.x / 32) + threadIdx.x / 32;
+    if (c >= g.n_chunks) return;
+    const unsigned char* dir = wire + 64;
+    const uint16_t* tab16 = reinterpret_cast<const uint16_t*>(wire + 64 + 16ull * g.n_chunks);
+    const uint64_t clen = chunk_len_dev(g, c);
+    const uint32_t t0 = c * g.tiles_per_chunk;
+    const uint32_t ntc = (uint32_t)((clen + kTile - 1) / kTile);
+    const uint32_t elen = *reinterpret_cast<const uint32_t*>(dir + 16ull * c + 8);
+    unsigned long long carry = 0;
+    bool ok = true, any = false, all = true;
+    for (uint32_t i0 = 0; i0 < ntc; i0 += 32) {
+        const uint32_t i = i0 + lane;
+        uint32_t len = 0;
+        bool l_ok = true, l_any = false, l_all = true;
+        if (i < ntc) {
+            const uint32_t e = tab16[t0 + i];
+            const uint64_t tl = clen - (uint64_t)i * kTile;
+            if (e == 0) l_all = false;
+            else {
+                l_any = true;
+                if (tl < kTile) { if (e != 0xFFFFu) l_ok = false; len = (uint32_t)tl; }
+                else if (e >= 258u && e <= 512u) len = 32u * e;
+                else l_ok = false;
+            }
+        }
+        uint32_t incl = len;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            uint32_t o = __shfl_up_sync(0xFFFFFFFFu, incl, d);
+            if (lane >= (uint32_t)d) incl += o;
+        }
+        if (i < ntc) ws.rel[t0 + i] = (uint32_t)(carry + incl - len);
+        carry += __shfl_sync(0xFFFFFFFFu, incl, 31);
+        ok = ok && __all_sync(0xFFFFFFFFu, l_ok);
+        any = any || __any_sync(0xFFFFFFFFu, l_any);
+        all = all && __all_sync(0xFFFFFFFFu, l_all);
+    }
+    if (any && !all) ok = false;
+    if (carry != elen) ok = false;
+    if (lane == 0) {
+        ws.cflag[c] = (any ? CF_PRESENT : 0u) | (ok ? 0u : CF_BAD3);
+        if (!ok) { atomicMin(&ws.ctrl->bad3_first, c); atomicAdd(&ws.ctrl->bad3_count, 1u); }
+        if (any) atomicAdd(&ws.ctrl->n_present, 1u);
+    }
+}
+
+// Step 3, across chunks (one block): payload offsets are the running sum of enc_len, the
+// totals match the header.  Sets the gate on failure.
+__global__ void __launch_bounds__(1024)
+k_decode_struct_scan(const unsigned char* __restrict__ wire, uint64_t wire_len, Geo g, Ws ws, wm_result* result)
+{
+    if (ld_volatile_u32(&ws.ctrl->gate)) return;
+    __shared__ unsigned long long s_warp[32];
+    __shared__ unsigned long long s_carry;
+    __shared__ uint32_t s_first, s_count;
+    const unsigned char* dir = wire + 64;
+    const uint32_t lane = threadIdx.x % 32, warp = threadIdx.x / 32;
+    if (threadIdx.x == 0) { s_carry = 0; s_first = 0xFFFFFFFFu; s_count = 0; }
+    __syncthreads();
+    for (uint32_t base = 0; base < g.n_chunks; base += 1024) {
+        const uint32_t c = base + threadIdx.x;
+        unsigned long long len = 0, po = 0;
+        if (c < g.n_chunks) {
+            po = *reinterpret_cast<const unsigned long long*>(dir + 16ull * c);
+            len = *reinterpret_cast<const uint32_t*>(dir + 16ull * c + 8);
+        }
+        unsigned long long incl = len;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            unsigned long long o = __shfl_up_sync(0xFFFFFFFFu, incl, d);
+            if (lane >= (uint32_t)d) incl += o;
+        }
+        if (lane == 31) s_warp[warp] = incl;
+        __syncthreads();
+        unsigned long long before = s_carry;
+        for (uint32_t w2 = 0; w2 < warp; w2++) before += s_warp[w2];
+        if (c < g.n_chunks && po != before + incl - len) {
+            // a chunk already counted by the per-chunk pass must not be counted twice
+            if (!(ws.cflag[c] & CF_BAD3)) {
+                ws.cflag[c] |= CF_BAD3;
+                atomicMin(&s_first, c);
+                atomicAdd(&s_count, 1u);
+            }
+        }
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            unsigned long long tot = 0;
+            for (int w2 = 0; w2 < 32; w2++) tot += s_warp[w2];
+            s_carry += tot;
+        }
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) {
+        uint32_t first = min(s_first, ws.ctrl->bad3_first);
+        uint32_t count = s_count + ws.ctrl->bad3_count;
+        if (count == 0 && (s_carry != ws.ctrl->payload_total || ws.ctrl->n_present != ws.ctrl->hdr_n_present)) {
+            first = 0; count = 1;
+        }
+        if (count) {
+            ws.ctrl->gate = (uint32_t)WM_ERR_STRUCT;
+            fill_result(result, ws.ctrl, wire_len, WM_ERR_STRUCT, first, count);
+        }
+    }
+}
+
+template <int TEAMS>
+__global__ void __launch_bounds__(TEAMS * 256, 1)
+k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restrict__ dst, Ws ws,
+         const Tables* __restrict__ tab)
+{
+    if (ld_volatile_u32(&ws.ctrl->gate)) return;
+    extern __shared__ __align__(16) unsigned char smem[];
+    SmemTables T = load_tables(smem, tab);
+    const uint32_t team = threadIdx.x / kTeamThreads, tt = threadIdx.x % kTeamThreads;
+    const uint32_t warp = tt / 32, lane = tt % 32;
+    TeamCtl* tc = reinterpret_cast<TeamCtl*>(smem + kSmemTables + team * kTeamSmemPlain);
+    const unsigned char* dir = wire + 64;
+    const uint16_t* tab16 = reinterpret_cast<const uint16_t*>(wire + 64 + 16ull * g.n_chunks);
+    const unsigned char* payload = wire + g.meta_end;
+
+    if (tt == 0) tc->next = atomicAdd(&ws.ctrl->ticket, 1u);
+    team_bar(team);
+    uint32_t t = tc->next;
+    while (t < g.n_tiles) {
+        team_bar(team);                                               // bar0
+        if (tt == 0) tc->next = atomicAdd(&ws.ctrl->ticket, 1u);
+        const uint32_t e = tab16[t];
+        const uint32_t c = t / g.tiles_per_chunk;
+        const bool first = (t % g.tiles_per_chunk) == 0;
+        bool have_digest = false;
+        if (e != 0) {
+            const unsigned char* src = payload + *reinterpret_cast<const unsigned long long*>(dir + 16ull * c) + ws.rel[t];
+            unsigned char* o = dst + (uint64_t)t * kTile;
+            uint32_t w[kWordsPerLane];
+            if (e == 0xFFFFu) {
+                const uint32_t len = g.tail_len;
+                for (uint32_t i = tt; i < len; i += kTeamThreads) o[i] = src[i];
+                load_tile_words_guarded(src, len, first, -8, warp, lane, w);
+                tile_digest_to_smem(T, w, false, warp, lane, tc);
+                have_digest = true;
+            } else if (e == 512u) {
+                load_tile_words(src, warp, lane, w);
+                unsigned char* p = o + warp * 2048u + lane * 4u;
+#pragma unroll
+                for (int i = 0; i < 16; i++) st_stream_u32(p + i * 128, w[i]);
+                tile_digest_to_smem(T, w, first, warp, lane, tc);
+                have_digest = true;
+            } else {
+                // PACK tile: validate the 32 descriptors (every warp does, the verdict is uniform)
+                const uint32_t desc = reinterpret_cast<const uint16_t*>(src)[lane];
+                const uint32_t base_l = desc & 0xFFu, wv = (desc >> 8) & 15u, chk = desc >> 12;
+                const bool bad = wv > 8u || chk != (((base_l & 15u) ^ (base_l >> 4) ^ wv ^ 5u) & 15u);
+                const bool anybad = __any_sync(0xFFFFFFFFu, bad);
+                uint32_t incl = wv;
+#pragma unroll
+                for (int d = 1; d < 32; d <<= 1) {
+                    uint32_t o2 = __shfl_up_sync(0xFFFFFFFFu, incl, d);
+                    if (lane >= (uint32_t)d) incl += o2;
+                }
+                const uint32_t S = __shfl_sync(0xFFFFFFFFu, incl, 31);
+                const int verdict = anybad ? 1 : (258u + S != e ? 2 : 0);
+                if (verdict) {
+                    if (tt == 0) {
+                        atomicMin(&ws.ctrl->bad4_key, (unsigned long long)t * 2ull + (verdict == 2 ? 1ull : 0ull));
+                        atomicOr(&ws.cflag[c], CF_BAD4);
+                    }
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 4; j++) {
+                        const uint32_t gi = 4 * warp + j;
+                        const uint32_t dg = __shfl_sync(0xFFFFFFFFu, desc, gi);
+                        const uint32_t exg = __shfl_sync(0xFFFFFFFFu, incl - wv, gi);
+                        const uint32_t base = dg & 0xFFu, wd = (dg >> 8) & 15u;
+                        const uint2 sm = *reinterpret_cast<const uint2*>(src + 64 + 256 * gi + 8 * lane);
+                        uint32_t ea = base * 0x01010101u, eb = ea;
+                        if (wd) {
+                            const unsigned char* rec = src + 8256 + 32 * exg;
+                            const uint32_t bo = lane * wd, a = bo & ~3u, sh = (bo & 3u) * 8u, rl = 32u * wd;
+                            const uint32_t w0 = *reinterpret_cast<const uint32_t*>(rec + a);
+                            const uint32_t w1 = (a + 4 < rl) ? *reinterpret_cast<const uint32_t*>(rec + a + 4) : 0u;
+                            const uint32_t w2 = (a + 8 < rl) ? *reinterpret_cast<const uint32_t*>(rec + a + 8) : 0u;
+                            const uint32_t lo = __funnelshift_r(w0, w1, sh), hi = __funnelshift_r(w1, w2, sh);
+                            const unsigned long long P = (unsigned long long)lo | ((unsigned long long)hi << 32);
+                            const uint32_t m4 = (wd == 8) ? 0xFFFFFFFFu : ((1u << (4 * wd)) - 1u);
+                            const uint32_t za = (uint32_t)P & m4, zb = (uint32_t)(P >> (4 * wd)) & m4;
+                            const uint32_t m2 = (1u << (2 * wd)) - 1u;
+                            const uint32_t ya = (za & m2) | ((za >> (2 * wd)) << 16);
+                            const uint32_t yb = (zb & m2) | ((zb >> (2 * wd)) << 16);
+                            const uint32_t m1 = ((1u << wd) - 1u) * 0x00010001u;
+                            const uint32_t da = (ya & m1) | ((ya & (m1 << wd)) << (8 - wd));
+                            const uint32_t db = (yb & m1) | ((yb & (m1 << wd)) << (8 - wd));
+                            // per-byte (base + d) & 0xFF
+                            const uint32_t b4 = ea;
+                            ea = ((da & 0x7F7F7F7Fu) + (b4 & 0x7F7F7F7Fu)) ^ ((da ^ b4) & 0x80808080u);
+                            eb = ((db & 0x7F7F7F7Fu) + (b4 & 0x7F7F7F7Fu)) ^ ((db ^ b4) & 0x80808080u);
+                        }
+                        uint32_t Tr[4];
+                        Tr[0] = __byte_perm(sm.x, ea, 0x5140);
+                        Tr[1] = __byte_perm(sm.x, ea, 0x7362);
+                        Tr[2] = __byte_perm(sm.y, eb, 0x5140);
+                        Tr[3] = __byte_perm(sm.y, eb, 0x7362);
+#pragma unroll
+                        for (int r = 0; r < 4; r++)
+                            w[4 * j + r] = ((Tr[r] >> 1) & 0x7FFF7FFFu) | ((Tr[r] << 15) & 0x80008000u);
+                    }
+                    unsigned char* p = o + warp * 2048u + lane * 4u;
+#pragma unroll
+                    for (int i = 0; i < 16; i++) st_stream_u32(p + i * 128, w[i]);
+                    tile_digest_to_smem(T, w, first, warp, lane, tc);
+                    have_digest = true;
+                }
+            }
+        }
+        team_bar(team);                                               // bar1
+        if (tt == 0 && have_digest) ws.dig[t] = team_digest(tc);
+        t = tc->next;
+    }
+}
+
+// Steps 5..8: chunk CRCs of the decoded bytes against the directory, stale check, cache CRC;
+// the last block to finish decides the status and, on success only, updates dst_crc_inout.
+__global__ void __launch_bounds__(1024)
+k_decode_finish(const unsigned char* __restrict__ wire, uint64_t wire_len, Geo g,
+                const unsigned char* __restrict__ dst, uint32_t* __restrict__ dst_crc, Ws ws,
+                const Tables* __restrict__ tab, wm_result* result)
+{
+    if (ld_volatile_u32(&ws.ctrl->gate)) return;
+    __shared__ uint32_t sHT[1024];
+    __shared__ uint32_t sT0[256];
+    __shared__ uint32_t sbuf[1024];
+    __shared__ bool s_last;
+    __shared__ int s_status;
+    load_ht_t0(sHT, sT0, tab);
+    const unsigned char* dir = wire + 64;
+    const uint32_t c = blockIdx.x * blockDim.x + threadIdx.x;
+    const bool step4_failed = ld_volatile_u32(reinterpret_cast<const uint32_t*>(&ws.ctrl->bad4_key)) != 0xFFFFFFFFu ||
+                              ld_volatile_u32(reinterpret_cast<const uint32_t*>(&ws.ctrl->bad4_key) + 1) != 0xFFFFFFFFu;
+    if (c < g.n_chunks) {
+        const uint32_t fl = ws.cflag[c];
+        const uint32_t want = *reinterpret_cast<const uint32_t*>(dir + 16ull * c + 12);
+        if (step4_failed) {
+            if (fl & CF_BAD4) { atomicMin(&ws.ctrl->bad4_first, c); atomicAdd(&ws.ctrl->bad4_count, 1u); }
+        } else if (fl & CF_PRESENT) {
+            const uint32_t got = chunk_crc_from_digests(g, sHT, sT0, ws.dig, dst, c);
+            if (got != want) { atomicMin(&ws.ctrl->bad5_first, c); atomicAdd(&ws.ctrl->bad5_count, 1u); }
+        } else {
+            if (dst_crc[c] != want) { atomicMin(&ws.ctrl->bad6_first, c); atomicAdd(&ws.ctrl->bad6_count, 1u); }
+        }
+    }
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        __threadfence();
+        s_last = atomicAdd(&ws.ctrl->done_a, 1u) == gridDim.x - 1;
+    }
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+    const uint32_t cache_crc = combine_chunk_crcs(g, reinterpret_cast<const uint32_t*>(dir + 12), 4, sbuf);
+    if (threadIdx.x == 0) {
+        int status = WM_OK;
+        uint32_t first = 0, count = 0;
+        const unsigned long long key = *reinterpret_cast<volatile unsigned long long*>(&ws.ctrl->bad4_key);
+        if (key != ~0ull) {
+            status = (key & 1ull) ? WM_ERR_STRUCT : WM_ERR_DESC;
+            first = ld_volatile_u32(&ws.ctrl->bad4_first); count = ld_volatile_u32(&ws.ctrl->bad4_count);
+        } else if (ld_volatile_u32(&ws.ctrl->bad5_count)) {
+            status = WM_ERR_CHUNK_CRC;
+            first = ld_volatile_u32(&ws.ctrl->bad5_first); count = ld_volatile_u32(&ws.ctrl->bad5_count);
+        } else if (ld_volatile_u32(&ws.ctrl->bad6_count)) {
+            status = WM_ERR_STALE;
+            first = ld_volatile_u32(&ws.ctrl->bad6_first); count = ld_volatile_u32(&ws.ctrl->bad6_count);
+        } else if (cache_crc != ws.ctrl->hdr_cache_crc) {
+            status = WM_ERR_CACHE_CRC;
+        }
+        fill_result(result, ws.ctrl, wire_len, status, first, count);
+        s_status = status;
+    }
+    __syncthreads();
+    if (s_status == WM_OK) {
+        for (uint32_t i = threadIdx.x; i < g.n_chunks; i += blockDim.x)
+            if (ws.cflag[i] & CF_PRESENT) dst_crc[i] = *reinterpret_cast<const uint32_t*>(dir + 16ull * i + 12);
+    }
+}
+
+// ------------------------------------------------------------------ host side
+
+constexpr int kTeams = 3;
+
+struct DeviceState {
+    Tables* tables = nullptr;
+    int sm_count = 0;
+    bool ready = false;
+};
+static DeviceState g_dev[64];
+static std::mutex g_mutex;
+static thread_local uint32_t g_launches = 0;
+
+static const DeviceState* device_state()
+{
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    std::lock_guard<std::mutex> lock(g_mutex);
+    DeviceState& s = g_dev[dev];
+    if (s.ready) return &s;
+    static Tables host;
+    build_tables(host);
+    if (cudaMalloc(&s.tables, sizeof(Tables)) != cudaSuccess) return nullptr;
+    if (cudaMemcpy(s.tables, &host, sizeof(Tables), cudaMemcpyHostToDevice) != cudaSuccess) return nullptr;
+    if (cudaDeviceGetAttribute(&s.sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return nullptr;
+    const int big = kSmemTables + kTeams * kTeamSmemEncode;
+    if (cudaFuncSetAttribute(k_encode<kTeams>, cudaFuncAttributeMaxDynamicSharedMemorySize, big) != cudaSuccess) return nullptr;
+    if (cudaFuncSetAttribute(k_decode<kTeams>, cudaFuncAttributeMaxDynamicSharedMemorySize, big) != cudaSuccess) return nullptr;
+    if (cudaFuncSetAttribute(k_tile_digests<kTeams>, cudaFuncAttributeMaxDynamicSharedMemorySize, big) != cudaSuccess) return nullptr;
+    if (cudaFuncSetAttribute(k_meta_crc, cudaFuncAttributeMaxDynamicSharedMemorySize, big) != cudaSuccess) return nullptr;
+    s.ready = true;
+    return &s;
+}
+
+static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+static wm_status launch_status()
+{
+    return cudaGetLastError() == cudaSuccess ? WM_OK : WM_ERR_CUDA;
+}
+
+}  // namespace wm
+
+using namespace wm;
+
+extern "C" {
+
+uint64_t wm_num_chunks(uint64_t nbytes, uint32_t chunk_bytes)
+{
+    return chunk_bytes ? (nbytes + chunk_bytes - 1) / chunk_bytes : 0;
+}
+
+uint64_t wm_num_tiles(uint64_t nbytes) { return (nbytes + kTile - 1) / kTile; }
+
+uint64_t wm_meta_bytes(uint64_t nbytes, uint32_t chunk_bytes)
+{
+    return (64ull + 16ull * wm_num_chunks(nbytes, chunk_bytes) + 2ull * wm_num_tiles(nbytes) + 31ull) & ~31ull;
+}
+
+uint64_t wm_wire_bound(uint64_t nbytes, uint32_t chunk_bytes) { return wm_meta_bytes(nbytes, chunk_bytes) + nbytes; }
+
+uint64_t wm_workspace_bytes(uint64_t nbytes, uint32_t chunk_bytes)
+{
+    Geo g;
+    if (!make_geo(nbytes, chunk_bytes, g)) return 0;
+    return ws_layout(g).total;
+}
+
+uint32_t wm_last_launch_count(void) { return g_launches; }
+
+wm_status wm_checksum(const void* cache, uint64_t nbytes, uint32_t chunk_bytes, uint32_t* crc_out,
+                      void* workspace, uint64_t workspace_bytes, void* stream)
+{
+    Geo g;
+    if (!cache || !crc_out || !workspace || !make_geo(nbytes, chunk_bytes, g)) return WM_ERR_ARG;
+    if (!aligned16(cache) || !aligned16(workspace) || workspace_bytes < ws_layout(g).total) return WM_ERR_ARG;
+    const DeviceState* ds = device_state();
+    if (!ds) return WM_ERR_CUDA;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    Ws ws = ws_carve(workspace, g);
+    const unsigned char* c = static_cast<const unsigned char*>(cache);
+    const uint32_t need = (g.n_tiles + kTeams - 1) / kTeams;
+    const uint32_t grid = need < (uint32_t)ds->sm_count ? need : (uint32_t)ds->sm_count;
+    k_tile_digests<kTeams><<<grid, kTeams * 256, kSmemTables + kTeams * kTeamSmemPlain, s>>>(c, g, ws, ds->tables);
+    k_checksum_finish<<<(g.n_chunks + 255) / 256, 256, 0, s>>>(c, g, ws, ds->tables, crc_out);
+    g_launches = 2;
+    return launch_status();
+}
+
+wm_status wm_dirty_diff(const void* cache, const void* prev, uint64_t nbytes, uint32_t chunk_bytes,
+                        uint8_t* dirty_out, uint32_t* dirty_idx_out, uint32_t* n_dirty_out,
+                        void* workspace, uint64_t workspace_bytes, void* stream)
+{
+    Geo g;
+    if (!cache || !prev || !dirty_out || !n_dirty_out || !workspace || !make_geo(nbytes, chunk_bytes, g)) return WM_ERR_ARG;
+    if (!aligned16(cache) || !aligned16(prev) || !aligned16(workspace) || workspace_bytes < ws_layout(g).total) return WM_ERR_ARG;
+    const DeviceState* ds = device_state();
+    if (!ds) return WM_ERR_CUDA;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    Ws ws = ws_carve(workspace, g);
+    k_diff_init<<<1, 32, 0, s>>>(ws);
+    const uint32_t want = (uint32_t)ds->sm_count * 4;
+    const uint32_t grid = g.n_chunks < want ? g.n_chunks : want;
+    k_diff<<<grid, 256, 0, s>>>(static_cast<const unsigned char*>(cache), static_cast<const unsigned char*>(prev), g, ws, dirty_out);
+    k_diff_compact<<<1, 1024, 0, s>>>(g, dirty_out, dirty_idx_out, n_dirty_out);
+    g_launches = 3;
+    return launch_status();
+}
+
+wm_status wm_encode(const void* cache, uint64_t nbytes, uint32_t chunk_bytes, const uint8_t* dirty,
+                    uint32_t* crc_inout, void* wire, uint64_t wire_cap, void* workspace, uint64_t workspace_bytes,
+                    wm_result* result, void* stream)
+{
+    Geo g;
+    if (!cache || !crc_inout || !wire || !workspace || !result || !make_geo(nbytes, chunk_bytes, g)) return WM_ERR_ARG;
+    if (!aligned16(cache) || !aligned16(wire) || !aligned16(workspace) || workspace_bytes < ws_layout(g).total ||
+        wire_cap < g.meta_end)
+        return WM_ERR_ARG;
+    const DeviceState* ds = device_state();
+    if (!ds) return WM_ERR_CUDA;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    Ws ws = ws_carve(workspace, g);
+    const unsigned char* c = static_cast<const unsigned char*>(cache);
+    unsigned char* w = static_cast<unsigned char*>(wire);
+    const uint32_t init_blocks = (g.n_tiles + 1023) / 1024 < 1024 ? (g.n_tiles + 1023) / 1024 : 1024;
+    k_encode_init<<<init_blocks ? init_blocks : 1, 1024, 0, s>>>(g, ws, w);
+    const uint32_t need = (g.n_tiles + kTeams - 1) / kTeams;
+    const uint32_t grid = need < (uint32_t)ds->sm_count ? need : (uint32_t)ds->sm_count;
+    k_encode<kTeams><<<grid, kTeams * 256, kSmemTables + kTeams * kTeamSmemEncode, s>>>(c, g, dirty, w, wire_cap, ws, ds->tables);
+    k_encode_finish<<<(g.n_chunks + 1023) / 1024, 1024, 0, s>>>(c, g, dirty, crc_inout, w, ws, ds->tables);
+    k_meta_crc<<<g.n_meta_slices, 256, kSmemTables + kTeamSmemPlain, s>>>(w, 0, g, ws, ds->tables, result, 0);
+    g_launches = 4;
+    return launch_status();
+}
+
+wm_status wm_decode_verify(const void* wire, uint64_t wire_len, void* dst, uint64_t nbytes, uint32_t chunk_bytes,
+                           uint32_t* dst_crc_inout, void* workspace, uint64_t workspace_bytes, wm_result* result,
+                           void* stream)
+{
+    Geo g;
+    if (!wire || !dst || !dst_crc_inout || !workspace || !result || !make_geo(nbytes, chunk_bytes, g)) return WM_ERR_ARG;
+    if (!aligned16(wire) || !aligned16(dst) || !aligned16(workspace) || workspace_bytes < ws_layout(g).total) return WM_ERR_ARG;
+    const DeviceState* ds = device_state();
+    if (!ds) return WM_ERR_CUDA;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    Ws ws = ws_carve(workspace, g);
+    const unsigned char* w = static_cast<const unsigned char*>(wire);
+    unsigned char* d = static_cast<unsigned char*>(dst);
+    k_decode_init<<<1, 64, 0, s>>>(ws);
+    // a wire shorter than the metadata is rejected by the header check before anything else is read
+    const uint32_t slices = wire_len >= g.meta_end ? g.n_meta_slices : 1;
+    k_meta_crc<<<slices, 256, kSmemTables + kTeamSmemPlain, s>>>(const_cast<unsigned char*>(w), wire_len, g, ws, ds->tables, result, 1);
+    k_decode_struct_chunks<<<(g.n_chunks + 7) / 8, 256, 0, s>>>(w, g, ws);
+    k_decode_struct_scan<<<1, 1024, 0, s>>>(w, wire_len, g, ws, result);
+    const uint32_t need = (g.n_tiles + kTeams - 1) / kTeams;
+    const uint32_t grid = need < (uint32_t)ds->sm_count ? need : (uint32_t)ds->sm_count;
+    k_decode<kTeams><<<grid, kTeams * 256, kSmemTables + kTeams * kTeamSmemPlain, s>>>(w, g, d, ws, ds->tables);
+    k_decode_finish<<<(g.n_chunks + 1023) / 1024, 1024, 0, s>>>(w, wire_len, g, d, dst_crc_inout, ws, ds->tables, result);
+    g_launches = 6;
+    return launch_status();
+}
+
+}  // extern "C"
