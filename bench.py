@@ -1,0 +1,409 @@
+#!/usr/bin/env python
+"""Benchmark of the session mover's data path on B200.
+
+One "step" is one pass of the whole path over one synthetic cache that is already resident
+in HBM: wm_checksum -> wm_dirty_diff (against a snapshot with three quarters of the chunks
+rewritten) -> wm_encode (full move: fused checksum + encode) -> wm_decode_verify into a shadow
+buffer.  `value` is raw cache bytes per second through that whole step; the per-call rates
+(the metric's "checksum+encode" and "decode+verify" figures) are in `calls`.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload engine] [--impl reference]
+
+N > 1 runs one independent replica per GPU (the path has no exchange step): launch with
+torch.distributed.run; rank 0 prints the one JSON line.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+FALLBACK_HBM_GBS = 6650.0
+# DRAM bytes per launch of the dominant kernel from an ncu capture (profiles/), or None.
+NCU_TRAFFIC_BYTES = {}
+
+
+def _peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            return float(json.load(open(p))["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clock, power and throttle reasons of one GPU through NVML while running."""
+
+    def __init__(self, index: int, uuid: str | None = None, period_s: float = 0.01):
+        self.index, self.uuid, self.period = index, uuid, period_s
+        self.samples, self._stop, self._thread = [], threading.Event(), None
+        self.max_mhz = None
+
+    def _run(self):
+        try:
+            import pynvml as nv
+            nv.nvmlInit()
+            h = None
+            if self.uuid:
+                try:
+                    h = nv.nvmlDeviceGetHandleByUUID(self.uuid)
+                except Exception:
+                    h = None
+            if h is None:
+                h = nv.nvmlDeviceGetHandleByIndex(self.index)
+            self.max_mhz = nv.nvmlDeviceGetMaxClockInfo(h, nv.NVML_CLOCK_SM)
+            while not self._stop.is_set():
+                mhz = nv.nvmlDeviceGetClockInfo(h, nv.NVML_CLOCK_SM)
+                try:
+                    reasons = nv.nvmlDeviceGetCurrentClocksEventReasons(h)
+                except Exception:
+                    reasons = nv.nvmlDeviceGetCurrentClocksThrottleReasons(h)
+                try:
+                    watts = nv.nvmlDeviceGetPowerUsage(h) / 1000.0
+                except Exception:
+                    watts = None
+                self.samples.append((mhz, reasons, watts))
+                time.sleep(self.period)
+        except Exception as e:  # NVML missing: report that instead of inventing clocks
+            self.samples.append(("error", str(e), None))
+
+    def __enter__(self):
+        self._thread = threading.Thread(target=self._run, daemon=True)
+        self._thread.start()
+        return self
+
+    def __exit__(self, *a):
+        self._stop.set()
+        self._thread.join(timeout=2)
+
+    def summary(self):
+        good = [s for s in self.samples if s[0] != "error"]
+        if not good:
+            return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": ["nvml_unavailable"], "samples": 0}
+        names = {0x8: "hw_slowdown", 0x40: "hw_thermal_slowdown", 0x20: "sw_thermal_slowdown",
+                 0x4: "sw_power_cap", 0x80: "hw_power_brake", 0x2: "applications_clocks_setting"}
+        seen = set()
+        for _, r, _ in good:
+            for bit, n in names.items():
+                if r & bit:
+                    seen.add(n)
+        watts = [w for _, _, w in good if w is not None]
+        return {"sm_mhz": statistics.median(s[0] for s in good), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(seen), "samples": len(good), "power_w_max": max(watts) if watts else None}
+
+
+def _dist():
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    return int(os.environ.get("RANK", "0")), int(os.environ.get("LOCAL_RANK", "0")), world
+
+
+def oracle_step(sample_cur, sample_prev, chunk_bytes):
+    """The CPU oracle's pass over one sample (same four calls as the GPU step)."""
+    import numpy as np
+    import oracle
+    crc = oracle.checksum(sample_cur, chunk_bytes)
+    dirty, _ = oracle.dirty_diff(sample_cur, sample_prev, chunk_bytes)
+    wire, crc2, res = oracle.encode(sample_cur, chunk_bytes)
+    out, _, r = oracle.decode_verify(wire, sample_cur.size, chunk_bytes)
+    assert res.status == 0 and r.status == 0 and np.array_equal(out, sample_cur) and np.array_equal(crc, crc2)
+    return int(dirty.sum())
+
+
+def cpu_baseline(cur_host, prev_host, chunk_bytes, target_s=12.0):
+    """Time the oracle, as it stands, on a bounded sample of the workload."""
+    n0 = min(cur_host.size, 8 * chunk_bytes)
+    t = time.perf_counter()
+    oracle_step(cur_host[:n0], prev_host[:n0], chunk_bytes)
+    dt = time.perf_counter() - t
+    chunks = max(8, min(cur_host.size // chunk_bytes, int(target_s / max(dt, 1e-6) * 8)))
+    n = min(cur_host.size, chunks * chunk_bytes)
+    t = time.perf_counter()
+    oracle_step(cur_host[:n], prev_host[:n], chunk_bytes)
+    dt = time.perf_counter() - t
+    return {"value": n / dt / 1e9, "unit": "GB/s", "cores": 1, "kind": "oracle",
+            "sample": f"first {n} bytes ({n // chunk_bytes} chunks) of the workload, one pass of "
+                      f"checksum+diff+encode+decode_verify, {dt:.1f} s, single thread"}
+
+
+def make_workload(name, device):
+    import torch
+    from paper_2607_10389_b200 import inputs
+    cfg = inputs.CONFIGS[name]
+    cur = inputs.make_cache(cfg, device)
+    # previous snapshot: the same cache before a generation step rewrote 75 % of its chunks
+    nc = (cfg.nbytes + cfg.chunk_bytes - 1) // cfg.chunk_bytes
+    mask = inputs.step_pattern(nc, 30, 0.75, seed=cfg.seed + 100)
+    prev = cur.clone()
+    inputs.apply_step(prev, cfg.chunk_bytes, mask, seed=cfg.seed + 200)
+    torch.cuda.synchronize()
+    return cfg, cur, prev, int(mask.sum())
+
+
+def run_reference(args):
+    """Reference arm: the CPU oracle timed on the host cores, a bounded sample per step."""
+    rank, _, world = _dist()
+    if rank != 0:
+        return
+    import numpy as np
+    from paper_2607_10389_b200 import inputs
+    name = args.workload
+    cfg = inputs.CONFIGS[name]
+    sample_chunks = 16
+    n = min(cfg.nbytes, sample_chunks * cfg.chunk_bytes)
+    # the sample is the head of a reduced cache of the same recipe (drawn on the CPU)
+    small = inputs.CONFIGS["engine_small"] if cfg.kind == "kv" else cfg
+    cur = inputs.make_cache(small, "cpu").numpy()
+    reps = -(-n // cur.size)
+    cur = np.tile(cur, reps)[:n].copy()
+    prev = cur.copy()
+    nc = n // cfg.chunk_bytes
+    mask = inputs.step_pattern(nc, 1, 0.75, seed=cfg.seed + 100).numpy()
+    rng = np.random.default_rng(cfg.seed)
+    for c in np.nonzero(mask)[0]:
+        prev[c * cfg.chunk_bytes:(c + 1) * cfg.chunk_bytes] = rng.integers(0, 256, cfg.chunk_bytes, dtype=np.uint8)
+    for _ in range(args.warmup):
+        oracle_step(cur, prev, cfg.chunk_bytes)
+    t = time.perf_counter()
+    for _ in range(args.steps):
+        oracle_step(cur, prev, cfg.chunk_bytes)
+    dt = (time.perf_counter() - t) / args.steps
+    v = n / dt / 1e9
+    sample = f"{n} bytes ({nc} chunks of {cfg.chunk_bytes}) of the {name} recipe per step, single thread"
+    print(json.dumps({
+        "impl": "reference", "metric": "raw-cache GB/s through checksum+diff+encode+decode_verify",
+        "value": v, "unit": "GB/s", "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "u8", "data": "synthetic",
+        "config": {"workload": name, "nbytes": cfg.nbytes, "chunk_bytes": cfg.chunk_bytes, "sample_bytes": n},
+        "cpu_baseline": {"value": v, "unit": "GB/s", "cores": 1, "kind": "oracle", "sample": sample},
+        "e2e": {"value": v, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=None)
+    ap.add_argument("--workload", default="engine")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--profile", action="store_true",
+                    help="profiler capture mode: round-trip check, warm-up and timed steps only")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        args.steps = 3 if args.steps is None else args.steps
+        args.warmup = 1 if args.warmup is None else args.warmup
+        return run_reference(args)
+    args.steps = 100 if args.steps is None else args.steps
+    args.warmup = 5 if args.warmup is None else max(args.warmup, 3)
+    if args.profile:
+        args.no_e2e = args.no_cpu_baseline = True
+
+    import numpy as np
+    import torch
+    from paper_2607_10389_b200 import binding as wm
+
+    rank, local_rank, world = _dist()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+
+    def barrier():
+        if world > 1:
+            torch.distributed.barrier()
+        torch.cuda.synchronize()
+
+    def max_over_ranks(x: float) -> float:
+        if world == 1:
+            return x
+        t = torch.tensor([x], dtype=torch.float64, device=dev)
+        torch.distributed.all_reduce(t, op=torch.distributed.ReduceOp.MAX)
+        return float(t.item())
+
+    cfg, cur, prev, n_rewritten = make_workload(args.workload, dev)
+    N, C = cfg.nbytes, cfg.chunk_bytes
+    nc = wm.num_chunks(N, C)
+    ws = wm.new_workspace(N, C, dev)
+    cap = wm.wire_bound(N, C)
+    wire = torch.empty(cap, dtype=torch.uint8, device=dev)
+    shadow = torch.empty(N, dtype=torch.uint8, device=dev)
+    crc_a = torch.zeros(nc, dtype=torch.int32, device=dev)
+    crc_b = torch.zeros(nc, dtype=torch.int32, device=dev)
+    crc_dst = torch.zeros(nc, dtype=torch.int32, device=dev)
+    dirty = torch.zeros(nc, dtype=torch.uint8, device=dev)
+    dirty_idx = torch.zeros(nc, dtype=torch.int32, device=dev)
+    n_dirty = torch.zeros(1, dtype=torch.int32, device=dev)
+    res_e, res_d = wm.new_result(dev), wm.new_result(dev)
+
+    state = {"wire_len": cap}
+    launches = {"n": 0}
+
+    def call_checksum():
+        wm.wm_checksum(cur, C, crc_a, ws)
+        launches["n"] += wm.last_launch_count()
+
+    def call_diff():
+        wm.wm_dirty_diff(cur, prev, C, dirty, dirty_idx, n_dirty, ws)
+        launches["n"] += wm.last_launch_count()
+
+    def call_encode():
+        wm.wm_encode(cur, C, None, crc_b, wire, ws, res_e)
+        launches["n"] += wm.last_launch_count()
+
+    def call_decode():
+        wm.wm_decode_verify(wire, state["wire_len"], shadow, C, crc_dst, ws, res_d)
+        launches["n"] += wm.last_launch_count()
+
+    def step():
+        call_checksum()
+        call_diff()
+        call_encode()
+        call_decode()
+
+    # first pass: learn wire_len, check the round trip before timing anything
+    call_encode()
+    r = wm.read_result(res_e)
+    if not r.ok:
+        raise SystemExit(f"encode failed: {r.status_name}")
+    state["wire_len"] = r.wire_len
+    step()
+    rd = wm.read_result(res_d)
+    if not rd.ok or not torch.equal(shadow, cur) or not torch.equal(crc_a, crc_b) or not torch.equal(crc_dst, crc_b):
+        raise SystemExit(f"round trip failed: {rd.status_name}")
+    if int(n_dirty.item()) != n_rewritten:
+        raise SystemExit("dirty count differs from the generated pattern")
+    W = r.wire_len
+
+    for _ in range(args.warmup):
+        step()
+    barrier()
+    launches["n"] = 0
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    try:
+        gpu_uuid = "GPU-" + str(torch.cuda.get_device_properties(dev).uuid)
+    except Exception:
+        gpu_uuid = None
+    with ClockSampler(local_rank, gpu_uuid) as clk:
+        ev0.record()
+        for _ in range(args.steps):
+            step()
+        ev1.record()
+        barrier()
+    ms_total = max_over_ranks(ev0.elapsed_time(ev1))
+    ms_step = ms_total / args.steps
+    gpu_launches = launches["n"]
+    value = world * N / (ms_step * 1e-3) / 1e9
+
+    if args.profile:
+        if rank == 0:
+            print(json.dumps({"profile_mode": True, "workload": args.workload, "ms_per_step": ms_step,
+                              "value": value, "gpu_launches": gpu_launches}))
+        return
+
+    # per-call and main-kernel times (separate pass; each call bracketed by events on the stream)
+    wm.timing_enable(True)
+    calls = {"checksum": (call_checksum, wm.KIND_CHECKSUM, N + 4 * nc),
+             "dirty_diff": (call_diff, wm.KIND_DIFF, None),
+             "encode": (call_encode, wm.KIND_ENCODE, N + W),
+             "decode_verify": (call_decode, wm.KIND_DECODE, N + W)}
+    reps = max(5, min(args.steps, 30))
+    peak, peak_kind = _peaks()
+    per_call = {}
+    for name, (fn, kind, alg_bytes) in calls.items():
+        call_ms, kern_ms = [], []
+        for _ in range(reps):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            fn()
+            b.record()
+            torch.cuda.synchronize()
+            call_ms.append(a.elapsed_time(b))
+            kern_ms.append(wm.timing_read_ms(kind))
+        cm, km = statistics.mean(call_ms), statistics.mean(kern_ms)
+        entry = {"call_ms": cm, "kernel_ms": km, "raw_gbs": N / (cm * 1e-3) / 1e9}
+        if alg_bytes:
+            entry["algorithmic_bytes"] = alg_bytes
+            entry["kernel_traffic_gbs"] = alg_bytes / (km * 1e-3) / 1e9
+            entry["frac_of_hbm_peak"] = entry["kernel_traffic_gbs"] / peak
+        per_call[name] = entry
+    wm.timing_enable(False)
+    # dirty diff: bytes it actually has to read (clean chunks in full on both sides)
+    per_call["dirty_diff"]["note"] = f"{n_rewritten} of {nc} chunks dirty; clean chunks are read in full on both sides"
+
+    enc = per_call["encode"]
+    roofline = {"bound": "hbm", "kernel": "k_encode (fused checksum+encode)",
+                "achieved": enc["kernel_traffic_gbs"], "peak": peak, "unit": "GB/s",
+                "frac": enc["kernel_traffic_gbs"] / peak, "peak_source": f"of {peak_kind}",
+                "traffic": NCU_TRAFFIC_BYTES.get(args.workload),
+                "algorithmic_bytes_per_launch": N + W,
+                "decode_frac": per_call["decode_verify"]["frac_of_hbm_peak"]}
+
+    # end to end: host cache in (pinned), verified wire image and result records out
+    e2e = None
+    if not args.no_e2e:
+        host_cache = torch.empty(N, dtype=torch.uint8, pin_memory=True)
+        host_cache.copy_(cur)
+        host_wire = torch.empty(W, dtype=torch.uint8, pin_memory=True)
+        host_res = torch.empty(80, dtype=torch.uint8, pin_memory=True)
+        e_steps = max(2, min(args.steps, 5))
+
+        def e2e_step():
+            cur.copy_(host_cache, non_blocking=True)
+            step()
+            host_wire.copy_(wire[:W], non_blocking=True)
+            host_res[:40].copy_(res_e, non_blocking=True)
+            host_res[40:].copy_(res_d, non_blocking=True)
+
+        e2e_step()
+        barrier()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(e_steps):
+            e2e_step()
+        b.record()
+        barrier()
+        e_ms = max_over_ranks(a.elapsed_time(b)) / e_steps
+        e2e = {"value": world * N / (e_ms * 1e-3) / 1e9, "unit": "GB/s", "h2d_bytes_per_step": N,
+               "d2h_bytes_per_step": W + 80, "steps": e_steps, "ms_per_step": e_ms}
+
+    base = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        sample_n = min(N, 64 * C)
+        base = cpu_baseline(cur[:sample_n].cpu().numpy(), prev[:sample_n].cpu().numpy(), C)
+
+    if rank == 0:
+        clocks = clk.summary()
+        out = {
+            "metric": "raw-cache GB/s through checksum+diff+encode+decode_verify",
+            "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "u8", "data": "synthetic",
+            "config": {"workload": args.workload, "nbytes": N, "chunk_bytes": C, "shape": list(cfg.shape),
+                       "wire_bytes": W, "ratio": W / N, "dirty_chunks": n_rewritten, "n_chunks": nc,
+                       "l2": "inputs larger than L2 (no flush needed)", "parallelism": "replicas only"},
+            "calls": per_call, "roofline": roofline, "cpu_baseline": base, "e2e": e2e,
+            "gpu_launches": gpu_launches, "clocks": clocks,
+        }
+        print(json.dumps(out))
+    if world > 1:
+        torch.distributed.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

@@ -155,8 +155,18 @@ wm_status wm_decode_verify(const void* wire, uint64_t wire_len, void* dst, uint6
                            uint32_t chunk_bytes, uint32_t* dst_crc_inout,
                            void* workspace, uint64_t workspace_bytes, wm_result* result, void* stream);
 
-/* Number of kernels the last call of each kind enqueued (for launch accounting). */
+/* Number of kernels the last call on this host thread enqueued (for launch accounting). */
 uint32_t wm_last_launch_count(void);
+
+/*
+ * Measurement aid (not part of the paper's method).  When enabled, every call records a CUDA
+ * event pair on the caller's stream around its main kernel: kind 0 = checksum tile digests,
+ * 1 = dirty diff compare, 2 = encode, 3 = decode.  wm_timing_read_ms waits for the most
+ * recent pair of that kind on the current device and returns its elapsed milliseconds
+ * (WM_ERR_CUDA if no such call was made while timing was enabled).  Process-wide switch.
+ */
+void wm_timing_enable(int on);
+int wm_timing_read_ms(int kind, float* ms);
 
 #ifdef __cplusplus
 }

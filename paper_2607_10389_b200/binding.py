@@ -22,7 +22,8 @@ STATUS = {
 }
 RESULT_BYTES = 40
 EXPORTS = ("wm_num_chunks", "wm_num_tiles", "wm_meta_bytes", "wm_wire_bound", "wm_workspace_bytes",
-           "wm_checksum", "wm_dirty_diff", "wm_encode", "wm_decode_verify", "wm_last_launch_count")
+           "wm_checksum", "wm_dirty_diff", "wm_encode", "wm_decode_verify", "wm_last_launch_count",
+           "wm_timing_enable", "wm_timing_read_ms")
 
 
 class WmError(RuntimeError):
@@ -44,6 +45,10 @@ def load_library() -> ctypes.CDLL:
         getattr(lib, n).argtypes = [u64, u32]
     lib.wm_last_launch_count.restype = u32
     lib.wm_last_launch_count.argtypes = []
+    lib.wm_timing_enable.restype = None
+    lib.wm_timing_enable.argtypes = [ctypes.c_int]
+    lib.wm_timing_read_ms.restype = ctypes.c_int
+    lib.wm_timing_read_ms.argtypes = [ctypes.c_int, ctypes.POINTER(ctypes.c_float)]
     lib.wm_checksum.restype = ctypes.c_int
     lib.wm_checksum.argtypes = [vp, u64, u32, vp, vp, u64, vp]
     lib.wm_dirty_diff.restype = ctypes.c_int
@@ -114,6 +119,19 @@ def workspace_bytes(nbytes: int, chunk_bytes: int) -> int:
 
 def last_launch_count() -> int:
     return int(lib().wm_last_launch_count())
+
+
+KIND_CHECKSUM, KIND_DIFF, KIND_ENCODE, KIND_DECODE = 0, 1, 2, 3
+
+
+def timing_enable(on: bool) -> None:
+    lib().wm_timing_enable(1 if on else 0)
+
+
+def timing_read_ms(kind: int) -> float:
+    ms = ctypes.c_float(0.0)
+    _check(lib().wm_timing_read_ms(kind, ctypes.byref(ms)), "wm_timing_read_ms")
+    return float(ms.value)
 
 
 def _dev_u8(t: torch.Tensor, what: str) -> torch.Tensor:

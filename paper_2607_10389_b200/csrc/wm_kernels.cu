@@ -45,12 +45,12 @@ struct Ctrl {                 // first 256 bytes of the workspace
     uint32_t done_a;
     uint32_t done_b;
     uint32_t n_present;
+    uint32_t scan_lock;
     uint32_t gate;            // decode: status of an earlier failing step (0 = none)
     uint32_t bad3_first, bad3_count;
     uint32_t bad4_first, bad4_count;
     uint32_t bad5_first, bad5_count;
     uint32_t bad6_first, bad6_count;
-    uint32_t pad0;
     unsigned long long bad4_key;   // lowest failing tile * 2 + (1 if STRUCT)
     unsigned long long payload_total;
     uint32_t hdr_n_present, hdr_cache_crc;
@@ -139,7 +139,6 @@ struct TeamCtl {
     uint32_t status;
     unsigned long long excl;
 };
-constexpr uint32_t kTeamSmemEncode = kTile + sizeof(TeamCtl);
 constexpr uint32_t kTeamSmemPlain = sizeof(TeamCtl);
 
 // Digest of the team's current tile from the words each lane holds; result in wdig[] (valid
@@ -365,48 +364,83 @@ __global__ void k_encode_init(Geo g, Ws ws, unsigned char* wire)
 constexpr unsigned long long kFlagA = 1ull << 62, kFlagP = 2ull << 62, kValMask = (1ull << 62) - 1;
 constexpr uint32_t kSpinLimit = 1u << 20;
 
-// Exclusive prefix of tile lengths for tile t (warp-wide decoupled look-back; every lane of
-// one warp calls).  Tiles are claimed in ticket order, so every predecessor belongs to a
-// team that is already running and publishes its own length before it waits for anything:
-// the wait below cannot deadlock.  It is bounded all the same; when the bound is hit the
-// call is poisoned and reports WM_ERR_TIMEOUT.
-__device__ unsigned long long lookback(unsigned long long* state, uint32_t t, uint32_t len, uint32_t lane, Ctrl* ctrl)
+// Placement of the encoded tiles: a chained scan with one dedicated scanner warp.
+//
+// state[t] starts at 0.  The team that encodes tile t publishes kFlagA | len(t) as soon as the
+// length is known.  One scanner warp (the winner of a lock among the extra warps every block
+// carries) walks the array in order, 256 entries per poll, turns every leading run of
+// published lengths into kFlagP | exclusive prefix, and moves on.  The owner of tile t then
+// reads its offset back from state[t].  Several hundred tiles are in flight at any time and
+// publish at about the same moment; letting each of them walk back to the nearest finished
+// prefix made the walk, not the data, the bottleneck.  The scanner is a warp that is running
+// by construction (it won the lock), so the owners' waits depend only on running code; all
+// waits are bounded all the same and end in WM_ERR_TIMEOUT.
+__device__ __forceinline__ void publish_len(unsigned long long* state, uint32_t t, uint32_t len)
 {
-    if (t == 0) {
-        if (lane == 0) st_volatile_u64(reinterpret_cast<uint64_t*>(&state[0]), kFlagP | len);
-        return 0;
+    st_volatile_u64(reinterpret_cast<uint64_t*>(&state[t]), kFlagA | len);
+}
+
+// Owner side: exclusive prefix of tile t (one lane spins; bounded).
+__device__ __forceinline__ unsigned long long wait_prefix(unsigned long long* state, uint32_t t, Ctrl* ctrl)
+{
+    for (uint32_t polls = 0; polls < kSpinLimit; polls++) {
+        const unsigned long long v = ld_volatile_u64(reinterpret_cast<const uint64_t*>(&state[t]));
+        if ((v >> 62) == 2) return v & kValMask;
+        if ((polls & 1023u) == 1023u && ld_volatile_u32(&ctrl->poison)) break;
     }
-    if (lane == 0) st_volatile_u64(reinterpret_cast<uint64_t*>(&state[t]), kFlagA | len);
-    unsigned long long excl = 0;
-    long long hi = (long long)t - 1;
-    uint32_t polls = 0;
-    bool failed = false;
-    while (true) {
-        const long long idx = hi - (long long)lane;
-        unsigned long long v;
-        while (true) {
-            v = idx >= 0 ? ld_volatile_u64(reinterpret_cast<const uint64_t*>(&state[idx])) : kFlagP;
-            if (__all_sync(0xFFFFFFFFu, (v >> 62) != 0)) break;
-            if (++polls > kSpinLimit) { failed = true; break; }
+    atomicOr(&ctrl->err, 2u);
+    atomicExch(&ctrl->poison, 1u);
+    return 0;
+}
+
+// Scanner side (one full warp).
+__device__ void scan_tile_lengths(unsigned long long* state, uint32_t n_tiles, uint32_t lane, Ctrl* ctrl)
+{
+    uint32_t f = 0, spins = 0;
+    unsigned long long base = 0;
+    while (f < n_tiles) {
+        unsigned long long v[8];
+#pragma unroll
+        for (int j = 0; j < 8; j++) {
+            const uint64_t idx = (uint64_t)f + 8u * lane + j;
+            v[j] = idx < n_tiles ? ld_volatile_u64(reinterpret_cast<const uint64_t*>(&state[idx])) : 0ull;
         }
-        if (failed) break;
-        const uint32_t pm = __ballot_sync(0xFFFFFFFFu, (v >> 62) == 2);
-        if (pm) {
-            const uint32_t first = __ffs(pm) - 1;
-            const uint32_t part = __reduce_add_sync(0xFFFFFFFFu, lane < first ? (uint32_t)(v & kValMask) : 0u);
-            const unsigned long long pv = __shfl_sync(0xFFFFFFFFu, v, first) & kValMask;
-            excl += part + pv;
-            break;
+        uint32_t r = 0, sum = 0;            // leading published entries of this lane and their sum
+#pragma unroll
+        for (int j = 0; j < 8; j++)
+            if (r == (uint32_t)j && (v[j] >> 62) == 1) { r++; sum += (uint32_t)(v[j] & kValMask); }
+        const uint32_t fm = __ballot_sync(0xFFFFFFFFu, r == 8);
+        const uint32_t lead = (fm == 0xFFFFFFFFu) ? 32u : (uint32_t)(__ffs(~fm) - 1);   // leading full lanes
+        const uint32_t contrib = lane <= lead ? sum : 0u;
+        uint32_t incl = contrib;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            uint32_t o = __shfl_up_sync(0xFFFFFFFFu, incl, d);
+            if (lane >= (uint32_t)d) incl += o;
         }
-        excl += __reduce_add_sync(0xFFFFFFFFu, (uint32_t)(v & kValMask));
-        hi -= 32;
+        const uint32_t cnt = lane < lead ? 8u : (lane == lead ? r : 0u);
+        unsigned long long run = base + (incl - contrib);
+#pragma unroll
+        for (int j = 0; j < 8; j++) {
+            if ((uint32_t)j < cnt) {
+                st_volatile_u64(reinterpret_cast<uint64_t*>(&state[(uint64_t)f + 8u * lane + j]), kFlagP | run);
+                run += v[j] & kValMask;
+            }
+        }
+        const uint32_t r_lead = __shfl_sync(0xFFFFFFFFu, r, lead & 31u);
+        const uint32_t k = 8u * lead + (lead < 32u ? r_lead : 0u);
+        base += __shfl_sync(0xFFFFFFFFu, incl, 31);
+        f += k;
+        if (k == 0) {
+            if (++spins > kSpinLimit || ((spins & 1023u) == 1023u && ld_volatile_u32(&ctrl->poison))) {
+                if (lane == 0) { atomicOr(&ctrl->err, 2u); atomicExch(&ctrl->poison, 1u); }
+                return;
+            }
+        } else {
+            spins = 0;
+        }
     }
-    if (failed) {
-        if (lane == 0) { atomicOr(&ctrl->err, 2u); atomicExch(&ctrl->poison, 1u); }
-        excl = 0;
-    }
-    if (lane == 0) st_volatile_u64(reinterpret_cast<uint64_t*>(&state[t]), kFlagP | (excl + len));
-    return excl;
+    if (lane == 0) ctrl->payload_total = base;
 }
 
 __device__ __forceinline__ uint32_t next_ticket(Ctrl* ctrl)
@@ -420,8 +454,53 @@ __device__ __forceinline__ uint32_t desc_of(uint32_t base, uint32_t w)
     return base | (w << 8) | ((((base & 15u) ^ (base >> 4) ^ w ^ 5u) & 15u) << 12);
 }
 
+struct EncTeamCtl {
+    uint32_t wtab[2][32];   // per group: base | w << 8 (double buffered by tile parity)
+    uint32_t wdig[2][8];    // per warp: its contribution to the tile digest
+    uint32_t next;          // ticket just claimed (>= n_tiles: none left)
+    uint32_t pad;
+    unsigned long long excl;
+};
+constexpr uint32_t kTeamSmemEncode = kTile + sizeof(EncTeamCtl);
+
+struct TileInfo {
+    bool valid, present, full, first;
+    uint32_t c, left;
+    uint64_t off;
+};
+
+__device__ __forceinline__ TileInfo tile_info(const Geo& g, const uint8_t* __restrict__ dirty, uint32_t t)
+{
+    TileInfo ti;
+    ti.valid = t < g.n_tiles;
+    ti.present = false; ti.full = false; ti.first = false; ti.c = 0; ti.left = 0; ti.off = 0;
+    if (!ti.valid) return ti;
+    ti.c = t / g.tiles_per_chunk;
+    ti.first = (t % g.tiles_per_chunk) == 0;
+    ti.present = !dirty || dirty[ti.c] != 0;
+    ti.off = (uint64_t)t * kTile;
+    const uint64_t left = g.nbytes - ti.off;
+    ti.full = left >= kTile;
+    ti.left = ti.full ? kTile : (uint32_t)left;
+    return ti;
+}
+
+__device__ __forceinline__ uint32_t encoded_len(const TileInfo& ti, uint32_t S)
+{
+    if (!ti.present) return 0;
+    if (!ti.full) return ti.left;
+    return S <= 253u ? 8256u + 32u * S : kTile;
+}
+
+// Single-pass fused checksum + encode.  Per team, software pipelined over tiles X (being
+// packed and written out) and Y (being checksummed and measured):
+//     pack X into shared memory | digest + exponent ranges of Y | publish len(Y) |
+//     look back for X's offset | claim Z and start its loads | copy X out
+// A team never waits for another team while it holds a claimed tile whose length is not yet
+// published: len(Y) goes out before the look-back for X starts, and Z is claimed only after
+// that look-back has returned.  This keeps every wait one hop long.
 template <int TEAMS>
-__global__ void __launch_bounds__(TEAMS * 256, 1)
+__global__ void __launch_bounds__(TEAMS * 256 + 32, 1)
 k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restrict__ dirty,
          unsigned char* __restrict__ wire, uint64_t wire_cap, Ws ws, const Tables* __restrict__ tab)
 {
@@ -429,71 +508,78 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
     SmemTables T = load_tables(smem, tab);
     const uint32_t team = threadIdx.x / kTeamThreads, tt = threadIdx.x % kTeamThreads;
     const uint32_t warp = tt / 32, lane = tt % 32;
+    if (team == TEAMS) {
+        // the extra warp: one of them, grid-wide, becomes the scanner; the others leave
+        uint32_t won = 0;
+        if (lane == 0) won = atomicCAS(&ws.ctrl->scan_lock, 0u, 1u) == 0u;
+        won = __shfl_sync(0xFFFFFFFFu, won, 0);
+        if (won) scan_tile_lengths(ws.state, g.n_tiles, lane, ws.ctrl);
+        return;
+    }
     unsigned char* out = smem + kSmemTables + team * kTeamSmemEncode;
-    TeamCtl* tc = reinterpret_cast<TeamCtl*>(out + kTile);
+    EncTeamCtl* tc = reinterpret_cast<EncTeamCtl*>(out + kTile);
     unsigned char* dir = wire + 64;
     uint16_t* tile_tab = reinterpret_cast<uint16_t*>(wire + 64 + 16ull * g.n_chunks);
 
-    if (tt == 0) tc->next = next_ticket(ws.ctrl);
-    team_bar(team);
-    uint32_t t = tc->next;
-    uint32_t nxt[kWordsPerLane];
-    {
-        const bool ok = t < g.n_tiles && (g.nbytes - (uint64_t)t * kTile) >= kTile &&
-                        (!dirty || dirty[t / g.tiles_per_chunk]);
-        if (ok) load_tile_words(cache + (uint64_t)t * kTile, warp, lane, nxt);
-    }
-
-    while (t < g.n_tiles) {
-        uint32_t cur[kWordsPerLane];
+    // digest and per-group exponent range of one tile; results go to wdig[par], wtab[par]
+    auto phase_a = [&](const TileInfo& ti, uint32_t (&d)[kWordsPerLane], uint32_t par) {
+        if (!ti.present) return;
+        if (!ti.full) load_tile_words_guarded(cache + ti.off, ti.left, ti.first, -8, warp, lane, d);
+        {
+            const uint32_t m = (ti.first && ti.full && warp == 0 && lane == 0) ? 0xFFFFFFFFu : 0u;
+            d[0] ^= m;
+            const uint32_t dg = warp_block_digest(T, d, lane);
+            d[0] ^= m;
+            const uint32_t v = warp_place(T, dg, warp, lane);
+            if (lane == 0) tc->wdig[par][warp] = v;
+        }
+        if (ti.full) {
 #pragma unroll
-        for (int i = 0; i < 16; i++) cur[i] = nxt[i];
-        const uint32_t c = t / g.tiles_per_chunk;
-        const bool first = (t % g.tiles_per_chunk) == 0;
-        const bool present = !dirty || dirty[c] != 0;
-        const uint64_t off = (uint64_t)t * kTile;
-        const uint64_t left = g.nbytes - off;
-        const bool full = left >= kTile;
-
-        team_bar(team);                                               // bar0
-        if (tt == 0) tc->next = next_ticket(ws.ctrl);
-
-        // ---- phase A: checksum digest, per-group exponent range
-        if (present) {
-            if (!full) load_tile_words_guarded(cache + off, (uint32_t)left, first, -8, warp, lane, cur);
-            tile_digest_to_smem(T, cur, first && full, warp, lane, tc);
-            if (full) {
-#pragma unroll
-                for (int j = 0; j < 4; j++) {
-                    const uint32_t a0 = cur[4 * j] & 0x7FFF7FFFu, a1 = cur[4 * j + 1] & 0x7FFF7FFFu;
-                    const uint32_t a2 = cur[4 * j + 2] & 0x7FFF7FFFu, a3 = cur[4 * j + 3] & 0x7FFF7FFFu;
-                    uint32_t mn = min_u16x2(min_u16x2(a0, a1), min_u16x2(a2, a3));
-                    uint32_t mx = max_u16x2(max_u16x2(a0, a1), max_u16x2(a2, a3));
-                    mn = min(mn & 0xFFFFu, mn >> 16);
-                    mx = max(mx & 0xFFFFu, mx >> 16);
-                    const uint32_t emin = __reduce_min_sync(0xFFFFFFFFu, mn) >> 7;
-                    const uint32_t emax = __reduce_max_sync(0xFFFFFFFFu, mx) >> 7;
-                    const uint32_t range = emax - emin;
-                    const uint32_t wd = 32u - __clz(range);
-                    if (lane == 0) tc->wtab[4 * warp + j] = emin | (wd << 8);
-                }
+            for (int j = 0; j < 4; j++) {
+                const uint32_t a0 = d[4 * j] & 0x7FFF7FFFu, a1 = d[4 * j + 1] & 0x7FFF7FFFu;
+                const uint32_t a2 = d[4 * j + 2] & 0x7FFF7FFFu, a3 = d[4 * j + 3] & 0x7FFF7FFFu;
+                uint32_t mn = min_u16x2(min_u16x2(a0, a1), min_u16x2(a2, a3));
+                uint32_t mx = max_u16x2(max_u16x2(a0, a1), max_u16x2(a2, a3));
+                mn = min(mn & 0xFFFFu, mn >> 16);
+                mx = max(mx & 0xFFFFu, mx >> 16);
+                const uint32_t emin = __reduce_min_sync(0xFFFFFFFFu, mn) >> 7;
+                const uint32_t emax = __reduce_max_sync(0xFFFFFFFFu, mx) >> 7;
+                const uint32_t wd = 32u - __clz(emax - emin);
+                if (lane == 0) tc->wtab[par][4 * warp + j] = emin | (wd << 8);
             }
         }
-        team_bar(team);                                               // bar1
+    };
+    auto sum_widths = [&](uint32_t par) {
+        return __reduce_add_sync(0xFFFFFFFFu, (tc->wtab[par][lane] >> 8) & 15u);
+    };
 
-        // ---- prefetch the next tile while this one is packed
-        const uint32_t tn = tc->next;
-        {
-            const bool ok = tn < g.n_tiles && (g.nbytes - (uint64_t)tn * kTile) >= kTile &&
-                            (!dirty || dirty[tn / g.tiles_per_chunk]);
-            if (ok) load_tile_words(cache + (uint64_t)tn * kTile, warp, lane, nxt);
-        }
+    // ---- prologue: X claimed, loaded, measured and published; Y claimed and loading
+    uint32_t dX[kWordsPerLane], dY[kWordsPerLane];
+    if (tt == 0) tc->next = next_ticket(ws.ctrl);
+    team_bar(team);
+    uint32_t tX = tc->next;
+    TileInfo iX = tile_info(g, dirty, tX);
+    if (iX.present && iX.full) load_tile_words(cache + iX.off, warp, lane, dX);
+    uint32_t par = 0;
+    phase_a(iX, dX, par);
+    team_bar(team);
+    if (warp == 0 && iX.valid) {
+        const uint32_t S = (iX.present && iX.full) ? sum_widths(par) : 0u;
+        if (lane == 0) { publish_len(ws.state, tX, encoded_len(iX, S)); tc->next = next_ticket(ws.ctrl); }
+    }
+    team_bar(team);
+    uint32_t tY = iX.valid ? tc->next : 0xFFFFFFFFu;
+    TileInfo iY = tile_info(g, dirty, tY);
+    if (iY.present && iY.full) load_tile_words(cache + iY.off, warp, lane, dY);
 
-        // ---- phase B: pack into shared memory (or decide RAW), look-back for the offset
+    while (iX.valid) {
+        team_bar(team);                                               // bar0: out buffer free
+
+        // ---- pack X
         uint32_t enc_len = 0, entry = 0;
-        bool packed = false;
-        if (present && full) {
-            const uint32_t wt = tc->wtab[lane];
+        bool staged = false;               // encoded tile sits in `out`
+        if (iX.present && iX.full) {
+            const uint32_t wt = tc->wtab[par][lane];
             const uint32_t wv = (wt >> 8) & 15u;
             uint32_t incl = wv;
 #pragma unroll
@@ -502,8 +588,8 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
                 if (lane >= (uint32_t)d) incl += o;
             }
             const uint32_t S = __shfl_sync(0xFFFFFFFFu, incl, 31);
+            staged = true;
             if (S <= 253u) {
-                packed = true;
                 enc_len = 8256u + 32u * S;
                 entry = 258u + S;
                 if (warp == 0) reinterpret_cast<uint16_t*>(out)[lane] = (uint16_t)desc_of(wt & 0xFFu, wv);
@@ -516,7 +602,7 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
                     uint32_t Tr[4];
 #pragma unroll
                     for (int r = 0; r < 4; r++) {
-                        const uint32_t W = cur[4 * j + r];
+                        const uint32_t W = dX[4 * j + r];
                         Tr[r] = ((W << 1) & 0xFFFEFFFEu) | ((W >> 15) & 0x00010001u);
                     }
                     const uint32_t sma = __byte_perm(Tr[0], Tr[1], 0x6420), smb = __byte_perm(Tr[2], Tr[3], 0x6420);
@@ -544,40 +630,67 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
             } else {
                 enc_len = kTile;
                 entry = 512u;
+                uint32_t* o32 = reinterpret_cast<uint32_t*>(out) + warp * 512u + lane;
+#pragma unroll
+                for (int i = 0; i < 16; i++) o32[i * 32] = dX[i];
             }
-        } else if (present) {
-            enc_len = (uint32_t)left;
+        } else if (iX.present) {
+            enc_len = iX.left;
             entry = 0xFFFFu;
         }
-        if (warp == 0) {
-            const unsigned long long e = lookback(ws.state, t, enc_len, lane, ws.ctrl);
-            if (lane == 0) tc->excl = e;
-        }
-        team_bar(team);                                               // bar2
 
-        // ---- phase C: move the encoded tile to its place in the wire image
+        // ---- measure Y (its data was requested one iteration ago)
+        phase_a(iY, dY, par ^ 1u);
+        team_bar(team);                                               // bar1: wtab[par^1] complete
+
+        if (warp == 0) {
+            if (iY.valid) {
+                const uint32_t S = (iY.present && iY.full) ? sum_widths(par ^ 1u) : 0u;
+                if (lane == 0) publish_len(ws.state, tY, encoded_len(iY, S));
+            }
+            if (lane == 0) {
+                tc->excl = wait_prefix(ws.state, tX, ws.ctrl);
+                tc->next = iY.valid ? next_ticket(ws.ctrl) : 0xFFFFFFFFu;
+            }
+        }
+        team_bar(team);                                               // bar2: offset known, out complete
+
+        // ---- claim Z, start its loads into X's (now free) registers
+        const uint32_t tZ = tc->next;
+        const TileInfo iZ = tile_info(g, dirty, tZ);
+        uint32_t dZ[kWordsPerLane];
+        if (iZ.present && iZ.full) load_tile_words(cache + iZ.off, warp, lane, dZ);
+
+        // ---- move X to its place in the wire image
         const unsigned long long excl = tc->excl;
-        if (present) {
+        if (iX.present) {
             const uint64_t dst = g.meta_end + excl;
             if (dst + enc_len > wire_cap) {
                 if (tt == 0) atomicOr(&ws.ctrl->err, 1u);
-            } else if (packed) {
+            } else if (staged) {
                 for (uint32_t i = tt * 16; i < enc_len; i += kTeamThreads * 16)
                     *reinterpret_cast<uint4*>(wire + dst + i) = *reinterpret_cast<const uint4*>(out + i);
-            } else if (full) {
-                unsigned char* p = wire + dst + warp * 2048u + lane * 4u;
-#pragma unroll
-                for (int i = 0; i < 16; i++) st_stream_u32(p + i * 128, cur[i]);
             } else {
-                for (uint32_t i = tt; i < enc_len; i += kTeamThreads) wire[dst + i] = cache[off + i];
+                for (uint32_t i = tt; i < enc_len; i += kTeamThreads) wire[dst + i] = cache[iX.off + i];
             }
         }
         if (tt == 0) {
-            tile_tab[t] = (uint16_t)entry;
-            if (present) ws.dig[t] = team_digest(tc);
-            if (first) *reinterpret_cast<unsigned long long*>(dir + 16ull * c) = excl;
+            tile_tab[tX] = (uint16_t)entry;
+            if (iX.present) {
+                uint32_t dg = 0;
+#pragma unroll
+                for (int i = 0; i < 8; i++) dg ^= tc->wdig[par][i];
+                ws.dig[tX] = dg;
+            }
+            if (iX.first) *reinterpret_cast<unsigned long long*>(dir + 16ull * iX.c) = excl;
         }
-        t = tn;
+
+        // ---- rotate
+        tX = tY; iX = iY;
+        tY = tZ; iY = iZ;
+#pragma unroll
+        for (int i = 0; i < 16; i++) { dX[i] = dY[i]; dY[i] = dZ[i]; }
+        par ^= 1u;
     }
 }
 
@@ -594,7 +707,7 @@ k_encode_finish(const unsigned char* __restrict__ cache, Geo g, const uint8_t* _
     __shared__ bool s_last;
     load_ht_t0(sHT, sT0, tab);
     unsigned char* dir = wire + 64;
-    const unsigned long long total = ws.state[g.n_tiles - 1] & kValMask;
+    const unsigned long long total = ws.ctrl->payload_total;
     const uint32_t c = blockIdx.x * blockDim.x + threadIdx.x;
     uint32_t present = 0;
     if (c < g.n_chunks) {
@@ -1072,12 +1185,29 @@ k_decode_finish(const unsigned char* __restrict__ wire, uint64_t wire_len, Geo g
 
 // ------------------------------------------------------------------ host side
 
-constexpr int kTeams = 3;
+#ifndef WM_TEAMS
+#define WM_TEAMS 3
+#endif
+constexpr int kTeams = WM_TEAMS;
 
 struct DeviceState {
     Tables* tables = nullptr;
     int sm_count = 0;
     bool ready = false;
+    cudaEvent_t ev[4][2] = {};   // optional timing of the four main kernels
+};
+static bool g_timing = false;
+
+struct MainKernelTimer {        // records events around a main kernel when timing is enabled
+    const DeviceState* ds; int kind; cudaStream_t s;
+    MainKernelTimer(const DeviceState* d, int k, cudaStream_t st) : ds(d), kind(k), s(st)
+    {
+        if (g_timing) cudaEventRecord(ds->ev[kind][0], s);
+    }
+    ~MainKernelTimer()
+    {
+        if (g_timing) cudaEventRecord(ds->ev[kind][1], s);
+    }
 };
 static DeviceState g_dev[64];
 static std::mutex g_mutex;
@@ -1100,6 +1230,9 @@ static const DeviceState* device_state()
     if (cudaFuncSetAttribute(k_decode<kTeams>, cudaFuncAttributeMaxDynamicSharedMemorySize, big) != cudaSuccess) return nullptr;
     if (cudaFuncSetAttribute(k_tile_digests<kTeams>, cudaFuncAttributeMaxDynamicSharedMemorySize, big) != cudaSuccess) return nullptr;
     if (cudaFuncSetAttribute(k_meta_crc, cudaFuncAttributeMaxDynamicSharedMemorySize, big) != cudaSuccess) return nullptr;
+    for (int k = 0; k < 4; k++)
+        for (int j = 0; j < 2; j++)
+            if (cudaEventCreate(&s.ev[k][j]) != cudaSuccess) return nullptr;
     s.ready = true;
     return &s;
 }
@@ -1140,6 +1273,16 @@ uint64_t wm_workspace_bytes(uint64_t nbytes, uint32_t chunk_bytes)
 
 uint32_t wm_last_launch_count(void) { return g_launches; }
 
+void wm_timing_enable(int on) { g_timing = on != 0; }
+
+int wm_timing_read_ms(int kind, float* ms)
+{
+    const DeviceState* ds = device_state();
+    if (!ds || kind < 0 || kind > 3 || !ms) return WM_ERR_ARG;
+    if (cudaEventSynchronize(ds->ev[kind][1]) != cudaSuccess) return WM_ERR_CUDA;
+    return cudaEventElapsedTime(ms, ds->ev[kind][0], ds->ev[kind][1]) == cudaSuccess ? WM_OK : WM_ERR_CUDA;
+}
+
 wm_status wm_checksum(const void* cache, uint64_t nbytes, uint32_t chunk_bytes, uint32_t* crc_out,
                       void* workspace, uint64_t workspace_bytes, void* stream)
 {
@@ -1153,7 +1296,10 @@ wm_status wm_checksum(const void* cache, uint64_t nbytes, uint32_t chunk_bytes, 
     const unsigned char* c = static_cast<const unsigned char*>(cache);
     const uint32_t need = (g.n_tiles + kTeams - 1) / kTeams;
     const uint32_t grid = need < (uint32_t)ds->sm_count ? need : (uint32_t)ds->sm_count;
-    k_tile_digests<kTeams><<<grid, kTeams * 256, kSmemTables + kTeams * kTeamSmemPlain, s>>>(c, g, ws, ds->tables);
+    {
+        MainKernelTimer timer(ds, 0, s);
+        k_tile_digests<kTeams><<<grid, kTeams * 256, kSmemTables + kTeams * kTeamSmemPlain, s>>>(c, g, ws, ds->tables);
+    }
     k_checksum_finish<<<(g.n_chunks + 255) / 256, 256, 0, s>>>(c, g, ws, ds->tables, crc_out);
     g_launches = 2;
     return launch_status();
@@ -1173,7 +1319,10 @@ wm_status wm_dirty_diff(const void* cache, const void* prev, uint64_t nbytes, ui
     k_diff_init<<<1, 32, 0, s>>>(ws);
     const uint32_t want = (uint32_t)ds->sm_count * 4;
     const uint32_t grid = g.n_chunks < want ? g.n_chunks : want;
-    k_diff<<<grid, 256, 0, s>>>(static_cast<const unsigned char*>(cache), static_cast<const unsigned char*>(prev), g, ws, dirty_out);
+    {
+        MainKernelTimer timer(ds, 1, s);
+        k_diff<<<grid, 256, 0, s>>>(static_cast<const unsigned char*>(cache), static_cast<const unsigned char*>(prev), g, ws, dirty_out);
+    }
     k_diff_compact<<<1, 1024, 0, s>>>(g, dirty_out, dirty_idx_out, n_dirty_out);
     g_launches = 3;
     return launch_status();
@@ -1198,7 +1347,10 @@ wm_status wm_encode(const void* cache, uint64_t nbytes, uint32_t chunk_bytes, co
     k_encode_init<<<init_blocks ? init_blocks : 1, 1024, 0, s>>>(g, ws, w);
     const uint32_t need = (g.n_tiles + kTeams - 1) / kTeams;
     const uint32_t grid = need < (uint32_t)ds->sm_count ? need : (uint32_t)ds->sm_count;
-    k_encode<kTeams><<<grid, kTeams * 256, kSmemTables + kTeams * kTeamSmemEncode, s>>>(c, g, dirty, w, wire_cap, ws, ds->tables);
+    {
+        MainKernelTimer timer(ds, 2, s);
+        k_encode<kTeams><<<grid, kTeams * 256 + 32, kSmemTables + kTeams * kTeamSmemEncode, s>>>(c, g, dirty, w, wire_cap, ws, ds->tables);
+    }
     k_encode_finish<<<(g.n_chunks + 1023) / 1024, 1024, 0, s>>>(c, g, dirty, crc_inout, w, ws, ds->tables);
     k_meta_crc<<<g.n_meta_slices, 256, kSmemTables + kTeamSmemPlain, s>>>(w, 0, g, ws, ds->tables, result, 0);
     g_launches = 4;
@@ -1226,7 +1378,10 @@ wm_status wm_decode_verify(const void* wire, uint64_t wire_len, void* dst, uint6
     k_decode_struct_scan<<<1, 1024, 0, s>>>(w, wire_len, g, ws, result);
     const uint32_t need = (g.n_tiles + kTeams - 1) / kTeams;
     const uint32_t grid = need < (uint32_t)ds->sm_count ? need : (uint32_t)ds->sm_count;
-    k_decode<kTeams><<<grid, kTeams * 256, kSmemTables + kTeams * kTeamSmemPlain, s>>>(w, g, d, ws, ds->tables);
+    {
+        MainKernelTimer timer(ds, 3, s);
+        k_decode<kTeams><<<grid, kTeams * 256, kSmemTables + kTeams * kTeamSmemPlain, s>>>(w, g, d, ws, ds->tables);
+    }
     k_decode_finish<<<(g.n_chunks + 1023) / 1024, 1024, 0, s>>>(w, wire_len, g, d, dst_crc_inout, ws, ds->tables, result);
     g_launches = 6;
     return launch_status();

@@ -49,6 +49,8 @@ CONFIGS = {
     # long-context cache
     "long": _kv("long", (32, 2, 8, 131072, 128), 4 << 20, 4, "kv"),
     "long8g": _kv("long8g", (32, 2, 8, 65536, 128), 4 << 20, 4, "kv"),
+    # engine-like cache small enough for a profiler capture, still larger than the 126 MB L2
+    "engine_256m": _kv("engine_256m", (5, 2, 16, 6400, 128), 1 << 20, 2, "kv"),
     # reduced engine-like cache for tests that also run the CPU oracle on everything
     "engine_small": _kv("engine_small", (3, 2, 4, 680, 128), 1 << 20, 2, "kv"),
 }
