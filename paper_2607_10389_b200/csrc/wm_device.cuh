@@ -7,6 +7,13 @@
 // apart, which makes its CRC contribution a Horner chain with ONE fixed multiplier
 // (x^1024, table G); the lane's place inside the row and the warp's place inside the tile
 // are folded in once per tile with two small nibble tables (NK, NW).
+//
+// Table lookups are the inner loop (one per byte), so their address arithmetic is reduced to
+// a single byte permute: the tables sit at a 64 KiB-aligned shared address, entry b of a
+// table starts at b*256 and holds one copy per lane (lane l only ever touches bank l: no
+// bank conflicts on data-dependent indices), so address = base | b << 8 | lane*4 is
+// PRMT(value, base | lane*4).  The second table of a pair lives 128 bytes further and is
+// reached through the load's immediate offset.
 #pragma once
 #include <cstdint>
 #include <cuda_runtime.h>
@@ -18,35 +25,61 @@ namespace wm {
 constexpr uint32_t kTile = 16384;
 constexpr uint32_t kTeamThreads = 256;
 constexpr uint32_t kWordsPerLane = 16;
+// Dynamic shared memory every table-using kernel asks for: the 144 KiB image plus 64 KiB
+// that the 64 KiB alignment splits into a part below and a part above the image.
+constexpr uint32_t kDynSmem = kImgBytes + 0x10000;
 
-// Shared-memory image of the tables.  G and NK are stored once per lane ("replicated") so
-// that lane l only ever touches bank l: data-dependent lookups are conflict free.
-constexpr uint32_t kSmemG = 4 * 256 * 32 * 4;      // 131072
-constexpr uint32_t kSmemNK = 8 * 16 * 32 * 4;      // 16384
-constexpr uint32_t kSmemNW = 8 * 8 * 16 * 4;       // 4096
-constexpr uint32_t kSmemTables = kSmemG + kSmemNK + kSmemNW;
+struct Smem {
+    uint32_t L01, L23, LNK;      // shared-window address of A01 / A23 / NK, or'ed with lane*4
+    const uint32_t* NW;          // warp-position nibble tables [8][8][16]
+    unsigned char* lo; uint32_t lo_bytes;    // free space below the image
+    unsigned char* hi; uint32_t hi_bytes;    // free space above the image
+    bool ok;
 
-struct SmemTables {
-    const uint32_t* G;    // [(k*256 + b)*32 + lane]
-    const uint32_t* NK;   // [(n*16 + v)*32 + lane]
-    const uint32_t* NW;   // [(w*8 + n)*16 + v]
+    // carve `bytes` (multiple of 16) from the free space; nullptr when it does not fit
+    __device__ unsigned char* take(uint32_t bytes)
+    {
+        unsigned char* p = nullptr;
+        if (lo_bytes >= bytes) { p = lo; lo += bytes; lo_bytes -= bytes; }
+        else if (hi_bytes >= bytes) { p = hi; hi += bytes; hi_bytes -= bytes; }
+        else ok = false;
+        return p;
+    }
 };
 
-__device__ __forceinline__ SmemTables load_tables(unsigned char* smem, const Tables* __restrict__ tab)
+// Copy the table image into shared memory (whole block; ends with __syncthreads).
+__device__ __forceinline__ Smem setup_smem(unsigned char* smem, const Tables* __restrict__ tab)
 {
-    uint32_t* G = reinterpret_cast<uint32_t*>(smem);
-    uint32_t* NK = reinterpret_cast<uint32_t*>(smem + kSmemG);
-    uint32_t* NW = reinterpret_cast<uint32_t*>(smem + kSmemG + kSmemNK);
-    const uint32_t* gG = &tab->G[0][0];
-    const uint32_t* gNK = &tab->NK[0][0][0];
-    const uint32_t* gNW = &tab->NW[0][0][0];
-    for (uint32_t i = threadIdx.x; i < 4 * 256 * 32; i += blockDim.x) G[i] = gG[i >> 5];
-    for (uint32_t i = threadIdx.x; i < 8 * 16 * 32; i += blockDim.x) NK[i] = gNK[(i & 31) * 128 + (i >> 5)];
-    for (uint32_t i = threadIdx.x; i < 8 * 8 * 16; i += blockDim.x) NW[i] = gNW[i];
+    Smem s;
+    const uint32_t base = (uint32_t)__cvta_generic_to_shared(smem);
+    const uint32_t tab0 = (base + 0xFFFFu) & ~0xFFFFu;
+    unsigned char* img = smem + (tab0 - base);
+    s.ok = true;
+    s.lo = smem; s.lo_bytes = tab0 - base;
+    s.hi = img + kImgBytes; s.hi_bytes = kDynSmem - kImgBytes - (tab0 - base);
+    const uint4* src = reinterpret_cast<const uint4*>(tab->image);
+    uint4* dst = reinterpret_cast<uint4*>(img);
+    for (uint32_t i = threadIdx.x; i < kImgBytes / 16; i += blockDim.x) dst[i] = src[i];
+    uint32_t* nw = reinterpret_cast<uint32_t*>(s.take(8 * 8 * 16 * 4));
+    if (nw) {
+        const uint32_t* gNW = &tab->NW[0][0][0];
+        for (uint32_t i = threadIdx.x; i < 8 * 8 * 16; i += blockDim.x) nw[i] = gNW[i];
+    }
+    s.NW = nw;
+    const uint32_t lane4 = (threadIdx.x & 31u) * 4u;
+    s.L01 = (tab0 + kImgA01) | lane4;
+    s.L23 = (tab0 + kImgA23) | lane4;
+    s.LNK = (tab0 + kImgNK) | lane4;
     __syncthreads();
-    SmemTables t;
-    t.G = G; t.NK = NK; t.NW = NW;
-    return t;
+    return s;
+}
+
+template <int OFF>
+__device__ __forceinline__ uint32_t lds_off(uint32_t addr)
+{
+    uint32_t v;
+    asm("ld.shared.u32 %0, [%1+%2];" : "=r"(v) : "r"(addr), "n"(OFF));
+    return v;
 }
 
 __device__ __forceinline__ void team_bar(uint32_t team)
@@ -54,46 +87,42 @@ __device__ __forceinline__ void team_bar(uint32_t team)
     asm volatile("bar.sync %0, %1;" ::"r"(team + 1), "r"(kTeamThreads) : "memory");
 }
 
-// One chain step: (state ^ word) advanced over 128 bytes.  Gl = G + lane.
-__device__ __forceinline__ uint32_t chain_step(const uint32_t* Gl, uint32_t x)
+// One chain step: (state ^ word) advanced over 128 bytes.
+__device__ __forceinline__ uint32_t chain_step(const Smem& S, uint32_t x)
 {
-    const char* p = reinterpret_cast<const char*>(Gl);
-    uint32_t a = *reinterpret_cast<const uint32_t*>(p + ((x << 7) & 0x7F80u));
-    uint32_t b = *reinterpret_cast<const uint32_t*>(p + 32768 + ((x >> 1) & 0x7F80u));
-    uint32_t c = *reinterpret_cast<const uint32_t*>(p + 65536 + ((x >> 9) & 0x7F80u));
-    uint32_t d = *reinterpret_cast<const uint32_t*>(p + 98304 + ((x >> 17) & 0x7F80u));
+    const uint32_t a = lds_off<0>(__byte_perm(x, S.L01, 0x7604));
+    const uint32_t b = lds_off<128>(__byte_perm(x, S.L01, 0x7614));
+    const uint32_t c = lds_off<0>(__byte_perm(x, S.L23, 0x7624));
+    const uint32_t d = lds_off<128>(__byte_perm(x, S.L23, 0x7634));
     return a ^ b ^ c ^ d;
 }
 
-// Lane finish: x advanced over 128 - 4*lane bytes.  NKl = NK + lane.
-__device__ __forceinline__ uint32_t lane_finish(const uint32_t* NKl, uint32_t x)
+// Lane finish: x advanced over 128 - 4*lane bytes (eight nibble lookups).
+__device__ __forceinline__ uint32_t lane_finish(const Smem& S, uint32_t x)
 {
-    const char* p = reinterpret_cast<const char*>(NKl);
-    uint32_t r = 0;
-#pragma unroll
-    for (int n = 0; n < 8; n++)
-        r ^= *reinterpret_cast<const uint32_t*>(p + n * 2048 + (((x >> (4 * n)) & 15u) << 7));
+    const uint32_t xe = x & 0x0F0F0F0Fu, xo = (x >> 4) & 0x0F0F0F0Fu;
+    uint32_t r = lds_off<0x0000>(__byte_perm(xe, S.LNK, 0x7604)) ^ lds_off<0x0080>(__byte_perm(xo, S.LNK, 0x7604));
+    r ^= lds_off<0x1000>(__byte_perm(xe, S.LNK, 0x7614)) ^ lds_off<0x1080>(__byte_perm(xo, S.LNK, 0x7614));
+    r ^= lds_off<0x2000>(__byte_perm(xe, S.LNK, 0x7624)) ^ lds_off<0x2080>(__byte_perm(xo, S.LNK, 0x7624));
+    r ^= lds_off<0x3000>(__byte_perm(xe, S.LNK, 0x7634)) ^ lds_off<0x3080>(__byte_perm(xo, S.LNK, 0x7634));
     return r;
 }
 
 // CRC state (zero start) of a warp's 2048-byte block from the 16 words each lane holds.
-__device__ __forceinline__ uint32_t warp_block_digest(const SmemTables& T, const uint32_t (&w)[kWordsPerLane],
-                                                      uint32_t lane)
+__device__ __forceinline__ uint32_t warp_block_digest(const Smem& S, const uint32_t (&w)[kWordsPerLane])
 {
-    const uint32_t* Gl = T.G + lane;
     uint32_t s = 0;
 #pragma unroll
-    for (int i = 0; i < 15; i++) s = chain_step(Gl, s ^ w[i]);
-    uint32_t r = lane_finish(T.NK + lane, s ^ w[15]);
-    return __reduce_xor_sync(0xFFFFFFFFu, r);
+    for (int i = 0; i < 15; i++) s = chain_step(S, s ^ w[i]);
+    return __reduce_xor_sync(0xFFFFFFFFu, lane_finish(S, s ^ w[15]));
 }
 
 // Place a warp's block digest inside the tile: advance over 2048*(7 - warp) bytes.  Returns the
 // warp's contribution to the tile digest in every lane.
-__device__ __forceinline__ uint32_t warp_place(const SmemTables& T, uint32_t digest, uint32_t warp, uint32_t lane)
+__device__ __forceinline__ uint32_t warp_place(const Smem& S, uint32_t digest, uint32_t warp, uint32_t lane)
 {
     uint32_t v = 0;
-    if (lane < 8) v = T.NW[(warp * 8 + lane) * 16 + ((digest >> (4 * lane)) & 15u)];
+    if (lane < 8) v = S.NW[(warp * 8 + lane) * 16 + ((digest >> (4 * lane)) & 15u)];
     return __reduce_xor_sync(0xFFFFFFFFu, v);
 }
 
@@ -165,31 +194,31 @@ __device__ __forceinline__ void load_tile_words(const unsigned char* tile, uint3
     for (int i = 0; i < 16; i++) w[i] = ld_stream_u32(p + i * 128);
 }
 
-// Any tile of `len` (1..16384) real bytes, right-aligned in a virtual tile whose leading
-// 16384 - len bytes are zero (leading zeros do not change a zero-start CRC state).  When
-// `first_in_chunk`, the chunk's first four bytes are complemented (the all-ones CRC init).
-// `skip_lo..skip_lo+3` (real byte offsets, or a negative value) are read as zero.
-__device__ __forceinline__ void load_tile_words_guarded(const unsigned char* tile, uint32_t len, bool first_in_chunk,
-                                                        int64_t skip_lo, uint32_t warp, uint32_t lane,
-                                                        uint32_t (&w)[kWordsPerLane])
+// One 32-bit word of a tile of `len` (1..16384) real bytes that is right-aligned in a virtual
+// tile whose leading 16384 - len bytes are zero (leading zeros do not change a zero-start CRC
+// state).  `vb` is the word's byte offset inside the virtual tile.  When `first_in_chunk`, the
+// chunk's first four bytes are complemented (the all-ones CRC init).  Rare path (one tile per
+// call at most), kept out of line.
+__device__ __noinline__ uint32_t guarded_word(const unsigned char* tile, uint32_t len, bool first_in_chunk, uint32_t vb)
 {
     const int64_t pad = (int64_t)kTile - (int64_t)len;
-#pragma unroll
-    for (int i = 0; i < 16; i++) {
-        int64_t vb = (int64_t)(warp * 16 + i) * 128 + lane * 4;
-        uint32_t word = 0;
-#pragma unroll
-        for (int j = 0; j < 4; j++) {
-            int64_t rb = vb + j - pad;
-            if (rb >= 0) {
-                uint32_t b = tile[rb];
-                if (rb >= skip_lo && rb < skip_lo + 4) b = 0;
-                if (first_in_chunk && rb < 4) b ^= 0xFFu;
-                word |= b << (8 * j);
-            }
+    uint32_t word = 0;
+    for (int j = 0; j < 4; j++) {
+        const int64_t rb = (int64_t)vb + j - pad;
+        if (rb >= 0) {
+            uint32_t b = tile[rb];
+            if (first_in_chunk && rb < 4) b ^= 0xFFu;
+            word |= b << (8 * j);
         }
-        w[i] = word;
     }
+    return word;
+}
+
+__device__ __forceinline__ void load_tile_words_guarded(const unsigned char* tile, uint32_t len, bool first_in_chunk,
+                                                        uint32_t warp, uint32_t lane, uint32_t (&w)[kWordsPerLane])
+{
+#pragma unroll
+    for (int i = 0; i < 16; i++) w[i] = guarded_word(tile, len, first_in_chunk, (warp * 16 + i) * 128 + lane * 4);
 }
 
 // CRC32C of a short run computed byte by byte (chunks shorter than four bytes).

@@ -36,6 +36,7 @@ struct Geo {
     uint32_t k_chunk;         // x^(8 chunk_bytes)
     uint32_t k_last_chunk;    // x^(8 last_chunk_len)
     uint32_t n_meta_slices;   // ceil(meta_end / 16384)
+    uint32_t tpc_shift;       // log2(tiles_per_chunk) when that is a power of two, else 32
 };
 
 struct Ctrl {                 // first 256 bytes of the workspace
@@ -122,7 +123,19 @@ static bool make_geo(uint64_t nbytes, uint32_t chunk_bytes, Geo& g)
     g.k_chunk = x_pow_bytes(chunk_bytes);
     g.k_last_chunk = x_pow_bytes(g.last_chunk_len);
     g.n_meta_slices = (uint32_t)((g.meta_end + kTile - 1) / kTile);
+    g.tpc_shift = 32;
+    for (uint32_t k = 0; k < 32; k++)
+        if (g.tiles_per_chunk == (1u << k)) g.tpc_shift = k;
     return true;
+}
+
+__device__ __forceinline__ uint32_t chunk_of(const Geo& g, uint32_t t)
+{
+    return g.tpc_shift < 32 ? t >> g.tpc_shift : t / g.tiles_per_chunk;
+}
+__device__ __forceinline__ bool first_in_chunk(const Geo& g, uint32_t t)
+{
+    return g.tpc_shift < 32 ? (t & (g.tiles_per_chunk - 1u)) == 0u : (t % g.tiles_per_chunk) == 0u;
 }
 
 __device__ __forceinline__ uint64_t chunk_len_dev(const Geo& g, uint32_t c)
@@ -133,33 +146,28 @@ __device__ __forceinline__ uint64_t chunk_len_dev(const Geo& g, uint32_t c)
 // ------------------------------------------------------------------ per-team shared state
 
 struct TeamCtl {
-    uint32_t wtab[32];     // per group: base | w << 8
-    uint32_t wdig[8];      // per warp: its contribution to the tile digest
-    uint32_t next;         // next tile ticket (0xFFFFFFFF: stop)
-    uint32_t status;
-    unsigned long long excl;
+    uint32_t wdig[2][8];   // per warp: its contribution to the tile digest (double buffered)
+    uint32_t next;
+    uint32_t pad[3];
 };
-constexpr uint32_t kTeamSmemPlain = sizeof(TeamCtl);
+static_assert(sizeof(TeamCtl) % 16 == 0, "team control block keeps 16-byte alignment");
 
-// Digest of the team's current tile from the words each lane holds; result in wdig[] (valid
-// for thread 0 after the next team barrier).  `init_fold`: complement the tile's first word.
-__device__ __forceinline__ void tile_digest_to_smem(const SmemTables& T, uint32_t (&w)[kWordsPerLane], bool init_fold,
-                                                    uint32_t warp, uint32_t lane, TeamCtl* tc)
+// A warp's contribution to the digest of the team's tile, from the 16 words each lane holds
+// (same value in every lane).  `init_fold`: complement the tile's first word, which folds the
+// CRC's all-ones start value into the first tile of a chunk.
+__device__ __forceinline__ uint32_t tile_digest_part(const Smem& S, uint32_t (&w)[kWordsPerLane], bool init_fold,
+                                                     uint32_t warp, uint32_t lane)
 {
     const uint32_t m = (init_fold && warp == 0 && lane == 0) ? 0xFFFFFFFFu : 0u;
     w[0] ^= m;
-    uint32_t d = warp_block_digest(T, w, lane);
+    const uint32_t d = warp_block_digest(S, w);
     w[0] ^= m;
-    uint32_t v = warp_place(T, d, warp, lane);
-    if (lane == 0) tc->wdig[warp] = v;
+    return warp_place(S, d, warp, lane);
 }
 
-__device__ __forceinline__ uint32_t team_digest(const TeamCtl* tc)
+__device__ __forceinline__ uint32_t xor8(const uint32_t* p)
 {
-    uint32_t d = 0;
-#pragma unroll
-    for (int i = 0; i < 8; i++) d ^= tc->wdig[i];
-    return d;
+    return p[0] ^ p[1] ^ p[2] ^ p[3] ^ p[4] ^ p[5] ^ p[6] ^ p[7];
 }
 
 // CRC32C of chunk c from its tiles' digests (Horner over tiles; the all-ones init was folded
@@ -230,28 +238,48 @@ __device__ uint32_t combine_chunk_crcs(const Geo& g, const uint32_t* crc, uint32
 
 // ------------------------------------------------------------------ wm_checksum
 
+// Tile digests of the whole cache: static striding over tiles, next tile's words prefetched
+// into registers while the current one is digested; one team barrier per tile.
 template <int TEAMS>
 __global__ void __launch_bounds__(TEAMS * 256, 1)
 k_tile_digests(const unsigned char* __restrict__ cache, Geo g, Ws ws, const Tables* __restrict__ tab)
 {
     extern __shared__ __align__(16) unsigned char smem[];
-    SmemTables T = load_tables(smem, tab);
+    Smem S = setup_smem(smem, tab);
     const uint32_t team = threadIdx.x / kTeamThreads, tt = threadIdx.x % kTeamThreads;
     const uint32_t warp = tt / 32, lane = tt % 32;
-    TeamCtl* tc = reinterpret_cast<TeamCtl*>(smem + kSmemTables + team * kTeamSmemPlain);
-    const uint32_t stride = gridDim.x * TEAMS;
-    for (uint32_t t = blockIdx.x * TEAMS + team; t < g.n_tiles; t += stride) {
-        const uint64_t off = (uint64_t)t * kTile;
-        const uint64_t left = g.nbytes - off;
-        const bool first = (t % g.tiles_per_chunk) == 0;
-        uint32_t w[kWordsPerLane];
-        bool fold;
-        if (left >= kTile) { load_tile_words(cache + off, warp, lane, w); fold = first; }
-        else { load_tile_words_guarded(cache + off, (uint32_t)left, first, -8, warp, lane, w); fold = false; }
-        tile_digest_to_smem(T, w, fold, warp, lane, tc);
+    TeamCtl* tc = reinterpret_cast<TeamCtl*>(S.take(TEAMS * sizeof(TeamCtl)));
+    if (!S.ok) { if (threadIdx.x == 0) atomicOr(&ws.ctrl->err, 4u); return; }
+    tc += team;
+    const uint64_t stride = (uint64_t)gridDim.x * TEAMS;
+    uint64_t t = (uint64_t)blockIdx.x * TEAMS + team;
+    uint32_t par = 0;
+
+    auto fetch = [&](uint64_t tile, uint32_t (&d)[kWordsPerLane]) {
+        if (tile < g.n_tiles && g.nbytes - tile * kTile >= kTile) load_tile_words(cache + tile * kTile, warp, lane, d);
+    };
+    auto process = [&](uint64_t tile, uint32_t (&d)[kWordsPerLane]) {
+        const uint64_t left = g.nbytes - tile * kTile;
+        const bool first = first_in_chunk(g, (uint32_t)tile);
+        const bool full = left >= kTile;
+        if (!full) load_tile_words_guarded(cache + tile * kTile, (uint32_t)left, first, warp, lane, d);
+        const uint32_t v = tile_digest_part(S, d, first && full, warp, lane);
+        if (lane == 0) tc->wdig[par][warp] = v;
         team_bar(team);
-        if (tt == 0) ws.dig[t] = team_digest(tc);
-        team_bar(team);
+        if (tt == 0) ws.dig[tile] = xor8(tc->wdig[par]);
+        par ^= 1u;
+    };
+
+    uint32_t da[kWordsPerLane], db[kWordsPerLane];
+    fetch(t, da);
+    while (t < g.n_tiles) {
+        fetch(t + stride, db);
+        process(t, da);
+        t += stride;
+        if (t >= g.n_tiles) break;
+        fetch(t + stride, da);
+        process(t, db);
+        t += stride;
     }
 }
 
@@ -461,25 +489,25 @@ struct EncTeamCtl {
     uint32_t pad;
     unsigned long long excl;
 };
+static_assert(sizeof(EncTeamCtl) % 16 == 0, "team control block keeps 16-byte alignment");
 constexpr uint32_t kTeamSmemEncode = kTile + sizeof(EncTeamCtl);
 
 struct TileInfo {
+    uint32_t t, c, left;
     bool valid, present, full, first;
-    uint32_t c, left;
-    uint64_t off;
 };
 
 __device__ __forceinline__ TileInfo tile_info(const Geo& g, const uint8_t* __restrict__ dirty, uint32_t t)
 {
     TileInfo ti;
+    ti.t = t;
     ti.valid = t < g.n_tiles;
-    ti.present = false; ti.full = false; ti.first = false; ti.c = 0; ti.left = 0; ti.off = 0;
+    ti.present = false; ti.full = false; ti.first = false; ti.c = 0; ti.left = 0;
     if (!ti.valid) return ti;
-    ti.c = t / g.tiles_per_chunk;
-    ti.first = (t % g.tiles_per_chunk) == 0;
+    ti.c = chunk_of(g, t);
+    ti.first = first_in_chunk(g, t);
     ti.present = !dirty || dirty[ti.c] != 0;
-    ti.off = (uint64_t)t * kTile;
-    const uint64_t left = g.nbytes - ti.off;
+    const uint64_t left = g.nbytes - (uint64_t)t * kTile;
     ti.full = left >= kTile;
     ti.left = ti.full ? kTile : (uint32_t)left;
     return ti;
@@ -492,22 +520,66 @@ __device__ __forceinline__ uint32_t encoded_len(const TileInfo& ti, uint32_t S)
     return S <= 253u ? 8256u + 32u * S : kTile;
 }
 
+// Bit-pack the lane's eight exponent deltas (e4a, e4b: bytes in coded order, each < 2^W after
+// the base is subtracted) into W bytes at ep.  W is a compile-time constant so that every
+// shift and mask is an immediate and the store uses the widest aligned form.
+template <int W>
+__device__ __forceinline__ void pack_group(uint32_t e4a, uint32_t e4b, uint32_t base, unsigned char* ep)
+{
+    const uint32_t b4 = base * 0x01010101u;
+    const uint32_t da = e4a - b4, db = e4b - b4;
+    if (W == 8) {
+        *reinterpret_cast<uint2*>(ep) = make_uint2(da, db);
+        return;
+    }
+    constexpr int V = W & 7;                              // W == 8 returned above; keeps shifts in range
+    constexpr uint32_t sh = 8 - V;
+    constexpr uint32_t m1 = ((1u << V) - 1u) * 0x00010001u;
+    constexpr uint32_t m2 = (1u << (2 * V)) - 1u;
+    const uint32_t ya = (da & m1) | ((da >> sh) & (m1 << V));
+    const uint32_t yb = (db & m1) | ((db >> sh) & (m1 << V));
+    const uint32_t za = (ya & m2) | ((ya >> (16 - 2 * V)) & (m2 << (2 * V)));
+    const uint32_t zb = (yb & m2) | ((yb >> (16 - 2 * V)) & (m2 << (2 * V)));
+    const uint32_t lo = za + (zb << (4 * V));            // disjoint bit fields: add == or
+    const uint32_t hi = (V > 4) ? (zb >> ((32 - 4 * V) & 31)) : 0u;
+    if (W == 1) ep[0] = (unsigned char)lo;
+    else if (W == 2) *reinterpret_cast<uint16_t*>(ep) = (uint16_t)lo;
+    else if (W == 3) { ep[0] = (unsigned char)lo; ep[1] = (unsigned char)(lo >> 8); ep[2] = (unsigned char)(lo >> 16); }
+    else if (W == 4) *reinterpret_cast<uint32_t*>(ep) = lo;
+    else if (W == 5) {
+        ep[0] = (unsigned char)lo; ep[1] = (unsigned char)(lo >> 8); ep[2] = (unsigned char)(lo >> 16);
+        ep[3] = (unsigned char)(lo >> 24); ep[4] = (unsigned char)hi;
+    } else if (W == 6) {
+        reinterpret_cast<uint16_t*>(ep)[0] = (uint16_t)lo; reinterpret_cast<uint16_t*>(ep)[1] = (uint16_t)(lo >> 16);
+        reinterpret_cast<uint16_t*>(ep)[2] = (uint16_t)hi;
+    } else {
+        ep[0] = (unsigned char)lo; ep[1] = (unsigned char)(lo >> 8); ep[2] = (unsigned char)(lo >> 16);
+        ep[3] = (unsigned char)(lo >> 24); ep[4] = (unsigned char)hi; ep[5] = (unsigned char)(hi >> 8);
+        ep[6] = (unsigned char)(hi >> 16);
+    }
+}
+
 // Single-pass fused checksum + encode.  Per team, software pipelined over tiles X (being
 // packed and written out) and Y (being checksummed and measured):
 //     pack X into shared memory | digest + exponent ranges of Y | publish len(Y) |
-//     look back for X's offset | claim Z and start its loads | copy X out
-// A team never waits for another team while it holds a claimed tile whose length is not yet
-// published: len(Y) goes out before the look-back for X starts, and Z is claimed only after
-// that look-back has returned.  This keeps every wait one hop long.
+//     wait for X's offset | claim Z and start its loads | copy X out
+// A team never waits while it holds a claimed tile whose length is not yet published: len(Y)
+// goes out before the wait for X starts, and Z is claimed only after that wait has returned.
 template <int TEAMS>
 __global__ void __launch_bounds__(TEAMS * 256 + 32, 1)
 k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restrict__ dirty,
          unsigned char* __restrict__ wire, uint64_t wire_cap, Ws ws, const Tables* __restrict__ tab)
 {
     extern __shared__ __align__(16) unsigned char smem[];
-    SmemTables T = load_tables(smem, tab);
+    Smem S = setup_smem(smem, tab);
     const uint32_t team = threadIdx.x / kTeamThreads, tt = threadIdx.x % kTeamThreads;
     const uint32_t warp = tt / 32, lane = tt % 32;
+    unsigned char* out = nullptr;
+    for (int i = 0; i < TEAMS; i++) {          // every thread carves the same blocks in the same order
+        unsigned char* p = S.take(kTeamSmemEncode);
+        if ((uint32_t)i == team) out = p;
+    }
+    if (!S.ok) { if (threadIdx.x == 0) atomicOr(&ws.ctrl->err, 4u); return; }
     if (team == TEAMS) {
         // the extra warp: one of them, grid-wide, becomes the scanner; the others leave
         uint32_t won = 0;
@@ -516,23 +588,16 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
         if (won) scan_tile_lengths(ws.state, g.n_tiles, lane, ws.ctrl);
         return;
     }
-    unsigned char* out = smem + kSmemTables + team * kTeamSmemEncode;
     EncTeamCtl* tc = reinterpret_cast<EncTeamCtl*>(out + kTile);
     unsigned char* dir = wire + 64;
     uint16_t* tile_tab = reinterpret_cast<uint16_t*>(wire + 64 + 16ull * g.n_chunks);
 
     // digest and per-group exponent range of one tile; results go to wdig[par], wtab[par]
-    auto phase_a = [&](const TileInfo& ti, uint32_t (&d)[kWordsPerLane], uint32_t par) {
+    auto measure = [&](const TileInfo& ti, uint32_t (&d)[kWordsPerLane], uint32_t par) {
         if (!ti.present) return;
-        if (!ti.full) load_tile_words_guarded(cache + ti.off, ti.left, ti.first, -8, warp, lane, d);
-        {
-            const uint32_t m = (ti.first && ti.full && warp == 0 && lane == 0) ? 0xFFFFFFFFu : 0u;
-            d[0] ^= m;
-            const uint32_t dg = warp_block_digest(T, d, lane);
-            d[0] ^= m;
-            const uint32_t v = warp_place(T, dg, warp, lane);
-            if (lane == 0) tc->wdig[par][warp] = v;
-        }
+        if (!ti.full) load_tile_words_guarded(cache + (uint64_t)ti.t * kTile, ti.left, ti.first, warp, lane, d);
+        const uint32_t v = tile_digest_part(S, d, ti.first && ti.full, warp, lane);
+        if (lane == 0) tc->wdig[par][warp] = v;
         if (ti.full) {
 #pragma unroll
             for (int j = 0; j < 4; j++) {
@@ -552,46 +617,32 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
     auto sum_widths = [&](uint32_t par) {
         return __reduce_add_sync(0xFFFFFFFFu, (tc->wtab[par][lane] >> 8) & 15u);
     };
+    auto fetch = [&](const TileInfo& ti, uint32_t (&d)[kWordsPerLane]) {
+        if (ti.present && ti.full) load_tile_words(cache + (uint64_t)ti.t * kTile, warp, lane, d);
+    };
 
-    // ---- prologue: X claimed, loaded, measured and published; Y claimed and loading
-    uint32_t dX[kWordsPerLane], dY[kWordsPerLane];
-    if (tt == 0) tc->next = next_ticket(ws.ctrl);
-    team_bar(team);
-    uint32_t tX = tc->next;
-    TileInfo iX = tile_info(g, dirty, tX);
-    if (iX.present && iX.full) load_tile_words(cache + iX.off, warp, lane, dX);
+    // One pipeline step: pack X (words in dP), measure Y (words in dM), place X, claim Z and
+    // start loading it into dP.  Returns with X <- Y, Y <- Z and the roles of dP / dM swapped.
+    TileInfo iX = tile_info(g, dirty, 0xFFFFFFFFu), iY = iX;
     uint32_t par = 0;
-    phase_a(iX, dX, par);
-    team_bar(team);
-    if (warp == 0 && iX.valid) {
-        const uint32_t S = (iX.present && iX.full) ? sum_widths(par) : 0u;
-        if (lane == 0) { publish_len(ws.state, tX, encoded_len(iX, S)); tc->next = next_ticket(ws.ctrl); }
-    }
-    team_bar(team);
-    uint32_t tY = iX.valid ? tc->next : 0xFFFFFFFFu;
-    TileInfo iY = tile_info(g, dirty, tY);
-    if (iY.present && iY.full) load_tile_words(cache + iY.off, warp, lane, dY);
-
-    while (iX.valid) {
+    auto step = [&](uint32_t (&dP)[kWordsPerLane], uint32_t (&dM)[kWordsPerLane]) {
         team_bar(team);                                               // bar0: out buffer free
-
-        // ---- pack X
         uint32_t enc_len = 0, entry = 0;
-        bool staged = false;               // encoded tile sits in `out`
+        bool staged = false;                                          // encoded tile sits in `out`
         if (iX.present && iX.full) {
             const uint32_t wt = tc->wtab[par][lane];
             const uint32_t wv = (wt >> 8) & 15u;
             uint32_t incl = wv;
 #pragma unroll
             for (int d = 1; d < 32; d <<= 1) {
-                uint32_t o = __shfl_up_sync(0xFFFFFFFFu, incl, d);
+                const uint32_t o = __shfl_up_sync(0xFFFFFFFFu, incl, d);
                 if (lane >= (uint32_t)d) incl += o;
             }
-            const uint32_t S = __shfl_sync(0xFFFFFFFFu, incl, 31);
+            const uint32_t Ssum = __shfl_sync(0xFFFFFFFFu, incl, 31);
             staged = true;
-            if (S <= 253u) {
-                enc_len = 8256u + 32u * S;
-                entry = 258u + S;
+            if (Ssum <= 253u) {
+                enc_len = 8256u + 32u * Ssum;
+                entry = 258u + Ssum;
                 if (warp == 0) reinterpret_cast<uint16_t*>(out)[lane] = (uint16_t)desc_of(wt & 0xFFu, wv);
 #pragma unroll
                 for (int j = 0; j < 4; j++) {
@@ -602,29 +653,23 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
                     uint32_t Tr[4];
 #pragma unroll
                     for (int r = 0; r < 4; r++) {
-                        const uint32_t W = dX[4 * j + r];
+                        const uint32_t W = dP[4 * j + r];
                         Tr[r] = ((W << 1) & 0xFFFEFFFEu) | ((W >> 15) & 0x00010001u);
                     }
                     const uint32_t sma = __byte_perm(Tr[0], Tr[1], 0x6420), smb = __byte_perm(Tr[2], Tr[3], 0x6420);
                     *reinterpret_cast<uint2*>(out + 64 + 256 * gi + 8 * lane) = make_uint2(sma, smb);
-                    if (wd) {
-                        const uint32_t b4 = base * 0x01010101u;
-                        const uint32_t da = __byte_perm(Tr[0], Tr[1], 0x7531) - b4;
-                        const uint32_t db = __byte_perm(Tr[2], Tr[3], 0x7531) - b4;
-                        const uint32_t sh = 8u - wd;
-                        const uint32_t ya = (da & 0x00FF00FFu) | ((da & 0xFF00FF00u) >> sh);
-                        const uint32_t yb = (db & 0x00FF00FFu) | ((db & 0xFF00FF00u) >> sh);
-                        const uint32_t za = (ya & 0xFFFFu) | ((ya >> 16) << (2 * wd));
-                        const uint32_t zb = (yb & 0xFFFFu) | ((yb >> 16) << (2 * wd));
-                        const unsigned long long P = (unsigned long long)za | ((unsigned long long)zb << (4 * wd));
-                        unsigned char* ep = out + 8256 + 32 * exg + lane * wd;
-                        if (wd == 4) *reinterpret_cast<uint32_t*>(ep) = (uint32_t)P;
-                        else if (wd == 8) *reinterpret_cast<uint2*>(ep) = make_uint2((uint32_t)P, (uint32_t)(P >> 32));
-                        else if ((wd & 1u) == 0) {
-                            for (uint32_t k = 0; k < wd; k += 2) *reinterpret_cast<uint16_t*>(ep + k) = (uint16_t)(P >> (8 * k));
-                        } else {
-                            for (uint32_t k = 0; k < wd; k++) ep[k] = (unsigned char)(P >> (8 * k));
-                        }
+                    const uint32_t e4a = __byte_perm(Tr[0], Tr[1], 0x7531), e4b = __byte_perm(Tr[2], Tr[3], 0x7531);
+                    unsigned char* ep = out + 8256 + 32 * exg + lane * wd;
+                    switch (wd) {          // uniform across the warp
+                        case 1: pack_group<1>(e4a, e4b, base, ep); break;
+                        case 2: pack_group<2>(e4a, e4b, base, ep); break;
+                        case 3: pack_group<3>(e4a, e4b, base, ep); break;
+                        case 4: pack_group<4>(e4a, e4b, base, ep); break;
+                        case 5: pack_group<5>(e4a, e4b, base, ep); break;
+                        case 6: pack_group<6>(e4a, e4b, base, ep); break;
+                        case 7: pack_group<7>(e4a, e4b, base, ep); break;
+                        case 8: pack_group<8>(e4a, e4b, base, ep); break;
+                        default: break;
                     }
                 }
             } else {
@@ -632,36 +677,31 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
                 entry = 512u;
                 uint32_t* o32 = reinterpret_cast<uint32_t*>(out) + warp * 512u + lane;
 #pragma unroll
-                for (int i = 0; i < 16; i++) o32[i * 32] = dX[i];
+                for (int i = 0; i < 16; i++) o32[i * 32] = dP[i];
             }
         } else if (iX.present) {
             enc_len = iX.left;
             entry = 0xFFFFu;
         }
 
-        // ---- measure Y (its data was requested one iteration ago)
-        phase_a(iY, dY, par ^ 1u);
+        measure(iY, dM, par ^ 1u);
         team_bar(team);                                               // bar1: wtab[par^1] complete
 
         if (warp == 0) {
             if (iY.valid) {
-                const uint32_t S = (iY.present && iY.full) ? sum_widths(par ^ 1u) : 0u;
-                if (lane == 0) publish_len(ws.state, tY, encoded_len(iY, S));
+                const uint32_t Sy = (iY.present && iY.full) ? sum_widths(par ^ 1u) : 0u;
+                if (lane == 0) publish_len(ws.state, iY.t, encoded_len(iY, Sy));
             }
             if (lane == 0) {
-                tc->excl = wait_prefix(ws.state, tX, ws.ctrl);
+                tc->excl = wait_prefix(ws.state, iX.t, ws.ctrl);
                 tc->next = iY.valid ? next_ticket(ws.ctrl) : 0xFFFFFFFFu;
             }
         }
         team_bar(team);                                               // bar2: offset known, out complete
 
-        // ---- claim Z, start its loads into X's (now free) registers
-        const uint32_t tZ = tc->next;
-        const TileInfo iZ = tile_info(g, dirty, tZ);
-        uint32_t dZ[kWordsPerLane];
-        if (iZ.present && iZ.full) load_tile_words(cache + iZ.off, warp, lane, dZ);
+        const TileInfo iZ = tile_info(g, dirty, tc->next);
+        fetch(iZ, dP);                                                // dP is free: X sits in `out`
 
-        // ---- move X to its place in the wire image
         const unsigned long long excl = tc->excl;
         if (iX.present) {
             const uint64_t dst = g.meta_end + excl;
@@ -671,26 +711,40 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
                 for (uint32_t i = tt * 16; i < enc_len; i += kTeamThreads * 16)
                     *reinterpret_cast<uint4*>(wire + dst + i) = *reinterpret_cast<const uint4*>(out + i);
             } else {
-                for (uint32_t i = tt; i < enc_len; i += kTeamThreads) wire[dst + i] = cache[iX.off + i];
+                const unsigned char* src = cache + (uint64_t)iX.t * kTile;
+                for (uint32_t i = tt; i < enc_len; i += kTeamThreads) wire[dst + i] = src[i];
             }
         }
         if (tt == 0) {
-            tile_tab[tX] = (uint16_t)entry;
-            if (iX.present) {
-                uint32_t dg = 0;
-#pragma unroll
-                for (int i = 0; i < 8; i++) dg ^= tc->wdig[par][i];
-                ws.dig[tX] = dg;
-            }
+            tile_tab[iX.t] = (uint16_t)entry;
+            if (iX.present) ws.dig[iX.t] = xor8(tc->wdig[par]);
             if (iX.first) *reinterpret_cast<unsigned long long*>(dir + 16ull * iX.c) = excl;
         }
-
-        // ---- rotate
-        tX = tY; iX = iY;
-        tY = tZ; iY = iZ;
-#pragma unroll
-        for (int i = 0; i < 16; i++) { dX[i] = dY[i]; dY[i] = dZ[i]; }
+        iX = iY;
+        iY = iZ;
         par ^= 1u;
+    };
+
+    // ---- prologue: X claimed, loaded, measured and published; Y claimed and loading
+    uint32_t dA[kWordsPerLane], dB[kWordsPerLane];
+    if (tt == 0) tc->next = next_ticket(ws.ctrl);
+    team_bar(team);
+    iX = tile_info(g, dirty, tc->next);
+    fetch(iX, dA);
+    measure(iX, dA, par);
+    team_bar(team);
+    if (warp == 0 && iX.valid) {
+        const uint32_t Sx = (iX.present && iX.full) ? sum_widths(par) : 0u;
+        if (lane == 0) { publish_len(ws.state, iX.t, encoded_len(iX, Sx)); tc->next = next_ticket(ws.ctrl); }
+    }
+    team_bar(team);
+    iY = tile_info(g, dirty, iX.valid ? tc->next : 0xFFFFFFFFu);
+    fetch(iY, dB);
+
+    while (iX.valid) {
+        step(dA, dB);
+        if (!iX.valid) break;
+        step(dB, dA);
     }
 }
 
@@ -766,9 +820,10 @@ k_meta_crc(unsigned char* wire, uint64_t wire_len, Geo g, Ws ws, const Tables* _
     extern __shared__ __align__(16) unsigned char smem[];
     __shared__ bool s_last;
     __shared__ int s_format_bad;
-    SmemTables T = load_tables(smem, tab);
+    Smem S = setup_smem(smem, tab);
     const uint32_t warp = threadIdx.x / 32, lane = threadIdx.x % 32;
-    TeamCtl* tc = reinterpret_cast<TeamCtl*>(smem + kSmemTables);
+    TeamCtl* tc = reinterpret_cast<TeamCtl*>(S.take(sizeof(TeamCtl)));
+    if (!S.ok) { if (threadIdx.x == 0) atomicOr(&ws.ctrl->err, 4u); return; }
 
     if (mode == 1) {
         // FORMAT check by every block (cheap, keeps the gate decision local)
@@ -815,10 +870,13 @@ k_meta_crc(unsigned char* wire, uint64_t wire_len, Geo g, Ws ws, const Tables* _
         }
         w[i] = v;
     }
-    tile_digest_to_smem(T, w, false, warp, lane, tc);
+    {
+        const uint32_t v = tile_digest_part(S, w, false, warp, lane);
+        if (lane == 0) tc->wdig[0][warp] = v;
+    }
     __syncthreads();
     if (threadIdx.x == 0) {
-        ws.mdig[s] = team_digest(tc);
+        ws.mdig[s] = xor8(tc->wdig[0]);
         __threadfence();
         s_last = atomicAdd(&ws.ctrl->done_b, 1u) == gridDim.x - 1;
     }
@@ -1003,6 +1061,58 @@ k_decode_struct_scan(const unsigned char* __restrict__ wire, uint64_t wire_len, 
     }
 }
 
+struct DecSlot {                 // what thread 0 prepares for a tile one iteration ahead
+    uint32_t t;                  // tile (>= n_tiles: none left)
+    uint32_t entry;              // tile table entry
+    uint32_t c;                  // chunk
+    uint32_t first;              // first tile of its chunk
+    unsigned long long src;      // offset of the encoded tile inside the wire image
+    unsigned long long pad;
+};
+struct DecTeamCtl {
+    uint32_t wdig[2][8];
+    DecSlot slot[2];
+};
+static_assert(sizeof(DecTeamCtl) % 16 == 0, "team control block keeps 16-byte alignment");
+
+// Inverse of pack_group: the lane's eight exponent bytes (two words, coded order) from the
+// aligned window (w0, w1, w2) that covers its W packed bytes; sh = 8 * (byte offset & 3).
+template <int W>
+__device__ __forceinline__ void unpack_group(uint32_t w0, uint32_t w1, uint32_t w2, uint32_t sh, uint32_t base,
+                                             uint32_t& ea, uint32_t& eb)
+{
+    const uint32_t lo = __funnelshift_r(w0, w1, sh);
+    const uint32_t hi = __funnelshift_r(w1, w2, sh);
+    uint32_t da, db;
+    if (W == 8) { da = lo; db = hi; }
+    else {
+        constexpr int V = W & 7;
+        constexpr uint32_t m4 = (1u << (4 * V)) - 1u;
+        constexpr uint32_t m2 = (1u << (2 * V)) - 1u;
+        constexpr uint32_t m1 = ((1u << V) - 1u) * 0x00010001u;
+        constexpr uint32_t sh1 = 8 - V;
+        const uint32_t za = lo & m4;
+        const uint32_t zb = (V <= 4 ? (lo >> (4 * V)) : __funnelshift_r(lo, hi, 4 * V)) & m4;
+        const uint32_t ya = (za & m2) | ((za << (16 - 2 * V)) & (m2 << 16));
+        const uint32_t yb = (zb & m2) | ((zb << (16 - 2 * V)) & (m2 << 16));
+        da = (ya & m1) | ((ya << sh1) & (m1 << 8));
+        db = (yb & m1) | ((yb << sh1) & (m1 << 8));
+    }
+    const uint32_t b4 = base * 0x01010101u;        // per byte (base + d) & 0xFF
+    ea = ((da & 0x7F7F7F7Fu) + (b4 & 0x7F7F7F7Fu)) ^ ((da ^ b4) & 0x80808080u);
+    eb = ((db & 0x7F7F7F7Fu) + (b4 & 0x7F7F7F7Fu)) ^ ((db ^ b4) & 0x80808080u);
+}
+
+__device__ __forceinline__ uint32_t ldg_u32(const void* p)
+{
+    uint32_t v;
+    asm volatile("ld.global.nc.u32 %0, [%1];" : "=r"(v) : "l"(p));
+    return v;
+}
+
+// Unpack + checksum of the decoded bytes.  Tiles are claimed by ticket; thread 0 of a team
+// looks up the next tile's table entry and source offset while the team decodes the current
+// one, so that chain of dependent loads is off the critical path.
 template <int TEAMS>
 __global__ void __launch_bounds__(TEAMS * 256, 1)
 k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restrict__ dst, Ws ws,
@@ -1010,43 +1120,53 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
 {
     if (ld_volatile_u32(&ws.ctrl->gate)) return;
     extern __shared__ __align__(16) unsigned char smem[];
-    SmemTables T = load_tables(smem, tab);
+    Smem S = setup_smem(smem, tab);
     const uint32_t team = threadIdx.x / kTeamThreads, tt = threadIdx.x % kTeamThreads;
     const uint32_t warp = tt / 32, lane = tt % 32;
-    TeamCtl* tc = reinterpret_cast<TeamCtl*>(smem + kSmemTables + team * kTeamSmemPlain);
+    DecTeamCtl* tc = reinterpret_cast<DecTeamCtl*>(S.take(TEAMS * sizeof(DecTeamCtl)));
+    if (!S.ok) { if (threadIdx.x == 0) atomicOr(&ws.ctrl->err, 4u); return; }
+    tc += team;
     const unsigned char* dir = wire + 64;
     const uint16_t* tab16 = reinterpret_cast<const uint16_t*>(wire + 64 + 16ull * g.n_chunks);
     const unsigned char* payload = wire + g.meta_end;
 
-    if (tt == 0) tc->next = atomicAdd(&ws.ctrl->ticket, 1u);
+    auto prepare = [&](DecSlot* sl) {       // thread 0 only
+        const uint32_t t = atomicAdd(&ws.ctrl->ticket, 1u);
+        sl->t = t;
+        if (t < g.n_tiles) {
+            const uint32_t e = tab16[t];
+            const uint32_t c = chunk_of(g, t);
+            sl->entry = e; sl->c = c; sl->first = first_in_chunk(g, t) ? 1u : 0u;
+            sl->src = e ? *reinterpret_cast<const unsigned long long*>(dir + 16ull * c) + ws.rel[t] : 0ull;
+        }
+    };
+
+    if (tt == 0) prepare(&tc->slot[0]);
     team_bar(team);
-    uint32_t t = tc->next;
-    while (t < g.n_tiles) {
-        team_bar(team);                                               // bar0
-        if (tt == 0) tc->next = atomicAdd(&ws.ctrl->ticket, 1u);
-        const uint32_t e = tab16[t];
-        const uint32_t c = t / g.tiles_per_chunk;
-        const bool first = (t % g.tiles_per_chunk) == 0;
+    uint32_t p = 0;
+    while (true) {
+        const DecSlot sl = tc->slot[p];
+        const uint32_t t = sl.t;
+        if (t >= g.n_tiles) break;
+        if (tt == 0) prepare(&tc->slot[p ^ 1u]);
+        const uint32_t e = sl.entry;
+        const bool first = sl.first != 0;
         bool have_digest = false;
         if (e != 0) {
-            const unsigned char* src = payload + *reinterpret_cast<const unsigned long long*>(dir + 16ull * c) + ws.rel[t];
+            const unsigned char* src = payload + sl.src;
             unsigned char* o = dst + (uint64_t)t * kTile;
             uint32_t w[kWordsPerLane];
+            bool fold = first;
+            bool decoded = true;
             if (e == 0xFFFFu) {
                 const uint32_t len = g.tail_len;
                 for (uint32_t i = tt; i < len; i += kTeamThreads) o[i] = src[i];
-                load_tile_words_guarded(src, len, first, -8, warp, lane, w);
-                tile_digest_to_smem(T, w, false, warp, lane, tc);
-                have_digest = true;
+                load_tile_words_guarded(src, len, first, warp, lane, w);
+                fold = false;
             } else if (e == 512u) {
                 load_tile_words(src, warp, lane, w);
-                unsigned char* p = o + warp * 2048u + lane * 4u;
-#pragma unroll
-                for (int i = 0; i < 16; i++) st_stream_u32(p + i * 128, w[i]);
-                tile_digest_to_smem(T, w, first, warp, lane, tc);
-                have_digest = true;
             } else {
-                // PACK tile: validate the 32 descriptors (every warp does, the verdict is uniform)
+                // PACK tile: validate the 32 descriptors (every warp does; the verdict is uniform)
                 const uint32_t desc = reinterpret_cast<const uint16_t*>(src)[lane];
                 const uint32_t base_l = desc & 0xFFu, wv = (desc >> 8) & 15u, chk = desc >> 12;
                 const bool bad = wv > 8u || chk != (((base_l & 15u) ^ (base_l >> 4) ^ wv ^ 5u) & 15u);
@@ -1054,66 +1174,75 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
                 uint32_t incl = wv;
 #pragma unroll
                 for (int d = 1; d < 32; d <<= 1) {
-                    uint32_t o2 = __shfl_up_sync(0xFFFFFFFFu, incl, d);
+                    const uint32_t o2 = __shfl_up_sync(0xFFFFFFFFu, incl, d);
                     if (lane >= (uint32_t)d) incl += o2;
                 }
-                const uint32_t S = __shfl_sync(0xFFFFFFFFu, incl, 31);
-                const int verdict = anybad ? 1 : (258u + S != e ? 2 : 0);
+                const uint32_t Ssum = __shfl_sync(0xFFFFFFFFu, incl, 31);
+                const int verdict = anybad ? 1 : (258u + Ssum != e ? 2 : 0);
                 if (verdict) {
+                    decoded = false;
                     if (tt == 0) {
                         atomicMin(&ws.ctrl->bad4_key, (unsigned long long)t * 2ull + (verdict == 2 ? 1ull : 0ull));
-                        atomicOr(&ws.cflag[c], CF_BAD4);
+                        atomicOr(&ws.cflag[sl.c], CF_BAD4);
                     }
                 } else {
+                    // issue every load of the warp's four groups, then unpack
+                    uint2 sm[4];
+                    uint32_t w0[4], w1[4], w2[4], dgv[4];
 #pragma unroll
                     for (int j = 0; j < 4; j++) {
                         const uint32_t gi = 4 * warp + j;
-                        const uint32_t dg = __shfl_sync(0xFFFFFFFFu, desc, gi);
+                        dgv[j] = __shfl_sync(0xFFFFFFFFu, desc, gi);
                         const uint32_t exg = __shfl_sync(0xFFFFFFFFu, incl - wv, gi);
-                        const uint32_t base = dg & 0xFFu, wd = (dg >> 8) & 15u;
-                        const uint2 sm = *reinterpret_cast<const uint2*>(src + 64 + 256 * gi + 8 * lane);
+                        const uint32_t wd = (dgv[j] >> 8) & 15u;
+                        sm[j] = *reinterpret_cast<const uint2*>(src + 64 + 256 * gi + 8 * lane);
+                        const unsigned char* rec = src + 8256 + 32 * exg;
+                        const uint32_t a = (lane * wd) & ~3u, rl = 32u * wd;
+                        w0[j] = (a < rl) ? ldg_u32(rec + a) : 0u;
+                        w1[j] = (a + 4 < rl) ? ldg_u32(rec + a + 4) : 0u;
+                        w2[j] = (a + 8 < rl) ? ldg_u32(rec + a + 8) : 0u;
+                    }
+#pragma unroll
+                    for (int j = 0; j < 4; j++) {
+                        const uint32_t base = dgv[j] & 0xFFu, wd = (dgv[j] >> 8) & 15u;
+                        const uint32_t sh = ((lane * wd) & 3u) * 8u;
                         uint32_t ea = base * 0x01010101u, eb = ea;
-                        if (wd) {
-                            const unsigned char* rec = src + 8256 + 32 * exg;
-                            const uint32_t bo = lane * wd, a = bo & ~3u, sh = (bo & 3u) * 8u, rl = 32u * wd;
-                            const uint32_t w0 = *reinterpret_cast<const uint32_t*>(rec + a);
-                            const uint32_t w1 = (a + 4 < rl) ? *reinterpret_cast<const uint32_t*>(rec + a + 4) : 0u;
-                            const uint32_t w2 = (a + 8 < rl) ? *reinterpret_cast<const uint32_t*>(rec + a + 8) : 0u;
-                            const uint32_t lo = __funnelshift_r(w0, w1, sh), hi = __funnelshift_r(w1, w2, sh);
-                            const unsigned long long P = (unsigned long long)lo | ((unsigned long long)hi << 32);
-                            const uint32_t m4 = (wd == 8) ? 0xFFFFFFFFu : ((1u << (4 * wd)) - 1u);
-                            const uint32_t za = (uint32_t)P & m4, zb = (uint32_t)(P >> (4 * wd)) & m4;
-                            const uint32_t m2 = (1u << (2 * wd)) - 1u;
-                            const uint32_t ya = (za & m2) | ((za >> (2 * wd)) << 16);
-                            const uint32_t yb = (zb & m2) | ((zb >> (2 * wd)) << 16);
-                            const uint32_t m1 = ((1u << wd) - 1u) * 0x00010001u;
-                            const uint32_t da = (ya & m1) | ((ya & (m1 << wd)) << (8 - wd));
-                            const uint32_t db = (yb & m1) | ((yb & (m1 << wd)) << (8 - wd));
-                            // per-byte (base + d) & 0xFF
-                            const uint32_t b4 = ea;
-                            ea = ((da & 0x7F7F7F7Fu) + (b4 & 0x7F7F7F7Fu)) ^ ((da ^ b4) & 0x80808080u);
-                            eb = ((db & 0x7F7F7F7Fu) + (b4 & 0x7F7F7F7Fu)) ^ ((db ^ b4) & 0x80808080u);
+                        switch (wd) {          // uniform across the warp
+                            case 1: unpack_group<1>(w0[j], w1[j], w2[j], sh, base, ea, eb); break;
+                            case 2: unpack_group<2>(w0[j], w1[j], w2[j], sh, base, ea, eb); break;
+                            case 3: unpack_group<3>(w0[j], w1[j], w2[j], sh, base, ea, eb); break;
+                            case 4: unpack_group<4>(w0[j], w1[j], w2[j], sh, base, ea, eb); break;
+                            case 5: unpack_group<5>(w0[j], w1[j], w2[j], sh, base, ea, eb); break;
+                            case 6: unpack_group<6>(w0[j], w1[j], w2[j], sh, base, ea, eb); break;
+                            case 7: unpack_group<7>(w0[j], w1[j], w2[j], sh, base, ea, eb); break;
+                            case 8: unpack_group<8>(w0[j], w1[j], w2[j], sh, base, ea, eb); break;
+                            default: break;
                         }
                         uint32_t Tr[4];
-                        Tr[0] = __byte_perm(sm.x, ea, 0x5140);
-                        Tr[1] = __byte_perm(sm.x, ea, 0x7362);
-                        Tr[2] = __byte_perm(sm.y, eb, 0x5140);
-                        Tr[3] = __byte_perm(sm.y, eb, 0x7362);
+                        Tr[0] = __byte_perm(sm[j].x, ea, 0x5140);
+                        Tr[1] = __byte_perm(sm[j].x, ea, 0x7362);
+                        Tr[2] = __byte_perm(sm[j].y, eb, 0x5140);
+                        Tr[3] = __byte_perm(sm[j].y, eb, 0x7362);
 #pragma unroll
                         for (int r = 0; r < 4; r++)
                             w[4 * j + r] = ((Tr[r] >> 1) & 0x7FFF7FFFu) | ((Tr[r] << 15) & 0x80008000u);
                     }
-                    unsigned char* p = o + warp * 2048u + lane * 4u;
-#pragma unroll
-                    for (int i = 0; i < 16; i++) st_stream_u32(p + i * 128, w[i]);
-                    tile_digest_to_smem(T, w, first, warp, lane, tc);
-                    have_digest = true;
                 }
             }
+            if (decoded) {
+                if (e != 0xFFFFu) {
+                    unsigned char* q = o + warp * 2048u + lane * 4u;
+#pragma unroll
+                    for (int i = 0; i < 16; i++) st_stream_u32(q + i * 128, w[i]);
+                }
+                const uint32_t v = tile_digest_part(S, w, fold, warp, lane);
+                if (lane == 0) tc->wdig[p][warp] = v;
+                have_digest = true;
+            }
         }
-        team_bar(team);                                               // bar1
-        if (tt == 0 && have_digest) ws.dig[t] = team_digest(tc);
-        t = tc->next;
+        team_bar(team);                                               // slot[p^1] and wdig[p] visible
+        if (tt == 0 && have_digest) ws.dig[t] = xor8(tc->wdig[p]);
+        p ^= 1u;
     }
 }
 
@@ -1188,7 +1317,11 @@ k_decode_finish(const unsigned char* __restrict__ wire, uint64_t wire_len, Geo g
 #ifndef WM_TEAMS
 #define WM_TEAMS 3
 #endif
-constexpr int kTeams = WM_TEAMS;
+constexpr int kTeams = WM_TEAMS;            // encode: teams per block (plus the scanner warp)
+#ifndef WM_TEAMS_PLAIN
+#define WM_TEAMS_PLAIN 4
+#endif
+constexpr int kTeamsPlain = WM_TEAMS_PLAIN;  // checksum / decode: teams per block
 
 struct DeviceState {
     Tables* tables = nullptr;
@@ -1225,10 +1358,10 @@ static const DeviceState* device_state()
     if (cudaMalloc(&s.tables, sizeof(Tables)) != cudaSuccess) return nullptr;
     if (cudaMemcpy(s.tables, &host, sizeof(Tables), cudaMemcpyHostToDevice) != cudaSuccess) return nullptr;
     if (cudaDeviceGetAttribute(&s.sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return nullptr;
-    const int big = kSmemTables + kTeams * kTeamSmemEncode;
+    const int big = kDynSmem;
     if (cudaFuncSetAttribute(k_encode<kTeams>, cudaFuncAttributeMaxDynamicSharedMemorySize, big) != cudaSuccess) return nullptr;
-    if (cudaFuncSetAttribute(k_decode<kTeams>, cudaFuncAttributeMaxDynamicSharedMemorySize, big) != cudaSuccess) return nullptr;
-    if (cudaFuncSetAttribute(k_tile_digests<kTeams>, cudaFuncAttributeMaxDynamicSharedMemorySize, big) != cudaSuccess) return nullptr;
+    if (cudaFuncSetAttribute(k_decode<kTeamsPlain>, cudaFuncAttributeMaxDynamicSharedMemorySize, big) != cudaSuccess) return nullptr;
+    if (cudaFuncSetAttribute(k_tile_digests<kTeamsPlain>, cudaFuncAttributeMaxDynamicSharedMemorySize, big) != cudaSuccess) return nullptr;
     if (cudaFuncSetAttribute(k_meta_crc, cudaFuncAttributeMaxDynamicSharedMemorySize, big) != cudaSuccess) return nullptr;
     for (int k = 0; k < 4; k++)
         for (int j = 0; j < 2; j++)
@@ -1294,11 +1427,11 @@ wm_status wm_checksum(const void* cache, uint64_t nbytes, uint32_t chunk_bytes, 
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     Ws ws = ws_carve(workspace, g);
     const unsigned char* c = static_cast<const unsigned char*>(cache);
-    const uint32_t need = (g.n_tiles + kTeams - 1) / kTeams;
+    const uint32_t need = (g.n_tiles + kTeamsPlain - 1) / kTeamsPlain;
     const uint32_t grid = need < (uint32_t)ds->sm_count ? need : (uint32_t)ds->sm_count;
     {
         MainKernelTimer timer(ds, 0, s);
-        k_tile_digests<kTeams><<<grid, kTeams * 256, kSmemTables + kTeams * kTeamSmemPlain, s>>>(c, g, ws, ds->tables);
+        k_tile_digests<kTeamsPlain><<<grid, kTeamsPlain * 256, kDynSmem, s>>>(c, g, ws, ds->tables);
     }
     k_checksum_finish<<<(g.n_chunks + 255) / 256, 256, 0, s>>>(c, g, ws, ds->tables, crc_out);
     g_launches = 2;
@@ -1349,10 +1482,10 @@ wm_status wm_encode(const void* cache, uint64_t nbytes, uint32_t chunk_bytes, co
     const uint32_t grid = need < (uint32_t)ds->sm_count ? need : (uint32_t)ds->sm_count;
     {
         MainKernelTimer timer(ds, 2, s);
-        k_encode<kTeams><<<grid, kTeams * 256 + 32, kSmemTables + kTeams * kTeamSmemEncode, s>>>(c, g, dirty, w, wire_cap, ws, ds->tables);
+        k_encode<kTeams><<<grid, kTeams * 256 + 32, kDynSmem, s>>>(c, g, dirty, w, wire_cap, ws, ds->tables);
     }
     k_encode_finish<<<(g.n_chunks + 1023) / 1024, 1024, 0, s>>>(c, g, dirty, crc_inout, w, ws, ds->tables);
-    k_meta_crc<<<g.n_meta_slices, 256, kSmemTables + kTeamSmemPlain, s>>>(w, 0, g, ws, ds->tables, result, 0);
+    k_meta_crc<<<g.n_meta_slices, 256, kDynSmem, s>>>(w, 0, g, ws, ds->tables, result, 0);
     g_launches = 4;
     return launch_status();
 }
@@ -1373,14 +1506,14 @@ wm_status wm_decode_verify(const void* wire, uint64_t wire_len, void* dst, uint6
     k_decode_init<<<1, 64, 0, s>>>(ws);
     // a wire shorter than the metadata is rejected by the header check before anything else is read
     const uint32_t slices = wire_len >= g.meta_end ? g.n_meta_slices : 1;
-    k_meta_crc<<<slices, 256, kSmemTables + kTeamSmemPlain, s>>>(const_cast<unsigned char*>(w), wire_len, g, ws, ds->tables, result, 1);
+    k_meta_crc<<<slices, 256, kDynSmem, s>>>(const_cast<unsigned char*>(w), wire_len, g, ws, ds->tables, result, 1);
     k_decode_struct_chunks<<<(g.n_chunks + 7) / 8, 256, 0, s>>>(w, g, ws);
     k_decode_struct_scan<<<1, 1024, 0, s>>>(w, wire_len, g, ws, result);
-    const uint32_t need = (g.n_tiles + kTeams - 1) / kTeams;
+    const uint32_t need = (g.n_tiles + kTeamsPlain - 1) / kTeamsPlain;
     const uint32_t grid = need < (uint32_t)ds->sm_count ? need : (uint32_t)ds->sm_count;
     {
         MainKernelTimer timer(ds, 3, s);
-        k_decode<kTeams><<<grid, kTeams * 256, kSmemTables + kTeams * kTeamSmemPlain, s>>>(w, g, d, ws, ds->tables);
+        k_decode<kTeamsPlain><<<grid, kTeamsPlain * 256, kDynSmem, s>>>(w, g, d, ws, ds->tables);
     }
     k_decode_finish<<<(g.n_chunks + 1023) / 1024, 1024, 0, s>>>(w, wire_len, g, d, dst_crc_inout, ws, ds->tables, result);
     g_launches = 6;

@@ -11,13 +11,21 @@ namespace wm {
 
 constexpr uint32_t kPolyReflected = 0x82F63B78u;
 
+// Byte offsets inside the shared-memory table image.  The image is placed at an address that
+// is a multiple of 64 KiB inside the shared window, so that "table base | value << 8 | lane
+// slot" can be put together with one byte permute.
+//   A01: entry b at b*256: 32 lane copies of G[0][b] (bytes 0..127), then of G[1][b]
+//   A23: the same for G[2], G[3]
+//   NK : four 4 KiB arrays, array j = nibbles 2j and 2j+1 of the lane-finish table:
+//        entry v at v*256: NK[lane][2j][v] for the 32 lanes, then NK[lane][2j+1][v]
+constexpr uint32_t kImgA01 = 0x00000, kImgA23 = 0x10000, kImgNK = 0x20000, kImgBytes = 0x24000;
+
 // Tables shared by all kernels; one copy lives in device memory per device.
 struct Tables {
-    uint32_t G[4][256];       // G[k][b]  = (b << 8k) advanced over 128 bytes (one row stride)
-    uint32_t NK[32][8][16];   // NK[l][n][v] = (v << 4n) advanced over 128 - 4l bytes (lane finish)
-    uint32_t NW[8][8][16];    // NW[w][n][v] = (v << 4n) advanced over 2048 (7 - w) bytes (warp position)
-    uint32_t HT[4][256];      // HT[k][b] = (b << 8k) advanced over 16384 bytes (one tile)
-    uint32_t T0[256];         // T0[b]    = b advanced over one byte (the classic table)
+    uint32_t image[kImgBytes / 4];   // the shared-memory image described above
+    uint32_t NW[8][8][16];           // NW[w][n][v] = (v << 4n) advanced over 2048 (7 - w) bytes
+    uint32_t HT[4][256];             // HT[k][b] = (b << 8k) advanced over 16384 bytes (one tile)
+    uint32_t T0[256];                // T0[b]    = b advanced over one byte (the classic table)
 };
 
 inline uint32_t times_x(uint32_t v) { return (v >> 1) ^ ((v & 1u) ? kPolyReflected : 0u); }
@@ -48,16 +56,21 @@ inline uint32_t x_pow_bytes(uint64_t n)
 inline void build_tables(Tables& t)
 {
     const uint32_t k128 = x_pow_bytes(128), kTile = x_pow_bytes(16384), k1 = x_pow_bytes(1);
+    // G[k][b] = (b << 8k) advanced over 128 bytes (one row stride of the word-strided chain)
     for (uint32_t k = 0; k < 4; k++)
         for (uint32_t b = 0; b < 256; b++) {
-            t.G[k][b] = mulmod(b << (8 * k), k128);
+            const uint32_t g = mulmod(b << (8 * k), k128);
+            uint32_t* dst = t.image + ((k < 2 ? kImgA01 : kImgA23) + b * 256 + (k & 1) * 128) / 4;
+            for (uint32_t l = 0; l < 32; l++) dst[l] = g;
             t.HT[k][b] = mulmod(b << (8 * k), kTile);
         }
     for (uint32_t b = 0; b < 256; b++) t.T0[b] = mulmod(b, k1);
+    // NK[l][n][v] = (v << 4n) advanced over 128 - 4l bytes (a lane's place inside its row)
     for (uint32_t l = 0; l < 32; l++) {
         const uint32_t kl = x_pow_bytes(128 - 4 * l);
         for (uint32_t n = 0; n < 8; n++)
-            for (uint32_t v = 0; v < 16; v++) t.NK[l][n][v] = mulmod(v << (4 * n), kl);
+            for (uint32_t v = 0; v < 16; v++)
+                t.image[(kImgNK + (n / 2) * 0x1000 + v * 256 + (n & 1) * 128) / 4 + l] = mulmod(v << (4 * n), kl);
     }
     for (uint32_t w = 0; w < 8; w++) {
         const uint32_t kw = x_pow_bytes(2048u * (7 - w));
