@@ -61,7 +61,7 @@ static_assert(sizeof(Ctrl) == 256, "control block is 256 bytes");
 
 struct Ws {
     Ctrl* ctrl;
-    unsigned long long* state;   // [n_tiles] look-back words
+    uint32_t* lbk;               // [n_tiles] placement look-back words
     uint32_t* dig;               // [n_tiles] tile digests
     uint32_t* rel;               // [n_tiles] decode: tile offset inside its chunk's payload
     uint32_t* cflag;             // [n_chunks] bit0 present, bit1..: failed step 3/4/5/6
@@ -97,7 +97,7 @@ static Ws ws_carve(void* base, const Geo& g)
     unsigned char* b = static_cast<unsigned char*>(base);
     Ws w;
     w.ctrl = reinterpret_cast<Ctrl*>(b);
-    w.state = reinterpret_cast<unsigned long long*>(b + L.state);
+    w.lbk = reinterpret_cast<uint32_t*>(b + L.state);
     w.dig = reinterpret_cast<uint32_t*>(b + L.dig);
     w.rel = reinterpret_cast<uint32_t*>(b + L.rel);
     w.cflag = reinterpret_cast<uint32_t*>(b + L.cflag);
@@ -382,38 +382,51 @@ __global__ void k_encode_init(Geo g, Ws ws, unsigned char* wire)
 {
     const uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
     const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
-    for (uint64_t t = i; t < g.n_tiles; t += stride) ws.state[t] = 0ull;
+    for (uint64_t t = i; t < g.n_tiles; t += stride) ws.lbk[t] = 0u;
     if (i < sizeof(Ctrl) / 4) reinterpret_cast<uint32_t*>(ws.ctrl)[i] = 0u;
     // zero padding between the tile table and the payload
     const uint64_t tab_end = 64ull + 16ull * g.n_chunks + 2ull * g.n_tiles;
     if (i < g.meta_end - tab_end) wire[tab_end + i] = 0;
 }
 
-constexpr unsigned long long kFlagA = 1ull << 62, kFlagP = 2ull << 62, kValMask = (1ull << 62) - 1;
+constexpr uint32_t kFlagA = 1u << 30, kFlagP = 2u << 30, kValMask = (1u << 30) - 1u;
 constexpr uint32_t kSpinLimit = 1u << 20;
+constexpr uint32_t kUnit = 32;              // placement words count in units of 32 bytes
 
 // Placement of the encoded tiles: a chained scan with one dedicated scanner warp.
 //
-// state[t] starts at 0.  The team that encodes tile t publishes kFlagA | len(t) as soon as the
-// length is known.  One scanner warp (the winner of a lock among the extra warps every block
-// carries) walks the array in order, 256 entries per poll, turns every leading run of
-// published lengths into kFlagP | exclusive prefix, and moves on.  The owner of tile t then
-// reads its offset back from state[t].  Several hundred tiles are in flight at any time and
-// publish at about the same moment; letting each of them walk back to the nearest finished
-// prefix made the walk, not the data, the bottleneck.  The scanner is a warp that is running
-// by construction (it won the lock), so the owners' waits depend only on running code; all
-// waits are bounded all the same and end in WM_ERR_TIMEOUT.
-__device__ __forceinline__ void publish_len(unsigned long long* state, uint32_t t, uint32_t len)
+// lbk[t] starts at 0.  The team that encodes tile t publishes kFlagA | len(t)/32 as soon as the
+// length is known.  One scanner warp (alone in the block that wins a lock at kernel start, so
+// that it has an SM's issue slots to itself) walks the array in order, 512 entries per poll,
+// turns every leading run of published lengths into kFlagP | (exclusive prefix)/32, and moves
+// on.  The owner of tile t then reads its offset back from lbk[t].  Every encoded length that
+// another tile has to add is a multiple of 32 (only the cache's last tile can be ragged, and
+// nothing follows it); 30 bits of 32-byte units cover 32 GiB of payload.
+//
+// Several hundred tiles are in flight at any time and publish at about the same moment;
+// letting each of them walk back to the nearest finished prefix made the walk, not the data,
+// the bottleneck, and assigning tiles statically made every round wait for its slowest team.
+// The scanner is running by construction (it won the lock), tiles are claimed in ticket
+// order, and a team publishes the length of a claimed tile without waiting for anyone, so the
+// owners' waits depend only on running code; they are bounded all the same and end in
+// WM_ERR_TIMEOUT.
+__device__ __forceinline__ void st_relaxed_u32(uint32_t* p, uint32_t v)
 {
-    st_volatile_u64(reinterpret_cast<uint64_t*>(&state[t]), kFlagA | len);
+    asm volatile("st.relaxed.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+__device__ __forceinline__ uint32_t ld_relaxed_u32(const uint32_t* p)
+{
+    uint32_t v;
+    asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
 }
 
-// Owner side: exclusive prefix of tile t (one lane spins; bounded).
-__device__ __forceinline__ unsigned long long wait_prefix(unsigned long long* state, uint32_t t, Ctrl* ctrl)
+// Owner side: exclusive prefix (bytes) of tile t (one lane spins; bounded).
+__device__ __forceinline__ unsigned long long wait_prefix(const uint32_t* lbk, uint32_t t, Ctrl* ctrl)
 {
     for (uint32_t polls = 0; polls < kSpinLimit; polls++) {
-        const unsigned long long v = ld_volatile_u64(reinterpret_cast<const uint64_t*>(&state[t]));
-        if ((v >> 62) == 2) return v & kValMask;
+        const uint32_t v = ld_relaxed_u32(lbk + t);
+        if ((v >> 30) == 2u) return (unsigned long long)(v & kValMask) * kUnit;
         if ((polls & 1023u) == 1023u && ld_volatile_u32(&ctrl->poison)) break;
     }
     atomicOr(&ctrl->err, 2u);
@@ -421,23 +434,54 @@ __device__ __forceinline__ unsigned long long wait_prefix(unsigned long long* st
     return 0;
 }
 
-// Scanner side (one full warp).
-__device__ void scan_tile_lengths(unsigned long long* state, uint32_t n_tiles, uint32_t lane, Ctrl* ctrl)
+// Scanner side (one full warp).  A poll copies 512 consecutive entries into shared memory with
+// coalesced asynchronous 16-byte copies (one round trip to L2, no registers held meanwhile);
+// lane l then owns entries 16 l .. 16 l + 15 of the window.
+constexpr int kScanPerLane = 16;
+__device__ void scan_tile_lengths(uint32_t* lbk, uint32_t n_tiles, uint32_t lane, Ctrl* ctrl, uint32_t* win)
 {
-    uint32_t f = 0, spins = 0;
-    unsigned long long base = 0;
+    uint64_t f = 0;                 // first unresolved entry
+    uint64_t base = 0;              // units before f
+    uint32_t spins = 0;
+#ifdef WM_DEBUG_COUNTERS
+    uint32_t dbg_iters = 0, dbg_empty = 0;
+#endif
     while (f < n_tiles) {
-        unsigned long long v[8];
+#ifdef WM_DEBUG_COUNTERS
+        dbg_iters++;
+#endif
+        const uint64_t w0 = f & ~3ull;                    // 16-byte aligned window start
+        const uint32_t skip = (uint32_t)(f - w0);         // entries before f (already resolved)
 #pragma unroll
-        for (int j = 0; j < 8; j++) {
-            const uint64_t idx = (uint64_t)f + 8u * lane + j;
-            v[j] = idx < n_tiles ? ld_volatile_u64(reinterpret_cast<const uint64_t*>(&state[idx])) : 0ull;
+        for (int q = 0; q < 4; q++) {
+            const uint32_t slot = 4u * (lane + 32u * q);
+            if (w0 + slot < n_tiles) {                    // n_tiles entries are padded to a multiple of 4
+                const uint32_t dst = (uint32_t)__cvta_generic_to_shared(win + slot);
+                asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(lbk + w0 + slot) : "memory");
+            } else {
+                *reinterpret_cast<uint4*>(win + slot) = make_uint4(0, 0, 0, 0);
+            }
         }
-        uint32_t r = 0, sum = 0;            // leading published entries of this lane and their sum
+        asm volatile("cp.async.commit_group;" ::: "memory");
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
+        __syncwarp();
+        uint32_t v[kScanPerLane];
 #pragma unroll
-        for (int j = 0; j < 8; j++)
-            if (r == (uint32_t)j && (v[j] >> 62) == 1) { r++; sum += (uint32_t)(v[j] & kValMask); }
-        const uint32_t fm = __ballot_sync(0xFFFFFFFFu, r == 8);
+        for (int q = 0; q < 4; q++) {
+            const uint4 x = *reinterpret_cast<const uint4*>(win + kScanPerLane * lane + 4 * q);
+            v[4 * q] = x.x; v[4 * q + 1] = x.y; v[4 * q + 2] = x.z; v[4 * q + 3] = x.w;
+        }
+        __syncwarp();
+        // leading published entries of this lane (entries before f count as published, value 0)
+        uint32_t r = 0, sum = 0;
+#pragma unroll
+        for (int j = 0; j < kScanPerLane; j++) {
+            const uint32_t rel = kScanPerLane * lane + j;
+            const bool old = rel < skip;
+            const bool in = w0 + rel < n_tiles;
+            if (r == (uint32_t)j && in && (old || (v[j] >> 30) == 1u)) { r++; if (!old) sum += v[j] & kValMask; }
+        }
+        const uint32_t fm = __ballot_sync(0xFFFFFFFFu, r == (uint32_t)kScanPerLane);
         const uint32_t lead = (fm == 0xFFFFFFFFu) ? 32u : (uint32_t)(__ffs(~fm) - 1);   // leading full lanes
         const uint32_t contrib = lane <= lead ? sum : 0u;
         uint32_t incl = contrib;
@@ -446,19 +490,24 @@ __device__ void scan_tile_lengths(unsigned long long* state, uint32_t n_tiles, u
             uint32_t o = __shfl_up_sync(0xFFFFFFFFu, incl, d);
             if (lane >= (uint32_t)d) incl += o;
         }
-        const uint32_t cnt = lane < lead ? 8u : (lane == lead ? r : 0u);
-        unsigned long long run = base + (incl - contrib);
+        const uint32_t cnt = lane < lead ? (uint32_t)kScanPerLane : (lane == lead ? r : 0u);
+        uint64_t run = base + (incl - contrib);
 #pragma unroll
-        for (int j = 0; j < 8; j++) {
-            if ((uint32_t)j < cnt) {
-                st_volatile_u64(reinterpret_cast<uint64_t*>(&state[(uint64_t)f + 8u * lane + j]), kFlagP | run);
+        for (int j = 0; j < kScanPerLane; j++) {
+            const uint32_t rel = kScanPerLane * lane + j;
+            if ((uint32_t)j < cnt && rel >= skip) {
+                st_relaxed_u32(lbk + w0 + rel, kFlagP | (uint32_t)run);
                 run += v[j] & kValMask;
             }
         }
         const uint32_t r_lead = __shfl_sync(0xFFFFFFFFu, r, lead & 31u);
-        const uint32_t k = 8u * lead + (lead < 32u ? r_lead : 0u);
+        const uint32_t k_all = (uint32_t)kScanPerLane * lead + (lead < 32u ? r_lead : 0u);   // includes `skip`
+        const uint32_t k = k_all > skip ? k_all - skip : 0u;
         base += __shfl_sync(0xFFFFFFFFu, incl, 31);
         f += k;
+#ifdef WM_DEBUG_COUNTERS
+        if (k == 0) dbg_empty++;
+#endif
         if (k == 0) {
             if (++spins > kSpinLimit || ((spins & 1023u) == 1023u && ld_volatile_u32(&ctrl->poison))) {
                 if (lane == 0) { atomicOr(&ctrl->err, 2u); atomicExch(&ctrl->poison, 1u); }
@@ -468,7 +517,9 @@ __device__ void scan_tile_lengths(unsigned long long* state, uint32_t n_tiles, u
             spins = 0;
         }
     }
-    if (lane == 0) ctrl->payload_total = base;
+#ifdef WM_DEBUG_COUNTERS
+    if (lane == 0) { ctrl->pad[0] = dbg_iters; ctrl->pad[1] = dbg_empty; }
+#endif
 }
 
 __device__ __forceinline__ uint32_t next_ticket(Ctrl* ctrl)
@@ -483,11 +534,12 @@ __device__ __forceinline__ uint32_t desc_of(uint32_t base, uint32_t w)
 }
 
 struct EncTeamCtl {
-    uint32_t wtab[2][32];   // per group: base | w << 8 (double buffered by tile parity)
-    uint32_t wdig[2][8];    // per warp: its contribution to the tile digest
+    uint32_t wtab[3][32];   // per group: base | w << 8 (one slot per tile in flight)
+    uint32_t wdig[3][8];    // per warp: its contribution to the tile digest
+    uint32_t wsum[3];       // sum of widths so far | warps arrived << 16 (the last warp publishes)
     uint32_t next;          // ticket just claimed (>= n_tiles: none left)
-    uint32_t pad;
     unsigned long long excl;
+    unsigned long long pad2;
 };
 static_assert(sizeof(EncTeamCtl) % 16 == 0, "team control block keeps 16-byte alignment");
 constexpr uint32_t kTeamSmemEncode = kTile + sizeof(EncTeamCtl);
@@ -559,18 +611,37 @@ __device__ __forceinline__ void pack_group(uint32_t e4a, uint32_t e4b, uint32_t 
     }
 }
 
-// Single-pass fused checksum + encode.  Per team, software pipelined over tiles X (being
-// packed and written out) and Y (being checksummed and measured):
-//     pack X into shared memory | digest + exponent ranges of Y | publish len(Y) |
-//     wait for X's offset | claim Z and start its loads | copy X out
-// A team never waits while it holds a claimed tile whose length is not yet published: len(Y)
-// goes out before the wait for X starts, and Z is claimed only after that wait has returned.
+// Single-pass fused checksum + encode.  Each team keeps three tiles in flight:
+//     A  measured two steps ago, packed and written out in this step
+//     B  measured one step ago, waiting for its offset
+//     C  checksummed and measured in this step (its length is published at once)
+// and per step does
+//     probe A's offset | pack A into shared memory | re-request B's words | digest + exponent
+//     ranges of C, publish len(C) | take A's offset (wait if the scanner is not there yet) |
+//     claim D, start its loads | copy A out.
+// The two steps between measuring a tile and needing its offset cover the time the scanner
+// needs (its poll plus the owner's read are two round trips to L2 under full load).  A tile's
+// words are not kept in registers over those two steps: they are read again for packing, one
+// step ahead, and come from L2 (a few hundred tiles, some tens of MB, were read in between).
+// A team never waits while it holds a claimed tile whose length is not on its way out: len(C)
+// is published by the team's own warps without waiting for anyone, and D is claimed only
+// after A's offset has arrived.
 template <int TEAMS>
-__global__ void __launch_bounds__(TEAMS * 256 + 32, 1)
+__global__ void __launch_bounds__(TEAMS * 256, 1)
 k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restrict__ dirty,
          unsigned char* __restrict__ wire, uint64_t wire_cap, Ws ws, const Tables* __restrict__ tab)
 {
     extern __shared__ __align__(16) unsigned char smem[];
+    // The first block to get here becomes the scanner: one warp of it, alone on its SM (a warp
+    // that shares its scheduler with six busy ones gets too few issue slots to keep up).
+    __shared__ uint32_t s_scanner;
+    if (threadIdx.x == 0) s_scanner = atomicCAS(&ws.ctrl->scan_lock, 0u, 1u) == 0u;
+    __syncthreads();
+    if (s_scanner) {
+        if (threadIdx.x < 32)
+            scan_tile_lengths(ws.lbk, g.n_tiles, threadIdx.x, ws.ctrl, reinterpret_cast<uint32_t*>(smem));
+        return;
+    }
     Smem S = setup_smem(smem, tab);
     const uint32_t team = threadIdx.x / kTeamThreads, tt = threadIdx.x % kTeamThreads;
     const uint32_t warp = tt / 32, lane = tt % 32;
@@ -580,25 +651,25 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
         if ((uint32_t)i == team) out = p;
     }
     if (!S.ok) { if (threadIdx.x == 0) atomicOr(&ws.ctrl->err, 4u); return; }
-    if (team == TEAMS) {
-        // the extra warp: one of them, grid-wide, becomes the scanner; the others leave
-        uint32_t won = 0;
-        if (lane == 0) won = atomicCAS(&ws.ctrl->scan_lock, 0u, 1u) == 0u;
-        won = __shfl_sync(0xFFFFFFFFu, won, 0);
-        if (won) scan_tile_lengths(ws.state, g.n_tiles, lane, ws.ctrl);
-        return;
-    }
     EncTeamCtl* tc = reinterpret_cast<EncTeamCtl*>(out + kTile);
     unsigned char* dir = wire + 64;
     uint16_t* tile_tab = reinterpret_cast<uint16_t*>(wire + 64 + 16ull * g.n_chunks);
+    auto info = [&](uint32_t t) { return tile_info(g, dirty, t); };
+    auto publish_len = [&](uint32_t t, uint32_t len) { st_relaxed_u32(ws.lbk + t, kFlagA | (len / kUnit)); };
 
-    // digest and per-group exponent range of one tile; results go to wdig[par], wtab[par]
+    // Digest and per-group exponent range of one tile; results go to wdig[par], wtab[par].  The
+    // tile's encoded length is published by whichever warp finishes last (no team barrier).
     auto measure = [&](const TileInfo& ti, uint32_t (&d)[kWordsPerLane], uint32_t par) {
-        if (!ti.present) return;
-        if (!ti.full) load_tile_words_guarded(cache + (uint64_t)ti.t * kTile, ti.left, ti.first, warp, lane, d);
+        if (!ti.valid) return;
+        if (!ti.present || !ti.full) {
+            if (warp == 0 && lane == 0) publish_len(ti.t, encoded_len(ti, 0));
+            if (!ti.present) return;
+            load_tile_words_guarded(cache + (uint64_t)ti.t * kTile, ti.left, ti.first, warp, lane, d);
+        }
         const uint32_t v = tile_digest_part(S, d, ti.first && ti.full, warp, lane);
         if (lane == 0) tc->wdig[par][warp] = v;
         if (ti.full) {
+            uint32_t mysum = 0;
 #pragma unroll
             for (int j = 0; j < 4; j++) {
                 const uint32_t a0 = d[4 * j] & 0x7FFF7FFFu, a1 = d[4 * j + 1] & 0x7FFF7FFFu;
@@ -610,23 +681,34 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
                 const uint32_t emin = __reduce_min_sync(0xFFFFFFFFu, mn) >> 7;
                 const uint32_t emax = __reduce_max_sync(0xFFFFFFFFu, mx) >> 7;
                 const uint32_t wd = 32u - __clz(emax - emin);
+                mysum += wd;
                 if (lane == 0) tc->wtab[par][4 * warp + j] = emin | (wd << 8);
             }
+            if (lane == 0) {
+                const uint32_t old = atomicAdd(&tc->wsum[par], mysum + (1u << 16));
+                if ((old >> 16) == 7u) {
+                    tc->wsum[par] = 0;
+                    publish_len(ti.t, encoded_len(ti, (old & 0xFFFFu) + mysum));
+                }
+            }
         }
-    };
-    auto sum_widths = [&](uint32_t par) {
-        return __reduce_add_sync(0xFFFFFFFFu, (tc->wtab[par][lane] >> 8) & 15u);
     };
     auto fetch = [&](const TileInfo& ti, uint32_t (&d)[kWordsPerLane]) {
         if (ti.present && ti.full) load_tile_words(cache + (uint64_t)ti.t * kTile, warp, lane, d);
     };
 
-    // One pipeline step: pack X (words in dP), measure Y (words in dM), place X, claim Z and
-    // start loading it into dP.  Returns with X <- Y, Y <- Z and the roles of dP / dM swapped.
-    TileInfo iX = tile_info(g, dirty, 0xFFFFFFFFu), iY = iX;
-    uint32_t par = 0;
+    // One pipeline step (X = A, W = B, Y = C above): pack X (words in dP), re-request W into dP,
+    // measure Y (words in dM), place X, claim Z and start loading it into dM.
+    TileInfo iX = info(0xFFFFFFFFu), iW = iX, iY = iX;
+    uint32_t par = 0;                  // slot of X; W has slot par+1, Y slot par+2 (mod 3)
+    auto nxt = [](uint32_t p) { return p == 2u ? 0u : p + 1u; };
     auto step = [&](uint32_t (&dP)[kWordsPerLane], uint32_t (&dM)[kWordsPerLane]) {
+        const uint32_t parW = nxt(par), parY = nxt(parW);
         team_bar(team);                                               // bar0: out buffer free
+        // X's length went out one step ago; ask for its offset now, use the answer later
+        const bool leader = (warp == 0 && lane == 0);
+        uint32_t pv = 0;
+        if (leader) pv = ld_relaxed_u32(ws.lbk + iX.t);
         uint32_t enc_len = 0, entry = 0;
         bool staged = false;                                          // encoded tile sits in `out`
         if (iX.present && iX.full) {
@@ -684,23 +766,42 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
             entry = 0xFFFFu;
         }
 
-        measure(iY, dM, par ^ 1u);
-        team_bar(team);                                               // bar1: wtab[par^1] complete
+        fetch(iW, dP);                      // W's words again, for the next step's pack
 
-        if (warp == 0) {
-            if (iY.valid) {
-                const uint32_t Sy = (iY.present && iY.full) ? sum_widths(par ^ 1u) : 0u;
-                if (lane == 0) publish_len(ws.state, iY.t, encoded_len(iY, Sy));
+        // fast path: the offset is already there, so this step will not wait and may claim Z now
+        uint32_t tk = 0xFFFFFFFFu;
+        bool claimed = false;
+        if (leader && (pv >> 30) == 2u) {
+            if (iY.valid) tk = next_ticket(ws.ctrl);
+            claimed = true;
+        }
+
+        // second chance: ask again before the checksum work, look at the answer after it
+        uint32_t pv1 = 0;
+        if (leader && !claimed) pv1 = ld_relaxed_u32(ws.lbk + iX.t);
+
+        measure(iY, dM, parY);
+
+        if (leader) {
+#ifdef WM_DEBUG_COUNTERS
+            atomicAdd(&ws.ctrl->pad[claimed ? 3 : ((pv1 >> 30) == 2u ? 4 : 2)], 1u);
+#endif
+            unsigned long long e;
+            if (claimed) {
+                e = (unsigned long long)(pv & kValMask) * kUnit;
+            } else {                        // len(Y) is on its way out; now it is safe to wait
+                e = (pv1 >> 30) == 2u ? (unsigned long long)(pv1 & kValMask) * kUnit
+                                      : wait_prefix(ws.lbk, iX.t, ws.ctrl);
+                if (iY.valid) tk = next_ticket(ws.ctrl);
             }
-            if (lane == 0) {
-                tc->excl = wait_prefix(ws.state, iX.t, ws.ctrl);
-                tc->next = iY.valid ? next_ticket(ws.ctrl) : 0xFFFFFFFFu;
-            }
+            tc->excl = e;
+            tc->next = tk;
+            if (iX.t + 1 == g.n_tiles) ws.ctrl->payload_total = e + enc_len;
         }
         team_bar(team);                                               // bar2: offset known, out complete
 
-        const TileInfo iZ = tile_info(g, dirty, tc->next);
-        fetch(iZ, dP);                                                // dP is free: X sits in `out`
+        const TileInfo iZ = info(tc->next);
+        fetch(iZ, dM);                                                // dM is free: Y has been measured
 
         const unsigned long long excl = tc->excl;
         if (iX.present) {
@@ -720,32 +821,34 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
             if (iX.present) ws.dig[iX.t] = xor8(tc->wdig[par]);
             if (iX.first) *reinterpret_cast<unsigned long long*>(dir + 16ull * iX.c) = excl;
         }
-        iX = iY;
+        iX = iW;
+        iW = iY;
         iY = iZ;
-        par ^= 1u;
+        par = parW;
     };
 
-    // ---- prologue: X claimed, loaded, measured and published; Y claimed and loading
-    uint32_t dA[kWordsPerLane], dB[kWordsPerLane];
-    if (tt == 0) tc->next = next_ticket(ws.ctrl);
+    // ---- prologue: X and W claimed, measured and published; Y claimed and loading; X's words
+    // requested again for the first pack
+    uint32_t dP[kWordsPerLane], dM[kWordsPerLane];
+    if (tt == 0) { tc->wsum[0] = 0; tc->wsum[1] = 0; tc->wsum[2] = 0; tc->next = next_ticket(ws.ctrl); }
     team_bar(team);
-    iX = tile_info(g, dirty, tc->next);
-    fetch(iX, dA);
-    measure(iX, dA, par);
+    iX = info(tc->next);
+    fetch(iX, dM);
+    measure(iX, dM, 0);
     team_bar(team);
-    if (warp == 0 && iX.valid) {
-        const uint32_t Sx = (iX.present && iX.full) ? sum_widths(par) : 0u;
-        if (lane == 0) { publish_len(ws.state, iX.t, encoded_len(iX, Sx)); tc->next = next_ticket(ws.ctrl); }
-    }
+    if (tt == 0) tc->next = iX.valid ? next_ticket(ws.ctrl) : 0xFFFFFFFFu;
     team_bar(team);
-    iY = tile_info(g, dirty, iX.valid ? tc->next : 0xFFFFFFFFu);
-    fetch(iY, dB);
+    iW = info(tc->next);
+    fetch(iW, dM);
+    measure(iW, dM, 1);
+    team_bar(team);
+    if (tt == 0) tc->next = iW.valid ? next_ticket(ws.ctrl) : 0xFFFFFFFFu;
+    team_bar(team);
+    iY = info(tc->next);
+    fetch(iY, dM);
+    fetch(iX, dP);
 
-    while (iX.valid) {
-        step(dA, dB);
-        if (!iX.valid) break;
-        step(dB, dA);
-    }
+    while (iX.valid) step(dP, dM);
 }
 
 // Directory (enc_len, crc), chunk CRCs, present count; the last block to finish combines the
@@ -1478,11 +1581,12 @@ wm_status wm_encode(const void* cache, uint64_t nbytes, uint32_t chunk_bytes, co
     unsigned char* w = static_cast<unsigned char*>(wire);
     const uint32_t init_blocks = (g.n_tiles + 1023) / 1024 < 1024 ? (g.n_tiles + 1023) / 1024 : 1024;
     k_encode_init<<<init_blocks ? init_blocks : 1, 1024, 0, s>>>(g, ws, w);
-    const uint32_t need = (g.n_tiles + kTeams - 1) / kTeams;
+    // one block per SM: one of them scans, the others encode
+    const uint32_t need = (g.n_tiles + kTeams - 1) / kTeams + 1;
     const uint32_t grid = need < (uint32_t)ds->sm_count ? need : (uint32_t)ds->sm_count;
     {
         MainKernelTimer timer(ds, 2, s);
-        k_encode<kTeams><<<grid, kTeams * 256 + 32, kDynSmem, s>>>(c, g, dirty, w, wire_cap, ws, ds->tables);
+        k_encode<kTeams><<<grid, kTeams * 256, kDynSmem, s>>>(c, g, dirty, w, wire_cap, ws, ds->tables);
     }
     k_encode_finish<<<(g.n_chunks + 1023) / 1024, 1024, 0, s>>>(c, g, dirty, crc_inout, w, ws, ds->tables);
     k_meta_crc<<<g.n_meta_slices, 256, kDynSmem, s>>>(w, 0, g, ws, ds->tables, result, 0);
