@@ -232,10 +232,26 @@ static uint32_t desc_check(uint32_t base, uint32_t w)
  *   S <= 253: PACK tile of 8256 + 32 S bytes (< 16384):
  *       desc[32]  u16 each: base | w << 8 | chk << 12
  *       SM[8192]  byte 256 g + k = SM of the element with coded position k in group g
- *       Epack_g   32 w_g bytes: d = E - base as an LSB-first bit string, the element
- *                 with coded position k in bits [k w, (k+1) w)
+ *       Epack_g   32 w_g bytes holding d = E - base, split into bit planes.  w = 8: one
+ *                 plane of 8 bits per element.  Otherwise the planes present are, in this
+ *                 order, a 4-bit plane (128 bytes) if w & 4, a 2-bit plane (64 bytes) if
+ *                 w & 2, a 1-bit plane (32 bytes) if w & 1; they take consecutive bits of d
+ *                 starting at bit 0 (w = 7: bits 0-3, 4-5, 6; w = 5: bits 0-3, 4).  Inside a
+ *                 p-bit plane, viewed as an LSB-first bit string, the element with coded
+ *                 position k occupies bits [k p, (k+1) p).
  *   else: RAW tile, the 16384 bytes verbatim.
  */
+
+/* Bit planes of a group of width w, in stored order: plane sizes in bits per element. */
+static int plane_widths(uint32_t w, uint32_t p[3])
+{
+    int n = 0;
+    if (w == 8u) { p[n++] = 8u; return n; }
+    if (w & 4u) p[n++] = 4u;
+    if (w & 2u) p[n++] = 2u;
+    if (w & 1u) p[n++] = 1u;
+    return n;
+}
 static uint32_t encode_full_tile(const uint8_t* src, uint8_t* out, uint32_t* entry)
 {
     uint32_t base[WMO_GROUPS_PER_TILE], w[WMO_GROUPS_PER_TILE], S = 0;
@@ -269,9 +285,16 @@ static uint32_t encode_full_tile(const uint8_t* src, uint8_t* out, uint32_t* ent
             uint32_t k = coded_pos(e);
             sm[256u * g + k] = (uint8_t)SM;
             uint32_t d = E - base[g];
-            for (uint32_t j = 0; j < w[g]; j++) {
-                uint32_t bit = k * w[g] + j;
-                if ((d >> j) & 1u) ep[bit / 8u] |= (uint8_t)(1u << (bit % 8u));
+            uint32_t pw[3], lo = 0;                  /* lo: first bit of d the plane takes */
+            int np = plane_widths(w[g], pw);
+            uint8_t* plane = ep;
+            for (int q = 0; q < np; q++) {
+                for (uint32_t j = 0; j < pw[q]; j++) {
+                    uint32_t bit = k * pw[q] + j;
+                    if ((d >> (lo + j)) & 1u) plane[bit / 8u] |= (uint8_t)(1u << (bit % 8u));
+                }
+                lo += pw[q];
+                plane += 32u * pw[q];
             }
         }
         ep += 32u * w[g];
@@ -388,9 +411,16 @@ static void decode_pack_tile(const uint8_t* in, uint8_t* dst)
         uint32_t base = desc & 0xFFu, w = (desc >> 8) & 0xFu;
         for (uint32_t e = 0; e < WMO_GROUP_ELEMS; e++) {
             uint32_t k = coded_pos(e), d = 0;
-            for (uint32_t j = 0; j < w; j++) {
-                uint32_t bit = k * w + j;
-                d |= (uint32_t)((ep[bit / 8u] >> (bit % 8u)) & 1u) << j;
+            uint32_t pw[3], lo = 0;
+            int np = plane_widths(w, pw);
+            const uint8_t* plane = ep;
+            for (int q = 0; q < np; q++) {
+                for (uint32_t j = 0; j < pw[q]; j++) {
+                    uint32_t bit = k * pw[q] + j;
+                    d |= (uint32_t)((plane[bit / 8u] >> (bit % 8u)) & 1u) << (lo + j);
+                }
+                lo += pw[q];
+                plane += 32u * pw[q];
             }
             uint32_t E = (base + d) & 0xFFu;
             uint32_t SM = sm[256u * g + k];

@@ -185,6 +185,29 @@ __device__ __forceinline__ uint32_t max_u16x2(uint32_t a, uint32_t b)
     return d;
 }
 
+// L2 residency hint: data that is read again soon is loaded with evict-last priority (the
+// plain streaming load marks its lines evict-first, and a line so marked is gone from L2 a few
+// microseconds later).
+__device__ __forceinline__ uint64_t l2_policy_evict_last()
+{
+    uint64_t pol;
+    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
+}
+__device__ __forceinline__ uint32_t ld_keep_u32(const void* p, uint64_t pol)
+{
+    uint32_t v;
+    asm volatile("ld.global.L1::no_allocate.L2::cache_hint.u32 %0, [%1], %2;" : "=r"(v) : "l"(p), "l"(pol));
+    return v;
+}
+__device__ __forceinline__ void load_tile_words_keep(const unsigned char* tile, uint32_t warp, uint32_t lane,
+                                                     uint32_t (&w)[16], uint64_t pol)
+{
+    const unsigned char* p = tile + warp * 2048u + lane * 4u;
+#pragma unroll
+    for (int i = 0; i < 16; i++) w[i] = ld_keep_u32(p + i * 128, pol);
+}
+
 // Full tile, fast path: lane's word of row 16*warp + i.
 __device__ __forceinline__ void load_tile_words(const unsigned char* tile, uint32_t warp, uint32_t lane,
                                                 uint32_t (&w)[kWordsPerLane])

@@ -534,15 +534,16 @@ __device__ __forceinline__ uint32_t desc_of(uint32_t base, uint32_t w)
 }
 
 struct EncTeamCtl {
-    uint32_t wtab[3][32];   // per group: base | w << 8 (one slot per tile in flight)
-    uint32_t wdig[3][8];    // per warp: its contribution to the tile digest
-    uint32_t wsum[3];       // sum of widths so far | warps arrived << 16 (the last warp publishes)
-    uint32_t next;          // ticket just claimed (>= n_tiles: none left)
-    unsigned long long excl;
-    unsigned long long pad2;
+    uint32_t wtab[8][32];   // per group: base | w << 8 (a ring of slots: one per tile in flight and
+                            // spares, so that a slot is rewritten long after its last read)
+    uint32_t wdig[8][8];    // per warp: its contribution to the tile digest
+    uint32_t wsum[8];       // sum of widths so far | warps arrived << 16 (the last warp publishes)
+    uint32_t next[2];       // ticket claimed in this step (>= n_tiles: none left), by step parity
+    uint32_t pad[2];
+    unsigned long long excl[2];   // offset of the tile packed in this step, by step parity
 };
 static_assert(sizeof(EncTeamCtl) % 16 == 0, "team control block keeps 16-byte alignment");
-constexpr uint32_t kTeamSmemEncode = kTile + sizeof(EncTeamCtl);
+constexpr uint32_t kTeamSmemEncode = sizeof(EncTeamCtl);
 
 struct TileInfo {
     uint32_t t, c, left;
@@ -572,60 +573,76 @@ __device__ __forceinline__ uint32_t encoded_len(const TileInfo& ti, uint32_t S)
     return S <= 253u ? 8256u + 32u * S : kTile;
 }
 
-// Bit-pack the lane's eight exponent deltas (e4a, e4b: bytes in coded order, each < 2^W after
-// the base is subtracted) into W bytes at ep.  W is a compile-time constant so that every
-// shift and mask is an immediate and the store uses the widest aligned form.
+__device__ __forceinline__ void stg_u8(void* p, uint32_t v)
+{
+    asm volatile("st.global.cs.u8 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+__device__ __forceinline__ void stg_u16(void* p, uint32_t v)
+{
+    asm volatile("st.global.cs.u16 [%0], %1;" ::"l"(p), "h"((unsigned short)v) : "memory");
+}
+__device__ __forceinline__ void stg_v2(void* p, uint32_t a, uint32_t b)
+{
+    asm volatile("st.global.cs.v2.u32 [%0], {%1, %2};" ::"l"(p), "r"(a), "r"(b) : "memory");
+}
+
+// Write the bit planes of one group straight to the wire image.  The lane holds the eight
+// exponent bytes of its elements (e4a, e4b, coded order); after the base is subtracted each
+// is < 2^W.  W = 8 is stored as it is; otherwise a 4-bit, a 2-bit and a 1-bit plane (those
+// whose bit is set in W) take consecutive bits of the deltas from bit 0.  In every plane lane
+// l owns an aligned 4 / 2 / 1-byte unit at l times that size, so each warp store covers one
+// contiguous, sector-aligned run of 128 / 64 / 32 bytes and nothing needs staging.
+//   nibbles : v | v >> 4 puts two 4-bit values side by side in bytes 0 and 2 of each word
+//   2 bits  : (t * 0x01041040) >> 24 gathers the four 2-bit fields of a word into one byte
+//   1 bit   : (t * 0x01020408) >> 24 gathers the four bits of a word into one nibble
+// (the partial products of both multiplications land on distinct bits, so no carry occurs).
 template <int W>
-__device__ __forceinline__ void pack_group(uint32_t e4a, uint32_t e4b, uint32_t base, unsigned char* ep)
+__device__ __forceinline__ void pack_group_planes(uint32_t e4a, uint32_t e4b, uint32_t base, unsigned char* rec,
+                                                  uint32_t lane)
 {
     const uint32_t b4 = base * 0x01010101u;
-    const uint32_t da = e4a - b4, db = e4b - b4;
+    uint32_t da = e4a - b4, db = e4b - b4;
     if (W == 8) {
-        *reinterpret_cast<uint2*>(ep) = make_uint2(da, db);
+        stg_v2(rec + 8 * lane, da, db);
         return;
     }
-    constexpr int V = W & 7;                              // W == 8 returned above; keeps shifts in range
-    constexpr uint32_t sh = 8 - V;
-    constexpr uint32_t m1 = ((1u << V) - 1u) * 0x00010001u;
-    constexpr uint32_t m2 = (1u << (2 * V)) - 1u;
-    const uint32_t ya = (da & m1) | ((da >> sh) & (m1 << V));
-    const uint32_t yb = (db & m1) | ((db >> sh) & (m1 << V));
-    const uint32_t za = (ya & m2) | ((ya >> (16 - 2 * V)) & (m2 << (2 * V)));
-    const uint32_t zb = (yb & m2) | ((yb >> (16 - 2 * V)) & (m2 << (2 * V)));
-    const uint32_t lo = za + (zb << (4 * V));            // disjoint bit fields: add == or
-    const uint32_t hi = (V > 4) ? (zb >> ((32 - 4 * V) & 31)) : 0u;
-    if (W == 1) ep[0] = (unsigned char)lo;
-    else if (W == 2) *reinterpret_cast<uint16_t*>(ep) = (uint16_t)lo;
-    else if (W == 3) { ep[0] = (unsigned char)lo; ep[1] = (unsigned char)(lo >> 8); ep[2] = (unsigned char)(lo >> 16); }
-    else if (W == 4) *reinterpret_cast<uint32_t*>(ep) = lo;
-    else if (W == 5) {
-        ep[0] = (unsigned char)lo; ep[1] = (unsigned char)(lo >> 8); ep[2] = (unsigned char)(lo >> 16);
-        ep[3] = (unsigned char)(lo >> 24); ep[4] = (unsigned char)hi;
-    } else if (W == 6) {
-        reinterpret_cast<uint16_t*>(ep)[0] = (uint16_t)lo; reinterpret_cast<uint16_t*>(ep)[1] = (uint16_t)(lo >> 16);
-        reinterpret_cast<uint16_t*>(ep)[2] = (uint16_t)hi;
-    } else {
-        ep[0] = (unsigned char)lo; ep[1] = (unsigned char)(lo >> 8); ep[2] = (unsigned char)(lo >> 16);
-        ep[3] = (unsigned char)(lo >> 24); ep[4] = (unsigned char)hi; ep[5] = (unsigned char)(hi >> 8);
-        ep[6] = (unsigned char)(hi >> 16);
+    unsigned char* p = rec;
+    if (W & 4) {
+        const uint32_t na = (W == 4) ? da : (da & 0x0F0F0F0Fu), nb = (W == 4) ? db : (db & 0x0F0F0F0Fu);
+        const uint32_t va = na | (na >> 4), vb = nb | (nb >> 4);
+        st_stream_u32(p + 4 * lane, __byte_perm(va, vb, 0x6420));
+        p += 128;
+        da >>= 4; db >>= 4;
+    }
+    if (W & 2) {
+        const uint32_t pa = (da & 0x03030303u) * 0x01041040u, pb = (db & 0x03030303u) * 0x01041040u;
+        stg_u16(p + 2 * lane, __byte_perm(pa, pb, 0x0073));
+        p += 64;
+        da >>= 2; db >>= 2;
+    }
+    if (W & 1) {
+        const uint32_t pa = (da & 0x01010101u) * 0x01020408u, pb = (db & 0x01010101u) * 0x01020408u;
+        const uint32_t x = __byte_perm(pa, pb, 0x0073);          // byte 0: a's nibble, byte 1: b's nibble
+        stg_u8(p + lane, x | (x >> 4));
     }
 }
 
 // Single-pass fused checksum + encode.  Each team keeps three tiles in flight:
-//     A  measured two steps ago, packed and written out in this step
-//     B  measured one step ago, waiting for its offset
-//     C  checksummed and measured in this step (its length is published at once)
+//     X  measured two steps ago, packed and written to the wire image in this step
+//     W  measured one step ago, waiting for its offset
+//     Y  checksummed and measured in this step (its length is published at once)
 // and per step does
-//     probe A's offset | pack A into shared memory | re-request B's words | digest + exponent
-//     ranges of C, publish len(C) | take A's offset (wait if the scanner is not there yet) |
-//     claim D, start its loads | copy A out.
+//     request X's offset and claim Z (two round trips to L2, answers used later) |
+//     digest + exponent ranges of Y, publish len(Y) | one team barrier | start loading Z |
+//     pack X straight into the wire image | re-request W's words for the next step.
 // The two steps between measuring a tile and needing its offset cover the time the scanner
-// needs (its poll plus the owner's read are two round trips to L2 under full load).  A tile's
-// words are not kept in registers over those two steps: they are read again for packing, one
-// step ahead, and come from L2 (a few hundred tiles, some tens of MB, were read in between).
-// A team never waits while it holds a claimed tile whose length is not on its way out: len(C)
-// is published by the team's own warps without waiting for anyone, and D is claimed only
-// after A's offset has arrived.
+// needs.  A tile's words are not kept in registers over those two steps: they are read again
+// for packing, one step ahead, and come from L2 (they were loaded with evict-last priority).
+// Packed data goes from registers to the wire image directly: in every region of a PACK tile
+// a lane owns an aligned unit at a lane-strided place, so each warp store is one contiguous
+// sector-aligned run.  Claiming Z before X's offset is known means that, if the scanner is
+// late, this team waits while Z's length is not out yet; with two steps of slack that is
+// rare, and it only delays: the teams that hold earlier tiles never depend on this one.
 template <int TEAMS>
 __global__ void __launch_bounds__(TEAMS * 256, 1)
 k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restrict__ dirty,
@@ -633,7 +650,7 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
 {
     extern __shared__ __align__(16) unsigned char smem[];
     // The first block to get here becomes the scanner: one warp of it, alone on its SM (a warp
-    // that shares its scheduler with six busy ones gets too few issue slots to keep up).
+    // that shares its scheduler with busy ones gets too few issue slots to keep up).
     __shared__ uint32_t s_scanner;
     if (threadIdx.x == 0) s_scanner = atomicCAS(&ws.ctrl->scan_lock, 0u, 1u) == 0u;
     __syncthreads();
@@ -645,21 +662,18 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
     Smem S = setup_smem(smem, tab);
     const uint32_t team = threadIdx.x / kTeamThreads, tt = threadIdx.x % kTeamThreads;
     const uint32_t warp = tt / 32, lane = tt % 32;
-    unsigned char* out = nullptr;
-    for (int i = 0; i < TEAMS; i++) {          // every thread carves the same blocks in the same order
-        unsigned char* p = S.take(kTeamSmemEncode);
-        if ((uint32_t)i == team) out = p;
-    }
+    EncTeamCtl* tc = reinterpret_cast<EncTeamCtl*>(S.take(TEAMS * kTeamSmemEncode));
     if (!S.ok) { if (threadIdx.x == 0) atomicOr(&ws.ctrl->err, 4u); return; }
-    EncTeamCtl* tc = reinterpret_cast<EncTeamCtl*>(out + kTile);
+    tc += team;
     unsigned char* dir = wire + 64;
     uint16_t* tile_tab = reinterpret_cast<uint16_t*>(wire + 64 + 16ull * g.n_chunks);
+    const uint64_t pol_keep = l2_policy_evict_last();
     auto info = [&](uint32_t t) { return tile_info(g, dirty, t); };
     auto publish_len = [&](uint32_t t, uint32_t len) { st_relaxed_u32(ws.lbk + t, kFlagA | (len / kUnit)); };
 
-    // Digest and per-group exponent range of one tile; results go to wdig[par], wtab[par].  The
-    // tile's encoded length is published by whichever warp finishes last (no team barrier).
-    auto measure = [&](const TileInfo& ti, uint32_t (&d)[kWordsPerLane], uint32_t par) {
+    // Digest and per-group exponent range of one tile; results go to slot `sl`.  The tile's
+    // encoded length is published by whichever warp finishes last (no team barrier).
+    auto measure = [&](const TileInfo& ti, uint32_t (&d)[kWordsPerLane], uint32_t sl) {
         if (!ti.valid) return;
         if (!ti.present || !ti.full) {
             if (warp == 0 && lane == 0) publish_len(ti.t, encoded_len(ti, 0));
@@ -667,188 +681,181 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
             load_tile_words_guarded(cache + (uint64_t)ti.t * kTile, ti.left, ti.first, warp, lane, d);
         }
         const uint32_t v = tile_digest_part(S, d, ti.first && ti.full, warp, lane);
-        if (lane == 0) tc->wdig[par][warp] = v;
+        if (lane == 0) tc->wdig[sl][warp] = v;
         if (ti.full) {
             uint32_t mysum = 0;
 #pragma unroll
             for (int j = 0; j < 4; j++) {
-                const uint32_t a0 = d[4 * j] & 0x7FFF7FFFu, a1 = d[4 * j + 1] & 0x7FFF7FFFu;
-                const uint32_t a2 = d[4 * j + 2] & 0x7FFF7FFFu, a3 = d[4 * j + 3] & 0x7FFF7FFFu;
+                // w << 1 drops the upper element's sign and leaves [E | m | junk bit] in each half
+                const uint32_t a0 = d[4 * j] * 2u, a1 = d[4 * j + 1] * 2u, a2 = d[4 * j + 2] * 2u, a3 = d[4 * j + 3] * 2u;
                 uint32_t mn = min_u16x2(min_u16x2(a0, a1), min_u16x2(a2, a3));
                 uint32_t mx = max_u16x2(max_u16x2(a0, a1), max_u16x2(a2, a3));
                 mn = min(mn & 0xFFFFu, mn >> 16);
                 mx = max(mx & 0xFFFFu, mx >> 16);
-                const uint32_t emin = __reduce_min_sync(0xFFFFFFFFu, mn) >> 7;
-                const uint32_t emax = __reduce_max_sync(0xFFFFFFFFu, mx) >> 7;
+                const uint32_t emin = __reduce_min_sync(0xFFFFFFFFu, mn) >> 8;
+                const uint32_t emax = __reduce_max_sync(0xFFFFFFFFu, mx) >> 8;
                 const uint32_t wd = 32u - __clz(emax - emin);
                 mysum += wd;
-                if (lane == 0) tc->wtab[par][4 * warp + j] = emin | (wd << 8);
+                if (lane == 0) tc->wtab[sl][4 * warp + j] = emin | (wd << 8);
             }
             if (lane == 0) {
-                const uint32_t old = atomicAdd(&tc->wsum[par], mysum + (1u << 16));
+                const uint32_t old = atomicAdd(&tc->wsum[sl], mysum + (1u << 16));
                 if ((old >> 16) == 7u) {
-                    tc->wsum[par] = 0;
+                    tc->wsum[sl] = 0;
                     publish_len(ti.t, encoded_len(ti, (old & 0xFFFFu) + mysum));
                 }
             }
         }
     };
-    auto fetch = [&](const TileInfo& ti, uint32_t (&d)[kWordsPerLane]) {
+    auto fetch = [&](const TileInfo& ti, uint32_t (&d)[kWordsPerLane]) {       // first read: keep in L2
+        if (ti.present && ti.full) load_tile_words_keep(cache + (uint64_t)ti.t * kTile, warp, lane, d, pol_keep);
+    };
+    auto refetch = [&](const TileInfo& ti, uint32_t (&d)[kWordsPerLane]) {     // second read: last use
         if (ti.present && ti.full) load_tile_words(cache + (uint64_t)ti.t * kTile, warp, lane, d);
     };
 
-    // One pipeline step (X = A, W = B, Y = C above): pack X (words in dP), re-request W into dP,
-    // measure Y (words in dM), place X, claim Z and start loading it into dM.
-    TileInfo iX = info(0xFFFFFFFFu), iW = iX, iY = iX;
-    uint32_t par = 0;                  // slot of X; W has slot par+1, Y slot par+2 (mod 3)
-    auto nxt = [](uint32_t p) { return p == 2u ? 0u : p + 1u; };
-    auto step = [&](uint32_t (&dP)[kWordsPerLane], uint32_t (&dM)[kWordsPerLane]) {
-        const uint32_t parW = nxt(par), parY = nxt(parW);
-        team_bar(team);                                               // bar0: out buffer free
-        // X's length went out one step ago; ask for its offset now, use the answer later
-        const bool leader = (warp == 0 && lane == 0);
-        uint32_t pv = 0;
-        if (leader) pv = ld_relaxed_u32(ws.lbk + iX.t);
+    // Pack tile X (words in d, widths in slot sl) into the wire image at payload offset excl.
+    auto pack = [&](const TileInfo& ti, const uint32_t (&d)[kWordsPerLane], uint32_t sl, unsigned long long excl) {
         uint32_t enc_len = 0, entry = 0;
-        bool staged = false;                                          // encoded tile sits in `out`
-        if (iX.present && iX.full) {
-            const uint32_t wt = tc->wtab[par][lane];
-            const uint32_t wv = (wt >> 8) & 15u;
-            uint32_t incl = wv;
+        if (ti.present) {
+            unsigned char* dst = wire + g.meta_end + excl;
+            if (ti.full) {
+                const uint32_t wt = tc->wtab[sl][lane];
+                const uint32_t wv = (wt >> 8) & 15u;
+                uint32_t incl = wv;
 #pragma unroll
-            for (int d = 1; d < 32; d <<= 1) {
-                const uint32_t o = __shfl_up_sync(0xFFFFFFFFu, incl, d);
-                if (lane >= (uint32_t)d) incl += o;
-            }
-            const uint32_t Ssum = __shfl_sync(0xFFFFFFFFu, incl, 31);
-            staged = true;
-            if (Ssum <= 253u) {
-                enc_len = 8256u + 32u * Ssum;
-                entry = 258u + Ssum;
-                if (warp == 0) reinterpret_cast<uint16_t*>(out)[lane] = (uint16_t)desc_of(wt & 0xFFu, wv);
+                for (int k = 1; k < 32; k <<= 1) {
+                    const uint32_t o = __shfl_up_sync(0xFFFFFFFFu, incl, k);
+                    if (lane >= (uint32_t)k) incl += o;
+                }
+                const uint32_t Ssum = __shfl_sync(0xFFFFFFFFu, incl, 31);
+                const bool packs = Ssum <= 253u;
+                enc_len = packs ? 8256u + 32u * Ssum : kTile;
+                entry = packs ? 258u + Ssum : 512u;
+                if (g.meta_end + excl + enc_len > wire_cap) {
+                    if (tt == 0) atomicOr(&ws.ctrl->err, 1u);
+                } else if (packs) {
+                    if (warp == 0) stg_u16(dst + 2 * lane, desc_of(wt & 0xFFu, wv));
 #pragma unroll
-                for (int j = 0; j < 4; j++) {
-                    const uint32_t gi = 4 * warp + j;
-                    const uint32_t wtg = __shfl_sync(0xFFFFFFFFu, wt, gi);
-                    const uint32_t exg = __shfl_sync(0xFFFFFFFFu, incl - wv, gi);
-                    const uint32_t base = wtg & 0xFFu, wd = (wtg >> 8) & 15u;
-                    uint32_t Tr[4];
+                    for (int j = 0; j < 4; j++) {
+                        const uint32_t gi = 4 * warp + j;
+                        const uint32_t wtg = __shfl_sync(0xFFFFFFFFu, wt, gi);
+                        const uint32_t exg = __shfl_sync(0xFFFFFFFFu, incl - wv, gi);
+                        const uint32_t base = wtg & 0xFFu, wd = (wtg >> 8) & 15u;
+                        uint32_t Tr[4];
 #pragma unroll
-                    for (int r = 0; r < 4; r++) {
-                        const uint32_t W = dP[4 * j + r];
-                        Tr[r] = ((W << 1) & 0xFFFEFFFEu) | ((W >> 15) & 0x00010001u);
+                        for (int r = 0; r < 4; r++) {
+                            const uint32_t Wd = d[4 * j + r];
+                            Tr[r] = ((Wd << 1) & 0xFFFEFFFEu) | ((Wd >> 15) & 0x00010001u);
+                        }
+                        stg_v2(dst + 64 + 256 * gi + 8 * lane, __byte_perm(Tr[0], Tr[1], 0x6420),
+                               __byte_perm(Tr[2], Tr[3], 0x6420));
+                        const uint32_t e4a = __byte_perm(Tr[0], Tr[1], 0x7531), e4b = __byte_perm(Tr[2], Tr[3], 0x7531);
+                        unsigned char* rec = dst + 8256 + 32 * exg;
+                        switch (wd) {          // uniform across the warp
+                            case 1: pack_group_planes<1>(e4a, e4b, base, rec, lane); break;
+                            case 2: pack_group_planes<2>(e4a, e4b, base, rec, lane); break;
+                            case 3: pack_group_planes<3>(e4a, e4b, base, rec, lane); break;
+                            case 4: pack_group_planes<4>(e4a, e4b, base, rec, lane); break;
+                            case 5: pack_group_planes<5>(e4a, e4b, base, rec, lane); break;
+                            case 6: pack_group_planes<6>(e4a, e4b, base, rec, lane); break;
+                            case 7: pack_group_planes<7>(e4a, e4b, base, rec, lane); break;
+                            case 8: pack_group_planes<8>(e4a, e4b, base, rec, lane); break;
+                            default: break;
+                        }
                     }
-                    const uint32_t sma = __byte_perm(Tr[0], Tr[1], 0x6420), smb = __byte_perm(Tr[2], Tr[3], 0x6420);
-                    *reinterpret_cast<uint2*>(out + 64 + 256 * gi + 8 * lane) = make_uint2(sma, smb);
-                    const uint32_t e4a = __byte_perm(Tr[0], Tr[1], 0x7531), e4b = __byte_perm(Tr[2], Tr[3], 0x7531);
-                    unsigned char* ep = out + 8256 + 32 * exg + lane * wd;
-                    switch (wd) {          // uniform across the warp
-                        case 1: pack_group<1>(e4a, e4b, base, ep); break;
-                        case 2: pack_group<2>(e4a, e4b, base, ep); break;
-                        case 3: pack_group<3>(e4a, e4b, base, ep); break;
-                        case 4: pack_group<4>(e4a, e4b, base, ep); break;
-                        case 5: pack_group<5>(e4a, e4b, base, ep); break;
-                        case 6: pack_group<6>(e4a, e4b, base, ep); break;
-                        case 7: pack_group<7>(e4a, e4b, base, ep); break;
-                        case 8: pack_group<8>(e4a, e4b, base, ep); break;
-                        default: break;
-                    }
+                } else {
+                    unsigned char* q = dst + warp * 2048u + lane * 4u;
+#pragma unroll
+                    for (int i = 0; i < 16; i++) st_stream_u32(q + i * 128, d[i]);
                 }
             } else {
-                enc_len = kTile;
-                entry = 512u;
-                uint32_t* o32 = reinterpret_cast<uint32_t*>(out) + warp * 512u + lane;
-#pragma unroll
-                for (int i = 0; i < 16; i++) o32[i * 32] = dP[i];
-            }
-        } else if (iX.present) {
-            enc_len = iX.left;
-            entry = 0xFFFFu;
-        }
-
-        fetch(iW, dP);                      // W's words again, for the next step's pack
-
-        // fast path: the offset is already there, so this step will not wait and may claim Z now
-        uint32_t tk = 0xFFFFFFFFu;
-        bool claimed = false;
-        if (leader && (pv >> 30) == 2u) {
-            if (iY.valid) tk = next_ticket(ws.ctrl);
-            claimed = true;
-        }
-
-        // second chance: ask again before the checksum work, look at the answer after it
-        uint32_t pv1 = 0;
-        if (leader && !claimed) pv1 = ld_relaxed_u32(ws.lbk + iX.t);
-
-        measure(iY, dM, parY);
-
-        if (leader) {
-#ifdef WM_DEBUG_COUNTERS
-            atomicAdd(&ws.ctrl->pad[claimed ? 3 : ((pv1 >> 30) == 2u ? 4 : 2)], 1u);
-#endif
-            unsigned long long e;
-            if (claimed) {
-                e = (unsigned long long)(pv & kValMask) * kUnit;
-            } else {                        // len(Y) is on its way out; now it is safe to wait
-                e = (pv1 >> 30) == 2u ? (unsigned long long)(pv1 & kValMask) * kUnit
-                                      : wait_prefix(ws.lbk, iX.t, ws.ctrl);
-                if (iY.valid) tk = next_ticket(ws.ctrl);
-            }
-            tc->excl = e;
-            tc->next = tk;
-            if (iX.t + 1 == g.n_tiles) ws.ctrl->payload_total = e + enc_len;
-        }
-        team_bar(team);                                               // bar2: offset known, out complete
-
-        const TileInfo iZ = info(tc->next);
-        fetch(iZ, dM);                                                // dM is free: Y has been measured
-
-        const unsigned long long excl = tc->excl;
-        if (iX.present) {
-            const uint64_t dst = g.meta_end + excl;
-            if (dst + enc_len > wire_cap) {
-                if (tt == 0) atomicOr(&ws.ctrl->err, 1u);
-            } else if (staged) {
-                for (uint32_t i = tt * 16; i < enc_len; i += kTeamThreads * 16)
-                    *reinterpret_cast<uint4*>(wire + dst + i) = *reinterpret_cast<const uint4*>(out + i);
-            } else {
-                const unsigned char* src = cache + (uint64_t)iX.t * kTile;
-                for (uint32_t i = tt; i < enc_len; i += kTeamThreads) wire[dst + i] = src[i];
+                enc_len = ti.left;
+                entry = 0xFFFFu;
+                if (g.meta_end + excl + enc_len > wire_cap) {
+                    if (tt == 0) atomicOr(&ws.ctrl->err, 1u);
+                } else {
+                    const unsigned char* src = cache + (uint64_t)ti.t * kTile;
+                    for (uint32_t i = tt; i < enc_len; i += kTeamThreads) dst[i] = src[i];
+                }
             }
         }
         if (tt == 0) {
-            tile_tab[iX.t] = (uint16_t)entry;
-            if (iX.present) ws.dig[iX.t] = xor8(tc->wdig[par]);
-            if (iX.first) *reinterpret_cast<unsigned long long*>(dir + 16ull * iX.c) = excl;
+            tile_tab[ti.t] = (uint16_t)entry;
+            if (ti.present) ws.dig[ti.t] = xor8(tc->wdig[sl]);
+            if (ti.first) *reinterpret_cast<unsigned long long*>(dir + 16ull * ti.c) = excl;
+            if (ti.t + 1 == g.n_tiles) ws.ctrl->payload_total = excl + enc_len;
         }
-        iX = iW;
-        iW = iY;
-        iY = iZ;
-        par = parW;
     };
 
-    // ---- prologue: X and W claimed, measured and published; Y claimed and loading; X's words
-    // requested again for the first pack
+    // Tiles in flight, oldest first: X (packed in this step), V, W (waiting for their offsets),
+    // Y (measured in this step).  Ring slots: X = sl, V = sl+1, W = sl+2, Y = sl+3 (mod 8).
+    TileInfo iX = info(0xFFFFFFFFu), iV = iX, iW = iX, iY = iX;
+    uint32_t sl = 0;
+    uint32_t par = 0;                  // step parity (selects next[] / excl[])
     uint32_t dP[kWordsPerLane], dM[kWordsPerLane];
-    if (tt == 0) { tc->wsum[0] = 0; tc->wsum[1] = 0; tc->wsum[2] = 0; tc->next = next_ticket(ws.ctrl); }
+    const bool leader = (warp == 0 && lane == 0);
+
+    // ---- prologue: X, V, W claimed, measured and published one after the other; Y claimed and
+    // loading; X's words requested again for the first pack; X's offset obtained
+    if (tt == 0) {
+        for (int i = 0; i < 8; i++) tc->wsum[i] = 0;
+        tc->next[0] = next_ticket(ws.ctrl);
+    }
     team_bar(team);
-    iX = info(tc->next);
+    iX = info(tc->next[0]);
     fetch(iX, dM);
     measure(iX, dM, 0);
+    if (tt == 0) tc->next[1] = iX.valid ? next_ticket(ws.ctrl) : 0xFFFFFFFFu;
     team_bar(team);
-    if (tt == 0) tc->next = iX.valid ? next_ticket(ws.ctrl) : 0xFFFFFFFFu;
+    iV = info(tc->next[1]);
+    fetch(iV, dM);
+    measure(iV, dM, 1);
+    if (tt == 0) tc->next[0] = iV.valid ? next_ticket(ws.ctrl) : 0xFFFFFFFFu;
     team_bar(team);
-    iW = info(tc->next);
+    iW = info(tc->next[0]);
     fetch(iW, dM);
-    measure(iW, dM, 1);
+    measure(iW, dM, 2);
+    if (tt == 0) {
+        tc->next[1] = iW.valid ? next_ticket(ws.ctrl) : 0xFFFFFFFFu;
+        tc->excl[0] = iX.valid ? wait_prefix(ws.lbk, iX.t, ws.ctrl) : 0ull;
+    }
     team_bar(team);
-    if (tt == 0) tc->next = iW.valid ? next_ticket(ws.ctrl) : 0xFFFFFFFFu;
-    team_bar(team);
-    iY = info(tc->next);
+    iY = info(tc->next[1]);
     fetch(iY, dM);
-    fetch(iX, dP);
+    refetch(iX, dP);
+    unsigned long long exclX = tc->excl[0];
+    team_bar(team);
 
-    while (iX.valid) step(dP, dM);
+    while (iX.valid) {
+        // two round trips to L2 whose answers are used at the end of the step: the ticket of
+        // the tile to load next, and the offset of the tile to pack in the next step
+        uint32_t pv = 0, tk = 0xFFFFFFFFu;
+        if (leader) {
+            if (iV.valid) pv = ld_relaxed_u32(ws.lbk + iV.t);
+            if (iY.valid) tk = next_ticket(ws.ctrl);
+        }
+        pack(iX, dP, sl, exclX);
+        refetch(iV, dP);                                              // V's words again, for the next pack
+        measure(iY, dM, (sl + 3u) & 7u);
+        if (leader) {
+#ifdef WM_DEBUG_COUNTERS
+            atomicAdd(&ws.ctrl->pad[(pv >> 30) == 2u ? 3 : 2], 1u);
+#endif
+            unsigned long long e = 0;
+            if (iV.valid)
+                e = (pv >> 30) == 2u ? (unsigned long long)(pv & kValMask) * kUnit : wait_prefix(ws.lbk, iV.t, ws.ctrl);
+            tc->excl[par] = e;
+            tc->next[par] = tk;
+        }
+        team_bar(team);            // offset and ticket visible; every warp is done with this step's slots
+        const TileInfo iZ = info(tc->next[par]);
+        fetch(iZ, dM);                                                // dM is free: Y has been measured
+        exclX = tc->excl[par];
+        iX = iV; iV = iW; iW = iY; iY = iZ;
+        sl = (sl + 1u) & 7u;
+        par ^= 1u;
+    }
 }
 
 // Directory (enc_len, crc), chunk CRCs, present count; the last block to finish combines the
@@ -1178,32 +1185,72 @@ struct DecTeamCtl {
 };
 static_assert(sizeof(DecTeamCtl) % 16 == 0, "team control block keeps 16-byte alignment");
 
-// Inverse of pack_group: the lane's eight exponent bytes (two words, coded order) from the
-// aligned window (w0, w1, w2) that covers its W packed bytes; sh = 8 * (byte offset & 3).
-template <int W>
-__device__ __forceinline__ void unpack_group(uint32_t w0, uint32_t w1, uint32_t w2, uint32_t sh, uint32_t base,
-                                             uint32_t& ea, uint32_t& eb)
+__device__ __forceinline__ uint32_t ldg_u8(const void* p)
 {
-    const uint32_t lo = __funnelshift_r(w0, w1, sh);
-    const uint32_t hi = __funnelshift_r(w1, w2, sh);
-    uint32_t da, db;
-    if (W == 8) { da = lo; db = hi; }
-    else {
-        constexpr int V = W & 7;
-        constexpr uint32_t m4 = (1u << (4 * V)) - 1u;
-        constexpr uint32_t m2 = (1u << (2 * V)) - 1u;
-        constexpr uint32_t m1 = ((1u << V) - 1u) * 0x00010001u;
-        constexpr uint32_t sh1 = 8 - V;
-        const uint32_t za = lo & m4;
-        const uint32_t zb = (V <= 4 ? (lo >> (4 * V)) : __funnelshift_r(lo, hi, 4 * V)) & m4;
-        const uint32_t ya = (za & m2) | ((za << (16 - 2 * V)) & (m2 << 16));
-        const uint32_t yb = (zb & m2) | ((zb << (16 - 2 * V)) & (m2 << 16));
-        da = (ya & m1) | ((ya << sh1) & (m1 << 8));
-        db = (yb & m1) | ((yb << sh1) & (m1 << 8));
+    uint32_t v;
+    asm volatile("ld.global.nc.u8 %0, [%1];" : "=r"(v) : "l"(p));
+    return v;
+}
+__device__ __forceinline__ uint32_t ldg_u16(const void* p)
+{
+    unsigned short v;
+    asm volatile("ld.global.nc.u16 %0, [%1];" : "=h"(v) : "l"(p));
+    return v;
+}
+
+// The raw plane words of one group, as loaded (aligned per-lane units, see pack_group_planes).
+struct PlaneWords { uint32_t p4, p2, p1, p8lo, p8hi; };
+
+__device__ __forceinline__ PlaneWords load_group_planes(const unsigned char* rec, uint32_t wd, uint32_t lane)
+{
+    PlaneWords pw;
+    pw.p4 = pw.p2 = pw.p1 = pw.p8lo = pw.p8hi = 0;
+    if (wd == 8u) {
+        const uint2 v = *reinterpret_cast<const uint2*>(rec + 8 * lane);
+        pw.p8lo = v.x; pw.p8hi = v.y;
+        return pw;
     }
-    const uint32_t b4 = base * 0x01010101u;        // per byte (base + d) & 0xFF
-    ea = ((da & 0x7F7F7F7Fu) + (b4 & 0x7F7F7F7Fu)) ^ ((da ^ b4) & 0x80808080u);
-    eb = ((db & 0x7F7F7F7Fu) + (b4 & 0x7F7F7F7Fu)) ^ ((db ^ b4) & 0x80808080u);
+    const unsigned char* p = rec;
+    if (wd & 4u) { pw.p4 = *reinterpret_cast<const uint32_t*>(p + 4 * lane); p += 128; }
+    if (wd & 2u) { pw.p2 = ldg_u16(p + 2 * lane); p += 64; }
+    if (wd & 1u) { pw.p1 = ldg_u8(p + lane); }
+    return pw;
+}
+
+// Inverse of pack_group_planes: the lane's eight exponent bytes (two words, coded order).
+template <int W>
+__device__ __forceinline__ void unpack_group_planes(const PlaneWords& pw, uint32_t base, uint32_t& ea, uint32_t& eb)
+{
+    uint32_t da = 0, db = 0;
+    if (W == 8) { da = pw.p8lo; db = pw.p8hi; }
+    else {
+        int sh = 0;
+        if (W & 4) {
+            const uint32_t t = __byte_perm(pw.p4, 0, 0x1100), u = __byte_perm(pw.p4, 0, 0x3322);
+            da = (t & 0x000F000Fu) | ((t >> 4) & 0x0F000F00u);
+            db = (u & 0x000F000Fu) | ((u >> 4) & 0x0F000F00u);
+            sh = 4;
+        }
+        if (W & 2) {        // byte -> four 2-bit fields, one per byte
+            uint32_t xa = pw.p2 & 0xFFu, xb = (pw.p2 >> 8) & 0xFFu;
+            xa = (xa * 0x1001u) & 0x000F000Fu; xa = (xa * 0x41u) & 0x03030303u;
+            xb = (xb * 0x1001u) & 0x000F000Fu; xb = (xb * 0x41u) & 0x03030303u;
+            da |= xa << sh; db |= xb << sh;
+            sh += 2;
+        }
+        if (W & 1) {        // nibble -> four bits, one per byte
+            const uint32_t xa = ((pw.p1 & 0xFu) * 0x00204081u) & 0x01010101u;
+            const uint32_t xb = (((pw.p1 >> 4) & 0xFu) * 0x00204081u) & 0x01010101u;
+            da |= xa << sh; db |= xb << sh;
+        }
+    }
+    const uint32_t b4 = base * 0x01010101u;
+    if (base + ((1u << W) - 1u) <= 255u) {        // no byte can wrap: plain add
+        ea = da + b4; eb = db + b4;
+    } else {                                      // per byte (base + d) & 0xFF
+        ea = ((da & 0x7F7F7F7Fu) + (b4 & 0x7F7F7F7Fu)) ^ ((da ^ b4) & 0x80808080u);
+        eb = ((db & 0x7F7F7F7Fu) + (b4 & 0x7F7F7F7Fu)) ^ ((db ^ b4) & 0x80808080u);
+    }
 }
 
 __device__ __forceinline__ uint32_t ldg_u32(const void* p)
@@ -1291,34 +1338,29 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
                 } else {
                     // issue every load of the warp's four groups, then unpack
                     uint2 sm[4];
-                    uint32_t w0[4], w1[4], w2[4], dgv[4];
+                    PlaneWords pw[4];
+                    uint32_t dgv[4];
 #pragma unroll
                     for (int j = 0; j < 4; j++) {
                         const uint32_t gi = 4 * warp + j;
                         dgv[j] = __shfl_sync(0xFFFFFFFFu, desc, gi);
                         const uint32_t exg = __shfl_sync(0xFFFFFFFFu, incl - wv, gi);
-                        const uint32_t wd = (dgv[j] >> 8) & 15u;
                         sm[j] = *reinterpret_cast<const uint2*>(src + 64 + 256 * gi + 8 * lane);
-                        const unsigned char* rec = src + 8256 + 32 * exg;
-                        const uint32_t a = (lane * wd) & ~3u, rl = 32u * wd;
-                        w0[j] = (a < rl) ? ldg_u32(rec + a) : 0u;
-                        w1[j] = (a + 4 < rl) ? ldg_u32(rec + a + 4) : 0u;
-                        w2[j] = (a + 8 < rl) ? ldg_u32(rec + a + 8) : 0u;
+                        pw[j] = load_group_planes(src + 8256 + 32 * exg, (dgv[j] >> 8) & 15u, lane);
                     }
 #pragma unroll
                     for (int j = 0; j < 4; j++) {
                         const uint32_t base = dgv[j] & 0xFFu, wd = (dgv[j] >> 8) & 15u;
-                        const uint32_t sh = ((lane * wd) & 3u) * 8u;
                         uint32_t ea = base * 0x01010101u, eb = ea;
                         switch (wd) {          // uniform across the warp
-                            case 1: unpack_group<1>(w0[j], w1[j], w2[j], sh, base, ea, eb); break;
-                            case 2: unpack_group<2>(w0[j], w1[j], w2[j], sh, base, ea, eb); break;
-                            case 3: unpack_group<3>(w0[j], w1[j], w2[j], sh, base, ea, eb); break;
-                            case 4: unpack_group<4>(w0[j], w1[j], w2[j], sh, base, ea, eb); break;
-                            case 5: unpack_group<5>(w0[j], w1[j], w2[j], sh, base, ea, eb); break;
-                            case 6: unpack_group<6>(w0[j], w1[j], w2[j], sh, base, ea, eb); break;
-                            case 7: unpack_group<7>(w0[j], w1[j], w2[j], sh, base, ea, eb); break;
-                            case 8: unpack_group<8>(w0[j], w1[j], w2[j], sh, base, ea, eb); break;
+                            case 1: unpack_group_planes<1>(pw[j], base, ea, eb); break;
+                            case 2: unpack_group_planes<2>(pw[j], base, ea, eb); break;
+                            case 3: unpack_group_planes<3>(pw[j], base, ea, eb); break;
+                            case 4: unpack_group_planes<4>(pw[j], base, ea, eb); break;
+                            case 5: unpack_group_planes<5>(pw[j], base, ea, eb); break;
+                            case 6: unpack_group_planes<6>(pw[j], base, ea, eb); break;
+                            case 7: unpack_group_planes<7>(pw[j], base, ea, eb); break;
+                            case 8: unpack_group_planes<8>(pw[j], base, ea, eb); break;
                             default: break;
                         }
                         uint32_t Tr[4];

@@ -112,19 +112,51 @@ def test_wide_group_bit_layout():
         assert ep[_coded(e)] == E[e] - 7
 
 
-def test_three_bit_group_against_python_bit_string():
-    rng = np.random.default_rng(1)
-    E = np.full(8192, 50)
-    d = rng.integers(0, 8, 256)
-    d[10], d[11] = 0, 7
-    E[5 * 256:6 * 256] = 50 + d
+def _planes_python(d, w):
+    """Bit planes of a group, built with Python integers: widths 4, 2, 1 present when the bit
+    of w is set, consecutive bits of d from bit 0; element with coded position k at bits
+    [k p, (k+1) p) of its p-bit plane."""
+    if w == 8:
+        widths = [8]
+    else:
+        widths = [p for p in (4, 2, 1) if w & p]
+    out, lo = b"", 0
+    for p in widths:
+        bits = 0
+        for e in range(256):
+            bits |= ((int(d[e]) >> lo) & ((1 << p) - 1)) << (p * _coded(e))
+        out += bits.to_bytes(32 * p, "little")
+        lo += p
+    return out
+
+
+@pytest.mark.parametrize("w", [1, 2, 3, 4, 5, 6, 7, 8])
+def test_group_bit_planes_against_python_integers(w):
+    rng = np.random.default_rng(w)
+    base = 0 if w == 8 else 50
+    E = np.full(8192, base)
+    d = rng.integers(0, 1 << w, 256)
+    d[10], d[11] = 0, (1 << w) - 1
+    E[5 * 256:6 * 256] = base + d
     wire, _, _ = oracle.encode(_bf16_tile(E), TILE)
     ep = wire[96 + 64 + 8192:]
-    assert len(ep) == 96
-    bits = 0
-    for e in range(256):
-        bits |= int(d[e]) << (3 * _coded(e))
-    assert ep.tobytes() == bits.to_bytes(96, "little")
+    assert len(ep) == 32 * w
+    assert ep.tobytes() == _planes_python(d, w)
+
+
+def test_five_bit_group_planes_by_hand():
+    # d = 0b10011 at memory element 7 only: nibble 3 in the 4-bit plane, bit 1 in the 1-bit plane
+    E = np.full(8192, 60)
+    E[7] = 60 + 0b10011
+    wire, _, _ = oracle.encode(_bf16_tile(E), TILE)
+    ep = wire[96 + 64 + 8192:]
+    assert len(ep) == 160
+    k = _coded(7)                       # r = 0, l = 3, h = 1 -> 25
+    assert k == 25
+    want = np.zeros(160, dtype=np.uint8)
+    want[k // 2] = 0x3 << (4 * (k % 2))      # 4-bit plane, 128 bytes
+    want[128 + k // 8] = 1 << (k % 8)        # 1-bit plane, 32 bytes
+    assert ep.tolist() == want.tolist()
 
 
 def test_raw_fallback_never_expands_beyond_metadata():
