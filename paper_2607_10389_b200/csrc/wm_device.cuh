@@ -208,6 +208,63 @@ __device__ __forceinline__ void load_tile_words_keep(const unsigned char* tile, 
     for (int i = 0; i < 16; i++) w[i] = ld_keep_u32(p + i * 128, pol);
 }
 
+// ---- bulk (TMA) copies of whole tiles into shared memory, tracked by an mbarrier ----
+// Loads that land in registers long before they are used tie up the warp's few scoreboards:
+// every later shared-memory or global access that shares one waits for them, so "prefetching
+// into registers" serialises instead of overlapping.  A bulk copy is issued by one thread,
+// holds no registers while in flight, and its completion is observed on an mbarrier.
+__device__ __forceinline__ void mbar_init(unsigned long long* bar, uint32_t count)
+{
+    const uint32_t a = (uint32_t)__cvta_generic_to_shared(bar);
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(a), "r"(count) : "memory");
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+
+// One 16-byte aligned copy of `bytes` (multiple of 16) from global to shared memory; the
+// mbarrier's pending byte count is raised first.  `policy`: an L2 cache policy or 0.
+__device__ __forceinline__ void bulk_load(void* smem_dst, const void* gsrc, uint32_t bytes, unsigned long long* bar,
+                                          uint64_t policy)
+{
+    const uint32_t d = (uint32_t)__cvta_generic_to_shared(smem_dst);
+    const uint32_t b = (uint32_t)__cvta_generic_to_shared(bar);
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(b), "r"(bytes) : "memory");
+    if (policy)
+        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
+                     ::"r"(d), "l"(gsrc), "r"(bytes), "r"(b), "l"(policy) : "memory");
+    else
+        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                     ::"r"(d), "l"(gsrc), "r"(bytes), "r"(b) : "memory");
+}
+
+// Wait for the phase with the given parity to complete (bounded).  Returns false on timeout.
+__device__ __forceinline__ bool mbar_wait(unsigned long long* bar, uint32_t parity)
+{
+    const uint32_t b = (uint32_t)__cvta_generic_to_shared(bar);
+    for (uint32_t i = 0; i < (1u << 22); i++) {
+        uint32_t done;
+        asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                     : "=r"(done) : "r"(b), "r"(parity) : "memory");
+        if (done) return true;
+    }
+    return false;
+}
+
+__device__ __forceinline__ uint64_t l2_policy_evict_first()
+{
+    uint64_t pol;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+    return pol;
+}
+
+// A staged tile's words for this lane: word `lane` of rows 16*warp .. 16*warp+15 (conflict free).
+__device__ __forceinline__ void read_staged_words(const unsigned char* stage, uint32_t warp, uint32_t lane,
+                                                  uint32_t (&w)[16])
+{
+    const uint32_t* p = reinterpret_cast<const uint32_t*>(stage) + warp * 512u + lane;
+#pragma unroll
+    for (int i = 0; i < 16; i++) w[i] = p[i * 32];
+}
+
 // Full tile, fast path: lane's word of row 16*warp + i.
 __device__ __forceinline__ void load_tile_words(const unsigned char* tile, uint32_t warp, uint32_t lane,
                                                 uint32_t (&w)[kWordsPerLane])

@@ -540,10 +540,12 @@ struct EncTeamCtl {
     uint32_t wsum[8];       // sum of widths so far | warps arrived << 16 (the last warp publishes)
     uint32_t next[2];       // ticket claimed in this step (>= n_tiles: none left), by step parity
     uint32_t pad[2];
-    unsigned long long excl[2];   // offset of the tile packed in this step, by step parity
+    unsigned long long excl[2];   // offset of the tile packed in the next step, by step parity
+    unsigned long long mbar;      // completion of the bulk copy into the team's stage
+    unsigned long long pad2;
 };
 static_assert(sizeof(EncTeamCtl) % 16 == 0, "team control block keeps 16-byte alignment");
-constexpr uint32_t kTeamSmemEncode = sizeof(EncTeamCtl);
+constexpr uint32_t kTeamSmemEncode = kTile + sizeof(EncTeamCtl);   // one 16 KiB stage + control
 
 struct TileInfo {
     uint32_t t, c, left;
@@ -627,22 +629,26 @@ __device__ __forceinline__ void pack_group_planes(uint32_t e4a, uint32_t e4b, ui
     }
 }
 
-// Single-pass fused checksum + encode.  Each team keeps three tiles in flight:
-//     X  measured two steps ago, packed and written to the wire image in this step
-//     W  measured one step ago, waiting for its offset
+// Single-pass fused checksum + encode.  Each team keeps four tiles in flight:
+//     X  measured three steps ago, packed and written to the wire image in this step
+//     V, W  measured two / one steps ago, waiting for their offsets
 //     Y  checksummed and measured in this step (its length is published at once)
-// and per step does
-//     request X's offset and claim Z (two round trips to L2, answers used later) |
-//     digest + exponent ranges of Y, publish len(Y) | one team barrier | start loading Z |
-//     pack X straight into the wire image | re-request W's words for the next step.
-// The two steps between measuring a tile and needing its offset cover the time the scanner
-// needs.  A tile's words are not kept in registers over those two steps: they are read again
-// for packing, one step ahead, and come from L2 (they were loaded with evict-last priority).
+// The team owns one 16 KiB stage in shared memory that bulk copies (TMA) fill; a tile's words
+// go through it twice, once for measuring and, three steps later, once more for packing (that
+// second read comes from L2: the first one asks for evict-last priority).  Per step:
+//     read X's words from the stage | start the copy of Y | pack X straight into the wire
+//     image | read Y's words from the stage | start the copy of V (next step's X) |
+//     digest + exponent ranges of Y, publish len(Y)
+// so each copy has the other phase's work to hide behind, only 16 words per lane are live at
+// any time, and no load sits in a register waiting to be used.  Meanwhile one lane has two
+// round trips to L2 in flight whose answers are needed a step later: the ticket of the tile
+// to measure next and the offset of the tile to pack next.
 // Packed data goes from registers to the wire image directly: in every region of a PACK tile
 // a lane owns an aligned unit at a lane-strided place, so each warp store is one contiguous
-// sector-aligned run.  Claiming Z before X's offset is known means that, if the scanner is
-// late, this team waits while Z's length is not out yet; with two steps of slack that is
-// rare, and it only delays: the teams that hold earlier tiles never depend on this one.
+// sector-aligned run.  Claiming a tile before the previous offset is known means that, if the
+// scanner is late, this team waits while that tile's length is not out yet; with three steps
+// of slack that is rare, and it only delays: the teams that hold earlier tiles never depend
+// on this one.
 template <int TEAMS>
 __global__ void __launch_bounds__(TEAMS * 256, 1)
 k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restrict__ dirty,
@@ -662,13 +668,31 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
     Smem S = setup_smem(smem, tab);
     const uint32_t team = threadIdx.x / kTeamThreads, tt = threadIdx.x % kTeamThreads;
     const uint32_t warp = tt / 32, lane = tt % 32;
-    EncTeamCtl* tc = reinterpret_cast<EncTeamCtl*>(S.take(TEAMS * kTeamSmemEncode));
+    unsigned char* stage = nullptr;
+    for (int i = 0; i < TEAMS; i++) {          // every thread carves the same blocks in the same order
+        unsigned char* p = S.take(kTeamSmemEncode);
+        if ((uint32_t)i == team) stage = p;
+    }
     if (!S.ok) { if (threadIdx.x == 0) atomicOr(&ws.ctrl->err, 4u); return; }
-    tc += team;
+    EncTeamCtl* tc = reinterpret_cast<EncTeamCtl*>(stage + kTile);
     unsigned char* dir = wire + 64;
     uint16_t* tile_tab = reinterpret_cast<uint16_t*>(wire + 64 + 16ull * g.n_chunks);
-    const uint64_t pol_keep = l2_policy_evict_last();
+    const uint64_t pol_keep = l2_policy_evict_last(), pol_last = l2_policy_evict_first();
+    uint32_t phase = 0;                // parity of the stage's next completion
     auto info = [&](uint32_t t) { return tile_info(g, dirty, t); };
+    // Start the bulk copy of a full tile into the stage (call after a team barrier that
+    // follows the last read of the stage; one thread issues).
+    auto stage_load = [&](const TileInfo& ti, uint64_t policy) {
+        if (tt == 0 && ti.present && ti.full) bulk_load(stage, cache + (uint64_t)ti.t * kTile, kTile, &tc->mbar, policy);
+    };
+    // Wait for it and take this lane's 16 words.
+    auto stage_read = [&](const TileInfo& ti, uint32_t (&d)[kWordsPerLane]) {
+        if (ti.present && ti.full) {
+            if (!mbar_wait(&tc->mbar, phase) && lane == 0) { atomicOr(&ws.ctrl->err, 2u); atomicExch(&ws.ctrl->poison, 1u); }
+            phase ^= 1u;
+            read_staged_words(stage, warp, lane, d);
+        }
+    };
     auto publish_len = [&](uint32_t t, uint32_t len) { st_relaxed_u32(ws.lbk + t, kFlagA | (len / kUnit)); };
 
     // Digest and per-group exponent range of one tile; results go to slot `sl`.  The tile's
@@ -707,13 +731,6 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
             }
         }
     };
-    auto fetch = [&](const TileInfo& ti, uint32_t (&d)[kWordsPerLane]) {       // first read: keep in L2
-        if (ti.present && ti.full) load_tile_words_keep(cache + (uint64_t)ti.t * kTile, warp, lane, d, pol_keep);
-    };
-    auto refetch = [&](const TileInfo& ti, uint32_t (&d)[kWordsPerLane]) {     // second read: last use
-        if (ti.present && ti.full) load_tile_words(cache + (uint64_t)ti.t * kTile, warp, lane, d);
-    };
-
     // Pack tile X (words in d, widths in slot sl) into the wire image at payload offset excl.
     auto pack = [&](const TileInfo& ti, const uint32_t (&d)[kWordsPerLane], uint32_t sl, unsigned long long excl) {
         uint32_t enc_len = 0, entry = 0;
@@ -793,51 +810,61 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
     TileInfo iX = info(0xFFFFFFFFu), iV = iX, iW = iX, iY = iX;
     uint32_t sl = 0;
     uint32_t par = 0;                  // step parity (selects next[] / excl[])
-    uint32_t dP[kWordsPerLane], dM[kWordsPerLane];
+    uint32_t d[kWordsPerLane];
     const bool leader = (warp == 0 && lane == 0);
 
-    // ---- prologue: X, V, W claimed, measured and published one after the other; Y claimed and
-    // loading; X's words requested again for the first pack; X's offset obtained
+    // ---- prologue: X, V, W claimed, measured and published one after the other; Y claimed;
+    // X's offset obtained; X's words requested again for the first pack
     if (tt == 0) {
         for (int i = 0; i < 8; i++) tc->wsum[i] = 0;
+        mbar_init(&tc->mbar, 1);
         tc->next[0] = next_ticket(ws.ctrl);
     }
     team_bar(team);
     iX = info(tc->next[0]);
-    fetch(iX, dM);
-    measure(iX, dM, 0);
+    stage_load(iX, pol_keep);
+    stage_read(iX, d);
+    measure(iX, d, 0);
     if (tt == 0) tc->next[1] = iX.valid ? next_ticket(ws.ctrl) : 0xFFFFFFFFu;
     team_bar(team);
     iV = info(tc->next[1]);
-    fetch(iV, dM);
-    measure(iV, dM, 1);
+    stage_load(iV, pol_keep);
+    stage_read(iV, d);
+    measure(iV, d, 1);
     if (tt == 0) tc->next[0] = iV.valid ? next_ticket(ws.ctrl) : 0xFFFFFFFFu;
     team_bar(team);
     iW = info(tc->next[0]);
-    fetch(iW, dM);
-    measure(iW, dM, 2);
+    stage_load(iW, pol_keep);
+    stage_read(iW, d);
+    measure(iW, d, 2);
+    uint32_t last_tk = 0xFFFFFFFFu;    // leader: the ticket it claimed last
     if (tt == 0) {
-        tc->next[1] = iW.valid ? next_ticket(ws.ctrl) : 0xFFFFFFFFu;
-        tc->excl[0] = iX.valid ? wait_prefix(ws.lbk, iX.t, ws.ctrl) : 0ull;
+        last_tk = iW.valid ? next_ticket(ws.ctrl) : 0xFFFFFFFFu;
+        tc->next[1] = last_tk;
+        tc->excl[1] = iX.valid ? wait_prefix(ws.lbk, iX.t, ws.ctrl) : 0ull;
     }
     team_bar(team);
-    iY = info(tc->next[1]);
-    fetch(iY, dM);
-    refetch(iX, dP);
-    unsigned long long exclX = tc->excl[0];
-    team_bar(team);
+    stage_load(iX, pol_last);          // X again, for the first pack
+    // from here on: next[par^1] / excl[par^1] hold what the previous step prepared
 
     while (iX.valid) {
-        // two round trips to L2 whose answers are used at the end of the step: the ticket of
-        // the tile to load next, and the offset of the tile to pack in the next step
+        // two round trips to L2 whose answers are used in the next step: the ticket of the tile
+        // to measure then, and the offset of the tile to pack then
         uint32_t pv = 0, tk = 0xFFFFFFFFu;
         if (leader) {
             if (iV.valid) pv = ld_relaxed_u32(ws.lbk + iV.t);
-            if (iY.valid) tk = next_ticket(ws.ctrl);
+            if (last_tk < g.n_tiles) tk = next_ticket(ws.ctrl);
         }
-        pack(iX, dP, sl, exclX);
-        refetch(iV, dP);                                              // V's words again, for the next pack
-        measure(iY, dM, (sl + 3u) & 7u);
+        stage_read(iX, d);
+        team_bar(team);                   // stage free; what the leader left at the end of the last step is visible
+        iY = info(tc->next[par ^ 1u]);
+        const unsigned long long exclX = tc->excl[par ^ 1u];
+        stage_load(iY, pol_keep);
+        pack(iX, d, sl, exclX);
+        stage_read(iY, d);
+        team_bar(team);                                               // stage free
+        stage_load(iV, pol_last);
+        measure(iY, d, (sl + 3u) & 7u);
         if (leader) {
 #ifdef WM_DEBUG_COUNTERS
             atomicAdd(&ws.ctrl->pad[(pv >> 30) == 2u ? 3 : 2], 1u);
@@ -847,12 +874,9 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
                 e = (pv >> 30) == 2u ? (unsigned long long)(pv & kValMask) * kUnit : wait_prefix(ws.lbk, iV.t, ws.ctrl);
             tc->excl[par] = e;
             tc->next[par] = tk;
+            last_tk = tk;
         }
-        team_bar(team);            // offset and ticket visible; every warp is done with this step's slots
-        const TileInfo iZ = info(tc->next[par]);
-        fetch(iZ, dM);                                                // dM is free: Y has been measured
-        exclX = tc->excl[par];
-        iX = iV; iV = iW; iW = iY; iY = iZ;
+        iX = iV; iV = iW; iW = iY;
         sl = (sl + 1u) & 7u;
         par ^= 1u;
     }
