@@ -25,9 +25,10 @@ namespace wm {
 constexpr uint32_t kTile = 16384;
 constexpr uint32_t kTeamThreads = 256;
 constexpr uint32_t kWordsPerLane = 16;
-// Dynamic shared memory every table-using kernel asks for: the 144 KiB image plus 64 KiB
-// that the 64 KiB alignment splits into a part below and a part above the image.
-constexpr uint32_t kDynSmem = kImgBytes + 0x10000;
+// Dynamic shared memory every table-using kernel asks for: the 144 KiB image plus 79 KiB
+// that the 64 KiB alignment splits into a part below and a part above the image (with the
+// window starting at 1 KiB: 63 KiB below, 16 KiB above).  227 KiB is the per-block maximum.
+constexpr uint32_t kDynSmem = kImgBytes + 0x10000 + 0x3C00;
 
 struct Smem {
     uint32_t L01, L23, LNK;      // shared-window address of A01 / A23 / NK, or'ed with lane*4

@@ -670,11 +670,12 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
     const uint32_t warp = tt / 32, lane = tt % 32;
     unsigned char* stage = nullptr;
     for (int i = 0; i < TEAMS; i++) {          // every thread carves the same blocks in the same order
-        unsigned char* p = S.take(kTeamSmemEncode);
+        unsigned char* p = S.take(kTile);
         if ((uint32_t)i == team) stage = p;
     }
+    EncTeamCtl* tc = reinterpret_cast<EncTeamCtl*>(S.take(TEAMS * sizeof(EncTeamCtl)));
     if (!S.ok) { if (threadIdx.x == 0) atomicOr(&ws.ctrl->err, 4u); return; }
-    EncTeamCtl* tc = reinterpret_cast<EncTeamCtl*>(stage + kTile);
+    tc += team;
     unsigned char* dir = wire + 64;
     uint16_t* tile_tab = reinterpret_cast<uint16_t*>(wire + 64 + 16ull * g.n_chunks);
     const uint64_t pol_keep = l2_policy_evict_last(), pol_last = l2_policy_evict_first();
@@ -1195,7 +1196,7 @@ k_decode_struct_scan(const unsigned char* __restrict__ wire, uint64_t wire_len, 
     }
 }
 
-struct DecSlot {                 // what thread 0 prepares for a tile one iteration ahead
+struct DecSlot {                 // what thread 0 prepares for a tile ahead of its turn
     uint32_t t;                  // tile (>= n_tiles: none left)
     uint32_t entry;              // tile table entry
     uint32_t c;                  // chunk
@@ -1205,39 +1206,30 @@ struct DecSlot {                 // what thread 0 prepares for a tile one iterat
 };
 struct DecTeamCtl {
     uint32_t wdig[2][8];
-    DecSlot slot[2];
+    DecSlot slot[4];             // ring: slot i & 3 belongs to the team's i-th tile
+    unsigned long long mbar;     // completion of the bulk copy into the team's stage
+    unsigned long long pad;
 };
 static_assert(sizeof(DecTeamCtl) % 16 == 0, "team control block keeps 16-byte alignment");
 
-__device__ __forceinline__ uint32_t ldg_u8(const void* p)
-{
-    uint32_t v;
-    asm volatile("ld.global.nc.u8 %0, [%1];" : "=r"(v) : "l"(p));
-    return v;
-}
-__device__ __forceinline__ uint32_t ldg_u16(const void* p)
-{
-    unsigned short v;
-    asm volatile("ld.global.nc.u16 %0, [%1];" : "=h"(v) : "l"(p));
-    return v;
-}
+// The plane words of one group as stored (aligned per-lane units, see pack_group_planes):
+// a = the 4-bit plane's word or the low half of an 8-bit plane; b = the 2-bit plane's 16 bits
+// in the low half and the 1-bit plane's byte in bits 16-23, or the high half of an 8-bit plane.
+struct PlaneWords { uint32_t a, b; };
 
-// The raw plane words of one group, as loaded (aligned per-lane units, see pack_group_planes).
-struct PlaneWords { uint32_t p4, p2, p1, p8lo, p8hi; };
-
-__device__ __forceinline__ PlaneWords load_group_planes(const unsigned char* rec, uint32_t wd, uint32_t lane)
+__device__ __forceinline__ PlaneWords read_group_planes(const unsigned char* rec, uint32_t wd, uint32_t lane)
 {
     PlaneWords pw;
-    pw.p4 = pw.p2 = pw.p1 = pw.p8lo = pw.p8hi = 0;
+    pw.a = 0; pw.b = 0;
     if (wd == 8u) {
         const uint2 v = *reinterpret_cast<const uint2*>(rec + 8 * lane);
-        pw.p8lo = v.x; pw.p8hi = v.y;
+        pw.a = v.x; pw.b = v.y;
         return pw;
     }
     const unsigned char* p = rec;
-    if (wd & 4u) { pw.p4 = *reinterpret_cast<const uint32_t*>(p + 4 * lane); p += 128; }
-    if (wd & 2u) { pw.p2 = ldg_u16(p + 2 * lane); p += 64; }
-    if (wd & 1u) { pw.p1 = ldg_u8(p + lane); }
+    if (wd & 4u) { pw.a = *reinterpret_cast<const uint32_t*>(p + 4 * lane); p += 128; }
+    if (wd & 2u) { pw.b = *reinterpret_cast<const uint16_t*>(p + 2 * lane); p += 64; }
+    if (wd & 1u) { pw.b |= (uint32_t)p[lane] << 16; }
     return pw;
 }
 
@@ -1246,25 +1238,25 @@ template <int W>
 __device__ __forceinline__ void unpack_group_planes(const PlaneWords& pw, uint32_t base, uint32_t& ea, uint32_t& eb)
 {
     uint32_t da = 0, db = 0;
-    if (W == 8) { da = pw.p8lo; db = pw.p8hi; }
+    if (W == 8) { da = pw.a; db = pw.b; }
     else {
         int sh = 0;
         if (W & 4) {
-            const uint32_t t = __byte_perm(pw.p4, 0, 0x1100), u = __byte_perm(pw.p4, 0, 0x3322);
+            const uint32_t t = __byte_perm(pw.a, 0, 0x1100), u = __byte_perm(pw.a, 0, 0x3322);
             da = (t & 0x000F000Fu) | ((t >> 4) & 0x0F000F00u);
             db = (u & 0x000F000Fu) | ((u >> 4) & 0x0F000F00u);
             sh = 4;
         }
         if (W & 2) {        // byte -> four 2-bit fields, one per byte
-            uint32_t xa = pw.p2 & 0xFFu, xb = (pw.p2 >> 8) & 0xFFu;
+            uint32_t xa = pw.b & 0xFFu, xb = (pw.b >> 8) & 0xFFu;
             xa = (xa * 0x1001u) & 0x000F000Fu; xa = (xa * 0x41u) & 0x03030303u;
             xb = (xb * 0x1001u) & 0x000F000Fu; xb = (xb * 0x41u) & 0x03030303u;
             da |= xa << sh; db |= xb << sh;
             sh += 2;
         }
         if (W & 1) {        // nibble -> four bits, one per byte
-            const uint32_t xa = ((pw.p1 & 0xFu) * 0x00204081u) & 0x01010101u;
-            const uint32_t xb = (((pw.p1 >> 4) & 0xFu) * 0x00204081u) & 0x01010101u;
+            const uint32_t xa = (((pw.b >> 16) & 0xFu) * 0x00204081u) & 0x01010101u;
+            const uint32_t xb = (((pw.b >> 20) & 0xFu) * 0x00204081u) & 0x01010101u;
             da |= xa << sh; db |= xb << sh;
         }
     }
@@ -1277,16 +1269,12 @@ __device__ __forceinline__ void unpack_group_planes(const PlaneWords& pw, uint32
     }
 }
 
-__device__ __forceinline__ uint32_t ldg_u32(const void* p)
-{
-    uint32_t v;
-    asm volatile("ld.global.nc.u32 %0, [%1];" : "=r"(v) : "l"(p));
-    return v;
-}
-
-// Unpack + checksum of the decoded bytes.  Tiles are claimed by ticket; thread 0 of a team
-// looks up the next tile's table entry and source offset while the team decodes the current
-// one, so that chain of dependent loads is off the critical path.
+// Unpack + checksum of the decoded bytes.  Tiles are claimed by ticket.  The team owns one
+// 16 KiB stage in shared memory; the encoded tile arrives there by one bulk copy (TMA) that is
+// started a tile ahead, each lane takes what it needs (descriptors, its 8 sign-mantissa bytes
+// and its plane words per group: at most 16 words) into registers, and the stage is handed to
+// the next copy while the team unpacks, stores and checksums.  Thread 0 looks up the table
+// entry and source offset two tiles ahead, so that chain of dependent loads is hidden too.
 template <int TEAMS>
 __global__ void __launch_bounds__(TEAMS * 256, 1)
 k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restrict__ dst, Ws ws,
@@ -1297,6 +1285,11 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
     Smem S = setup_smem(smem, tab);
     const uint32_t team = threadIdx.x / kTeamThreads, tt = threadIdx.x % kTeamThreads;
     const uint32_t warp = tt / 32, lane = tt % 32;
+    unsigned char* stage = nullptr;
+    for (int i = 0; i < TEAMS; i++) {          // every thread carves the same blocks in the same order
+        unsigned char* p = S.take(kTile);
+        if ((uint32_t)i == team) stage = p;
+    }
     DecTeamCtl* tc = reinterpret_cast<DecTeamCtl*>(S.take(TEAMS * sizeof(DecTeamCtl)));
     if (!S.ok) { if (threadIdx.x == 0) atomicOr(&ws.ctrl->err, 4u); return; }
     tc += team;
@@ -1314,88 +1307,112 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
             sl->src = e ? *reinterpret_cast<const unsigned long long*>(dir + 16ull * c) + ws.rel[t] : 0ull;
         }
     };
+    // staged tiles: full RAW and PACK tiles (everything except absent tiles and the ragged tail)
+    auto staged = [&](const DecSlot& sl) { return sl.t < g.n_tiles && sl.entry >= 258u && sl.entry <= 512u; };
+    auto start_copy = [&](const DecSlot& sl) {   // thread 0 only
+        if (staged(sl)) bulk_load(stage, payload + sl.src, 32u * sl.entry, &tc->mbar, 0);
+    };
 
-    if (tt == 0) prepare(&tc->slot[0]);
+    if (tt == 0) {
+        mbar_init(&tc->mbar, 1);
+        prepare(&tc->slot[0]);
+        prepare(&tc->slot[1]);
+        start_copy(tc->slot[0]);
+    }
     team_bar(team);
-    uint32_t p = 0;
-    while (true) {
-        const DecSlot sl = tc->slot[p];
+    uint32_t phase = 0;
+    for (uint32_t it = 0;; it++) {
+        const DecSlot sl = tc->slot[it & 3u];
         const uint32_t t = sl.t;
         if (t >= g.n_tiles) break;
-        if (tt == 0) prepare(&tc->slot[p ^ 1u]);
         const uint32_t e = sl.entry;
         const bool first = sl.first != 0;
-        bool have_digest = false;
-        if (e != 0) {
-            const unsigned char* src = payload + sl.src;
-            unsigned char* o = dst + (uint64_t)t * kTile;
-            uint32_t w[kWordsPerLane];
-            bool fold = first;
-            bool decoded = true;
-            if (e == 0xFFFFu) {
-                const uint32_t len = g.tail_len;
-                for (uint32_t i = tt; i < len; i += kTeamThreads) o[i] = src[i];
-                load_tile_words_guarded(src, len, first, warp, lane, w);
-                fold = false;
-            } else if (e == 512u) {
-                load_tile_words(src, warp, lane, w);
+        const uint32_t p = it & 1u;
+        bool have_digest = false, decoded = true, fold = first;
+        uint32_t w[kWordsPerLane];
+        uint32_t desc = 0, incl = 0, wv = 0;
+        uint2 sm[4];
+        PlaneWords pw[4];
+        const bool is_pack = e >= 258u && e < 512u;
+
+        // ---- phase 1: everything this lane needs from the stage goes into registers
+        if (staged(sl)) {
+            if (!mbar_wait(&tc->mbar, phase) && lane == 0) { atomicOr(&ws.ctrl->err, 2u); }
+            phase ^= 1u;
+            if (!is_pack) {
+                read_staged_words(stage, warp, lane, w);
             } else {
-                // PACK tile: validate the 32 descriptors (every warp does; the verdict is uniform)
-                const uint32_t desc = reinterpret_cast<const uint16_t*>(src)[lane];
-                const uint32_t base_l = desc & 0xFFu, wv = (desc >> 8) & 15u, chk = desc >> 12;
+                desc = reinterpret_cast<const uint16_t*>(stage)[lane];
+                wv = (desc >> 8) & 15u;
+                const uint32_t base_l = desc & 0xFFu, chk = desc >> 12;
                 const bool bad = wv > 8u || chk != (((base_l & 15u) ^ (base_l >> 4) ^ wv ^ 5u) & 15u);
                 const bool anybad = __any_sync(0xFFFFFFFFu, bad);
-                uint32_t incl = wv;
+                incl = wv;
 #pragma unroll
-                for (int d = 1; d < 32; d <<= 1) {
-                    const uint32_t o2 = __shfl_up_sync(0xFFFFFFFFu, incl, d);
-                    if (lane >= (uint32_t)d) incl += o2;
+                for (int k = 1; k < 32; k <<= 1) {
+                    const uint32_t o2 = __shfl_up_sync(0xFFFFFFFFu, incl, k);
+                    if (lane >= (uint32_t)k) incl += o2;
                 }
                 const uint32_t Ssum = __shfl_sync(0xFFFFFFFFu, incl, 31);
                 const int verdict = anybad ? 1 : (258u + Ssum != e ? 2 : 0);
-                if (verdict) {
+                if (verdict) {               // every warp reaches the same verdict
                     decoded = false;
                     if (tt == 0) {
                         atomicMin(&ws.ctrl->bad4_key, (unsigned long long)t * 2ull + (verdict == 2 ? 1ull : 0ull));
                         atomicOr(&ws.cflag[sl.c], CF_BAD4);
                     }
                 } else {
-                    // issue every load of the warp's four groups, then unpack
-                    uint2 sm[4];
-                    PlaneWords pw[4];
-                    uint32_t dgv[4];
 #pragma unroll
                     for (int j = 0; j < 4; j++) {
                         const uint32_t gi = 4 * warp + j;
-                        dgv[j] = __shfl_sync(0xFFFFFFFFu, desc, gi);
+                        const uint32_t dg = __shfl_sync(0xFFFFFFFFu, desc, gi);
                         const uint32_t exg = __shfl_sync(0xFFFFFFFFu, incl - wv, gi);
-                        sm[j] = *reinterpret_cast<const uint2*>(src + 64 + 256 * gi + 8 * lane);
-                        pw[j] = load_group_planes(src + 8256 + 32 * exg, (dgv[j] >> 8) & 15u, lane);
+                        sm[j] = *reinterpret_cast<const uint2*>(stage + 64 + 256 * gi + 8 * lane);
+                        pw[j] = read_group_planes(stage + 8256 + 32 * exg, (dg >> 8) & 15u, lane);
                     }
+                }
+            }
+        }
+        team_bar(team);                      // stage free; slot[it+1] (prepared last step) visible
+        if (tt == 0) {
+            start_copy(tc->slot[(it + 1u) & 3u]);
+            prepare(&tc->slot[(it + 2u) & 3u]);
+        }
+
+        // ---- phase 2: unpack, store, checksum
+        if (e != 0) {
+            unsigned char* o = dst + (uint64_t)t * kTile;
+            if (e == 0xFFFFu) {
+                const unsigned char* src = payload + sl.src;
+                const uint32_t len = g.tail_len;
+                for (uint32_t i = tt; i < len; i += kTeamThreads) o[i] = src[i];
+                load_tile_words_guarded(src, len, first, warp, lane, w);
+                fold = false;
+            } else if (is_pack && decoded) {
 #pragma unroll
-                    for (int j = 0; j < 4; j++) {
-                        const uint32_t base = dgv[j] & 0xFFu, wd = (dgv[j] >> 8) & 15u;
-                        uint32_t ea = base * 0x01010101u, eb = ea;
-                        switch (wd) {          // uniform across the warp
-                            case 1: unpack_group_planes<1>(pw[j], base, ea, eb); break;
-                            case 2: unpack_group_planes<2>(pw[j], base, ea, eb); break;
-                            case 3: unpack_group_planes<3>(pw[j], base, ea, eb); break;
-                            case 4: unpack_group_planes<4>(pw[j], base, ea, eb); break;
-                            case 5: unpack_group_planes<5>(pw[j], base, ea, eb); break;
-                            case 6: unpack_group_planes<6>(pw[j], base, ea, eb); break;
-                            case 7: unpack_group_planes<7>(pw[j], base, ea, eb); break;
-                            case 8: unpack_group_planes<8>(pw[j], base, ea, eb); break;
-                            default: break;
-                        }
-                        uint32_t Tr[4];
-                        Tr[0] = __byte_perm(sm[j].x, ea, 0x5140);
-                        Tr[1] = __byte_perm(sm[j].x, ea, 0x7362);
-                        Tr[2] = __byte_perm(sm[j].y, eb, 0x5140);
-                        Tr[3] = __byte_perm(sm[j].y, eb, 0x7362);
-#pragma unroll
-                        for (int r = 0; r < 4; r++)
-                            w[4 * j + r] = ((Tr[r] >> 1) & 0x7FFF7FFFu) | ((Tr[r] << 15) & 0x80008000u);
+                for (int j = 0; j < 4; j++) {
+                    const uint32_t dg = __shfl_sync(0xFFFFFFFFu, desc, 4 * warp + j);
+                    const uint32_t base = dg & 0xFFu, wd = (dg >> 8) & 15u;
+                    uint32_t ea = base * 0x01010101u, eb = ea;
+                    switch (wd) {          // uniform across the warp
+                        case 1: unpack_group_planes<1>(pw[j], base, ea, eb); break;
+                        case 2: unpack_group_planes<2>(pw[j], base, ea, eb); break;
+                        case 3: unpack_group_planes<3>(pw[j], base, ea, eb); break;
+                        case 4: unpack_group_planes<4>(pw[j], base, ea, eb); break;
+                        case 5: unpack_group_planes<5>(pw[j], base, ea, eb); break;
+                        case 6: unpack_group_planes<6>(pw[j], base, ea, eb); break;
+                        case 7: unpack_group_planes<7>(pw[j], base, ea, eb); break;
+                        case 8: unpack_group_planes<8>(pw[j], base, ea, eb); break;
+                        default: break;
                     }
+                    uint32_t Tr[4];
+                    Tr[0] = __byte_perm(sm[j].x, ea, 0x5140);
+                    Tr[1] = __byte_perm(sm[j].x, ea, 0x7362);
+                    Tr[2] = __byte_perm(sm[j].y, eb, 0x5140);
+                    Tr[3] = __byte_perm(sm[j].y, eb, 0x7362);
+#pragma unroll
+                    for (int r = 0; r < 4; r++)
+                        w[4 * j + r] = ((Tr[r] >> 1) & 0x7FFF7FFFu) | ((Tr[r] << 15) & 0x80008000u);
                 }
             }
             if (decoded) {
@@ -1409,9 +1426,8 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
                 have_digest = true;
             }
         }
-        team_bar(team);                                               // slot[p^1] and wdig[p] visible
+        team_bar(team);                      // wdig[p] complete; thread 0's slot writes visible
         if (tt == 0 && have_digest) ws.dig[t] = xor8(tc->wdig[p]);
-        p ^= 1u;
     }
 }
 
