@@ -238,8 +238,16 @@ __device__ uint32_t combine_chunk_crcs(const Geo& g, const uint32_t* crc, uint32
 
 // ------------------------------------------------------------------ wm_checksum
 
-// Tile digests of the whole cache: static striding over tiles, next tile's words prefetched
-// into registers while the current one is digested; one team barrier per tile.
+// Tile digests of the whole cache: static striding over tiles.  Each team owns one 16 KiB stage
+// that bulk copies (TMA) fill; the team takes its 16 words per lane out of the stage, hands
+// the stage to the copy of its next tile and digests from registers meanwhile.
+struct DigTeamCtl {
+    uint32_t wdig[2][8];
+    unsigned long long mbar;
+    unsigned long long pad;
+};
+static_assert(sizeof(DigTeamCtl) % 16 == 0, "team control block keeps 16-byte alignment");
+
 template <int TEAMS>
 __global__ void __launch_bounds__(TEAMS * 256, 1)
 k_tile_digests(const unsigned char* __restrict__ cache, Geo g, Ws ws, const Tables* __restrict__ tab)
@@ -248,38 +256,44 @@ k_tile_digests(const unsigned char* __restrict__ cache, Geo g, Ws ws, const Tabl
     Smem S = setup_smem(smem, tab);
     const uint32_t team = threadIdx.x / kTeamThreads, tt = threadIdx.x % kTeamThreads;
     const uint32_t warp = tt / 32, lane = tt % 32;
-    TeamCtl* tc = reinterpret_cast<TeamCtl*>(S.take(TEAMS * sizeof(TeamCtl)));
+    unsigned char* stage = nullptr;
+    for (int i = 0; i < TEAMS; i++) {          // every thread carves the same blocks in the same order
+        unsigned char* p = S.take(kTile);
+        if ((uint32_t)i == team) stage = p;
+    }
+    DigTeamCtl* tc = reinterpret_cast<DigTeamCtl*>(S.take(TEAMS * sizeof(DigTeamCtl)));
     if (!S.ok) { if (threadIdx.x == 0) atomicOr(&ws.ctrl->err, 4u); return; }
     tc += team;
     const uint64_t stride = (uint64_t)gridDim.x * TEAMS;
-    uint64_t t = (uint64_t)blockIdx.x * TEAMS + team;
-    uint32_t par = 0;
-
-    auto fetch = [&](uint64_t tile, uint32_t (&d)[kWordsPerLane]) {
-        if (tile < g.n_tiles && g.nbytes - tile * kTile >= kTile) load_tile_words(cache + tile * kTile, warp, lane, d);
+    const uint64_t pol = l2_policy_evict_first();
+    auto full = [&](uint64_t tile) { return tile < g.n_tiles && g.nbytes - tile * kTile >= kTile; };
+    auto start_copy = [&](uint64_t tile) {     // thread 0 only
+        if (full(tile)) bulk_load(stage, cache + tile * kTile, kTile, &tc->mbar, pol);
     };
-    auto process = [&](uint64_t tile, uint32_t (&d)[kWordsPerLane]) {
-        const uint64_t left = g.nbytes - tile * kTile;
-        const bool first = first_in_chunk(g, (uint32_t)tile);
-        const bool full = left >= kTile;
-        if (!full) load_tile_words_guarded(cache + tile * kTile, (uint32_t)left, first, warp, lane, d);
-        const uint32_t v = tile_digest_part(S, d, first && full, warp, lane);
+
+    uint64_t t = (uint64_t)blockIdx.x * TEAMS + team;
+    if (tt == 0) { mbar_init(&tc->mbar, 1); start_copy(t); }
+    team_bar(team);
+    uint32_t phase = 0, par = 0;
+    for (; t < g.n_tiles; t += stride) {
+        const bool first = first_in_chunk(g, (uint32_t)t);
+        uint32_t d[kWordsPerLane];
+        bool fold = first;
+        if (full(t)) {
+            if (!mbar_wait(&tc->mbar, phase) && lane == 0) atomicOr(&ws.ctrl->err, 2u);
+            phase ^= 1u;
+            read_staged_words(stage, warp, lane, d);
+        } else {
+            load_tile_words_guarded(cache + t * kTile, (uint32_t)(g.nbytes - t * kTile), first, warp, lane, d);
+            fold = false;
+        }
+        team_bar(team);                          // stage free; wdig[par] of two tiles ago consumed
+        if (tt == 0) start_copy(t + stride);
+        const uint32_t v = tile_digest_part(S, d, fold, warp, lane);
         if (lane == 0) tc->wdig[par][warp] = v;
         team_bar(team);
-        if (tt == 0) ws.dig[tile] = xor8(tc->wdig[par]);
+        if (tt == 0) ws.dig[t] = xor8(tc->wdig[par]);
         par ^= 1u;
-    };
-
-    uint32_t da[kWordsPerLane], db[kWordsPerLane];
-    fetch(t, da);
-    while (t < g.n_tiles) {
-        fetch(t + stride, db);
-        process(t, da);
-        t += stride;
-        if (t >= g.n_tiles) break;
-        fetch(t + stride, da);
-        process(t, db);
-        t += stride;
     }
 }
 
