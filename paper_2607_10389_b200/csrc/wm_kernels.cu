@@ -822,7 +822,10 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
 
     // Tiles in flight, oldest first: X (packed in this step), V, W (waiting for their offsets),
     // Y (measured in this step).  Ring slots: X = sl, V = sl+1, W = sl+2, Y = sl+3 (mod 8).
-    TileInfo iX = info(0xFFFFFFFFu), iV = iX, iW = iX, iY = iX;
+    // Only the tile numbers are carried from step to step (0xFFFFFFFF: none); what follows from
+    // a number (chunk, full / ragged, present) is worked out where it is used.
+    constexpr uint32_t kNone = 0xFFFFFFFFu;
+    uint32_t tX = kNone, tV = kNone, tW = kNone, tY = kNone;
     uint32_t sl = 0;
     uint32_t par = 0;                  // step parity (selects next[] / excl[])
     uint32_t d[kWordsPerLane];
@@ -836,62 +839,62 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
         tc->next[0] = next_ticket(ws.ctrl);
     }
     team_bar(team);
-    iX = info(tc->next[0]);
-    stage_load(iX, pol_keep);
-    stage_read(iX, d);
-    measure(iX, d, 0);
-    if (tt == 0) tc->next[1] = iX.valid ? next_ticket(ws.ctrl) : 0xFFFFFFFFu;
+    tX = tc->next[0];
+    { const TileInfo i = info(tX); stage_load(i, pol_keep); stage_read(i, d); measure(i, d, 0); }
+    if (tt == 0) tc->next[1] = tX < g.n_tiles ? next_ticket(ws.ctrl) : kNone;
     team_bar(team);
-    iV = info(tc->next[1]);
-    stage_load(iV, pol_keep);
-    stage_read(iV, d);
-    measure(iV, d, 1);
-    if (tt == 0) tc->next[0] = iV.valid ? next_ticket(ws.ctrl) : 0xFFFFFFFFu;
+    tV = tc->next[1];
+    { const TileInfo i = info(tV); stage_load(i, pol_keep); stage_read(i, d); measure(i, d, 1); }
+    if (tt == 0) tc->next[0] = tV < g.n_tiles ? next_ticket(ws.ctrl) : kNone;
     team_bar(team);
-    iW = info(tc->next[0]);
-    stage_load(iW, pol_keep);
-    stage_read(iW, d);
-    measure(iW, d, 2);
-    uint32_t last_tk = 0xFFFFFFFFu;    // leader: the ticket it claimed last
+    tW = tc->next[0];
+    { const TileInfo i = info(tW); stage_load(i, pol_keep); stage_read(i, d); measure(i, d, 2); }
+    uint32_t last_tk = kNone;          // leader: the ticket it claimed last
     if (tt == 0) {
-        last_tk = iW.valid ? next_ticket(ws.ctrl) : 0xFFFFFFFFu;
+        last_tk = tW < g.n_tiles ? next_ticket(ws.ctrl) : kNone;
         tc->next[1] = last_tk;
-        tc->excl[1] = iX.valid ? wait_prefix(ws.lbk, iX.t, ws.ctrl) : 0ull;
+        tc->excl[1] = tX < g.n_tiles ? wait_prefix(ws.lbk, tX, ws.ctrl) : 0ull;
     }
     team_bar(team);
-    stage_load(iX, pol_last);          // X again, for the first pack
+    stage_load(info(tX), pol_last);    // X again, for the first pack
     // from here on: next[par^1] / excl[par^1] hold what the previous step prepared
 
-    while (iX.valid) {
+    while (tX < g.n_tiles) {
         // two round trips to L2 whose answers are used in the next step: the ticket of the tile
         // to measure then, and the offset of the tile to pack then
-        uint32_t pv = 0, tk = 0xFFFFFFFFu;
+        uint32_t pv = 0, tk = kNone;
         if (leader) {
-            if (iV.valid) pv = ld_relaxed_u32(ws.lbk + iV.t);
+            if (tV < g.n_tiles) pv = ld_relaxed_u32(ws.lbk + tV);
             if (last_tk < g.n_tiles) tk = next_ticket(ws.ctrl);
         }
-        stage_read(iX, d);
-        team_bar(team);                   // stage free; what the leader left at the end of the last step is visible
-        iY = info(tc->next[par ^ 1u]);
-        const unsigned long long exclX = tc->excl[par ^ 1u];
-        stage_load(iY, pol_keep);
-        pack(iX, d, sl, exclX);
-        stage_read(iY, d);
-        team_bar(team);                                               // stage free
-        stage_load(iV, pol_last);
-        measure(iY, d, (sl + 3u) & 7u);
+        {
+            const TileInfo iX = info(tX);
+            stage_read(iX, d);
+            team_bar(team);               // stage free; what the leader left at the end of the last step is visible
+            tY = tc->next[par ^ 1u];
+            const unsigned long long exclX = tc->excl[par ^ 1u];
+            stage_load(info(tY), pol_keep);
+            pack(iX, d, sl, exclX);
+        }
+        {
+            const TileInfo iY = info(tY);
+            stage_read(iY, d);
+            team_bar(team);                                           // stage free
+            stage_load(info(tV), pol_last);
+            measure(iY, d, (sl + 3u) & 7u);
+        }
         if (leader) {
 #ifdef WM_DEBUG_COUNTERS
             atomicAdd(&ws.ctrl->pad[(pv >> 30) == 2u ? 3 : 2], 1u);
 #endif
             unsigned long long e = 0;
-            if (iV.valid)
-                e = (pv >> 30) == 2u ? (unsigned long long)(pv & kValMask) * kUnit : wait_prefix(ws.lbk, iV.t, ws.ctrl);
+            if (tV < g.n_tiles)
+                e = (pv >> 30) == 2u ? (unsigned long long)(pv & kValMask) * kUnit : wait_prefix(ws.lbk, tV, ws.ctrl);
             tc->excl[par] = e;
             tc->next[par] = tk;
             last_tk = tk;
         }
-        iX = iV; iV = iW; iW = iY;
+        tX = tV; tV = tW; tW = tY;
         sl = (sl + 1u) & 7u;
         par ^= 1u;
     }
@@ -1514,7 +1517,7 @@ k_decode_finish(const unsigned char* __restrict__ wire, uint64_t wire_len, Geo g
 // ------------------------------------------------------------------ host side
 
 #ifndef WM_TEAMS
-#define WM_TEAMS 3
+#define WM_TEAMS 4
 #endif
 constexpr int kTeams = WM_TEAMS;            // encode: teams per block (plus the scanner warp)
 #ifndef WM_TEAMS_PLAIN
