@@ -37,6 +37,7 @@ struct Geo {
     uint32_t k_last_chunk;    // x^(8 last_chunk_len)
     uint32_t n_meta_slices;   // ceil(meta_end / 16384)
     uint32_t tpc_shift;       // log2(tiles_per_chunk) when that is a power of two, else 32
+    uint32_t n_full_tiles;    // tiles of exactly 16384 bytes
 };
 
 struct Ctrl {                 // first 256 bytes of the workspace
@@ -123,6 +124,7 @@ static bool make_geo(uint64_t nbytes, uint32_t chunk_bytes, Geo& g)
     g.k_chunk = x_pow_bytes(chunk_bytes);
     g.k_last_chunk = x_pow_bytes(g.last_chunk_len);
     g.n_meta_slices = (uint32_t)((g.meta_end + kTile - 1) / kTile);
+    g.n_full_tiles = (uint32_t)(nbytes / kTile);
     g.tpc_shift = 32;
     for (uint32_t k = 0; k < 32; k++)
         if (g.tiles_per_chunk == (1u << k)) g.tpc_shift = k;
@@ -548,10 +550,12 @@ __device__ __forceinline__ uint32_t desc_of(uint32_t base, uint32_t w)
 }
 
 struct EncTeamCtl {
-    uint32_t wtab[8][32];   // per group: base | w << 8 (a ring of slots: one per tile in flight and
-                            // spares, so that a slot is rewritten long after its last read)
+    uint32_t wtab[8][32];   // per group: base | w << 8 | (sum of the widths before it) << 16 (a ring of
+                            // slots: one per tile in flight and spares, so that a slot is rewritten
+                            // long after its last read)
     uint32_t wdig[8][8];    // per warp: its contribution to the tile digest
     uint32_t wsum[8];       // sum of widths so far | warps arrived << 16 (the last warp publishes)
+    uint32_t ssum[8];       // sum of the 32 widths of the slot's tile (set by that last warp)
     uint32_t next[2];       // ticket claimed in this step (>= n_tiles: none left), by step parity
     uint32_t pad[2];
     unsigned long long excl[2];   // offset of the tile packed in the next step, by step parity
@@ -562,30 +566,32 @@ static_assert(sizeof(EncTeamCtl) % 16 == 0, "team control block keeps 16-byte al
 constexpr uint32_t kTeamSmemEncode = kTile + sizeof(EncTeamCtl);   // one 16 KiB stage + control
 
 struct TileInfo {
-    uint32_t t, c, left;
+    uint32_t t, c;
     bool valid, present, full, first;
 };
 
+__device__ __forceinline__ uint32_t tile_left(const Geo& g, uint32_t t)      // bytes of a ragged tile
+{
+    return (uint32_t)(g.nbytes - (uint64_t)t * kTile);
+}
+
+template <bool MASKED>
 __device__ __forceinline__ TileInfo tile_info(const Geo& g, const uint8_t* __restrict__ dirty, uint32_t t)
 {
     TileInfo ti;
     ti.t = t;
     ti.valid = t < g.n_tiles;
-    ti.present = false; ti.full = false; ti.first = false; ti.c = 0; ti.left = 0;
-    if (!ti.valid) return ti;
+    ti.full = t < g.n_full_tiles;
     ti.c = chunk_of(g, t);
     ti.first = first_in_chunk(g, t);
-    ti.present = !dirty || dirty[ti.c] != 0;
-    const uint64_t left = g.nbytes - (uint64_t)t * kTile;
-    ti.full = left >= kTile;
-    ti.left = ti.full ? kTile : (uint32_t)left;
+    ti.present = ti.valid && (!MASKED || dirty[ti.valid ? ti.c : 0] != 0);
     return ti;
 }
 
-__device__ __forceinline__ uint32_t encoded_len(const TileInfo& ti, uint32_t S)
+__device__ __forceinline__ uint32_t encoded_len(const Geo& g, const TileInfo& ti, uint32_t S)
 {
     if (!ti.present) return 0;
-    if (!ti.full) return ti.left;
+    if (!ti.full) return tile_left(g, ti.t);
     return S <= 253u ? 8256u + 32u * S : kTile;
 }
 
@@ -663,7 +669,7 @@ __device__ __forceinline__ void pack_group_planes(uint32_t e4a, uint32_t e4b, ui
 // scanner is late, this team waits while that tile's length is not out yet; with three steps
 // of slack that is rare, and it only delays: the teams that hold earlier tiles never depend
 // on this one.
-template <int TEAMS>
+template <int TEAMS, bool MASKED>
 __global__ void __launch_bounds__(TEAMS * 256, 1)
 k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restrict__ dirty,
          unsigned char* __restrict__ wire, uint64_t wire_cap, Ws ws, const Tables* __restrict__ tab)
@@ -694,7 +700,7 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
     uint16_t* tile_tab = reinterpret_cast<uint16_t*>(wire + 64 + 16ull * g.n_chunks);
     const uint64_t pol_keep = l2_policy_evict_last(), pol_last = l2_policy_evict_first();
     uint32_t phase = 0;                // parity of the stage's next completion
-    auto info = [&](uint32_t t) { return tile_info(g, dirty, t); };
+    auto info = [&](uint32_t t) { return tile_info<MASKED>(g, dirty, t); };
     // Start the bulk copy of a full tile into the stage (call after a team barrier that
     // follows the last read of the stage; one thread issues).
     auto stage_load = [&](const TileInfo& ti, uint64_t policy) {
@@ -715,9 +721,9 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
     auto measure = [&](const TileInfo& ti, uint32_t (&d)[kWordsPerLane], uint32_t sl) {
         if (!ti.valid) return;
         if (!ti.present || !ti.full) {
-            if (warp == 0 && lane == 0) publish_len(ti.t, encoded_len(ti, 0));
+            if (warp == 0 && lane == 0) publish_len(ti.t, encoded_len(g, ti, 0));
             if (!ti.present) return;
-            load_tile_words_guarded(cache + (uint64_t)ti.t * kTile, ti.left, ti.first, warp, lane, d);
+            load_tile_words_guarded(cache + (uint64_t)ti.t * kTile, tile_left(g, ti.t), ti.first, warp, lane, d);
         }
         const uint32_t v = tile_digest_part(S, d, ti.first && ti.full, warp, lane);
         if (lane == 0) tc->wdig[sl][warp] = v;
@@ -737,11 +743,27 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
                 mysum += wd;
                 if (lane == 0) tc->wtab[sl][4 * warp + j] = emin | (wd << 8);
             }
+            // the warp that arrives last turns the 32 widths into offsets and publishes the length
+            uint32_t last = 0;
             if (lane == 0) {
-                const uint32_t old = atomicAdd(&tc->wsum[sl], mysum + (1u << 16));
-                if ((old >> 16) == 7u) {
+                __threadfence_block();
+                last = (atomicAdd(&tc->wsum[sl], 1u) == 7u) ? 1u : 0u;
+            }
+            if (__shfl_sync(0xFFFFFFFFu, last, 0)) {
+                __threadfence_block();
+                const uint32_t wt = *reinterpret_cast<volatile uint32_t*>(&tc->wtab[sl][lane]);
+                const uint32_t wv = (wt >> 8) & 15u;
+                uint32_t incl = wv;
+#pragma unroll
+                for (int k = 1; k < 32; k <<= 1) {
+                    const uint32_t o = __shfl_up_sync(0xFFFFFFFFu, incl, k);
+                    if (lane >= (uint32_t)k) incl += o;
+                }
+                tc->wtab[sl][lane] = (wt & 0xFFFFu) | ((incl - wv) << 16);
+                if (lane == 31) {
+                    tc->ssum[sl] = incl;
                     tc->wsum[sl] = 0;
-                    publish_len(ti.t, encoded_len(ti, (old & 0xFFFFu) + mysum));
+                    publish_len(ti.t, encoded_len(g, ti, incl));
                 }
             }
         }
@@ -752,27 +774,22 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
         if (ti.present) {
             unsigned char* dst = wire + g.meta_end + excl;
             if (ti.full) {
-                const uint32_t wt = tc->wtab[sl][lane];
-                const uint32_t wv = (wt >> 8) & 15u;
-                uint32_t incl = wv;
-#pragma unroll
-                for (int k = 1; k < 32; k <<= 1) {
-                    const uint32_t o = __shfl_up_sync(0xFFFFFFFFu, incl, k);
-                    if (lane >= (uint32_t)k) incl += o;
-                }
-                const uint32_t Ssum = __shfl_sync(0xFFFFFFFFu, incl, 31);
+                const uint32_t Ssum = tc->ssum[sl];
                 const bool packs = Ssum <= 253u;
                 enc_len = packs ? 8256u + 32u * Ssum : kTile;
                 entry = packs ? 258u + Ssum : 512u;
                 if (g.meta_end + excl + enc_len > wire_cap) {
                     if (tt == 0) atomicOr(&ws.ctrl->err, 1u);
                 } else if (packs) {
-                    if (warp == 0) stg_u16(dst + 2 * lane, desc_of(wt & 0xFFu, wv));
+                    if (warp == 0) {
+                        const uint32_t wt = tc->wtab[sl][lane];
+                        stg_u16(dst + 2 * lane, desc_of(wt & 0xFFu, (wt >> 8) & 15u));
+                    }
 #pragma unroll
                     for (int j = 0; j < 4; j++) {
                         const uint32_t gi = 4 * warp + j;
-                        const uint32_t wtg = __shfl_sync(0xFFFFFFFFu, wt, gi);
-                        const uint32_t exg = __shfl_sync(0xFFFFFFFFu, incl - wv, gi);
+                        const uint32_t wtg = tc->wtab[sl][gi];
+                        const uint32_t exg = wtg >> 16;
                         const uint32_t base = wtg & 0xFFu, wd = (wtg >> 8) & 15u;
                         uint32_t Tr[4];
 #pragma unroll
@@ -802,7 +819,7 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
                     for (int i = 0; i < 16; i++) st_stream_u32(q + i * 128, d[i]);
                 }
             } else {
-                enc_len = ti.left;
+                enc_len = tile_left(g, ti.t);
                 entry = 0xFFFFu;
                 if (g.meta_end + excl + enc_len > wire_cap) {
                     if (tt == 0) atomicOr(&ws.ctrl->err, 1u);
@@ -1561,7 +1578,8 @@ static const DeviceState* device_state()
     if (cudaMemcpy(s.tables, &host, sizeof(Tables), cudaMemcpyHostToDevice) != cudaSuccess) return nullptr;
     if (cudaDeviceGetAttribute(&s.sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return nullptr;
     const int big = kDynSmem;
-    if (cudaFuncSetAttribute(k_encode<kTeams>, cudaFuncAttributeMaxDynamicSharedMemorySize, big) != cudaSuccess) return nullptr;
+    if (cudaFuncSetAttribute(k_encode<kTeams, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, big) != cudaSuccess) return nullptr;
+    if (cudaFuncSetAttribute(k_encode<kTeams, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, big) != cudaSuccess) return nullptr;
     if (cudaFuncSetAttribute(k_decode<kTeamsPlain>, cudaFuncAttributeMaxDynamicSharedMemorySize, big) != cudaSuccess) return nullptr;
     if (cudaFuncSetAttribute(k_tile_digests<kTeamsPlain>, cudaFuncAttributeMaxDynamicSharedMemorySize, big) != cudaSuccess) return nullptr;
     if (cudaFuncSetAttribute(k_meta_crc, cudaFuncAttributeMaxDynamicSharedMemorySize, big) != cudaSuccess) return nullptr;
@@ -1685,7 +1703,8 @@ wm_status wm_encode(const void* cache, uint64_t nbytes, uint32_t chunk_bytes, co
     const uint32_t grid = need < (uint32_t)ds->sm_count ? need : (uint32_t)ds->sm_count;
     {
         MainKernelTimer timer(ds, 2, s);
-        k_encode<kTeams><<<grid, kTeams * 256, kDynSmem, s>>>(c, g, dirty, w, wire_cap, ws, ds->tables);
+        if (dirty) k_encode<kTeams, true><<<grid, kTeams * 256, kDynSmem, s>>>(c, g, dirty, w, wire_cap, ws, ds->tables);
+        else k_encode<kTeams, false><<<grid, kTeams * 256, kDynSmem, s>>>(c, g, dirty, w, wire_cap, ws, ds->tables);
     }
     k_encode_finish<<<(g.n_chunks + 1023) / 1024, 1024, 0, s>>>(c, g, dirty, crc_inout, w, ws, ds->tables);
     k_meta_crc<<<g.n_meta_slices, 256, kDynSmem, s>>>(w, 0, g, ws, ds->tables, result, 0);
