@@ -183,10 +183,23 @@ __device__ uint32_t chunk_crc_from_digests(const Geo& g, const uint32_t* HT, con
     const uint32_t ntc = (uint32_t)((clen + kTile - 1) / kTile);
     const bool ragged = (clen % kTile) != 0;
     uint32_t st = 0;
-    for (uint32_t i = 0; i < ntc; i++) {
+    uint32_t i = 0;
+    // full tiles, eight at a time: the digests are fetched first (independent loads), then folded
+    const uint32_t n_plain = ragged ? ntc - 1 : ntc;
+    if ((t0 & 3u) == 0) {
+        for (; i + 8 <= n_plain; i += 8) {
+            const uint4 a = __ldcg(reinterpret_cast<const uint4*>(dig + t0 + i));
+            const uint4 b = __ldcg(reinterpret_cast<const uint4*>(dig + t0 + i + 4));
+            st = advance_tile(HT, st) ^ a.x; st = advance_tile(HT, st) ^ a.y;
+            st = advance_tile(HT, st) ^ a.z; st = advance_tile(HT, st) ^ a.w;
+            st = advance_tile(HT, st) ^ b.x; st = advance_tile(HT, st) ^ b.y;
+            st = advance_tile(HT, st) ^ b.z; st = advance_tile(HT, st) ^ b.w;
+        }
+    }
+    for (; i < ntc; i++) {
         if (i + 1 == ntc && ragged) st = mulmod_dev(st, g.k_tail);
         else st = advance_tile(HT, st);
-        st ^= dig[t0 + i];
+        st ^= __ldcg(dig + t0 + i);
     }
     return ~st;
 }
@@ -198,9 +211,35 @@ __device__ __forceinline__ void load_ht_t0(uint32_t* sHT, uint32_t* sT0, const T
     __syncthreads();
 }
 
+// Table of products with one fixed multiplier M (block of 1024 threads; ends with a block
+// barrier): tab[256 k + v] = (v << 8k) * M, so that a * M is four lookups.
+__device__ void build_mul_table(uint32_t* tab, uint32_t M)
+{
+    const uint32_t k = threadIdx.x >> 8, v = threadIdx.x & 255u;
+    // bit 8k+j of (v << 8k) is the coefficient of x^(31-8k-j): start at M x^(24-8k) for j = 7
+    uint32_t b = M;
+    for (uint32_t i = 0; i < 24u - 8u * k; i++) b = (b >> 1) ^ (kPolyReflected & (0u - (b & 1u)));
+    uint32_t r = 0;
+#pragma unroll
+    for (int j = 7; j >= 0; j--) {
+        r ^= b & (0u - ((v >> j) & 1u));
+        b = (b >> 1) ^ (kPolyReflected & (0u - (b & 1u)));
+    }
+    tab[threadIdx.x] = r;
+    __syncthreads();
+}
+__device__ __forceinline__ uint32_t mul_by_table(const uint32_t* tab, uint32_t a)
+{
+    return tab[a & 0xFF] ^ tab[256 + ((a >> 8) & 0xFF)] ^ tab[512 + ((a >> 16) & 0xFF)] ^ tab[768 + (a >> 24)];
+}
+
 // CRC32C of the concatenation of all chunks from their finished CRCs (block-wide; every
 // thread of a 1024-thread block must call).  crc(A||B) = crc(A) x^(8 len B) + crc(B).
-__device__ uint32_t combine_chunk_crcs(const Geo& g, const uint32_t* crc, uint32_t stride_words, uint32_t* sbuf)
+// Each thread folds a run of chunks, then a tree folds the runs; every product is with a
+// multiplier shared by the whole block, so it goes through a table built for that multiplier.
+// stab: 1024 words for the table, sbuf: 1024 words.
+__device__ uint32_t combine_chunk_crcs(const Geo& g, const uint32_t* crc, uint32_t stride_words, uint32_t* stab,
+                                       uint32_t* sbuf)
 {
     const uint32_t n = g.n_chunks;
     if (n == 1) return __ldcg(&crc[0]);
@@ -208,30 +247,24 @@ __device__ uint32_t combine_chunk_crcs(const Geo& g, const uint32_t* crc, uint32
     const uint32_t T = blockDim.x;                  // 1024
     const uint32_t R = (m + T - 1) / T;             // run per thread
     const uint64_t pad = (uint64_t)T * R - m;       // leading empty slots
-    uint32_t acc = 0;
+    build_mul_table(stab, g.k_chunk);
+    uint32_t acc = 0, M = 0x80000000u;              // M becomes k_chunk^R
     for (uint32_t s = 0; s < R; s++) {
         uint64_t slot = (uint64_t)threadIdx.x * R + s;
         uint32_t v = slot >= pad ? __ldcg(&crc[(slot - pad) * stride_words]) : 0u;
-        acc = (acc ? mulmod_dev(acc, g.k_chunk) : 0u) ^ v;
-    }
-    // multiplier of one run: k_chunk^R
-    uint32_t M = 0x80000000u, b = g.k_chunk;
-    for (uint32_t e = R; e; e >>= 1) {
-        if (e & 1u) M = mulmod_dev(M, b);
-        if (e > 1) b = mulmod_dev(b, b);
+        acc = mul_by_table(stab, acc) ^ v;
+        M = mul_by_table(stab, M);
     }
     sbuf[threadIdx.x] = acc;
     __syncthreads();
     for (uint32_t width = T / 2; width >= 1; width >>= 1) {
+        build_mul_table(stab, M);
         uint32_t v = 0;
-        if (threadIdx.x < width) {
-            uint32_t a = sbuf[2 * threadIdx.x], c2 = sbuf[2 * threadIdx.x + 1];
-            v = (a ? mulmod_dev(a, M) : 0u) ^ c2;
-        }
+        if (threadIdx.x < width) v = mul_by_table(stab, sbuf[2 * threadIdx.x]) ^ sbuf[2 * threadIdx.x + 1];
+        M = mul_by_table(stab, M);
         __syncthreads();
         if (threadIdx.x < width) sbuf[threadIdx.x] = v;
         __syncthreads();
-        M = mulmod_dev(M, M);
     }
     uint32_t fold = sbuf[0];
     __syncthreads();
@@ -927,6 +960,7 @@ k_encode_finish(const unsigned char* __restrict__ cache, Geo g, const uint8_t* _
     __shared__ uint32_t sHT[1024];
     __shared__ uint32_t sT0[256];
     __shared__ uint32_t sbuf[1024];
+    __shared__ uint32_t stab[1024];
     __shared__ bool s_last;
     load_ht_t0(sHT, sT0, tab);
     unsigned char* dir = wire + 64;
@@ -958,7 +992,7 @@ k_encode_finish(const unsigned char* __restrict__ cache, Geo g, const uint8_t* _
     __syncthreads();
     if (!s_last) return;
     __threadfence();
-    const uint32_t cache_crc = combine_chunk_crcs(g, reinterpret_cast<const uint32_t*>(dir + 12), 4, sbuf);
+    const uint32_t cache_crc = combine_chunk_crcs(g, reinterpret_cast<const uint32_t*>(dir + 12), 4, stab, sbuf);
     if (threadIdx.x == 0) {
         const uint32_t n_present = ld_volatile_u32(&ws.ctrl->n_present);
         uint32_t* h = reinterpret_cast<uint32_t*>(wire);
@@ -978,11 +1012,11 @@ k_encode_finish(const unsigned char* __restrict__ cache, Geo g, const uint8_t* _
 
 // CRC32C of the metadata region wire[0, meta_end) with the meta_crc field read as zero.
 // The region is right-aligned in a whole number of virtual 16 KiB slices (leading zeros),
-// one block (one team) per slice; the last block to finish folds the slice digests.
+// one team per slice, four teams per block; the last block to finish folds the slice digests.
 //   mode 0 (encode): store the CRC into the header and write the result record.
 //   mode 1 (decode): check the header against the call (FORMAT), then the CRC (META_CRC);
 //                    on failure set the gate and write the result record.
-__global__ void __launch_bounds__(256, 1)
+__global__ void __launch_bounds__(1024, 1)
 k_meta_crc(unsigned char* wire, uint64_t wire_len, Geo g, Ws ws, const Tables* __restrict__ tab,
            wm_result* result, int mode)
 {
@@ -990,9 +1024,13 @@ k_meta_crc(unsigned char* wire, uint64_t wire_len, Geo g, Ws ws, const Tables* _
     __shared__ bool s_last;
     __shared__ int s_format_bad;
     Smem S = setup_smem(smem, tab);
-    const uint32_t warp = threadIdx.x / 32, lane = threadIdx.x % 32;
-    TeamCtl* tc = reinterpret_cast<TeamCtl*>(S.take(sizeof(TeamCtl)));
+    const uint32_t team = threadIdx.x / kTeamThreads, tt = threadIdx.x % kTeamThreads;
+    const uint32_t warp = tt / 32, lane = tt % 32;
+    TeamCtl* tc = reinterpret_cast<TeamCtl*>(S.take(4 * sizeof(TeamCtl)));
+    uint32_t* sHT = reinterpret_cast<uint32_t*>(S.take(4096));
     if (!S.ok) { if (threadIdx.x == 0) atomicOr(&ws.ctrl->err, 4u); return; }
+    tc += team;
+    sHT[threadIdx.x] = (&tab->HT[0][0])[threadIdx.x];
 
     if (mode == 1) {
         // FORMAT check by every block (cheap, keeps the gate decision local)
@@ -1025,27 +1063,29 @@ k_meta_crc(unsigned char* wire, uint64_t wire_len, Geo g, Ws ws, const Tables* _
     }
 
     const uint64_t pad = (uint64_t)g.n_meta_slices * kTile - g.meta_end;    // multiple of 4
-    const uint32_t s = blockIdx.x;
-    uint32_t w[kWordsPerLane];
+    const uint32_t s = blockIdx.x * 4 + team;
+    if (s < g.n_meta_slices) {
+        uint32_t w[kWordsPerLane];
 #pragma unroll
-    for (int i = 0; i < 16; i++) {
-        const uint64_t vb = (uint64_t)s * kTile + (warp * 16 + i) * 128 + lane * 4;
-        uint32_t v = 0;
-        if (vb >= pad) {
-            const uint64_t rb = vb - pad;
-            v = *reinterpret_cast<const uint32_t*>(wire + rb);
-            if (rb == 52) v = 0;
-            if (rb == 0) v ^= 0xFFFFFFFFu;
+        for (int i = 0; i < 16; i++) {
+            const uint64_t vb = (uint64_t)s * kTile + (warp * 16 + i) * 128 + lane * 4;
+            uint32_t v = 0;
+            if (vb >= pad) {
+                const uint64_t rb = vb - pad;
+                v = *reinterpret_cast<const uint32_t*>(wire + rb);
+                if (rb == 52) v = 0;
+                if (rb == 0) v ^= 0xFFFFFFFFu;
+            }
+            w[i] = v;
         }
-        w[i] = v;
-    }
-    {
         const uint32_t v = tile_digest_part(S, w, false, warp, lane);
         if (lane == 0) tc->wdig[0][warp] = v;
     }
     __syncthreads();
+    if (tt == 0 && s < g.n_meta_slices) ws.mdig[s] = xor8(tc->wdig[0]);
+    __threadfence();
+    __syncthreads();
     if (threadIdx.x == 0) {
-        ws.mdig[s] = xor8(tc->wdig[0]);
         __threadfence();
         s_last = atomicAdd(&ws.ctrl->done_b, 1u) == gridDim.x - 1;
     }
@@ -1054,7 +1094,7 @@ k_meta_crc(unsigned char* wire, uint64_t wire_len, Geo g, Ws ws, const Tables* _
     __threadfence();
     uint32_t st = 0;
     for (uint32_t i = 0; i < g.n_meta_slices; i++) {
-        st = advance_tile(&tab->HT[0][0], st);
+        st = advance_tile(sHT, st);
         st ^= ld_volatile_u32(&ws.mdig[i]);
     }
     const uint32_t crc = ~st;
@@ -1476,6 +1516,7 @@ k_decode_finish(const unsigned char* __restrict__ wire, uint64_t wire_len, Geo g
     __shared__ uint32_t sHT[1024];
     __shared__ uint32_t sT0[256];
     __shared__ uint32_t sbuf[1024];
+    __shared__ uint32_t stab[1024];
     __shared__ bool s_last;
     __shared__ int s_status;
     load_ht_t0(sHT, sT0, tab);
@@ -1504,7 +1545,7 @@ k_decode_finish(const unsigned char* __restrict__ wire, uint64_t wire_len, Geo g
     __syncthreads();
     if (!s_last) return;
     __threadfence();
-    const uint32_t cache_crc = combine_chunk_crcs(g, reinterpret_cast<const uint32_t*>(dir + 12), 4, sbuf);
+    const uint32_t cache_crc = combine_chunk_crcs(g, reinterpret_cast<const uint32_t*>(dir + 12), 4, stab, sbuf);
     if (threadIdx.x == 0) {
         int status = WM_OK;
         uint32_t first = 0, count = 0;
@@ -1707,7 +1748,7 @@ wm_status wm_encode(const void* cache, uint64_t nbytes, uint32_t chunk_bytes, co
         else k_encode<kTeams, false><<<grid, kTeams * 256, kDynSmem, s>>>(c, g, dirty, w, wire_cap, ws, ds->tables);
     }
     k_encode_finish<<<(g.n_chunks + 1023) / 1024, 1024, 0, s>>>(c, g, dirty, crc_inout, w, ws, ds->tables);
-    k_meta_crc<<<g.n_meta_slices, 256, kDynSmem, s>>>(w, 0, g, ws, ds->tables, result, 0);
+    k_meta_crc<<<(g.n_meta_slices + 3) / 4, 1024, kDynSmem, s>>>(w, 0, g, ws, ds->tables, result, 0);
     g_launches = 4;
     return launch_status();
 }
@@ -1728,7 +1769,7 @@ wm_status wm_decode_verify(const void* wire, uint64_t wire_len, void* dst, uint6
     k_decode_init<<<1, 64, 0, s>>>(ws);
     // a wire shorter than the metadata is rejected by the header check before anything else is read
     const uint32_t slices = wire_len >= g.meta_end ? g.n_meta_slices : 1;
-    k_meta_crc<<<slices, 256, kDynSmem, s>>>(const_cast<unsigned char*>(w), wire_len, g, ws, ds->tables, result, 1);
+    k_meta_crc<<<(slices + 3) / 4, 1024, kDynSmem, s>>>(const_cast<unsigned char*>(w), wire_len, g, ws, ds->tables, result, 1);
     k_decode_struct_chunks<<<(g.n_chunks + 7) / 8, 256, 0, s>>>(w, g, ws);
     k_decode_struct_scan<<<1, 1024, 0, s>>>(w, wire_len, g, ws, result);
     const uint32_t need = (g.n_tiles + kTeamsPlain - 1) / kTeamsPlain;
