@@ -211,6 +211,8 @@ __device__ __forceinline__ void load_ht_t0(uint32_t* sHT, uint32_t* sT0, const T
     __syncthreads();
 }
 
+constexpr uint32_t kFinishChunks = 128;      // chunks folded per block of the finish kernels
+
 // Table of products with one fixed multiplier M (block of 1024 threads; ends with a block
 // barrier): tab[256 k + v] = (v << 8k) * M, so that a * M is four lookups.
 __device__ void build_mul_table(uint32_t* tab, uint32_t M)
@@ -965,9 +967,11 @@ k_encode_finish(const unsigned char* __restrict__ cache, Geo g, const uint8_t* _
     load_ht_t0(sHT, sT0, tab);
     unsigned char* dir = wire + 64;
     const unsigned long long total = ws.ctrl->payload_total;
-    const uint32_t c = blockIdx.x * blockDim.x + threadIdx.x;
+    // only kFinishChunks threads of a block fold chunks (the lookups of a full block would queue
+    // up on one SM's shared memory); all of them take part in the last block's combine
+    const uint32_t c = blockIdx.x * kFinishChunks + threadIdx.x;
     uint32_t present = 0;
-    if (c < g.n_chunks) {
+    if (threadIdx.x < kFinishChunks && c < g.n_chunks) {
         present = (!dirty || dirty[c]) ? 1u : 0u;
         uint32_t crc;
         if (present) {
@@ -1521,10 +1525,10 @@ k_decode_finish(const unsigned char* __restrict__ wire, uint64_t wire_len, Geo g
     __shared__ int s_status;
     load_ht_t0(sHT, sT0, tab);
     const unsigned char* dir = wire + 64;
-    const uint32_t c = blockIdx.x * blockDim.x + threadIdx.x;
+    const uint32_t c = blockIdx.x * kFinishChunks + threadIdx.x;
     const bool step4_failed = ld_volatile_u32(reinterpret_cast<const uint32_t*>(&ws.ctrl->bad4_key)) != 0xFFFFFFFFu ||
                               ld_volatile_u32(reinterpret_cast<const uint32_t*>(&ws.ctrl->bad4_key) + 1) != 0xFFFFFFFFu;
-    if (c < g.n_chunks) {
+    if (threadIdx.x < kFinishChunks && c < g.n_chunks) {
         const uint32_t fl = ws.cflag[c];
         const uint32_t want = *reinterpret_cast<const uint32_t*>(dir + 16ull * c + 12);
         if (step4_failed) {
@@ -1747,7 +1751,7 @@ wm_status wm_encode(const void* cache, uint64_t nbytes, uint32_t chunk_bytes, co
         if (dirty) k_encode<kTeams, true><<<grid, kTeams * 256, kDynSmem, s>>>(c, g, dirty, w, wire_cap, ws, ds->tables);
         else k_encode<kTeams, false><<<grid, kTeams * 256, kDynSmem, s>>>(c, g, dirty, w, wire_cap, ws, ds->tables);
     }
-    k_encode_finish<<<(g.n_chunks + 1023) / 1024, 1024, 0, s>>>(c, g, dirty, crc_inout, w, ws, ds->tables);
+    k_encode_finish<<<(g.n_chunks + kFinishChunks - 1) / kFinishChunks, 1024, 0, s>>>(c, g, dirty, crc_inout, w, ws, ds->tables);
     k_meta_crc<<<(g.n_meta_slices + 3) / 4, 1024, kDynSmem, s>>>(w, 0, g, ws, ds->tables, result, 0);
     g_launches = 4;
     return launch_status();
@@ -1778,7 +1782,7 @@ wm_status wm_decode_verify(const void* wire, uint64_t wire_len, void* dst, uint6
         MainKernelTimer timer(ds, 3, s);
         k_decode<kTeamsPlain><<<grid, kTeamsPlain * 256, kDynSmem, s>>>(w, g, d, ws, ds->tables);
     }
-    k_decode_finish<<<(g.n_chunks + 1023) / 1024, 1024, 0, s>>>(w, wire_len, g, d, dst_crc_inout, ws, ds->tables, result);
+    k_decode_finish<<<(g.n_chunks + kFinishChunks - 1) / kFinishChunks, 1024, 0, s>>>(w, wire_len, g, d, dst_crc_inout, ws, ds->tables, result);
     g_launches = 6;
     return launch_status();
 }
