@@ -238,13 +238,15 @@ __device__ __forceinline__ void bulk_load(void* smem_dst, const void* gsrc, uint
 }
 
 // Wait for the phase with the given parity to complete (bounded).  Returns false on timeout.
+// try_wait suspends the thread in hardware until the phase completes or the time hint runs
+// out, so a waiting warp does not burn issue slots that the other teams on the SM need.
 __device__ __forceinline__ bool mbar_wait(unsigned long long* bar, uint32_t parity)
 {
     const uint32_t b = (uint32_t)__cvta_generic_to_shared(bar);
-    for (uint32_t i = 0; i < (1u << 22); i++) {
+    for (uint32_t i = 0; i < 4096u; i++) {
         uint32_t done;
-        asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-                     : "=r"(done) : "r"(b), "r"(parity) : "memory");
+        asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                     : "=r"(done) : "r"(b), "r"(parity), "r"(500000u) : "memory");
         if (done) return true;
     }
     return false;
