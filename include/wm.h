@@ -155,6 +155,30 @@ wm_status wm_decode_verify(const void* wire, uint64_t wire_len, void* dst, uint6
                            uint32_t chunk_bytes, uint32_t* dst_crc_inout,
                            void* workspace, uint64_t workspace_bytes, wm_result* result, void* stream);
 
+/*
+ * wm_checksum_noalloc - wm_checksum for callers that cannot allocate device memory.
+ * The paper has no counterpart to this call; it exists for hosts that may not call cudaMalloc
+ * at the point where they need a checksum: code running inside a stream capture or under an
+ * allocator that has been frozen for the life of a serving process, plug-ins that are handed
+ * a stream and buffers but no allocation rights, and start-up or recovery paths that must not
+ * touch the device heap.  Same result as wm_checksum, bit for bit, but the scratch memory and
+ * the constant tables sit in arrays built into the library image (about 1.2 MiB that every
+ * GPU loading the library keeps until the process exits), so the call takes no workspace.
+ *   - Limit: nbytes <= WM_NOALLOC_MAX_BYTES (4 GiB); larger inputs return WM_ERR_ARG and
+ *     nothing is launched.  All other argument rules are those of wm_checksum.
+ *   - The first call on a device looks up the arrays' device addresses and uploads the
+ *     tables (a synchronous copy).  Make that first call before any stream capture.
+ *   - The call itself allocates nothing: no cudaMalloc, cudaFree or allocating library call.
+ *   - There is one scratch array per device and every call uses it.  It keeps the previous
+ *     call's contents (the part that must start at zero is cleared on the stream), and two
+ *     calls whose kernels overlap on the GPU (different streams, no ordering) race on it:
+ *     order such calls on one stream or with events.
+ */
+#define WM_NOALLOC_MAX_BYTES (4ull << 30)
+#define WM_NOALLOC_SCRATCH_BYTES ((1u << 20) + 4096u)
+wm_status wm_checksum_noalloc(const void* cache, uint64_t nbytes, uint32_t chunk_bytes,
+                              uint32_t* crc_out, void* stream);
+
 /* Number of kernels the last call on this host thread enqueued (for launch accounting). */
 uint32_t wm_last_launch_count(void);
 

@@ -23,7 +23,7 @@ STATUS = {
 RESULT_BYTES = 40
 EXPORTS = ("wm_num_chunks", "wm_num_tiles", "wm_meta_bytes", "wm_wire_bound", "wm_workspace_bytes",
            "wm_checksum", "wm_dirty_diff", "wm_encode", "wm_decode_verify", "wm_last_launch_count",
-           "wm_timing_enable", "wm_timing_read_ms")
+           "wm_timing_enable", "wm_timing_read_ms", "wm_checksum_noalloc")
 
 
 class WmError(RuntimeError):
@@ -51,6 +51,8 @@ def load_library() -> ctypes.CDLL:
     lib.wm_timing_read_ms.argtypes = [ctypes.c_int, ctypes.POINTER(ctypes.c_float)]
     lib.wm_checksum.restype = ctypes.c_int
     lib.wm_checksum.argtypes = [vp, u64, u32, vp, vp, u64, vp]
+    lib.wm_checksum_noalloc.restype = ctypes.c_int
+    lib.wm_checksum_noalloc.argtypes = [vp, u64, u32, vp, vp]
     lib.wm_dirty_diff.restype = ctypes.c_int
     lib.wm_dirty_diff.argtypes = [vp, vp, u64, u32, vp, vp, vp, vp, u64, vp]
     lib.wm_encode.restype = ctypes.c_int
@@ -169,6 +171,20 @@ def wm_checksum(cache: torch.Tensor, chunk_bytes: int, crc_out: torch.Tensor, wo
     nbytes = cache.numel() * cache.element_size()
     _check(lib().wm_checksum(cache.data_ptr(), nbytes, chunk_bytes, crc_out.data_ptr(), workspace.data_ptr(),
                              workspace.numel(), _stream(stream)), "wm_checksum")
+
+
+NOALLOC_MAX_BYTES = 4 << 30
+
+
+def wm_checksum_noalloc(cache: torch.Tensor, chunk_bytes: int, crc_out: torch.Tensor, stream=None,
+                        nbytes: int | None = None) -> None:
+    """wm_checksum without a workspace argument: scratch and tables are built into the library,
+    for callers that may not allocate device memory.  `nbytes` overrides the tensor's size
+    (used to exercise the size limit without allocating a buffer that large)."""
+    _dev_u8(cache, "cache")
+    n = cache.numel() * cache.element_size() if nbytes is None else int(nbytes)
+    _check(lib().wm_checksum_noalloc(cache.data_ptr(), n, chunk_bytes, crc_out.data_ptr(), _stream(stream)),
+           "wm_checksum_noalloc")
 
 
 def wm_dirty_diff(cache: torch.Tensor, prev: torch.Tensor, chunk_bytes: int, dirty_out: torch.Tensor,

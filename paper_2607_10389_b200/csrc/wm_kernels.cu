@@ -1703,6 +1703,75 @@ wm_status wm_checksum(const void* cache, uint64_t nbytes, uint32_t chunk_bytes, 
     return launch_status();
 }
 
+// ---- wm_checksum_noalloc: the checksum call for callers that must not allocate -------------
+//
+// Scratch and tables live in the library image itself: two file-scope __device__ arrays that
+// every GPU loading the library carries until the process exits.  In host code their names
+// are host-side stand-ins, not device addresses, so the addresses are asked for once per
+// device with cudaGetSymbolAddress (with that device current) and only those go to kernels.
+static __device__ __align__(256) unsigned char g_na_scratch[WM_NOALLOC_SCRATCH_BYTES];
+static __device__ __align__(256) unsigned char g_na_tables[sizeof(wm::Tables)];
+
+namespace wm {
+struct NoAllocState {
+    unsigned char* scratch = nullptr;
+    Tables* tables = nullptr;
+    int sm_count = 0;
+    bool ready = false;
+};
+static NoAllocState g_na[64];
+
+static const NoAllocState* noalloc_state()
+{
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    std::lock_guard<std::mutex> lock(g_mutex);
+    NoAllocState& s = g_na[dev];
+    if (s.ready) return &s;
+    void* p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_na_scratch) != cudaSuccess || !p) return nullptr;
+    s.scratch = static_cast<unsigned char*>(p);
+    p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_na_tables) != cudaSuccess || !p) return nullptr;
+    s.tables = static_cast<Tables*>(p);
+    static Tables host;                          // static storage: no heap, no device allocation
+    build_tables(host);
+    if (cudaMemcpy(s.tables, &host, sizeof(Tables), cudaMemcpyHostToDevice) != cudaSuccess) return nullptr;
+    if (cudaDeviceGetAttribute(&s.sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return nullptr;
+    if (cudaFuncSetAttribute(k_tile_digests<kTeamsPlain>, cudaFuncAttributeMaxDynamicSharedMemorySize, kDynSmem)
+        != cudaSuccess)
+        return nullptr;
+    s.ready = true;
+    return &s;
+}
+}  // namespace wm
+
+wm_status wm_checksum_noalloc(const void* cache, uint64_t nbytes, uint32_t chunk_bytes, uint32_t* crc_out, void* stream)
+{
+    Geo g;
+    if (!cache || !crc_out || !make_geo(nbytes, chunk_bytes, g) || !aligned16(cache)) return WM_ERR_ARG;
+    if (nbytes > WM_NOALLOC_MAX_BYTES) return WM_ERR_ARG;          // the built-in scratch holds no more
+    const NoAllocState* ns = noalloc_state();
+    if (!ns) return WM_ERR_CUDA;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    // scratch: a control block, then one 32-bit digest per tile
+    static_assert(WM_NOALLOC_SCRATCH_BYTES >= sizeof(Ctrl) + 4ull * (WM_NOALLOC_MAX_BYTES / WM_TILE_BYTES + 1),
+                  "built-in scratch covers the stated maximum");
+    Ws ws;
+    memset(&ws, 0, sizeof ws);
+    ws.ctrl = reinterpret_cast<Ctrl*>(ns->scratch);
+    ws.dig = reinterpret_cast<uint32_t*>(ns->scratch + sizeof(Ctrl));
+    // the array keeps the last call's contents; only the control block has to start at zero
+    if (cudaMemsetAsync(ns->scratch, 0, sizeof(Ctrl), s) != cudaSuccess) return WM_ERR_CUDA;
+    const unsigned char* c = static_cast<const unsigned char*>(cache);
+    const uint32_t need = (g.n_tiles + kTeamsPlain - 1) / kTeamsPlain;
+    const uint32_t grid = need < (uint32_t)ns->sm_count ? need : (uint32_t)ns->sm_count;
+    k_tile_digests<kTeamsPlain><<<grid, kTeamsPlain * 256, kDynSmem, s>>>(c, g, ws, ns->tables);
+    k_checksum_finish<<<(g.n_chunks + 255) / 256, 256, 0, s>>>(c, g, ws, ns->tables, crc_out);
+    g_launches = 2;
+    return launch_status();
+}
+
 wm_status wm_dirty_diff(const void* cache, const void* prev, uint64_t nbytes, uint32_t chunk_bytes,
                         uint8_t* dirty_out, uint32_t* dirty_idx_out, uint32_t* n_dirty_out,
                         void* workspace, uint64_t workspace_bytes, void* stream)
