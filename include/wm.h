@@ -117,7 +117,12 @@ wm_status wm_dirty_diff(const void* cache, const void* prev, uint64_t nbytes, ui
  *           base = min E, w = bit length of (max E - base); a tile packs iff sum w <= 253
  *           (length 8256 + 32*sum w), else it is stored raw.  Inside a group, element e
  *           (memory order) has coded position k = 8*((e%64)/2) + 2*(e/64) + (e%2); SM[256 g + k]
- *           is its SM byte and bits [k w, (k+1) w) of Epack_g (LSB-first) hold E - base.
+ *           is its SM byte.  Epack_g (32 w bytes) stores d = E - base as bit planes, in this
+ *           order, each present iff w has that bit: for w < 8 a 4-bit plane (128 bytes), a
+ *           2-bit plane (64 bytes), a 1-bit plane (32 bytes); for w = 8 one 8-bit plane (256
+ *           bytes).  The planes take consecutive bits of d from bit 0 upwards (w = 7: bits
+ *           0..3, 4..5, 6); element k sits at bits [k p, (k+1) p) of its p-bit plane, LSB first.
+ *           The payload is limited to 32 GiB (WM_ERR_ARG beyond that).
  *
  *   dirty     [dev] u8[n_chunks] or NULL (NULL = every chunk present: the fused
  *             checksum+encode of a full move)

@@ -3,8 +3,8 @@
 // Kernel map (every call enqueues a short chain on the caller's stream, no host sync):
 //   wm_checksum      : k_tile_digests -> k_checksum_finish
 //   wm_dirty_diff    : k_diff_init -> k_diff -> k_diff_compact
-//   wm_encode        : k_encode_init -> k_encode (single pass, decoupled look-back over tile
-//                      lengths) -> k_encode_finish (directory, cache CRC, header)
+//   wm_encode        : k_encode_init -> k_encode (single pass; teams publish tile lengths, one
+//                      scanner warp turns them into payload offsets) -> k_encode_finish (directory, cache CRC, header)
 //                      -> k_meta_crc (metadata CRC, result)
 //   wm_decode_verify : k_decode_init -> k_meta_crc (header + metadata CRC gate)
 //                      -> k_decode_struct_chunks -> k_decode_struct_scan (structure gate)
@@ -106,6 +106,10 @@ static Ws ws_carve(void* base, const Geo& g)
     w.mdig = reinterpret_cast<uint32_t*>(b + L.mdig);
     return w;
 }
+
+// Payload offsets travel between blocks as 30-bit counts of 32-byte units, and the payload is
+// never longer than the cache, so the codec entry points take caches up to 32 GiB.
+constexpr uint64_t kMaxCodecBytes = 32ull << 30;
 
 static bool make_geo(uint64_t nbytes, uint32_t chunk_bytes, Geo& g)
 {
@@ -1804,6 +1808,7 @@ wm_status wm_encode(const void* cache, uint64_t nbytes, uint32_t chunk_bytes, co
     if (!aligned16(cache) || !aligned16(wire) || !aligned16(workspace) || workspace_bytes < ws_layout(g).total ||
         wire_cap < g.meta_end)
         return WM_ERR_ARG;
+    if (nbytes > kMaxCodecBytes) return WM_ERR_ARG;
     const DeviceState* ds = device_state();
     if (!ds) return WM_ERR_CUDA;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
@@ -1833,6 +1838,7 @@ wm_status wm_decode_verify(const void* wire, uint64_t wire_len, void* dst, uint6
     Geo g;
     if (!wire || !dst || !dst_crc_inout || !workspace || !result || !make_geo(nbytes, chunk_bytes, g)) return WM_ERR_ARG;
     if (!aligned16(wire) || !aligned16(dst) || !aligned16(workspace) || workspace_bytes < ws_layout(g).total) return WM_ERR_ARG;
+    if (nbytes > kMaxCodecBytes) return WM_ERR_ARG;
     const DeviceState* ds = device_state();
     if (!ds) return WM_ERR_CUDA;
     cudaStream_t s = static_cast<cudaStream_t>(stream);

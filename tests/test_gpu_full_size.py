@@ -1,0 +1,262 @@
+"""Parity at the full workload sizes, in the launch configuration the benchmark times.
+
+The oracle cannot run a multi-gigabyte cache in seconds, so these tests compare what it can
+compute one by one (sampled chunks: CRC, encoded payload bytes, tile table entries; the whole
+metadata block, which is small) and properties that hold at any size (directory offsets are the
+running sum of lengths, the decoded shadow equals the cache byte for byte, a flipped bit is
+rejected and nothing is installed).
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2607_10389_b200 import binding as wm
+from paper_2607_10389_b200 import inputs
+
+pytestmark = pytest.mark.gpu
+
+TILE = 16384
+
+
+class Job:
+    """Buffers of one geometry, reused over the calls of a test."""
+
+    def __init__(self, nbytes, chunk):
+        self.n, self.chunk = nbytes, chunk
+        self.nc = wm.num_chunks(nbytes, chunk)
+        self.nt = wm.num_tiles(nbytes)
+        self.meta_end = wm.meta_bytes(nbytes, chunk)
+        self.cap = wm.wire_bound(nbytes, chunk)
+        self.ws = wm.new_workspace(nbytes, chunk)
+        self.ws2 = wm.new_workspace(nbytes, chunk)
+        self.wire = torch.empty(self.cap, dtype=torch.uint8, device="cuda")
+        self.res_e, self.res_d = wm.new_result(), wm.new_result()
+
+    def meta(self):
+        m = self.wire[: self.meta_end].cpu().numpy()
+        hdr = m[:64]
+        directory = m[64: 64 + 16 * self.nc]
+        off = directory.view(np.uint64).reshape(self.nc, 2)[:, 0].copy()
+        ln = directory.view(np.uint32).reshape(self.nc, 4)[:, 2].copy()
+        crc = directory.view(np.uint32).reshape(self.nc, 4)[:, 3].copy()
+        tab = m[64 + 16 * self.nc: 64 + 16 * self.nc + 2 * self.nt].view(np.uint16).copy()
+        return m, hdr, off, ln, crc, tab
+
+
+def check_meta_against_oracle(job, m, hdr, off, ln, crc, present):
+    """Header, directory sums, metadata CRC and whole-cache CRC, recomputed with the oracle's CRC."""
+    assert bytes(hdr[:4]) == b"WMV1"
+    assert int(hdr[8:16].view(np.uint64)[0]) == job.n and int(hdr[16:20].view(np.uint32)[0]) == job.chunk
+    assert int(hdr[24:28].view(np.uint32)[0]) == job.nc and int(hdr[28:32].view(np.uint32)[0]) == int(present.sum())
+    run = np.concatenate([[0], np.cumsum(ln.astype(np.uint64) * present)])[:-1]
+    assert np.array_equal(off[present == 1], run[present == 1])
+    assert (ln[present == 0] == 0).all()
+    payload = int((ln.astype(np.uint64) * present).sum())
+    assert int(hdr[32:40].view(np.uint64)[0]) == payload
+    assert int(hdr[40:48].view(np.uint64)[0]) == job.meta_end + payload
+    z = m.copy()
+    z[52:56] = 0
+    assert oracle.crc32c(z) == int(hdr[52:56].view(np.uint32)[0])
+    acc = int(crc[0])
+    for c in range(1, job.nc):
+        acc = oracle.crc_combine(acc, int(crc[c]), min(job.chunk, job.n - c * job.chunk))
+    assert acc == int(hdr[48:52].view(np.uint32)[0])
+
+
+def check_chunks_against_oracle(job, cache, chunks, off, ln, crc, tab):
+    """Each sampled chunk, encoded alone by the oracle, gives the bytes found in the wire image."""
+    tpc = job.chunk // TILE
+    for c in chunks:
+        lo, hi = c * job.chunk, min((c + 1) * job.chunk, job.n)
+        raw = cache[lo:hi].cpu().numpy()
+        w1, crc1, r1 = oracle.encode(raw, job.chunk)
+        assert r1.status == 0
+        assert int(crc1[0]) == int(crc[c]) == oracle.crc32c(raw), f"chunk {c}: crc"
+        me = oracle.meta_end(hi - lo, job.chunk)
+        pay = w1[me: r1.wire_len]
+        assert pay.size == int(ln[c]), f"chunk {c}: encoded length"
+        a = job.meta_end + int(off[c])
+        got = job.wire[a: a + pay.size].cpu().numpy()
+        assert np.array_equal(got, pay), f"chunk {c}: payload bytes"
+        nt1 = oracle.num_tiles(hi - lo)
+        tab1 = w1[64 + 16: 64 + 16 + 2 * nt1].view(np.uint16)
+        assert np.array_equal(tab[c * tpc: c * tpc + nt1], tab1), f"chunk {c}: tile table"
+
+
+def sample_chunks(nc, k, seed):
+    rng = np.random.default_rng(seed)
+    s = {0, 1, nc - 2, nc - 1} | set(int(x) for x in rng.integers(0, nc, k))
+    return sorted(c for c in s if 0 <= c < nc)
+
+
+def test_engine_cache_full_move_sampled_against_oracle():
+    cfg = inputs.CONFIGS["engine"]
+    cur = inputs.make_cache(cfg, "cuda")
+    job = Job(cfg.nbytes, cfg.chunk_bytes)
+    crc_a = torch.zeros(job.nc, dtype=torch.int32, device="cuda")
+    crc_b = torch.zeros(job.nc, dtype=torch.int32, device="cuda")
+    wm.wm_checksum(cur, job.chunk, crc_a, job.ws)
+    wm.wm_encode(cur, job.chunk, None, crc_b, job.wire, job.ws, job.res_e)
+    r = wm.read_result(job.res_e)
+    assert r.ok and r.n_present == job.nc
+    assert torch.equal(crc_a, crc_b)
+    m, hdr, off, ln, crc, tab = job.meta()
+    assert np.array_equal(crc, crc_a.cpu().numpy().view(np.uint32))
+    present = np.ones(job.nc, dtype=np.uint64)
+    check_meta_against_oracle(job, m, hdr, off, ln, crc, present)
+    assert r.wire_len == int(hdr[40:48].view(np.uint64)[0]) and r.cache_crc == int(hdr[48:52].view(np.uint32)[0])
+    assert 0.70 < r.wire_len / job.n < 0.80        # the exponent plane carries the saving
+    check_chunks_against_oracle(job, cur, sample_chunks(job.nc, 10, 1), off, ln, crc, tab)
+
+    shadow = torch.zeros(job.n, dtype=torch.uint8, device="cuda")
+    crc_dst = torch.zeros(job.nc, dtype=torch.int32, device="cuda")
+    wm.wm_decode_verify(job.wire, r.wire_len, shadow, job.chunk, crc_dst, job.ws, job.res_d)
+    rd = wm.read_result(job.res_d)
+    assert rd.ok and rd.cache_crc == r.cache_crc and rd.n_present == job.nc
+    assert torch.equal(shadow, cur) and torch.equal(crc_dst, crc_b)
+
+
+def test_random_cache_takes_the_raw_path_and_a_flipped_bit_is_rejected():
+    cfg = inputs.CONFIGS["random"]
+    cur = inputs.make_cache(cfg, "cuda")
+    job = Job(cfg.nbytes, cfg.chunk_bytes)
+    crc = torch.zeros(job.nc, dtype=torch.int32, device="cuda")
+    wm.wm_encode(cur, job.chunk, None, crc, job.wire, job.ws, job.res_e)
+    r = wm.read_result(job.res_e)
+    assert r.ok
+    m, hdr, off, ln, dcrc, tab = job.meta()
+    # incompressible data: every tile raw, the image is the cache plus its metadata and no more
+    assert (tab == 512).all()
+    assert r.payload_bytes == job.n and r.wire_len == job.meta_end + job.n
+    assert (ln == job.chunk).all()
+    check_meta_against_oracle(job, m, hdr, off, ln, dcrc, np.ones(job.nc, dtype=np.uint64))
+    check_chunks_against_oracle(job, cur, sample_chunks(job.nc, 4, 2), off, ln, dcrc, tab)
+
+    shadow = torch.zeros(job.n, dtype=torch.uint8, device="cuda")
+    crc_dst = torch.zeros(job.nc, dtype=torch.int32, device="cuda")
+    wm.wm_decode_verify(job.wire, r.wire_len, shadow, job.chunk, crc_dst, job.ws, job.res_d)
+    assert wm.read_result(job.res_d).ok and torch.equal(shadow, cur) and torch.equal(crc_dst, crc)
+
+    # one flipped payload bit: the chunk that holds it is named, and no checksum is installed
+    bad_chunk = 611
+    pos = job.meta_end + bad_chunk * job.chunk + 123457
+    job.wire[pos] ^= 0x10
+    crc_dst.fill_(77)
+    wm.wm_decode_verify(job.wire, r.wire_len, shadow, job.chunk, crc_dst, job.ws, job.res_d)
+    rd = wm.read_result(job.res_d)
+    assert rd.status_name == "ERR_CHUNK_CRC" and rd.first_bad_chunk == bad_chunk and rd.n_bad_chunks == 1
+    assert (crc_dst == 77).all()
+    job.wire[pos] ^= 0x10
+    # one flipped metadata bit (a directory length): stopped at the metadata CRC
+    job.wire[64 + 16 * 5 + 8] ^= 0x01
+    wm.wm_decode_verify(job.wire, r.wire_len, shadow, job.chunk, crc_dst, job.ws, job.res_d)
+    assert wm.read_result(job.res_d).status_name == "ERR_META_CRC"
+    assert (crc_dst == 77).all()
+    job.wire[64 + 16 * 5 + 8] ^= 0x01
+    wm.wm_decode_verify(job.wire, r.wire_len, shadow, job.chunk, crc_dst, job.ws, job.res_d)
+    assert wm.read_result(job.res_d).ok and torch.equal(crc_dst, crc)
+
+
+def test_long_context_cache_beyond_4gib_offsets():
+    """17 GB cache: payload offsets and tile numbers pass 2^32 bytes / 2^20 tiles."""
+    cfg = inputs.CONFIGS["long"]
+    free, _ = torch.cuda.mem_get_info()
+    if free < 4 * cfg.nbytes:
+        pytest.skip("not enough free device memory for the long-context cache")
+    cur = inputs.make_cache(cfg, "cuda")
+    job = Job(cfg.nbytes, cfg.chunk_bytes)
+    crc_a = torch.zeros(job.nc, dtype=torch.int32, device="cuda")
+    crc_b = torch.zeros(job.nc, dtype=torch.int32, device="cuda")
+    wm.wm_checksum(cur, job.chunk, crc_a, job.ws)
+    wm.wm_encode(cur, job.chunk, None, crc_b, job.wire, job.ws, job.res_e)
+    r = wm.read_result(job.res_e)
+    assert r.ok and torch.equal(crc_a, crc_b)
+    assert r.payload_bytes > (1 << 32)
+    m, hdr, off, ln, crc, tab = job.meta()
+    check_meta_against_oracle(job, m, hdr, off, ln, crc, np.ones(job.nc, dtype=np.uint64))
+    # chunks on both sides of the 4 GiB payload offset, and the ends
+    k = int(np.searchsorted(off, 1 << 32))
+    check_chunks_against_oracle(job, cur, sorted({0, k - 1, k, k + 1, job.nc - 1}), off, ln, crc, tab)
+    shadow = torch.zeros(job.n, dtype=torch.uint8, device="cuda")
+    crc_dst = torch.zeros(job.nc, dtype=torch.int32, device="cuda")
+    wm.wm_decode_verify(job.wire, r.wire_len, shadow, job.chunk, crc_dst, job.ws, job.res_d)
+    assert wm.read_result(job.res_d).ok
+    assert torch.equal(shadow, cur) and torch.equal(crc_dst, crc_b)
+
+
+def test_precopy_step_loop_on_two_streams():
+    """Twenty generation steps of the engine cache.  Source stream: rewrite three quarters of the
+    chunks, diff against the last snapshot, encode only the dirty chunks.  Destination stream:
+    decode, verify, install into the destination copy while the source already works on the
+    next step.  After every step the destination must equal the source's snapshot."""
+    cfg = inputs.CONFIGS["engine"]
+    steps = 20
+    cur = inputs.make_cache(cfg, "cuda")
+    job = Job(cfg.nbytes, cfg.chunk_bytes)
+    wires = [job.wire, torch.empty_like(job.wire)]
+    src, dstream = torch.cuda.Stream(), torch.cuda.Stream()
+    res_d = [wm.new_result(), wm.new_result()]
+    crc_src = torch.zeros(job.nc, dtype=torch.int32, device="cuda")
+    crc_dst = torch.zeros(job.nc, dtype=torch.int32, device="cuda")
+    dirty = torch.zeros(job.nc, dtype=torch.uint8, device="cuda")
+    idx = torch.zeros(job.nc, dtype=torch.int32, device="cuda")
+    n_dirty = torch.zeros(1, dtype=torch.int32, device="cuda")
+
+    # step 0 of the protocol: a full move brings the destination level with the source
+    wm.wm_encode(cur, job.chunk, None, crc_src, wires[0], job.ws, job.res_e)
+    r = wm.read_result(job.res_e)
+    dst = torch.zeros(job.n, dtype=torch.uint8, device="cuda")
+    wm.wm_decode_verify(wires[0], r.wire_len, dst, job.chunk, crc_dst, job.ws, job.res_d)
+    assert r.ok and wm.read_result(job.res_d).ok and torch.equal(dst, cur)
+    prev = cur.clone()
+    torch.cuda.synchronize()
+
+    oracle_steps = {0, 7, 19}
+    pending = None                       # (step, result record) of the decode still in flight
+    for k in range(steps):
+        mask = inputs.step_pattern(job.nc, cfg.shape[0], 0.75, seed=1000 + k)
+        wire = wires[(k + 1) % 2]
+        with torch.cuda.stream(src):
+            inputs.apply_step(cur, job.chunk, mask, seed=5000 + k)
+            wm.wm_dirty_diff(cur, prev, job.chunk, dirty, idx, n_dirty, job.ws, stream=src)
+            wm.wm_encode(cur, job.chunk, dirty, crc_src, wire, job.ws, job.res_e, stream=src)
+            r = wm.read_result(job.res_e)                  # waits for the source stream only
+            nd = int(n_dirty.item())
+            assert r.ok and r.n_present == nd == int(mask.sum())
+            assert torch.equal(dirty.cpu(), mask)
+            assert torch.equal(idx[:nd].cpu().long(), torch.nonzero(mask).flatten())
+            if k in oracle_steps:
+                job.wire = wire
+                m, hdr, off, ln, crc, tab = job.meta()
+                present = mask.numpy().astype(np.uint64)
+                check_meta_against_oracle(job, m, hdr, off, ln, crc, present)
+                some = [int(c) for c in torch.nonzero(mask).flatten()[[0, nd // 2, nd - 1]]]
+                check_chunks_against_oracle(job, cur, some, off, ln, crc, tab)
+                absent = [int(c) for c in torch.nonzero(mask == 0).flatten()[:2]]
+                tpc = job.chunk // TILE
+                for c in absent:
+                    assert (tab[c * tpc:(c + 1) * tpc] == 0).all()
+            encoded = torch.cuda.Event()
+            encoded.record(src)
+        if pending is not None:
+            # the previous step's install ran beside this step's source work; settle it now
+            dstream.synchronize()
+            pk, rec = pending
+            rd = wm.read_result(rec)
+            assert rd.ok, f"step {pk}: {rd.status_name}"
+            assert torch.equal(dst, prev), f"step {pk}: destination differs from the snapshot"
+            assert torch.equal(crc_dst, crc_prev)
+        with torch.cuda.stream(src):
+            prev.copy_(cur, non_blocking=True)             # snapshot for the next diff
+            crc_prev = crc_src.clone()
+            snap = torch.cuda.Event()
+            snap.record(src)
+        with torch.cuda.stream(dstream):
+            dstream.wait_event(encoded)
+            wm.wm_decode_verify(wire, r.wire_len, dst, job.chunk, crc_dst, job.ws2, res_d[k % 2], stream=dstream)
+        pending = (k, res_d[k % 2])
+        snap.synchronize()
+    dstream.synchronize()
+    rd = wm.read_result(pending[1])
+    assert rd.ok and torch.equal(dst, cur) and torch.equal(crc_dst, crc_src)
