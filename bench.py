@@ -26,8 +26,10 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 
 FALLBACK_HBM_GBS = 6650.0
-# DRAM bytes per launch of the dominant kernel from an ncu capture (profiles/), or None.
-NCU_TRAFFIC_BYTES = {}
+# DRAM bytes read + written per launch of the encode kernel, from single-pass ncu captures of this
+# benchmark (dram__bytes_read.sum + dram__bytes_write.sum; summaries under profiles/).  A workload
+# without a capture reports null.
+NCU_TRAFFIC_BYTES = {"engine": 1671874432 + 1207008896, "engine_256m": 262465024 + 144592896}
 
 
 # the headline metric as the baseline file words it; a step is one pass of the whole path:
