@@ -7,7 +7,7 @@
 //                      scanner warp turns them into payload offsets) -> k_encode_finish (directory, cache CRC, header)
 //                      -> k_meta_crc (metadata CRC, result)
 //   wm_decode_verify : k_decode_init -> k_meta_crc (header + metadata CRC gate)
-//                      -> k_decode_struct_chunks -> k_decode_struct_scan (structure gate)
+//                      -> k_decode_struct (structure gate)
 //                      -> k_decode (unpack + CRC of decoded bytes) -> k_decode_finish
 #include <cstdint>
 #include <cstdio>
@@ -38,6 +38,17 @@ struct Geo {
     uint32_t n_meta_slices;   // ceil(meta_end / 16384)
     uint32_t tpc_shift;       // log2(tiles_per_chunk) when that is a power of two, else 32
     uint32_t n_full_tiles;    // tiles of exactly 16384 bytes
+    uint32_t finish_cb;       // chunks handled by one block of the finish kernels
+};
+
+// Powers of k_chunk = x^(8 chunk_bytes), by 7-bit digit of the exponent: k_chunk^e is the product
+// of d0[e & 127], d1[(e >> 7) & 127], d2[(e >> 14) & 127] and, beyond 2^21 chunks, of the
+// squares hi[j] = k_chunk^(2^(21+j)) that the remaining bits select.  Built on the host once per
+// geometry and handed to the finish kernels as an argument.
+struct ChunkPowers {
+    uint32_t d0[128], d1[128], d2[128];
+    uint32_t hi[11];
+    uint32_t pad;
 };
 
 struct Ctrl {                 // first 256 bytes of the workspace
@@ -56,7 +67,9 @@ struct Ctrl {                 // first 256 bytes of the workspace
     unsigned long long bad4_key;   // lowest failing tile * 2 + (1 if STRUCT)
     unsigned long long payload_total;
     uint32_t hdr_n_present, hdr_cache_crc;
-    uint32_t pad[42];
+    uint32_t cache_acc;       // XOR of the chunks' terms of the whole-cache CRC
+    uint32_t done_c;
+    uint32_t pad[40];
 };
 static_assert(sizeof(Ctrl) == 256, "control block is 256 bytes");
 
@@ -111,11 +124,19 @@ static Ws ws_carve(void* base, const Geo& g)
 // never longer than the cache, so the codec entry points take caches up to 32 GiB.
 constexpr uint64_t kMaxCodecBytes = 32ull << 30;
 
+constexpr uint32_t kFinishDigests = 8192;    // tile digests a finish block stages in shared memory
+constexpr uint32_t kFinishChunks = 128;      // at most this many chunks per finish block
+
 static bool make_geo(uint64_t nbytes, uint32_t chunk_bytes, Geo& g)
 {
     if (nbytes == 0 || chunk_bytes == 0 || chunk_bytes % kTile != 0 || chunk_bytes > (1u << 30)) return false;
     uint64_t nt = (nbytes + kTile - 1) / kTile;
     if (nt > 0xFFFFFFFFull) return false;
+    // the powers below cost a few microseconds of host time: keep the last geometry per thread
+    static thread_local Geo last;
+    static thread_local bool have_last = false;
+    if (have_last && last.nbytes == nbytes && last.chunk_bytes == chunk_bytes) { g = last; return true; }
+    have_last = false;
     g.nbytes = nbytes;
     g.chunk_bytes = chunk_bytes;
     g.tiles_per_chunk = chunk_bytes / kTile;
@@ -132,7 +153,32 @@ static bool make_geo(uint64_t nbytes, uint32_t chunk_bytes, Geo& g)
     g.tpc_shift = 32;
     for (uint32_t k = 0; k < 32; k++)
         if (g.tiles_per_chunk == (1u << k)) g.tpc_shift = k;
+    uint32_t cb = kFinishDigests / g.tiles_per_chunk;
+    g.finish_cb = cb > kFinishChunks ? kFinishChunks : (cb ? cb : 1u);
+    last = g;
+    have_last = true;
     return true;
+}
+
+// The powers for g (kept per thread for the last chunk size: about 400 products to build).
+static const ChunkPowers& chunk_powers(const Geo& g)
+{
+    static thread_local ChunkPowers cp;
+    static thread_local uint32_t for_k = 0;
+    static thread_local bool have = false;
+    if (have && for_k == g.k_chunk) return cp;
+    uint32_t step = g.k_chunk;
+    uint32_t* digit[3] = {cp.d0, cp.d1, cp.d2};
+    for (int d = 0; d < 3; d++) {
+        uint32_t v = 0x80000000u;                       // the polynomial 1
+        for (int i = 0; i < 128; i++) { digit[d][i] = v; v = mulmod(v, step); }
+        step = v;                                       // step^128
+    }
+    for (int j = 0; j < 11; j++) { cp.hi[j] = step; step = mulmod(step, step); }
+    cp.pad = 0;
+    for_k = g.k_chunk;
+    have = true;
+    return cp;
 }
 
 __device__ __forceinline__ uint32_t chunk_of(const Geo& g, uint32_t t)
@@ -215,66 +261,76 @@ __device__ __forceinline__ void load_ht_t0(uint32_t* sHT, uint32_t* sT0, const T
     __syncthreads();
 }
 
-constexpr uint32_t kFinishChunks = 128;      // chunks folded per block of the finish kernels
+// Finish blocks: a block owns g.finish_cb consecutive chunks.  Their tiles' digests are one
+// contiguous run, copied to shared memory with coalesced loads (one round trip to L2 for the
+// block instead of one per few digests of a serial fold); thread i then folds chunk c0 + i out
+// of shared memory.  A chunk's digests sit at stride tiles_per_chunk + 1 so that the threads'
+// reads fall on different banks.  Chunks with more tiles than the stage holds are folded
+// from global memory.  Block-wide: every thread calls; ends with a block barrier.
+struct FinishStage {
+    uint32_t dig[kFinishDigests + kFinishChunks];
+};
 
-// Table of products with one fixed multiplier M (block of 1024 threads; ends with a block
-// barrier): tab[256 k + v] = (v << 8k) * M, so that a * M is four lookups.
-__device__ void build_mul_table(uint32_t* tab, uint32_t M)
+__device__ void stage_chunk_digests(const Geo& g, FinishStage& st, const uint32_t* __restrict__ dig, uint32_t c0)
 {
-    const uint32_t k = threadIdx.x >> 8, v = threadIdx.x & 255u;
-    // bit 8k+j of (v << 8k) is the coefficient of x^(31-8k-j): start at M x^(24-8k) for j = 7
-    uint32_t b = M;
-    for (uint32_t i = 0; i < 24u - 8u * k; i++) b = (b >> 1) ^ (kPolyReflected & (0u - (b & 1u)));
-    uint32_t r = 0;
-#pragma unroll
-    for (int j = 7; j >= 0; j--) {
-        r ^= b & (0u - ((v >> j) & 1u));
-        b = (b >> 1) ^ (kPolyReflected & (0u - (b & 1u)));
+    const uint32_t tpc = g.tiles_per_chunk;
+    if (tpc <= kFinishDigests) {
+        const uint64_t t0 = (uint64_t)c0 * tpc;
+        uint64_t t1 = t0 + (uint64_t)g.finish_cb * tpc;
+        if (t1 > g.n_tiles) t1 = g.n_tiles;
+        for (uint32_t i = threadIdx.x; t0 + i < t1; i += blockDim.x) {
+            const uint32_t ch = g.tpc_shift < 32 ? i >> g.tpc_shift : i / tpc;
+            st.dig[i + ch] = __ldcg(dig + t0 + i);          // ch * (tpc + 1) + (i - ch * tpc)
+        }
     }
-    tab[threadIdx.x] = r;
     __syncthreads();
 }
-__device__ __forceinline__ uint32_t mul_by_table(const uint32_t* tab, uint32_t a)
+
+// CRC32C of chunk c = c0 + i from the staged digests (Horner over tiles; the all-ones start
+// value was folded into the first tile's digest, the final complement is applied here).
+__device__ uint32_t chunk_crc_staged(const Geo& g, const uint32_t* HT, const uint32_t* T0, const FinishStage& st,
+                                     const uint32_t* dig, const unsigned char* bytes, uint32_t c, uint32_t i)
 {
-    return tab[a & 0xFF] ^ tab[256 + ((a >> 8) & 0xFF)] ^ tab[512 + ((a >> 16) & 0xFF)] ^ tab[768 + (a >> 24)];
+    if (g.tiles_per_chunk > kFinishDigests) return chunk_crc_from_digests(g, HT, T0, dig, bytes, c);
+    const uint64_t clen = chunk_len_dev(g, c);
+    if (clen < 4) return crc_bytewise(T0, bytes + (uint64_t)c * g.chunk_bytes, (uint32_t)clen);
+    const uint32_t ntc = (uint32_t)((clen + kTile - 1) / kTile);
+    const bool ragged = (clen % kTile) != 0;
+    const uint32_t* d = st.dig + (size_t)i * (g.tiles_per_chunk + 1u);
+    uint32_t s = 0;
+    const uint32_t n_plain = ragged ? ntc - 1 : ntc;
+    for (uint32_t k = 0; k < n_plain; k++) s = advance_tile(HT, s) ^ d[k];
+    if (ragged) s = mulmod_dev(s, g.k_tail) ^ d[ntc - 1];
+    return ~s;
 }
 
-// CRC32C of the concatenation of all chunks from their finished CRCs (block-wide; every
-// thread of a 1024-thread block must call).  crc(A||B) = crc(A) x^(8 len B) + crc(B).
-// Each thread folds a run of chunks, then a tree folds the runs; every product is with a
-// multiplier shared by the whole block, so it goes through a table built for that multiplier.
-// stab: 1024 words for the table, sbuf: 1024 words.
-__device__ uint32_t combine_chunk_crcs(const Geo& g, const uint32_t* crc, uint32_t stride_words, uint32_t* stab,
-                                       uint32_t* sbuf)
+// Chunk c's term of the whole-cache CRC: crc(A || B) = crc(A) x^(8 len B) + crc(B), so the CRC
+// of all chunks in a row is the sum over chunks of crc_c times x^(8 * bytes after chunk c).
+// Every chunk but the last has the same length: the factor is k_last_chunk * k_chunk^e with
+// e = number of full chunks after c.
+__device__ uint32_t cache_crc_term(const Geo& g, const ChunkPowers& cp, uint32_t crc, uint32_t c)
 {
-    const uint32_t n = g.n_chunks;
-    if (n == 1) return __ldcg(&crc[0]);
-    const uint32_t m = n - 1;                       // chunks of full length
-    const uint32_t T = blockDim.x;                  // 1024
-    const uint32_t R = (m + T - 1) / T;             // run per thread
-    const uint64_t pad = (uint64_t)T * R - m;       // leading empty slots
-    build_mul_table(stab, g.k_chunk);
-    uint32_t acc = 0, M = 0x80000000u;              // M becomes k_chunk^R
-    for (uint32_t s = 0; s < R; s++) {
-        uint64_t slot = (uint64_t)threadIdx.x * R + s;
-        uint32_t v = slot >= pad ? __ldcg(&crc[(slot - pad) * stride_words]) : 0u;
-        acc = mul_by_table(stab, acc) ^ v;
-        M = mul_by_table(stab, M);
-    }
-    sbuf[threadIdx.x] = acc;
+    if (c + 1 == g.n_chunks) return crc;
+    uint32_t e = g.n_chunks - 2u - c;
+    uint32_t f = mulmod_dev(crc, g.k_last_chunk);
+    if (e & 127u) f = mulmod_dev(f, cp.d0[e & 127u]);
+    if ((e >> 7) & 127u) f = mulmod_dev(f, cp.d1[(e >> 7) & 127u]);
+    if ((e >> 14) & 127u) f = mulmod_dev(f, cp.d2[(e >> 14) & 127u]);
+    e >>= 21;
+    for (uint32_t j = 0; e; j++, e >>= 1)
+        if (e & 1u) f = mulmod_dev(f, cp.hi[j]);
+    return f;
+}
+
+// XOR the threads' terms into ctrl->cache_acc (block-wide; one atomic per block).
+__device__ void accumulate_cache_crc(Ctrl* ctrl, uint32_t term, uint32_t* s_acc)
+{
+    if (threadIdx.x == 0) *s_acc = 0;
     __syncthreads();
-    for (uint32_t width = T / 2; width >= 1; width >>= 1) {
-        build_mul_table(stab, M);
-        uint32_t v = 0;
-        if (threadIdx.x < width) v = mul_by_table(stab, sbuf[2 * threadIdx.x]) ^ sbuf[2 * threadIdx.x + 1];
-        M = mul_by_table(stab, M);
-        __syncthreads();
-        if (threadIdx.x < width) sbuf[threadIdx.x] = v;
-        __syncthreads();
-    }
-    uint32_t fold = sbuf[0];
+    const uint32_t w = __reduce_xor_sync(0xFFFFFFFFu, term);
+    if ((threadIdx.x & 31u) == 0 && w) atomicXor(s_acc, w);
     __syncthreads();
-    return mulmod_dev(fold, g.k_last_chunk) ^ __ldcg(&crc[(uint64_t)m * stride_words]);
+    if (threadIdx.x == 0 && *s_acc) atomicXor(&ctrl->cache_acc, *s_acc);
 }
 
 // ------------------------------------------------------------------ wm_checksum
@@ -338,14 +394,19 @@ k_tile_digests(const unsigned char* __restrict__ cache, Geo g, Ws ws, const Tabl
     }
 }
 
-__global__ void k_checksum_finish(const unsigned char* __restrict__ cache, Geo g, Ws ws,
-                                  const Tables* __restrict__ tab, uint32_t* __restrict__ crc_out)
+__global__ void __launch_bounds__(1024)
+k_checksum_finish(const unsigned char* __restrict__ cache, Geo g, Ws ws, const Tables* __restrict__ tab,
+                  uint32_t* __restrict__ crc_out)
 {
     __shared__ uint32_t sHT[1024];
     __shared__ uint32_t sT0[256];
+    __shared__ FinishStage stage;
     load_ht_t0(sHT, sT0, tab);
-    uint32_t c = blockIdx.x * blockDim.x + threadIdx.x;
-    if (c < g.n_chunks) crc_out[c] = chunk_crc_from_digests(g, sHT, sT0, ws.dig, cache, c);
+    const uint32_t c0 = blockIdx.x * g.finish_cb;
+    stage_chunk_digests(g, stage, ws.dig, c0);
+    const uint32_t c = c0 + threadIdx.x;
+    if (threadIdx.x < g.finish_cb && c < g.n_chunks)
+        crc_out[c] = chunk_crc_staged(g, sHT, sT0, stage, ws.dig, cache, c, threadIdx.x);
 }
 
 // ------------------------------------------------------------------ wm_dirty_diff
@@ -961,25 +1022,27 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
 __global__ void __launch_bounds__(1024)
 k_encode_finish(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restrict__ dirty,
                 uint32_t* __restrict__ crc_inout, unsigned char* __restrict__ wire, Ws ws,
-                const Tables* __restrict__ tab)
+                const Tables* __restrict__ tab, const __grid_constant__ ChunkPowers cp)
 {
     __shared__ uint32_t sHT[1024];
     __shared__ uint32_t sT0[256];
-    __shared__ uint32_t sbuf[1024];
-    __shared__ uint32_t stab[1024];
+    __shared__ FinishStage stage;
+    __shared__ uint32_t s_acc;
     __shared__ bool s_last;
     load_ht_t0(sHT, sT0, tab);
+    const uint32_t c0 = blockIdx.x * g.finish_cb;
+    stage_chunk_digests(g, stage, ws.dig, c0);
     unsigned char* dir = wire + 64;
     const unsigned long long total = ws.ctrl->payload_total;
-    // only kFinishChunks threads of a block fold chunks (the lookups of a full block would queue
-    // up on one SM's shared memory); all of them take part in the last block's combine
-    const uint32_t c = blockIdx.x * kFinishChunks + threadIdx.x;
-    uint32_t present = 0;
-    if (threadIdx.x < kFinishChunks && c < g.n_chunks) {
+    // only finish_cb threads of a block fold chunks (the lookups of a full block would queue up
+    // on one SM's shared memory)
+    const uint32_t c = c0 + threadIdx.x;
+    uint32_t present = 0, term = 0;
+    if (threadIdx.x < g.finish_cb && c < g.n_chunks) {
         present = (!dirty || dirty[c]) ? 1u : 0u;
         uint32_t crc;
         if (present) {
-            crc = chunk_crc_from_digests(g, sHT, sT0, ws.dig, cache, c);
+            crc = chunk_crc_staged(g, sHT, sT0, stage, ws.dig, cache, c, threadIdx.x);
             crc_inout[c] = crc;
         } else {
             crc = crc_inout[c];
@@ -989,8 +1052,9 @@ k_encode_finish(const unsigned char* __restrict__ cache, Geo g, const uint8_t* _
                                           ? *reinterpret_cast<const unsigned long long*>(dir + 16ull * (c + 1)) : total;
         *reinterpret_cast<uint32_t*>(dir + 16ull * c + 8) = (uint32_t)(nx - po);
         *reinterpret_cast<uint32_t*>(dir + 16ull * c + 12) = crc;
+        term = cache_crc_term(g, cp, crc, c);
     }
-    __threadfence();
+    accumulate_cache_crc(ws.ctrl, term, &s_acc);
     const uint32_t cnt = __syncthreads_count(present);
     if (threadIdx.x == 0) {
         if (cnt) atomicAdd(&ws.ctrl->n_present, cnt);
@@ -998,24 +1062,22 @@ k_encode_finish(const unsigned char* __restrict__ cache, Geo g, const uint8_t* _
         s_last = atomicAdd(&ws.ctrl->done_a, 1u) == gridDim.x - 1;
     }
     __syncthreads();
-    if (!s_last) return;
+    if (!s_last || threadIdx.x != 0) return;
     __threadfence();
-    const uint32_t cache_crc = combine_chunk_crcs(g, reinterpret_cast<const uint32_t*>(dir + 12), 4, stab, sbuf);
-    if (threadIdx.x == 0) {
-        const uint32_t n_present = ld_volatile_u32(&ws.ctrl->n_present);
-        uint32_t* h = reinterpret_cast<uint32_t*>(wire);
-        h[0] = 0x31564D57u;                                  // "WMV1"
-        h[1] = 1u | ((dirty ? 1u : 0u) << 16);               // version, flags
-        h[2] = (uint32_t)g.nbytes; h[3] = (uint32_t)(g.nbytes >> 32);
-        h[4] = g.chunk_bytes; h[5] = kTile; h[6] = g.n_chunks; h[7] = n_present;
-        h[8] = (uint32_t)total; h[9] = (uint32_t)(total >> 32);
-        const unsigned long long wl = g.meta_end + total;
-        h[10] = (uint32_t)wl; h[11] = (uint32_t)(wl >> 32);
-        h[12] = cache_crc; h[13] = 0u; h[14] = 0u; h[15] = 0u;
-        ws.ctrl->hdr_cache_crc = cache_crc;
-        ws.ctrl->hdr_n_present = n_present;
-        ws.ctrl->payload_total = total;
-    }
+    const uint32_t cache_crc = ld_volatile_u32(&ws.ctrl->cache_acc);
+    const uint32_t n_present = ld_volatile_u32(&ws.ctrl->n_present);
+    uint32_t* h = reinterpret_cast<uint32_t*>(wire);
+    h[0] = 0x31564D57u;                                  // "WMV1"
+    h[1] = 1u | ((dirty ? 1u : 0u) << 16);               // version, flags
+    h[2] = (uint32_t)g.nbytes; h[3] = (uint32_t)(g.nbytes >> 32);
+    h[4] = g.chunk_bytes; h[5] = kTile; h[6] = g.n_chunks; h[7] = n_present;
+    h[8] = (uint32_t)total; h[9] = (uint32_t)(total >> 32);
+    const unsigned long long wl = g.meta_end + total;
+    h[10] = (uint32_t)wl; h[11] = (uint32_t)(wl >> 32);
+    h[12] = cache_crc; h[13] = 0u; h[14] = 0u; h[15] = 0u;
+    ws.ctrl->hdr_cache_crc = cache_crc;
+    ws.ctrl->hdr_n_present = n_present;
+    ws.ctrl->payload_total = total;
 }
 
 // CRC32C of the metadata region wire[0, meta_end) with the meta_crc field read as zero.
@@ -1036,6 +1098,7 @@ k_meta_crc(unsigned char* wire, uint64_t wire_len, Geo g, Ws ws, const Tables* _
     const uint32_t warp = tt / 32, lane = tt % 32;
     TeamCtl* tc = reinterpret_cast<TeamCtl*>(S.take(4 * sizeof(TeamCtl)));
     uint32_t* sHT = reinterpret_cast<uint32_t*>(S.take(4096));
+    uint32_t* s_dig = reinterpret_cast<uint32_t*>(S.take(4096));
     if (!S.ok) { if (threadIdx.x == 0) atomicOr(&ws.ctrl->err, 4u); return; }
     tc += team;
     sHT[threadIdx.x] = (&tab->HT[0][0])[threadIdx.x];
@@ -1098,13 +1161,20 @@ k_meta_crc(unsigned char* wire, uint64_t wire_len, Geo g, Ws ws, const Tables* _
         s_last = atomicAdd(&ws.ctrl->done_b, 1u) == gridDim.x - 1;
     }
     __syncthreads();
-    if (!s_last || threadIdx.x != 0) return;
+    if (!s_last) return;
     __threadfence();
+    // fold the slice digests: fetched 1024 at a time by the whole block (one round trip to L2
+    // per batch, not one per digest), folded by one thread out of shared memory
     uint32_t st = 0;
-    for (uint32_t i = 0; i < g.n_meta_slices; i++) {
-        st = advance_tile(sHT, st);
-        st ^= ld_volatile_u32(&ws.mdig[i]);
+    for (uint32_t b0 = 0; b0 < g.n_meta_slices; b0 += 1024) {
+        const uint32_t nb = min(1024u, g.n_meta_slices - b0);
+        __syncthreads();
+        if (threadIdx.x < nb) s_dig[threadIdx.x] = ld_volatile_u32(&ws.mdig[b0 + threadIdx.x]);
+        __syncthreads();
+        if (threadIdx.x == 0)
+            for (uint32_t i = 0; i < nb; i++) st = advance_tile(sHT, st) ^ s_dig[i];
     }
+    if (threadIdx.x != 0) return;
     const uint32_t crc = ~st;
     if (mode == 0) {
         reinterpret_cast<uint32_t*>(wire)[13] = crc;
@@ -1166,78 +1236,80 @@ __device__ __forceinline__ void fill_result(wm_result* result, const Ctrl* ctrl,
     *result = r;
 }
 
-// Step 3, per chunk (one warp each): tile entries against the chunk's length and enc_len;
-// also produces each tile's offset inside its chunk's payload.
-__global__ void __launch_bounds__(256)
-k_decode_struct_chunks(const unsigned char* __restrict__ wire, Geo g, Ws ws)
-{
-    if (ld_volatile_u32(&ws.ctrl->gate)) return;
-    const uint32_t lane = threadIdx.x % 32;
-    const uint32_t c = blockIdx.x * (blockDim.x / 32) + threadIdx.x / 32;
-    if (c >= g.n_chunks) return;
-    const unsigned char* dir = wire + 64;
-    const uint16_t* tab16 = reinterpret_cast<const uint16_t*>(wire + 64 + 16ull * g.n_chunks);
-    const uint64_t clen = chunk_len_dev(g, c);
-    const uint32_t t0 = c * g.tiles_per_chunk;
-    const uint32_t ntc = (uint32_t)((clen + kTile - 1) / kTile);
-    const uint32_t elen = *reinterpret_cast<const uint32_t*>(dir + 16ull * c + 8);
-    unsigned long long carry = 0;
-    bool ok = true, any = false, all = true;
-    for (uint32_t i0 = 0; i0 < ntc; i0 += 32) {
-        const uint32_t i = i0 + lane;
-        uint32_t len = 0;
-        bool l_ok = true, l_any = false, l_all = true;
-        if (i < ntc) {
-            const uint32_t e = tab16[t0 + i];
-            const uint64_t tl = clen - (uint64_t)i * kTile;
-            if (e == 0) l_all = false;
-            else {
-                l_any = true;
-                if (tl < kTile) { if (e != 0xFFFFu) l_ok = false; len = (uint32_t)tl; }
-                else if (e >= 258u && e <= 512u) len = 32u * e;
-                else l_ok = false;
-            }
-        }
-        uint32_t incl = len;
-#pragma unroll
-        for (int d = 1; d < 32; d <<= 1) {
-            uint32_t o = __shfl_up_sync(0xFFFFFFFFu, incl, d);
-            if (lane >= (uint32_t)d) incl += o;
-        }
-        if (i < ntc) ws.rel[t0 + i] = (uint32_t)(carry + incl - len);
-        carry += __shfl_sync(0xFFFFFFFFu, incl, 31);
-        ok = ok && __all_sync(0xFFFFFFFFu, l_ok);
-        any = any || __any_sync(0xFFFFFFFFu, l_any);
-        all = all && __all_sync(0xFFFFFFFFu, l_all);
-    }
-    if (any && !all) ok = false;
-    if (carry != elen) ok = false;
-    if (lane == 0) {
-        ws.cflag[c] = (any ? CF_PRESENT : 0u) | (ok ? 0u : CF_BAD3);
-        if (!ok) { atomicMin(&ws.ctrl->bad3_first, c); atomicAdd(&ws.ctrl->bad3_count, 1u); }
-        if (any) atomicAdd(&ws.ctrl->n_present, 1u);
-    }
-}
-
-// Step 3, across chunks (one block): payload offsets are the running sum of enc_len, the
-// totals match the header.  Sets the gate on failure.
+// Step 3.  Per chunk (one warp each): tile entries against the chunk's length and enc_len; also
+// produces each tile's offset inside its chunk's payload.  Across chunks (the last block to
+// finish): payload offsets are the running sum of enc_len and the totals match the header.
+// Sets the gate on failure.
 __global__ void __launch_bounds__(1024)
-k_decode_struct_scan(const unsigned char* __restrict__ wire, uint64_t wire_len, Geo g, Ws ws, wm_result* result)
+k_decode_struct(const unsigned char* __restrict__ wire, uint64_t wire_len, Geo g, Ws ws, wm_result* result)
 {
     if (ld_volatile_u32(&ws.ctrl->gate)) return;
     __shared__ unsigned long long s_warp[32];
     __shared__ unsigned long long s_carry;
     __shared__ uint32_t s_first, s_count;
-    const unsigned char* dir = wire + 64;
+    __shared__ bool s_last;
     const uint32_t lane = threadIdx.x % 32, warp = threadIdx.x / 32;
-    if (threadIdx.x == 0) { s_carry = 0; s_first = 0xFFFFFFFFu; s_count = 0; }
+    const unsigned char* dir = wire + 64;
+    const uint16_t* tab16 = reinterpret_cast<const uint16_t*>(wire + 64 + 16ull * g.n_chunks);
+    const uint32_t c = blockIdx.x * 32u + warp;
+    if (c < g.n_chunks) {
+        const uint64_t clen = chunk_len_dev(g, c);
+        const uint32_t t0 = c * g.tiles_per_chunk;
+        const uint32_t ntc = (uint32_t)((clen + kTile - 1) / kTile);
+        const uint32_t elen = *reinterpret_cast<const uint32_t*>(dir + 16ull * c + 8);
+        unsigned long long carry = 0;
+        bool ok = true, any = false, all = true;
+        for (uint32_t i0 = 0; i0 < ntc; i0 += 32) {
+            const uint32_t i = i0 + lane;
+            uint32_t len = 0;
+            bool l_ok = true, l_any = false, l_all = true;
+            if (i < ntc) {
+                const uint32_t e = tab16[t0 + i];
+                const uint64_t tl = clen - (uint64_t)i * kTile;
+                if (e == 0) l_all = false;
+                else {
+                    l_any = true;
+                    if (tl < kTile) { if (e != 0xFFFFu) l_ok = false; len = (uint32_t)tl; }
+                    else if (e >= 258u && e <= 512u) len = 32u * e;
+                    else l_ok = false;
+                }
+            }
+            uint32_t incl = len;
+#pragma unroll
+            for (int d = 1; d < 32; d <<= 1) {
+                uint32_t o = __shfl_up_sync(0xFFFFFFFFu, incl, d);
+                if (lane >= (uint32_t)d) incl += o;
+            }
+            if (i < ntc) ws.rel[t0 + i] = (uint32_t)(carry + incl - len);
+            carry += __shfl_sync(0xFFFFFFFFu, incl, 31);
+            ok = ok && __all_sync(0xFFFFFFFFu, l_ok);
+            any = any || __any_sync(0xFFFFFFFFu, l_any);
+            all = all && __all_sync(0xFFFFFFFFu, l_all);
+        }
+        if (any && !all) ok = false;
+        if (carry != elen) ok = false;
+        if (lane == 0) {
+            ws.cflag[c] = (any ? CF_PRESENT : 0u) | (ok ? 0u : CF_BAD3);
+            if (!ok) { atomicMin(&ws.ctrl->bad3_first, c); atomicAdd(&ws.ctrl->bad3_count, 1u); }
+            if (any) atomicAdd(&ws.ctrl->n_present, 1u);
+        }
+    }
+    __threadfence();
     __syncthreads();
+    if (threadIdx.x == 0) {
+        s_carry = 0; s_first = 0xFFFFFFFFu; s_count = 0;
+        __threadfence();
+        s_last = atomicAdd(&ws.ctrl->done_c, 1u) == gridDim.x - 1;
+    }
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
     for (uint32_t base = 0; base < g.n_chunks; base += 1024) {
-        const uint32_t c = base + threadIdx.x;
+        const uint32_t cc = base + threadIdx.x;
         unsigned long long len = 0, po = 0;
-        if (c < g.n_chunks) {
-            po = *reinterpret_cast<const unsigned long long*>(dir + 16ull * c);
-            len = *reinterpret_cast<const uint32_t*>(dir + 16ull * c + 8);
+        if (cc < g.n_chunks) {
+            po = *reinterpret_cast<const unsigned long long*>(dir + 16ull * cc);
+            len = *reinterpret_cast<const uint32_t*>(dir + 16ull * cc + 8);
         }
         unsigned long long incl = len;
 #pragma unroll
@@ -1249,11 +1321,12 @@ k_decode_struct_scan(const unsigned char* __restrict__ wire, uint64_t wire_len, 
         __syncthreads();
         unsigned long long before = s_carry;
         for (uint32_t w2 = 0; w2 < warp; w2++) before += s_warp[w2];
-        if (c < g.n_chunks && po != before + incl - len) {
+        if (cc < g.n_chunks && po != before + incl - len) {
             // a chunk already counted by the per-chunk pass must not be counted twice
-            if (!(ws.cflag[c] & CF_BAD3)) {
-                ws.cflag[c] |= CF_BAD3;
-                atomicMin(&s_first, c);
+            const uint32_t fl = ld_volatile_u32(&ws.cflag[cc]);
+            if (!(fl & CF_BAD3)) {
+                ws.cflag[cc] = fl | CF_BAD3;
+                atomicMin(&s_first, cc);
                 atomicAdd(&s_count, 1u);
             }
         }
@@ -1266,9 +1339,10 @@ k_decode_struct_scan(const unsigned char* __restrict__ wire, uint64_t wire_len, 
         __syncthreads();
     }
     if (threadIdx.x == 0) {
-        uint32_t first = min(s_first, ws.ctrl->bad3_first);
-        uint32_t count = s_count + ws.ctrl->bad3_count;
-        if (count == 0 && (s_carry != ws.ctrl->payload_total || ws.ctrl->n_present != ws.ctrl->hdr_n_present)) {
+        uint32_t first = min(s_first, ld_volatile_u32(&ws.ctrl->bad3_first));
+        uint32_t count = s_count + ld_volatile_u32(&ws.ctrl->bad3_count);
+        if (count == 0 && (s_carry != ws.ctrl->payload_total ||
+                           ld_volatile_u32(&ws.ctrl->n_present) != ws.ctrl->hdr_n_present)) {
             first = 0; count = 1;
         }
         if (count) {
@@ -1518,33 +1592,37 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
 __global__ void __launch_bounds__(1024)
 k_decode_finish(const unsigned char* __restrict__ wire, uint64_t wire_len, Geo g,
                 const unsigned char* __restrict__ dst, uint32_t* __restrict__ dst_crc, Ws ws,
-                const Tables* __restrict__ tab, wm_result* result)
+                const Tables* __restrict__ tab, wm_result* result, const __grid_constant__ ChunkPowers cp)
 {
     if (ld_volatile_u32(&ws.ctrl->gate)) return;
     __shared__ uint32_t sHT[1024];
     __shared__ uint32_t sT0[256];
-    __shared__ uint32_t sbuf[1024];
-    __shared__ uint32_t stab[1024];
+    __shared__ FinishStage stage;
+    __shared__ uint32_t s_acc;
     __shared__ bool s_last;
     __shared__ int s_status;
     load_ht_t0(sHT, sT0, tab);
+    const uint32_t c0 = blockIdx.x * g.finish_cb;
+    stage_chunk_digests(g, stage, ws.dig, c0);
     const unsigned char* dir = wire + 64;
-    const uint32_t c = blockIdx.x * kFinishChunks + threadIdx.x;
+    const uint32_t c = c0 + threadIdx.x;
     const bool step4_failed = ld_volatile_u32(reinterpret_cast<const uint32_t*>(&ws.ctrl->bad4_key)) != 0xFFFFFFFFu ||
                               ld_volatile_u32(reinterpret_cast<const uint32_t*>(&ws.ctrl->bad4_key) + 1) != 0xFFFFFFFFu;
-    if (threadIdx.x < kFinishChunks && c < g.n_chunks) {
+    uint32_t term = 0;
+    if (threadIdx.x < g.finish_cb && c < g.n_chunks) {
         const uint32_t fl = ws.cflag[c];
         const uint32_t want = *reinterpret_cast<const uint32_t*>(dir + 16ull * c + 12);
         if (step4_failed) {
             if (fl & CF_BAD4) { atomicMin(&ws.ctrl->bad4_first, c); atomicAdd(&ws.ctrl->bad4_count, 1u); }
         } else if (fl & CF_PRESENT) {
-            const uint32_t got = chunk_crc_from_digests(g, sHT, sT0, ws.dig, dst, c);
+            const uint32_t got = chunk_crc_staged(g, sHT, sT0, stage, ws.dig, dst, c, threadIdx.x);
             if (got != want) { atomicMin(&ws.ctrl->bad5_first, c); atomicAdd(&ws.ctrl->bad5_count, 1u); }
         } else {
             if (dst_crc[c] != want) { atomicMin(&ws.ctrl->bad6_first, c); atomicAdd(&ws.ctrl->bad6_count, 1u); }
         }
+        term = cache_crc_term(g, cp, want, c);
     }
-    __threadfence();
+    accumulate_cache_crc(ws.ctrl, term, &s_acc);
     __syncthreads();
     if (threadIdx.x == 0) {
         __threadfence();
@@ -1553,8 +1631,8 @@ k_decode_finish(const unsigned char* __restrict__ wire, uint64_t wire_len, Geo g
     __syncthreads();
     if (!s_last) return;
     __threadfence();
-    const uint32_t cache_crc = combine_chunk_crcs(g, reinterpret_cast<const uint32_t*>(dir + 12), 4, stab, sbuf);
     if (threadIdx.x == 0) {
+        const uint32_t cache_crc = ld_volatile_u32(&ws.ctrl->cache_acc);
         int status = WM_OK;
         uint32_t first = 0, count = 0;
         const unsigned long long key = *reinterpret_cast<volatile unsigned long long*>(&ws.ctrl->bad4_key);
@@ -1702,7 +1780,7 @@ wm_status wm_checksum(const void* cache, uint64_t nbytes, uint32_t chunk_bytes, 
         MainKernelTimer timer(ds, 0, s);
         k_tile_digests<kTeamsPlain><<<grid, kTeamsPlain * 256, kDynSmem, s>>>(c, g, ws, ds->tables);
     }
-    k_checksum_finish<<<(g.n_chunks + 255) / 256, 256, 0, s>>>(c, g, ws, ds->tables, crc_out);
+    k_checksum_finish<<<(g.n_chunks + g.finish_cb - 1) / g.finish_cb, 1024, 0, s>>>(c, g, ws, ds->tables, crc_out);
     g_launches = 2;
     return launch_status();
 }
@@ -1771,7 +1849,7 @@ wm_status wm_checksum_noalloc(const void* cache, uint64_t nbytes, uint32_t chunk
     const uint32_t need = (g.n_tiles + kTeamsPlain - 1) / kTeamsPlain;
     const uint32_t grid = need < (uint32_t)ns->sm_count ? need : (uint32_t)ns->sm_count;
     k_tile_digests<kTeamsPlain><<<grid, kTeamsPlain * 256, kDynSmem, s>>>(c, g, ws, ns->tables);
-    k_checksum_finish<<<(g.n_chunks + 255) / 256, 256, 0, s>>>(c, g, ws, ns->tables, crc_out);
+    k_checksum_finish<<<(g.n_chunks + g.finish_cb - 1) / g.finish_cb, 1024, 0, s>>>(c, g, ws, ns->tables, crc_out);
     g_launches = 2;
     return launch_status();
 }
@@ -1825,7 +1903,7 @@ wm_status wm_encode(const void* cache, uint64_t nbytes, uint32_t chunk_bytes, co
         if (dirty) k_encode<kTeams, true><<<grid, kTeams * 256, kDynSmem, s>>>(c, g, dirty, w, wire_cap, ws, ds->tables);
         else k_encode<kTeams, false><<<grid, kTeams * 256, kDynSmem, s>>>(c, g, dirty, w, wire_cap, ws, ds->tables);
     }
-    k_encode_finish<<<(g.n_chunks + kFinishChunks - 1) / kFinishChunks, 1024, 0, s>>>(c, g, dirty, crc_inout, w, ws, ds->tables);
+    k_encode_finish<<<(g.n_chunks + g.finish_cb - 1) / g.finish_cb, 1024, 0, s>>>(c, g, dirty, crc_inout, w, ws, ds->tables, chunk_powers(g));
     k_meta_crc<<<(g.n_meta_slices + 3) / 4, 1024, kDynSmem, s>>>(w, 0, g, ws, ds->tables, result, 0);
     g_launches = 4;
     return launch_status();
@@ -1849,16 +1927,15 @@ wm_status wm_decode_verify(const void* wire, uint64_t wire_len, void* dst, uint6
     // a wire shorter than the metadata is rejected by the header check before anything else is read
     const uint32_t slices = wire_len >= g.meta_end ? g.n_meta_slices : 1;
     k_meta_crc<<<(slices + 3) / 4, 1024, kDynSmem, s>>>(const_cast<unsigned char*>(w), wire_len, g, ws, ds->tables, result, 1);
-    k_decode_struct_chunks<<<(g.n_chunks + 7) / 8, 256, 0, s>>>(w, g, ws);
-    k_decode_struct_scan<<<1, 1024, 0, s>>>(w, wire_len, g, ws, result);
+    k_decode_struct<<<(g.n_chunks + 31) / 32, 1024, 0, s>>>(w, wire_len, g, ws, result);
     const uint32_t need = (g.n_tiles + kTeamsPlain - 1) / kTeamsPlain;
     const uint32_t grid = need < (uint32_t)ds->sm_count ? need : (uint32_t)ds->sm_count;
     {
         MainKernelTimer timer(ds, 3, s);
         k_decode<kTeamsPlain><<<grid, kTeamsPlain * 256, kDynSmem, s>>>(w, g, d, ws, ds->tables);
     }
-    k_decode_finish<<<(g.n_chunks + kFinishChunks - 1) / kFinishChunks, 1024, 0, s>>>(w, wire_len, g, d, dst_crc_inout, ws, ds->tables, result);
-    g_launches = 6;
+    k_decode_finish<<<(g.n_chunks + g.finish_cb - 1) / g.finish_cb, 1024, 0, s>>>(w, wire_len, g, d, dst_crc_inout, ws, ds->tables, result, chunk_powers(g));
+    g_launches = 5;
     return launch_status();
 }
 
