@@ -259,6 +259,44 @@ __device__ __forceinline__ uint64_t l2_policy_evict_first()
     return pol;
 }
 
+// ---- tensor memory as a parking place for tiles in flight ----
+// Each SM has 256 KB of tensor memory (128 lanes x 512 columns of 32 bits) next to its shared
+// memory.  Nothing here multiplies matrices, so it is free, and it takes exactly the shape of
+// what a team has to park: thread i of a warp owns lane 32 * (warp % 4) + i, and one
+// instruction moves 16 consecutive columns between that lane and 16 registers.  A tile that has
+// been measured waits there for its place in the wire image instead of being fetched again.
+// The block allocates all 512 columns once (it is alone on its SM) and must free them before
+// it exits.  All of these are warp-wide (.sync.aligned): every lane of the warp executes them.
+__device__ __forceinline__ void tmem_alloc_all(uint32_t* smem_result)
+{
+    const uint32_t a = (uint32_t)__cvta_generic_to_shared(smem_result);
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(a) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_free_all(uint32_t taddr)
+{
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_fence_before_sync() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tmem_fence_after_sync() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+
+// 16 registers -> 16 columns of this thread's lane, and back (each waits for its completion).
+__device__ __forceinline__ void tmem_store16(uint32_t taddr, const uint32_t (&w)[16])
+{
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
+                 ::"r"(taddr), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7]),
+                   "r"(w[8]), "r"(w[9]), "r"(w[10]), "r"(w[11]), "r"(w[12]), "r"(w[13]), "r"(w[14]), "r"(w[15]) : "memory");
+    asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_load16(uint32_t taddr, uint32_t (&w)[16])
+{
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+                 : "=r"(w[0]), "=r"(w[1]), "=r"(w[2]), "=r"(w[3]), "=r"(w[4]), "=r"(w[5]), "=r"(w[6]), "=r"(w[7]),
+                   "=r"(w[8]), "=r"(w[9]), "=r"(w[10]), "=r"(w[11]), "=r"(w[12]), "=r"(w[13]), "=r"(w[14]), "=r"(w[15])
+                 : "r"(taddr) : "memory");
+    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+}
+
 // A staged tile's words for this lane: word `lane` of rows 16*warp .. 16*warp+15 (conflict free).
 __device__ __forceinline__ void read_staged_words(const unsigned char* stage, uint32_t warp, uint32_t lane,
                                                   uint32_t (&w)[16])

@@ -753,16 +753,15 @@ __device__ __forceinline__ void pack_group_planes(uint32_t e4a, uint32_t e4b, ui
 //     X  measured three steps ago, packed and written to the wire image in this step
 //     V, W  measured two / one steps ago, waiting for their offsets
 //     Y  checksummed and measured in this step (its length is published at once)
-// The team owns one 16 KiB stage in shared memory that bulk copies (TMA) fill; a tile's words
-// go through it twice, once for measuring and, three steps later, once more for packing (that
-// second read comes from L2: the first one asks for evict-last priority).  Per step:
-//     read X's words from the stage | start the copy of Y | pack X straight into the wire
-//     image | read Y's words from the stage | start the copy of V (next step's X) |
-//     digest + exponent ranges of Y, publish len(Y)
-// so each copy has the other phase's work to hide behind, only 16 words per lane are live at
-// any time, and no load sits in a register waiting to be used.  Meanwhile one lane has two
-// round trips to L2 in flight whose answers are needed a step later: the ticket of the tile
-// to measure next and the offset of the tile to pack next.
+// The team owns one 16 KiB stage in shared memory that bulk copies (TMA) fill, one tile per
+// step, each copy started a whole step before its tile is needed.  A measured tile's words
+// (16 registers per lane) are parked in tensor memory until its offset is known, so a tile is
+// read from memory once and nothing waits in registers.  Per step:
+//     take Y's words from the stage | team barrier | start the copy of the next Y |
+//     digest + exponent ranges of Y, publish len(Y) | park Y | fetch X | pack X straight into
+//     the wire image
+// Meanwhile one lane has two round trips to L2 in flight whose answers are needed a step later:
+// the ticket of the tile to measure two steps on and the offset of the tile to pack next.
 // Packed data goes from registers to the wire image directly: in every region of a PACK tile
 // a lane owns an aligned unit at a lane-strided place, so each warp store is one contiguous
 // sector-aligned run.  Claiming a tile before the previous offset is known means that, if the
@@ -798,7 +797,7 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
     tc += team;
     unsigned char* dir = wire + 64;
     uint16_t* tile_tab = reinterpret_cast<uint16_t*>(wire + 64 + 16ull * g.n_chunks);
-    const uint64_t pol_keep = l2_policy_evict_last(), pol_last = l2_policy_evict_first();
+    const uint64_t pol_last = l2_policy_evict_first();     // every tile is read once
     uint32_t phase = 0;                // parity of the stage's next completion
     auto info = [&](uint32_t t) { return tile_info<MASKED>(g, dirty, t); };
     // Start the bulk copy of a full tile into the stage (call after a team barrier that
@@ -937,68 +936,66 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
         }
     };
 
+    // Tensor memory for the tiles in flight: allocated by the block's first warp, the address
+    // goes round through shared memory.  Warp w of the block owns lanes 32 (w % 4) .. + 31 and
+    // 64 columns from 64 (w / 4): four slots of 16 columns, one per tile in flight.
+    __shared__ uint32_t s_tmem;
+    if (threadIdx.x < 32) tmem_alloc_all(&s_tmem);
+    tmem_fence_before_sync();
+    __syncthreads();
+    tmem_fence_after_sync();
+    const uint32_t wc = threadIdx.x / 32;
+    const uint32_t tmem_warp = s_tmem + ((32u * (wc & 3u)) << 16) + 64u * (wc >> 2);
+
     // Tiles in flight, oldest first: X (packed in this step), V, W (waiting for their offsets),
-    // Y (measured in this step).  Ring slots: X = sl, V = sl+1, W = sl+2, Y = sl+3 (mod 8).
-    // Only the tile numbers are carried from step to step (0xFFFFFFFF: none); what follows from
-    // a number (chunk, full / ragged, present) is worked out where it is used.
+    // Y (measured in this step).  Ring slots of the widths: X = sl, V = sl+1, W = sl+2, Y = sl+3
+    // (mod 8); tensor memory slots: Y = step mod 4, X = (step + 1) mod 4 (where it was put three
+    // steps ago).  Only the tile numbers are carried from step to step (>= n_tiles: none); what
+    // follows from a number (chunk, full / ragged, present) is worked out where it is used.
     constexpr uint32_t kNone = 0xFFFFFFFFu;
     uint32_t tX = kNone, tV = kNone, tW = kNone, tY = kNone;
     uint32_t sl = 0;
     uint32_t par = 0;                  // step parity (selects next[] / excl[])
+    uint32_t step = 0;
     uint32_t d[kWordsPerLane];
     const bool leader = (warp == 0 && lane == 0);
+    uint32_t last_tk = kNone;          // leader: the ticket it claimed last
 
-    // ---- prologue: X, V, W claimed, measured and published one after the other; Y claimed;
-    // X's offset obtained; X's words requested again for the first pack
+    // ---- prologue: the tiles of the first two steps are claimed, the first one's copy started
     if (tt == 0) {
         for (int i = 0; i < 8; i++) tc->wsum[i] = 0;
         mbar_init(&tc->mbar, 1);
-        tc->next[0] = next_ticket(ws.ctrl);
-    }
-    team_bar(team);
-    tX = tc->next[0];
-    { const TileInfo i = info(tX); stage_load(i, pol_keep); stage_read(i, d); measure(i, d, 0); }
-    if (tt == 0) tc->next[1] = tX < g.n_tiles ? next_ticket(ws.ctrl) : kNone;
-    team_bar(team);
-    tV = tc->next[1];
-    { const TileInfo i = info(tV); stage_load(i, pol_keep); stage_read(i, d); measure(i, d, 1); }
-    if (tt == 0) tc->next[0] = tV < g.n_tiles ? next_ticket(ws.ctrl) : kNone;
-    team_bar(team);
-    tW = tc->next[0];
-    { const TileInfo i = info(tW); stage_load(i, pol_keep); stage_read(i, d); measure(i, d, 2); }
-    uint32_t last_tk = kNone;          // leader: the ticket it claimed last
-    if (tt == 0) {
-        last_tk = tW < g.n_tiles ? next_ticket(ws.ctrl) : kNone;
+        const uint32_t t0 = next_ticket(ws.ctrl);
+        last_tk = t0 < g.n_tiles ? next_ticket(ws.ctrl) : kNone;
+        tc->next[0] = t0;
         tc->next[1] = last_tk;
-        tc->excl[1] = tX < g.n_tiles ? wait_prefix(ws.lbk, tX, ws.ctrl) : 0ull;
+        tc->excl[0] = 0ull;
+        tc->excl[1] = 0ull;
     }
     team_bar(team);
-    stage_load(info(tX), pol_last);    // X again, for the first pack
-    // from here on: next[par^1] / excl[par^1] hold what the previous step prepared
+    tY = tc->next[0];
+    stage_load(info(tY), pol_last);
 
-    while (tX < g.n_tiles) {
-        // two round trips to L2 whose answers are used in the next step: the ticket of the tile
-        // to measure then, and the offset of the tile to pack then
+    while (tX < g.n_tiles || tV < g.n_tiles || tW < g.n_tiles || tY < g.n_tiles) {
+        // two round trips to L2 whose answers are used at the end of the step: the ticket of the
+        // tile to measure two steps on, and the offset of the tile to pack in the next step
         uint32_t pv = 0, tk = kNone;
         if (leader) {
             if (tV < g.n_tiles) pv = ld_relaxed_u32(ws.lbk + tV);
             if (last_tk < g.n_tiles) tk = next_ticket(ws.ctrl);
         }
-        {
-            const TileInfo iX = info(tX);
-            stage_read(iX, d);
-            team_bar(team);               // stage free; what the leader left at the end of the last step is visible
-            tY = tc->next[par ^ 1u];
-            const unsigned long long exclX = tc->excl[par ^ 1u];
-            stage_load(info(tY), pol_keep);
+        const TileInfo iY = info(tY);
+        stage_read(iY, d);
+        team_bar(team);                   // stage free; what the leader left at the end of the last step is visible
+        const uint32_t tN = tc->next[par ^ 1u];
+        const unsigned long long exclX = tc->excl[par ^ 1u];
+        stage_load(info(tN), pol_last);   // has the whole step to arrive
+        measure(iY, d, (sl + 3u) & 7u);
+        if (iY.present && iY.full) tmem_store16(tmem_warp + 16u * (step & 3u), d);
+        const TileInfo iX = info(tX);
+        if (iX.valid) {
+            if (iX.present && iX.full) tmem_load16(tmem_warp + 16u * ((step + 1u) & 3u), d);
             pack(iX, d, sl, exclX);
-        }
-        {
-            const TileInfo iY = info(tY);
-            stage_read(iY, d);
-            team_bar(team);                                           // stage free
-            stage_load(info(tV), pol_last);
-            measure(iY, d, (sl + 3u) & 7u);
         }
         if (leader) {
 #ifdef WM_DEBUG_COUNTERS
@@ -1011,10 +1008,15 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
             tc->next[par] = tk;
             last_tk = tk;
         }
-        tX = tV; tV = tW; tW = tY;
+        tX = tV; tV = tW; tW = tY; tY = tN;
         sl = (sl + 1u) & 7u;
         par ^= 1u;
+        step++;
     }
+    // every warp is done with its tensor memory: hand it back before the block exits
+    tmem_fence_before_sync();
+    __syncthreads();
+    if (threadIdx.x < 32) tmem_free_all(s_tmem);
 }
 
 // Directory (enc_len, crc), chunk CRCs, present count; the last block to finish combines the
