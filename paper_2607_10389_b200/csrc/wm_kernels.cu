@@ -537,6 +537,18 @@ __device__ __forceinline__ uint32_t ld_relaxed_u32(const uint32_t* p)
     return v;
 }
 
+// Give up: waits end early once the flag is up, and the ticket counter jumps past every tile,
+// so that nobody claims another one (claiming itself never has to look at the flag).
+__device__ __forceinline__ void raise_poison(Ctrl* ctrl)
+{
+    atomicExch(&ctrl->poison, 1u);
+    atomicMax(&ctrl->ticket, 0x7FFF0000u);
+}
+__device__ __forceinline__ uint32_t next_ticket(Ctrl* ctrl)
+{
+    return atomicAdd(&ctrl->ticket, 1u);
+}
+
 // Owner side: exclusive prefix (bytes) of tile t (one lane spins; bounded).
 __device__ __forceinline__ unsigned long long wait_prefix(const uint32_t* lbk, uint32_t t, Ctrl* ctrl)
 {
@@ -546,7 +558,7 @@ __device__ __forceinline__ unsigned long long wait_prefix(const uint32_t* lbk, u
         if ((polls & 1023u) == 1023u && ld_volatile_u32(&ctrl->poison)) break;
     }
     atomicOr(&ctrl->err, 2u);
-    atomicExch(&ctrl->poison, 1u);
+    raise_poison(ctrl);
     return 0;
 }
 
@@ -626,7 +638,7 @@ __device__ void scan_tile_lengths(uint32_t* lbk, uint32_t n_tiles, uint32_t lane
 #endif
         if (k == 0) {
             if (++spins > kSpinLimit || ((spins & 1023u) == 1023u && ld_volatile_u32(&ctrl->poison))) {
-                if (lane == 0) { atomicOr(&ctrl->err, 2u); atomicExch(&ctrl->poison, 1u); }
+                if (lane == 0) { atomicOr(&ctrl->err, 2u); raise_poison(ctrl); }
                 return;
             }
         } else {
@@ -636,12 +648,6 @@ __device__ void scan_tile_lengths(uint32_t* lbk, uint32_t n_tiles, uint32_t lane
 #ifdef WM_DEBUG_COUNTERS
     if (lane == 0) { ctrl->pad[0] = dbg_iters; ctrl->pad[1] = dbg_empty; }
 #endif
-}
-
-__device__ __forceinline__ uint32_t next_ticket(Ctrl* ctrl)
-{
-    if (ld_volatile_u32(&ctrl->poison)) return 0xFFFFFFFFu;
-    return atomicAdd(&ctrl->ticket, 1u);
 }
 
 __device__ __forceinline__ uint32_t desc_of(uint32_t base, uint32_t w)
@@ -665,34 +671,9 @@ struct EncTeamCtl {
 static_assert(sizeof(EncTeamCtl) % 16 == 0, "team control block keeps 16-byte alignment");
 constexpr uint32_t kTeamSmemEncode = kTile + sizeof(EncTeamCtl);   // one 16 KiB stage + control
 
-struct TileInfo {
-    uint32_t t, c;
-    bool valid, present, full, first;
-};
-
 __device__ __forceinline__ uint32_t tile_left(const Geo& g, uint32_t t)      // bytes of a ragged tile
 {
     return (uint32_t)(g.nbytes - (uint64_t)t * kTile);
-}
-
-template <bool MASKED>
-__device__ __forceinline__ TileInfo tile_info(const Geo& g, const uint8_t* __restrict__ dirty, uint32_t t)
-{
-    TileInfo ti;
-    ti.t = t;
-    ti.valid = t < g.n_tiles;
-    ti.full = t < g.n_full_tiles;
-    ti.c = chunk_of(g, t);
-    ti.first = first_in_chunk(g, t);
-    ti.present = ti.valid && (!MASKED || dirty[ti.valid ? ti.c : 0] != 0);
-    return ti;
-}
-
-__device__ __forceinline__ uint32_t encoded_len(const Geo& g, const TileInfo& ti, uint32_t S)
-{
-    if (!ti.present) return 0;
-    if (!ti.full) return tile_left(g, ti.t);
-    return S <= 253u ? 8256u + 32u * S : kTile;
 }
 
 __device__ __forceinline__ void stg_u8(void* p, uint32_t v)
@@ -768,6 +749,21 @@ __device__ __forceinline__ void pack_group_planes(uint32_t e4a, uint32_t e4b, ui
 // scanner is late, this team waits while that tile's length is not out yet; with three steps
 // of slack that is rare, and it only delays: the teams that hold earlier tiles never depend
 // on this one.
+// A tile as a team passes it round: its number in the low 30 bits, kQFirst when it is the first
+// tile of its chunk, kQPresent when its chunk is encoded; kQNone: no tile.  (The codec takes
+// caches of at most 2^21 tiles, so a number never reaches the flag bits.)
+constexpr uint32_t kQPresent = 1u << 31, kQFirst = 1u << 30, kQTile = (1u << 30) - 1u, kQNone = kQTile;
+
+template <bool MASKED>
+__device__ __forceinline__ uint32_t describe_tile(const Geo& g, const uint8_t* __restrict__ dirty, uint32_t t)
+{
+    if (t >= g.n_tiles) return kQNone;
+    uint32_t q = t;
+    if (first_in_chunk(g, t)) q |= kQFirst;
+    if (!MASKED || dirty[chunk_of(g, t)] != 0) q |= kQPresent;
+    return q;
+}
+
 template <int TEAMS, bool MASKED>
 __global__ void __launch_bounds__(TEAMS * 256, 1)
 k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restrict__ dirty,
@@ -777,6 +773,7 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
     // The first block to get here becomes the scanner: one warp of it, alone on its SM (a warp
     // that shares its scheduler with busy ones gets too few issue slots to keep up).
     __shared__ uint32_t s_scanner;
+    __shared__ uint32_t s_tmem;
     if (threadIdx.x == 0) s_scanner = atomicCAS(&ws.ctrl->scan_lock, 0u, 1u) == 0u;
     __syncthreads();
     if (s_scanner) {
@@ -795,39 +792,96 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
     EncTeamCtl* tc = reinterpret_cast<EncTeamCtl*>(S.take(TEAMS * sizeof(EncTeamCtl)));
     if (!S.ok) { if (threadIdx.x == 0) atomicOr(&ws.ctrl->err, 4u); return; }
     tc += team;
-    unsigned char* dir = wire + 64;
-    uint16_t* tile_tab = reinterpret_cast<uint16_t*>(wire + 64 + 16ull * g.n_chunks);
-    const uint64_t pol_last = l2_policy_evict_first();     // every tile is read once
-    uint32_t phase = 0;                // parity of the stage's next completion
-    auto info = [&](uint32_t t) { return tile_info<MASKED>(g, dirty, t); };
-    // Start the bulk copy of a full tile into the stage (call after a team barrier that
-    // follows the last read of the stage; one thread issues).
-    auto stage_load = [&](const TileInfo& ti, uint64_t policy) {
-        if (tt == 0 && ti.present && ti.full) bulk_load(stage, cache + (uint64_t)ti.t * kTile, kTile, &tc->mbar, policy);
-    };
-    // Wait for it and take this lane's 16 words.
-    auto stage_read = [&](const TileInfo& ti, uint32_t (&d)[kWordsPerLane]) {
-        if (ti.present && ti.full) {
-            if (!mbar_wait(&tc->mbar, phase) && lane == 0) { atomicOr(&ws.ctrl->err, 2u); atomicExch(&ws.ctrl->poison, 1u); }
-            phase ^= 1u;
-            read_staged_words(stage, warp, lane, d);
-        }
-    };
-    auto publish_len = [&](uint32_t t, uint32_t len) { st_relaxed_u32(ws.lbk + t, kFlagA | (len / kUnit)); };
 
-    // Digest and per-group exponent range of one tile; results go to slot `sl`.  The tile's
-    // encoded length is published by whichever warp finishes last (no team barrier).
-    auto measure = [&](const TileInfo& ti, uint32_t (&d)[kWordsPerLane], uint32_t sl) {
-        if (!ti.valid) return;
-        if (!ti.present || !ti.full) {
-            if (warp == 0 && lane == 0) publish_len(ti.t, encoded_len(g, ti, 0));
-            if (!ti.present) return;
-            load_tile_words_guarded(cache + (uint64_t)ti.t * kTile, tile_left(g, ti.t), ti.first, warp, lane, d);
+    // Tensor memory for the tiles in flight: allocated by the block's first warp, the address
+    // goes round through shared memory.  Warp w of the block owns lanes 32 (w % 4) .. + 31 and
+    // 64 columns from 64 (w / 4): four slots of 16 columns, one per tile in flight.
+    if (threadIdx.x < 32) tmem_alloc_all(&s_tmem);
+    tmem_fence_before_sync();
+    __syncthreads();
+    tmem_fence_after_sync();
+    const uint32_t wc = threadIdx.x / 32;
+    const uint32_t tmem_warp = s_tmem + ((32u * (wc & 3u)) << 16) + 64u * (wc >> 2);
+
+    unsigned char* const dir = wire + 64;
+    uint16_t* const tile_tab = reinterpret_cast<uint16_t*>(wire + 64 + 16ull * g.n_chunks);
+    unsigned char* const payload = wire + g.meta_end;
+    const uint64_t room = wire_cap - g.meta_end;                 // payload bytes that fit
+    const uint64_t pol_once = l2_policy_evict_first();           // every tile is read once
+    const uint32_t* const my_words = reinterpret_cast<const uint32_t*>(stage) + warp * 512u + lane;
+    const uint32_t sm_off = 64u + 1024u * warp + 8u * lane;      // this lane's place in a group's sign-mantissa run
+    const bool leader = (tt == 0);
+    uint32_t phase = 0;                // parity of the stage's next completion
+
+    auto is_tile = [](uint32_t q) { return (q & kQTile) != kQNone; };
+    auto is_hot = [&](uint32_t q) { return q >= kQPresent && (q & kQTile) < g.n_full_tiles; };   // present and full
+    auto publish_len = [&](uint32_t t, uint32_t len) { st_relaxed_u32(ws.lbk + t, kFlagA | (len / kUnit)); };
+    auto start_copy = [&](uint32_t q) {          // thread 0 of the team, after the barrier that frees the stage
+        if (is_hot(q)) bulk_load(stage, cache + (uint64_t)(q & kQTile) * kTile, kTile, &tc->mbar, pol_once);
+    };
+
+    // Tiles in flight, oldest first: X (packed in this step), V, W (waiting for their offsets),
+    // Y (measured in this step).  Ring slots of the widths: X = sl, V = sl+1, W = sl+2, Y = sl+3
+    // (mod 8); tensor memory slots: Y = step mod 4, X = (step + 1) mod 4 (where it was put three
+    // steps ago).
+    uint32_t qX = kQNone, qV = kQNone, qW = kQNone, qY = kQNone;
+    uint32_t sl = 0;
+    uint32_t par = 0;                  // step parity (selects next[] / excl[])
+    uint32_t step = 0;
+    uint32_t d[kWordsPerLane];
+    bool claiming = false;             // leader: the last ticket it claimed was a tile
+
+    // ---- prologue: the tiles of the first two steps are claimed, the first one's copy started
+    if (leader) {
+        for (int i = 0; i < 8; i++) tc->wsum[i] = 0;
+        mbar_init(&tc->mbar, 1);
+        const uint32_t q0 = describe_tile<MASKED>(g, dirty, next_ticket(ws.ctrl));
+        const uint32_t q1 = is_tile(q0) ? describe_tile<MASKED>(g, dirty, next_ticket(ws.ctrl)) : kQNone;
+        claiming = is_tile(q1);
+        tc->next[0] = q0;
+        tc->next[1] = q1;
+        tc->excl[0] = 0ull;
+        tc->excl[1] = 0ull;
+    }
+    team_bar(team);
+    qY = tc->next[0];
+    if (leader) start_copy(qY);
+
+    uint32_t trouble = 0;              // sticky: 1 the image does not fit, 2 a copy never arrived
+    while (((qX & qV & qW & qY) & kQTile) != kQNone) {
+        const bool hotY = is_hot(qY);
+        if (hotY) {
+            if (!mbar_wait(&tc->mbar, phase)) trouble |= 2u;
+            phase ^= 1u;
+#pragma unroll
+            for (int i = 0; i < 16; i++) d[i] = my_words[i * 32];
         }
-        const uint32_t v = tile_digest_part(S, d, ti.first && ti.full, warp, lane);
-        if (lane == 0) tc->wdig[sl][warp] = v;
-        if (ti.full) {
-            uint32_t mysum = 0;
+        team_bar(team);                   // stage free; what the leader left at the end of the last step is visible
+        const uint32_t qN = tc->next[par ^ 1u];
+        const unsigned long long exclX = tc->excl[par ^ 1u];
+        // The leader starts the copy of the next tile (it has the whole step to arrive) and two
+        // round trips to L2 whose answers are used at the end of the step: the ticket of the
+        // tile to measure two steps on, and the offset of the tile to pack in the next step.
+        uint32_t pv = 0, tk = 0xFFFFFFFFu;
+        if (leader) {
+            start_copy(qN);
+            if (is_tile(qV)) pv = ld_relaxed_u32(ws.lbk + (qV & kQTile));
+            if (claiming) tk = next_ticket(ws.ctrl);
+        }
+
+        // ---- Y: digest, exponent ranges, length out, words parked
+        const uint32_t slY = (sl + 3u) & 7u;
+        const uint32_t tYn = qY & kQTile;
+        if (hotY) {
+#ifdef WM_AB_NOCRC
+            const uint32_t v = d[3];
+#else
+            const uint32_t v = tile_digest_part(S, d, (qY & kQFirst) != 0, warp, lane);
+#endif
+            uint32_t gw[4];               // per group: base | width << 8
+#ifdef WM_AB_NOMINMAX
+            gw[0] = gw[1] = gw[2] = gw[3] = 100u | (4u << 8);
+#else
 #pragma unroll
             for (int j = 0; j < 4; j++) {
                 // w << 1 drops the upper element's sign and leaves [E | m | junk bit] in each half
@@ -838,19 +892,21 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
                 mx = max(mx & 0xFFFFu, mx >> 16);
                 const uint32_t emin = __reduce_min_sync(0xFFFFFFFFu, mn) >> 8;
                 const uint32_t emax = __reduce_max_sync(0xFFFFFFFFu, mx) >> 8;
-                const uint32_t wd = 32u - __clz(emax - emin);
-                mysum += wd;
-                if (lane == 0) tc->wtab[sl][4 * warp + j] = emin | (wd << 8);
+                gw[j] = emin | ((32u - __clz(emax - emin)) << 8);
             }
-            // the warp that arrives last turns the 32 widths into offsets and publishes the length
+#endif
+            // one lane leaves the warp's results; the warp that arrives last turns the 32 widths
+            // into offsets and publishes the tile's length
             uint32_t last = 0;
             if (lane == 0) {
+                tc->wdig[slY][warp] = v;
+                *reinterpret_cast<uint4*>(&tc->wtab[slY][4 * warp]) = make_uint4(gw[0], gw[1], gw[2], gw[3]);
                 __threadfence_block();
-                last = (atomicAdd(&tc->wsum[sl], 1u) == 7u) ? 1u : 0u;
+                last = (atomicAdd(&tc->wsum[slY], 1u) == 7u) ? 1u : 0u;
             }
             if (__shfl_sync(0xFFFFFFFFu, last, 0)) {
                 __threadfence_block();
-                const uint32_t wt = *reinterpret_cast<volatile uint32_t*>(&tc->wtab[sl][lane]);
+                const uint32_t wt = *reinterpret_cast<volatile uint32_t*>(&tc->wtab[slY][lane]);
                 const uint32_t wv = (wt >> 8) & 15u;
                 uint32_t incl = wv;
 #pragma unroll
@@ -858,160 +914,132 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
                     const uint32_t o = __shfl_up_sync(0xFFFFFFFFu, incl, k);
                     if (lane >= (uint32_t)k) incl += o;
                 }
-                tc->wtab[sl][lane] = (wt & 0xFFFFu) | ((incl - wv) << 16);
+                tc->wtab[slY][lane] = (wt & 0xFFFFu) | ((incl - wv) << 16);
                 if (lane == 31) {
-                    tc->ssum[sl] = incl;
-                    tc->wsum[sl] = 0;
-                    publish_len(ti.t, encoded_len(g, ti, incl));
+                    tc->ssum[slY] = incl;
+                    tc->wsum[slY] = 0;
+                    publish_len(tYn, incl <= 253u ? 8256u + 32u * incl : kTile);
                 }
             }
+#ifndef WM_AB_NOTMEM
+            tmem_store16(tmem_warp + 16u * (step & 3u), d);
+#endif
+        } else if (is_tile(qY)) {
+            // rare: a tile of an absent chunk (length 0) or the ragged last tile (stored raw)
+            const bool present = qY >= kQPresent;
+            if (tt == 0) publish_len(tYn, present ? tile_left(g, tYn) : 0u);
+            if (present) {
+                load_tile_words_guarded(cache + (uint64_t)tYn * kTile, tile_left(g, tYn), (qY & kQFirst) != 0, warp, lane, d);
+                const uint32_t v = tile_digest_part(S, d, false, warp, lane);
+                if (lane == 0) tc->wdig[slY][warp] = v;
+            }
         }
-    };
-    // Pack tile X (words in d, widths in slot sl) into the wire image at payload offset excl.
-    auto pack = [&](const TileInfo& ti, const uint32_t (&d)[kWordsPerLane], uint32_t sl, unsigned long long excl) {
-        uint32_t enc_len = 0, entry = 0;
-        if (ti.present) {
-            unsigned char* dst = wire + g.meta_end + excl;
-            if (ti.full) {
-                const uint32_t Ssum = tc->ssum[sl];
-                const bool packs = Ssum <= 253u;
-                enc_len = packs ? 8256u + 32u * Ssum : kTile;
-                entry = packs ? 258u + Ssum : 512u;
-                if (g.meta_end + excl + enc_len > wire_cap) {
-                    if (tt == 0) atomicOr(&ws.ctrl->err, 1u);
-                } else if (packs) {
-                    if (warp == 0) {
-                        const uint32_t wt = tc->wtab[sl][lane];
-                        stg_u16(dst + 2 * lane, desc_of(wt & 0xFFu, (wt >> 8) & 15u));
-                    }
-#pragma unroll
-                    for (int j = 0; j < 4; j++) {
-                        const uint32_t gi = 4 * warp + j;
-                        const uint32_t wtg = tc->wtab[sl][gi];
-                        const uint32_t exg = wtg >> 16;
-                        const uint32_t base = wtg & 0xFFu, wd = (wtg >> 8) & 15u;
-                        uint32_t Tr[4];
-#pragma unroll
-                        for (int r = 0; r < 4; r++) {
-                            const uint32_t Wd = d[4 * j + r];
-                            Tr[r] = ((Wd << 1) & 0xFFFEFFFEu) | ((Wd >> 15) & 0x00010001u);
-                        }
-                        stg_v2(dst + 64 + 256 * gi + 8 * lane, __byte_perm(Tr[0], Tr[1], 0x6420),
-                               __byte_perm(Tr[2], Tr[3], 0x6420));
-                        const uint32_t e4a = __byte_perm(Tr[0], Tr[1], 0x7531), e4b = __byte_perm(Tr[2], Tr[3], 0x7531);
-                        unsigned char* rec = dst + 8256 + 32 * exg;
-                        switch (wd) {          // uniform across the warp
-                            case 1: pack_group_planes<1>(e4a, e4b, base, rec, lane); break;
-                            case 2: pack_group_planes<2>(e4a, e4b, base, rec, lane); break;
-                            case 3: pack_group_planes<3>(e4a, e4b, base, rec, lane); break;
-                            case 4: pack_group_planes<4>(e4a, e4b, base, rec, lane); break;
-                            case 5: pack_group_planes<5>(e4a, e4b, base, rec, lane); break;
-                            case 6: pack_group_planes<6>(e4a, e4b, base, rec, lane); break;
-                            case 7: pack_group_planes<7>(e4a, e4b, base, rec, lane); break;
-                            case 8: pack_group_planes<8>(e4a, e4b, base, rec, lane); break;
-                            default: break;
-                        }
-                    }
-                } else {
-                    unsigned char* q = dst + warp * 2048u + lane * 4u;
-#pragma unroll
-                    for (int i = 0; i < 16; i++) st_stream_u32(q + i * 128, d[i]);
+
+        // ---- X: its words back from tensor memory, packed straight into the wire image
+        const uint32_t tXn = qX & kQTile;
+        if (is_hot(qX)) {
+#ifndef WM_AB_NOTMEM
+            tmem_load16(tmem_warp + 16u * ((step + 1u) & 3u), d);
+#endif
+            const uint32_t Ssum = tc->ssum[sl];
+            const bool packs = Ssum <= 253u;
+            const uint32_t enc_len = packs ? 8256u + 32u * Ssum : kTile;
+            unsigned char* const dst = payload + exclX;
+            if (exclX + enc_len > room) {
+                trouble |= 1u;
+            } else if (packs) {
+#ifndef WM_AB_NOPACK
+                if (warp == 0) {
+                    const uint32_t wt = tc->wtab[sl][lane];
+                    stg_u16(dst + 2 * lane, desc_of(wt & 0xFFu, (wt >> 8) & 15u));
                 }
+                unsigned char* const sm_dst = dst + sm_off;
+                unsigned char* const pl_dst = dst + 8256;
+                const uint4 g4 = *reinterpret_cast<const uint4*>(&tc->wtab[sl][4 * warp]);
+                const uint32_t gq[4] = {g4.x, g4.y, g4.z, g4.w};
+#pragma unroll
+                for (int j = 0; j < 4; j++) {
+                    const uint32_t wtg = gq[j];
+                    const uint32_t base = wtg & 0xFFu, wd = (wtg >> 8) & 15u;
+                    uint32_t Tr[4];
+#pragma unroll
+                    for (int r = 0; r < 4; r++) {
+                        const uint32_t Wd = d[4 * j + r];
+                        Tr[r] = ((Wd << 1) & 0xFFFEFFFEu) | ((Wd >> 15) & 0x00010001u);
+                    }
+                    stg_v2(sm_dst + 256 * j, __byte_perm(Tr[0], Tr[1], 0x6420), __byte_perm(Tr[2], Tr[3], 0x6420));
+                    const uint32_t e4a = __byte_perm(Tr[0], Tr[1], 0x7531), e4b = __byte_perm(Tr[2], Tr[3], 0x7531);
+                    unsigned char* rec = pl_dst + 32u * (wtg >> 16);
+                    if (wd == 4u) pack_group_planes<4>(e4a, e4b, base, rec, lane);      // by far the most frequent width
+                    else switch (wd) {     // uniform across the warp
+                        case 1: pack_group_planes<1>(e4a, e4b, base, rec, lane); break;
+                        case 2: pack_group_planes<2>(e4a, e4b, base, rec, lane); break;
+                        case 3: pack_group_planes<3>(e4a, e4b, base, rec, lane); break;
+                        case 5: pack_group_planes<5>(e4a, e4b, base, rec, lane); break;
+                        case 6: pack_group_planes<6>(e4a, e4b, base, rec, lane); break;
+                        case 7: pack_group_planes<7>(e4a, e4b, base, rec, lane); break;
+                        case 8: pack_group_planes<8>(e4a, e4b, base, rec, lane); break;
+                        default: break;
+                    }
+                }
+#else
+                if (d[5] == 0x12345678u) stg_u8(dst + lane, d[1]);
+#endif
             } else {
-                enc_len = tile_left(g, ti.t);
-                entry = 0xFFFFu;
-                if (g.meta_end + excl + enc_len > wire_cap) {
-                    if (tt == 0) atomicOr(&ws.ctrl->err, 1u);
-                } else {
-                    const unsigned char* src = cache + (uint64_t)ti.t * kTile;
-                    for (uint32_t i = tt; i < enc_len; i += kTeamThreads) dst[i] = src[i];
-                }
+                unsigned char* q = dst + warp * 2048u + lane * 4u;
+#pragma unroll
+                for (int i = 0; i < 16; i++) st_stream_u32(q + i * 128, d[i]);
+            }
+        } else if (qX >= kQPresent) {
+            // rare: the ragged last tile, stored raw
+            const uint32_t enc_len = tile_left(g, tXn);
+            if (exclX + enc_len > room) {
+                trouble |= 1u;
+            } else {
+                const unsigned char* src = cache + (uint64_t)tXn * kTile;
+                unsigned char* dst = payload + exclX;
+                for (uint32_t i = tt; i < enc_len; i += kTeamThreads) dst[i] = src[i];
             }
         }
-        if (tt == 0) {
-            tile_tab[ti.t] = (uint16_t)entry;
-            if (ti.present) ws.dig[ti.t] = xor8(tc->wdig[sl]);
-            if (ti.first) *reinterpret_cast<unsigned long long*>(dir + 16ull * ti.c) = excl;
-            if (ti.t + 1 == g.n_tiles) ws.ctrl->payload_total = excl + enc_len;
-        }
-    };
 
-    // Tensor memory for the tiles in flight: allocated by the block's first warp, the address
-    // goes round through shared memory.  Warp w of the block owns lanes 32 (w % 4) .. + 31 and
-    // 64 columns from 64 (w / 4): four slots of 16 columns, one per tile in flight.
-    __shared__ uint32_t s_tmem;
-    if (threadIdx.x < 32) tmem_alloc_all(&s_tmem);
-    tmem_fence_before_sync();
-    __syncthreads();
-    tmem_fence_after_sync();
-    const uint32_t wc = threadIdx.x / 32;
-    const uint32_t tmem_warp = s_tmem + ((32u * (wc & 3u)) << 16) + 64u * (wc >> 2);
-
-    // Tiles in flight, oldest first: X (packed in this step), V, W (waiting for their offsets),
-    // Y (measured in this step).  Ring slots of the widths: X = sl, V = sl+1, W = sl+2, Y = sl+3
-    // (mod 8); tensor memory slots: Y = step mod 4, X = (step + 1) mod 4 (where it was put three
-    // steps ago).  Only the tile numbers are carried from step to step (>= n_tiles: none); what
-    // follows from a number (chunk, full / ragged, present) is worked out where it is used.
-    constexpr uint32_t kNone = 0xFFFFFFFFu;
-    uint32_t tX = kNone, tV = kNone, tW = kNone, tY = kNone;
-    uint32_t sl = 0;
-    uint32_t par = 0;                  // step parity (selects next[] / excl[])
-    uint32_t step = 0;
-    uint32_t d[kWordsPerLane];
-    const bool leader = (warp == 0 && lane == 0);
-    uint32_t last_tk = kNone;          // leader: the ticket it claimed last
-
-    // ---- prologue: the tiles of the first two steps are claimed, the first one's copy started
-    if (tt == 0) {
-        for (int i = 0; i < 8; i++) tc->wsum[i] = 0;
-        mbar_init(&tc->mbar, 1);
-        const uint32_t t0 = next_ticket(ws.ctrl);
-        last_tk = t0 < g.n_tiles ? next_ticket(ws.ctrl) : kNone;
-        tc->next[0] = t0;
-        tc->next[1] = last_tk;
-        tc->excl[0] = 0ull;
-        tc->excl[1] = 0ull;
-    }
-    team_bar(team);
-    tY = tc->next[0];
-    stage_load(info(tY), pol_last);
-
-    while (tX < g.n_tiles || tV < g.n_tiles || tW < g.n_tiles || tY < g.n_tiles) {
-        // two round trips to L2 whose answers are used at the end of the step: the ticket of the
-        // tile to measure two steps on, and the offset of the tile to pack in the next step
-        uint32_t pv = 0, tk = kNone;
         if (leader) {
-            if (tV < g.n_tiles) pv = ld_relaxed_u32(ws.lbk + tV);
-            if (last_tk < g.n_tiles) tk = next_ticket(ws.ctrl);
-        }
-        const TileInfo iY = info(tY);
-        stage_read(iY, d);
-        team_bar(team);                   // stage free; what the leader left at the end of the last step is visible
-        const uint32_t tN = tc->next[par ^ 1u];
-        const unsigned long long exclX = tc->excl[par ^ 1u];
-        stage_load(info(tN), pol_last);   // has the whole step to arrive
-        measure(iY, d, (sl + 3u) & 7u);
-        if (iY.present && iY.full) tmem_store16(tmem_warp + 16u * (step & 3u), d);
-        const TileInfo iX = info(tX);
-        if (iX.valid) {
-            if (iX.present && iX.full) tmem_load16(tmem_warp + 16u * ((step + 1u) & 3u), d);
-            pack(iX, d, sl, exclX);
-        }
-        if (leader) {
+            // what is left to note about X: table entry, digest, where its chunk starts, the total
+            if (is_tile(qX)) {
+                uint32_t entry = 0, enc_len = 0;
+                if (qX >= kQPresent) {
+                    if (tXn < g.n_full_tiles) {
+                        const uint32_t Ssum = tc->ssum[sl];
+                        entry = Ssum <= 253u ? 258u + Ssum : 512u;
+                        enc_len = 32u * entry;
+                    } else {
+                        entry = 0xFFFFu;
+                        enc_len = tile_left(g, tXn);
+                    }
+                    ws.dig[tXn] = xor8(tc->wdig[sl]);
+                }
+                tile_tab[tXn] = (uint16_t)entry;
+                if (qX & kQFirst) *reinterpret_cast<unsigned long long*>(dir + 16ull * chunk_of(g, tXn)) = exclX;
+                if (tXn + 1 == g.n_tiles) ws.ctrl->payload_total = exclX + enc_len;
+            }
 #ifdef WM_DEBUG_COUNTERS
             atomicAdd(&ws.ctrl->pad[(pv >> 30) == 2u ? 3 : 2], 1u);
 #endif
             unsigned long long e = 0;
-            if (tV < g.n_tiles)
-                e = (pv >> 30) == 2u ? (unsigned long long)(pv & kValMask) * kUnit : wait_prefix(ws.lbk, tV, ws.ctrl);
+            if (is_tile(qV))
+                e = (pv >> 30) == 2u ? (unsigned long long)(pv & kValMask) * kUnit : wait_prefix(ws.lbk, qV & kQTile, ws.ctrl);
+            uint32_t qn2 = kQNone;
+            if (claiming) { qn2 = describe_tile<MASKED>(g, dirty, tk); claiming = is_tile(qn2); }
             tc->excl[par] = e;
-            tc->next[par] = tk;
-            last_tk = tk;
+            tc->next[par] = qn2;
         }
-        tX = tV; tV = tW; tW = tY; tY = tN;
+        qX = qV; qV = qW; qW = qY; qY = qN;
         sl = (sl + 1u) & 7u;
         par ^= 1u;
         step++;
+    }
+    if (trouble && lane == 0) {
+        atomicOr(&ws.ctrl->err, trouble);
+        if (trouble & 2u) raise_poison(ws.ctrl);
     }
     // every warp is done with its tensor memory: hand it back before the block exits
     tmem_fence_before_sync();
