@@ -878,14 +878,18 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
 #else
             const uint32_t v = tile_digest_part(S, d, (qY & kQFirst) != 0, warp, lane);
 #endif
+            // From here on the words are kept rotated left by one bit: each half then reads
+            // [E | mantissa | a sign bit], E in its high byte (the two sign bits of a word
+            // land in each other's half; the packing step puts them right).
+#pragma unroll
+            for (int i = 0; i < 16; i++) d[i] = __funnelshift_l(d[i], d[i], 1);
             uint32_t gw[4];               // per group: base | width << 8
 #ifdef WM_AB_NOMINMAX
             gw[0] = gw[1] = gw[2] = gw[3] = 100u | (4u << 8);
 #else
 #pragma unroll
             for (int j = 0; j < 4; j++) {
-                // w << 1 drops the upper element's sign and leaves [E | m | junk bit] in each half
-                const uint32_t a0 = d[4 * j] * 2u, a1 = d[4 * j + 1] * 2u, a2 = d[4 * j + 2] * 2u, a3 = d[4 * j + 3] * 2u;
+                const uint32_t a0 = d[4 * j], a1 = d[4 * j + 1], a2 = d[4 * j + 2], a3 = d[4 * j + 3];
                 uint32_t mn = min_u16x2(min_u16x2(a0, a1), min_u16x2(a2, a3));
                 uint32_t mx = max_u16x2(max_u16x2(a0, a1), max_u16x2(a2, a3));
                 mn = min(mn & 0xFFFFu, mn >> 16);
@@ -961,14 +965,12 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
                 for (int j = 0; j < 4; j++) {
                     const uint32_t wtg = gq[j];
                     const uint32_t base = wtg & 0xFFu, wd = (wtg >> 8) & 15u;
-                    uint32_t Tr[4];
-#pragma unroll
-                    for (int r = 0; r < 4; r++) {
-                        const uint32_t Wd = d[4 * j + r];
-                        Tr[r] = ((Wd << 1) & 0xFFFEFFFEu) | ((Wd >> 15) & 0x00010001u);
-                    }
-                    stg_v2(sm_dst + 256 * j, __byte_perm(Tr[0], Tr[1], 0x6420), __byte_perm(Tr[2], Tr[3], 0x6420));
-                    const uint32_t e4a = __byte_perm(Tr[0], Tr[1], 0x7531), e4b = __byte_perm(Tr[2], Tr[3], 0x7531);
+                    // bytes 0 and 2 of a rotated word: mantissa << 1 | the other element's sign;
+                    // bytes 1 and 3: the exponents.  Gather, then swap bit 0 inside byte pairs.
+                    const uint32_t sa = __byte_perm(d[4 * j], d[4 * j + 1], 0x6420), sb = __byte_perm(d[4 * j + 2], d[4 * j + 3], 0x6420);
+                    const uint32_t ya = __byte_perm(sa, sa, 0x2301), yb = __byte_perm(sb, sb, 0x2301);
+                    stg_v2(sm_dst + 256 * j, (sa & 0xFEFEFEFEu) | (ya & 0x01010101u), (sb & 0xFEFEFEFEu) | (yb & 0x01010101u));
+                    const uint32_t e4a = __byte_perm(d[4 * j], d[4 * j + 1], 0x7531), e4b = __byte_perm(d[4 * j + 2], d[4 * j + 3], 0x7531);
                     unsigned char* rec = pl_dst + 32u * (wtg >> 16);
                     if (wd == 4u) pack_group_planes<4>(e4a, e4b, base, rec, lane);      // by far the most frequent width
                     else switch (wd) {     // uniform across the warp
@@ -988,7 +990,7 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
             } else {
                 unsigned char* q = dst + warp * 2048u + lane * 4u;
 #pragma unroll
-                for (int i = 0; i < 16; i++) st_stream_u32(q + i * 128, d[i]);
+                for (int i = 0; i < 16; i++) st_stream_u32(q + i * 128, __funnelshift_r(d[i], d[i], 1));
             }
         } else if (qX >= kQPresent) {
             // rare: the ragged last tile, stored raw
