@@ -1213,7 +1213,7 @@ k_meta_crc(unsigned char* wire, uint64_t wire_len, Geo g, Ws ws, const Tables* _
         wm_result r;
         memset(&r, 0, sizeof r);
         const uint32_t err = ld_volatile_u32(&ws.ctrl->err);
-        r.status = (err & 2u) ? WM_ERR_TIMEOUT : (err & 1u) ? WM_ERR_CAPACITY : WM_OK;
+        r.status = (err & 4u) ? WM_ERR_CUDA : (err & 2u) ? WM_ERR_TIMEOUT : (err & 1u) ? WM_ERR_CAPACITY : WM_OK;
         r.n_present = ws.ctrl->hdr_n_present;
         r.payload_bytes = ws.ctrl->payload_total;
         r.wire_len = g.meta_end + ws.ctrl->payload_total;
@@ -1384,13 +1384,10 @@ k_decode_struct(const unsigned char* __restrict__ wire, uint64_t wire_len, Geo g
     }
 }
 
-struct DecSlot {                 // what thread 0 prepares for a tile ahead of its turn
+struct DecSlot {                 // what the team's first thread prepares for a tile ahead of its turn
     uint32_t t;                  // tile (>= n_tiles: none left)
-    uint32_t entry;              // tile table entry
-    uint32_t c;                  // chunk
-    uint32_t first;              // first tile of its chunk
-    unsigned long long src;      // offset of the encoded tile inside the wire image
-    unsigned long long pad;
+    uint32_t entry;              // tile table entry | (first tile of its chunk) << 16
+    unsigned long long src;      // offset of the encoded tile inside the payload
 };
 struct DecTeamCtl {
     uint32_t wdig[2][8];
@@ -1461,8 +1458,10 @@ __device__ __forceinline__ void unpack_group_planes(const PlaneWords& pw, uint32
 // 16 KiB stage in shared memory; the encoded tile arrives there by one bulk copy (TMA) that is
 // started a tile ahead, each lane takes what it needs (descriptors, its 8 sign-mantissa bytes
 // and its plane words per group: at most 16 words) into registers, and the stage is handed to
-// the next copy while the team unpacks, stores and checksums.  Thread 0 looks up the table
-// entry and source offset two tiles ahead, so that chain of dependent loads is hidden too.
+// the next copy while the team unpacks, stores and checksums.  One team barrier per tile.
+// The team's first thread prepares tiles ahead of their turn, one dependent step per tile so
+// that it never sits waiting for an answer from L2: claim a ticket (three tiles ahead), look
+// up that tile's table entry and offsets (two ahead), start its copy (one ahead).
 template <int TEAMS>
 __global__ void __launch_bounds__(TEAMS * 256, 1)
 k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restrict__ dst, Ws ws,
@@ -1481,61 +1480,71 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
     DecTeamCtl* tc = reinterpret_cast<DecTeamCtl*>(S.take(TEAMS * sizeof(DecTeamCtl)));
     if (!S.ok) { if (threadIdx.x == 0) atomicOr(&ws.ctrl->err, 4u); return; }
     tc += team;
-    const unsigned char* dir = wire + 64;
-    const uint16_t* tab16 = reinterpret_cast<const uint16_t*>(wire + 64 + 16ull * g.n_chunks);
-    const unsigned char* payload = wire + g.meta_end;
+    const unsigned char* const dir = wire + 64;
+    const uint16_t* const tab16 = reinterpret_cast<const uint16_t*>(wire + 64 + 16ull * g.n_chunks);
+    const unsigned char* const payload = wire + g.meta_end;
+    const bool leader = (tt == 0);
+    constexpr uint32_t kNone = 0xFFFFFFFFu;
 
-    auto prepare = [&](DecSlot* sl) {       // thread 0 only
-        const uint32_t t = atomicAdd(&ws.ctrl->ticket, 1u);
+    // a tile's entry word and payload offset (blocking: prologue only)
+    auto lookup = [&](uint32_t t, DecSlot* sl) {
         sl->t = t;
+        sl->entry = 0; sl->src = 0;
         if (t < g.n_tiles) {
             const uint32_t e = tab16[t];
-            const uint32_t c = chunk_of(g, t);
-            sl->entry = e; sl->c = c; sl->first = first_in_chunk(g, t) ? 1u : 0u;
-            sl->src = e ? *reinterpret_cast<const unsigned long long*>(dir + 16ull * c) + ws.rel[t] : 0ull;
+            sl->entry = e | (first_in_chunk(g, t) ? 0x10000u : 0u);
+            if (e) sl->src = *reinterpret_cast<const unsigned long long*>(dir + 16ull * chunk_of(g, t)) + ws.rel[t];
         }
     };
     // staged tiles: full RAW and PACK tiles (everything except absent tiles and the ragged tail)
-    auto staged = [&](const DecSlot& sl) { return sl.t < g.n_tiles && sl.entry >= 258u && sl.entry <= 512u; };
-    auto start_copy = [&](const DecSlot& sl) {   // thread 0 only
-        if (staged(sl)) bulk_load(stage, payload + sl.src, 32u * sl.entry, &tc->mbar, 0);
+    auto start_copy = [&](const DecSlot& sl) {   // leader only
+        const uint32_t e = sl.entry & 0xFFFFu;
+        if (sl.t < g.n_tiles && e >= 258u && e <= 512u) bulk_load(stage, payload + sl.src, 32u * e, &tc->mbar, 0);
     };
 
-    if (tt == 0) {
+    uint32_t t_look = kNone;           // leader: the tile whose look-ups are under way in this step
+    if (leader) {
         mbar_init(&tc->mbar, 1);
-        prepare(&tc->slot[0]);
-        prepare(&tc->slot[1]);
+        lookup(atomicAdd(&ws.ctrl->ticket, 1u), &tc->slot[0]);
+        lookup(atomicAdd(&ws.ctrl->ticket, 1u), &tc->slot[1]);
+        t_look = atomicAdd(&ws.ctrl->ticket, 1u);
+        tc->slot[2].t = t_look;
         start_copy(tc->slot[0]);
     }
     team_bar(team);
     uint32_t phase = 0;
+    uint32_t trouble = 0;              // sticky: a copy never arrived
+    uint32_t t_done = kNone;           // leader: tile whose digest parts wait in wdig[(it - 1) & 1]
     for (uint32_t it = 0;; it++) {
-        const DecSlot sl = tc->slot[it & 3u];
-        const uint32_t t = sl.t;
-        if (t >= g.n_tiles) break;
-        const uint32_t e = sl.entry;
-        const bool first = sl.first != 0;
+        const uint32_t t = tc->slot[it & 3u].t;
+        if (t >= g.n_tiles) {
+            team_bar(team);
+            if (leader && t_done != kNone) ws.dig[t_done] = xor8(tc->wdig[(it & 1u) ^ 1u]);
+            break;
+        }
+        const uint32_t ew = tc->slot[it & 3u].entry;
+        const uint32_t e = ew & 0xFFFFu;
         const uint32_t p = it & 1u;
-        bool have_digest = false, decoded = true, fold = first;
+        const bool is_pack = e >= 258u && e < 512u;
+        bool decoded = true;
         uint32_t w[kWordsPerLane];
-        uint32_t desc = 0, incl = 0, wv = 0;
+        uint32_t desc = 0;
         uint2 sm[4];
         PlaneWords pw[4];
-        const bool is_pack = e >= 258u && e < 512u;
 
         // ---- phase 1: everything this lane needs from the stage goes into registers
-        if (staged(sl)) {
-            if (!mbar_wait(&tc->mbar, phase) && lane == 0) { atomicOr(&ws.ctrl->err, 2u); }
+        if (e >= 258u && e <= 512u) {
+            if (!mbar_wait(&tc->mbar, phase)) trouble = 1u;
             phase ^= 1u;
             if (!is_pack) {
                 read_staged_words(stage, warp, lane, w);
             } else {
                 desc = reinterpret_cast<const uint16_t*>(stage)[lane];
-                wv = (desc >> 8) & 15u;
+                const uint32_t wv = (desc >> 8) & 15u;
                 const uint32_t base_l = desc & 0xFFu, chk = desc >> 12;
                 const bool bad = wv > 8u || chk != (((base_l & 15u) ^ (base_l >> 4) ^ wv ^ 5u) & 15u);
                 const bool anybad = __any_sync(0xFFFFFFFFu, bad);
-                incl = wv;
+                uint32_t incl = wv;
 #pragma unroll
                 for (int k = 1; k < 32; k <<= 1) {
                     const uint32_t o2 = __shfl_up_sync(0xFFFFFFFFu, incl, k);
@@ -1545,48 +1554,63 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
                 const int verdict = anybad ? 1 : (258u + Ssum != e ? 2 : 0);
                 if (verdict) {               // every warp reaches the same verdict
                     decoded = false;
-                    if (tt == 0) {
+                    if (leader) {
                         atomicMin(&ws.ctrl->bad4_key, (unsigned long long)t * 2ull + (verdict == 2 ? 1ull : 0ull));
-                        atomicOr(&ws.cflag[sl.c], CF_BAD4);
+                        atomicOr(&ws.cflag[chunk_of(g, t)], CF_BAD4);
                     }
                 } else {
+                    // this lane keeps, in desc, the descriptor of group 4 warp + (lane & 3) with the
+                    // group's offset in the plane area in the high half
+                    const uint32_t mine = (desc & 0xFFFFu) | ((incl - wv) << 16);
+                    desc = __shfl_sync(0xFFFFFFFFu, mine, 4 * warp + (lane & 3u));
 #pragma unroll
                     for (int j = 0; j < 4; j++) {
-                        const uint32_t gi = 4 * warp + j;
-                        const uint32_t dg = __shfl_sync(0xFFFFFFFFu, desc, gi);
-                        const uint32_t exg = __shfl_sync(0xFFFFFFFFu, incl - wv, gi);
-                        sm[j] = *reinterpret_cast<const uint2*>(stage + 64 + 256 * gi + 8 * lane);
-                        pw[j] = read_group_planes(stage + 8256 + 32 * exg, (dg >> 8) & 15u, lane);
+                        const uint32_t dg = __shfl_sync(0xFFFFFFFFu, desc, j);
+                        sm[j] = *reinterpret_cast<const uint2*>(stage + 64 + 256 * (4 * warp + j) + 8 * lane);
+                        pw[j] = read_group_planes(stage + 8256 + 32 * (dg >> 16), (dg >> 8) & 15u, lane);
                     }
                 }
             }
         }
-        team_bar(team);                      // stage free; slot[it+1] (prepared last step) visible
-        if (tt == 0) {
+        team_bar(team);                      // stage free; the slots the leader filled last step visible;
+                                             // the previous tile's digest parts complete
+        // The leader: next tile's copy; the previous tile's digest; look-ups for the tile two
+        // ahead and the ticket of the tile three ahead (answers taken at the end of the step).
+        uint32_t l_e = 0, l_rel = 0, l_tk = kNone;
+        unsigned long long l_po = 0;
+        if (leader) {
             start_copy(tc->slot[(it + 1u) & 3u]);
-            prepare(&tc->slot[(it + 2u) & 3u]);
+            if (t_done != kNone) ws.dig[t_done] = xor8(tc->wdig[p ^ 1u]);
+            if (t_look < g.n_tiles) {
+                l_e = tab16[t_look];
+                l_rel = __ldcg(ws.rel + t_look);
+                l_po = *reinterpret_cast<const unsigned long long*>(dir + 16ull * chunk_of(g, t_look));
+                l_tk = atomicAdd(&ws.ctrl->ticket, 1u);
+            }
         }
 
         // ---- phase 2: unpack, store, checksum
+        bool have_digest = false;
         if (e != 0) {
             unsigned char* o = dst + (uint64_t)t * kTile;
+            bool fold = (ew >> 16) != 0;
             if (e == 0xFFFFu) {
-                const unsigned char* src = payload + sl.src;
+                const unsigned char* src = payload + tc->slot[it & 3u].src;
                 const uint32_t len = g.tail_len;
                 for (uint32_t i = tt; i < len; i += kTeamThreads) o[i] = src[i];
-                load_tile_words_guarded(src, len, first, warp, lane, w);
+                load_tile_words_guarded(src, len, fold, warp, lane, w);
                 fold = false;
             } else if (is_pack && decoded) {
 #pragma unroll
                 for (int j = 0; j < 4; j++) {
-                    const uint32_t dg = __shfl_sync(0xFFFFFFFFu, desc, 4 * warp + j);
+                    const uint32_t dg = __shfl_sync(0xFFFFFFFFu, desc, j);
                     const uint32_t base = dg & 0xFFu, wd = (dg >> 8) & 15u;
                     uint32_t ea = base * 0x01010101u, eb = ea;
-                    switch (wd) {          // uniform across the warp
+                    if (wd == 4u) unpack_group_planes<4>(pw[j], base, ea, eb);       // by far the most frequent width
+                    else switch (wd) {     // uniform across the warp
                         case 1: unpack_group_planes<1>(pw[j], base, ea, eb); break;
                         case 2: unpack_group_planes<2>(pw[j], base, ea, eb); break;
                         case 3: unpack_group_planes<3>(pw[j], base, ea, eb); break;
-                        case 4: unpack_group_planes<4>(pw[j], base, ea, eb); break;
                         case 5: unpack_group_planes<5>(pw[j], base, ea, eb); break;
                         case 6: unpack_group_planes<6>(pw[j], base, ea, eb); break;
                         case 7: unpack_group_planes<7>(pw[j], base, ea, eb); break;
@@ -1614,9 +1638,20 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
                 have_digest = true;
             }
         }
-        team_bar(team);                      // wdig[p] complete; thread 0's slot writes visible
-        if (tt == 0 && have_digest) ws.dig[t] = xor8(tc->wdig[p]);
+        if (leader) {
+            t_done = have_digest ? t : kNone;
+            if (t_look < g.n_tiles) {
+                DecSlot* s2 = &tc->slot[(it + 2u) & 3u];
+                s2->entry = l_e | (first_in_chunk(g, t_look) ? 0x10000u : 0u);
+                s2->src = l_po + l_rel;
+                tc->slot[(it + 3u) & 3u].t = l_tk;
+            } else {
+                tc->slot[(it + 3u) & 3u].t = kNone;
+            }
+            t_look = l_tk;
+        }
     }
+    if (trouble && lane == 0) atomicOr(&ws.ctrl->err, 2u);
 }
 
 // Steps 5..8: chunk CRCs of the decoded bytes against the directory, stale check, cache CRC;
@@ -1668,7 +1703,10 @@ k_decode_finish(const unsigned char* __restrict__ wire, uint64_t wire_len, Geo g
         int status = WM_OK;
         uint32_t first = 0, count = 0;
         const unsigned long long key = *reinterpret_cast<volatile unsigned long long*>(&ws.ctrl->bad4_key);
-        if (key != ~0ull) {
+        const uint32_t err = ld_volatile_u32(&ws.ctrl->err);
+        if (err) {                     // the kernels themselves failed: nothing can be said about the image
+            status = (err & 4u) ? WM_ERR_CUDA : WM_ERR_TIMEOUT;
+        } else if (key != ~0ull) {
             status = (key & 1ull) ? WM_ERR_STRUCT : WM_ERR_DESC;
             first = ld_volatile_u32(&ws.ctrl->bad4_first); count = ld_volatile_u32(&ws.ctrl->bad4_count);
         } else if (ld_volatile_u32(&ws.ctrl->bad5_count)) {
