@@ -1544,13 +1544,9 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
                 const uint32_t base_l = desc & 0xFFu, chk = desc >> 12;
                 const bool bad = wv > 8u || chk != (((base_l & 15u) ^ (base_l >> 4) ^ wv ^ 5u) & 15u);
                 const bool anybad = __any_sync(0xFFFFFFFFu, bad);
-                uint32_t incl = wv;
-#pragma unroll
-                for (int k = 1; k < 32; k <<= 1) {
-                    const uint32_t o2 = __shfl_up_sync(0xFFFFFFFFu, incl, k);
-                    if (lane >= (uint32_t)k) incl += o2;
-                }
-                const uint32_t Ssum = __shfl_sync(0xFFFFFFFFu, incl, 31);
+                // sum of all 32 widths, and of the widths of the groups before this warp's four
+                const uint32_t Ssum = __reduce_add_sync(0xFFFFFFFFu, wv);
+                const uint32_t before = __reduce_add_sync(0xFFFFFFFFu, lane < 4u * warp ? wv : 0u);
                 const int verdict = anybad ? 1 : (258u + Ssum != e ? 2 : 0);
                 if (verdict) {               // every warp reaches the same verdict
                     decoded = false;
@@ -1559,10 +1555,17 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
                         atomicOr(&ws.cflag[chunk_of(g, t)], CF_BAD4);
                     }
                 } else {
-                    // this lane keeps, in desc, the descriptor of group 4 warp + (lane & 3) with the
+                    // lanes 0..3 end up with the descriptors of the warp's four groups, each with its
                     // group's offset in the plane area in the high half
-                    const uint32_t mine = (desc & 0xFFFFu) | ((incl - wv) << 16);
-                    desc = __shfl_sync(0xFFFFFFFFu, mine, 4 * warp + (lane & 3u));
+                    const uint32_t own = __shfl_sync(0xFFFFFFFFu, desc, 4 * warp + (lane & 3u)) & 0xFFFFu;
+                    const uint32_t wo = (own >> 8) & 15u;
+                    uint32_t off = before;                          // running offset over the four groups
+                    const uint32_t w0 = __shfl_sync(0xFFFFFFFFu, wo, 0), w1 = __shfl_sync(0xFFFFFFFFu, wo, 1),
+                                   w2 = __shfl_sync(0xFFFFFFFFu, wo, 2);
+                    if ((lane & 3u) >= 1u) off += w0;
+                    if ((lane & 3u) >= 2u) off += w1;
+                    if ((lane & 3u) == 3u) off += w2;
+                    desc = own | (off << 16);
 #pragma unroll
                     for (int j = 0; j < 4; j++) {
                         const uint32_t dg = __shfl_sync(0xFFFFFFFFu, desc, j);
@@ -1601,6 +1604,10 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
                 load_tile_words_guarded(src, len, fold, warp, lane, w);
                 fold = false;
             } else if (is_pack && decoded) {
+#ifdef WM_AB_D_NOUNPACK
+#pragma unroll
+                for (int j = 0; j < 4; j++) { w[4 * j] = sm[j].x; w[4 * j + 1] = sm[j].y; w[4 * j + 2] = pw[j].a; w[4 * j + 3] = pw[j].b; }
+#else
 #pragma unroll
                 for (int j = 0; j < 4; j++) {
                     const uint32_t dg = __shfl_sync(0xFFFFFFFFu, desc, j);
@@ -1617,23 +1624,35 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
                         case 8: unpack_group_planes<8>(pw[j], base, ea, eb); break;
                         default: break;
                     }
-                    uint32_t Tr[4];
-                    Tr[0] = __byte_perm(sm[j].x, ea, 0x5140);
-                    Tr[1] = __byte_perm(sm[j].x, ea, 0x7362);
-                    Tr[2] = __byte_perm(sm[j].y, eb, 0x5140);
-                    Tr[3] = __byte_perm(sm[j].y, eb, 0x7362);
-#pragma unroll
-                    for (int r = 0; r < 4; r++)
-                        w[4 * j + r] = ((Tr[r] >> 1) & 0x7FFF7FFFu) | ((Tr[r] << 15) & 0x80008000u);
+                    // A word rotated left by one bit reads [E | m << 1 | sign of the other half] in
+                    // each half: swap bit 0 inside the byte pairs of the sign-mantissa words, put
+                    // the exponent bytes beside them, rotate back.
+                    const uint32_t xa = __byte_perm(sm[j].x, sm[j].x, 0x2301), xb = __byte_perm(sm[j].y, sm[j].y, 0x2301);
+                    const uint32_t sa = (sm[j].x & 0xFEFEFEFEu) | (xa & 0x01010101u), sb = (sm[j].y & 0xFEFEFEFEu) | (xb & 0x01010101u);
+                    const uint32_t r0 = __byte_perm(sa, ea, 0x5140), r1 = __byte_perm(sa, ea, 0x7362);
+                    const uint32_t r2 = __byte_perm(sb, eb, 0x5140), r3 = __byte_perm(sb, eb, 0x7362);
+                    w[4 * j] = __funnelshift_r(r0, r0, 1);
+                    w[4 * j + 1] = __funnelshift_r(r1, r1, 1);
+                    w[4 * j + 2] = __funnelshift_r(r2, r2, 1);
+                    w[4 * j + 3] = __funnelshift_r(r3, r3, 1);
                 }
+#endif
             }
             if (decoded) {
+#ifndef WM_AB_D_NOSTORE
                 if (e != 0xFFFFu) {
                     unsigned char* q = o + warp * 2048u + lane * 4u;
 #pragma unroll
                     for (int i = 0; i < 16; i++) st_stream_u32(q + i * 128, w[i]);
                 }
+#else
+                if (w[7] == 0x12345678u && e != 0xFFFFu) st_stream_u32(o + lane * 4u, w[2] ^ w[9] ^ w[12] ^ w[15] ^ w[0] ^ w[5]);
+#endif
+#ifdef WM_AB_D_NOCRC
+                const uint32_t v = w[3] ^ w[6] ^ w[8] ^ w[13] ^ w[1] ^ w[4] ^ w[10] ^ w[11] ^ w[14];
+#else
                 const uint32_t v = tile_digest_part(S, w, fold, warp, lane);
+#endif
                 if (lane == 0) tc->wdig[p][warp] = v;
                 have_digest = true;
             }
