@@ -83,6 +83,36 @@ __device__ __forceinline__ uint32_t lds_off(uint32_t addr)
     return v;
 }
 
+// Loads of data that other threads or the copy engine write (stages, team control blocks),
+// addressed by 32-bit shared-window addresses so that the address arithmetic stays in 32 bits.
+// volatile: they keep their place relative to the barriers and mbarrier waits around them.
+template <int OFF>
+__device__ __forceinline__ uint32_t lds_now(uint32_t addr)
+{
+    uint32_t v;
+    asm volatile("ld.shared.u32 %0, [%1+%2];" : "=r"(v) : "r"(addr), "n"(OFF));
+    return v;
+}
+template <int OFF>
+__device__ __forceinline__ uint2 lds_now_v2(uint32_t addr)
+{
+    uint2 v;
+    asm volatile("ld.shared.v2.u32 {%0, %1}, [%2+%3];" : "=r"(v.x), "=r"(v.y) : "r"(addr), "n"(OFF));
+    return v;
+}
+__device__ __forceinline__ uint32_t lds_now_u16(uint32_t addr)
+{
+    uint32_t v;
+    asm volatile("{\n\t.reg .u16 t;\n\tld.shared.u16 t, [%1];\n\tcvt.u32.u16 %0, t;\n\t}" : "=r"(v) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ uint32_t lds_now_u8(uint32_t addr)
+{
+    uint32_t v;
+    asm volatile("ld.shared.u8 %0, [%1];" : "=r"(v) : "r"(addr));
+    return v;
+}
+
 __device__ __forceinline__ void team_bar(uint32_t team)
 {
     asm volatile("bar.sync %0, %1;" ::"r"(team + 1), "r"(kTeamThreads) : "memory");

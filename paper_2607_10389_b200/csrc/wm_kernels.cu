@@ -1402,19 +1402,19 @@ static_assert(sizeof(DecTeamCtl) % 16 == 0, "team control block keeps 16-byte al
 // in the low half and the 1-bit plane's byte in bits 16-23, or the high half of an 8-bit plane.
 struct PlaneWords { uint32_t a, b; };
 
-__device__ __forceinline__ PlaneWords read_group_planes(const unsigned char* rec, uint32_t wd, uint32_t lane)
+// rec: shared-window address of the group's planes; l4 / l2 / l1: 4, 2, 1 times the lane number
+__device__ __forceinline__ PlaneWords read_group_planes(uint32_t rec, uint32_t wd, uint32_t l4, uint32_t l2, uint32_t l1)
 {
     PlaneWords pw;
     pw.a = 0; pw.b = 0;
     if (wd == 8u) {
-        const uint2 v = *reinterpret_cast<const uint2*>(rec + 8 * lane);
+        const uint2 v = lds_now_v2<0>(rec + 2u * l4);
         pw.a = v.x; pw.b = v.y;
         return pw;
     }
-    const unsigned char* p = rec;
-    if (wd & 4u) { pw.a = *reinterpret_cast<const uint32_t*>(p + 4 * lane); p += 128; }
-    if (wd & 2u) { pw.b = *reinterpret_cast<const uint16_t*>(p + 2 * lane); p += 64; }
-    if (wd & 1u) { pw.b |= (uint32_t)p[lane] << 16; }
+    if (wd & 4u) { pw.a = lds_now<0>(rec + l4); rec += 128u; }
+    if (wd & 2u) { pw.b = lds_now_u16(rec + l2); rec += 64u; }
+    if (wd & 1u) { pw.b |= lds_now_u8(rec + l1) << 16; }
     return pw;
 }
 
@@ -1485,6 +1485,8 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
     const unsigned char* const payload = wire + g.meta_end;
     const bool leader = (tt == 0);
     constexpr uint32_t kNone = 0xFFFFFFFFu;
+    const uint32_t stage_s = (uint32_t)__cvta_generic_to_shared(stage);
+    const uint32_t sm_s = stage_s + 64u + 1024u * warp + 8u * lane;     // this lane's sign-mantissa bytes, group 4 warp
 
     // a tile's entry word and payload offset (blocking: prologue only)
     auto lookup = [&](uint32_t t, DecSlot* sl) {
@@ -1539,7 +1541,11 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
             if (!is_pack) {
                 read_staged_words(stage, warp, lane, w);
             } else {
-                desc = reinterpret_cast<const uint16_t*>(stage)[lane];
+#ifdef WM_AB_D_NOP1
+                desc = 100u | (4u << 8);
+                for (int j = 0; j < 4; j++) { sm[j] = make_uint2(lane, it); pw[j].a = t; pw[j].b = e; }
+#else
+                desc = lds_now_u16(stage_s + 2u * lane);
                 const uint32_t wv = (desc >> 8) & 15u;
                 const uint32_t base_l = desc & 0xFFu, chk = desc >> 12;
                 const bool bad = wv > 8u || chk != (((base_l & 15u) ^ (base_l >> 4) ^ wv ^ 5u) & 15u);
@@ -1569,10 +1575,11 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
 #pragma unroll
                     for (int j = 0; j < 4; j++) {
                         const uint32_t dg = __shfl_sync(0xFFFFFFFFu, desc, j);
-                        sm[j] = *reinterpret_cast<const uint2*>(stage + 64 + 256 * (4 * warp + j) + 8 * lane);
-                        pw[j] = read_group_planes(stage + 8256 + 32 * (dg >> 16), (dg >> 8) & 15u, lane);
+                        sm[j] = j == 0 ? lds_now_v2<0>(sm_s) : j == 1 ? lds_now_v2<256>(sm_s) : j == 2 ? lds_now_v2<512>(sm_s) : lds_now_v2<768>(sm_s);
+                        pw[j] = read_group_planes(stage_s + 8256u + 32u * (dg >> 16), (dg >> 8) & 15u, 4u * lane, 2u * lane, lane);
                     }
                 }
+#endif
             }
         }
         team_bar(team);                      // stage free; the slots the leader filled last step visible;
