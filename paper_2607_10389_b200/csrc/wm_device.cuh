@@ -113,6 +113,16 @@ __device__ __forceinline__ uint32_t lds_now_u8(uint32_t addr)
     return v;
 }
 
+// Programmatic dependent launch.  Every call enqueues a short chain of kernels; each kernel but
+// the first is launched with permission to start before its predecessor has finished.  It then
+// sets up what does not depend on the predecessor (tables into shared memory, allocations) and
+// waits here; the wait returns once the predecessor has completed and its writes are visible.
+// Every block of such a kernel must pass the wait before it exits or reads anything the chain
+// produced.  A kernel tells the scheduler that its successor may be brought in with
+// grid_dep_launch (the successor's blocks take SM resources as they become free).
+__device__ __forceinline__ void grid_dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_dep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 __device__ __forceinline__ void team_bar(uint32_t team)
 {
     asm volatile("bar.sync %0, %1;" ::"r"(team + 1), "r"(kTeamThreads) : "memory");

@@ -349,6 +349,7 @@ template <int TEAMS>
 __global__ void __launch_bounds__(TEAMS * 256, 1)
 k_tile_digests(const unsigned char* __restrict__ cache, Geo g, Ws ws, const Tables* __restrict__ tab)
 {
+    grid_dep_launch();
     extern __shared__ __align__(16) unsigned char smem[];
     Smem S = setup_smem(smem, tab);
     const uint32_t team = threadIdx.x / kTeamThreads, tt = threadIdx.x % kTeamThreads;
@@ -402,6 +403,7 @@ k_checksum_finish(const unsigned char* __restrict__ cache, Geo g, Ws ws, const T
     __shared__ uint32_t sT0[256];
     __shared__ FinishStage stage;
     load_ht_t0(sHT, sT0, tab);
+    grid_dep_wait();
     const uint32_t c0 = blockIdx.x * g.finish_cb;
     stage_chunk_digests(g, stage, ws.dig, c0);
     const uint32_t c = c0 + threadIdx.x;
@@ -413,6 +415,7 @@ k_checksum_finish(const unsigned char* __restrict__ cache, Geo g, Ws ws, const T
 
 __global__ void k_diff_init(Ws ws)
 {
+    grid_dep_launch();
     if (threadIdx.x == 0 && blockIdx.x == 0) { ws.ctrl->ticket = 0; ws.ctrl->n_present = 0; }
 }
 
@@ -424,6 +427,8 @@ k_diff(const unsigned char* __restrict__ cache, const unsigned char* __restrict_
 {
     __shared__ uint32_t s_chunk;
     constexpr uint32_t kStep = 256 * 16 * 8;      // bytes per block step
+    grid_dep_wait();
+    grid_dep_launch();
     while (true) {
         __syncthreads();
         if (threadIdx.x == 0) s_chunk = atomicAdd(&ws.ctrl->ticket, 1u);
@@ -470,6 +475,7 @@ k_diff_compact(Geo g, const uint8_t* __restrict__ dirty, uint32_t* __restrict__ 
     __shared__ uint32_t s_warp[32];
     __shared__ uint32_t s_carry;
     const uint32_t lane = threadIdx.x % 32, warp = threadIdx.x / 32;
+    grid_dep_wait();
     if (threadIdx.x == 0) s_carry = 0;
     __syncthreads();
     for (uint32_t base = 0; base < g.n_chunks; base += 1024) {
@@ -496,6 +502,7 @@ k_diff_compact(Geo g, const uint8_t* __restrict__ dirty, uint32_t* __restrict__ 
 
 __global__ void k_encode_init(Geo g, Ws ws, unsigned char* wire)
 {
+    grid_dep_launch();
     const uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
     const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
     for (uint64_t t = i; t < g.n_tiles; t += stride) ws.lbk[t] = 0u;
@@ -774,14 +781,16 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
     // that shares its scheduler with busy ones gets too few issue slots to keep up).
     __shared__ uint32_t s_scanner;
     __shared__ uint32_t s_tmem;
+    Smem S = setup_smem(smem, tab);
+    grid_dep_wait();                   // from here on the control block and the length table are ready
+    grid_dep_launch();
     if (threadIdx.x == 0) s_scanner = atomicCAS(&ws.ctrl->scan_lock, 0u, 1u) == 0u;
     __syncthreads();
     if (s_scanner) {
-        if (threadIdx.x < 32)
-            scan_tile_lengths(ws.lbk, g.n_tiles, threadIdx.x, ws.ctrl, reinterpret_cast<uint32_t*>(smem));
+        uint32_t* win = reinterpret_cast<uint32_t*>(S.take(2048));      // 512 entries
+        if (threadIdx.x < 32 && win) scan_tile_lengths(ws.lbk, g.n_tiles, threadIdx.x, ws.ctrl, win);
         return;
     }
-    Smem S = setup_smem(smem, tab);
     const uint32_t team = threadIdx.x / kTeamThreads, tt = threadIdx.x % kTeamThreads;
     const uint32_t warp = tt / 32, lane = tt % 32;
     unsigned char* stage = nullptr;
@@ -1062,6 +1071,8 @@ k_encode_finish(const unsigned char* __restrict__ cache, Geo g, const uint8_t* _
     __shared__ uint32_t s_acc;
     __shared__ bool s_last;
     load_ht_t0(sHT, sT0, tab);
+    grid_dep_wait();
+    grid_dep_launch();
     const uint32_t c0 = blockIdx.x * g.finish_cb;
     stage_chunk_digests(g, stage, ws.dig, c0);
     unsigned char* dir = wire + 64;
@@ -1134,6 +1145,8 @@ k_meta_crc(unsigned char* wire, uint64_t wire_len, Geo g, Ws ws, const Tables* _
     if (!S.ok) { if (threadIdx.x == 0) atomicOr(&ws.ctrl->err, 4u); return; }
     tc += team;
     sHT[threadIdx.x] = (&tab->HT[0][0])[threadIdx.x];
+    grid_dep_wait();
+    grid_dep_launch();
 
     if (mode == 1) {
         // FORMAT check by every block (cheap, keeps the gate decision local)
@@ -1242,6 +1255,7 @@ k_meta_crc(unsigned char* wire, uint64_t wire_len, Geo g, Ws ws, const Tables* _
 
 __global__ void k_decode_init(Ws ws)
 {
+    grid_dep_launch();
     if (blockIdx.x == 0 && threadIdx.x < sizeof(Ctrl) / 4) {
         uint32_t v = 0;
         const uint32_t i = threadIdx.x;
@@ -1275,6 +1289,8 @@ __device__ __forceinline__ void fill_result(wm_result* result, const Ctrl* ctrl,
 __global__ void __launch_bounds__(1024)
 k_decode_struct(const unsigned char* __restrict__ wire, uint64_t wire_len, Geo g, Ws ws, wm_result* result)
 {
+    grid_dep_wait();
+    grid_dep_launch();
     if (ld_volatile_u32(&ws.ctrl->gate)) return;
     __shared__ unsigned long long s_warp[32];
     __shared__ unsigned long long s_carry;
@@ -1467,9 +1483,11 @@ __global__ void __launch_bounds__(TEAMS * 256, 1)
 k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restrict__ dst, Ws ws,
          const Tables* __restrict__ tab)
 {
-    if (ld_volatile_u32(&ws.ctrl->gate)) return;
     extern __shared__ __align__(16) unsigned char smem[];
     Smem S = setup_smem(smem, tab);
+    grid_dep_wait();
+    grid_dep_launch();
+    if (ld_volatile_u32(&ws.ctrl->gate)) return;
     const uint32_t team = threadIdx.x / kTeamThreads, tt = threadIdx.x % kTeamThreads;
     const uint32_t warp = tt / 32, lane = tt % 32;
     unsigned char* stage = nullptr;
@@ -1687,7 +1705,6 @@ k_decode_finish(const unsigned char* __restrict__ wire, uint64_t wire_len, Geo g
                 const unsigned char* __restrict__ dst, uint32_t* __restrict__ dst_crc, Ws ws,
                 const Tables* __restrict__ tab, wm_result* result, const __grid_constant__ ChunkPowers cp)
 {
-    if (ld_volatile_u32(&ws.ctrl->gate)) return;
     __shared__ uint32_t sHT[1024];
     __shared__ uint32_t sT0[256];
     __shared__ FinishStage stage;
@@ -1695,6 +1712,8 @@ k_decode_finish(const unsigned char* __restrict__ wire, uint64_t wire_len, Geo g
     __shared__ bool s_last;
     __shared__ int s_status;
     load_ht_t0(sHT, sT0, tab);
+    grid_dep_wait();
+    if (ld_volatile_u32(&ws.ctrl->gate)) return;
     const uint32_t c0 = blockIdx.x * g.finish_cb;
     stage_chunk_digests(g, stage, ws.dig, c0);
     const unsigned char* dir = wire + 64;
@@ -1813,6 +1832,24 @@ static const DeviceState* device_state()
     return &s;
 }
 
+// Launch a kernel that may start before the kernel enqueued just before it on the stream has
+// finished (it waits inside, see grid_dep_wait).
+template <typename... Params, typename... Args>
+static void launch_after(void (*kernel)(Params...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, Args&&... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    cudaLaunchKernelEx(&cfg, kernel, static_cast<Params>(args)...);
+}
+
 static bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 static wm_status launch_status()
@@ -1876,7 +1913,7 @@ wm_status wm_checksum(const void* cache, uint64_t nbytes, uint32_t chunk_bytes, 
         MainKernelTimer timer(ds, 0, s);
         k_tile_digests<kTeamsPlain><<<grid, kTeamsPlain * 256, kDynSmem, s>>>(c, g, ws, ds->tables);
     }
-    k_checksum_finish<<<(g.n_chunks + g.finish_cb - 1) / g.finish_cb, 1024, 0, s>>>(c, g, ws, ds->tables, crc_out);
+    launch_after(k_checksum_finish, (g.n_chunks + g.finish_cb - 1) / g.finish_cb, 1024, 0, s, c, g, ws, ds->tables, crc_out);
     g_launches = 2;
     return launch_status();
 }
@@ -1945,7 +1982,7 @@ wm_status wm_checksum_noalloc(const void* cache, uint64_t nbytes, uint32_t chunk
     const uint32_t need = (g.n_tiles + kTeamsPlain - 1) / kTeamsPlain;
     const uint32_t grid = need < (uint32_t)ns->sm_count ? need : (uint32_t)ns->sm_count;
     k_tile_digests<kTeamsPlain><<<grid, kTeamsPlain * 256, kDynSmem, s>>>(c, g, ws, ns->tables);
-    k_checksum_finish<<<(g.n_chunks + g.finish_cb - 1) / g.finish_cb, 1024, 0, s>>>(c, g, ws, ns->tables, crc_out);
+    launch_after(k_checksum_finish, (g.n_chunks + g.finish_cb - 1) / g.finish_cb, 1024, 0, s, c, g, ws, ns->tables, crc_out);
     g_launches = 2;
     return launch_status();
 }
@@ -1966,9 +2003,9 @@ wm_status wm_dirty_diff(const void* cache, const void* prev, uint64_t nbytes, ui
     const uint32_t grid = g.n_chunks < want ? g.n_chunks : want;
     {
         MainKernelTimer timer(ds, 1, s);
-        k_diff<<<grid, 256, 0, s>>>(static_cast<const unsigned char*>(cache), static_cast<const unsigned char*>(prev), g, ws, dirty_out);
+        launch_after(k_diff, grid, 256, 0, s, static_cast<const unsigned char*>(cache), static_cast<const unsigned char*>(prev), g, ws, dirty_out);
     }
-    k_diff_compact<<<1, 1024, 0, s>>>(g, dirty_out, dirty_idx_out, n_dirty_out);
+    launch_after(k_diff_compact, 1, 1024, 0, s, g, dirty_out, dirty_idx_out, n_dirty_out);
     g_launches = 3;
     return launch_status();
 }
@@ -1996,11 +2033,12 @@ wm_status wm_encode(const void* cache, uint64_t nbytes, uint32_t chunk_bytes, co
     const uint32_t grid = need < (uint32_t)ds->sm_count ? need : (uint32_t)ds->sm_count;
     {
         MainKernelTimer timer(ds, 2, s);
-        if (dirty) k_encode<kTeams, true><<<grid, kTeams * 256, kDynSmem, s>>>(c, g, dirty, w, wire_cap, ws, ds->tables);
-        else k_encode<kTeams, false><<<grid, kTeams * 256, kDynSmem, s>>>(c, g, dirty, w, wire_cap, ws, ds->tables);
+        if (dirty) launch_after(k_encode<kTeams, true>, grid, kTeams * 256, kDynSmem, s, c, g, dirty, w, wire_cap, ws, ds->tables);
+        else launch_after(k_encode<kTeams, false>, grid, kTeams * 256, kDynSmem, s, c, g, dirty, w, wire_cap, ws, ds->tables);
     }
-    k_encode_finish<<<(g.n_chunks + g.finish_cb - 1) / g.finish_cb, 1024, 0, s>>>(c, g, dirty, crc_inout, w, ws, ds->tables, chunk_powers(g));
-    k_meta_crc<<<(g.n_meta_slices + 3) / 4, 1024, kDynSmem, s>>>(w, 0, g, ws, ds->tables, result, 0);
+    launch_after(k_encode_finish, (g.n_chunks + g.finish_cb - 1) / g.finish_cb, 1024, 0, s, c, g, dirty, crc_inout, w, ws, ds->tables,
+                 chunk_powers(g));
+    launch_after(k_meta_crc, (g.n_meta_slices + 3) / 4, 1024, kDynSmem, s, w, (uint64_t)0, g, ws, ds->tables, result, 0);
     g_launches = 4;
     return launch_status();
 }
@@ -2022,15 +2060,16 @@ wm_status wm_decode_verify(const void* wire, uint64_t wire_len, void* dst, uint6
     k_decode_init<<<1, 64, 0, s>>>(ws);
     // a wire shorter than the metadata is rejected by the header check before anything else is read
     const uint32_t slices = wire_len >= g.meta_end ? g.n_meta_slices : 1;
-    k_meta_crc<<<(slices + 3) / 4, 1024, kDynSmem, s>>>(const_cast<unsigned char*>(w), wire_len, g, ws, ds->tables, result, 1);
-    k_decode_struct<<<(g.n_chunks + 31) / 32, 1024, 0, s>>>(w, wire_len, g, ws, result);
+    launch_after(k_meta_crc, (slices + 3) / 4, 1024, kDynSmem, s, const_cast<unsigned char*>(w), wire_len, g, ws, ds->tables, result, 1);
+    launch_after(k_decode_struct, (g.n_chunks + 31) / 32, 1024, 0, s, w, wire_len, g, ws, result);
     const uint32_t need = (g.n_tiles + kTeamsPlain - 1) / kTeamsPlain;
     const uint32_t grid = need < (uint32_t)ds->sm_count ? need : (uint32_t)ds->sm_count;
     {
         MainKernelTimer timer(ds, 3, s);
-        k_decode<kTeamsPlain><<<grid, kTeamsPlain * 256, kDynSmem, s>>>(w, g, d, ws, ds->tables);
+        launch_after(k_decode<kTeamsPlain>, grid, kTeamsPlain * 256, kDynSmem, s, w, g, d, ws, ds->tables);
     }
-    k_decode_finish<<<(g.n_chunks + g.finish_cb - 1) / g.finish_cb, 1024, 0, s>>>(w, wire_len, g, d, dst_crc_inout, ws, ds->tables, result, chunk_powers(g));
+    launch_after(k_decode_finish, (g.n_chunks + g.finish_cb - 1) / g.finish_cb, 1024, 0, s, w, wire_len, g, d, dst_crc_inout, ws, ds->tables,
+                 result, chunk_powers(g));
     g_launches = 5;
     return launch_status();
 }
