@@ -155,6 +155,83 @@ def make_workload(name, device):
     return cfg, cur, prev, int(mask.sum())
 
 
+def precopy_loop(wm, inputs, cfg, cur, prev, dst, wire_a, ws_a, dev, peak, steps=20):
+    """Twenty generation steps on two streams; returns per-step time and per-step dirty bytes."""
+    import torch
+    N, C = cfg.nbytes, cfg.chunk_bytes
+    nc = wm.num_chunks(N, C)
+    wires = [wire_a, torch.empty_like(wire_a)]
+    ws_b = wm.new_workspace(N, C, dev)
+    src, dstream = torch.cuda.Stream(), torch.cuda.Stream()
+    crc_src = torch.zeros(nc, dtype=torch.int32, device=dev)
+    crc_dst = torch.zeros(nc, dtype=torch.int32, device=dev)
+    dirty = torch.zeros(nc, dtype=torch.uint8, device=dev)
+    n_dirty = torch.zeros(1, dtype=torch.int32, device=dev)
+    res_e = [wm.new_result(dev) for _ in range(steps)]
+    res_d = [wm.new_result(dev) for _ in range(steps)]
+    # level the two sides first (full move), and keep pristine copies to restore afterwards
+    keep_cur, keep_prev = cur.clone(), prev.clone()
+    wm.wm_encode(cur, C, None, crc_src, wires[0], ws_a, res_e[0])
+    r = wm.read_result(res_e[0])
+    wm.wm_decode_verify(wires[0], r.wire_len, dst, C, crc_dst, ws_a, res_d[0])
+    if not wm.read_result(res_d[0]).ok:
+        raise SystemExit("pre-copy loop: levelling move failed")
+    prev.copy_(cur)
+    masks = [inputs.step_pattern(nc, cfg.shape[0], 0.75, seed=1000 + k) for k in range(steps)]
+    # The rewrites stand for the engine's own writes, so they sit outside the timed events: per
+    # step one event pair brackets diff + encode on the source stream, another the decode on the
+    # destination stream.
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(5)] for _ in range(steps)]
+    torch.cuda.synchronize()
+    wall0 = time.perf_counter()
+    lens = []
+    for k in range(steps):
+        wire = wires[(k + 1) % 2]
+        with torch.cuda.stream(src):
+            ev[k][4].record(src)
+            inputs.apply_step(cur, C, masks[k], seed=5000 + k)
+            ev[k][0].record(src)
+            wm.wm_dirty_diff(cur, prev, C, dirty, None, n_dirty, ws_a, stream=src)
+            wm.wm_encode(cur, C, dirty, crc_src, wire, ws_a, res_e[k], stream=src)
+            ev[k][1].record(src)
+            rr = wm.read_result(res_e[k])                 # the destination needs wire_len
+            if not rr.ok:
+                raise SystemExit(f"pre-copy loop: encode failed at step {k}: {rr.status_name}")
+            lens.append((rr.wire_len, rr.n_present))
+            prev.copy_(cur, non_blocking=True)
+        with torch.cuda.stream(dstream):
+            dstream.wait_event(ev[k][1])
+            ev[k][2].record(dstream)
+            wm.wm_decode_verify(wire, rr.wire_len, dst, C, crc_dst, ws_b, res_d[k], stream=dstream)
+            ev[k][3].record(dstream)
+    torch.cuda.synchronize()
+    wall_ms = (time.perf_counter() - wall0) * 1e3 / steps
+    for k in range(steps):
+        if not wm.read_result(res_d[k]).ok:
+            raise SystemExit(f"pre-copy loop: decode failed at step {k}")
+    if not torch.equal(dst, cur) or not torch.equal(crc_dst, crc_src):
+        raise SystemExit("pre-copy loop: destination differs from the source after the last step")
+    src_ms = [ev[k][0].elapsed_time(ev[k][1]) for k in range(steps)]
+    dst_ms = [ev[k][2].elapsed_time(ev[k][3]) for k in range(steps)]
+    dirty_bytes = [min(n * C, N) for _, n in lens]
+    mean_dirty = sum(dirty_bytes) / steps
+    mean_wire = sum(w for w, _ in lens) / steps
+    cur.copy_(keep_cur)
+    prev.copy_(keep_prev)
+    torch.cuda.synchronize()
+    s_ms, d_ms = statistics.mean(src_ms), statistics.mean(dst_ms)
+    rewrite_ms = statistics.mean(ev[k][4].elapsed_time(ev[k][0]) for k in range(steps))
+    return {"steps": steps, "streams": 2, "dirty_fraction": mean_dirty / N, "wire_bytes_per_step": mean_wire,
+            "wall_ms_per_step": wall_ms, "rewrite_ms_per_step": rewrite_ms,
+            "source_ms_per_step": s_ms, "dest_ms_per_step": d_ms,
+            "source_dirty_gbs": mean_dirty / (s_ms * 1e-3) / 1e9, "dest_dirty_gbs": mean_dirty / (d_ms * 1e-3) / 1e9,
+            "dest_frac_of_hbm_peak": (mean_dirty + mean_wire) / (d_ms * 1e-3) / 1e9 / peak,
+            "note": "source = wm_dirty_diff + wm_encode(dirty chunks only); dest = wm_decode_verify into the live "
+                    "copy; the destination of step k runs beside the source of step k+1, so each stream's time includes waiting for "
+                    "SMs the other holds; wall = host clock over the whole loop per step, rewrite = the stand-in for the "
+                    "engine's own writes"}
+
+
 def run_reference(args):
     """Reference arm: the CPU oracle timed on the host cores, a bounded sample per step."""
     rank, _, world = _dist()
@@ -206,6 +283,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-loop", action="store_true", help="skip the pre-copy step loop")
     ap.add_argument("--profile", action="store_true",
                     help="profiler capture mode: round-trip check, warm-up and timed steps only")
     args = ap.parse_args()
@@ -216,11 +294,12 @@ def main():
     args.steps = 100 if args.steps is None else args.steps
     args.warmup = 5 if args.warmup is None else max(args.warmup, 3)
     if args.profile:
-        args.no_e2e = args.no_cpu_baseline = True
+        args.no_e2e = args.no_cpu_baseline = args.no_loop = True
 
     import numpy as np
     import torch
     from paper_2607_10389_b200 import binding as wm
+    from paper_2607_10389_b200 import inputs as inputs_mod
 
     rank, local_rank, world = _dist()
     if not torch.cuda.is_available():
@@ -371,6 +450,13 @@ def main():
                 "decode_frac": per_call["decode_verify"]["frac_of_hbm_peak"],
                 "decode_call_frac": per_call["decode_verify"]["call_frac_of_hbm_peak"]}
 
+    # pre-copy step loop (the fifth workload): per generation step the source rewrites three
+    # quarters of the chunks, then diff -> encode(dirty only) on one stream and
+    # decode-verify-install on another (two wire buffers), 20 steps, device-timed as a whole
+    loop = None
+    if not args.no_loop and args.workload in ("engine", "engine_256m"):
+        loop = precopy_loop(wm, inputs_mod, cfg, cur, prev, shadow, wire, ws, dev, peak)
+
     # end to end: host cache in (pinned), verified wire image and result records out
     e2e = None
     if not args.no_e2e:
@@ -414,7 +500,7 @@ def main():
             "config": {"workload": args.workload, "nbytes": N, "chunk_bytes": C, "shape": list(cfg.shape),
                        "wire_bytes": W, "ratio": W / N, "dirty_chunks": n_rewritten, "n_chunks": nc,
                        "l2": "inputs larger than L2 (no flush needed)", "parallelism": "replicas only"},
-            "calls": per_call, "roofline": roofline, "cpu_baseline": base, "e2e": e2e,
+            "calls": per_call, "roofline": roofline, "precopy_loop": loop, "cpu_baseline": base, "e2e": e2e,
             "gpu_launches": gpu_launches, "clocks": clocks,
         }
         print(json.dumps(out))
