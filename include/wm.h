@@ -18,6 +18,10 @@
  *     small or not 16-byte aligned, wire_cap below the metadata size), WM_ERR_CUDA for
  *     a launch failure, else WM_OK.
  *   - Calls that share a workspace must be ordered on one stream (or by events).
+ *   - A call enqueues a short chain of kernels; all but the first are launched with
+ *     programmatic stream serialization (they may start while their predecessor drains and
+ *     wait inside before touching its results).  Work enqueued by the caller before or after
+ *     a call keeps ordinary stream order.
  *   - All integers in the wire image are little-endian.  Tile = 16384 bytes, group = 256
  *     bf16 elements; n_chunks = ceil(nbytes / chunk_bytes), n_tiles = ceil(nbytes / 16384).
  */
@@ -150,6 +154,9 @@ wm_status wm_encode(const void* cache, uint64_t nbytes, uint32_t chunk_bytes, co
  *   6 absent chunk: dst_crc_inout[c] equals its directory CRC      WM_ERR_STALE
  *   7 the directory CRCs combine to header.cache_crc               WM_ERR_CACHE_CRC
  *   8 only then dst_crc_inout[c] <- crc for present chunks, status WM_OK
+ * A bounded device-side wait that ran out (a bulk copy that never arrived) gives WM_ERR_TIMEOUT
+ * ahead of steps 4..7: the kernels failed, nothing can be said about the image, nothing is
+ * installed.
  *   dst           [dev] nbytes bytes, 16-byte aligned: the SHADOW slot.  Present chunks are
  *                 written, absent chunks are left as they are.  On any failure its content is
  *                 unspecified (never written outside [dst, dst+nbytes)) and dst_crc_inout is
