@@ -167,6 +167,39 @@ __device__ __forceinline__ uint32_t warp_place(const Smem& S, uint32_t digest, u
     return __reduce_xor_sync(0xFFFFFFFFu, v);
 }
 
+// ---- the same digest with small tables, for kernels that see a few hundred kilobytes ----
+// Copying the 144 KiB lane-replicated image costs more than such a kernel's whole work.  Here
+// the chain uses one copy of the four byte tables (4 KiB in shared memory, taken from lane 0's
+// column of the image; lookups may collide on a bank) and the two once-per-tile steps read the
+// nibble tables straight from global memory.  Same result as warp_block_digest + warp_place.
+__device__ __forceinline__ void load_small_chain_tables(uint32_t* sG, const Tables* __restrict__ tab)
+{
+    for (uint32_t i = threadIdx.x; i < 1024; i += blockDim.x) {
+        const uint32_t k = i >> 8, b = i & 255u;
+        sG[i] = tab->image[((k < 2 ? kImgA01 : kImgA23) + b * 256u + (k & 1u) * 128u) / 4u];
+    }
+    __syncthreads();
+}
+__device__ __forceinline__ uint32_t tile_digest_part_small(const uint32_t* sG, const Tables* __restrict__ tab,
+                                                           const uint32_t (&w)[kWordsPerLane], uint32_t warp, uint32_t lane)
+{
+    uint32_t s = 0;
+#pragma unroll
+    for (int i = 0; i < 15; i++) {
+        const uint32_t x = s ^ w[i];
+        s = sG[x & 0xFFu] ^ sG[256u + ((x >> 8) & 0xFFu)] ^ sG[512u + ((x >> 16) & 0xFFu)] ^ sG[768u + (x >> 24)];
+    }
+    const uint32_t x = s ^ w[15];
+    uint32_t r = 0;
+#pragma unroll
+    for (uint32_t n = 0; n < 8; n++)
+        r ^= __ldg(&tab->image[(kImgNK + (n / 2u) * 0x1000u + ((x >> (4u * n)) & 15u) * 256u + (n & 1u) * 128u) / 4u + lane]);
+    const uint32_t digest = __reduce_xor_sync(0xFFFFFFFFu, r);
+    uint32_t v = 0;
+    if (lane < 8) v = __ldg(&tab->NW[warp][lane][(digest >> (4 * lane)) & 15u]);
+    return __reduce_xor_sync(0xFFFFFFFFu, v);
+}
+
 // Generic product of two residues (bitwise; used a handful of times per call).
 __device__ __forceinline__ uint32_t mulmod_dev(uint32_t a, uint32_t b)
 {

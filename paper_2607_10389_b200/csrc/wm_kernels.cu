@@ -6,8 +6,7 @@
 //   wm_encode        : k_encode_init -> k_encode (single pass; teams publish tile lengths, one
 //                      scanner warp turns them into payload offsets) -> k_encode_finish (directory, cache CRC, header)
 //                      -> k_meta_crc (metadata CRC, result)
-//   wm_decode_verify : k_decode_init -> k_meta_crc (header + metadata CRC gate)
-//                      -> k_decode_struct (structure gate)
+//   wm_decode_verify : k_decode_init -> k_decode_check (header, metadata CRC, structure: the gate)
 //                      -> k_decode (unpack + CRC of decoded bytes) -> k_decode_finish
 #include <cstdint>
 #include <cstdio>
@@ -1123,61 +1122,81 @@ k_encode_finish(const unsigned char* __restrict__ cache, Geo g, const uint8_t* _
     ws.ctrl->payload_total = total;
 }
 
-// CRC32C of the metadata region wire[0, meta_end) with the meta_crc field read as zero.
-// The region is right-aligned in a whole number of virtual 16 KiB slices (leading zeros),
-// one team per slice, four teams per block; the last block to finish folds the slice digests.
-//   mode 0 (encode): store the CRC into the header and write the result record.
-//   mode 1 (decode): check the header against the call (FORMAT), then the CRC (META_CRC);
-//                    on failure set the gate and write the result record.
+// ---- metadata CRC and structure checks ----
+// CRC32C of the metadata region wire[0, meta_end) with the meta_crc field read as zero.  The
+// region is right-aligned in a whole number of virtual 16 KiB slices (leading zeros), one team
+// per slice, four teams per block; the last block to finish folds the slice digests.  These
+// kernels see a few hundred kilobytes: they use the small tables.
+
+// The header against the call's arguments (decode step 1).
+__device__ __forceinline__ bool header_matches(const unsigned char* wire, uint64_t wire_len, const Geo& g)
+{
+    if (wire_len < 64) return false;
+    const uint32_t* h = reinterpret_cast<const uint32_t*>(wire);
+    const unsigned long long nb = h[2] | ((unsigned long long)h[3] << 32);
+    const unsigned long long pb = h[8] | ((unsigned long long)h[9] << 32);
+    const unsigned long long wl = h[10] | ((unsigned long long)h[11] << 32);
+    return !(h[0] != 0x31564D57u || (h[1] & 0xFFFFu) != 1u || (h[1] >> 16) > 1u || nb != g.nbytes ||
+             h[4] != g.chunk_bytes || h[5] != kTile || h[6] != g.n_chunks || wl != wire_len ||
+             wire_len < g.meta_end || pb != wire_len - g.meta_end);
+}
+
+// One team: its warps' parts of the digest of metadata slice s go to wdig[0..7].
+__device__ __forceinline__ void meta_slice_parts(const unsigned char* wire, const Geo& g, uint32_t s, const uint32_t* sG,
+                                                 const Tables* __restrict__ tab, uint32_t* wdig, uint32_t warp, uint32_t lane)
+{
+    const uint64_t pad = (uint64_t)g.n_meta_slices * kTile - g.meta_end;    // multiple of 4
+    uint32_t w[kWordsPerLane];
+#pragma unroll
+    for (int i = 0; i < 16; i++) {
+        const uint64_t vb = (uint64_t)s * kTile + (warp * 16 + i) * 128 + lane * 4;
+        uint32_t v = 0;
+        if (vb >= pad) {
+            const uint64_t rb = vb - pad;
+            v = *reinterpret_cast<const uint32_t*>(wire + rb);
+            if (rb == 52) v = 0;                      // the meta_crc field reads as zero
+            if (rb == 0) v ^= 0xFFFFFFFFu;            // the CRC's all-ones start value
+        }
+        w[i] = v;
+    }
+    const uint32_t v = tile_digest_part_small(sG, tab, w, warp, lane);
+    if (lane == 0) wdig[warp] = v;
+}
+
+// Whole block: fold the slice digests (fetched 1024 at a time, one round trip to L2 per batch,
+// folded by one thread out of shared memory).  The CRC is valid in thread 0.
+__device__ uint32_t fold_meta_digests(const Geo& g, const Ws& ws, const uint32_t* sHT, uint32_t* s_dig)
+{
+    uint32_t st = 0;
+    for (uint32_t b0 = 0; b0 < g.n_meta_slices; b0 += 1024) {
+        const uint32_t nb = min(1024u, g.n_meta_slices - b0);
+        __syncthreads();
+        if (threadIdx.x < nb) s_dig[threadIdx.x] = ld_volatile_u32(&ws.mdig[b0 + threadIdx.x]);
+        __syncthreads();
+        if (threadIdx.x == 0)
+            for (uint32_t i = 0; i < nb; i++) st = advance_tile(sHT, st) ^ s_dig[i];
+    }
+    return ~st;
+}
+
+// Encode: the metadata CRC goes into the header, the result record is written.  This kernel
+// starts while k_encode_finish still runs, so copying the large tables costs nothing here and
+// the digest itself is the fast one.
 __global__ void __launch_bounds__(1024, 1)
-k_meta_crc(unsigned char* wire, uint64_t wire_len, Geo g, Ws ws, const Tables* __restrict__ tab,
-           wm_result* result, int mode)
+k_meta_crc(unsigned char* wire, Geo g, Ws ws, const Tables* __restrict__ tab, wm_result* result)
 {
     extern __shared__ __align__(16) unsigned char smem[];
     __shared__ bool s_last;
-    __shared__ int s_format_bad;
     Smem S = setup_smem(smem, tab);
     const uint32_t team = threadIdx.x / kTeamThreads, tt = threadIdx.x % kTeamThreads;
     const uint32_t warp = tt / 32, lane = tt % 32;
-    TeamCtl* tc = reinterpret_cast<TeamCtl*>(S.take(4 * sizeof(TeamCtl)));
+    uint32_t* s_wdig = reinterpret_cast<uint32_t*>(S.take(4 * 8 * 4));
     uint32_t* sHT = reinterpret_cast<uint32_t*>(S.take(4096));
     uint32_t* s_dig = reinterpret_cast<uint32_t*>(S.take(4096));
-    if (!S.ok) { if (threadIdx.x == 0) atomicOr(&ws.ctrl->err, 4u); return; }
-    tc += team;
+    if (!S.ok) { if (threadIdx.x == 0) atomicOr(&ws.ctrl->err, 4u); grid_dep_wait(); return; }
+    s_wdig += 8 * team;
     sHT[threadIdx.x] = (&tab->HT[0][0])[threadIdx.x];
     grid_dep_wait();
-    grid_dep_launch();
-
-    if (mode == 1) {
-        // FORMAT check by every block (cheap, keeps the gate decision local)
-        if (threadIdx.x == 0) {
-            int bad = 0;
-            if (wire_len < 64) bad = 1;
-            else {
-                const uint32_t* h = reinterpret_cast<const uint32_t*>(wire);
-                const unsigned long long nb = h[2] | ((unsigned long long)h[3] << 32);
-                const unsigned long long pb = h[8] | ((unsigned long long)h[9] << 32);
-                const unsigned long long wl = h[10] | ((unsigned long long)h[11] << 32);
-                if (h[0] != 0x31564D57u || (h[1] & 0xFFFFu) != 1u || (h[1] >> 16) > 1u || nb != g.nbytes ||
-                    h[4] != g.chunk_bytes || h[5] != kTile || h[6] != g.n_chunks || wl != wire_len ||
-                    wire_len < g.meta_end || pb != wire_len - g.meta_end)
-                    bad = 1;
-            }
-            s_format_bad = bad;
-        }
-        __syncthreads();
-        if (s_format_bad) {
-            if (blockIdx.x == 0 && threadIdx.x == 0) {
-                ws.ctrl->gate = (uint32_t)WM_ERR_FORMAT;
-                wm_result r;
-                memset(&r, 0, sizeof r);
-                r.status = WM_ERR_FORMAT;
-                *result = r;
-            }
-            return;
-        }
-    }
-
     const uint64_t pad = (uint64_t)g.n_meta_slices * kTile - g.meta_end;    // multiple of 4
     const uint32_t s = blockIdx.x * 4 + team;
     if (s < g.n_meta_slices) {
@@ -1189,16 +1208,16 @@ k_meta_crc(unsigned char* wire, uint64_t wire_len, Geo g, Ws ws, const Tables* _
             if (vb >= pad) {
                 const uint64_t rb = vb - pad;
                 v = *reinterpret_cast<const uint32_t*>(wire + rb);
-                if (rb == 52) v = 0;
-                if (rb == 0) v ^= 0xFFFFFFFFu;
+                if (rb == 52) v = 0;                      // the meta_crc field reads as zero
+                if (rb == 0) v ^= 0xFFFFFFFFu;            // the CRC's all-ones start value
             }
             w[i] = v;
         }
         const uint32_t v = tile_digest_part(S, w, false, warp, lane);
-        if (lane == 0) tc->wdig[0][warp] = v;
+        if (lane == 0) s_wdig[warp] = v;
     }
     __syncthreads();
-    if (tt == 0 && s < g.n_meta_slices) ws.mdig[s] = xor8(tc->wdig[0]);
+    if (tt == 0 && s < g.n_meta_slices) ws.mdig[s] = xor8(s_wdig);
     __threadfence();
     __syncthreads();
     if (threadIdx.x == 0) {
@@ -1208,47 +1227,18 @@ k_meta_crc(unsigned char* wire, uint64_t wire_len, Geo g, Ws ws, const Tables* _
     __syncthreads();
     if (!s_last) return;
     __threadfence();
-    // fold the slice digests: fetched 1024 at a time by the whole block (one round trip to L2
-    // per batch, not one per digest), folded by one thread out of shared memory
-    uint32_t st = 0;
-    for (uint32_t b0 = 0; b0 < g.n_meta_slices; b0 += 1024) {
-        const uint32_t nb = min(1024u, g.n_meta_slices - b0);
-        __syncthreads();
-        if (threadIdx.x < nb) s_dig[threadIdx.x] = ld_volatile_u32(&ws.mdig[b0 + threadIdx.x]);
-        __syncthreads();
-        if (threadIdx.x == 0)
-            for (uint32_t i = 0; i < nb; i++) st = advance_tile(sHT, st) ^ s_dig[i];
-    }
+    const uint32_t crc = fold_meta_digests(g, ws, sHT, s_dig);
     if (threadIdx.x != 0) return;
-    const uint32_t crc = ~st;
-    if (mode == 0) {
-        reinterpret_cast<uint32_t*>(wire)[13] = crc;
-        wm_result r;
-        memset(&r, 0, sizeof r);
-        const uint32_t err = ld_volatile_u32(&ws.ctrl->err);
-        r.status = (err & 4u) ? WM_ERR_CUDA : (err & 2u) ? WM_ERR_TIMEOUT : (err & 1u) ? WM_ERR_CAPACITY : WM_OK;
-        r.n_present = ws.ctrl->hdr_n_present;
-        r.payload_bytes = ws.ctrl->payload_total;
-        r.wire_len = g.meta_end + ws.ctrl->payload_total;
-        r.cache_crc = ws.ctrl->hdr_cache_crc;
-        *result = r;
-    } else {
-        const uint32_t* h = reinterpret_cast<const uint32_t*>(wire);
-        ws.ctrl->hdr_n_present = h[7];
-        ws.ctrl->hdr_cache_crc = h[12];
-        ws.ctrl->payload_total = h[8] | ((unsigned long long)h[9] << 32);
-        if (crc != h[13]) {
-            ws.ctrl->gate = (uint32_t)WM_ERR_META_CRC;
-            wm_result r;
-            memset(&r, 0, sizeof r);
-            r.status = WM_ERR_META_CRC;
-            r.n_present = h[7];
-            r.payload_bytes = ws.ctrl->payload_total;
-            r.wire_len = wire_len;
-            r.cache_crc = h[12];
-            *result = r;
-        }
-    }
+    reinterpret_cast<uint32_t*>(wire)[13] = crc;
+    wm_result r;
+    memset(&r, 0, sizeof r);
+    const uint32_t err = ld_volatile_u32(&ws.ctrl->err);
+    r.status = (err & 4u) ? WM_ERR_CUDA : (err & 2u) ? WM_ERR_TIMEOUT : (err & 1u) ? WM_ERR_CAPACITY : WM_OK;
+    r.n_present = ws.ctrl->hdr_n_present;
+    r.payload_bytes = ws.ctrl->payload_total;
+    r.wire_len = g.meta_end + ws.ctrl->payload_total;
+    r.cache_crc = ws.ctrl->hdr_cache_crc;
+    *result = r;
 }
 
 // ------------------------------------------------------------------ wm_decode_verify
@@ -1282,64 +1272,96 @@ __device__ __forceinline__ void fill_result(wm_result* result, const Ctrl* ctrl,
     *result = r;
 }
 
-// Step 3.  Per chunk (one warp each): tile entries against the chunk's length and enc_len; also
-// produces each tile's offset inside its chunk's payload.  Across chunks (the last block to
-// finish): payload offsets are the running sum of enc_len and the totals match the header.
-// Sets the gate on failure.
+// Decode steps 1-3 in one kernel.  The first blocks digest the metadata slices (four teams
+// each), the others check the structure chunk by chunk (one warp per chunk: tile entries
+// against the chunk's length and enc_len; also each tile's offset inside its chunk's payload).
+// Neither part follows anything it reads: every index comes from the call's geometry, so the
+// structure pass is safe on damaged metadata and can run beside the CRC.  The last block to
+// finish decides in the specified order: metadata CRC first (WM_ERR_META_CRC), then the
+// structure (WM_ERR_STRUCT: per-chunk findings, payload offsets as the running sum of enc_len,
+// totals against the header).  A header that does not match the call stops every block at
+// once (WM_ERR_FORMAT).  A failure sets the gate that keeps the later kernels out.
 __global__ void __launch_bounds__(1024)
-k_decode_struct(const unsigned char* __restrict__ wire, uint64_t wire_len, Geo g, Ws ws, wm_result* result)
+k_decode_check(const unsigned char* __restrict__ wire, uint64_t wire_len, Geo g, Ws ws,
+               const Tables* __restrict__ tab, wm_result* result, uint32_t meta_blocks)
 {
-    grid_dep_wait();
-    grid_dep_launch();
-    if (ld_volatile_u32(&ws.ctrl->gate)) return;
+    __shared__ uint32_t sG[1024];
+    __shared__ uint32_t sHT[1024];
+    __shared__ uint32_t s_dig[1024];
+    __shared__ uint32_t s_wdig[4][8];
     __shared__ unsigned long long s_warp[32];
     __shared__ unsigned long long s_carry;
     __shared__ uint32_t s_first, s_count;
     __shared__ bool s_last;
-    const uint32_t lane = threadIdx.x % 32, warp = threadIdx.x / 32;
-    const unsigned char* dir = wire + 64;
-    const uint16_t* tab16 = reinterpret_cast<const uint16_t*>(wire + 64 + 16ull * g.n_chunks);
-    const uint32_t c = blockIdx.x * 32u + warp;
-    if (c < g.n_chunks) {
-        const uint64_t clen = chunk_len_dev(g, c);
-        const uint32_t t0 = c * g.tiles_per_chunk;
-        const uint32_t ntc = (uint32_t)((clen + kTile - 1) / kTile);
-        const uint32_t elen = *reinterpret_cast<const uint32_t*>(dir + 16ull * c + 8);
-        unsigned long long carry = 0;
-        bool ok = true, any = false, all = true;
-        for (uint32_t i0 = 0; i0 < ntc; i0 += 32) {
-            const uint32_t i = i0 + lane;
-            uint32_t len = 0;
-            bool l_ok = true, l_any = false, l_all = true;
-            if (i < ntc) {
-                const uint32_t e = tab16[t0 + i];
-                const uint64_t tl = clen - (uint64_t)i * kTile;
-                if (e == 0) l_all = false;
-                else {
-                    l_any = true;
-                    if (tl < kTile) { if (e != 0xFFFFu) l_ok = false; len = (uint32_t)tl; }
-                    else if (e >= 258u && e <= 512u) len = 32u * e;
-                    else l_ok = false;
-                }
-            }
-            uint32_t incl = len;
-#pragma unroll
-            for (int d = 1; d < 32; d <<= 1) {
-                uint32_t o = __shfl_up_sync(0xFFFFFFFFu, incl, d);
-                if (lane >= (uint32_t)d) incl += o;
-            }
-            if (i < ntc) ws.rel[t0 + i] = (uint32_t)(carry + incl - len);
-            carry += __shfl_sync(0xFFFFFFFFu, incl, 31);
-            ok = ok && __all_sync(0xFFFFFFFFu, l_ok);
-            any = any || __any_sync(0xFFFFFFFFu, l_any);
-            all = all && __all_sync(0xFFFFFFFFu, l_all);
+    __shared__ int s_format_bad;
+    const uint32_t lane = threadIdx.x % 32, wblk = threadIdx.x / 32;
+    sHT[threadIdx.x] = (&tab->HT[0][0])[threadIdx.x];
+    load_small_chain_tables(sG, tab);
+    grid_dep_wait();
+    grid_dep_launch();
+    if (threadIdx.x == 0) s_format_bad = header_matches(wire, wire_len, g) ? 0 : 1;
+    __syncthreads();
+    if (s_format_bad) {
+        if (blockIdx.x == 0 && threadIdx.x == 0) {
+            ws.ctrl->gate = (uint32_t)WM_ERR_FORMAT;
+            wm_result r;
+            memset(&r, 0, sizeof r);
+            r.status = WM_ERR_FORMAT;
+            *result = r;
         }
-        if (any && !all) ok = false;
-        if (carry != elen) ok = false;
-        if (lane == 0) {
-            ws.cflag[c] = (any ? CF_PRESENT : 0u) | (ok ? 0u : CF_BAD3);
-            if (!ok) { atomicMin(&ws.ctrl->bad3_first, c); atomicAdd(&ws.ctrl->bad3_count, 1u); }
-            if (any) atomicAdd(&ws.ctrl->n_present, 1u);
+        return;
+    }
+    const unsigned char* dir = wire + 64;
+    if (blockIdx.x < meta_blocks) {
+        const uint32_t team = threadIdx.x / kTeamThreads, tt = threadIdx.x % kTeamThreads;
+        const uint32_t s = blockIdx.x * 4 + team;
+        if (s < g.n_meta_slices) meta_slice_parts(wire, g, s, sG, tab, s_wdig[team], tt / 32, lane);
+        __syncthreads();
+        if (tt == 0 && s < g.n_meta_slices) ws.mdig[s] = xor8(s_wdig[team]);
+    } else {
+        const uint16_t* tab16 = reinterpret_cast<const uint16_t*>(wire + 64 + 16ull * g.n_chunks);
+        const uint32_t c = (blockIdx.x - meta_blocks) * 32u + wblk;
+        if (c < g.n_chunks) {
+            const uint64_t clen = chunk_len_dev(g, c);
+            const uint32_t t0 = c * g.tiles_per_chunk;
+            const uint32_t ntc = (uint32_t)((clen + kTile - 1) / kTile);
+            const uint32_t elen = *reinterpret_cast<const uint32_t*>(dir + 16ull * c + 8);
+            unsigned long long carry = 0;
+            bool ok = true, any = false, all = true;
+            for (uint32_t i0 = 0; i0 < ntc; i0 += 32) {
+                const uint32_t i = i0 + lane;
+                uint32_t len = 0;
+                bool l_ok = true, l_any = false, l_all = true;
+                if (i < ntc) {
+                    const uint32_t e = tab16[t0 + i];
+                    const uint64_t tl = clen - (uint64_t)i * kTile;
+                    if (e == 0) l_all = false;
+                    else {
+                        l_any = true;
+                        if (tl < kTile) { if (e != 0xFFFFu) l_ok = false; len = (uint32_t)tl; }
+                        else if (e >= 258u && e <= 512u) len = 32u * e;
+                        else l_ok = false;
+                    }
+                }
+                uint32_t incl = len;
+#pragma unroll
+                for (int d = 1; d < 32; d <<= 1) {
+                    uint32_t o = __shfl_up_sync(0xFFFFFFFFu, incl, d);
+                    if (lane >= (uint32_t)d) incl += o;
+                }
+                if (i < ntc) ws.rel[t0 + i] = (uint32_t)(carry + incl - len);
+                carry += __shfl_sync(0xFFFFFFFFu, incl, 31);
+                ok = ok && __all_sync(0xFFFFFFFFu, l_ok);
+                any = any || __any_sync(0xFFFFFFFFu, l_any);
+                all = all && __all_sync(0xFFFFFFFFu, l_all);
+            }
+            if (any && !all) ok = false;
+            if (carry != elen) ok = false;
+            if (lane == 0) {
+                ws.cflag[c] = (any ? CF_PRESENT : 0u) | (ok ? 0u : CF_BAD3);
+                if (!ok) { atomicMin(&ws.ctrl->bad3_first, c); atomicAdd(&ws.ctrl->bad3_count, 1u); }
+                if (any) atomicAdd(&ws.ctrl->n_present, 1u);
+            }
         }
     }
     __threadfence();
@@ -1347,11 +1369,37 @@ k_decode_struct(const unsigned char* __restrict__ wire, uint64_t wire_len, Geo g
     if (threadIdx.x == 0) {
         s_carry = 0; s_first = 0xFFFFFFFFu; s_count = 0;
         __threadfence();
-        s_last = atomicAdd(&ws.ctrl->done_c, 1u) == gridDim.x - 1;
+        s_last = atomicAdd(&ws.ctrl->done_b, 1u) == gridDim.x - 1;
     }
     __syncthreads();
     if (!s_last) return;
     __threadfence();
+
+    // ---- the last block: metadata CRC first
+    const uint32_t crc = fold_meta_digests(g, ws, sHT, s_dig);
+    if (threadIdx.x == 0) {
+        const uint32_t* h = reinterpret_cast<const uint32_t*>(wire);
+        ws.ctrl->hdr_n_present = h[7];
+        ws.ctrl->hdr_cache_crc = h[12];
+        ws.ctrl->payload_total = h[8] | ((unsigned long long)h[9] << 32);
+        s_format_bad = 0;
+        if (crc != h[13]) {
+            s_format_bad = 1;
+            ws.ctrl->gate = (uint32_t)WM_ERR_META_CRC;
+            wm_result r;
+            memset(&r, 0, sizeof r);
+            r.status = WM_ERR_META_CRC;
+            r.n_present = h[7];
+            r.payload_bytes = ws.ctrl->payload_total;
+            r.wire_len = wire_len;
+            r.cache_crc = h[12];
+            *result = r;
+        }
+    }
+    __syncthreads();
+    if (s_format_bad) return;
+
+    // ---- then the structure across chunks
     for (uint32_t base = 0; base < g.n_chunks; base += 1024) {
         const uint32_t cc = base + threadIdx.x;
         unsigned long long len = 0, po = 0;
@@ -1365,10 +1413,10 @@ k_decode_struct(const unsigned char* __restrict__ wire, uint64_t wire_len, Geo g
             unsigned long long o = __shfl_up_sync(0xFFFFFFFFu, incl, d);
             if (lane >= (uint32_t)d) incl += o;
         }
-        if (lane == 31) s_warp[warp] = incl;
+        if (lane == 31) s_warp[wblk] = incl;
         __syncthreads();
         unsigned long long before = s_carry;
-        for (uint32_t w2 = 0; w2 < warp; w2++) before += s_warp[w2];
+        for (uint32_t w2 = 0; w2 < wblk; w2++) before += s_warp[w2];
         if (cc < g.n_chunks && po != before + incl - len) {
             // a chunk already counted by the per-chunk pass must not be counted twice
             const uint32_t fl = ld_volatile_u32(&ws.cflag[cc]);
@@ -2038,7 +2086,7 @@ wm_status wm_encode(const void* cache, uint64_t nbytes, uint32_t chunk_bytes, co
     }
     launch_after(k_encode_finish, (g.n_chunks + g.finish_cb - 1) / g.finish_cb, 1024, 0, s, c, g, dirty, crc_inout, w, ws, ds->tables,
                  chunk_powers(g));
-    launch_after(k_meta_crc, (g.n_meta_slices + 3) / 4, 1024, kDynSmem, s, w, (uint64_t)0, g, ws, ds->tables, result, 0);
+    launch_after(k_meta_crc, (g.n_meta_slices + 3) / 4, 1024, kDynSmem, s, w, g, ws, ds->tables, result);
     g_launches = 4;
     return launch_status();
 }
@@ -2059,9 +2107,8 @@ wm_status wm_decode_verify(const void* wire, uint64_t wire_len, void* dst, uint6
     unsigned char* d = static_cast<unsigned char*>(dst);
     k_decode_init<<<1, 64, 0, s>>>(ws);
     // a wire shorter than the metadata is rejected by the header check before anything else is read
-    const uint32_t slices = wire_len >= g.meta_end ? g.n_meta_slices : 1;
-    launch_after(k_meta_crc, (slices + 3) / 4, 1024, kDynSmem, s, const_cast<unsigned char*>(w), wire_len, g, ws, ds->tables, result, 1);
-    launch_after(k_decode_struct, (g.n_chunks + 31) / 32, 1024, 0, s, w, wire_len, g, ws, result);
+    const uint32_t meta_blocks = (g.n_meta_slices + 3) / 4;
+    launch_after(k_decode_check, meta_blocks + (g.n_chunks + 31) / 32, 1024, 0, s, w, wire_len, g, ws, ds->tables, result, meta_blocks);
     const uint32_t need = (g.n_tiles + kTeamsPlain - 1) / kTeamsPlain;
     const uint32_t grid = need < (uint32_t)ds->sm_count ? need : (uint32_t)ds->sm_count;
     {
@@ -2070,7 +2117,7 @@ wm_status wm_decode_verify(const void* wire, uint64_t wire_len, void* dst, uint6
     }
     launch_after(k_decode_finish, (g.n_chunks + g.finish_cb - 1) / g.finish_cb, 1024, 0, s, w, wire_len, g, d, dst_crc_inout, ws, ds->tables,
                  result, chunk_powers(g));
-    g_launches = 5;
+    g_launches = 4;
     return launch_status();
 }
 
