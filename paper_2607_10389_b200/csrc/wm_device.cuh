@@ -219,25 +219,9 @@ __device__ __forceinline__ uint32_t advance_tile(const uint32_t* HT, uint32_t s)
     return HT[s & 0xFF] ^ HT[256 + ((s >> 8) & 0xFF)] ^ HT[512 + ((s >> 16) & 0xFF)] ^ HT[768 + (s >> 24)];
 }
 
-__device__ __forceinline__ uint32_t ld_stream_u32(const void* p)
-{
-    uint32_t v;
-    asm volatile("ld.global.cs.u32 %0, [%1];" : "=r"(v) : "l"(p));
-    return v;
-}
 __device__ __forceinline__ void st_stream_u32(void* p, uint32_t v)
 {
     asm volatile("st.global.cs.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
-}
-__device__ __forceinline__ uint64_t ld_volatile_u64(const uint64_t* p)
-{
-    uint64_t v;
-    asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
-    return v;
-}
-__device__ __forceinline__ void st_volatile_u64(uint64_t* p, uint64_t v)
-{
-    asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
 }
 __device__ __forceinline__ uint32_t ld_volatile_u32(const uint32_t* p)
 {
@@ -257,29 +241,6 @@ __device__ __forceinline__ uint32_t max_u16x2(uint32_t a, uint32_t b)
     uint32_t d;
     asm("max.u16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
     return d;
-}
-
-// L2 residency hint: data that is read again soon is loaded with evict-last priority (the
-// plain streaming load marks its lines evict-first, and a line so marked is gone from L2 a few
-// microseconds later).
-__device__ __forceinline__ uint64_t l2_policy_evict_last()
-{
-    uint64_t pol;
-    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(pol));
-    return pol;
-}
-__device__ __forceinline__ uint32_t ld_keep_u32(const void* p, uint64_t pol)
-{
-    uint32_t v;
-    asm volatile("ld.global.L1::no_allocate.L2::cache_hint.u32 %0, [%1], %2;" : "=r"(v) : "l"(p), "l"(pol));
-    return v;
-}
-__device__ __forceinline__ void load_tile_words_keep(const unsigned char* tile, uint32_t warp, uint32_t lane,
-                                                     uint32_t (&w)[16], uint64_t pol)
-{
-    const unsigned char* p = tile + warp * 2048u + lane * 4u;
-#pragma unroll
-    for (int i = 0; i < 16; i++) w[i] = ld_keep_u32(p + i * 128, pol);
 }
 
 // ---- bulk (TMA) copies of whole tiles into shared memory, tracked by an mbarrier ----
@@ -377,15 +338,6 @@ __device__ __forceinline__ void read_staged_words(const unsigned char* stage, ui
     const uint32_t* p = reinterpret_cast<const uint32_t*>(stage) + warp * 512u + lane;
 #pragma unroll
     for (int i = 0; i < 16; i++) w[i] = p[i * 32];
-}
-
-// Full tile, fast path: lane's word of row 16*warp + i.
-__device__ __forceinline__ void load_tile_words(const unsigned char* tile, uint32_t warp, uint32_t lane,
-                                                uint32_t (&w)[kWordsPerLane])
-{
-    const unsigned char* p = tile + warp * 2048u + lane * 4u;
-#pragma unroll
-    for (int i = 0; i < 16; i++) w[i] = ld_stream_u32(p + i * 128);
 }
 
 // One 32-bit word of a tile of `len` (1..16384) real bytes that is right-aligned in a virtual

@@ -67,8 +67,7 @@ struct Ctrl {                 // first 256 bytes of the workspace
     unsigned long long payload_total;
     uint32_t hdr_n_present, hdr_cache_crc;
     uint32_t cache_acc;       // XOR of the chunks' terms of the whole-cache CRC
-    uint32_t done_c;
-    uint32_t pad[40];
+    uint32_t pad[41];
 };
 static_assert(sizeof(Ctrl) == 256, "control block is 256 bytes");
 
@@ -193,15 +192,6 @@ __device__ __forceinline__ uint64_t chunk_len_dev(const Geo& g, uint32_t c)
 {
     return (c + 1 == g.n_chunks) ? g.last_chunk_len : g.chunk_bytes;
 }
-
-// ------------------------------------------------------------------ per-team shared state
-
-struct TeamCtl {
-    uint32_t wdig[2][8];   // per warp: its contribution to the tile digest (double buffered)
-    uint32_t next;
-    uint32_t pad[3];
-};
-static_assert(sizeof(TeamCtl) % 16 == 0, "team control block keeps 16-byte alignment");
 
 // A warp's contribution to the digest of the team's tile, from the 16 words each lane holds
 // (same value in every lane).  `init_fold`: complement the tile's first word, which folds the
@@ -675,7 +665,6 @@ struct EncTeamCtl {
     unsigned long long pad2;
 };
 static_assert(sizeof(EncTeamCtl) % 16 == 0, "team control block keeps 16-byte alignment");
-constexpr uint32_t kTeamSmemEncode = kTile + sizeof(EncTeamCtl);   // one 16 KiB stage + control
 
 __device__ __forceinline__ uint32_t tile_left(const Geo& g, uint32_t t)      // bytes of a ragged tile
 {
