@@ -168,6 +168,37 @@ wm_status wm_decode_verify(const void* wire, uint64_t wire_len, void* dst, uint6
                            void* workspace, uint64_t workspace_bytes, wm_result* result, void* stream);
 
 /*
+ * Leaf mode - the cache as the engine holds it: a list of tensors, not one buffer.
+ * Paper: the mover flattens the live cache before the transfer and rehydrates it after
+ * (Section 1 and Section 4.1: flatten, transfer, CRC-verify, rehydrate; Section 5: the movable
+ * set is 420 tensors, 450 leaves with the control flags).  These two calls read the leaves
+ * where they are and write the decoded bytes where they belong, which removes the flatten copy
+ * before wm_encode and the rehydrate copy after wm_decode_verify (each a read and a write of
+ * the whole cache).  The logical cache is the concatenation of the leaves in table order;
+ * chunks, tiles and the wire image are exactly those of that concatenation, so the image is
+ * byte for byte what wm_encode produces from the flattened buffer, and either decode call
+ * accepts it.
+ *   leaves    [dev] n_leaves entries (1..4096), read on the stream.  Every ptr is 16-byte
+ *             aligned device memory; every nbytes is positive and, for all leaves but the
+ *             last, a multiple of 16384; the sizes add up to nbytes.  A table that breaks
+ *             these rules gives result->status WM_ERR_ARG and nothing is read or written
+ *             through it.
+ * Everything else is as in wm_encode / wm_decode_verify.
+ */
+typedef struct {
+    const void* ptr;     /* [dev] first byte of the leaf */
+    uint64_t    nbytes;
+} wm_leaf;
+
+wm_status wm_encode_leaves(const wm_leaf* leaves, uint32_t n_leaves, uint64_t nbytes, uint32_t chunk_bytes,
+                           const uint8_t* dirty, uint32_t* crc_inout, void* wire, uint64_t wire_cap,
+                           void* workspace, uint64_t workspace_bytes, wm_result* result, void* stream);
+
+wm_status wm_decode_verify_leaves(const void* wire, uint64_t wire_len, const wm_leaf* dst_leaves, uint32_t n_leaves,
+                                  uint64_t nbytes, uint32_t chunk_bytes, uint32_t* dst_crc_inout,
+                                  void* workspace, uint64_t workspace_bytes, wm_result* result, void* stream);
+
+/*
  * wm_checksum_noalloc - wm_checksum for callers that cannot allocate device memory.
  * The paper has no counterpart to this call; it exists for hosts that may not call cudaMalloc
  * at the point where they need a checksum: code running inside a stream capture or under an

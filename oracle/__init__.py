@@ -13,8 +13,11 @@ from .wm_oracle import (  # noqa: F401
     crc_bitwise,
     crc_combine,
     decode_verify,
+    decode_verify_leaves,
     dirty_diff,
     encode,
+    encode_leaves,
+    flatten_leaves,
     meta_end,
     num_chunks,
     num_tiles,

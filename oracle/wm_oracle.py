@@ -191,3 +191,27 @@ def decode_verify(wire, nbytes: int, chunk_bytes: int, dst=None, dst_crc=None, w
                                    nbytes, chunk_bytes, _ptr(crc), ctypes.byref(res))
     _check(st, "decode_verify")
     return out, crc, _result(res)
+
+
+def flatten_leaves(leaves) -> np.ndarray:
+    """The logical cache of the leaf-mode calls: the leaves' bytes one after the other."""
+    return np.concatenate([_bytes_view(x) for x in leaves]) if len(leaves) else np.zeros(0, dtype=np.uint8)
+
+
+def encode_leaves(leaves, chunk_bytes: int, dirty=None, crc_in=None, wire_cap: int | None = None):
+    """Leaf mode is defined by the flat calls: the image of a list of leaves is the image of their
+    concatenation.  Returns what encode() returns."""
+    return encode(flatten_leaves(leaves), chunk_bytes, dirty=dirty, crc_in=crc_in, wire_cap=wire_cap)
+
+
+def decode_verify_leaves(wire, leaves, chunk_bytes: int, dst_crc=None, wire_len: int | None = None):
+    """Decode into a list of leaves (arrays whose sizes give the split).  Returns (new leaves,
+    crc vector, Result); on failure the leaves come back as the flat decoder left its buffer."""
+    sizes = [_bytes_view(x).size for x in leaves]
+    flat = flatten_leaves(leaves)
+    out, crc, res = decode_verify(wire, flat.size, chunk_bytes, dst=flat, dst_crc=dst_crc, wire_len=wire_len)
+    parts, o = [], 0
+    for n in sizes:
+        parts.append(out[o:o + n].copy())
+        o += n
+    return parts, crc, res

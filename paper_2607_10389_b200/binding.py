@@ -23,7 +23,8 @@ STATUS = {
 RESULT_BYTES = 40
 EXPORTS = ("wm_num_chunks", "wm_num_tiles", "wm_meta_bytes", "wm_wire_bound", "wm_workspace_bytes",
            "wm_checksum", "wm_dirty_diff", "wm_encode", "wm_decode_verify", "wm_last_launch_count",
-           "wm_timing_enable", "wm_timing_read_ms", "wm_checksum_noalloc")
+           "wm_timing_enable", "wm_timing_read_ms", "wm_checksum_noalloc", "wm_encode_leaves",
+           "wm_decode_verify_leaves")
 
 
 class WmError(RuntimeError):
@@ -59,6 +60,10 @@ def load_library() -> ctypes.CDLL:
     lib.wm_encode.argtypes = [vp, u64, u32, vp, vp, vp, u64, vp, u64, vp, vp]
     lib.wm_decode_verify.restype = ctypes.c_int
     lib.wm_decode_verify.argtypes = [vp, u64, vp, u64, u32, vp, vp, u64, vp, vp]
+    lib.wm_encode_leaves.restype = ctypes.c_int
+    lib.wm_encode_leaves.argtypes = [vp, u32, u64, u32, vp, vp, vp, u64, vp, u64, vp, vp]
+    lib.wm_decode_verify_leaves.restype = ctypes.c_int
+    lib.wm_decode_verify_leaves.argtypes = [vp, u64, vp, u32, u64, u32, vp, vp, u64, vp, vp]
     return lib
 
 
@@ -220,3 +225,36 @@ def wm_decode_verify(wire: torch.Tensor, wire_len: int, dst: torch.Tensor, chunk
     _check(lib().wm_decode_verify(wire.data_ptr(), int(wire_len), dst.data_ptr(), nbytes, chunk_bytes,
                                   dst_crc_inout.data_ptr(), workspace.data_ptr(), workspace.numel(),
                                   result.data_ptr(), _stream(stream)), "wm_decode_verify")
+
+
+def make_leaf_table(tensors, device="cuda") -> torch.Tensor:
+    """Device table of (ptr, nbytes) pairs, one per tensor, in the order given: the `wm_leaf`
+    array of the leaf-mode calls.  The tensors must stay alive while the table is in use."""
+    rows = []
+    for t in tensors:
+        if not t.is_cuda or not t.is_contiguous():
+            raise WmError("leaves must be contiguous CUDA tensors")
+        rows.append((t.data_ptr(), t.numel() * t.element_size()))
+    table = torch.tensor(rows, dtype=torch.int64).reshape(-1, 2)
+    return table.to(device)
+
+
+def wm_encode_leaves(leaf_table: torch.Tensor, nbytes: int, chunk_bytes: int, dirty, crc_inout: torch.Tensor,
+                     wire: torch.Tensor, workspace: torch.Tensor, result: torch.Tensor, stream=None,
+                     wire_cap=None) -> None:
+    _dev_u8(wire, "wire")
+    cap = wire.numel() if wire_cap is None else int(wire_cap)
+    _check(lib().wm_encode_leaves(leaf_table.data_ptr(), leaf_table.shape[0], int(nbytes), chunk_bytes,
+                                  None if dirty is None else dirty.data_ptr(), crc_inout.data_ptr(), wire.data_ptr(),
+                                  cap, workspace.data_ptr(), workspace.numel(), result.data_ptr(), _stream(stream)),
+           "wm_encode_leaves")
+
+
+def wm_decode_verify_leaves(wire: torch.Tensor, wire_len: int, leaf_table: torch.Tensor, nbytes: int,
+                            chunk_bytes: int, dst_crc_inout: torch.Tensor, workspace: torch.Tensor,
+                            result: torch.Tensor, stream=None) -> None:
+    _dev_u8(wire, "wire")
+    _check(lib().wm_decode_verify_leaves(wire.data_ptr(), int(wire_len), leaf_table.data_ptr(), leaf_table.shape[0],
+                                         int(nbytes), chunk_bytes, dst_crc_inout.data_ptr(), workspace.data_ptr(),
+                                         workspace.numel(), result.data_ptr(), _stream(stream)),
+           "wm_decode_verify_leaves")

@@ -79,6 +79,7 @@ struct Ws {
     uint32_t* cflag;             // [n_chunks] bit0 present, bit1..: failed step 3/4/5/6
     uint32_t* ccrc;              // [n_chunks]
     uint32_t* mdig;              // [n_meta_slices]
+    unsigned char** tptr;        // [n_tiles] leaf mode: where each tile of the logical cache lives
 };
 
 constexpr uint32_t CF_PRESENT = 1, CF_BAD3 = 2, CF_BAD4 = 4, CF_BAD5 = 8, CF_BAD6 = 16;
@@ -86,7 +87,7 @@ constexpr uint32_t CF_PRESENT = 1, CF_BAD3 = 2, CF_BAD4 = 4, CF_BAD5 = 8, CF_BAD
 static inline uint64_t align16(uint64_t v) { return (v + 15) & ~(uint64_t)15; }
 
 struct WsLayout {
-    uint64_t state, dig, rel, cflag, ccrc, mdig, total;
+    uint64_t state, dig, rel, cflag, ccrc, mdig, tptr, total;
 };
 
 static WsLayout ws_layout(const Geo& g)
@@ -99,6 +100,7 @@ static WsLayout ws_layout(const Geo& g)
     L.cflag = o; o = align16(o + 4ull * g.n_chunks);
     L.ccrc = o;  o = align16(o + 4ull * g.n_chunks);
     L.mdig = o;  o = align16(o + 4ull * g.n_meta_slices);
+    L.tptr = o;  o = align16(o + 8ull * g.n_tiles);
     L.total = o;
     return L;
 }
@@ -115,6 +117,7 @@ static Ws ws_carve(void* base, const Geo& g)
     w.cflag = reinterpret_cast<uint32_t*>(b + L.cflag);
     w.ccrc = reinterpret_cast<uint32_t*>(b + L.ccrc);
     w.mdig = reinterpret_cast<uint32_t*>(b + L.mdig);
+    w.tptr = reinterpret_cast<unsigned char**>(b + L.tptr);
     return w;
 }
 
@@ -211,13 +214,22 @@ __device__ __forceinline__ uint32_t xor8(const uint32_t* p)
     return p[0] ^ p[1] ^ p[2] ^ p[3] ^ p[4] ^ p[5] ^ p[6] ^ p[7];
 }
 
+// First byte of chunk c: in the flat buffer, or (leaf mode, flat == nullptr) where the chunk's
+// first tile lives.  Only chunks shorter than four bytes are ever read through it.
+__device__ __forceinline__ const unsigned char* chunk_first_byte(const Geo& g, const Ws& ws, const unsigned char* flat, uint32_t c)
+{
+    if (flat) return flat + (uint64_t)c * g.chunk_bytes;
+    return chunk_len_dev(g, c) < 4 ? ws.tptr[(uint64_t)c * g.tiles_per_chunk] : nullptr;
+}
+
 // CRC32C of chunk c from its tiles' digests (Horner over tiles; the all-ones init was folded
-// into the first tile's digest, the final complement is applied here).
+// into the first tile's digest, the final complement is applied here).  `bytes`: the chunk's
+// first byte (read only when the chunk is shorter than four bytes).
 __device__ uint32_t chunk_crc_from_digests(const Geo& g, const uint32_t* HT, const uint32_t* T0,
                                            const uint32_t* dig, const unsigned char* bytes, uint32_t c)
 {
     const uint64_t clen = chunk_len_dev(g, c);
-    if (clen < 4) return crc_bytewise(T0, bytes + (uint64_t)c * g.chunk_bytes, (uint32_t)clen);
+    if (clen < 4) return crc_bytewise(T0, bytes, (uint32_t)clen);
     const uint32_t t0 = c * g.tiles_per_chunk;
     const uint32_t ntc = (uint32_t)((clen + kTile - 1) / kTile);
     const bool ragged = (clen % kTile) != 0;
@@ -282,7 +294,7 @@ __device__ uint32_t chunk_crc_staged(const Geo& g, const uint32_t* HT, const uin
 {
     if (g.tiles_per_chunk > kFinishDigests) return chunk_crc_from_digests(g, HT, T0, dig, bytes, c);
     const uint64_t clen = chunk_len_dev(g, c);
-    if (clen < 4) return crc_bytewise(T0, bytes + (uint64_t)c * g.chunk_bytes, (uint32_t)clen);
+    if (clen < 4) return crc_bytewise(T0, bytes, (uint32_t)clen);
     const uint32_t ntc = (uint32_t)((clen + kTile - 1) / kTile);
     const bool ragged = (clen % kTile) != 0;
     const uint32_t* d = st.dig + (size_t)i * (g.tiles_per_chunk + 1u);
@@ -397,7 +409,7 @@ k_checksum_finish(const unsigned char* __restrict__ cache, Geo g, Ws ws, const T
     stage_chunk_digests(g, stage, ws.dig, c0);
     const uint32_t c = c0 + threadIdx.x;
     if (threadIdx.x < g.finish_cb && c < g.n_chunks)
-        crc_out[c] = chunk_crc_staged(g, sHT, sT0, stage, ws.dig, cache, c, threadIdx.x);
+        crc_out[c] = chunk_crc_staged(g, sHT, sT0, stage, ws.dig, cache + (uint64_t)c * g.chunk_bytes, c, threadIdx.x);
 }
 
 // ------------------------------------------------------------------ wm_dirty_diff
@@ -485,6 +497,98 @@ k_diff_compact(Geo g, const uint8_t* __restrict__ dirty, uint32_t* __restrict__ 
         __syncthreads();
     }
     if (threadIdx.x == 0) *n_out = s_carry;
+}
+
+// ------------------------------------------------------------------ leaf tables
+
+// Leaf mode: the logical cache is the concatenation of `n` leaves (tensors).  Every leaf but
+// the last is a whole number of tiles, so a tile never straddles two leaves and all that the
+// main kernels need is where each tile lives: tptr[t].  Every block recomputes the leaves'
+// first tiles in shared memory (at most 4096 leaves), then the blocks share the tiles.
+// A table that breaks the rules (a leaf that is empty, misaligned or not a whole number of
+// tiles before the last, or sizes that do not add up to nbytes) raises error bit 8; in decode
+// mode it also closes the gate and writes the result record.
+constexpr uint32_t kMaxLeaves = 4096;
+__global__ void __launch_bounds__(1024)
+k_leaf_map(const wm_leaf* __restrict__ leaves, uint32_t n, Geo g, Ws ws, wm_result* result, int decode)
+{
+    __shared__ uint32_t s_start[kMaxLeaves + 1];       // first tile of each leaf; [n] = total tiles
+    __shared__ uint32_t s_wsum[32];
+    __shared__ uint32_t s_bad;
+    const uint32_t lane = threadIdx.x % 32, warp = threadIdx.x / 32;
+    grid_dep_wait();
+    grid_dep_launch();
+    if (threadIdx.x == 0) s_bad = 0;
+    __syncthreads();
+    // thread i owns leaves 4i .. 4i+3
+    uint32_t cnt[4], bad = 0;
+    unsigned long long bytes = 0;
+#pragma unroll
+    for (int k = 0; k < 4; k++) {
+        const uint32_t i = 4 * threadIdx.x + k;
+        cnt[k] = 0;
+        if (i < n) {
+            const unsigned long long nb = leaves[i].nbytes;
+            const unsigned long long p = reinterpret_cast<unsigned long long>(leaves[i].ptr);
+            if (nb == 0 || (p & 15ull) != 0 || (i + 1 < n && nb % kTile != 0)) bad = 1;
+            bytes += nb;
+            cnt[k] = (uint32_t)((nb + kTile - 1) / kTile);
+        }
+    }
+    const uint32_t mine = cnt[0] + cnt[1] + cnt[2] + cnt[3];
+    uint32_t incl = mine;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        const uint32_t o = __shfl_up_sync(0xFFFFFFFFu, incl, d);
+        if (lane >= (uint32_t)d) incl += o;
+    }
+    if (lane == 31) s_wsum[warp] = incl;
+    // total bytes: the sum is exact modulo 2^64, which is all the comparison below needs
+    unsigned long long tot = bytes;
+#pragma unroll
+    for (int d = 16; d >= 1; d >>= 1) tot += __shfl_xor_sync(0xFFFFFFFFu, tot, d);
+    __shared__ unsigned long long s_bytes[32];
+    if (lane == 0) s_bytes[warp] = tot;
+    if (bad) s_bad = 1;
+    __syncthreads();
+    uint32_t before = 0;
+    for (uint32_t w2 = 0; w2 < warp; w2++) before += s_wsum[w2];
+    uint32_t run = before + incl - mine;
+#pragma unroll
+    for (int k = 0; k < 4; k++) {
+        const uint32_t i = 4 * threadIdx.x + k;
+        if (i < n) s_start[i] = run;
+        run += cnt[k];
+    }
+    if (threadIdx.x == 0) {
+        unsigned long long all = 0;
+        for (int w2 = 0; w2 < 32; w2++) all += s_bytes[w2];
+        if (all != g.nbytes) s_bad = 1;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) s_start[n] = g.n_tiles;
+    __syncthreads();
+    if (s_bad) {
+        if (blockIdx.x == 0 && threadIdx.x == 0) {
+            atomicOr(&ws.ctrl->err, 8u);
+            if (decode) {
+                ws.ctrl->gate = (uint32_t)WM_ERR_ARG;
+                wm_result r;
+                memset(&r, 0, sizeof r);
+                r.status = WM_ERR_ARG;
+                *result = r;
+            }
+        }
+        return;
+    }
+    for (uint32_t t = blockIdx.x * blockDim.x + threadIdx.x; t < g.n_tiles; t += gridDim.x * blockDim.x) {
+        uint32_t lo = 0, hi = n;                       // the leaf with start[lo] <= t < start[lo + 1]
+        while (hi - lo > 1) {
+            const uint32_t mid = (lo + hi) / 2;
+            if (s_start[mid] <= t) lo = mid; else hi = mid;
+        }
+        ws.tptr[t] = const_cast<unsigned char*>(static_cast<const unsigned char*>(leaves[lo].ptr)) + (uint64_t)(t - s_start[lo]) * kTile;
+    }
 }
 
 // ------------------------------------------------------------------ wm_encode
@@ -663,6 +767,7 @@ struct EncTeamCtl {
     unsigned long long excl[2];   // offset of the tile packed in the next step, by step parity
     unsigned long long mbar;      // completion of the bulk copy into the team's stage
     unsigned long long pad2;
+    const unsigned char* nptr[2]; // leaf mode: where the tile in next[] lives, by step parity
 };
 static_assert(sizeof(EncTeamCtl) % 16 == 0, "team control block keeps 16-byte alignment");
 
@@ -759,7 +864,7 @@ __device__ __forceinline__ uint32_t describe_tile(const Geo& g, const uint8_t* _
     return q;
 }
 
-template <int TEAMS, bool MASKED>
+template <int TEAMS, bool MASKED, bool LEAVES>
 __global__ void __launch_bounds__(TEAMS * 256, 1)
 k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restrict__ dirty,
          unsigned char* __restrict__ wire, uint64_t wire_cap, Ws ws, const Tables* __restrict__ tab)
@@ -772,6 +877,7 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
     Smem S = setup_smem(smem, tab);
     grid_dep_wait();                   // from here on the control block and the length table are ready
     grid_dep_launch();
+    if (LEAVES && (ld_volatile_u32(&ws.ctrl->err) & 8u)) return;      // the leaf table was rejected
     if (threadIdx.x == 0) s_scanner = atomicCAS(&ws.ctrl->scan_lock, 0u, 1u) == 0u;
     __syncthreads();
     if (s_scanner) {
@@ -813,8 +919,12 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
     auto is_tile = [](uint32_t q) { return (q & kQTile) != kQNone; };
     auto is_hot = [&](uint32_t q) { return q >= kQPresent && (q & kQTile) < g.n_full_tiles; };   // present and full
     auto publish_len = [&](uint32_t t, uint32_t len) { st_relaxed_u32(ws.lbk + t, kFlagA | (len / kUnit)); };
-    auto start_copy = [&](uint32_t q) {          // thread 0 of the team, after the barrier that frees the stage
-        if (is_hot(q)) bulk_load(stage, cache + (uint64_t)(q & kQTile) * kTile, kTile, &tc->mbar, pol_once);
+    // where tile t lives: the flat cache, or (leaf mode) the table that k_leaf_map filled
+    auto tile_src = [&](uint32_t t) -> const unsigned char* {
+        return LEAVES ? ws.tptr[t] : cache + (uint64_t)t * kTile;
+    };
+    auto start_copy = [&](uint32_t q, const unsigned char* src) {   // thread 0 of the team, after the barrier that frees the stage
+        if (is_hot(q)) bulk_load(stage, src, kTile, &tc->mbar, pol_once);
     };
 
     // Tiles in flight, oldest first: X (packed in this step), V, W (waiting for their offsets),
@@ -828,7 +938,10 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
     uint32_t d[kWordsPerLane];
     bool claiming = false;             // leader: the last ticket it claimed was a tile
 
-    // ---- prologue: the tiles of the first two steps are claimed, the first one's copy started
+    // ---- prologue: the tiles of the first two steps are claimed, the first one's copy started.
+    // Leaf mode claims one step further ahead: a tile's address is looked up in the step between
+    // its claim and its hand-over, so that the leader never waits for that answer either.
+    uint32_t qA = kQNone;              // leader, leaf mode: claimed and described, address on its way
     if (leader) {
         for (int i = 0; i < 8; i++) tc->wsum[i] = 0;
         mbar_init(&tc->mbar, 1);
@@ -839,10 +952,15 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
         tc->next[1] = q1;
         tc->excl[0] = 0ull;
         tc->excl[1] = 0ull;
+        if (LEAVES) {
+            tc->nptr[0] = is_tile(q0) ? tile_src(q0 & kQTile) : nullptr;
+            tc->nptr[1] = is_tile(q1) ? tile_src(q1 & kQTile) : nullptr;
+            if (claiming) { qA = describe_tile<MASKED>(g, dirty, next_ticket(ws.ctrl)); claiming = is_tile(qA); }
+        }
     }
     team_bar(team);
     qY = tc->next[0];
-    if (leader) start_copy(qY);
+    if (leader) start_copy(qY, LEAVES ? tc->nptr[0] : tile_src(qY & kQTile));
 
     uint32_t trouble = 0;              // sticky: 1 the image does not fit, 2 a copy never arrived
     while (((qX & qV & qW & qY) & kQTile) != kQNone) {
@@ -860,10 +978,12 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
         // round trips to L2 whose answers are used at the end of the step: the ticket of the
         // tile to measure two steps on, and the offset of the tile to pack in the next step.
         uint32_t pv = 0, tk = 0xFFFFFFFFu;
+        const unsigned char* pA = nullptr;
         if (leader) {
-            start_copy(qN);
+            start_copy(qN, LEAVES ? tc->nptr[par ^ 1u] : tile_src(qN & kQTile));
             if (is_tile(qV)) pv = ld_relaxed_u32(ws.lbk + (qV & kQTile));
             if (claiming) tk = next_ticket(ws.ctrl);
+            if (LEAVES && is_tile(qA)) pA = tile_src(qA & kQTile);
         }
 
         // ---- Y: digest, exponent ranges, length out, words parked
@@ -930,7 +1050,7 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
             const bool present = qY >= kQPresent;
             if (tt == 0) publish_len(tYn, present ? tile_left(g, tYn) : 0u);
             if (present) {
-                load_tile_words_guarded(cache + (uint64_t)tYn * kTile, tile_left(g, tYn), (qY & kQFirst) != 0, warp, lane, d);
+                load_tile_words_guarded(tile_src(tYn), tile_left(g, tYn), (qY & kQFirst) != 0, warp, lane, d);
                 const uint32_t v = tile_digest_part(S, d, false, warp, lane);
                 if (lane == 0) tc->wdig[slY][warp] = v;
             }
@@ -995,7 +1115,7 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
             if (exclX + enc_len > room) {
                 trouble |= 1u;
             } else {
-                const unsigned char* src = cache + (uint64_t)tXn * kTile;
+                const unsigned char* src = tile_src(tXn);
                 unsigned char* dst = payload + exclX;
                 for (uint32_t i = tt; i < enc_len; i += kTeamThreads) dst[i] = src[i];
             }
@@ -1029,7 +1149,13 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
             uint32_t qn2 = kQNone;
             if (claiming) { qn2 = describe_tile<MASKED>(g, dirty, tk); claiming = is_tile(qn2); }
             tc->excl[par] = e;
-            tc->next[par] = qn2;
+            if (LEAVES) {              // hand over the tile whose address arrived during this step
+                tc->next[par] = qA;
+                tc->nptr[par] = pA;
+                qA = qn2;
+            } else {
+                tc->next[par] = qn2;
+            }
         }
         qX = qV; qV = qW; qW = qY; qY = qN;
         sl = (sl + 1u) & 7u;
@@ -1069,11 +1195,12 @@ k_encode_finish(const unsigned char* __restrict__ cache, Geo g, const uint8_t* _
     // on one SM's shared memory)
     const uint32_t c = c0 + threadIdx.x;
     uint32_t present = 0, term = 0;
-    if (threadIdx.x < g.finish_cb && c < g.n_chunks) {
+    const bool dead = (ld_volatile_u32(&ws.ctrl->err) & 8u) != 0;      // leaf mode: the table was rejected
+    if (!dead && threadIdx.x < g.finish_cb && c < g.n_chunks) {
         present = (!dirty || dirty[c]) ? 1u : 0u;
         uint32_t crc;
         if (present) {
-            crc = chunk_crc_staged(g, sHT, sT0, stage, ws.dig, cache, c, threadIdx.x);
+            crc = chunk_crc_staged(g, sHT, sT0, stage, ws.dig, chunk_first_byte(g, ws, cache, c), c, threadIdx.x);
             crc_inout[c] = crc;
         } else {
             crc = crc_inout[c];
@@ -1222,7 +1349,7 @@ k_meta_crc(unsigned char* wire, Geo g, Ws ws, const Tables* __restrict__ tab, wm
     wm_result r;
     memset(&r, 0, sizeof r);
     const uint32_t err = ld_volatile_u32(&ws.ctrl->err);
-    r.status = (err & 4u) ? WM_ERR_CUDA : (err & 2u) ? WM_ERR_TIMEOUT : (err & 1u) ? WM_ERR_CAPACITY : WM_OK;
+    r.status = (err & 8u) ? WM_ERR_ARG : (err & 4u) ? WM_ERR_CUDA : (err & 2u) ? WM_ERR_TIMEOUT : (err & 1u) ? WM_ERR_CAPACITY : WM_OK;
     r.n_present = ws.ctrl->hdr_n_present;
     r.payload_bytes = ws.ctrl->payload_total;
     r.wire_len = g.meta_end + ws.ctrl->payload_total;
@@ -1288,6 +1415,7 @@ k_decode_check(const unsigned char* __restrict__ wire, uint64_t wire_len, Geo g,
     load_small_chain_tables(sG, tab);
     grid_dep_wait();
     grid_dep_launch();
+    if (ld_volatile_u32(&ws.ctrl->gate)) return;        // leaf mode: the destination table was rejected
     if (threadIdx.x == 0) s_format_bad = header_matches(wire, wire_len, g) ? 0 : 1;
     __syncthreads();
     if (s_format_bad) {
@@ -1515,7 +1643,7 @@ __device__ __forceinline__ void unpack_group_planes(const PlaneWords& pw, uint32
 // The team's first thread prepares tiles ahead of their turn, one dependent step per tile so
 // that it never sits waiting for an answer from L2: claim a ticket (three tiles ahead), look
 // up that tile's table entry and offsets (two ahead), start its copy (one ahead).
-template <int TEAMS>
+template <int TEAMS, bool LEAVES>
 __global__ void __launch_bounds__(TEAMS * 256, 1)
 k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restrict__ dst, Ws ws,
          const Tables* __restrict__ tab)
@@ -1581,6 +1709,8 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
         }
         const uint32_t ew = tc->slot[it & 3u].entry;
         const uint32_t e = ew & 0xFFFFu;
+        // leaf mode: where this tile goes (asked for now, needed when the stores begin)
+        unsigned char* const o_leaf = LEAVES ? ws.tptr[t] : nullptr;
         const uint32_t p = it & 1u;
         const bool is_pack = e >= 258u && e < 512u;
         bool decoded = true;
@@ -1657,7 +1787,7 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
         // ---- phase 2: unpack, store, checksum
         bool have_digest = false;
         if (e != 0) {
-            unsigned char* o = dst + (uint64_t)t * kTile;
+            unsigned char* o = LEAVES ? o_leaf : dst + (uint64_t)t * kTile;
             bool fold = (ew >> 16) != 0;
             if (e == 0xFFFFu) {
                 const unsigned char* src = payload + tc->slot[it & 3u].src;
@@ -1764,7 +1894,7 @@ k_decode_finish(const unsigned char* __restrict__ wire, uint64_t wire_len, Geo g
         if (step4_failed) {
             if (fl & CF_BAD4) { atomicMin(&ws.ctrl->bad4_first, c); atomicAdd(&ws.ctrl->bad4_count, 1u); }
         } else if (fl & CF_PRESENT) {
-            const uint32_t got = chunk_crc_staged(g, sHT, sT0, stage, ws.dig, dst, c, threadIdx.x);
+            const uint32_t got = chunk_crc_staged(g, sHT, sT0, stage, ws.dig, chunk_first_byte(g, ws, dst, c), c, threadIdx.x);
             if (got != want) { atomicMin(&ws.ctrl->bad5_first, c); atomicAdd(&ws.ctrl->bad5_count, 1u); }
         } else {
             if (dst_crc[c] != want) { atomicMin(&ws.ctrl->bad6_first, c); atomicAdd(&ws.ctrl->bad6_count, 1u); }
@@ -1857,9 +1987,12 @@ static const DeviceState* device_state()
     if (cudaMemcpy(s.tables, &host, sizeof(Tables), cudaMemcpyHostToDevice) != cudaSuccess) return nullptr;
     if (cudaDeviceGetAttribute(&s.sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return nullptr;
     const int big = kDynSmem;
-    if (cudaFuncSetAttribute(k_encode<kTeams, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, big) != cudaSuccess) return nullptr;
-    if (cudaFuncSetAttribute(k_encode<kTeams, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, big) != cudaSuccess) return nullptr;
-    if (cudaFuncSetAttribute(k_decode<kTeamsPlain>, cudaFuncAttributeMaxDynamicSharedMemorySize, big) != cudaSuccess) return nullptr;
+    if (cudaFuncSetAttribute(k_encode<kTeams, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, big) != cudaSuccess) return nullptr;
+    if (cudaFuncSetAttribute(k_encode<kTeams, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, big) != cudaSuccess) return nullptr;
+    if (cudaFuncSetAttribute(k_encode<kTeams, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, big) != cudaSuccess) return nullptr;
+    if (cudaFuncSetAttribute(k_encode<kTeams, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, big) != cudaSuccess) return nullptr;
+    if (cudaFuncSetAttribute(k_decode<kTeamsPlain, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, big) != cudaSuccess) return nullptr;
+    if (cudaFuncSetAttribute(k_decode<kTeamsPlain, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, big) != cudaSuccess) return nullptr;
     if (cudaFuncSetAttribute(k_tile_digests<kTeamsPlain>, cudaFuncAttributeMaxDynamicSharedMemorySize, big) != cudaSuccess) return nullptr;
     if (cudaFuncSetAttribute(k_meta_crc, cudaFuncAttributeMaxDynamicSharedMemorySize, big) != cudaSuccess) return nullptr;
     for (int k = 0; k < 4; k++)
@@ -2047,14 +2180,15 @@ wm_status wm_dirty_diff(const void* cache, const void* prev, uint64_t nbytes, ui
     return launch_status();
 }
 
-wm_status wm_encode(const void* cache, uint64_t nbytes, uint32_t chunk_bytes, const uint8_t* dirty,
-                    uint32_t* crc_inout, void* wire, uint64_t wire_cap, void* workspace, uint64_t workspace_bytes,
-                    wm_result* result, void* stream)
+// Both forms of the encode call: a flat cache (leaves == nullptr) or a table of leaves.
+static wm_status encode_any(const void* cache, const wm_leaf* leaves, uint32_t n_leaves, uint64_t nbytes, uint32_t chunk_bytes,
+                            const uint8_t* dirty, uint32_t* crc_inout, void* wire, uint64_t wire_cap, void* workspace,
+                            uint64_t workspace_bytes, wm_result* result, void* stream)
 {
     Geo g;
-    if (!cache || !crc_inout || !wire || !workspace || !result || !make_geo(nbytes, chunk_bytes, g)) return WM_ERR_ARG;
-    if (!aligned16(cache) || !aligned16(wire) || !aligned16(workspace) || workspace_bytes < ws_layout(g).total ||
-        wire_cap < g.meta_end)
+    if (!crc_inout || !wire || !workspace || !result || !make_geo(nbytes, chunk_bytes, g)) return WM_ERR_ARG;
+    if (leaves ? (n_leaves == 0 || n_leaves > kMaxLeaves) : (!cache || !aligned16(cache))) return WM_ERR_ARG;
+    if (!aligned16(wire) || !aligned16(workspace) || workspace_bytes < ws_layout(g).total || wire_cap < g.meta_end)
         return WM_ERR_ARG;
     if (nbytes > kMaxCodecBytes) return WM_ERR_ARG;
     const DeviceState* ds = device_state();
@@ -2065,28 +2199,55 @@ wm_status wm_encode(const void* cache, uint64_t nbytes, uint32_t chunk_bytes, co
     unsigned char* w = static_cast<unsigned char*>(wire);
     const uint32_t init_blocks = (g.n_tiles + 1023) / 1024 < 1024 ? (g.n_tiles + 1023) / 1024 : 1024;
     k_encode_init<<<init_blocks ? init_blocks : 1, 1024, 0, s>>>(g, ws, w);
+    if (leaves) {
+        const uint32_t map_blocks = (g.n_tiles + 4095) / 4096 < 64 ? (g.n_tiles + 4095) / 4096 : 64;
+        launch_after(k_leaf_map, map_blocks ? map_blocks : 1, 1024, 0, s, leaves, n_leaves, g, ws, result, 0);
+    }
     // one block per SM: one of them scans, the others encode
     const uint32_t need = (g.n_tiles + kTeams - 1) / kTeams + 1;
     const uint32_t grid = need < (uint32_t)ds->sm_count ? need : (uint32_t)ds->sm_count;
     {
         MainKernelTimer timer(ds, 2, s);
-        if (dirty) launch_after(k_encode<kTeams, true>, grid, kTeams * 256, kDynSmem, s, c, g, dirty, w, wire_cap, ws, ds->tables);
-        else launch_after(k_encode<kTeams, false>, grid, kTeams * 256, kDynSmem, s, c, g, dirty, w, wire_cap, ws, ds->tables);
+        if (leaves) {
+            if (dirty) launch_after(k_encode<kTeams, true, true>, grid, kTeams * 256, kDynSmem, s, c, g, dirty, w, wire_cap, ws, ds->tables);
+            else launch_after(k_encode<kTeams, false, true>, grid, kTeams * 256, kDynSmem, s, c, g, dirty, w, wire_cap, ws, ds->tables);
+        } else {
+            if (dirty) launch_after(k_encode<kTeams, true, false>, grid, kTeams * 256, kDynSmem, s, c, g, dirty, w, wire_cap, ws, ds->tables);
+            else launch_after(k_encode<kTeams, false, false>, grid, kTeams * 256, kDynSmem, s, c, g, dirty, w, wire_cap, ws, ds->tables);
+        }
     }
     launch_after(k_encode_finish, (g.n_chunks + g.finish_cb - 1) / g.finish_cb, 1024, 0, s, c, g, dirty, crc_inout, w, ws, ds->tables,
                  chunk_powers(g));
     launch_after(k_meta_crc, (g.n_meta_slices + 3) / 4, 1024, kDynSmem, s, w, g, ws, ds->tables, result);
-    g_launches = 4;
+    g_launches = leaves ? 5 : 4;
     return launch_status();
 }
 
-wm_status wm_decode_verify(const void* wire, uint64_t wire_len, void* dst, uint64_t nbytes, uint32_t chunk_bytes,
-                           uint32_t* dst_crc_inout, void* workspace, uint64_t workspace_bytes, wm_result* result,
-                           void* stream)
+wm_status wm_encode(const void* cache, uint64_t nbytes, uint32_t chunk_bytes, const uint8_t* dirty,
+                    uint32_t* crc_inout, void* wire, uint64_t wire_cap, void* workspace, uint64_t workspace_bytes,
+                    wm_result* result, void* stream)
+{
+    if (!cache) return WM_ERR_ARG;
+    return encode_any(cache, nullptr, 0, nbytes, chunk_bytes, dirty, crc_inout, wire, wire_cap, workspace, workspace_bytes, result, stream);
+}
+
+wm_status wm_encode_leaves(const wm_leaf* leaves, uint32_t n_leaves, uint64_t nbytes, uint32_t chunk_bytes, const uint8_t* dirty,
+                           uint32_t* crc_inout, void* wire, uint64_t wire_cap, void* workspace, uint64_t workspace_bytes,
+                           wm_result* result, void* stream)
+{
+    if (!leaves) return WM_ERR_ARG;
+    return encode_any(nullptr, leaves, n_leaves, nbytes, chunk_bytes, dirty, crc_inout, wire, wire_cap, workspace, workspace_bytes, result, stream);
+}
+
+// Both forms of the decode call: a flat shadow buffer (leaves == nullptr) or a table of leaves.
+static wm_status decode_any(const void* wire, uint64_t wire_len, void* dst, const wm_leaf* leaves, uint32_t n_leaves, uint64_t nbytes,
+                            uint32_t chunk_bytes, uint32_t* dst_crc_inout, void* workspace, uint64_t workspace_bytes,
+                            wm_result* result, void* stream)
 {
     Geo g;
-    if (!wire || !dst || !dst_crc_inout || !workspace || !result || !make_geo(nbytes, chunk_bytes, g)) return WM_ERR_ARG;
-    if (!aligned16(wire) || !aligned16(dst) || !aligned16(workspace) || workspace_bytes < ws_layout(g).total) return WM_ERR_ARG;
+    if (!wire || !dst_crc_inout || !workspace || !result || !make_geo(nbytes, chunk_bytes, g)) return WM_ERR_ARG;
+    if (leaves ? (n_leaves == 0 || n_leaves > kMaxLeaves) : (!dst || !aligned16(dst))) return WM_ERR_ARG;
+    if (!aligned16(wire) || !aligned16(workspace) || workspace_bytes < ws_layout(g).total) return WM_ERR_ARG;
     if (nbytes > kMaxCodecBytes) return WM_ERR_ARG;
     const DeviceState* ds = device_state();
     if (!ds) return WM_ERR_CUDA;
@@ -2095,6 +2256,10 @@ wm_status wm_decode_verify(const void* wire, uint64_t wire_len, void* dst, uint6
     const unsigned char* w = static_cast<const unsigned char*>(wire);
     unsigned char* d = static_cast<unsigned char*>(dst);
     k_decode_init<<<1, 64, 0, s>>>(ws);
+    if (leaves) {
+        const uint32_t map_blocks = (g.n_tiles + 4095) / 4096 < 64 ? (g.n_tiles + 4095) / 4096 : 64;
+        launch_after(k_leaf_map, map_blocks ? map_blocks : 1, 1024, 0, s, leaves, n_leaves, g, ws, result, 1);
+    }
     // a wire shorter than the metadata is rejected by the header check before anything else is read
     const uint32_t meta_blocks = (g.n_meta_slices + 3) / 4;
     launch_after(k_decode_check, meta_blocks + (g.n_chunks + 31) / 32, 1024, 0, s, w, wire_len, g, ws, ds->tables, result, meta_blocks);
@@ -2102,12 +2267,30 @@ wm_status wm_decode_verify(const void* wire, uint64_t wire_len, void* dst, uint6
     const uint32_t grid = need < (uint32_t)ds->sm_count ? need : (uint32_t)ds->sm_count;
     {
         MainKernelTimer timer(ds, 3, s);
-        launch_after(k_decode<kTeamsPlain>, grid, kTeamsPlain * 256, kDynSmem, s, w, g, d, ws, ds->tables);
+        if (leaves) launch_after(k_decode<kTeamsPlain, true>, grid, kTeamsPlain * 256, kDynSmem, s, w, g, d, ws, ds->tables);
+        else launch_after(k_decode<kTeamsPlain, false>, grid, kTeamsPlain * 256, kDynSmem, s, w, g, d, ws, ds->tables);
     }
     launch_after(k_decode_finish, (g.n_chunks + g.finish_cb - 1) / g.finish_cb, 1024, 0, s, w, wire_len, g, d, dst_crc_inout, ws, ds->tables,
                  result, chunk_powers(g));
-    g_launches = 4;
+    g_launches = leaves ? 5 : 4;
     return launch_status();
+}
+
+wm_status wm_decode_verify(const void* wire, uint64_t wire_len, void* dst, uint64_t nbytes, uint32_t chunk_bytes,
+                           uint32_t* dst_crc_inout, void* workspace, uint64_t workspace_bytes, wm_result* result,
+                           void* stream)
+{
+    if (!dst) return WM_ERR_ARG;
+    return decode_any(wire, wire_len, dst, nullptr, 0, nbytes, chunk_bytes, dst_crc_inout, workspace, workspace_bytes, result, stream);
+}
+
+wm_status wm_decode_verify_leaves(const void* wire, uint64_t wire_len, const wm_leaf* dst_leaves, uint32_t n_leaves, uint64_t nbytes,
+                                  uint32_t chunk_bytes, uint32_t* dst_crc_inout, void* workspace, uint64_t workspace_bytes,
+                                  wm_result* result, void* stream)
+{
+    if (!dst_leaves) return WM_ERR_ARG;
+    return decode_any(wire, wire_len, nullptr, dst_leaves, n_leaves, nbytes, chunk_bytes, dst_crc_inout, workspace, workspace_bytes, result,
+                      stream);
 }
 
 }  // extern "C"

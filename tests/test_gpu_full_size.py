@@ -260,3 +260,33 @@ def test_precopy_step_loop_on_two_streams():
     dstream.synchronize()
     rd = wm.read_result(pending[1])
     assert rd.ok and torch.equal(dst, cur) and torch.equal(crc_dst, crc_src)
+
+
+def test_engine_cache_as_sixty_leaves_gives_the_flat_image():
+    """The engine cache as the model holds it: one key and one value tensor per layer (60 leaves
+    of 27.85 MB).  Leaf-mode encode must produce the flat call's image byte for byte, and
+    leaf-mode decode must fill separate destination tensors with the source's bytes."""
+    cfg = inputs.CONFIGS["engine"]
+    cur = inputs.make_cache(cfg, "cuda")
+    job = Job(cfg.nbytes, cfg.chunk_bytes)
+    n_leaves = cfg.shape[0] * cfg.shape[1]
+    leaf_bytes = cfg.nbytes // n_leaves
+    assert leaf_bytes % TILE == 0
+    leaves = [cur[i * leaf_bytes:(i + 1) * leaf_bytes].clone() for i in range(n_leaves)]
+    table = wm.make_leaf_table(leaves)
+    crc_flat = torch.zeros(job.nc, dtype=torch.int32, device="cuda")
+    crc_leaf = torch.zeros(job.nc, dtype=torch.int32, device="cuda")
+    wm.wm_encode(cur, job.chunk, None, crc_flat, job.wire, job.ws, job.res_e)
+    r_flat = wm.read_result(job.res_e)
+    wire_leaf = torch.empty_like(job.wire)
+    wm.wm_encode_leaves(table, job.n, job.chunk, None, crc_leaf, wire_leaf, job.ws, job.res_e)
+    r_leaf = wm.read_result(job.res_e)
+    assert r_flat.ok and r_leaf.ok
+    assert (r_leaf.wire_len, r_leaf.cache_crc, r_leaf.n_present) == (r_flat.wire_len, r_flat.cache_crc, r_flat.n_present)
+    assert torch.equal(wire_leaf[: r_leaf.wire_len], job.wire[: r_flat.wire_len]) and torch.equal(crc_leaf, crc_flat)
+    dst = [torch.zeros_like(x) for x in leaves]
+    dtable = wm.make_leaf_table(dst)
+    crc_dst = torch.zeros(job.nc, dtype=torch.int32, device="cuda")
+    wm.wm_decode_verify_leaves(wire_leaf, r_leaf.wire_len, dtable, job.n, job.chunk, crc_dst, job.ws, job.res_d)
+    assert wm.read_result(job.res_d).ok and torch.equal(crc_dst, crc_flat)
+    assert all(torch.equal(a, b) for a, b in zip(dst, leaves))

@@ -1,0 +1,139 @@
+"""Leaf mode: the cache as a list of tensors.  Its definition is the flat call on the leaves'
+concatenation, so the oracle side is that concatenation; the GPU side reads and writes the
+leaves in place and must give the same image, checksums, verdicts and bytes."""
+import numpy as np
+import pytest
+
+import oracle
+
+TILE = 16384
+
+
+def split_sizes(nbytes, cuts):
+    """Leaf sizes for a cache of nbytes cut at the given tile numbers (ascending)."""
+    edges = [0] + [c * TILE for c in cuts] + [nbytes]
+    return [b - a for a, b in zip(edges[:-1], edges[1:])]
+
+
+def test_oracle_leaf_calls_are_the_flat_calls_on_the_concatenation():
+    rng = np.random.default_rng(7)
+    flat = (rng.normal(size=3 * 65536 // 2 + 700).astype(np.float32).view(np.uint32) >> 16).astype(np.uint16).view(np.uint8)
+    sizes = split_sizes(flat.size, [1, 5, 6])
+    leaves, o = [], 0
+    for n in sizes:
+        leaves.append(flat[o:o + n].copy())
+        o += n
+    assert np.array_equal(oracle.flatten_leaves(leaves), flat)
+    w0, c0, r0 = oracle.encode(flat, 65536)
+    w1, c1, r1 = oracle.encode_leaves(leaves, 65536)
+    assert np.array_equal(w0, w1) and np.array_equal(c0, c1) and r0.wire_len == r1.wire_len
+    blank = [np.zeros_like(x) for x in leaves]
+    out, crc, r = oracle.decode_verify_leaves(w1, blank, 65536)
+    assert r.status == 0 and np.array_equal(crc, c0)
+    assert all(np.array_equal(a, b) for a, b in zip(out, leaves))
+    assert all(not x.any() for x in blank)                     # the caller's arrays are the live state
+
+
+gpu = pytest.mark.gpu
+
+
+def _setup(nbytes, chunk, cuts, seed):
+    import torch
+    from paper_2607_10389_b200 import binding as wm
+    g = torch.Generator(device="cuda").manual_seed(seed)
+    flat = torch.randn(((nbytes + 1) // 2,), generator=g, device="cuda").to(torch.bfloat16).view(torch.uint8)[:nbytes].contiguous()
+    sizes = split_sizes(nbytes, cuts)
+    leaves, o = [], 0
+    for n in sizes:                      # separate allocations, as an engine's tensors are
+        leaves.append(flat[o:o + n].clone())
+        o += n
+    return torch, wm, flat, leaves
+
+
+@gpu
+@pytest.mark.parametrize("nbytes,chunk,cuts", [
+    (5 * 65536 + 3 * TILE + 1000, 65536, [1, 2, 9, 17]),       # ragged last leaf, chunks straddle leaves
+    (40 * TILE, 8 * TILE, [8, 16, 24, 32]),                    # leaves on chunk boundaries
+    (64 * TILE, 65536, list(range(1, 64))),                    # one tile per leaf
+    (3 * TILE + 2, 65536, []),                                 # a single leaf
+])
+def test_leaf_encode_and_decode_match_the_oracle(nbytes, chunk, cuts):
+    torch, wm, flat, leaves = _setup(nbytes, chunk, cuts, seed=nbytes % 1000)
+    nc = wm.num_chunks(nbytes, chunk)
+    ws = wm.new_workspace(nbytes, chunk)
+    cap = wm.wire_bound(nbytes, chunk)
+    res = wm.new_result()
+    table = wm.make_leaf_table(leaves)
+    for dirty_np in (None, (np.arange(nc) % 3 != 1).astype(np.uint8)):
+        crc_in = (np.arange(nc, dtype=np.uint64) * 2654435761 % (1 << 32)).astype(np.uint32)
+        want_wire, want_crc, want = oracle.encode_leaves([x.cpu().numpy() for x in leaves], chunk, dirty=dirty_np,
+                                                          crc_in=crc_in.astype(np.uint32))
+        wire = torch.full((cap + 64,), 0xA5, dtype=torch.uint8, device="cuda")
+        crc = torch.from_numpy(crc_in.astype(np.uint32).view(np.int32).copy()).cuda()
+        dirty = None if dirty_np is None else torch.from_numpy(dirty_np).cuda()
+        wm.wm_encode_leaves(table, nbytes, chunk, dirty, crc, wire, ws, res, wire_cap=cap)
+        r = wm.read_result(res)
+        assert (r.status, r.wire_len, r.n_present, r.cache_crc) == (want.status, want.wire_len, want.n_present, want.cache_crc)
+        got = wire.cpu().numpy()
+        assert np.array_equal(got[: r.wire_len], want_wire) and (got[cap:] == 0xA5).all()
+        assert np.array_equal(crc.cpu().numpy().view(np.uint32), want_crc)
+        # the flat call gives the same image
+        wire2 = torch.zeros(cap, dtype=torch.uint8, device="cuda")
+        crc2 = torch.from_numpy(crc_in.astype(np.uint32).view(np.int32).copy()).cuda()
+        wm.wm_encode(flat, chunk, dirty, crc2, wire2, ws, res)
+        assert torch.equal(wire2[: r.wire_len], wire[: r.wire_len])
+
+        # decode into fresh leaves that hold the old content of the absent chunks
+        old = flat.clone()
+        if dirty_np is not None:
+            for c in np.nonzero(dirty_np)[0]:
+                old[c * chunk: min((c + 1) * chunk, nbytes)] = 0x11
+        dst_leaves, o = [], 0
+        for x in leaves:
+            dst_leaves.append(old[o:o + x.numel()].clone())
+            o += x.numel()
+        dtable = wm.make_leaf_table(dst_leaves)
+        dcrc = crc.clone()
+        wm.wm_decode_verify_leaves(wire, r.wire_len, dtable, nbytes, chunk, dcrc, ws, res)
+        rd = wm.read_result(res)
+        assert rd.ok and rd.cache_crc == want.cache_crc
+        assert all(torch.equal(a, b) for a, b in zip(dst_leaves, leaves))
+        # one flipped payload bit is caught on the way into the leaves
+        wire[r.wire_len - 5] ^= 4
+        wm.wm_decode_verify_leaves(wire, r.wire_len, dtable, nbytes, chunk, dcrc, ws, res)
+        assert wm.read_result(res).status_name == "ERR_CHUNK_CRC"
+
+
+@gpu
+def test_leaf_table_that_breaks_the_rules_is_rejected():
+    torch, wm, flat, leaves = _setup(8 * TILE, 65536, [2, 5], seed=3)
+    nbytes, chunk = 8 * TILE, 65536
+    nc = wm.num_chunks(nbytes, chunk)
+    ws, res = wm.new_workspace(nbytes, chunk), wm.new_result()
+    cap = wm.wire_bound(nbytes, chunk)
+    wire = torch.zeros(cap, dtype=torch.uint8, device="cuda")
+    crc = torch.zeros(nc, dtype=torch.int32, device="cuda")
+    good = wm.make_leaf_table(leaves)
+    wm.wm_encode_leaves(good, nbytes, chunk, None, crc, wire, ws, res)
+    r = wm.read_result(res)
+    assert r.ok
+    bad_tables = []
+    t = good.clone(); t[0, 1] -= 16; t[1, 1] += 16; bad_tables.append(t)          # a middle leaf that is not whole tiles
+    t = good.clone(); t[2, 1] += TILE; bad_tables.append(t)                        # sizes do not add up
+    t = good.clone(); t[1, 0] += 4; bad_tables.append(t)                           # misaligned leaf
+    t = good.clone(); t[1, 1] = 0; bad_tables.append(t)                            # empty leaf
+    for t in bad_tables:
+        wm.wm_encode_leaves(t, nbytes, chunk, None, crc, wire, ws, res)
+        assert wm.read_result(res).status_name == "ERR_ARG"
+    # decode: a bad destination table is refused before anything is written
+    wm.wm_encode_leaves(good, nbytes, chunk, None, crc, wire, ws, res)
+    dst = [torch.full_like(x, 0x33) for x in leaves]
+    for t in bad_tables:
+        dt = wm.make_leaf_table(dst)
+        dt[:, 1] = t[:, 1]
+        if not torch.equal(t[:, 0], good[:, 0]):
+            dt[1, 0] += 4
+        dcrc = torch.zeros(nc, dtype=torch.int32, device="cuda")
+        wm.wm_decode_verify_leaves(wire, r.wire_len, dt, nbytes, chunk, dcrc, ws, res)
+        assert wm.read_result(res).status_name == "ERR_ARG"
+        assert all((x == 0x33).all() for x in dst) and not dcrc.any()
