@@ -255,6 +255,12 @@ static int plane_widths(uint32_t w, uint32_t p[3])
 static uint32_t encode_full_tile(const uint8_t* src, uint8_t* out, uint32_t* entry)
 {
     uint32_t base[WMO_GROUPS_PER_TILE], w[WMO_GROUPS_PER_TILE], S = 0;
+    /* a tile whose 16384 bytes are all zero (unused allocation) has entry 1 and no payload */
+    {
+        uint32_t any = 0;
+        for (uint32_t i = 0; i < WMO_TILE; i++) any |= src[i];
+        if (!any) { *entry = 1u; return 0; }
+    }
     for (uint32_t g = 0; g < WMO_GROUPS_PER_TILE; g++) {
         uint32_t mn = 255, mx = 0;
         for (uint32_t e = 0; e < WMO_GROUP_ELEMS; e++) {
@@ -313,7 +319,8 @@ static uint32_t encode_full_tile(const uint8_t* src, uint8_t* out, uint32_t* ent
  *           24 u32 n_chunks 28 u32 n_present     32 u64 payload_bytes
  *           40 u64 wire_len 48 u32 cache_crc     52 u32 meta_crc   56 8 zero bytes
  *   chunk_dir[c]: u64 payload_off | u32 enc_len | u32 crc
- *   tile_tab[t] : 0 absent | 258..511 PACK of 32*value bytes | 512 RAW full tile |
+ *   tile_tab[t] : 0 absent | 1 ZERO full tile (all bytes zero, no payload) |
+ *                 258..511 PACK of 32*value bytes | 512 RAW full tile |
  *                 0xFFFF RAW partial tail tile
  *   payload: encoded tiles of present chunks in ascending order, no padding.
  *
@@ -498,6 +505,7 @@ int wmo_decode_verify(const uint8_t* wire, uint64_t wire_len, uint8_t* dst, uint
                 if (e == 0) { all = 0; continue; }
                 any = 1;
                 if (tlen < WMO_TILE) { if (e != 0xFFFFu) ok = 0; sum += tlen; }
+                else if (e == 1u) sum += 0;                /* ZERO tile: full tiles only, no payload */
                 else if (e >= 258u && e <= 512u) sum += 32u * (uint64_t)e;
                 else ok = 0;
             }
@@ -522,7 +530,7 @@ int wmo_decode_verify(const uint8_t* wire, uint64_t wire_len, uint8_t* dst, uint
             for (uint64_t i = 0; i < ntc; i++) {
                 uint32_t e = get16(tab + 2u * (t0 + i));
                 if (e == 0) break;
-                uint64_t tlen = (e == 0xFFFFu) ? clen - i * WMO_TILE : 32u * (uint64_t)e;
+                uint64_t tlen = (e == 0xFFFFu) ? clen - i * WMO_TILE : (e == 1u) ? 0 : 32u * (uint64_t)e;
                 if (e >= 258u && e <= 511u) {
                     const uint8_t* in = payload + off;
                     int tile_status = WMO_OK; uint32_t S = 0;
@@ -556,8 +564,9 @@ int wmo_decode_verify(const uint8_t* wire, uint64_t wire_len, uint8_t* dst, uint
             uint8_t* out = dst + c * (uint64_t)chunk_bytes;
             for (uint64_t i = 0; i < ntc; i++) {
                 uint32_t e = get16(tab + 2u * (t0 + i));
-                uint64_t tlen = (e == 0xFFFFu) ? clen - i * WMO_TILE : 32u * (uint64_t)e;
-                if (e == 512u || e == 0xFFFFu) memcpy(out + i * WMO_TILE, payload + off, tlen);
+                uint64_t tlen = (e == 0xFFFFu) ? clen - i * WMO_TILE : (e == 1u) ? 0 : 32u * (uint64_t)e;
+                if (e == 1u) memset(out + i * WMO_TILE, 0, WMO_TILE);
+                else if (e == 512u || e == 0xFFFFu) memcpy(out + i * WMO_TILE, payload + off, tlen);
                 else decode_pack_tile(payload + off, out + i * WMO_TILE);
                 off += tlen;
             }

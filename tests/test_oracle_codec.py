@@ -380,3 +380,84 @@ def test_capacity_error_reports_needed_size():
         oracle.encode(a, TILE, wire_cap=oracle.meta_end(len(a), TILE) - 1)
     with pytest.raises(ValueError):
         oracle.encode(a, 1000)
+
+
+# ---------------------------------------------------------------- ZERO tiles (unused allocation)
+
+def _rand_tile(seed):
+    rng = np.random.default_rng(seed)
+    return (rng.normal(size=8192).astype(np.float32).view(np.uint32) >> 16).astype("<u2").view(np.uint8)
+
+
+def test_zero_tiles_have_entry_one_and_no_payload():
+    a, b = _rand_tile(1), _rand_tile(2)
+    z = np.zeros(TILE, dtype=np.uint8)
+    cache = np.concatenate([a, z, z, b])
+    wire, crc, res = oracle.encode(cache, 4 * TILE)
+    wa, _, ra = oracle.encode(a, TILE)
+    wb, _, rb = oracle.encode(b, TILE)
+    ea, eb = wa[96:ra.wire_len], wb[96:rb.wire_len]
+    tab = _tab(wire, 1, 4).tolist()
+    assert tab == [int(_tab(wa, 1, 1)[0]), 1, 1, int(_tab(wb, 1, 1)[0])]
+    me = oracle.meta_end(4 * TILE, 4 * TILE)
+    assert res.payload_bytes == ea.size + eb.size and res.wire_len == me + ea.size + eb.size
+    assert np.array_equal(wire[me:me + ea.size], ea) and np.array_equal(wire[me + ea.size:], eb)
+    assert _dir(wire, 1)[0][:2] == (0, ea.size + eb.size)
+    assert int(crc[0]) == oracle.crc32c(cache)               # the checksum is of the raw bytes, zeros included
+    out, dcrc, r = oracle.decode_verify(wire, cache.size, 4 * TILE, dst=np.full(cache.size, 0xEE, np.uint8))
+    assert r.status == 0 and np.array_equal(out, cache)
+
+
+def test_all_zero_cache_is_metadata_plus_its_ragged_tail():
+    n = 3 * TILE + 100
+    cache = np.zeros(n, dtype=np.uint8)
+    wire, crc, res = oracle.encode(cache, 2 * TILE)
+    assert _tab(wire, 2, 4).tolist() == [1, 1, 1, 0xFFFF]
+    assert res.payload_bytes == 100 and res.wire_len == oracle.meta_end(n, 2 * TILE) + 100
+    assert [d[1] for d in _dir(wire, 2)] == [0, 100]
+    out, _, r = oracle.decode_verify(wire, n, 2 * TILE, dst=np.full(n, 7, np.uint8))
+    assert r.status == 0 and not out.any()
+
+
+@pytest.mark.parametrize("word", [0x8000, 0x0001, 0x0080])
+def test_only_all_zero_bytes_make_a_zero_tile(word):
+    # minus zero, the smallest denormal and the smallest normal exponent are data, not emptiness
+    tile = np.zeros(8192, dtype="<u2")
+    tile[4711] = word
+    wire, _, res = oracle.encode(tile.view(np.uint8), TILE)
+    assert _tab(wire, 1, 1)[0] >= 258 and res.payload_bytes >= 8256
+    out, _, r = oracle.decode_verify(wire, TILE, TILE)
+    assert r.status == 0 and np.array_equal(out, tile.view(np.uint8))
+
+
+def _refresh_meta_crc(wire, nbytes, chunk):
+    me = oracle.meta_end(nbytes, chunk)
+    w = wire.copy()
+    w[52:56] = 0
+    w[52:56] = np.frombuffer(struct.pack("<I", oracle.crc32c(w[:me])), dtype=np.uint8)
+    return w
+
+
+def test_zero_entry_is_checked_like_any_other():
+    a = _rand_tile(3)
+    cache = np.concatenate([a, np.zeros(TILE, np.uint8), a[:500]])
+    n, chunk = cache.size, 4 * TILE
+    wire, crc, res = oracle.encode(cache, chunk)
+    assert _tab(wire, 1, 3).tolist()[1:] == [1, 0xFFFF]
+    tab_off = 64 + 16
+    # a ZERO entry where a ragged tile belongs: the structure check refuses it
+    w = wire.copy(); w[tab_off + 4: tab_off + 6] = (1, 0)
+    assert oracle.decode_verify(_refresh_meta_crc(w, n, chunk), n, chunk)[2].status_name == "ERR_STRUCT"
+    # a data tile relabelled as ZERO: lengths no longer add up
+    w = wire.copy(); w[tab_off: tab_off + 2] = (1, 0)
+    assert oracle.decode_verify(_refresh_meta_crc(w, n, chunk), n, chunk)[2].status_name == "ERR_STRUCT"
+    # the same with the directory length patched as well: caught by the chunk CRC
+    e0 = int(_tab(wire, 1, 3)[0]) * 32
+    w[64 + 8: 64 + 12] = np.frombuffer(struct.pack("<I", 500), dtype=np.uint8)
+    w = np.concatenate([w[:oracle.meta_end(n, chunk)], w[oracle.meta_end(n, chunk) + e0:]])
+    w[32:40] = np.frombuffer(struct.pack("<Q", 500), dtype=np.uint8)
+    w[40:48] = np.frombuffer(struct.pack("<Q", w.size), dtype=np.uint8)
+    assert oracle.decode_verify(_refresh_meta_crc(w, n, chunk), n, chunk)[2].status_name == "ERR_CHUNK_CRC"
+    # without fixing the metadata CRC any of these stops at the metadata check
+    w = wire.copy(); w[tab_off + 2] ^= 1
+    assert oracle.decode_verify(w, n, chunk)[2].status_name == "ERR_META_CRC"
