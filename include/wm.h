@@ -107,12 +107,14 @@ wm_status wm_dirty_diff(const void* cache, const void* prev, uint64_t nbytes, ui
  * decoded bytes).  The paper fixes those properties, not a layout; WM1 is this library's:
  *
  *   header[64] | chunk_dir[16*n_chunks] | tile_tab[2*n_tiles] | zero pad to 32 | payload
- *   header: 0 "WMV1" | 4 u16 version=1 | 6 u16 flags (bit0: a dirty mask was given) |
+ *   header: 0 "WMV1" | 4 u16 version=1 | 6 u16 flags (bit0: a dirty mask was given; bit1:
+ *           the ZERO tile option, see wm_zero_tiles_enable) |
  *           8 u64 nbytes | 16 u32 chunk_bytes | 20 u32 tile_bytes=16384 | 24 u32 n_chunks |
  *           28 u32 n_present | 32 u64 payload_bytes | 40 u64 wire_len | 48 u32 cache_crc |
  *           52 u32 meta_crc (CRC32C of the metadata with this field as zero) | 56 zero[8]
  *   chunk_dir[c]: u64 payload_off | u32 enc_len | u32 crc
- *   tile_tab[t] (u16): 0 tile of an absent chunk | 258..511 PACK tile of 32*value bytes |
+ *   tile_tab[t] (u16): 0 tile of an absent chunk | 1 ZERO tile: a full tile whose bytes are
+ *           all zero, no payload (only in images with flags bit1) | 258..511 PACK tile of 32*value bytes |
  *           512 RAW full tile | 0xFFFF RAW partial tail tile (nbytes mod 16384 bytes)
  *   payload: encoded tiles of present chunks in ascending order, no padding
  *   PACK tile (32 groups of 256 elements): desc[32] u16 (base | w<<8 | chk<<12,
@@ -166,6 +168,19 @@ wm_status wm_encode(const void* cache, uint64_t nbytes, uint32_t chunk_bytes, co
 wm_status wm_decode_verify(const void* wire, uint64_t wire_len, void* dst, uint64_t nbytes,
                            uint32_t chunk_bytes, uint32_t* dst_crc_inout,
                            void* workspace, uint64_t workspace_bytes, wm_result* result, void* stream);
+
+/*
+ * wm_zero_tiles_enable - encoder option: ship unused (all-zero) memory as table entries.
+ * Paper: at least 19.4 % of the movable set is an allocation that no step writes or reads
+ * (Section 3.3).  Read here as zero-filled memory: with the option on, a full tile of a
+ * present chunk whose 16384 bytes are all zero gets tile_tab entry 1 and no payload bytes
+ * (without it such a tile packs to 8256 bytes), and header flags bit1 is set.  Only the
+ * all-zero byte pattern qualifies (minus zero and denormals are data).  The decoder accepts
+ * entry 1 in images that declare the option and writes zeros, which it checksums like any
+ * decoded tile.  Process-wide switch, off by default (the detection costs the encoder about
+ * 3 % on caches without such tiles); applies to wm_encode and wm_encode_leaves.
+ */
+void wm_zero_tiles_enable(int on);
 
 /*
  * Leaf mode - the cache as the engine holds it: a list of tensors, not one buffer.

@@ -252,11 +252,11 @@ static int plane_widths(uint32_t w, uint32_t p[3])
     if (w & 1u) p[n++] = 1u;
     return n;
 }
-static uint32_t encode_full_tile(const uint8_t* src, uint8_t* out, uint32_t* entry)
+static uint32_t encode_full_tile(const uint8_t* src, uint8_t* out, uint32_t* entry, int zero_tiles)
 {
     uint32_t base[WMO_GROUPS_PER_TILE], w[WMO_GROUPS_PER_TILE], S = 0;
-    /* a tile whose 16384 bytes are all zero (unused allocation) has entry 1 and no payload */
-    {
+    /* option: a tile whose 16384 bytes are all zero (unused allocation) has entry 1 and no payload */
+    if (zero_tiles) {
         uint32_t any = 0;
         for (uint32_t i = 0; i < WMO_TILE; i++) any |= src[i];
         if (!any) { *entry = 1u; return 0; }
@@ -314,7 +314,8 @@ static uint32_t encode_full_tile(const uint8_t* src, uint8_t* out, uint32_t* ent
  *   header[64] | chunk_dir[16 n_chunks] | tile_tab[2 n_tiles] | zero pad to a
  *   multiple of 32 (= meta_end) | payload
  *
- *   header:  0 "WMV1"   4 u16 version=1   6 u16 flags (bit0: a dirty mask was given)
+ *   header:  0 "WMV1"   4 u16 version=1   6 u16 flags (bit0: a dirty mask was given;
+ *            bit1: ZERO tile option)
  *            8 u64 nbytes   16 u32 chunk_bytes   20 u32 tile_bytes=16384
  *           24 u32 n_chunks 28 u32 n_present     32 u64 payload_bytes
  *           40 u64 wire_len 48 u32 cache_crc     52 u32 meta_crc   56 8 zero bytes
@@ -331,8 +332,21 @@ static uint32_t encode_full_tile(const uint8_t* src, uint8_t* out, uint32_t* ent
  * `dirty` may be NULL (every chunk present).  crc_inout[c] is written for present
  * chunks and read for absent ones.  Returns the status also stored in *res.
  */
+#define WMO_FLAG_MASKED 1u       /* header flags: a dirty mask was given             */
+#define WMO_FLAG_ZERO_TILES 2u   /* header flags: all-zero tiles are table entries   */
+
+int wmo_encode_opt(const uint8_t* cache, uint64_t nbytes, uint32_t chunk_bytes, const uint8_t* dirty,
+                   uint32_t* crc_inout, uint8_t* wire, uint64_t wire_cap, int zero_tiles, wmo_result* res);
+
 int wmo_encode(const uint8_t* cache, uint64_t nbytes, uint32_t chunk_bytes, const uint8_t* dirty,
                uint32_t* crc_inout, uint8_t* wire, uint64_t wire_cap, wmo_result* res)
+{
+    return wmo_encode_opt(cache, nbytes, chunk_bytes, dirty, crc_inout, wire, wire_cap, 0, res);
+}
+
+/* zero_tiles != 0: the ZERO tile option (tile table entry 1), recorded in header flags bit 1. */
+int wmo_encode_opt(const uint8_t* cache, uint64_t nbytes, uint32_t chunk_bytes, const uint8_t* dirty,
+                   uint32_t* crc_inout, uint8_t* wire, uint64_t wire_cap, int zero_tiles, wmo_result* res)
 {
     if (!cache || !crc_inout || !wire || !res || !args_ok(nbytes, chunk_bytes)) return WMO_ERR_ARG;
     uint64_t nc = wmo_num_chunks(nbytes, chunk_bytes), nt = wmo_num_tiles(nbytes);
@@ -361,7 +375,7 @@ int wmo_encode(const uint8_t* cache, uint64_t nbytes, uint32_t chunk_bytes, cons
                 uint64_t tlen = clen - o < WMO_TILE ? clen - o : WMO_TILE;
                 uint32_t entry, elen;
                 if (tlen < WMO_TILE) { memcpy(tile_buf, cp + o, tlen); entry = 0xFFFFu; elen = (uint32_t)tlen; }
-                else elen = encode_full_tile(cp + o, tile_buf, &entry);
+                else elen = encode_full_tile(cp + o, tile_buf, &entry, zero_tiles);
                 put16(tab + 2u * t, entry);
                 if (!overflow && meta_end + off + enc_len + elen <= wire_cap)
                     memcpy(wire + meta_end + off + enc_len, tile_buf, elen);
@@ -380,7 +394,7 @@ int wmo_encode(const uint8_t* cache, uint64_t nbytes, uint32_t chunk_bytes, cons
 
     memcpy(wire, "WMV1", 4);
     put16(wire + 4, 1);
-    put16(wire + 6, dirty ? 1u : 0u);
+    put16(wire + 6, (dirty ? WMO_FLAG_MASKED : 0u) | (zero_tiles ? WMO_FLAG_ZERO_TILES : 0u));
     put64(wire + 8, nbytes);
     put32(wire + 16, chunk_bytes);
     put32(wire + 20, WMO_TILE);
@@ -463,13 +477,14 @@ int wmo_decode_verify(const uint8_t* wire, uint64_t wire_len, uint8_t* dst, uint
 
     /* 1 */
     if (wire_len < WMO_HEADER || memcmp(wire, "WMV1", 4) != 0 || get16(wire + 4) != 1 ||
-        get16(wire + 6) > 1 || get64(wire + 8) != nbytes || get32(wire + 16) != chunk_bytes ||
+        get16(wire + 6) > 3 || get64(wire + 8) != nbytes || get32(wire + 16) != chunk_bytes ||
         get32(wire + 20) != WMO_TILE || get32(wire + 24) != nc || get64(wire + 40) != wire_len ||
         wire_len < meta_end || get64(wire + 32) != wire_len - meta_end) {
         fail(res, WMO_ERR_FORMAT, 0, 0);
         return res->status;
     }
     uint64_t payload_bytes = get64(wire + 32);
+    int zero_ok = (get16(wire + 6) & 2u) != 0;      /* entry 1 is legal only in an image that declares the option */
     uint32_t n_present_hdr = get32(wire + 28);
     uint32_t cache_crc_hdr = get32(wire + 48);
     res->wire_len = wire_len; res->payload_bytes = payload_bytes;
@@ -505,7 +520,7 @@ int wmo_decode_verify(const uint8_t* wire, uint64_t wire_len, uint8_t* dst, uint
                 if (e == 0) { all = 0; continue; }
                 any = 1;
                 if (tlen < WMO_TILE) { if (e != 0xFFFFu) ok = 0; sum += tlen; }
-                else if (e == 1u) sum += 0;                /* ZERO tile: full tiles only, no payload */
+                else if (e == 1u && zero_ok) sum += 0;     /* ZERO tile: full tiles only, no payload */
                 else if (e >= 258u && e <= 512u) sum += 32u * (uint64_t)e;
                 else ok = 0;
             }

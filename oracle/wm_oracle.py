@@ -85,6 +85,8 @@ def _load():
     lib.wmo_dirty_diff.argtypes = [u8p, u8p, u64, u32, u8p, u32p, u32p]
     lib.wmo_encode.restype = ctypes.c_int
     lib.wmo_encode.argtypes = [u8p, u64, u32, u8p, u32p, u8p, u64, ctypes.POINTER(_CResult)]
+    lib.wmo_encode_opt.restype = ctypes.c_int
+    lib.wmo_encode_opt.argtypes = [u8p, u64, u32, u8p, u32p, u8p, u64, ctypes.c_int, ctypes.POINTER(_CResult)]
     lib.wmo_decode_verify.restype = ctypes.c_int
     lib.wmo_decode_verify.argtypes = [u8p, u64, u8p, u64, u32, u32p, ctypes.POINTER(_CResult)]
     _lib = lib
@@ -161,8 +163,9 @@ def dirty_diff(cache, prev, chunk_bytes: int):
     return dirty, idx[: int(n[0])].copy()
 
 
-def encode(cache, chunk_bytes: int, dirty=None, crc_in=None, wire_cap: int | None = None):
-    """Return (wire u8[wire_len or wire_cap], crc u32[n_chunks], Result)."""
+def encode(cache, chunk_bytes: int, dirty=None, crc_in=None, wire_cap: int | None = None, zero_tiles: bool = False):
+    """Return (wire u8[wire_len or wire_cap], crc u32[n_chunks], Result).  ``zero_tiles``: the
+    option that ships a full tile of all-zero bytes as a table entry without payload."""
     b = _bytes_view(cache)
     nc = num_chunks(b.size, chunk_bytes)
     cap = wire_bound(b.size, chunk_bytes) if wire_cap is None else int(wire_cap)
@@ -170,8 +173,8 @@ def encode(cache, chunk_bytes: int, dirty=None, crc_in=None, wire_cap: int | Non
     crc = np.zeros(nc, dtype=np.uint32) if crc_in is None else np.array(crc_in, dtype=np.uint32).copy()
     d = None if dirty is None else np.ascontiguousarray(dirty, dtype=np.uint8)
     res = _CResult()
-    st = _load().wmo_encode(_ptr(b), b.size, chunk_bytes, None if d is None else _ptr(d), _ptr(crc),
-                            _ptr(wire), cap, ctypes.byref(res))
+    st = _load().wmo_encode_opt(_ptr(b), b.size, chunk_bytes, None if d is None else _ptr(d), _ptr(crc),
+                                _ptr(wire), cap, 1 if zero_tiles else 0, ctypes.byref(res))
     _check(st, "encode")
     r = _result(res)
     if r.status == 0:
@@ -198,10 +201,12 @@ def flatten_leaves(leaves) -> np.ndarray:
     return np.concatenate([_bytes_view(x) for x in leaves]) if len(leaves) else np.zeros(0, dtype=np.uint8)
 
 
-def encode_leaves(leaves, chunk_bytes: int, dirty=None, crc_in=None, wire_cap: int | None = None):
+def encode_leaves(leaves, chunk_bytes: int, dirty=None, crc_in=None, wire_cap: int | None = None,
+                  zero_tiles: bool = False):
     """Leaf mode is defined by the flat calls: the image of a list of leaves is the image of their
     concatenation.  Returns what encode() returns."""
-    return encode(flatten_leaves(leaves), chunk_bytes, dirty=dirty, crc_in=crc_in, wire_cap=wire_cap)
+    return encode(flatten_leaves(leaves), chunk_bytes, dirty=dirty, crc_in=crc_in, wire_cap=wire_cap,
+                  zero_tiles=zero_tiles)
 
 
 def decode_verify_leaves(wire, leaves, chunk_bytes: int, dst_crc=None, wire_len: int | None = None):

@@ -24,7 +24,7 @@ RESULT_BYTES = 40
 EXPORTS = ("wm_num_chunks", "wm_num_tiles", "wm_meta_bytes", "wm_wire_bound", "wm_workspace_bytes",
            "wm_checksum", "wm_dirty_diff", "wm_encode", "wm_decode_verify", "wm_last_launch_count",
            "wm_timing_enable", "wm_timing_read_ms", "wm_checksum_noalloc", "wm_encode_leaves",
-           "wm_decode_verify_leaves")
+           "wm_decode_verify_leaves", "wm_zero_tiles_enable")
 
 
 class WmError(RuntimeError):
@@ -48,6 +48,8 @@ def load_library() -> ctypes.CDLL:
     lib.wm_last_launch_count.argtypes = []
     lib.wm_timing_enable.restype = None
     lib.wm_timing_enable.argtypes = [ctypes.c_int]
+    lib.wm_zero_tiles_enable.restype = None
+    lib.wm_zero_tiles_enable.argtypes = [ctypes.c_int]
     lib.wm_timing_read_ms.restype = ctypes.c_int
     lib.wm_timing_read_ms.argtypes = [ctypes.c_int, ctypes.POINTER(ctypes.c_float)]
     lib.wm_checksum.restype = ctypes.c_int
@@ -133,6 +135,11 @@ KIND_CHECKSUM, KIND_DIFF, KIND_ENCODE, KIND_DECODE = 0, 1, 2, 3
 
 def timing_enable(on: bool) -> None:
     lib().wm_timing_enable(1 if on else 0)
+
+
+def zero_tiles_enable(on: bool) -> None:
+    """Encoder option: full tiles of all-zero bytes become table entries without payload."""
+    lib().wm_zero_tiles_enable(1 if on else 0)
 
 
 def timing_read_ms(kind: int) -> float:

@@ -853,6 +853,9 @@ __device__ __forceinline__ void pack_group_planes(uint32_t e4a, uint32_t e4b, ui
 // tile of its chunk, kQPresent when its chunk is encoded; kQNone: no tile.  (The codec takes
 // caches of at most 2^21 tiles, so a number never reaches the flag bits.)
 constexpr uint32_t kQPresent = 1u << 31, kQFirst = 1u << 30, kQTile = (1u << 30) - 1u, kQNone = kQTile;
+// Marks in a team's width table: on a warp's first entry, all 2 KiB of the warp's rows are zero;
+// as the sum of the widths, the tile is all zero.
+constexpr uint32_t kWarpAllZero = 0x8000u, kSumZeroTile = 0xFFFFu;
 
 template <bool MASKED>
 __device__ __forceinline__ uint32_t describe_tile(const Geo& g, const uint8_t* __restrict__ dirty, uint32_t t)
@@ -864,7 +867,7 @@ __device__ __forceinline__ uint32_t describe_tile(const Geo& g, const uint8_t* _
     return q;
 }
 
-template <int TEAMS, bool MASKED, bool LEAVES>
+template <int TEAMS, bool MASKED, bool LEAVES, bool ZEROS>
 __global__ void __launch_bounds__(TEAMS * 256, 1)
 k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restrict__ dirty,
          unsigned char* __restrict__ wire, uint64_t wire_cap, Ws ws, const Tables* __restrict__ tab)
@@ -1016,6 +1019,14 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
                 gw[j] = emin | ((32u - __clz(emax - emin)) << 8);
             }
 #endif
+            // Option ZEROS.  Unused memory: when all four groups have exponent 0 throughout (rare in live data)
+            // look at the words themselves; a warp whose 2 KiB are all zero marks its first entry.
+            if (ZEROS && (gw[0] | gw[1] | gw[2] | gw[3]) == 0u) {
+                uint32_t any = 0;
+#pragma unroll
+                for (int i = 0; i < 16; i++) any |= d[i];
+                if (!__any_sync(0xFFFFFFFFu, any != 0u)) gw[0] = kWarpAllZero;
+            }
             // one lane leaves the warp's results; the warp that arrives last turns the 32 widths
             // into offsets and publishes the tile's length
             uint32_t last = 0;
@@ -1036,10 +1047,12 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
                     if (lane >= (uint32_t)k) incl += o;
                 }
                 tc->wtab[slY][lane] = (wt & 0xFFFFu) | ((incl - wv) << 16);
+                // unused memory (every warp's first entry carries the mark): no payload
+                const bool zero_tile = ZEROS && __all_sync(0xFFFFFFFFu, (lane & 3u) != 0u || (wt & kWarpAllZero) != 0u);
                 if (lane == 31) {
-                    tc->ssum[slY] = incl;
+                    tc->ssum[slY] = zero_tile ? kSumZeroTile : incl;
                     tc->wsum[slY] = 0;
-                    publish_len(tYn, incl <= 253u ? 8256u + 32u * incl : kTile);
+                    publish_len(tYn, zero_tile ? 0u : incl <= 253u ? 8256u + 32u * incl : kTile);
                 }
             }
 #ifndef WM_AB_NOTMEM
@@ -1064,7 +1077,8 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
 #endif
             const uint32_t Ssum = tc->ssum[sl];
             const bool packs = Ssum <= 253u;
-            const uint32_t enc_len = packs ? 8256u + 32u * Ssum : kTile;
+            // (a tile of all-zero bytes, marked in ssum, is its table entry and nothing else)
+            const uint32_t enc_len = packs ? 8256u + 32u * Ssum : (ZEROS && Ssum == kSumZeroTile) ? 0u : kTile;
             unsigned char* const dst = payload + exclX;
             if (exclX + enc_len > room) {
                 trouble |= 1u;
@@ -1104,7 +1118,7 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
 #else
                 if (d[5] == 0x12345678u) stg_u8(dst + lane, d[1]);
 #endif
-            } else {
+            } else if (enc_len) {
                 unsigned char* q = dst + warp * 2048u + lane * 4u;
 #pragma unroll
                 for (int i = 0; i < 16; i++) st_stream_u32(q + i * 128, __funnelshift_r(d[i], d[i], 1));
@@ -1128,8 +1142,8 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
                 if (qX >= kQPresent) {
                     if (tXn < g.n_full_tiles) {
                         const uint32_t Ssum = tc->ssum[sl];
-                        entry = Ssum <= 253u ? 258u + Ssum : 512u;
-                        enc_len = 32u * entry;
+                        entry = Ssum <= 253u ? 258u + Ssum : (ZEROS && Ssum == kSumZeroTile) ? 1u : 512u;
+                        enc_len = entry == 1u ? 0u : 32u * entry;
                     } else {
                         entry = 0xFFFFu;
                         enc_len = tile_left(g, tXn);
@@ -1177,7 +1191,7 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
 __global__ void __launch_bounds__(1024)
 k_encode_finish(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restrict__ dirty,
                 uint32_t* __restrict__ crc_inout, unsigned char* __restrict__ wire, Ws ws,
-                const Tables* __restrict__ tab, const __grid_constant__ ChunkPowers cp)
+                const Tables* __restrict__ tab, const __grid_constant__ ChunkPowers cp, uint32_t zero_tiles)
 {
     __shared__ uint32_t sHT[1024];
     __shared__ uint32_t sT0[256];
@@ -1226,7 +1240,7 @@ k_encode_finish(const unsigned char* __restrict__ cache, Geo g, const uint8_t* _
     const uint32_t n_present = ld_volatile_u32(&ws.ctrl->n_present);
     uint32_t* h = reinterpret_cast<uint32_t*>(wire);
     h[0] = 0x31564D57u;                                  // "WMV1"
-    h[1] = 1u | ((dirty ? 1u : 0u) << 16);               // version, flags
+    h[1] = 1u | ((dirty ? 1u : 0u) << 16) | ((zero_tiles ? 2u : 0u) << 16);      // version, flags
     h[2] = (uint32_t)g.nbytes; h[3] = (uint32_t)(g.nbytes >> 32);
     h[4] = g.chunk_bytes; h[5] = kTile; h[6] = g.n_chunks; h[7] = n_present;
     h[8] = (uint32_t)total; h[9] = (uint32_t)(total >> 32);
@@ -1252,7 +1266,7 @@ __device__ __forceinline__ bool header_matches(const unsigned char* wire, uint64
     const unsigned long long nb = h[2] | ((unsigned long long)h[3] << 32);
     const unsigned long long pb = h[8] | ((unsigned long long)h[9] << 32);
     const unsigned long long wl = h[10] | ((unsigned long long)h[11] << 32);
-    return !(h[0] != 0x31564D57u || (h[1] & 0xFFFFu) != 1u || (h[1] >> 16) > 1u || nb != g.nbytes ||
+    return !(h[0] != 0x31564D57u || (h[1] & 0xFFFFu) != 1u || (h[1] >> 16) > 3u || nb != g.nbytes ||
              h[4] != g.chunk_bytes || h[5] != kTile || h[6] != g.n_chunks || wl != wire_len ||
              wire_len < g.meta_end || pb != wire_len - g.meta_end);
 }
@@ -1429,6 +1443,7 @@ k_decode_check(const unsigned char* __restrict__ wire, uint64_t wire_len, Geo g,
         return;
     }
     const unsigned char* dir = wire + 64;
+    const bool zero_ok = ((reinterpret_cast<const uint32_t*>(wire)[1] >> 17) & 1u) != 0u;   // the image declares the option
     if (blockIdx.x < meta_blocks) {
         const uint32_t team = threadIdx.x / kTeamThreads, tt = threadIdx.x % kTeamThreads;
         const uint32_t s = blockIdx.x * 4 + team;
@@ -1456,6 +1471,7 @@ k_decode_check(const unsigned char* __restrict__ wire, uint64_t wire_len, Geo g,
                     else {
                         l_any = true;
                         if (tl < kTile) { if (e != 0xFFFFu) l_ok = false; len = (uint32_t)tl; }
+                        else if (e == 1u && zero_ok) len = 0;       // a tile of zeros: no payload
                         else if (e >= 258u && e <= 512u) len = 32u * e;
                         else l_ok = false;
                     }
@@ -1766,6 +1782,10 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
                 }
 #endif
             }
+        } else if (e == 1u) {
+            // a tile of zeros: nothing was shipped; from here on it goes the way of a raw tile
+#pragma unroll
+            for (int i = 0; i < 16; i++) w[i] = 0u;
         }
         team_bar(team);                      // stage free; the slots the leader filled last step visible;
                                              // the previous tile's digest parts complete
@@ -1958,6 +1978,7 @@ struct DeviceState {
     cudaEvent_t ev[4][2] = {};   // optional timing of the four main kernels
 };
 static bool g_timing = false;
+static bool g_zero_tiles = false;   // wm_zero_tiles_enable
 
 struct MainKernelTimer {        // records events around a main kernel when timing is enabled
     const DeviceState* ds; int kind; cudaStream_t s;
@@ -1987,10 +2008,14 @@ static const DeviceState* device_state()
     if (cudaMemcpy(s.tables, &host, sizeof(Tables), cudaMemcpyHostToDevice) != cudaSuccess) return nullptr;
     if (cudaDeviceGetAttribute(&s.sm_count, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return nullptr;
     const int big = kDynSmem;
-    if (cudaFuncSetAttribute(k_encode<kTeams, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, big) != cudaSuccess) return nullptr;
-    if (cudaFuncSetAttribute(k_encode<kTeams, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, big) != cudaSuccess) return nullptr;
-    if (cudaFuncSetAttribute(k_encode<kTeams, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, big) != cudaSuccess) return nullptr;
-    if (cudaFuncSetAttribute(k_encode<kTeams, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, big) != cudaSuccess) return nullptr;
+    {
+        const void* enc[] = {(const void*)k_encode<kTeams, false, false, false>, (const void*)k_encode<kTeams, true, false, false>,
+                             (const void*)k_encode<kTeams, false, true, false>,  (const void*)k_encode<kTeams, true, true, false>,
+                             (const void*)k_encode<kTeams, false, false, true>,  (const void*)k_encode<kTeams, true, false, true>,
+                             (const void*)k_encode<kTeams, false, true, true>,   (const void*)k_encode<kTeams, true, true, true>};
+        for (const void* f : enc)
+            if (cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, big) != cudaSuccess) return nullptr;
+    }
     if (cudaFuncSetAttribute(k_decode<kTeamsPlain, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, big) != cudaSuccess) return nullptr;
     if (cudaFuncSetAttribute(k_decode<kTeamsPlain, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, big) != cudaSuccess) return nullptr;
     if (cudaFuncSetAttribute(k_tile_digests<kTeamsPlain>, cudaFuncAttributeMaxDynamicSharedMemorySize, big) != cudaSuccess) return nullptr;
@@ -2057,6 +2082,8 @@ uint64_t wm_workspace_bytes(uint64_t nbytes, uint32_t chunk_bytes)
 uint32_t wm_last_launch_count(void) { return g_launches; }
 
 void wm_timing_enable(int on) { g_timing = on != 0; }
+
+void wm_zero_tiles_enable(int on) { g_zero_tiles = on != 0; }
 
 int wm_timing_read_ms(int kind, float* ms)
 {
@@ -2208,16 +2235,21 @@ static wm_status encode_any(const void* cache, const wm_leaf* leaves, uint32_t n
     const uint32_t grid = need < (uint32_t)ds->sm_count ? need : (uint32_t)ds->sm_count;
     {
         MainKernelTimer timer(ds, 2, s);
-        if (leaves) {
-            if (dirty) launch_after(k_encode<kTeams, true, true>, grid, kTeams * 256, kDynSmem, s, c, g, dirty, w, wire_cap, ws, ds->tables);
-            else launch_after(k_encode<kTeams, false, true>, grid, kTeams * 256, kDynSmem, s, c, g, dirty, w, wire_cap, ws, ds->tables);
-        } else {
-            if (dirty) launch_after(k_encode<kTeams, true, false>, grid, kTeams * 256, kDynSmem, s, c, g, dirty, w, wire_cap, ws, ds->tables);
-            else launch_after(k_encode<kTeams, false, false>, grid, kTeams * 256, kDynSmem, s, c, g, dirty, w, wire_cap, ws, ds->tables);
+        const int variant = (dirty ? 1 : 0) | (leaves ? 2 : 0) | (g_zero_tiles ? 4 : 0);
+        auto go = [&](auto kernel) { launch_after(kernel, grid, kTeams * 256, kDynSmem, s, c, g, dirty, w, wire_cap, ws, ds->tables); };
+        switch (variant) {
+            case 0: go(k_encode<kTeams, false, false, false>); break;
+            case 1: go(k_encode<kTeams, true, false, false>); break;
+            case 2: go(k_encode<kTeams, false, true, false>); break;
+            case 3: go(k_encode<kTeams, true, true, false>); break;
+            case 4: go(k_encode<kTeams, false, false, true>); break;
+            case 5: go(k_encode<kTeams, true, false, true>); break;
+            case 6: go(k_encode<kTeams, false, true, true>); break;
+            default: go(k_encode<kTeams, true, true, true>); break;
         }
     }
     launch_after(k_encode_finish, (g.n_chunks + g.finish_cb - 1) / g.finish_cb, 1024, 0, s, c, g, dirty, crc_inout, w, ws, ds->tables,
-                 chunk_powers(g));
+                 chunk_powers(g), g_zero_tiles ? 1u : 0u);
     launch_after(k_meta_crc, (g.n_meta_slices + 3) / 4, 1024, kDynSmem, s, w, g, ws, ds->tables, result);
     g_launches = leaves ? 5 : 4;
     return launch_status();

@@ -277,3 +277,47 @@ def test_repeatable_and_grid_independent_bytes(G):
     w1, _, r1, _ = g.encode(a)
     w2, _, r2, _ = g.encode(a)
     assert r1.wire_len == r2.wire_len and np.array_equal(w1[: r1.wire_len], w2[: r2.wire_len])
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("layout", ["some", "all", "first_of_chunk", "masked"])
+def test_zero_tiles_match_the_oracle(layout):
+    """Tiles of all-zero bytes (unused allocation) become table entries without payload."""
+    from gpu_util import Gpu, same_result, to_dev
+    rng = np.random.default_rng(11)
+    chunk = 4 * TILE
+    nt = 13
+    n = nt * TILE + 700
+    a = (rng.normal(size=(n + 1) // 2).astype(np.float32).view(np.uint32) >> 16).astype("<u2").view(np.uint8)[:n].copy()
+    zero = {"some": [1, 2, 6, 11], "all": list(range(nt)), "first_of_chunk": [0, 4, 8, 12], "masked": [1, 5, 6, 7]}[layout]
+    for t in zero:
+        a[t * TILE:(t + 1) * TILE] = 0
+    if layout == "all":
+        a[nt * TILE:] = 0
+    a[3 * TILE + 10:3 * TILE + 12] = (0, 0x80) if layout != "all" else (0, 0)      # a minus zero stays data
+    nc = (n + chunk - 1) // chunk
+    dirty = (np.arange(nc) % 2 == 1).astype(np.uint8) if layout == "masked" else None
+    crc_in = np.full(nc, 0x12345678, dtype=np.uint32)
+    from paper_2607_10389_b200 import binding as wm
+    want_wire, want_crc, want = oracle.encode(a, chunk, dirty=dirty, crc_in=crc_in, zero_tiles=True)
+    plain_wire, _, plain = oracle.encode(a, chunk, dirty=dirty, crc_in=crc_in)
+    g = Gpu(n, chunk)
+    # without the option the zeros pack like any constant tile ...
+    wire0, _, r0, _ = g.encode(to_dev(a), dirty=dirty, crc_in=crc_in)
+    assert same_result(r0, plain) and np.array_equal(wire0[: r0.wire_len], plain_wire)
+    # ... with it they are table entries
+    wm.zero_tiles_enable(True)
+    try:
+        wire, crc, r, wire_dev = g.encode(to_dev(a), dirty=dirty, crc_in=crc_in)
+    finally:
+        wm.zero_tiles_enable(False)
+    assert same_result(r, want) and r.wire_len < r0.wire_len
+    assert np.array_equal(wire[: r.wire_len], want_wire) and np.array_equal(crc, want_crc)
+    old = np.full(n, 0x5A, dtype=np.uint8)
+    if dirty is not None:
+        for c in np.nonzero(dirty == 0)[0]:
+            old[c * chunk:(c + 1) * chunk] = a[c * chunk:(c + 1) * chunk]
+    want_out, want_dcrc, want_r = oracle.decode_verify(want_wire, n, chunk, dst=old, dst_crc=want_crc)
+    out, dcrc, rd = g.decode(wire_dev, r.wire_len, dst=old, dst_crc=want_crc)
+    assert same_result(rd, want_r) and rd.ok
+    assert np.array_equal(out, want_out) and np.array_equal(out, a) and np.array_equal(dcrc, want_dcrc)

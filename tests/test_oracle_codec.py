@@ -393,7 +393,7 @@ def test_zero_tiles_have_entry_one_and_no_payload():
     a, b = _rand_tile(1), _rand_tile(2)
     z = np.zeros(TILE, dtype=np.uint8)
     cache = np.concatenate([a, z, z, b])
-    wire, crc, res = oracle.encode(cache, 4 * TILE)
+    wire, crc, res = oracle.encode(cache, 4 * TILE, zero_tiles=True)
     wa, _, ra = oracle.encode(a, TILE)
     wb, _, rb = oracle.encode(b, TILE)
     ea, eb = wa[96:ra.wire_len], wb[96:rb.wire_len]
@@ -411,7 +411,7 @@ def test_zero_tiles_have_entry_one_and_no_payload():
 def test_all_zero_cache_is_metadata_plus_its_ragged_tail():
     n = 3 * TILE + 100
     cache = np.zeros(n, dtype=np.uint8)
-    wire, crc, res = oracle.encode(cache, 2 * TILE)
+    wire, crc, res = oracle.encode(cache, 2 * TILE, zero_tiles=True)
     assert _tab(wire, 2, 4).tolist() == [1, 1, 1, 0xFFFF]
     assert res.payload_bytes == 100 and res.wire_len == oracle.meta_end(n, 2 * TILE) + 100
     assert [d[1] for d in _dir(wire, 2)] == [0, 100]
@@ -424,7 +424,7 @@ def test_only_all_zero_bytes_make_a_zero_tile(word):
     # minus zero, the smallest denormal and the smallest normal exponent are data, not emptiness
     tile = np.zeros(8192, dtype="<u2")
     tile[4711] = word
-    wire, _, res = oracle.encode(tile.view(np.uint8), TILE)
+    wire, _, res = oracle.encode(tile.view(np.uint8), TILE, zero_tiles=True)
     assert _tab(wire, 1, 1)[0] >= 258 and res.payload_bytes >= 8256
     out, _, r = oracle.decode_verify(wire, TILE, TILE)
     assert r.status == 0 and np.array_equal(out, tile.view(np.uint8))
@@ -442,7 +442,7 @@ def test_zero_entry_is_checked_like_any_other():
     a = _rand_tile(3)
     cache = np.concatenate([a, np.zeros(TILE, np.uint8), a[:500]])
     n, chunk = cache.size, 4 * TILE
-    wire, crc, res = oracle.encode(cache, chunk)
+    wire, crc, res = oracle.encode(cache, chunk, zero_tiles=True)
     assert _tab(wire, 1, 3).tolist()[1:] == [1, 0xFFFF]
     tab_off = 64 + 16
     # a ZERO entry where a ragged tile belongs: the structure check refuses it
@@ -461,3 +461,22 @@ def test_zero_entry_is_checked_like_any_other():
     # without fixing the metadata CRC any of these stops at the metadata check
     w = wire.copy(); w[tab_off + 2] ^= 1
     assert oracle.decode_verify(w, n, chunk)[2].status_name == "ERR_META_CRC"
+
+
+def test_zero_tiles_are_an_option_recorded_in_the_header():
+    cache = np.concatenate([_rand_tile(5), np.zeros(TILE, np.uint8)])
+    plain, _, rp = oracle.encode(cache, 2 * TILE)
+    opt, _, ro = oracle.encode(cache, 2 * TILE, zero_tiles=True)
+    assert _hdr(plain)["flags"] == 0 and _hdr(opt)["flags"] == 2
+    assert _tab(plain, 1, 2).tolist()[1] == 258 and _tab(opt, 1, 2).tolist()[1] == 1     # zeros pack to 8256 bytes without it
+    assert rp.wire_len - ro.wire_len == 8256
+    for w in (plain, opt):
+        out, _, r = oracle.decode_verify(w, cache.size, 2 * TILE)
+        assert r.status == 0 and np.array_equal(out, cache)
+    # entry 1 in an image that does not declare the option is a structure error
+    w = opt.copy(); w[6] = 0
+    assert oracle.decode_verify(_refresh_meta_crc(w, cache.size, 2 * TILE), cache.size, 2 * TILE)[2].status_name == "ERR_STRUCT"
+    # with a dirty mask both flag bits are set
+    two = np.concatenate([cache, cache])
+    m, _, _ = oracle.encode(two, 2 * TILE, dirty=np.array([1, 0], np.uint8), crc_in=np.zeros(2, np.uint32), zero_tiles=True)
+    assert _hdr(m)["flags"] == 3
