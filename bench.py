@@ -172,6 +172,11 @@ def make_workload(name, device):
     from paper_2607_10389_b200 import inputs
     cfg = inputs.CONFIGS[name]
     cur = inputs.make_cache(cfg, device)
+    if cfg.kind == "llm":
+        # previous snapshot: the same window before the last 16 tokens were appended
+        prev, mask = inputs.before_append(cur, cfg, 16)
+        torch.cuda.synchronize()
+        return cfg, cur, prev, int(mask.sum())
     # previous snapshot: the same cache before a generation step rewrote 75 % of its chunks
     nc = (cfg.nbytes + cfg.chunk_bytes - 1) // cfg.chunk_bytes
     mask = inputs.step_pattern(nc, 30, 0.75, seed=cfg.seed + 100)
@@ -363,6 +368,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-loop", action="store_true", help="skip the pre-copy step loop")
+    ap.add_argument("--zero-tiles", action="store_true", help="encoder option: all-zero tiles as table entries")
     ap.add_argument("--profile", action="store_true",
                     help="profiler capture mode: round-trip check, warm-up and timed steps only")
     args = ap.parse_args()
@@ -389,6 +395,7 @@ def main():
     group = Replicas("nccl", dev)
     barrier, max_over_ranks = group.barrier, group.max_over_ranks
 
+    wm.zero_tiles_enable(args.zero_tiles)
     cfg, cur, prev, n_rewritten = make_workload(args.workload, dev)
     N, C = cfg.nbytes, cfg.chunk_bytes
     nc = wm.num_chunks(N, C)
@@ -584,7 +591,8 @@ def main():
             "dtype": "u8", "data": "synthetic",
             "config": {"workload": args.workload, "nbytes": N, "chunk_bytes": C, "shape": list(cfg.shape),
                        "wire_bytes": W, "ratio": W / N, "dirty_chunks": n_rewritten, "n_chunks": nc,
-                       "l2": "inputs larger than L2 (no flush needed)", "parallelism": "replicas only"},
+                       "l2": "inputs larger than L2 (no flush needed)", "parallelism": "replicas only",
+                       "zero_tiles": bool(args.zero_tiles)},
             "calls": per_call, "roofline": roofline, "precopy_loop": loop, "leaf_mode": leaf, "cpu_baseline": base, "e2e": e2e,
             "gpu_launches": gpu_launches, "clocks": clocks,
         }

@@ -28,14 +28,15 @@ class CacheConfig:
     nbytes: int
     chunk_bytes: int
     seed: int
-    kind: str             # "gauss" | "kv" | "bytes"
+    kind: str             # "gauss" | "kv" | "bytes" | "llm"
+    fill: float = 1.0     # "llm": fraction of the token window that holds data (the rest is zero)
 
 
-def _kv(name, shape, chunk, seed, kind):
+def _kv(name, shape, chunk, seed, kind, fill=1.0):
     n = 2
     for s in shape:
         n *= s
-    return CacheConfig(name, tuple(shape), n, chunk, seed, kind)
+    return CacheConfig(name, tuple(shape), n, chunk, seed, kind, fill)
 
 
 CONFIGS = {
@@ -51,6 +52,11 @@ CONFIGS = {
     "long8g": _kv("long8g", (32, 2, 8, 65536, 128), 4 << 20, 4, "kv"),
     # engine-like cache small enough for a profiler capture, still larger than the 126 MB L2
     "engine_256m": _kv("engine_256m", (5, 2, 16, 6400, 128), 1 << 20, 2, "kv"),
+    # append-only text-model cache (Section 3.3: 24 layers, a window that fills from 0.249 towards
+    # 0.727, a step appends tokens and rewrites nothing): allocated for the whole window, zero
+    # beyond the tokens written so far
+    "llm_append": _kv("llm_append", (24, 2, 8, 16384, 128), 64 * 1024, 6, "llm", 0.249),
+    "llm_append_small": _kv("llm_append_small", (2, 2, 2, 2048, 128), 64 * 1024, 6, "llm", 0.249),
     # reduced engine-like cache for tests that also run the CPU oracle on everything
     "engine_small": _kv("engine_small", (3, 2, 4, 680, 128), 1 << 20, 2, "kv"),
 }
@@ -75,6 +81,16 @@ def make_cache(cfg: CacheConfig, device="cpu") -> torch.Tensor:
         return out
     layers, two, heads, tokens, dim = cfg.shape
     assert two == 2
+    if cfg.kind == "llm":
+        out = torch.zeros(cfg.shape, dtype=torch.bfloat16, device=device)
+        filled = filled_tokens(cfg)
+        for layer in range(layers):
+            k = torch.randn((heads, filled, dim), generator=g, device=device)
+            v = torch.randn((heads, filled, dim), generator=g, device=device)
+            scale = torch.exp(0.5 * torch.randn((heads, 1, dim), generator=g, device=device))
+            out[layer, 0, :, :filled] = (k * scale).to(torch.bfloat16)
+            out[layer, 1, :, :filled] = v.to(torch.bfloat16)
+        return out.view(-1).view(torch.uint8)
     out = torch.empty(cfg.shape, dtype=torch.bfloat16, device=device)
     for layer in range(layers):
         k = torch.randn((heads, tokens, dim), generator=g, device=device)
@@ -149,3 +165,27 @@ def apply_step(cache_u8: torch.Tensor, chunk_bytes: int, mask: torch.Tensor, see
         lo, hi = idx[i] * chunk_bytes, min((idx[j] + 1) * chunk_bytes, n)
         cache_u8[lo:hi] = fresh_like(cache_u8, seed * 1000003 + idx[i], lo, hi + ((hi - lo) & 1))[: hi - lo]
         i = j + 1
+
+
+def filled_tokens(cfg: CacheConfig) -> int:
+    """Tokens of an "llm" cache's window that hold data."""
+    return int(round(cfg.fill * cfg.shape[3]))
+
+
+def before_append(cache_u8: torch.Tensor, cfg: CacheConfig, appended: int):
+    """The previous snapshot of an append-only cache: the same bytes without the last `appended`
+    tokens of every (layer, key/value, head) row block.  Returns (prev, dirty u8[n_chunks]): the
+    chunks that hold those tokens are the only ones that differ."""
+    layers, two, heads, tokens, dim = cfg.shape
+    filled = filled_tokens(cfg)
+    prev = cache_u8.clone()
+    view = prev.view(torch.bfloat16).view(cfg.shape)
+    view[:, :, :, filled - appended:filled] = 0
+    nc = (cfg.nbytes + cfg.chunk_bytes - 1) // cfg.chunk_bytes
+    mask = torch.zeros(nc, dtype=torch.uint8)
+    row = dim * 2
+    for blk in range(layers * two * heads):
+        lo = (blk * tokens + filled - appended) * row
+        hi = (blk * tokens + filled) * row
+        mask[lo // cfg.chunk_bytes:(hi - 1) // cfg.chunk_bytes + 1] = 1
+    return prev, mask

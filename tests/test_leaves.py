@@ -137,3 +137,53 @@ def test_leaf_table_that_breaks_the_rules_is_rejected():
         wm.wm_decode_verify_leaves(wire, r.wire_len, dt, nbytes, chunk, dcrc, ws, res)
         assert wm.read_result(res).status_name == "ERR_ARG"
         assert all((x == 0x33).all() for x in dst) and not dcrc.any()
+
+
+def test_append_only_workload_dirties_only_the_chunks_that_hold_the_new_tokens():
+    from paper_2607_10389_b200 import inputs
+    cfg = inputs.CONFIGS["llm_append_small"]
+    a = inputs.make_cache(cfg, "cpu")
+    prev, mask = inputs.before_append(a, cfg, 16)
+    d, idx = oracle.dirty_diff(a.numpy(), prev.numpy(), cfg.chunk_bytes)
+    assert np.array_equal(d, mask.numpy()) and 0 < int(d.sum()) <= d.size // 8
+    plain = oracle.encode(a.numpy(), cfg.chunk_bytes)[2]
+    opt = oracle.encode(a.numpy(), cfg.chunk_bytes, zero_tiles=True)[2]
+    # three quarters of the window are unused: without the option they still cost half their size
+    assert 0.5 < plain.wire_len / cfg.nbytes < 0.6 and 0.15 < opt.wire_len / cfg.nbytes < 0.25
+
+
+@gpu
+def test_append_only_step_with_zero_tiles_matches_the_oracle():
+    import torch
+    from paper_2607_10389_b200 import binding as wm
+    from paper_2607_10389_b200 import inputs
+    cfg = inputs.CONFIGS["llm_append_small"]
+    cur = inputs.make_cache(cfg, "cuda")
+    prev, mask = inputs.before_append(cur, cfg, 16)
+    n, chunk = cfg.nbytes, cfg.chunk_bytes
+    nc = wm.num_chunks(n, chunk)
+    ws, res = wm.new_workspace(n, chunk), wm.new_result()
+    cap = wm.wire_bound(n, chunk)
+    dirty = torch.zeros(nc, dtype=torch.uint8, device="cuda")
+    nd = torch.zeros(1, dtype=torch.int32, device="cuda")
+    wm.wm_dirty_diff(cur, prev, chunk, dirty, None, nd, ws)
+    assert torch.equal(dirty.cpu(), mask)
+    crc_prev = torch.from_numpy(oracle.checksum(prev.cpu().numpy(), chunk).view(np.int32).copy()).cuda()
+    wm.zero_tiles_enable(True)
+    try:
+        for d_np, d_dev, crc0 in ((None, None, torch.zeros_like(crc_prev)), (mask.numpy(), dirty, crc_prev)):
+            want_wire, want_crc, want = oracle.encode(cur.cpu().numpy(), chunk, dirty=d_np,
+                                                      crc_in=crc0.cpu().numpy().view(np.uint32), zero_tiles=True)
+            wire = torch.zeros(cap, dtype=torch.uint8, device="cuda")
+            crc = crc0.clone()
+            wm.wm_encode(cur, chunk, d_dev, crc, wire, ws, res)
+            r = wm.read_result(res)
+            assert (r.status, r.wire_len, r.n_present, r.cache_crc) == (want.status, want.wire_len, want.n_present, want.cache_crc)
+            assert np.array_equal(wire[: r.wire_len].cpu().numpy(), want_wire)
+            assert np.array_equal(crc.cpu().numpy().view(np.uint32), want_crc)
+            dst = prev.clone() if d_np is not None else torch.full_like(cur, 0x77)
+            dcrc = crc_prev.clone()
+            wm.wm_decode_verify(wire, r.wire_len, dst, chunk, dcrc, ws, res)
+            assert wm.read_result(res).ok and torch.equal(dst, cur)
+    finally:
+        wm.zero_tiles_enable(False)
