@@ -1135,25 +1135,26 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
             }
         }
 
-        if (leader) {
-            // what is left to note about X: table entry, digest, where its chunk starts, the total
-            if (is_tile(qX)) {
-                uint32_t entry = 0, enc_len = 0;
-                if (qX >= kQPresent) {
-                    if (tXn < g.n_full_tiles) {
-                        const uint32_t Ssum = tc->ssum[sl];
-                        entry = Ssum <= 253u ? 258u + Ssum : (ZEROS && Ssum == kSumZeroTile) ? 1u : 512u;
-                        enc_len = entry == 1u ? 0u : 32u * entry;
-                    } else {
-                        entry = 0xFFFFu;
-                        enc_len = tile_left(g, tXn);
-                    }
-                    ws.dig[tXn] = xor8(tc->wdig[sl]);
+        // What is left to note about X (table entry, digest, where its chunk starts, the total) is
+        // done by the second warp's first lane: the leader's warp is the one the team waits for.
+        if (tt == 32u && is_tile(qX)) {
+            uint32_t entry = 0, enc_len = 0;
+            if (qX >= kQPresent) {
+                if (tXn < g.n_full_tiles) {
+                    const uint32_t Ssum = tc->ssum[sl];
+                    entry = Ssum <= 253u ? 258u + Ssum : (ZEROS && Ssum == kSumZeroTile) ? 1u : 512u;
+                    enc_len = (ZEROS && entry == 1u) ? 0u : 32u * entry;
+                } else {
+                    entry = 0xFFFFu;
+                    enc_len = tile_left(g, tXn);
                 }
-                tile_tab[tXn] = (uint16_t)entry;
-                if (qX & kQFirst) *reinterpret_cast<unsigned long long*>(dir + 16ull * chunk_of(g, tXn)) = exclX;
-                if (tXn + 1 == g.n_tiles) ws.ctrl->payload_total = exclX + enc_len;
+                ws.dig[tXn] = xor8(tc->wdig[sl]);
             }
+            tile_tab[tXn] = (uint16_t)entry;
+            if (qX & kQFirst) *reinterpret_cast<unsigned long long*>(dir + 16ull * chunk_of(g, tXn)) = exclX;
+            if (tXn + 1 == g.n_tiles) ws.ctrl->payload_total = exclX + enc_len;
+        }
+        if (leader) {
 #ifdef WM_DEBUG_COUNTERS
             atomicAdd(&ws.ctrl->pad[(pv >> 30) == 2u ? 3 : 2], 1u);
 #endif
