@@ -1716,12 +1716,12 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
     team_bar(team);
     uint32_t phase = 0;
     uint32_t trouble = 0;              // sticky: a copy never arrived
-    uint32_t t_done = kNone;           // leader: tile whose digest parts wait in wdig[(it - 1) & 1]
+    uint32_t t_done = kNone;           // tile whose digest parts wait in wdig[(it - 1) & 1]
     for (uint32_t it = 0;; it++) {
         const uint32_t t = tc->slot[it & 3u].t;
         if (t >= g.n_tiles) {
             team_bar(team);
-            if (leader && t_done != kNone) ws.dig[t_done] = xor8(tc->wdig[(it & 1u) ^ 1u]);
+            if (tt == 32u && t_done != kNone) ws.dig[t_done] = xor8(tc->wdig[(it & 1u) ^ 1u]);
             break;
         }
         const uint32_t ew = tc->slot[it & 3u].entry;
@@ -1794,9 +1794,10 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
         // ahead and the ticket of the tile three ahead (answers taken at the end of the step).
         uint32_t l_e = 0, l_rel = 0, l_tk = kNone;
         unsigned long long l_po = 0;
+        // (spread over three warps: the team waits for whichever warp has the most to do)
+        if (tt == 64u) start_copy(tc->slot[(it + 1u) & 3u]);
+        if (tt == 32u && t_done != kNone) ws.dig[t_done] = xor8(tc->wdig[p ^ 1u]);
         if (leader) {
-            start_copy(tc->slot[(it + 1u) & 3u]);
-            if (t_done != kNone) ws.dig[t_done] = xor8(tc->wdig[p ^ 1u]);
             if (t_look < g.n_tiles) {
                 l_e = tab16[t_look];
                 l_rel = __ldcg(ws.rel + t_look);
@@ -1870,8 +1871,8 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
                 have_digest = true;
             }
         }
+        t_done = have_digest ? t : kNone;
         if (leader) {
-            t_done = have_digest ? t : kNone;
             if (t_look < g.n_tiles) {
                 DecSlot* s2 = &tc->slot[(it + 2u) & 3u];
                 s2->entry = l_e | (first_in_chunk(g, t_look) ? 0x10000u : 0u);
