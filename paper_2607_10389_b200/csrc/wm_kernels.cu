@@ -977,14 +977,16 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
         team_bar(team);                   // stage free; what the leader left at the end of the last step is visible
         const uint32_t qN = tc->next[par ^ 1u];
         const unsigned long long exclX = tc->excl[par ^ 1u];
-        // The leader starts the copy of the next tile (it has the whole step to arrive) and two
-        // round trips to L2 whose answers are used at the end of the step: the ticket of the
-        // tile to measure two steps on, and the offset of the tile to pack in the next step.
+        // The team's single-lane chores are spread over its warps, because the team waits for
+        // whichever warp has the most to do.  Warp 2 starts the copy of the next tile (it has the
+        // whole step to arrive).  Two round trips to L2 are started now and used at the end of the
+        // step: the ticket of the tile to measure two steps on (warp 0, the leader) and the offset
+        // of the tile to pack in the next step (warp 3).  Warp 1 notes what is left about X.
         uint32_t pv = 0, tk = 0xFFFFFFFFu;
         const unsigned char* pA = nullptr;
+        if (tt == 64u) start_copy(qN, LEAVES ? tc->nptr[par ^ 1u] : tile_src(qN & kQTile));
+        if (tt == 96u && is_tile(qV)) pv = ld_relaxed_u32(ws.lbk + (qV & kQTile));
         if (leader) {
-            start_copy(qN, LEAVES ? tc->nptr[par ^ 1u] : tile_src(qN & kQTile));
-            if (is_tile(qV)) pv = ld_relaxed_u32(ws.lbk + (qV & kQTile));
             if (claiming) tk = next_ticket(ws.ctrl);
             if (LEAVES && is_tile(qA)) pA = tile_src(qA & kQTile);
         }
@@ -1155,15 +1157,8 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
             if (tXn + 1 == g.n_tiles) ws.ctrl->payload_total = exclX + enc_len;
         }
         if (leader) {
-#ifdef WM_DEBUG_COUNTERS
-            atomicAdd(&ws.ctrl->pad[(pv >> 30) == 2u ? 3 : 2], 1u);
-#endif
-            unsigned long long e = 0;
-            if (is_tile(qV))
-                e = (pv >> 30) == 2u ? (unsigned long long)(pv & kValMask) * kUnit : wait_prefix(ws.lbk, qV & kQTile, ws.ctrl);
             uint32_t qn2 = kQNone;
             if (claiming) { qn2 = describe_tile<MASKED>(g, dirty, tk); claiming = is_tile(qn2); }
-            tc->excl[par] = e;
             if (LEAVES) {              // hand over the tile whose address arrived during this step
                 tc->next[par] = qA;
                 tc->nptr[par] = pA;
@@ -1171,6 +1166,15 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
             } else {
                 tc->next[par] = qn2;
             }
+        }
+        if (tt == 96u) {
+#ifdef WM_DEBUG_COUNTERS
+            atomicAdd(&ws.ctrl->pad[(pv >> 30) == 2u ? 3 : 2], 1u);
+#endif
+            unsigned long long e = 0;
+            if (is_tile(qV))
+                e = (pv >> 30) == 2u ? (unsigned long long)(pv & kValMask) * kUnit : wait_prefix(ws.lbk, qV & kQTile, ws.ctrl);
+            tc->excl[par] = e;
         }
         qX = qV; qV = qW; qW = qY; qY = qN;
         sl = (sl + 1u) & 7u;
