@@ -1086,7 +1086,7 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
                 trouble |= 1u;
             } else if (packs) {
 #ifndef WM_AB_NOPACK
-                if (warp == 0) {
+                if (warp == 5) {           // (any one warp: not one that has a single-lane chore)
                     const uint32_t wt = tc->wtab[sl][lane];
                     stg_u16(dst + 2 * lane, desc_of(wt & 0xFFu, (wt >> 8) & 15u));
                 }
@@ -1137,9 +1137,11 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
             }
         }
 
-        // What is left to note about X (table entry, digest, where its chunk starts, the total) is
-        // done by the second warp's first lane: the leader's warp is the one the team waits for.
-        if (tt == 32u && is_tile(qX)) {
+        // What is left to note about X is done by two other warps' first lanes (the leader's
+        // warp is the one the team waits for): the digest by warp 1; the table entry, where its
+        // chunk starts and the total by warp 4.
+        if (tt == 32u && qX >= kQPresent && is_tile(qX)) ws.dig[tXn] = xor8(tc->wdig[sl]);
+        if (tt == 128u && is_tile(qX)) {
             uint32_t entry = 0, enc_len = 0;
             if (qX >= kQPresent) {
                 if (tXn < g.n_full_tiles) {
@@ -1150,7 +1152,6 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
                     entry = 0xFFFFu;
                     enc_len = tile_left(g, tXn);
                 }
-                ws.dig[tXn] = xor8(tc->wdig[sl]);
             }
             tile_tab[tXn] = (uint16_t)entry;
             if (qX & kQFirst) *reinterpret_cast<unsigned long long*>(dir + 16ull * chunk_of(g, tXn)) = exclX;
