@@ -1709,13 +1709,11 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
         if (sl.t < g.n_tiles && e >= 258u && e <= 512u) bulk_load(stage, payload + sl.src, 32u * e, &tc->mbar, 0);
     };
 
-    uint32_t t_look = kNone;           // leader: the tile whose look-ups are under way in this step
     if (leader) {
         mbar_init(&tc->mbar, 1);
         lookup(atomicAdd(&ws.ctrl->ticket, 1u), &tc->slot[0]);
         lookup(atomicAdd(&ws.ctrl->ticket, 1u), &tc->slot[1]);
-        t_look = atomicAdd(&ws.ctrl->ticket, 1u);
-        tc->slot[2].t = t_look;
+        tc->slot[2].t = atomicAdd(&ws.ctrl->ticket, 1u);      // its look-ups happen in the first step
         start_copy(tc->slot[0]);
     }
     team_bar(team);
@@ -1802,13 +1800,18 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
         // (spread over three warps: the team waits for whichever warp has the most to do)
         if (tt == 64u) start_copy(tc->slot[(it + 1u) & 3u]);
         if (tt == 32u && t_done != kNone) ws.dig[t_done] = xor8(tc->wdig[p ^ 1u]);
-        if (leader) {
+        uint32_t t_look = kNone;           // warps 0 and 3: the tile claimed a step ago (two tiles ahead)
+        if (leader) {                      // its table entry and offsets
+            t_look = tc->slot[(it + 2u) & 3u].t;
             if (t_look < g.n_tiles) {
                 l_e = tab16[t_look];
                 l_rel = __ldcg(ws.rel + t_look);
                 l_po = *reinterpret_cast<const unsigned long long*>(dir + 16ull * chunk_of(g, t_look));
-                l_tk = atomicAdd(&ws.ctrl->ticket, 1u);
             }
+        }
+        if (tt == 96u) {                   // the ticket of the tile three ahead
+            t_look = tc->slot[(it + 2u) & 3u].t;
+            if (t_look < g.n_tiles) l_tk = atomicAdd(&ws.ctrl->ticket, 1u);
         }
 
         // ---- phase 2: unpack, store, checksum
@@ -1877,17 +1880,12 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
             }
         }
         t_done = have_digest ? t : kNone;
-        if (leader) {
-            if (t_look < g.n_tiles) {
-                DecSlot* s2 = &tc->slot[(it + 2u) & 3u];
-                s2->entry = l_e | (first_in_chunk(g, t_look) ? 0x10000u : 0u);
-                s2->src = l_po + l_rel;
-                tc->slot[(it + 3u) & 3u].t = l_tk;
-            } else {
-                tc->slot[(it + 3u) & 3u].t = kNone;
-            }
-            t_look = l_tk;
+        if (leader && t_look < g.n_tiles) {
+            DecSlot* s2 = &tc->slot[(it + 2u) & 3u];
+            s2->entry = l_e | (first_in_chunk(g, t_look) ? 0x10000u : 0u);
+            s2->src = l_po + l_rel;
         }
+        if (tt == 96u) tc->slot[(it + 3u) & 3u].t = l_tk;      // (none once the tickets have run out)
     }
     if (trouble && lane == 0) atomicOr(&ws.ctrl->err, 2u);
 }
