@@ -756,7 +756,7 @@ __device__ __forceinline__ uint32_t desc_of(uint32_t base, uint32_t w)
 }
 
 struct EncTeamCtl {
-    uint32_t wtab[8][32];   // per group: base | w << 8 | (sum of the widths before it) << 16 (a ring of
+    uint32_t wtab[8][32];   // per group: base | w << 8 (| the all-zero mark on a warp's first entry) (a ring of
                             // slots: one per tile in flight and spares, so that a slot is rewritten
                             // long after its last read)
     uint32_t wdig[8][8];    // per warp: its contribution to the tile digest
@@ -1040,21 +1040,16 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
             }
             if (__shfl_sync(0xFFFFFFFFu, last, 0)) {
                 __threadfence_block();
+                // (kept short: this warp is the one the team's length waits for; the groups'
+                // places inside the tile are worked out by each warp when it packs)
                 const uint32_t wt = *reinterpret_cast<volatile uint32_t*>(&tc->wtab[slY][lane]);
-                const uint32_t wv = (wt >> 8) & 15u;
-                uint32_t incl = wv;
-#pragma unroll
-                for (int k = 1; k < 32; k <<= 1) {
-                    const uint32_t o = __shfl_up_sync(0xFFFFFFFFu, incl, k);
-                    if (lane >= (uint32_t)k) incl += o;
-                }
-                tc->wtab[slY][lane] = (wt & 0xFFFFu) | ((incl - wv) << 16);
+                const uint32_t total = __reduce_add_sync(0xFFFFFFFFu, (wt >> 8) & 15u);
                 // unused memory (every warp's first entry carries the mark): no payload
                 const bool zero_tile = ZEROS && __all_sync(0xFFFFFFFFu, (lane & 3u) != 0u || (wt & kWarpAllZero) != 0u);
-                if (lane == 31) {
-                    tc->ssum[slY] = zero_tile ? kSumZeroTile : incl;
+                if (lane == 0) {
+                    tc->ssum[slY] = zero_tile ? kSumZeroTile : total;
                     tc->wsum[slY] = 0;
-                    publish_len(tYn, zero_tile ? 0u : incl <= 253u ? 8256u + 32u * incl : kTile);
+                    publish_len(tYn, zero_tile ? 0u : total <= 253u ? 8256u + 32u * total : kTile);
                 }
             }
 #ifndef WM_AB_NOTMEM
@@ -1092,6 +1087,9 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
                 }
                 unsigned char* const sm_dst = dst + sm_off;
                 unsigned char* const pl_dst = dst + 8256;
+                // widths of all 32 groups (one per lane): 32-byte units before this warp's first group
+                const uint32_t wall = (tc->wtab[sl][lane] >> 8) & 15u;
+                uint32_t before = __reduce_add_sync(0xFFFFFFFFu, lane < 4u * warp ? wall : 0u);
                 const uint4 g4 = *reinterpret_cast<const uint4*>(&tc->wtab[sl][4 * warp]);
                 const uint32_t gq[4] = {g4.x, g4.y, g4.z, g4.w};
 #pragma unroll
@@ -1104,7 +1102,8 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
                     const uint32_t ya = __byte_perm(sa, sa, 0x2301), yb = __byte_perm(sb, sb, 0x2301);
                     stg_v2(sm_dst + 256 * j, (sa & 0xFEFEFEFEu) | (ya & 0x01010101u), (sb & 0xFEFEFEFEu) | (yb & 0x01010101u));
                     const uint32_t e4a = __byte_perm(d[4 * j], d[4 * j + 1], 0x7531), e4b = __byte_perm(d[4 * j + 2], d[4 * j + 3], 0x7531);
-                    unsigned char* rec = pl_dst + 32u * (wtg >> 16);
+                    unsigned char* rec = pl_dst + 32u * before;
+                    before += wd;
                     if (wd == 4u) pack_group_planes<4>(e4a, e4b, base, rec, lane);      // by far the most frequent width
                     else switch (wd) {     // uniform across the warp
                         case 1: pack_group_planes<1>(e4a, e4b, base, rec, lane); break;
