@@ -371,9 +371,13 @@ k_tile_digests(const unsigned char* __restrict__ cache, Geo g, Ws ws, const Tabl
     };
 
     uint64_t t = (uint64_t)blockIdx.x * TEAMS + team;
-    if (tt == 0) { mbar_init(&tc->mbar, 1); start_copy(t); }
+    if (tt == 64u) { mbar_init(&tc->mbar, 1); start_copy(t); }
     team_bar(team);
     uint32_t phase = 0, par = 0;
+    uint64_t t_done = ~0ull;                     // tile whose digest parts wait in wdig[par ^ 1]
+    // One team barrier per tile.  The single-lane chores sit on different warps (the team waits
+    // for whichever warp has the most to do): warp 2 starts the next copy, warp 1 folds and
+    // stores the previous tile's digest once the barrier has made its parts complete.
     for (; t < g.n_tiles; t += stride) {
         const bool first = first_in_chunk(g, (uint32_t)t);
         uint32_t d[kWordsPerLane];
@@ -386,14 +390,16 @@ k_tile_digests(const unsigned char* __restrict__ cache, Geo g, Ws ws, const Tabl
             load_tile_words_guarded(cache + t * kTile, (uint32_t)(g.nbytes - t * kTile), first, warp, lane, d);
             fold = false;
         }
-        team_bar(team);                          // stage free; wdig[par] of two tiles ago consumed
-        if (tt == 0) start_copy(t + stride);
+        team_bar(team);                          // stage free; the previous tile's digest parts complete
+        if (tt == 64u) start_copy(t + stride);
+        if (tt == 32u && t_done != ~0ull) ws.dig[t_done] = xor8(tc->wdig[par ^ 1u]);
         const uint32_t v = tile_digest_part(S, d, fold, warp, lane);
         if (lane == 0) tc->wdig[par][warp] = v;
-        team_bar(team);
-        if (tt == 0) ws.dig[t] = xor8(tc->wdig[par]);
+        t_done = t;
         par ^= 1u;
     }
+    team_bar(team);
+    if (tt == 32u && t_done != ~0ull) ws.dig[t_done] = xor8(tc->wdig[par ^ 1u]);
 }
 
 __global__ void __launch_bounds__(1024)
