@@ -1020,10 +1020,12 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
                 const uint32_t a0 = d[4 * j], a1 = d[4 * j + 1], a2 = d[4 * j + 2], a3 = d[4 * j + 3];
                 uint32_t mn = min_u16x2(min_u16x2(a0, a1), min_u16x2(a2, a3));
                 uint32_t mx = max_u16x2(max_u16x2(a0, a1), max_u16x2(a2, a3));
-                mn = min(mn & 0xFFFFu, mn >> 16);
-                mx = max(mx & 0xFFFFu, mx >> 16);
-                const uint32_t emin = __reduce_min_sync(0xFFFFFFFFu, mn) >> 8;
-                const uint32_t emax = __reduce_max_sync(0xFFFFFFFFu, mx) >> 8;
+                // both halves get the smaller (larger) of the two, so that the word as a whole
+                // orders like its halves and one warp reduction per bound does
+                mn = min_u16x2(mn, __byte_perm(mn, mn, 0x1032));
+                mx = max_u16x2(mx, __byte_perm(mx, mx, 0x1032));
+                const uint32_t emin = (__reduce_min_sync(0xFFFFFFFFu, mn) >> 8) & 0xFFu;
+                const uint32_t emax = (__reduce_max_sync(0xFFFFFFFFu, mx) >> 8) & 0xFFu;
                 gw[j] = emin | ((32u - __clz(emax - emin)) << 8);
             }
 #endif
