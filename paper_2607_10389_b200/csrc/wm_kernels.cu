@@ -847,8 +847,13 @@ __device__ __forceinline__ void pack_group_planes(uint32_t e4a, uint32_t e4b, ui
 //     take Y's words from the stage | team barrier | start the copy of the next Y |
 //     digest + exponent ranges of Y, publish len(Y) | park Y | fetch X | pack X straight into
 //     the wire image
-// Meanwhile one lane has two round trips to L2 in flight whose answers are needed a step later:
-// the ticket of the tile to measure two steps on and the offset of the tile to pack next.
+// Meanwhile two round trips to L2 are in flight whose answers are needed a step later: the
+// ticket of the tile to measure two steps on and the offset of the tile to pack next.  These and
+// the other single-lane chores of a step sit on different warps: the team passes one barrier per
+// tile, so it runs at the pace of the warp that has the most to do.
+// Template switches: MASKED (a dirty mask was given), LEAVES (the cache is a table of tensors;
+// tickets are claimed one step further ahead so that a tile's address can be looked up on the
+// way), ZEROS (the zero-tile option).
 // Packed data goes from registers to the wire image directly: in every region of a PACK tile
 // a lane owns an aligned unit at a lane-strided place, so each warp store is one contiguous
 // sector-aligned run.  Claiming a tile before the previous offset is known means that, if the
@@ -1669,9 +1674,11 @@ __device__ __forceinline__ void unpack_group_planes(const PlaneWords& pw, uint32
 // started a tile ahead, each lane takes what it needs (descriptors, its 8 sign-mantissa bytes
 // and its plane words per group: at most 16 words) into registers, and the stage is handed to
 // the next copy while the team unpacks, stores and checksums.  One team barrier per tile.
-// The team's first thread prepares tiles ahead of their turn, one dependent step per tile so
-// that it never sits waiting for an answer from L2: claim a ticket (three tiles ahead), look
-// up that tile's table entry and offsets (two ahead), start its copy (one ahead).
+// Tiles are prepared ahead of their turn, one dependent step per tile so that nobody sits
+// waiting for an answer from L2: claim a ticket (three tiles ahead, warp 3), look up that
+// tile's table entry and offsets (two ahead, warp 0), start its copy (one ahead, warp 2); warp 1
+// folds and stores the previous tile's digest.  (Spread over warps because the team runs at
+// the pace of its slowest one.)  LEAVES: the decoded tiles go to a table of tensors.
 template <int TEAMS, bool LEAVES>
 __global__ void __launch_bounds__(TEAMS * 256, 1)
 k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restrict__ dst, Ws ws,
