@@ -523,6 +523,20 @@ def main():
             entry["frac_of_nominal_8tbs"] = entry["kernel_traffic_gbs"] / 8000.0
         per_call[name] = entry
     wm.timing_enable(False)
+    # verify-before-write decode (two passes over the image): back-to-back time per call
+    for _ in range(3):
+        wm.wm_decode_verify_strict(wire, state["wire_len"], shadow, C, crc_dst, ws, res_d)
+    torch.cuda.synchronize()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    for _ in range(reps):
+        wm.wm_decode_verify_strict(wire, state["wire_len"], shadow, C, crc_dst, ws, res_d)
+    b.record()
+    torch.cuda.synchronize()
+    if not wm.read_result(res_d).ok:
+        raise SystemExit("strict decode failed")
+    per_call["decode_verify_strict"] = {"call_ms": a.elapsed_time(b) / reps, "reps": reps,
+                                        "note": "wm_decode_verify_strict: nothing is stored before the verdict"}
     # dirty diff: bytes it actually has to read (clean chunks in full on both sides)
     per_call["dirty_diff"]["note"] = f"{n_rewritten} of {nc} chunks dirty; clean chunks are read in full on both sides"
 

@@ -170,6 +170,23 @@ wm_status wm_decode_verify(const void* wire, uint64_t wire_len, void* dst, uint6
                            void* workspace, uint64_t workspace_bytes, wm_result* result, void* stream);
 
 /*
+ * wm_decode_verify_strict - verify first, write afterwards.
+ * Paper: "the destination is bit-identical to the source, or nothing is installed" (Section 1;
+ * Section 4.1: a torn state can never be installed).  wm_decode_verify gives that guarantee
+ * through the caller's shadow buffer; this call gives it for a buffer that is decoded into in
+ * place (the live cache of a pre-copy round): a first pass unpacks and checksums the image
+ * without storing a byte, the verdict is taken with all of wm_decode_verify's checks, and only
+ * after WM_OK does a second pass unpack again and store.  On any failure dst and
+ * dst_crc_inout are left exactly as they were.  Same arguments and result as
+ * wm_decode_verify; the image is read twice, so the call takes about 1.7 times as long.  The
+ * wire image must not change between the two passes (it is the caller's buffer on the
+ * caller's stream).
+ */
+wm_status wm_decode_verify_strict(const void* wire, uint64_t wire_len, void* dst, uint64_t nbytes,
+                                  uint32_t chunk_bytes, uint32_t* dst_crc_inout,
+                                  void* workspace, uint64_t workspace_bytes, wm_result* result, void* stream);
+
+/*
  * wm_zero_tiles_enable - encoder option: ship unused (all-zero) memory as table entries.
  * Paper: at least 19.4 % of the movable set is an allocation that no step writes or reads
  * (Section 3.3).  Read here as zero-filled memory: with the option on, a full tile of a

@@ -14,6 +14,7 @@ from .wm_oracle import (  # noqa: F401
     crc_combine,
     decode_verify,
     decode_verify_leaves,
+    decode_verify_strict,
     dirty_diff,
     encode,
     encode_leaves,

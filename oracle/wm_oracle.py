@@ -220,3 +220,12 @@ def decode_verify_leaves(wire, leaves, chunk_bytes: int, dst_crc=None, wire_len:
         parts.append(out[o:o + n].copy())
         o += n
     return parts, crc, res
+
+
+def decode_verify_strict(wire, nbytes: int, chunk_bytes: int, dst, dst_crc, wire_len: int | None = None):
+    """Verify first, write afterwards: what decode_verify returns when it succeeds; on any failure
+    the destination and its CRC vector come back exactly as they were given."""
+    out, crc, res = decode_verify(wire, nbytes, chunk_bytes, dst=dst, dst_crc=dst_crc, wire_len=wire_len)
+    if res.status != 0:
+        return _bytes_view(dst).copy(), np.array(dst_crc, dtype=np.uint32).copy(), res
+    return out, crc, res

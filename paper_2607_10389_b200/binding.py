@@ -24,7 +24,7 @@ RESULT_BYTES = 40
 EXPORTS = ("wm_num_chunks", "wm_num_tiles", "wm_meta_bytes", "wm_wire_bound", "wm_workspace_bytes",
            "wm_checksum", "wm_dirty_diff", "wm_encode", "wm_decode_verify", "wm_last_launch_count",
            "wm_timing_enable", "wm_timing_read_ms", "wm_checksum_noalloc", "wm_encode_leaves",
-           "wm_decode_verify_leaves", "wm_zero_tiles_enable")
+           "wm_decode_verify_leaves", "wm_zero_tiles_enable", "wm_decode_verify_strict")
 
 
 class WmError(RuntimeError):
@@ -62,6 +62,8 @@ def load_library() -> ctypes.CDLL:
     lib.wm_encode.argtypes = [vp, u64, u32, vp, vp, vp, u64, vp, u64, vp, vp]
     lib.wm_decode_verify.restype = ctypes.c_int
     lib.wm_decode_verify.argtypes = [vp, u64, vp, u64, u32, vp, vp, u64, vp, vp]
+    lib.wm_decode_verify_strict.restype = ctypes.c_int
+    lib.wm_decode_verify_strict.argtypes = [vp, u64, vp, u64, u32, vp, vp, u64, vp, vp]
     lib.wm_encode_leaves.restype = ctypes.c_int
     lib.wm_encode_leaves.argtypes = [vp, u32, u64, u32, vp, vp, vp, u64, vp, u64, vp, vp]
     lib.wm_decode_verify_leaves.restype = ctypes.c_int
@@ -232,6 +234,18 @@ def wm_decode_verify(wire: torch.Tensor, wire_len: int, dst: torch.Tensor, chunk
     _check(lib().wm_decode_verify(wire.data_ptr(), int(wire_len), dst.data_ptr(), nbytes, chunk_bytes,
                                   dst_crc_inout.data_ptr(), workspace.data_ptr(), workspace.numel(),
                                   result.data_ptr(), _stream(stream)), "wm_decode_verify")
+
+
+def wm_decode_verify_strict(wire: torch.Tensor, wire_len: int, dst: torch.Tensor, chunk_bytes: int,
+                            dst_crc_inout: torch.Tensor, workspace: torch.Tensor, result: torch.Tensor,
+                            stream=None) -> None:
+    """wm_decode_verify that stores nothing until every check has passed."""
+    _dev_u8(wire, "wire")
+    _dev_u8(dst, "dst")
+    nbytes = dst.numel() * dst.element_size()
+    _check(lib().wm_decode_verify_strict(wire.data_ptr(), int(wire_len), dst.data_ptr(), nbytes, chunk_bytes,
+                                         dst_crc_inout.data_ptr(), workspace.data_ptr(), workspace.numel(),
+                                         result.data_ptr(), _stream(stream)), "wm_decode_verify_strict")
 
 
 def make_leaf_table(tensors, device="cuda") -> torch.Tensor:

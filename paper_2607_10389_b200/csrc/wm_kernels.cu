@@ -1679,7 +1679,9 @@ __device__ __forceinline__ void unpack_group_planes(const PlaneWords& pw, uint32
 // tile's table entry and offsets (two ahead, warp 0), start its copy (one ahead, warp 2); warp 1
 // folds and stores the previous tile's digest.  (Spread over warps because the team runs at
 // the pace of its slowest one.)  LEAVES: the decoded tiles go to a table of tensors.
-template <int TEAMS, bool LEAVES>
+// MODE 0: unpack, store, checksum (the normal call).  Strict calls run the kernel twice: MODE 1
+// unpacks and checksums without storing anything; MODE 2, after the verdict, unpacks and stores.
+template <int TEAMS, bool LEAVES, int MODE>
 __global__ void __launch_bounds__(TEAMS * 256, 1)
 k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restrict__ dst, Ws ws,
          const Tables* __restrict__ tab)
@@ -1836,8 +1838,8 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
             if (e == 0xFFFFu) {
                 const unsigned char* src = payload + tc->slot[it & 3u].src;
                 const uint32_t len = g.tail_len;
-                for (uint32_t i = tt; i < len; i += kTeamThreads) o[i] = src[i];
-                load_tile_words_guarded(src, len, fold, warp, lane, w);
+                if (MODE != 1) for (uint32_t i = tt; i < len; i += kTeamThreads) o[i] = src[i];
+                if (MODE != 2) load_tile_words_guarded(src, len, fold, warp, lane, w);
                 fold = false;
             } else if (is_pack && decoded) {
 #ifdef WM_AB_D_NOUNPACK
@@ -1876,7 +1878,7 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
             }
             if (decoded) {
 #ifndef WM_AB_D_NOSTORE
-                if (e != 0xFFFFu) {
+                if (MODE != 1 && e != 0xFFFFu) {
                     unsigned char* q = o + warp * 2048u + lane * 4u;
 #pragma unroll
                     for (int i = 0; i < 16; i++) st_stream_u32(q + i * 128, w[i]);
@@ -1884,13 +1886,15 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
 #else
                 if (w[7] == 0x12345678u && e != 0xFFFFu) st_stream_u32(o + lane * 4u, w[2] ^ w[9] ^ w[12] ^ w[15] ^ w[0] ^ w[5]);
 #endif
+                if (MODE != 2) {
 #ifdef WM_AB_D_NOCRC
-                const uint32_t v = w[3] ^ w[6] ^ w[8] ^ w[13] ^ w[1] ^ w[4] ^ w[10] ^ w[11] ^ w[14];
+                    const uint32_t v = w[3] ^ w[6] ^ w[8] ^ w[13] ^ w[1] ^ w[4] ^ w[10] ^ w[11] ^ w[14];
 #else
-                const uint32_t v = tile_digest_part(S, w, fold, warp, lane);
+                    const uint32_t v = tile_digest_part(S, w, fold, warp, lane);
 #endif
-                if (lane == 0) tc->wdig[p][warp] = v;
-                have_digest = true;
+                    if (lane == 0) tc->wdig[p][warp] = v;
+                    have_digest = true;
+                }
             }
         }
         t_done = have_digest ? t : kNone;
@@ -1909,7 +1913,7 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
 __global__ void __launch_bounds__(1024)
 k_decode_finish(const unsigned char* __restrict__ wire, uint64_t wire_len, Geo g,
                 const unsigned char* __restrict__ dst, uint32_t* __restrict__ dst_crc, Ws ws,
-                const Tables* __restrict__ tab, wm_result* result, const __grid_constant__ ChunkPowers cp)
+                const Tables* __restrict__ tab, wm_result* result, const __grid_constant__ ChunkPowers cp, uint32_t strict)
 {
     __shared__ uint32_t sHT[1024];
     __shared__ uint32_t sT0[256];
@@ -1933,7 +1937,12 @@ k_decode_finish(const unsigned char* __restrict__ wire, uint64_t wire_len, Geo g
         if (step4_failed) {
             if (fl & CF_BAD4) { atomicMin(&ws.ctrl->bad4_first, c); atomicAdd(&ws.ctrl->bad4_count, 1u); }
         } else if (fl & CF_PRESENT) {
-            const uint32_t got = chunk_crc_staged(g, sHT, sT0, stage, ws.dig, chunk_first_byte(g, ws, dst, c), c, threadIdx.x);
+            // (a chunk shorter than four bytes is checksummed byte by byte: from dst, or, in a strict
+            // call, where nothing has been stored yet, from its raw copy in the wire image)
+            const unsigned char* tiny = chunk_first_byte(g, ws, dst, c);
+            if (strict && chunk_len_dev(g, c) < 4)
+                tiny = wire + g.meta_end + *reinterpret_cast<const unsigned long long*>(dir + 16ull * c);
+            const uint32_t got = chunk_crc_staged(g, sHT, sT0, stage, ws.dig, tiny, c, threadIdx.x);
             if (got != want) { atomicMin(&ws.ctrl->bad5_first, c); atomicAdd(&ws.ctrl->bad5_count, 1u); }
         } else {
             if (dst_crc[c] != want) { atomicMin(&ws.ctrl->bad6_first, c); atomicAdd(&ws.ctrl->bad6_count, 1u); }
@@ -1971,6 +1980,10 @@ k_decode_finish(const unsigned char* __restrict__ wire, uint64_t wire_len, Geo g
         }
         fill_result(result, ws.ctrl, wire_len, status, first, count);
         s_status = status;
+        if (strict) {                  // the storing pass follows: it starts from ticket 0 and stays out after a failure
+            ws.ctrl->ticket = 0;
+            if (status != WM_OK) ws.ctrl->gate = (uint32_t)status;
+        }
     }
     __syncthreads();
     if (s_status == WM_OK) {
@@ -2035,8 +2048,13 @@ static const DeviceState* device_state()
         for (const void* f : enc)
             if (cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, big) != cudaSuccess) return nullptr;
     }
-    if (cudaFuncSetAttribute(k_decode<kTeamsPlain, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, big) != cudaSuccess) return nullptr;
-    if (cudaFuncSetAttribute(k_decode<kTeamsPlain, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, big) != cudaSuccess) return nullptr;
+    {
+        const void* dec[] = {(const void*)k_decode<kTeamsPlain, false, 0>, (const void*)k_decode<kTeamsPlain, true, 0>,
+                             (const void*)k_decode<kTeamsPlain, false, 1>, (const void*)k_decode<kTeamsPlain, true, 1>,
+                             (const void*)k_decode<kTeamsPlain, false, 2>, (const void*)k_decode<kTeamsPlain, true, 2>};
+        for (const void* f : dec)
+            if (cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, big) != cudaSuccess) return nullptr;
+    }
     if (cudaFuncSetAttribute(k_tile_digests<kTeamsPlain>, cudaFuncAttributeMaxDynamicSharedMemorySize, big) != cudaSuccess) return nullptr;
     if (cudaFuncSetAttribute(k_meta_crc, cudaFuncAttributeMaxDynamicSharedMemorySize, big) != cudaSuccess) return nullptr;
     for (int k = 0; k < 4; k++)
@@ -2291,9 +2309,10 @@ wm_status wm_encode_leaves(const wm_leaf* leaves, uint32_t n_leaves, uint64_t nb
 }
 
 // Both forms of the decode call: a flat shadow buffer (leaves == nullptr) or a table of leaves.
+// strict: nothing is stored until every check has passed (two passes over the wire image).
 static wm_status decode_any(const void* wire, uint64_t wire_len, void* dst, const wm_leaf* leaves, uint32_t n_leaves, uint64_t nbytes,
                             uint32_t chunk_bytes, uint32_t* dst_crc_inout, void* workspace, uint64_t workspace_bytes,
-                            wm_result* result, void* stream)
+                            wm_result* result, void* stream, bool strict)
 {
     Geo g;
     if (!wire || !dst_crc_inout || !workspace || !result || !make_geo(nbytes, chunk_bytes, g)) return WM_ERR_ARG;
@@ -2316,14 +2335,19 @@ static wm_status decode_any(const void* wire, uint64_t wire_len, void* dst, cons
     launch_after(k_decode_check, meta_blocks + (g.n_chunks + 31) / 32, 1024, 0, s, w, wire_len, g, ws, ds->tables, result, meta_blocks);
     const uint32_t need = (g.n_tiles + kTeamsPlain - 1) / kTeamsPlain;
     const uint32_t grid = need < (uint32_t)ds->sm_count ? need : (uint32_t)ds->sm_count;
+    auto pass = [&](auto flat_kernel, auto leaf_kernel) {
+        if (leaves) launch_after(leaf_kernel, grid, kTeamsPlain * 256, kDynSmem, s, w, g, d, ws, ds->tables);
+        else launch_after(flat_kernel, grid, kTeamsPlain * 256, kDynSmem, s, w, g, d, ws, ds->tables);
+    };
     {
         MainKernelTimer timer(ds, 3, s);
-        if (leaves) launch_after(k_decode<kTeamsPlain, true>, grid, kTeamsPlain * 256, kDynSmem, s, w, g, d, ws, ds->tables);
-        else launch_after(k_decode<kTeamsPlain, false>, grid, kTeamsPlain * 256, kDynSmem, s, w, g, d, ws, ds->tables);
+        if (strict) pass(k_decode<kTeamsPlain, false, 1>, k_decode<kTeamsPlain, true, 1>);
+        else pass(k_decode<kTeamsPlain, false, 0>, k_decode<kTeamsPlain, true, 0>);
     }
     launch_after(k_decode_finish, (g.n_chunks + g.finish_cb - 1) / g.finish_cb, 1024, 0, s, w, wire_len, g, d, dst_crc_inout, ws, ds->tables,
-                 result, chunk_powers(g));
-    g_launches = leaves ? 5 : 4;
+                 result, chunk_powers(g), strict ? 1u : 0u);
+    if (strict) pass(k_decode<kTeamsPlain, false, 2>, k_decode<kTeamsPlain, true, 2>);
+    g_launches = (leaves ? 5 : 4) + (strict ? 1 : 0);
     return launch_status();
 }
 
@@ -2332,7 +2356,17 @@ wm_status wm_decode_verify(const void* wire, uint64_t wire_len, void* dst, uint6
                            void* stream)
 {
     if (!dst) return WM_ERR_ARG;
-    return decode_any(wire, wire_len, dst, nullptr, 0, nbytes, chunk_bytes, dst_crc_inout, workspace, workspace_bytes, result, stream);
+    return decode_any(wire, wire_len, dst, nullptr, 0, nbytes, chunk_bytes, dst_crc_inout, workspace, workspace_bytes, result, stream,
+                      false);
+}
+
+wm_status wm_decode_verify_strict(const void* wire, uint64_t wire_len, void* dst, uint64_t nbytes, uint32_t chunk_bytes,
+                                  uint32_t* dst_crc_inout, void* workspace, uint64_t workspace_bytes, wm_result* result,
+                                  void* stream)
+{
+    if (!dst) return WM_ERR_ARG;
+    return decode_any(wire, wire_len, dst, nullptr, 0, nbytes, chunk_bytes, dst_crc_inout, workspace, workspace_bytes, result, stream,
+                      true);
 }
 
 wm_status wm_decode_verify_leaves(const void* wire, uint64_t wire_len, const wm_leaf* dst_leaves, uint32_t n_leaves, uint64_t nbytes,
@@ -2341,7 +2375,7 @@ wm_status wm_decode_verify_leaves(const void* wire, uint64_t wire_len, const wm_
 {
     if (!dst_leaves) return WM_ERR_ARG;
     return decode_any(wire, wire_len, nullptr, dst_leaves, n_leaves, nbytes, chunk_bytes, dst_crc_inout, workspace, workspace_bytes, result,
-                      stream);
+                      stream, false);
 }
 
 }  // extern "C"
