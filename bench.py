@@ -316,6 +316,61 @@ def leaf_mode(wm, cfg, cur, wire, ws, dev, W, peak, reps=20):
     return out
 
 
+def tail_schedule(wm, cfg, cur, shadow, wire, ws, dev, W, reps=8, super_mbs=(64, 128, 256)):
+    """Verification placement: the move cut into super-chunks on three streams (encode, a device-to-device
+    copy standing in for the wire, decode + verify), against the same three stages run one after the
+    other on the whole cache.  `exposed_ms` is what remains after the last wire byte has arrived."""
+    import statistics
+    import torch
+    from paper_2607_10389_b200 import tail_schedule as ts
+    N, C = cfg.nbytes, cfg.chunk_bytes
+    nc = wm.num_chunks(N, C)
+    crc_s = torch.zeros(nc, dtype=torch.int32, device=dev)
+    crc_d = torch.zeros(nc, dtype=torch.int32, device=dev)
+    res_e, res_d = wm.new_result(dev), wm.new_result(dev)
+    recv = torch.empty(W, dtype=torch.uint8, device=dev)
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+    tot, exp = [], []
+    for i in range(reps + 2):
+        torch.cuda.synchronize()
+        ev[0].record()
+        wm.wm_encode(cur, C, None, crc_s, wire, ws, res_e)
+        wl = wm.read_result(res_e).wire_len              # the sender learns the image length
+        recv[:wl].copy_(wire[:wl], non_blocking=True)
+        ev[1].record()
+        wm.wm_decode_verify(recv, wl, shadow, C, crc_d, ws, res_d)
+        ev[2].record()
+        torch.cuda.synchronize()
+        if i >= 2:
+            tot.append(ev[0].elapsed_time(ev[2]))
+            exp.append(ev[1].elapsed_time(ev[2]))
+    if not wm.read_result(res_d).ok:
+        raise SystemExit("tail schedule: sequential move failed")
+    out = {"sequential": {"total_ms": statistics.median(tot), "exposed_ms": statistics.median(exp)}, "pipelined": []}
+    for mb in super_mbs:
+        sup = mb << 20
+        if sup % C or sup >= N:
+            continue
+        sched = ts.TailSchedule(N, C, sup, dev)
+        tot, exp = [], []
+        for i in range(reps + 2):
+            shadow[:4096].zero_()
+            rep = sched.move(cur, shadow, crc_s, crc_d)
+            if not rep.ok:
+                raise SystemExit("tail schedule: a part failed")
+            if i >= 2:
+                tot.append(rep.total_ms)
+                exp.append(rep.exposed_ms)
+        if not torch.equal(shadow, cur):
+            raise SystemExit("tail schedule: destination differs from the source")
+        out["pipelined"].append({"super_mib": mb, "parts": len(sched.parts), "total_ms": statistics.median(tot),
+                                 "exposed_ms": statistics.median(exp), "launches": sched.launches})
+        del sched
+    out["note"] = ("total = first encode starts -> last verification ends; exposed = last wire copy ends -> last "
+                   "verification ends; the wire is a device-to-device copy; medians of %d moves" % reps)
+    return out
+
+
 def run_reference(args):
     """Reference arm: the CPU oracle timed on the host cores, a bounded sample per step."""
     rank, _, world = _dist()
@@ -563,6 +618,11 @@ def main():
     if not args.no_loop and cfg.kind == "kv":
         leaf = leaf_mode(wm, cfg, cur, wire, ws, dev, W, peak)
 
+    # verification placement: super-chunks on three streams against the whole cache stage by stage
+    tail = None
+    if not args.no_loop and args.workload in ("engine", "engine_256m"):
+        tail = tail_schedule(wm, cfg, cur, shadow, wire, ws, dev, W)
+
     # end to end: host cache in (pinned), verified wire image and result records out
     e2e = None
     if not args.no_e2e:
@@ -644,7 +704,8 @@ def main():
                        "wire_bytes": W, "ratio": W / N, "dirty_chunks": n_rewritten, "n_chunks": nc,
                        "l2": "inputs larger than L2 (no flush needed)", "parallelism": "replicas only",
                        "zero_tiles": bool(args.zero_tiles)},
-            "calls": per_call, "roofline": roofline, "precopy_loop": loop, "leaf_mode": leaf, "cpu_baseline": base, "e2e": e2e,
+            "calls": per_call, "roofline": roofline, "precopy_loop": loop, "leaf_mode": leaf, "tail_schedule": tail,
+            "cpu_baseline": base, "e2e": e2e,
             "gpu_launches": gpu_launches, "clocks": clocks,
         }
         print(json.dumps(out))
