@@ -592,6 +592,20 @@ def main():
         raise SystemExit("strict decode failed")
     per_call["decode_verify_strict"] = {"call_ms": a.elapsed_time(b) / reps, "reps": reps,
                                         "note": "wm_decode_verify_strict: nothing is stored before the verdict"}
+    # the checksum step with the CRC-32 polynomial of zlib (same kernels, other tables)
+    crc_z = torch.zeros(nc, dtype=torch.int32, device=dev)
+    for _ in range(3):
+        wm.wm_checksum_poly(cur, C, wm.POLY_ZLIB, crc_z, ws)
+    torch.cuda.synchronize()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    for _ in range(reps):
+        wm.wm_checksum_poly(cur, C, wm.POLY_ZLIB, crc_z, ws)
+    b.record()
+    torch.cuda.synchronize()
+    zm = a.elapsed_time(b) / reps
+    per_call["checksum_zlib_polynomial"] = {"call_ms": zm, "reps": reps,
+                                            "call_frac_of_hbm_peak": (N + 4 * nc) / (zm * 1e-3) / 1e9 / peak}
     # dirty diff: bytes it actually has to read (clean chunks in full on both sides)
     per_call["dirty_diff"]["note"] = f"{n_rewritten} of {nc} chunks dirty; clean chunks are read in full on both sides"
 

@@ -86,6 +86,22 @@ wm_status wm_checksum(const void* cache, uint64_t nbytes, uint32_t chunk_bytes,
                       uint32_t* crc_out, void* workspace, uint64_t workspace_bytes, void* stream);
 
 /*
+ * wm_checksum_poly - wm_checksum with the CRC polynomial as an argument.
+ * Paper: the verification plane (Section 6.5) measures its chunk CRC with zlib's CRC-32 on the
+ * CPU side, while the wire format of this library fixes CRC32C.  This call offers both for the
+ * checksum step alone; wm_encode and wm_decode_verify always use CRC32C.
+ *   polynomial  WM_POLY_CRC32C (the same as wm_checksum) or WM_POLY_ZLIB (reflected 0xEDB88320,
+ *               init and final xor all ones; "123456789" -> 0xCBF43926, what zlib's crc32 returns);
+ *               anything else returns WM_ERR_ARG and launches nothing
+ * All other arguments, layouts and errors are those of wm_checksum.  The first WM_POLY_ZLIB
+ * call on a device allocates and uploads that polynomial's tables (synchronous, once).
+ */
+#define WM_POLY_CRC32C 0
+#define WM_POLY_ZLIB 1
+wm_status wm_checksum_poly(const void* cache, uint64_t nbytes, uint32_t chunk_bytes, int polynomial,
+                           uint32_t* crc_out, void* workspace, uint64_t workspace_bytes, void* stream);
+
+/*
  * wm_dirty_diff - which chunks changed since the previous snapshot.
  * Paper: live pre-copy (Appendix G: round 0 ships every chunk, each later round the dirty
  * ones) and the measured dirty fraction per generation step (Section 3.3).  The compare is

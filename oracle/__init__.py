@@ -9,6 +9,7 @@ from .wm_oracle import (  # noqa: F401
     Result,
     build,
     checksum,
+    checksum_poly,
     crc32c,
     crc_bitwise,
     crc_combine,

@@ -149,6 +149,13 @@ def checksum(cache, chunk_bytes: int) -> np.ndarray:
     return out
 
 
+def checksum_poly(cache, chunk_bytes: int, poly: int) -> np.ndarray:
+    """The checksum step with another polynomial: the bit-at-a-time definition, chunk by chunk."""
+    b = _bytes_view(cache)
+    n = num_chunks(b.size, chunk_bytes)
+    return np.array([crc_bitwise(b[c * chunk_bytes: (c + 1) * chunk_bytes], poly) for c in range(n)], dtype=np.uint32)
+
+
 def dirty_diff(cache, prev, chunk_bytes: int):
     """Return (dirty u8[n_chunks], dirty_idx u32[n_dirty])."""
     a, p = _bytes_view(cache), _bytes_view(prev)

@@ -24,7 +24,7 @@ RESULT_BYTES = 40
 EXPORTS = ("wm_num_chunks", "wm_num_tiles", "wm_meta_bytes", "wm_wire_bound", "wm_workspace_bytes",
            "wm_checksum", "wm_dirty_diff", "wm_encode", "wm_decode_verify", "wm_last_launch_count",
            "wm_timing_enable", "wm_timing_read_ms", "wm_checksum_noalloc", "wm_encode_leaves",
-           "wm_decode_verify_leaves", "wm_zero_tiles_enable", "wm_decode_verify_strict")
+           "wm_decode_verify_leaves", "wm_zero_tiles_enable", "wm_decode_verify_strict", "wm_checksum_poly")
 
 
 class WmError(RuntimeError):
@@ -54,6 +54,8 @@ def load_library() -> ctypes.CDLL:
     lib.wm_timing_read_ms.argtypes = [ctypes.c_int, ctypes.POINTER(ctypes.c_float)]
     lib.wm_checksum.restype = ctypes.c_int
     lib.wm_checksum.argtypes = [vp, u64, u32, vp, vp, u64, vp]
+    lib.wm_checksum_poly.restype = ctypes.c_int
+    lib.wm_checksum_poly.argtypes = [vp, u64, u32, ctypes.c_int, vp, vp, u64, vp]
     lib.wm_checksum_noalloc.restype = ctypes.c_int
     lib.wm_checksum_noalloc.argtypes = [vp, u64, u32, vp, vp]
     lib.wm_dirty_diff.restype = ctypes.c_int
@@ -185,6 +187,18 @@ def wm_checksum(cache: torch.Tensor, chunk_bytes: int, crc_out: torch.Tensor, wo
     nbytes = cache.numel() * cache.element_size()
     _check(lib().wm_checksum(cache.data_ptr(), nbytes, chunk_bytes, crc_out.data_ptr(), workspace.data_ptr(),
                              workspace.numel(), _stream(stream)), "wm_checksum")
+
+
+POLY_CRC32C, POLY_ZLIB = 0, 1
+
+
+def wm_checksum_poly(cache: torch.Tensor, chunk_bytes: int, polynomial: int, crc_out: torch.Tensor,
+                     workspace: torch.Tensor, stream=None) -> None:
+    """wm_checksum with the polynomial chosen by the caller (POLY_CRC32C or POLY_ZLIB)."""
+    _dev_u8(cache, "cache")
+    nbytes = cache.numel() * cache.element_size()
+    _check(lib().wm_checksum_poly(cache.data_ptr(), nbytes, chunk_bytes, int(polynomial), crc_out.data_ptr(),
+                                  workspace.data_ptr(), workspace.numel(), _stream(stream)), "wm_checksum_poly")
 
 
 NOALLOC_MAX_BYTES = 4 << 30

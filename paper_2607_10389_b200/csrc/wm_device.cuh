@@ -201,14 +201,14 @@ __device__ __forceinline__ uint32_t tile_digest_part_small(const uint32_t* sG, c
 }
 
 // Generic product of two residues (bitwise; used a handful of times per call).
-__device__ __forceinline__ uint32_t mulmod_dev(uint32_t a, uint32_t b)
+__device__ __forceinline__ uint32_t mulmod_dev(uint32_t a, uint32_t b, uint32_t poly = kPolyReflected)
 {
     uint32_t r = 0;
 #pragma unroll 8
     for (int i = 0; i < 32; i++) {
         r ^= b & (0u - (a >> 31));
         a <<= 1;
-        b = (b >> 1) ^ (kPolyReflected & (0u - (b & 1u)));
+        b = (b >> 1) ^ (poly & (0u - (b & 1u)));
     }
     return r;
 }

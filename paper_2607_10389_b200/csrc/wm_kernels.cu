@@ -38,6 +38,7 @@ struct Geo {
     uint32_t tpc_shift;       // log2(tiles_per_chunk) when that is a power of two, else 32
     uint32_t n_full_tiles;    // tiles of exactly 16384 bytes
     uint32_t finish_cb;       // chunks handled by one block of the finish kernels
+    uint32_t poly;            // reflected CRC polynomial of the k_* powers (CRC32C except in wm_checksum_poly)
 };
 
 // Powers of k_chunk = x^(8 chunk_bytes), by 7-bit digit of the exponent: k_chunk^e is the product
@@ -156,6 +157,7 @@ static bool make_geo(uint64_t nbytes, uint32_t chunk_bytes, Geo& g)
         if (g.tiles_per_chunk == (1u << k)) g.tpc_shift = k;
     uint32_t cb = kFinishDigests / g.tiles_per_chunk;
     g.finish_cb = cb > kFinishChunks ? kFinishChunks : (cb ? cb : 1u);
+    g.poly = kPolyReflected;
     last = g;
     have_last = true;
     return true;
@@ -248,7 +250,7 @@ __device__ uint32_t chunk_crc_from_digests(const Geo& g, const uint32_t* HT, con
         }
     }
     for (; i < ntc; i++) {
-        if (i + 1 == ntc && ragged) st = mulmod_dev(st, g.k_tail);
+        if (i + 1 == ntc && ragged) st = mulmod_dev(st, g.k_tail, g.poly);
         else st = advance_tile(HT, st);
         st ^= __ldcg(dig + t0 + i);
     }
@@ -301,7 +303,7 @@ __device__ uint32_t chunk_crc_staged(const Geo& g, const uint32_t* HT, const uin
     uint32_t s = 0;
     const uint32_t n_plain = ragged ? ntc - 1 : ntc;
     for (uint32_t k = 0; k < n_plain; k++) s = advance_tile(HT, s) ^ d[k];
-    if (ragged) s = mulmod_dev(s, g.k_tail) ^ d[ntc - 1];
+    if (ragged) s = mulmod_dev(s, g.k_tail, g.poly) ^ d[ntc - 1];
     return ~s;
 }
 
@@ -2005,6 +2007,7 @@ constexpr int kTeamsPlain = WM_TEAMS_PLAIN;  // checksum / decode: teams per blo
 
 struct DeviceState {
     Tables* tables = nullptr;
+    Tables* tables_zlib = nullptr;   // built on the first wm_checksum_poly call that asks for it
     int sm_count = 0;
     bool ready = false;
     cudaEvent_t ev[4][2] = {};   // optional timing of the four main kernels
@@ -2148,6 +2151,54 @@ wm_status wm_checksum(const void* cache, uint64_t nbytes, uint32_t chunk_bytes, 
         k_tile_digests<kTeamsPlain><<<grid, kTeamsPlain * 256, kDynSmem, s>>>(c, g, ws, ds->tables);
     }
     launch_after(k_checksum_finish, (g.n_chunks + g.finish_cb - 1) / g.finish_cb, 1024, 0, s, c, g, ws, ds->tables, crc_out);
+    g_launches = 2;
+    return launch_status();
+}
+
+// The checksum call with the polynomial as an argument.  The tile kernel and the finish kernel
+// are the ones wm_checksum runs: the polynomial lives in the tables and in the geometry's powers.
+static const Tables* zlib_tables()
+{
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    std::lock_guard<std::mutex> lock(g_mutex);
+    DeviceState& s = g_dev[dev];
+    if (s.tables_zlib) return s.tables_zlib;
+    static Tables host;
+    build_tables(host, kPolyZlib);
+    Tables* p = nullptr;
+    if (cudaMalloc(&p, sizeof(Tables)) != cudaSuccess) return nullptr;
+    if (cudaMemcpy(p, &host, sizeof(Tables), cudaMemcpyHostToDevice) != cudaSuccess) { cudaFree(p); return nullptr; }
+    s.tables_zlib = p;
+    return p;
+}
+
+wm_status wm_checksum_poly(const void* cache, uint64_t nbytes, uint32_t chunk_bytes, int polynomial, uint32_t* crc_out,
+                           void* workspace, uint64_t workspace_bytes, void* stream)
+{
+    if (polynomial == WM_POLY_CRC32C) return wm_checksum(cache, nbytes, chunk_bytes, crc_out, workspace, workspace_bytes, stream);
+    if (polynomial != WM_POLY_ZLIB) return WM_ERR_ARG;
+    Geo g;
+    if (!cache || !crc_out || !workspace || !make_geo(nbytes, chunk_bytes, g)) return WM_ERR_ARG;
+    if (!aligned16(cache) || !aligned16(workspace) || workspace_bytes < ws_layout(g).total) return WM_ERR_ARG;
+    const DeviceState* ds = device_state();
+    if (!ds) return WM_ERR_CUDA;
+    const Tables* tab = zlib_tables();
+    if (!tab) return WM_ERR_CUDA;
+    g.poly = kPolyZlib;
+    g.k_tail = x_pow_bytes(g.tail_len, kPolyZlib);
+    g.k_chunk = x_pow_bytes(g.chunk_bytes, kPolyZlib);
+    g.k_last_chunk = x_pow_bytes(g.last_chunk_len, kPolyZlib);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    Ws ws = ws_carve(workspace, g);
+    const unsigned char* c = static_cast<const unsigned char*>(cache);
+    const uint32_t need = (g.n_tiles + kTeamsPlain - 1) / kTeamsPlain;
+    const uint32_t grid = need < (uint32_t)ds->sm_count ? need : (uint32_t)ds->sm_count;
+    {
+        MainKernelTimer timer(ds, 0, s);
+        k_tile_digests<kTeamsPlain><<<grid, kTeamsPlain * 256, kDynSmem, s>>>(c, g, ws, tab);
+    }
+    launch_after(k_checksum_finish, (g.n_chunks + g.finish_cb - 1) / g.finish_cb, 1024, 0, s, c, g, ws, tab, crc_out);
     g_launches = 2;
     return launch_status();
 }
