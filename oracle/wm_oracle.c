@@ -252,14 +252,185 @@ static int plane_widths(uint32_t w, uint32_t p[3])
     if (w & 1u) p[n++] = 1u;
     return n;
 }
-static uint32_t encode_full_tile(const uint8_t* src, uint8_t* out, uint32_t* entry, int zero_tiles)
+
+/* ------------------------------------------------- ENT tiles (option) ---
+ * Entropy-coded exponents (the variant of the codec the paper measured codes the exponent
+ * plane with an entropy coder; Section 6.4).  An image that sets header flags bit 2 stores a
+ * full tile either as an ENT tile or raw; the sign-mantissa plane is the one of a PACK tile.
+ *
+ * A tile is eight shares of 16 rows (row = 128 bytes = 64 elements).  Share s has 32 strands;
+ * strand l holds the 32 elements at 32-bit word l of the share's rows, row after row, low half
+ * first: element i of the strand is tile element 64 (16 s + i / 2) + 2 l + i % 2.
+ *
+ *   anchor_s = (sum of the share's 1024 exponents + 512) >> 10      (the rounded mean)
+ *   u = E - anchor_s is coded with a fixed prefix code; the bits of a codeword are listed in
+ *   the order they are written, and a strand is an LSB-first bit string:
+ *        u:   0    +1    -1    -2     +2     -3     -4      -5       +3        -6
+ *      bits:  00   10    01    1100   1110   1101   11110   111110   1111110   11111110
+ *      any other u: 11111111 followed by the eight bits of E itself, low bit first (16 bits)
+ *   (as numbers, first bit = bit 0: 0, 1, 2, 3, 7, 11, 15, 31, 63, 127, 255 | E << 8).
+ *
+ * The 32 strands of a share are cut into 16-bit halfwords (the last one zero-filled) and
+ * interleaved into one stream in the order a reader needs them: the reader walks i = 0..31;
+ * at step i every strand whose codeword i is not complete in the halfwords it has taken so
+ * far takes the next halfword of the stream, strands in ascending order; then every strand
+ * consumes its codeword i.  (A codeword is at most 16 bits, so one halfword always suffices.)
+ *
+ *   ENT tile:  anchor[8] u8 | count[8] u16 (halfwords in each share's stream) | 40 zero bytes
+ *              SM[8192] as in a PACK tile | the eight streams | zero fill to a multiple of 32
+ *   entry = 0x8000 | length / 32, used iff the length is below 16384; else the tile is raw.
+ */
+static const int      ent_sym[10]  = {0, 1, -1, -2, 2, -3, -4, -5, 3, -6};
+static const uint32_t ent_len[10]  = {2, 2, 2, 4, 4, 4, 5, 6, 7, 8};
+static const uint32_t ent_bits[10] = {0, 1, 2, 3, 7, 11, 15, 31, 63, 127};
+
+static uint32_t ent_elem(uint32_t share, uint32_t strand, uint32_t i)
+{
+    return 64u * (16u * share + i / 2u) + 2u * strand + i % 2u;
+}
+
+static void ent_codeword(uint32_t E, uint32_t anchor, uint32_t* bits, uint32_t* len)
+{
+    int u = (int)E - (int)anchor;
+    for (int k = 0; k < 10; k++)
+        if (u == ent_sym[k]) { *bits = ent_bits[k]; *len = ent_len[k]; return; }
+    *bits = 255u | (E << 8);
+    *len = 16u;
+}
+
+/* Length and symbol of the codeword at the low end of `buf` (bits beyond the valid ones are
+ * zero).  Returns the length; *E receives the exponent. */
+static uint32_t ent_parse(uint32_t buf, uint32_t anchor, uint32_t* E)
+{
+    for (int k = 0; k < 10; k++)
+        if ((buf & ((1u << ent_len[k]) - 1u)) == ent_bits[k]) {
+            *E = (uint32_t)((int)anchor + ent_sym[k]) & 0xFFu;
+            return ent_len[k];
+        }
+    *E = (buf >> 8) & 0xFFu;
+    return 16u;
+}
+
+/* Encode the exponents of one tile as ENT streams.  Returns the tile's length in bytes (a
+ * multiple of 32; it may exceed the tile size, in which case the caller stores the tile raw
+ * and `out` is not used).  `out` must hold 64 + 8192 + 8 * 32 * 64 + 32 bytes. */
+static uint32_t encode_ent_tile(const uint8_t* src, uint8_t* out)
+{
+    uint32_t hw_total = 0;
+    memset(out, 0, 64);
+    uint8_t* stream = out + 64 + 8192;
+    for (uint32_t s = 0; s < 8; s++) {
+        uint32_t sum = 0;
+        for (uint32_t e = 0; e < 1024; e++) sum += (get16(src + 2u * (1024u * s + e)) >> 7) & 0xFFu;
+        uint32_t anchor = (sum + 512u) >> 10;
+        out[s] = (uint8_t)anchor;
+        /* every strand as a bit string, and the bits used up to and including codeword i */
+        static uint8_t bit[32][32 * 16 + 16];
+        uint32_t upto[32][32];
+        memset(bit, 0, sizeof bit);
+        for (uint32_t l = 0; l < 32; l++) {
+            uint32_t n = 0;
+            for (uint32_t i = 0; i < 32; i++) {
+                uint32_t E = (get16(src + 2u * ent_elem(s, l, i)) >> 7) & 0xFFu, cw, len;
+                ent_codeword(E, anchor, &cw, &len);
+                for (uint32_t b = 0; b < len; b++) bit[l][n + b] = (uint8_t)((cw >> b) & 1u);
+                n += len;
+                upto[l][i] = n;
+            }
+        }
+        uint32_t taken[32] = {0}, count = 0;
+        for (uint32_t i = 0; i < 32; i++)
+            for (uint32_t l = 0; l < 32; l++)
+                if (upto[l][i] > 16u * taken[l]) {
+                    uint32_t hw = 0;
+                    for (uint32_t b = 0; b < 16; b++) hw |= (uint32_t)bit[l][16u * taken[l] + b] << b;
+                    put16(stream + 2u * (hw_total + count), hw);
+                    taken[l]++;
+                    count++;
+                }
+        put16(out + 8 + 2u * s, count);
+        hw_total += count;
+    }
+    uint32_t len = 8256u + 2u * hw_total;
+    while (len % 32u) out[len++] = 0;
+    /* sign-mantissa plane: the PACK tile's */
+    for (uint32_t g = 0; g < WMO_GROUPS_PER_TILE; g++)
+        for (uint32_t e = 0; e < WMO_GROUP_ELEMS; e++) {
+            uint32_t v = get16(src + 2u * (g * WMO_GROUP_ELEMS + e));
+            out[64u + 256u * g + coded_pos(e)] = (uint8_t)(((v & 0x7Fu) << 1) | (v >> 15));
+        }
+    return len;
+}
+
+/* Header of an ENT tile against its table entry: every share's count within what 32 strands
+ * of 32 codewords can need, and the length they add up to.  Returns 0 when it fits. */
+static int ent_header_bad(const uint8_t* in, uint32_t entry)
+{
+    uint32_t total = 0;
+    for (uint32_t s = 0; s < 8; s++) {
+        uint32_t c = get16(in + 8 + 2u * s);
+        if (c < 128u || c > 1024u) return 1;
+        total += c;
+    }
+    return ((8256u + 2u * total + 31u) / 32u) != (entry & 0x7FFFu);
+}
+
+/* Read the eight streams of an ENT tile whose header fits.  With dst != NULL the tile is
+ * written there.  Returns 0 when every stream is used up exactly and the bits left over in every
+ * strand's last halfword are zero, 1 otherwise. */
+static int decode_ent_tile(const uint8_t* in, uint8_t* dst)
+{
+    const uint8_t* stream = in + 64 + 8192;
+    int bad = 0;
+    for (uint32_t s = 0; s < 8; s++) {
+        uint32_t anchor = in[s], count = get16(in + 8 + 2u * s), pos = 0;
+        uint32_t buf[32] = {0}, avail[32] = {0};
+        for (uint32_t i = 0; i < 32; i++)
+            for (uint32_t l = 0; l < 32; l++) {
+                uint32_t E;
+                if (ent_parse(buf[l], anchor, &E) > avail[l]) {
+                    uint32_t hw = 0;
+                    if (pos < count) hw = get16(stream + 2u * pos); else bad = 1;
+                    pos++;
+                    buf[l] |= hw << avail[l];
+                    avail[l] += 16u;
+                }
+                uint32_t len = ent_parse(buf[l], anchor, &E);
+                buf[l] >>= len;
+                avail[l] -= len;
+                if (dst) {
+                    uint32_t e = ent_elem(s, l, i);
+                    uint32_t SM = in[64u + 256u * (e / 256u) + coded_pos(e % 256u)];
+                    put16(dst + 2u * e, ((SM & 1u) << 15) | (E << 7) | (SM >> 1));
+                }
+            }
+        if (pos != count) bad = 1;
+        for (uint32_t l = 0; l < 32; l++)
+            if (buf[l]) bad = 1;                 /* the fill bits of a strand's last halfword are zero */
+        stream += 2u * count;
+    }
+    return bad;
+}
+
+#define WMO_OPT_ZERO_TILES 1   /* encoder options */
+#define WMO_OPT_ENTROPY 2
+
+static uint32_t encode_full_tile(const uint8_t* src, uint8_t* out, uint32_t* entry, int options)
 {
     uint32_t base[WMO_GROUPS_PER_TILE], w[WMO_GROUPS_PER_TILE], S = 0;
     /* option: a tile whose 16384 bytes are all zero (unused allocation) has entry 1 and no payload */
-    if (zero_tiles) {
+    if (options & WMO_OPT_ZERO_TILES) {
         uint32_t any = 0;
         for (uint32_t i = 0; i < WMO_TILE; i++) any |= src[i];
         if (!any) { *entry = 1u; return 0; }
+    }
+    /* option: entropy-coded exponents; the tile is an ENT tile when that is shorter than raw */
+    if (options & WMO_OPT_ENTROPY) {
+        uint32_t len = encode_ent_tile(src, out);
+        if (len < WMO_TILE) { *entry = 0x8000u | (len / 32u); return len; }
+        memcpy(out, src, WMO_TILE);
+        *entry = 512u;
+        return WMO_TILE;
     }
     for (uint32_t g = 0; g < WMO_GROUPS_PER_TILE; g++) {
         uint32_t mn = 255, mx = 0;
@@ -315,14 +486,14 @@ static uint32_t encode_full_tile(const uint8_t* src, uint8_t* out, uint32_t* ent
  *   multiple of 32 (= meta_end) | payload
  *
  *   header:  0 "WMV1"   4 u16 version=1   6 u16 flags (bit0: a dirty mask was given;
- *            bit1: ZERO tile option)
+ *            bit1: ZERO tile option; bit2: ENT tiles instead of PACK tiles)
  *            8 u64 nbytes   16 u32 chunk_bytes   20 u32 tile_bytes=16384
  *           24 u32 n_chunks 28 u32 n_present     32 u64 payload_bytes
  *           40 u64 wire_len 48 u32 cache_crc     52 u32 meta_crc   56 8 zero bytes
  *   chunk_dir[c]: u64 payload_off | u32 enc_len | u32 crc
  *   tile_tab[t] : 0 absent | 1 ZERO full tile (all bytes zero, no payload) |
  *                 258..511 PACK of 32*value bytes | 512 RAW full tile |
- *                 0xFFFF RAW partial tail tile
+ *                 0x8000 | n, n = 259..511: ENT of 32 n bytes | 0xFFFF RAW partial tail tile
  *   payload: encoded tiles of present chunks in ascending order, no padding.
  *
  * cache_crc is the CRC32C of the whole cache, obtained by combining the directory
@@ -334,9 +505,10 @@ static uint32_t encode_full_tile(const uint8_t* src, uint8_t* out, uint32_t* ent
  */
 #define WMO_FLAG_MASKED 1u       /* header flags: a dirty mask was given             */
 #define WMO_FLAG_ZERO_TILES 2u   /* header flags: all-zero tiles are table entries   */
+#define WMO_FLAG_ENTROPY 4u      /* header flags: ENT tiles instead of PACK tiles    */
 
 int wmo_encode_opt(const uint8_t* cache, uint64_t nbytes, uint32_t chunk_bytes, const uint8_t* dirty,
-                   uint32_t* crc_inout, uint8_t* wire, uint64_t wire_cap, int zero_tiles, wmo_result* res);
+                   uint32_t* crc_inout, uint8_t* wire, uint64_t wire_cap, int options, wmo_result* res);
 
 int wmo_encode(const uint8_t* cache, uint64_t nbytes, uint32_t chunk_bytes, const uint8_t* dirty,
                uint32_t* crc_inout, uint8_t* wire, uint64_t wire_cap, wmo_result* res)
@@ -344,9 +516,10 @@ int wmo_encode(const uint8_t* cache, uint64_t nbytes, uint32_t chunk_bytes, cons
     return wmo_encode_opt(cache, nbytes, chunk_bytes, dirty, crc_inout, wire, wire_cap, 0, res);
 }
 
-/* zero_tiles != 0: the ZERO tile option (tile table entry 1), recorded in header flags bit 1. */
+/* options: WMO_OPT_ZERO_TILES (tile table entry 1; header flags bit 1), WMO_OPT_ENTROPY (ENT tiles
+ * instead of PACK tiles; header flags bit 2). */
 int wmo_encode_opt(const uint8_t* cache, uint64_t nbytes, uint32_t chunk_bytes, const uint8_t* dirty,
-                   uint32_t* crc_inout, uint8_t* wire, uint64_t wire_cap, int zero_tiles, wmo_result* res)
+                   uint32_t* crc_inout, uint8_t* wire, uint64_t wire_cap, int options, wmo_result* res)
 {
     if (!cache || !crc_inout || !wire || !res || !args_ok(nbytes, chunk_bytes)) return WMO_ERR_ARG;
     uint64_t nc = wmo_num_chunks(nbytes, chunk_bytes), nt = wmo_num_tiles(nbytes);
@@ -357,7 +530,7 @@ int wmo_encode_opt(const uint8_t* cache, uint64_t nbytes, uint32_t chunk_bytes, 
 
     uint8_t* dir = wire + WMO_HEADER;
     uint8_t* tab = dir + 16u * nc;
-    uint8_t* tile_buf = (uint8_t*)malloc(WMO_TILE);
+    uint8_t* tile_buf = (uint8_t*)malloc(2 * WMO_TILE);     /* an ENT attempt may run past the tile size */
     uint64_t off = 0;              /* payload bytes emitted so far */
     uint32_t n_present = 0, cache_crc = 0;
     int overflow = 0;
@@ -375,7 +548,7 @@ int wmo_encode_opt(const uint8_t* cache, uint64_t nbytes, uint32_t chunk_bytes, 
                 uint64_t tlen = clen - o < WMO_TILE ? clen - o : WMO_TILE;
                 uint32_t entry, elen;
                 if (tlen < WMO_TILE) { memcpy(tile_buf, cp + o, tlen); entry = 0xFFFFu; elen = (uint32_t)tlen; }
-                else elen = encode_full_tile(cp + o, tile_buf, &entry, zero_tiles);
+                else elen = encode_full_tile(cp + o, tile_buf, &entry, options);
                 put16(tab + 2u * t, entry);
                 if (!overflow && meta_end + off + enc_len + elen <= wire_cap)
                     memcpy(wire + meta_end + off + enc_len, tile_buf, elen);
@@ -394,7 +567,8 @@ int wmo_encode_opt(const uint8_t* cache, uint64_t nbytes, uint32_t chunk_bytes, 
 
     memcpy(wire, "WMV1", 4);
     put16(wire + 4, 1);
-    put16(wire + 6, (dirty ? WMO_FLAG_MASKED : 0u) | (zero_tiles ? WMO_FLAG_ZERO_TILES : 0u));
+    put16(wire + 6, (dirty ? WMO_FLAG_MASKED : 0u) | ((options & WMO_OPT_ZERO_TILES) ? WMO_FLAG_ZERO_TILES : 0u) |
+                        ((options & WMO_OPT_ENTROPY) ? WMO_FLAG_ENTROPY : 0u));
     put64(wire + 8, nbytes);
     put32(wire + 16, chunk_bytes);
     put32(wire + 20, WMO_TILE);
@@ -457,7 +631,9 @@ static void decode_pack_tile(const uint8_t* in, uint8_t* dst)
  *  2 meta_crc                                                       -> META_CRC
  *  3 directory / tile-table structure                               -> STRUCT
  *  4 every PACK tile, in tile order: descriptors (w <= 8, check nibble) -> DESC,
- *    then 258 + sum w equals the tile entry                         -> STRUCT
+ *    then 258 + sum w equals the tile entry                         -> STRUCT;
+ *    every ENT tile: stream counts in range and adding up to the entry -> STRUCT,
+ *    then each stream used up exactly by its 1024 codewords, fill bits zero -> DESC
  *    (status of the lowest failing tile; n_bad_chunks = chunks with a failing tile)
  *  5 decode; CRC32C of each decoded chunk equals its directory CRC  -> CHUNK_CRC
  *  6 absent chunk: dst_crc_inout[c] equals its directory CRC        -> STALE
@@ -477,7 +653,7 @@ int wmo_decode_verify(const uint8_t* wire, uint64_t wire_len, uint8_t* dst, uint
 
     /* 1 */
     if (wire_len < WMO_HEADER || memcmp(wire, "WMV1", 4) != 0 || get16(wire + 4) != 1 ||
-        get16(wire + 6) > 3 || get64(wire + 8) != nbytes || get32(wire + 16) != chunk_bytes ||
+        get16(wire + 6) > 7 || get64(wire + 8) != nbytes || get32(wire + 16) != chunk_bytes ||
         get32(wire + 20) != WMO_TILE || get32(wire + 24) != nc || get64(wire + 40) != wire_len ||
         wire_len < meta_end || get64(wire + 32) != wire_len - meta_end) {
         fail(res, WMO_ERR_FORMAT, 0, 0);
@@ -485,6 +661,7 @@ int wmo_decode_verify(const uint8_t* wire, uint64_t wire_len, uint8_t* dst, uint
     }
     uint64_t payload_bytes = get64(wire + 32);
     int zero_ok = (get16(wire + 6) & 2u) != 0;      /* entry 1 is legal only in an image that declares the option */
+    int ent_on = (get16(wire + 6) & 4u) != 0;       /* ENT entries only with the flag, PACK entries only without */
     uint32_t n_present_hdr = get32(wire + 28);
     uint32_t cache_crc_hdr = get32(wire + 48);
     res->wire_len = wire_len; res->payload_bytes = payload_bytes;
@@ -521,7 +698,8 @@ int wmo_decode_verify(const uint8_t* wire, uint64_t wire_len, uint8_t* dst, uint
                 any = 1;
                 if (tlen < WMO_TILE) { if (e != 0xFFFFu) ok = 0; sum += tlen; }
                 else if (e == 1u && zero_ok) sum += 0;     /* ZERO tile: full tiles only, no payload */
-                else if (e >= 258u && e <= 512u) sum += 32u * (uint64_t)e;
+                else if (e == 512u || (!ent_on && e >= 258u && e <= 511u)) sum += 32u * (uint64_t)e;
+                else if (ent_on && e >= (0x8000u | 259u) && e <= (0x8000u | 511u)) sum += 32u * (uint64_t)(e & 0x7FFFu);
                 else ok = 0;
             }
             if (any && !all) ok = 0;                   /* a chunk is present as a whole or not at all */
@@ -545,8 +723,17 @@ int wmo_decode_verify(const uint8_t* wire, uint64_t wire_len, uint8_t* dst, uint
             for (uint64_t i = 0; i < ntc; i++) {
                 uint32_t e = get16(tab + 2u * (t0 + i));
                 if (e == 0) break;
-                uint64_t tlen = (e == 0xFFFFu) ? clen - i * WMO_TILE : (e == 1u) ? 0 : 32u * (uint64_t)e;
-                if (e >= 258u && e <= 511u) {
+                uint64_t tlen = (e == 0xFFFFu) ? clen - i * WMO_TILE : (e == 1u) ? 0 : 32u * (uint64_t)(e & 0x7FFFu);
+                if (e != 0xFFFFu && (e & 0x8000u)) {
+                    /* ENT tile: the header against the entry -> STRUCT, then every stream must be used up exactly -> DESC */
+                    int tile_status = WMO_OK;
+                    if (ent_header_bad(payload + off, e)) tile_status = WMO_ERR_STRUCT;
+                    else if (decode_ent_tile(payload + off, NULL)) tile_status = WMO_ERR_DESC;
+                    if (tile_status != WMO_OK) {
+                        chunk_bad = 1;
+                        if (status == WMO_OK) status = tile_status;
+                    }
+                } else if (e >= 258u && e <= 511u) {
                     const uint8_t* in = payload + off;
                     int tile_status = WMO_OK; uint32_t S = 0;
                     for (uint32_t g = 0; g < WMO_GROUPS_PER_TILE; g++) {
@@ -579,8 +766,9 @@ int wmo_decode_verify(const uint8_t* wire, uint64_t wire_len, uint8_t* dst, uint
             uint8_t* out = dst + c * (uint64_t)chunk_bytes;
             for (uint64_t i = 0; i < ntc; i++) {
                 uint32_t e = get16(tab + 2u * (t0 + i));
-                uint64_t tlen = (e == 0xFFFFu) ? clen - i * WMO_TILE : (e == 1u) ? 0 : 32u * (uint64_t)e;
+                uint64_t tlen = (e == 0xFFFFu) ? clen - i * WMO_TILE : (e == 1u) ? 0 : 32u * (uint64_t)(e & 0x7FFFu);
                 if (e == 1u) memset(out + i * WMO_TILE, 0, WMO_TILE);
+                else if (e != 0xFFFFu && (e & 0x8000u)) decode_ent_tile(payload + off, out + i * WMO_TILE);
                 else if (e == 512u || e == 0xFFFFu) memcpy(out + i * WMO_TILE, payload + off, tlen);
                 else decode_pack_tile(payload + off, out + i * WMO_TILE);
                 off += tlen;

@@ -1,0 +1,249 @@
+"""The ENT tile option of the oracle (entropy-coded exponents) against what the format fixes:
+hand-built tiles whose streams can be written down without running the coder, the completeness
+of the prefix code, Shannon's bound, round trips, and the decoder's verdicts on damaged tiles.
+"""
+import struct
+
+import numpy as np
+import pytest
+
+import oracle
+
+TILE = 16384
+META1 = 96            # one chunk of one tile: header 64 + directory 16 + table 2, rounded up to 32
+
+# the code as the format states it: u -> (bits in writing order)
+CODE = {0: "00", 1: "10", -1: "01", -2: "1100", 2: "1110", -3: "1101", -4: "11110", -5: "111110", 3: "1111110",
+        -6: "11111110"}
+ESC = "11111111"
+
+
+def _tile_of(value_u16):
+    return np.full(8192, value_u16, dtype="<u2")
+
+
+def _encode_one_tile(v):
+    wire, crc, res = oracle.encode(v.view(np.uint8), TILE, entropy=True)
+    assert res.status == 0 and oracle.meta_end(TILE, TILE) == META1
+    flags = struct.unpack_from("<H", wire, 6)[0]
+    entry = struct.unpack_from("<H", wire, 64 + 16)[0]
+    return wire, flags, entry, wire[META1:]
+
+
+def test_prefix_code_is_complete_and_prefix_free():
+    words = list(CODE.values()) + [ESC]
+    assert sum(2.0 ** -len(w) for w in words) == 1.0                      # Kraft with equality
+    for a in words:
+        for b in words:
+            assert a == b or not b.startswith(a)
+
+
+def test_constant_tile_by_hand():
+    """All elements 1.0 (0x3F80): every anchor is 127, every codeword is '00', a strand is 64 zero
+    bits = 4 halfwords, a share's stream 128 zero halfwords."""
+    wire, flags, entry, t = _encode_one_tile(_tile_of(0x3F80))
+    assert flags == 4 and entry == (0x8000 | 322) and t.size == 322 * 32 == 8256 + 8 * 128 * 2
+    want = np.zeros(322 * 32, dtype=np.uint8)
+    want[0:8] = 127
+    want[8:24] = np.full(8, 128, dtype="<u2").view(np.uint8)
+    assert np.array_equal(t, want)
+    out, _, r = oracle.decode_verify(wire, TILE, TILE)
+    assert r.status == 0 and np.array_equal(out.view("<u2"), _tile_of(0x3F80))
+
+
+def test_one_different_element_lands_where_the_format_says():
+    """Share 3, strand 5, element 7 of the strand is 2.0: u = +1, written '10' at bits 14-15 of the
+    strand's first halfword; with 2-bit codewords everywhere strand l takes its k-th halfword at
+    step 8 k, so that halfword is number 32 k + l of the share's stream."""
+    v = _tile_of(0x3F80)
+    elem = 64 * (16 * 3 + 7 // 2) + 2 * 5 + 7 % 2
+    v[elem] = 0x4000
+    wire, flags, entry, t = _encode_one_tile(v)
+    assert entry == (0x8000 | 322)
+    streams = t[8256:].view("<u2")
+    want = np.zeros(1024, dtype="<u2")
+    want[3 * 128 + 0 * 32 + 5] = 1 << 14
+    assert np.array_equal(streams[:1024], want)
+    sm = t[64:8256]
+    assert not sm.any()                                     # sign and mantissa bits are all zero
+    out, _, r = oracle.decode_verify(wire, TILE, TILE)
+    assert r.status == 0 and np.array_equal(out.view("<u2"), v)
+
+
+def test_a_strand_of_escapes_is_interleaved_as_the_reader_needs_it():
+    """Share 0, strand 0 holds 2^20 (E = 147), everything else 1.0 (E = 127): the share's mean is
+    127.6, anchor 128.  Strand 0 is 32 escapes of 16 bits (0xFF, then E), one halfword per step;
+    the other strands code u = -1 as '01', one halfword per 8 steps."""
+    v = _tile_of(0x3F80)
+    for i in range(32):
+        v[64 * (i // 2) + i % 2] = 147 << 7
+    wire, flags, entry, t = _encode_one_tile(v)
+    assert t[0] == 128 and list(t[1:8]) == [127] * 7
+    counts = t[8:24].view("<u2")
+    assert list(counts) == [32 + 31 * 4] + [128] * 7
+    s = t[8256:].view("<u2")
+    esc, m1 = 0xFF | (147 << 8), 0xAAAA                     # '01' eight times, LSB first
+    assert s[0] == esc and np.all(s[1:32] == m1)            # step 0: every strand, in order
+    assert np.all(s[32:39] == esc)                          # steps 1..7: strand 0 alone
+    assert s[39] == esc and np.all(s[40:71] == m1)          # step 8: strand 0, then the others' second halfword
+    assert np.all(s[71:78] == esc)                          # steps 9..15
+    assert np.all(s[156:156 + 128 * 7] == 0)                # shares 1..7: all '00'
+    out, _, r = oracle.decode_verify(wire, TILE, TILE)
+    assert r.status == 0 and np.array_equal(out.view("<u2"), v)
+
+
+def _gauss(n, seed, scale=1.0):
+    rng = np.random.default_rng(seed)
+    return ((rng.normal(size=n) * scale).astype(np.float32).view(np.uint32) >> 16).astype("<u2")
+
+
+def _strand_view(v):
+    """exponents as [tile, share, row, strand, half] -> [tile, share, strand, i]"""
+    E = ((v >> 7) & 0xFF).astype(np.int64).reshape(-1, 8, 16, 32, 2)
+    return E.transpose(0, 1, 3, 2, 4).reshape(E.shape[0], 8, 32, 32)
+
+
+def test_sizes_follow_the_code_lengths_and_respect_shannon():
+    v = np.concatenate([_gauss(8192 * 3, 5), _gauss(8192 * 2, 6, 37.0), _gauss(8192, 7, 1e-3)])
+    n_tiles = v.size // 8192
+    wire, crc, res = oracle.encode(v.view(np.uint8), 2 * TILE, entropy=True)
+    me = oracle.meta_end(v.size * 2, 2 * TILE)
+    entries = wire[64 + 16 * 3: 64 + 16 * 3 + 2 * n_tiles].view("<u2")
+    E = _strand_view(v)
+    anchor = (E.sum(axis=(2, 3)) + 512) >> 10
+    u = E - anchor[:, :, None, None]
+    L = np.full(u.shape, 16)
+    for k, w in CODE.items():
+        L[u == k] = len(w)
+    halfwords = -(-L.sum(axis=3) // 16)
+    want_len = (8256 + 2 * halfwords.sum(axis=(1, 2)) + 31) // 32 * 32
+    assert np.array_equal(entries.astype(np.int64), np.where(want_len < TILE, 0x8000 | (want_len // 32), 512))
+    assert res.wire_len == me + int(np.minimum(want_len, TILE).sum())
+    # no uniquely decodable code beats the empirical entropy of what it codes
+    for t in range(n_tiles):
+        for s in range(8):
+            c = np.bincount(E[t, s].ravel(), minlength=256).astype(float)
+            p = c[c > 0] / 1024.0
+            assert L[t, s].sum() >= 1024.0 * -(p * np.log2(p)).sum() - 1e-6
+    # and on Gaussian data it stays within half a bit of it on average, far below the plane packing
+    w_pack, _, r_pack = oracle.encode(v.view(np.uint8), 2 * TILE)
+    assert res.wire_len < 0.93 * r_pack.wire_len
+
+
+@pytest.mark.parametrize("n,chunk", [(5 * TILE + 300, 2 * TILE), (4 * TILE, 4 * TILE), (TILE - 2, TILE), (9 * TILE + 1, 4 * TILE)])
+def test_round_trip_masks_and_special_values(n, chunk):
+    rng = np.random.default_rng(n)
+    a = _gauss((n + 1) // 2, n).view(np.uint8)[:n].copy()
+    if n >= 2 * TILE:
+        a[TILE:2 * TILE] = rng.integers(0, 256, TILE, dtype=np.uint8)       # incompressible: stays raw
+        sp = a[:TILE].view("<u2")
+        sp[:6] = [0x7FC0, 0xFF80, 0x0001, 0x8000, 0x7F80, 0x0000]           # NaN, -Inf, denormal, -0, Inf, 0
+    nc = oracle.num_chunks(n, chunk)
+    wire, crc, res = oracle.encode(a, chunk, entropy=True)
+    assert res.status == 0 and np.array_equal(crc, oracle.checksum(a, chunk))
+    out, dcrc, r = oracle.decode_verify(wire, n, chunk)
+    assert r.status == 0 and np.array_equal(out, a) and np.array_equal(dcrc, crc)
+    if n >= 2 * TILE:
+        entries = wire[64 + 16 * nc: 64 + 16 * nc + 4].view("<u2")
+        assert entries[1] == 512 and entries[0] & 0x8000
+    # with a mask: absent chunks are trusted, the rest is coded the same way
+    dirty = (np.arange(nc) % 2 == 0).astype(np.uint8)
+    wire2, crc2, res2 = oracle.encode(a, chunk, dirty=dirty, crc_in=crc, entropy=True)
+    base = a.copy()
+    out2, _, r2 = oracle.decode_verify(wire2, n, chunk, dst=base, dst_crc=crc)
+    assert res2.status == 0 and r2.status == 0 and np.array_equal(out2, a)
+    assert struct.unpack_from("<H", wire2, 6)[0] == 5
+    # both options together: a zero tile is an entry, the rest ENT
+    if n >= 3 * TILE:
+        z = a.copy()
+        z[2 * TILE:3 * TILE] = 0
+        wz, _, rz = oracle.encode(z, chunk, zero_tiles=True, entropy=True)
+        oz, _, rdz = oracle.decode_verify(wz, n, chunk)
+        assert rz.status == 0 and rdz.status == 0 and np.array_equal(oz, z)
+        assert struct.unpack_from("<H", wz, 64 + 16 * nc + 4)[0] == 1 and struct.unpack_from("<H", wz, 6)[0] == 6
+
+
+def _reseal(w, n, chunk):
+    me = oracle.meta_end(n, chunk)
+    z = w[:me].copy()
+    z[52:56] = 0
+    w[52:56] = np.frombuffer(struct.pack("<I", oracle.crc32c(z)), dtype=np.uint8)
+    return w
+
+
+def test_damaged_ent_tiles_are_refused_with_the_right_status():
+    n, chunk = 4 * TILE, 2 * TILE
+    a = _gauss(n // 2, 21).view(np.uint8)
+    wire, crc, res = oracle.encode(a, chunk, entropy=True)
+    me = oracle.meta_end(n, chunk)
+    entries = wire[64 + 16 * 2: 64 + 16 * 2 + 8].view("<u2")
+    len0 = 32 * int(entries[0] & 0x7FFF)
+    # a count that no longer adds up to the entry: structure
+    w = wire.copy()
+    w[me + 8] ^= 16                       # 16 halfwords = one 32-byte unit
+    assert oracle.decode_verify(w, n, chunk)[2].status_name == "ERR_STRUCT"
+    # counts moved between shares (sum unchanged): the streams are no longer used up exactly
+    w = wire.copy()
+    c = w[me + 8: me + 24].view("<u2")
+    c[0] += 1
+    c[1] -= 1
+    r = oracle.decode_verify(w, n, chunk)[2]
+    assert r.status_name == "ERR_DESC" and r.first_bad_chunk == 0 and r.n_bad_chunks == 1
+    # in the second tile of the second chunk: lowest failing tile decides, chunk 1 is reported
+    w = wire.copy()
+    off = me + len0 + 32 * int(entries[1] & 0x7FFF) + 32 * int(entries[2] & 0x7FFF)
+    c = w[off + 8: off + 24].view("<u2")
+    c[6] += 2
+    c[7] -= 2
+    r = oracle.decode_verify(w, n, chunk)[2]
+    assert r.status_name == "ERR_DESC" and r.first_bad_chunk == 1
+    # a flipped bit inside a stream: either the streams no longer fit (DESC) or the bytes differ (CHUNK_CRC)
+    seen = set()
+    for k in range(0, 600, 7):
+        w = wire.copy()
+        w[me + 8256 + k] ^= 1 << (k % 8)
+        seen.add(oracle.decode_verify(w, n, chunk)[2].status_name)
+    assert seen <= {"ERR_DESC", "ERR_CHUNK_CRC"} and "ERR_CHUNK_CRC" in seen
+    # an ENT entry in an image that does not declare the option, and a PACK entry in one that does
+    w = wire.copy()
+    w[6] = 0
+    assert oracle.decode_verify(_reseal(w, n, chunk), n, chunk)[2].status_name == "ERR_STRUCT"
+    wp, _, _ = oracle.encode(a, chunk)
+    wp = wp.copy()
+    wp[6] = 4
+    assert oracle.decode_verify(_reseal(wp, n, chunk), n, chunk)[2].status_name == "ERR_STRUCT"
+    # flags above 7 are no format this decoder knows
+    w = wire.copy()
+    w[6] = 12
+    assert oracle.decode_verify(_reseal(w, n, chunk), n, chunk)[2].status_name == "ERR_FORMAT"
+
+
+def test_default_images_are_unchanged_by_the_option():
+    a = _gauss(3 * 8192, 31).view(np.uint8)
+    w0, _, r0 = oracle.encode(a, TILE)
+    assert struct.unpack_from("<H", w0, 6)[0] == 0 and not (w0[64 + 48: 64 + 48 + 6].view("<u2") & 0x8000).any()
+
+
+def test_every_codeword_bit_by_bit():
+    """Share 0, strand 0 starts with one element for each coded u (in the table's order), all else
+    is E = 127.  The strand's bit string is the codewords as the format lists them; where its six
+    halfwords sit in the stream follows from when it runs out of bits (steps 0, 5, 8, 12, 20, 28)
+    against the other strands' steps 0, 8, 16, 24."""
+    us = [0, 1, -1, -2, 2, -3, -4, -5, 3, -6]
+    v = _tile_of(0x3F80)
+    for i, u in enumerate(us):
+        v[64 * (i // 2) + i % 2] = (127 + u) << 7
+    wire, flags, entry, t = _encode_one_tile(v)
+    assert t[0] == 127
+    bits = "".join(CODE[u] for u in us) + "00" * 22
+    assert len(bits) == 88
+    bits += "0" * 8
+    hw = [sum(int(bits[16 * k + b]) << b for b in range(16)) for k in range(6)]
+    s = t[8256:].view("<u2")
+    assert struct.unpack_from("<H", t, 8)[0] == 6 + 31 * 4
+    where = [0, 32, 33, 65, 97, 129]
+    assert [int(s[i]) for i in where] == hw
+    others = np.delete(s[:130], where)
+    assert not others.any()
+    out, _, r = oracle.decode_verify(wire, TILE, TILE)
+    assert r.status == 0 and np.array_equal(out.view("<u2"), v)
