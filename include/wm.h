@@ -216,6 +216,33 @@ wm_status wm_decode_verify_strict(const void* wire, uint64_t wire_len, void* dst
 void wm_zero_tiles_enable(int on);
 
 /*
+ * wm_entropy_enable - codec option: entropy-coded exponents (ENT tiles instead of PACK tiles).
+ * Paper: the codec it measured entropy-codes the exponent plane inside the verified envelope
+ * (Section 6.4); the bit-plane packing of the default format stops at a fixed number of bits
+ * per group.  With the option on, wm_encode / wm_encode_leaves store a full tile of a present
+ * chunk as an ENT tile or raw, and set header flags bit 2; the wm_decode_verify family then
+ * expects such images.  A decode call whose option differs from the image's flag returns
+ * WM_ERR_FORMAT.  While this option is on, the zero-tile option is ignored.  Process-wide, off
+ * by default; set it on both ends of a move before the calls are issued.
+ *
+ * ENT tile (entry 0x8000 | length / 32 in the tile table, length < 16384, else the tile is raw):
+ *   a tile is eight shares of 16 rows (row = 128 bytes); share s has 32 strands, strand l = the 32
+ *   elements at 32-bit word l of the share's rows, row after row, low half first.
+ *   anchor_s = (sum of the share's 1024 exponents + 512) >> 10.  u = E - anchor_s is coded
+ *       u:    0   +1   -1   -2    +2    -3    -4     -5      +3       -6        other
+ *       bits: 00  10   01   1100  1110  1101  11110  111110  1111110  11111110  11111111 + E (8 bits, low first)
+ *   (in writing order; a strand is an LSB-first bit string, zero-filled to whole 16-bit halfwords).
+ *   A share's strands are interleaved into one stream in the order a reader needs them: at step
+ *   i = 0..31 every strand whose codeword i is not complete in the halfwords it has taken so far
+ *   takes the stream's next halfword, strands in ascending order.
+ *   Layout: anchor[8] u8 | count[8] u16 (halfwords per stream) | 40 zero bytes | SM[8192] as in
+ *   a PACK tile | the eight streams | zero fill to a multiple of 32 bytes.
+ * Decode checks (step 4): counts within 128..1024 and adding up to the entry (else WM_ERR_STRUCT);
+ * every stream used up exactly and the fill bits of every strand zero (else WM_ERR_DESC).
+ */
+void wm_entropy_enable(int on);
+
+/*
  * Leaf mode - the cache as the engine holds it: a list of tensors, not one buffer.
  * Paper: the mover flattens the live cache before the transfer and rehydrates it after
  * (Section 1 and Section 4.1: flatten, transfer, CRC-verify, rehydrate; Section 5: the movable

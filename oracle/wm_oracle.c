@@ -643,8 +643,19 @@ static void decode_pack_tile(const uint8_t* in, uint8_t* dst)
  * contents of dst are unspecified (bounded to [dst, dst+nbytes)) and dst_crc_inout
  * is unchanged; the caller must not install dst.
  */
+int wmo_decode_verify_opt(const uint8_t* wire, uint64_t wire_len, uint8_t* dst, uint64_t nbytes,
+                          uint32_t chunk_bytes, uint32_t* dst_crc_inout, int expect_entropy, wmo_result* res);
+
 int wmo_decode_verify(const uint8_t* wire, uint64_t wire_len, uint8_t* dst, uint64_t nbytes,
                       uint32_t chunk_bytes, uint32_t* dst_crc_inout, wmo_result* res)
+{
+    return wmo_decode_verify_opt(wire, wire_len, dst, nbytes, chunk_bytes, dst_crc_inout, -1, res);
+}
+
+/* expect_entropy: -1 accepts both kinds of image; 0 / 1: a receiver that was told which codec
+ * option the sender uses treats an image of the other kind as a format error (step 1). */
+int wmo_decode_verify_opt(const uint8_t* wire, uint64_t wire_len, uint8_t* dst, uint64_t nbytes,
+                          uint32_t chunk_bytes, uint32_t* dst_crc_inout, int expect_entropy, wmo_result* res)
 {
     if (!wire || !dst || !dst_crc_inout || !res || !args_ok(nbytes, chunk_bytes)) return WMO_ERR_ARG;
     memset(res, 0, sizeof *res);
@@ -653,7 +664,8 @@ int wmo_decode_verify(const uint8_t* wire, uint64_t wire_len, uint8_t* dst, uint
 
     /* 1 */
     if (wire_len < WMO_HEADER || memcmp(wire, "WMV1", 4) != 0 || get16(wire + 4) != 1 ||
-        get16(wire + 6) > 7 || get64(wire + 8) != nbytes || get32(wire + 16) != chunk_bytes ||
+        get16(wire + 6) > 7 || (expect_entropy >= 0 && (int)((get16(wire + 6) >> 2) & 1u) != expect_entropy) ||
+        get64(wire + 8) != nbytes || get32(wire + 16) != chunk_bytes ||
         get32(wire + 20) != WMO_TILE || get32(wire + 24) != nc || get64(wire + 40) != wire_len ||
         wire_len < meta_end || get64(wire + 32) != wire_len - meta_end) {
         fail(res, WMO_ERR_FORMAT, 0, 0);

@@ -89,6 +89,8 @@ def _load():
     lib.wmo_encode_opt.argtypes = [u8p, u64, u32, u8p, u32p, u8p, u64, ctypes.c_int, ctypes.POINTER(_CResult)]
     lib.wmo_decode_verify.restype = ctypes.c_int
     lib.wmo_decode_verify.argtypes = [u8p, u64, u8p, u64, u32, u32p, ctypes.POINTER(_CResult)]
+    lib.wmo_decode_verify_opt.restype = ctypes.c_int
+    lib.wmo_decode_verify_opt.argtypes = [u8p, u64, u8p, u64, u32, u32p, ctypes.c_int, ctypes.POINTER(_CResult)]
     _lib = lib
     return lib
 
@@ -191,16 +193,20 @@ def encode(cache, chunk_bytes: int, dirty=None, crc_in=None, wire_cap: int | Non
     return wire, crc, r
 
 
-def decode_verify(wire, nbytes: int, chunk_bytes: int, dst=None, dst_crc=None, wire_len: int | None = None):
+def decode_verify(wire, nbytes: int, chunk_bytes: int, dst=None, dst_crc=None, wire_len: int | None = None,
+                  expect_entropy: bool | None = None):
     """Return (dst u8[nbytes], dst_crc u32[n_chunks], Result).  ``dst`` and ``dst_crc`` are
-    copied first, so the caller's arrays play the part of the live state and stay untouched."""
+    copied first, so the caller's arrays play the part of the live state and stay untouched.
+    ``expect_entropy``: None accepts images with and without ENT tiles; True / False is a receiver
+    that knows the sender's option and refuses the other kind as a format error."""
     w = _bytes_view(wire)
     nc = num_chunks(nbytes, chunk_bytes)
     out = np.zeros(nbytes, dtype=np.uint8) if dst is None else _bytes_view(dst).copy()
     crc = np.zeros(nc, dtype=np.uint32) if dst_crc is None else np.array(dst_crc, dtype=np.uint32).copy()
     res = _CResult()
-    st = _load().wmo_decode_verify(_ptr(w), w.size if wire_len is None else int(wire_len), _ptr(out),
-                                   nbytes, chunk_bytes, _ptr(crc), ctypes.byref(res))
+    st = _load().wmo_decode_verify_opt(_ptr(w), w.size if wire_len is None else int(wire_len), _ptr(out),
+                                       nbytes, chunk_bytes, _ptr(crc),
+                                       -1 if expect_entropy is None else int(bool(expect_entropy)), ctypes.byref(res))
     _check(st, "decode_verify")
     return out, crc, _result(res)
 

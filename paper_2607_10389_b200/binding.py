@@ -24,7 +24,7 @@ RESULT_BYTES = 40
 EXPORTS = ("wm_num_chunks", "wm_num_tiles", "wm_meta_bytes", "wm_wire_bound", "wm_workspace_bytes",
            "wm_checksum", "wm_dirty_diff", "wm_encode", "wm_decode_verify", "wm_last_launch_count",
            "wm_timing_enable", "wm_timing_read_ms", "wm_checksum_noalloc", "wm_encode_leaves",
-           "wm_decode_verify_leaves", "wm_zero_tiles_enable", "wm_decode_verify_strict", "wm_checksum_poly")
+           "wm_decode_verify_leaves", "wm_zero_tiles_enable", "wm_decode_verify_strict", "wm_checksum_poly", "wm_entropy_enable")
 
 
 class WmError(RuntimeError):
@@ -50,6 +50,8 @@ def load_library() -> ctypes.CDLL:
     lib.wm_timing_enable.argtypes = [ctypes.c_int]
     lib.wm_zero_tiles_enable.restype = None
     lib.wm_zero_tiles_enable.argtypes = [ctypes.c_int]
+    lib.wm_entropy_enable.restype = None
+    lib.wm_entropy_enable.argtypes = [ctypes.c_int]
     lib.wm_timing_read_ms.restype = ctypes.c_int
     lib.wm_timing_read_ms.argtypes = [ctypes.c_int, ctypes.POINTER(ctypes.c_float)]
     lib.wm_checksum.restype = ctypes.c_int
@@ -146,6 +148,12 @@ def zero_tiles_enable(on: bool) -> None:
     lib().wm_zero_tiles_enable(1 if on else 0)
 
 
+def entropy_enable(on: bool) -> None:
+    """Codec option: entropy-coded exponents (ENT tiles).  Applies to the encode calls (what they
+    write) and to the decode calls (what they expect) of this process."""
+    lib().wm_entropy_enable(1 if on else 0)
+
+
 def timing_read_ms(kind: int) -> float:
     ms = ctypes.c_float(0.0)
     _check(lib().wm_timing_read_ms(kind, ctypes.byref(ms)), "wm_timing_read_ms")
@@ -198,7 +206,7 @@ def wm_checksum_poly(cache: torch.Tensor, chunk_bytes: int, polynomial: int, crc
     _dev_u8(cache, "cache")
     nbytes = cache.numel() * cache.element_size()
     _check(lib().wm_checksum_poly(cache.data_ptr(), nbytes, chunk_bytes, int(polynomial), crc_out.data_ptr(),
-                                  workspace.data_ptr(), workspace.numel(), _stream(stream)), "wm_checksum_poly")
+                                  workspace.data_ptr(), workspace.numel(), _stream(stream)), "wm_checksum_poly", "wm_entropy_enable")
 
 
 NOALLOC_MAX_BYTES = 4 << 30

@@ -838,6 +838,63 @@ __device__ __forceinline__ void pack_group_planes(uint32_t e4a, uint32_t e4b, ui
     }
 }
 
+
+// ---- ENT tiles: entropy-coded exponents (an encoder option; header flags bit 2) --------------
+// A warp's 2 KiB of a tile (16 rows) is one share; lane l's 32 elements (its 16 words, low half
+// first) are strand l.  Every exponent is coded as u = E - anchor with a fixed prefix code, the
+// anchor being the rounded mean of the share's exponents; a strand is an LSB-first bit string
+// cut into halfwords, and the 32 strands of a share are interleaved in the order a reader
+// needs them: at step i every strand whose codeword i is not complete in what it has taken so
+// far takes the stream's next halfword, strands in ascending order.
+//   u        -6  -5  -4  -3  -2  -1   0   1   2   3   other
+//   length    8   6   5   4   4   2   2   2   4   7   16 (eight ones, then E itself)
+//   bits    127  31  15  11   3   2   0   1   7  63   255 | E << 8        (first bit = bit 0)
+// ent_slot: 0..9 for u = -6..3, 10 for everything else.
+__device__ __forceinline__ uint32_t ent_slot(uint32_t E, uint32_t anchor)
+{
+    return min(E - anchor + 6u, 10u);
+}
+__device__ __forceinline__ uint32_t ent_length(uint32_t slot)
+{
+    // (length - 1) per slot, four bits each: 7 5 4 3 3 1 1 1 3 6 15
+    return (uint32_t)((0xF6311133457ull >> (4u * slot)) & 15ull) + 1u;
+}
+__device__ __forceinline__ uint32_t ent_word(uint32_t slot, uint32_t E)
+{
+    if (slot >= 10u) return 255u | (E << 8);
+    if (slot >= 8u) return slot == 8u ? 7u : 63u;
+    return __byte_perm(0x0B0F1F7Fu, 0x01000203u, slot) & 0xFFu;
+}
+// Bytes of an ENT tile whose eight streams hold `halfwords` halfwords in all (a multiple of 32;
+// 16384 or more means that the tile is stored raw instead).
+__device__ __forceinline__ uint32_t ent_tile_bytes(uint32_t halfwords)
+{
+    return (8256u + 2u * halfwords + 31u) & ~31u;
+}
+// Decoder side: length of the codeword at the low end of `buf` (zero beyond the valid bits).
+__device__ __forceinline__ uint32_t ent_parse_length(uint32_t buf)
+{
+    if ((buf & 3u) != 3u) return 2u;
+    if ((buf & 12u) != 12u) return 4u;
+    const uint32_t k = __ffs(~(buf >> 4)) - 1u;          // ones after the four
+    return k < 4u ? 5u + k : 16u;
+}
+// ... and the exponent it stands for.
+__device__ __forceinline__ uint32_t ent_parse_value(uint32_t buf, uint32_t anchor)
+{
+    uint32_t u;
+    if ((buf & 3u) != 3u) {
+        u = (0xFF0100u >> (8u * (buf & 3u))) & 0xFFu;                 // 0, +1, -1
+    } else if ((buf & 12u) != 12u) {
+        u = (0xFD02FEu >> (8u * ((buf >> 2) & 3u))) & 0xFFu;          // -2, +2, -3
+    } else {
+        const uint32_t k = __ffs(~(buf >> 4)) - 1u;
+        if (k >= 4u) return (buf >> 8) & 0xFFu;
+        u = (0xFA03FBFCu >> (8u * k)) & 0xFFu;                        // -4, -5, +3, -6
+    }
+    return (anchor + u) & 0xFFu;
+}
+
 // Single-pass fused checksum + encode.  Each team keeps four tiles in flight:
 //     X  measured three steps ago, packed and written to the wire image in this step
 //     V, W  measured two / one steps ago, waiting for their offsets
@@ -880,7 +937,7 @@ __device__ __forceinline__ uint32_t describe_tile(const Geo& g, const uint8_t* _
     return q;
 }
 
-template <int TEAMS, bool MASKED, bool LEAVES, bool ZEROS>
+template <int TEAMS, bool MASKED, bool LEAVES, bool ZEROS, bool ENT = false>
 __global__ void __launch_bounds__(TEAMS * 256, 1)
 k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restrict__ dirty,
          unsigned char* __restrict__ wire, uint64_t wire_cap, Ws ws, const Tables* __restrict__ tab)
@@ -1019,6 +1076,21 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
 #pragma unroll
             for (int i = 0; i < 16; i++) d[i] = __funnelshift_l(d[i], d[i], 1);
             uint32_t gw[4];               // per group: base | width << 8
+            if (ENT) {
+                // the share's anchor (rounded mean of its 1024 exponents: bytes 1 and 3 of a rotated
+                // word) and the halfwords its 32 strands need
+                uint32_t acc = 0;
+#pragma unroll
+                for (int i = 0; i < 16; i++) acc += (d[i] >> 8) & 0x00FF00FFu;
+                const uint32_t anchor = (__reduce_add_sync(0xFFFFFFFFu, (acc & 0xFFFFu) + (acc >> 16)) + 512u) >> 10;
+                uint32_t bits = 0;
+#pragma unroll
+                for (int i = 0; i < 16; i++)
+                    bits += ent_length(ent_slot((d[i] >> 8) & 0xFFu, anchor)) + ent_length(ent_slot(d[i] >> 24, anchor));
+                const uint32_t count = __reduce_add_sync(0xFFFFFFFFu, (bits + 15u) >> 4);
+                gw[0] = anchor | (count << 8);
+                gw[1] = gw[2] = gw[3] = 0u;
+            } else {
 #ifdef WM_AB_NOMINMAX
             gw[0] = gw[1] = gw[2] = gw[3] = 100u | (4u << 8);
 #else
@@ -1036,6 +1108,7 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
                 gw[j] = emin | ((32u - __clz(emax - emin)) << 8);
             }
 #endif
+            }
             // Option ZEROS.  Unused memory: when all four groups have exponent 0 throughout (rare in live data)
             // look at the words themselves; a warp whose 2 KiB are all zero marks its first entry.
             if (ZEROS && (gw[0] | gw[1] | gw[2] | gw[3]) == 0u) {
@@ -1058,13 +1131,15 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
                 // (kept short: this warp is the one the team's length waits for; the groups'
                 // places inside the tile are worked out by each warp when it packs)
                 const uint32_t wt = *reinterpret_cast<volatile uint32_t*>(&tc->wtab[slY][lane]);
-                const uint32_t total = __reduce_add_sync(0xFFFFFFFFu, (wt >> 8) & 15u);
+                // (ENT: every warp's first entry carries its stream's halfwords, the other three are zero)
+                const uint32_t total = __reduce_add_sync(0xFFFFFFFFu, ENT ? wt >> 8 : (wt >> 8) & 15u);
                 // unused memory (every warp's first entry carries the mark): no payload
                 const bool zero_tile = ZEROS && __all_sync(0xFFFFFFFFu, (lane & 3u) != 0u || (wt & kWarpAllZero) != 0u);
                 if (lane == 0) {
                     tc->ssum[slY] = zero_tile ? kSumZeroTile : total;
                     tc->wsum[slY] = 0;
-                    publish_len(tYn, zero_tile ? 0u : total <= 253u ? 8256u + 32u * total : kTile);
+                    if (ENT) publish_len(tYn, ent_tile_bytes(total) < kTile ? ent_tile_bytes(total) : kTile);
+                    else publish_len(tYn, zero_tile ? 0u : total <= 253u ? 8256u + 32u * total : kTile);
                 }
             }
 #ifndef WM_AB_NOTMEM
@@ -1088,12 +1163,59 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
             tmem_load16(tmem_warp + 16u * ((step + 1u) & 3u), d);
 #endif
             const uint32_t Ssum = tc->ssum[sl];
-            const bool packs = Ssum <= 253u;
+            const bool packs = ENT ? ent_tile_bytes(Ssum) < kTile : Ssum <= 253u;
             // (a tile of all-zero bytes, marked in ssum, is its table entry and nothing else)
-            const uint32_t enc_len = packs ? 8256u + 32u * Ssum : (ZEROS && Ssum == kSumZeroTile) ? 0u : kTile;
+            const uint32_t enc_len = ENT ? (packs ? ent_tile_bytes(Ssum) : kTile)
+                                         : packs ? 8256u + 32u * Ssum : (ZEROS && Ssum == kSumZeroTile) ? 0u : kTile;
             unsigned char* const dst = payload + exclX;
             if (exclX + enc_len > room) {
                 trouble |= 1u;
+            } else if (ENT && packs) {
+                // header: anchors, stream lengths, 40 zero bytes; zero fill behind the last stream
+                if (warp == 5) {
+                    if (lane < 8u) {
+                        const uint32_t wt = tc->wtab[sl][4u * lane];
+                        stg_u8(dst + lane, wt & 0xFFu);
+                        stg_u16(dst + 8u + 2u * lane, wt >> 8);
+                    } else if (lane < 18u) {
+                        st_stream_u32(dst + 24u + 4u * (lane - 8u), 0u);
+                    }
+                    if (2u * lane < enc_len - 8256u - 2u * Ssum) stg_u16(dst + 8256u + 2u * Ssum + 2u * lane, 0u);
+                }
+                unsigned char* const sm_dst = dst + sm_off;
+#pragma unroll
+                for (int j = 0; j < 4; j++) {
+                    const uint32_t sa = __byte_perm(d[4 * j], d[4 * j + 1], 0x6420), sb = __byte_perm(d[4 * j + 2], d[4 * j + 3], 0x6420);
+                    const uint32_t ya = __byte_perm(sa, sa, 0x2301), yb = __byte_perm(sb, sb, 0x2301);
+                    stg_v2(sm_dst + 256 * j, (sa & 0xFEFEFEFEu) | (ya & 0x01010101u), (sb & 0xFEFEFEFEu) | (yb & 0x01010101u));
+                }
+                // this share's stream: it starts behind the streams of the warps before it
+                const uint32_t wall = tc->wtab[sl][lane] >> 8;
+                const uint32_t before = __reduce_add_sync(0xFFFFFFFFu, lane < 4u * warp ? wall : 0u);
+                const uint32_t anchor = tc->wtab[sl][4u * warp] & 0xFFu;
+                unsigned char* const hw_dst = dst + 8256u + 2u * before;
+                const uint32_t lt_mask = (1u << lane) - 1u;
+                // acc: the strand's bits from the start of the halfword it took last (number `pend` of
+                // the stream) on; n of them are valid.  Step 0: every strand takes one halfword.
+                uint32_t acc = 0, n = 0, pend = lane, pos = 32;
+#pragma unroll
+                for (int i = 0; i < 32; i++) {
+                    const uint32_t E = (i & 1) ? d[i >> 1] >> 24 : (d[i >> 1] >> 8) & 0xFFu;
+                    const uint32_t slot = ent_slot(E, anchor);
+                    acc |= ent_word(slot, E) << n;
+                    n += ent_length(slot);
+                    if (i == 0) continue;
+                    const bool more = n > 16u;             // the codeword runs past what the strand has taken
+                    const uint32_t takers = __ballot_sync(0xFFFFFFFFu, more);
+                    if (more) {
+                        stg_u16(hw_dst + 2u * pend, acc & 0xFFFFu);
+                        acc >>= 16;
+                        n -= 16u;
+                        pend = pos + __popc(takers & lt_mask);
+                    }
+                    pos += __popc(takers);
+                }
+                stg_u16(hw_dst + 2u * pend, acc & 0xFFFFu);
             } else if (packs) {
 #ifndef WM_AB_NOPACK
                 if (warp == 5) {           // (any one warp: not one that has a single-lane chore)
@@ -1160,8 +1282,14 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
             if (qX >= kQPresent) {
                 if (tXn < g.n_full_tiles) {
                     const uint32_t Ssum = tc->ssum[sl];
-                    entry = Ssum <= 253u ? 258u + Ssum : (ZEROS && Ssum == kSumZeroTile) ? 1u : 512u;
-                    enc_len = (ZEROS && entry == 1u) ? 0u : 32u * entry;
+                    if (ENT) {
+                        const uint32_t nb = ent_tile_bytes(Ssum);
+                        entry = nb < kTile ? 0x8000u | (nb / 32u) : 512u;
+                        enc_len = nb < kTile ? nb : kTile;
+                    } else {
+                        entry = Ssum <= 253u ? 258u + Ssum : (ZEROS && Ssum == kSumZeroTile) ? 1u : 512u;
+                        enc_len = (ZEROS && entry == 1u) ? 0u : 32u * entry;
+                    }
                 } else {
                     entry = 0xFFFFu;
                     enc_len = tile_left(g, tXn);
@@ -1211,7 +1339,7 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
 __global__ void __launch_bounds__(1024)
 k_encode_finish(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restrict__ dirty,
                 uint32_t* __restrict__ crc_inout, unsigned char* __restrict__ wire, Ws ws,
-                const Tables* __restrict__ tab, const __grid_constant__ ChunkPowers cp, uint32_t zero_tiles)
+                const Tables* __restrict__ tab, const __grid_constant__ ChunkPowers cp, uint32_t option_flags)
 {
     __shared__ uint32_t sHT[1024];
     __shared__ uint32_t sT0[256];
@@ -1260,7 +1388,7 @@ k_encode_finish(const unsigned char* __restrict__ cache, Geo g, const uint8_t* _
     const uint32_t n_present = ld_volatile_u32(&ws.ctrl->n_present);
     uint32_t* h = reinterpret_cast<uint32_t*>(wire);
     h[0] = 0x31564D57u;                                  // "WMV1"
-    h[1] = 1u | ((dirty ? 1u : 0u) << 16) | ((zero_tiles ? 2u : 0u) << 16);      // version, flags
+    h[1] = 1u | ((dirty ? 1u : 0u) << 16) | (option_flags << 16);      // version, flags (bit 1 zero tiles, bit 2 ENT tiles)
     h[2] = (uint32_t)g.nbytes; h[3] = (uint32_t)(g.nbytes >> 32);
     h[4] = g.chunk_bytes; h[5] = kTile; h[6] = g.n_chunks; h[7] = n_present;
     h[8] = (uint32_t)total; h[9] = (uint32_t)(total >> 32);
@@ -1279,14 +1407,14 @@ k_encode_finish(const unsigned char* __restrict__ cache, Geo g, const uint8_t* _
 // kernels see a few hundred kilobytes: they use the small tables.
 
 // The header against the call's arguments (decode step 1).
-__device__ __forceinline__ bool header_matches(const unsigned char* wire, uint64_t wire_len, const Geo& g)
+__device__ __forceinline__ bool header_matches(const unsigned char* wire, uint64_t wire_len, const Geo& g, uint32_t expect_ent)
 {
     if (wire_len < 64) return false;
     const uint32_t* h = reinterpret_cast<const uint32_t*>(wire);
     const unsigned long long nb = h[2] | ((unsigned long long)h[3] << 32);
     const unsigned long long pb = h[8] | ((unsigned long long)h[9] << 32);
     const unsigned long long wl = h[10] | ((unsigned long long)h[11] << 32);
-    return !(h[0] != 0x31564D57u || (h[1] & 0xFFFFu) != 1u || (h[1] >> 16) > 3u || nb != g.nbytes ||
+    return !(h[0] != 0x31564D57u || (h[1] & 0xFFFFu) != 1u || (h[1] >> 16) > 7u || ((h[1] >> 18) & 1u) != expect_ent || nb != g.nbytes ||
              h[4] != g.chunk_bytes || h[5] != kTile || h[6] != g.n_chunks || wl != wire_len ||
              wire_len < g.meta_end || pb != wire_len - g.meta_end);
 }
@@ -1433,7 +1561,7 @@ __device__ __forceinline__ void fill_result(wm_result* result, const Ctrl* ctrl,
 // once (WM_ERR_FORMAT).  A failure sets the gate that keeps the later kernels out.
 __global__ void __launch_bounds__(1024)
 k_decode_check(const unsigned char* __restrict__ wire, uint64_t wire_len, Geo g, Ws ws,
-               const Tables* __restrict__ tab, wm_result* result, uint32_t meta_blocks)
+               const Tables* __restrict__ tab, wm_result* result, uint32_t meta_blocks, uint32_t expect_ent)
 {
     __shared__ uint32_t sG[1024];
     __shared__ uint32_t sHT[1024];
@@ -1450,7 +1578,7 @@ k_decode_check(const unsigned char* __restrict__ wire, uint64_t wire_len, Geo g,
     grid_dep_wait();
     grid_dep_launch();
     if (ld_volatile_u32(&ws.ctrl->gate)) return;        // leaf mode: the destination table was rejected
-    if (threadIdx.x == 0) s_format_bad = header_matches(wire, wire_len, g) ? 0 : 1;
+    if (threadIdx.x == 0) s_format_bad = header_matches(wire, wire_len, g, expect_ent) ? 0 : 1;
     __syncthreads();
     if (s_format_bad) {
         if (blockIdx.x == 0 && threadIdx.x == 0) {
@@ -1492,7 +1620,8 @@ k_decode_check(const unsigned char* __restrict__ wire, uint64_t wire_len, Geo g,
                         l_any = true;
                         if (tl < kTile) { if (e != 0xFFFFu) l_ok = false; len = (uint32_t)tl; }
                         else if (e == 1u && zero_ok) len = 0;       // a tile of zeros: no payload
-                        else if (e >= 258u && e <= 512u) len = 32u * e;
+                        else if (e == 512u || (!expect_ent && e >= 258u && e <= 511u)) len = 32u * e;
+                        else if (expect_ent && e >= (0x8000u | 259u) && e <= (0x8000u | 511u)) len = 32u * (e & 0x7FFFu);   // ENT tile
                         else l_ok = false;
                     }
                 }
@@ -1683,7 +1812,7 @@ __device__ __forceinline__ void unpack_group_planes(const PlaneWords& pw, uint32
 // the pace of its slowest one.)  LEAVES: the decoded tiles go to a table of tensors.
 // MODE 0: unpack, store, checksum (the normal call).  Strict calls run the kernel twice: MODE 1
 // unpacks and checksums without storing anything; MODE 2, after the verdict, unpacks and stores.
-template <int TEAMS, bool LEAVES, int MODE>
+template <int TEAMS, bool LEAVES, int MODE, bool ENT = false>
 __global__ void __launch_bounds__(TEAMS * 256, 1)
 k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restrict__ dst, Ws ws,
          const Tables* __restrict__ tab)
@@ -1722,9 +1851,11 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
         }
     };
     // staged tiles: full RAW and PACK tiles (everything except absent tiles and the ragged tail)
+    // (ENT images: raw tiles and ENT tiles, entry 0x8000 | length / 32)
+    auto is_staged = [](uint32_t e) { return ENT ? (e == 512u || (e > 0x8000u && e != 0xFFFFu)) : (e >= 258u && e <= 512u); };
     auto start_copy = [&](const DecSlot& sl) {   // leader only
         const uint32_t e = sl.entry & 0xFFFFu;
-        if (sl.t < g.n_tiles && e >= 258u && e <= 512u) bulk_load(stage, payload + sl.src, 32u * e, &tc->mbar, 0);
+        if (sl.t < g.n_tiles && is_staged(e)) bulk_load(stage, payload + sl.src, 32u * (e & 0x7FFFu), &tc->mbar, 0);
     };
 
     if (leader) {
@@ -1750,7 +1881,7 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
         // leaf mode: where this tile goes (asked for now, needed when the stores begin)
         unsigned char* const o_leaf = LEAVES ? ws.tptr[t] : nullptr;
         const uint32_t p = it & 1u;
-        const bool is_pack = e >= 258u && e < 512u;
+        const bool is_pack = ENT ? (e > 0x8000u && e != 0xFFFFu) : (e >= 258u && e < 512u);     // a coded tile
         bool decoded = true;
         uint32_t w[kWordsPerLane];
         uint32_t desc = 0;
@@ -1758,11 +1889,63 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
         PlaneWords pw[4];
 
         // ---- phase 1: everything this lane needs from the stage goes into registers
-        if (e >= 258u && e <= 512u) {
+        if (is_staged(e)) {
             if (!mbar_wait(&tc->mbar, phase)) trouble = 1u;
             phase ^= 1u;
             if (!is_pack) {
                 read_staged_words(stage, warp, lane, w);
+            } else if (ENT) {
+                // ENT tile.  Header: the eight stream lengths against the entry (structure); then this
+                // warp reads its share's stream the way the format interleaves it: at step i every
+                // strand whose codeword i is not complete in the bits it holds takes the stream's next
+                // halfword, strands in ascending order.  The stream must be used up exactly and the
+                // bits left in every strand must be zero (descriptor error otherwise).
+                const uint32_t cnt = lane < 8u ? lds_now_u16(stage_s + 8u + 2u * lane) : 0u;
+                const bool cnt_bad = lane < 8u && (cnt < 128u || cnt > 1024u);
+                const uint32_t total = __reduce_add_sync(0xFFFFFFFFu, cnt);
+                const uint32_t before = __reduce_add_sync(0xFFFFFFFFu, lane < warp ? cnt : 0u);
+                const uint32_t mine = __shfl_sync(0xFFFFFFFFu, cnt, warp);
+                int verdict = (__any_sync(0xFFFFFFFFu, cnt_bad) || ent_tile_bytes(total) != 32u * (e & 0x7FFFu)) ? 2 : 0;
+                if (!verdict) {
+                    const uint32_t anchor = lds_now_u8(stage_s + warp);
+                    const uint32_t st = stage_s + 8256u + 2u * before;
+                    const uint32_t lt_mask = (1u << lane) - 1u;
+                    uint32_t buf = 0, avail = 0, pos = 0, ew[8];
+                    bool over = false;
+#pragma unroll
+                    for (int j = 0; j < 8; j++) ew[j] = 0u;
+#pragma unroll
+                    for (int i = 0; i < 32; i++) {
+                        const bool more = ent_parse_length(buf) > avail;
+                        const uint32_t takers = __ballot_sync(0xFFFFFFFFu, more);
+                        if (more) {
+                            const uint32_t idx = pos + __popc(takers & lt_mask);
+                            uint32_t hw = 0;
+                            if (idx < mine) hw = lds_now_u16(st + 2u * idx); else over = true;
+                            buf |= hw << avail;
+                            avail += 16u;
+                        }
+                        pos += __popc(takers);
+                        const uint32_t len = ent_parse_length(buf);
+                        ew[i >> 2] |= ent_parse_value(buf, anchor) << (8 * (i & 3));
+                        buf >>= len;
+                        avail -= len;
+                    }
+                    if (__any_sync(0xFFFFFFFFu, over || buf != 0u) || pos != mine) verdict = 1;
+#pragma unroll
+                    for (int j = 0; j < 4; j++) {
+                        sm[j] = j == 0 ? lds_now_v2<0>(sm_s) : j == 1 ? lds_now_v2<256>(sm_s) : j == 2 ? lds_now_v2<512>(sm_s) : lds_now_v2<768>(sm_s);
+                        pw[j].a = ew[2 * j];
+                        pw[j].b = ew[2 * j + 1];
+                    }
+                }
+                if (verdict) {               // (a stream that does not fit is this warp's finding alone)
+                    decoded = false;
+                    if (lane == 0) {
+                        atomicMin(&ws.ctrl->bad4_key, (unsigned long long)t * 2ull + (verdict == 2 ? 1ull : 0ull));
+                        atomicOr(&ws.cflag[chunk_of(g, t)], CF_BAD4);
+                    }
+                }
             } else {
 #ifdef WM_AB_D_NOP1
                 desc = 100u | (4u << 8);
@@ -1853,7 +2036,8 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
                     const uint32_t dg = __shfl_sync(0xFFFFFFFFu, desc, j);
                     const uint32_t base = dg & 0xFFu, wd = (dg >> 8) & 15u;
                     uint32_t ea = base * 0x01010101u, eb = ea;
-                    if (wd == 4u) unpack_group_planes<4>(pw[j], base, ea, eb);       // by far the most frequent width
+                    if (ENT) { ea = pw[j].a; eb = pw[j].b; }       // the exponent bytes are already there
+                    else if (wd == 4u) unpack_group_planes<4>(pw[j], base, ea, eb);       // by far the most frequent width
                     else switch (wd) {     // uniform across the warp
                         case 1: unpack_group_planes<1>(pw[j], base, ea, eb); break;
                         case 2: unpack_group_planes<2>(pw[j], base, ea, eb); break;
@@ -2014,6 +2198,7 @@ struct DeviceState {
 };
 static bool g_timing = false;
 static bool g_zero_tiles = false;   // wm_zero_tiles_enable
+static bool g_entropy = false;      // wm_entropy_enable
 
 struct MainKernelTimer {        // records events around a main kernel when timing is enabled
     const DeviceState* ds; int kind; cudaStream_t s;
@@ -2047,14 +2232,19 @@ static const DeviceState* device_state()
         const void* enc[] = {(const void*)k_encode<kTeams, false, false, false>, (const void*)k_encode<kTeams, true, false, false>,
                              (const void*)k_encode<kTeams, false, true, false>,  (const void*)k_encode<kTeams, true, true, false>,
                              (const void*)k_encode<kTeams, false, false, true>,  (const void*)k_encode<kTeams, true, false, true>,
-                             (const void*)k_encode<kTeams, false, true, true>,   (const void*)k_encode<kTeams, true, true, true>};
+                             (const void*)k_encode<kTeams, false, true, true>,   (const void*)k_encode<kTeams, true, true, true>,
+                             (const void*)k_encode<kTeams, false, false, false, true>, (const void*)k_encode<kTeams, true, false, false, true>,
+                             (const void*)k_encode<kTeams, false, true, false, true>,  (const void*)k_encode<kTeams, true, true, false, true>};
         for (const void* f : enc)
             if (cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, big) != cudaSuccess) return nullptr;
     }
     {
         const void* dec[] = {(const void*)k_decode<kTeamsPlain, false, 0>, (const void*)k_decode<kTeamsPlain, true, 0>,
                              (const void*)k_decode<kTeamsPlain, false, 1>, (const void*)k_decode<kTeamsPlain, true, 1>,
-                             (const void*)k_decode<kTeamsPlain, false, 2>, (const void*)k_decode<kTeamsPlain, true, 2>};
+                             (const void*)k_decode<kTeamsPlain, false, 2>, (const void*)k_decode<kTeamsPlain, true, 2>,
+                             (const void*)k_decode<kTeamsPlain, false, 0, true>, (const void*)k_decode<kTeamsPlain, true, 0, true>,
+                             (const void*)k_decode<kTeamsPlain, false, 1, true>, (const void*)k_decode<kTeamsPlain, true, 1, true>,
+                             (const void*)k_decode<kTeamsPlain, false, 2, true>, (const void*)k_decode<kTeamsPlain, true, 2, true>};
         for (const void* f : dec)
             if (cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, big) != cudaSuccess) return nullptr;
     }
@@ -2124,6 +2314,7 @@ uint32_t wm_last_launch_count(void) { return g_launches; }
 void wm_timing_enable(int on) { g_timing = on != 0; }
 
 void wm_zero_tiles_enable(int on) { g_zero_tiles = on != 0; }
+void wm_entropy_enable(int on) { g_entropy = on != 0; }
 
 int wm_timing_read_ms(int kind, float* ms)
 {
@@ -2323,7 +2514,8 @@ static wm_status encode_any(const void* cache, const wm_leaf* leaves, uint32_t n
     const uint32_t grid = need < (uint32_t)ds->sm_count ? need : (uint32_t)ds->sm_count;
     {
         MainKernelTimer timer(ds, 2, s);
-        const int variant = (dirty ? 1 : 0) | (leaves ? 2 : 0) | (g_zero_tiles ? 4 : 0);
+        // the entropy option takes precedence over the zero-tile option
+        const int variant = (dirty ? 1 : 0) | (leaves ? 2 : 0) | (g_entropy ? 8 : g_zero_tiles ? 4 : 0);
         auto go = [&](auto kernel) { launch_after(kernel, grid, kTeams * 256, kDynSmem, s, c, g, dirty, w, wire_cap, ws, ds->tables); };
         switch (variant) {
             case 0: go(k_encode<kTeams, false, false, false>); break;
@@ -2333,11 +2525,15 @@ static wm_status encode_any(const void* cache, const wm_leaf* leaves, uint32_t n
             case 4: go(k_encode<kTeams, false, false, true>); break;
             case 5: go(k_encode<kTeams, true, false, true>); break;
             case 6: go(k_encode<kTeams, false, true, true>); break;
-            default: go(k_encode<kTeams, true, true, true>); break;
+            case 7: go(k_encode<kTeams, true, true, true>); break;
+            case 8: go(k_encode<kTeams, false, false, false, true>); break;
+            case 9: go(k_encode<kTeams, true, false, false, true>); break;
+            case 10: go(k_encode<kTeams, false, true, false, true>); break;
+            default: go(k_encode<kTeams, true, true, false, true>); break;
         }
     }
     launch_after(k_encode_finish, (g.n_chunks + g.finish_cb - 1) / g.finish_cb, 1024, 0, s, c, g, dirty, crc_inout, w, ws, ds->tables,
-                 chunk_powers(g), g_zero_tiles ? 1u : 0u);
+                 chunk_powers(g), g_entropy ? 4u : g_zero_tiles ? 2u : 0u);
     launch_after(k_meta_crc, (g.n_meta_slices + 3) / 4, 1024, kDynSmem, s, w, g, ws, ds->tables, result);
     g_launches = leaves ? 5 : 4;
     return launch_status();
@@ -2383,7 +2579,9 @@ static wm_status decode_any(const void* wire, uint64_t wire_len, void* dst, cons
     }
     // a wire shorter than the metadata is rejected by the header check before anything else is read
     const uint32_t meta_blocks = (g.n_meta_slices + 3) / 4;
-    launch_after(k_decode_check, meta_blocks + (g.n_chunks + 31) / 32, 1024, 0, s, w, wire_len, g, ws, ds->tables, result, meta_blocks);
+    const bool ent = g_entropy;      // the option says which kind of image the call expects
+    launch_after(k_decode_check, meta_blocks + (g.n_chunks + 31) / 32, 1024, 0, s, w, wire_len, g, ws, ds->tables, result, meta_blocks,
+                 ent ? 1u : 0u);
     const uint32_t need = (g.n_tiles + kTeamsPlain - 1) / kTeamsPlain;
     const uint32_t grid = need < (uint32_t)ds->sm_count ? need : (uint32_t)ds->sm_count;
     auto pass = [&](auto flat_kernel, auto leaf_kernel) {
@@ -2392,12 +2590,20 @@ static wm_status decode_any(const void* wire, uint64_t wire_len, void* dst, cons
     };
     {
         MainKernelTimer timer(ds, 3, s);
-        if (strict) pass(k_decode<kTeamsPlain, false, 1>, k_decode<kTeamsPlain, true, 1>);
-        else pass(k_decode<kTeamsPlain, false, 0>, k_decode<kTeamsPlain, true, 0>);
+        if (ent) {
+            if (strict) pass(k_decode<kTeamsPlain, false, 1, true>, k_decode<kTeamsPlain, true, 1, true>);
+            else pass(k_decode<kTeamsPlain, false, 0, true>, k_decode<kTeamsPlain, true, 0, true>);
+        } else {
+            if (strict) pass(k_decode<kTeamsPlain, false, 1>, k_decode<kTeamsPlain, true, 1>);
+            else pass(k_decode<kTeamsPlain, false, 0>, k_decode<kTeamsPlain, true, 0>);
+        }
     }
     launch_after(k_decode_finish, (g.n_chunks + g.finish_cb - 1) / g.finish_cb, 1024, 0, s, w, wire_len, g, d, dst_crc_inout, ws, ds->tables,
                  result, chunk_powers(g), strict ? 1u : 0u);
-    if (strict) pass(k_decode<kTeamsPlain, false, 2>, k_decode<kTeamsPlain, true, 2>);
+    if (strict) {
+        if (ent) pass(k_decode<kTeamsPlain, false, 2, true>, k_decode<kTeamsPlain, true, 2, true>);
+        else pass(k_decode<kTeamsPlain, false, 2>, k_decode<kTeamsPlain, true, 2>);
+    }
     g_launches = (leaves ? 5 : 4) + (strict ? 1 : 0);
     return launch_status();
 }
