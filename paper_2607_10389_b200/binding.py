@@ -206,7 +206,7 @@ def wm_checksum_poly(cache: torch.Tensor, chunk_bytes: int, polynomial: int, crc
     _dev_u8(cache, "cache")
     nbytes = cache.numel() * cache.element_size()
     _check(lib().wm_checksum_poly(cache.data_ptr(), nbytes, chunk_bytes, int(polynomial), crc_out.data_ptr(),
-                                  workspace.data_ptr(), workspace.numel(), _stream(stream)), "wm_checksum_poly", "wm_entropy_enable")
+                                  workspace.data_ptr(), workspace.numel(), _stream(stream)), "wm_checksum_poly")
 
 
 NOALLOC_MAX_BYTES = 4 << 30
