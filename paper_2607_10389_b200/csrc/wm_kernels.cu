@@ -854,16 +854,21 @@ __device__ __forceinline__ uint32_t ent_slot(uint32_t E, uint32_t anchor)
 {
     return min(E - anchor + 6u, 10u);
 }
+// Both tables are byte look-ups done with permutes (no branches: the lanes of a warp hold
+// different slots): slots 0..7 from one pair of words, 8..10 from a third.
+__device__ __forceinline__ uint32_t ent_lut(uint32_t lo, uint32_t hi, uint32_t top, uint32_t slot)
+{
+    const uint32_t a = __byte_perm(lo, hi, slot), b = __byte_perm(top, 0u, slot & 7u);
+    return (slot < 8u ? a : b) & 0xFFu;
+}
 __device__ __forceinline__ uint32_t ent_length(uint32_t slot)
 {
-    // (length - 1) per slot, four bits each: 7 5 4 3 3 1 1 1 3 6 15
-    return (uint32_t)((0xF6311133457ull >> (4u * slot)) & 15ull) + 1u;
+    return ent_lut(0x04050608u, 0x02020204u, 0x00100704u, slot);      // 8 6 5 4 | 4 2 2 2 | 4 7 16
 }
 __device__ __forceinline__ uint32_t ent_word(uint32_t slot, uint32_t E)
 {
-    if (slot >= 10u) return 255u | (E << 8);
-    if (slot >= 8u) return slot == 8u ? 7u : 63u;
-    return __byte_perm(0x0B0F1F7Fu, 0x01000203u, slot) & 0xFFu;
+    const uint32_t w = ent_lut(0x0B0F1F7Fu, 0x01000203u, 0x00FF3F07u, slot);       // 127 31 15 11 | 3 2 0 1 | 7 63 255
+    return w | (slot == 10u ? E << 8 : 0u);
 }
 // Bytes of an ENT tile whose eight streams hold `halfwords` halfwords in all (a multiple of 32;
 // 16384 or more means that the tile is stored raw instead).
@@ -871,28 +876,23 @@ __device__ __forceinline__ uint32_t ent_tile_bytes(uint32_t halfwords)
 {
     return (8256u + 2u * halfwords + 31u) & ~31u;
 }
-// Decoder side: length of the codeword at the low end of `buf` (zero beyond the valid bits).
-__device__ __forceinline__ uint32_t ent_parse_length(uint32_t buf)
+// Decoder side.  A codeword is s ones and a zero (s < 8; eight ones: the escape), followed for
+// s = 0 and s = 2 by one more bit x:  s = 0: u = -x;  1: +1;  2: -2 - x;  3: +2;  4..7: -4, -5, +3, -6.
+// ent_ones: s, capped at 8, of the codeword at the low end of `buf` (zero beyond the valid bits).
+__device__ __forceinline__ uint32_t ent_ones(uint32_t buf)
 {
-    if ((buf & 3u) != 3u) return 2u;
-    if ((buf & 12u) != 12u) return 4u;
-    const uint32_t k = __ffs(~(buf >> 4)) - 1u;          // ones after the four
-    return k < 4u ? 5u + k : 16u;
+    return min((uint32_t)__ffs(~buf) - 1u, 8u);
 }
-// ... and the exponent it stands for.
-__device__ __forceinline__ uint32_t ent_parse_value(uint32_t buf, uint32_t anchor)
+__device__ __forceinline__ uint32_t ent_parse_length(uint32_t s)
 {
-    uint32_t u;
-    if ((buf & 3u) != 3u) {
-        u = (0xFF0100u >> (8u * (buf & 3u))) & 0xFFu;                 // 0, +1, -1
-    } else if ((buf & 12u) != 12u) {
-        u = (0xFD02FEu >> (8u * ((buf >> 2) & 3u))) & 0xFFu;          // -2, +2, -3
-    } else {
-        const uint32_t k = __ffs(~(buf >> 4)) - 1u;
-        if (k >= 4u) return (buf >> 8) & 0xFFu;
-        u = (0xFA03FBFCu >> (8u * k)) & 0xFFu;                        // -4, -5, +3, -6
-    }
-    return (anchor + u) & 0xFFu;
+    const uint32_t l = __byte_perm(0x04040202u, 0x08070605u, s & 7u) & 0xFFu;       // 2 2 4 4 | 5 6 7 8
+    return s == 8u ? 16u : l;
+}
+__device__ __forceinline__ uint32_t ent_parse_value(uint32_t buf, uint32_t s, uint32_t anchor)
+{
+    const uint32_t base = __byte_perm(0x02FE0100u, 0xFA03FBFCu, s & 7u);            // 0 +1 -2 +2 | -4 -5 +3 -6
+    const uint32_t x = ((s & 5u) == 0u) ? (buf >> (s + 1u)) & 1u : 0u;
+    return s == 8u ? (buf >> 8) & 0xFFu : (anchor + base - x) & 0xFFu;
 }
 
 // Single-pass fused checksum + encode.  Each team keeps four tiles in flight:
@@ -947,6 +947,8 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
     // that shares its scheduler with busy ones gets too few issue slots to keep up).
     __shared__ uint32_t s_scanner;
     __shared__ uint32_t s_tmem;
+    __shared__ uint32_t s_ent[16];     // ENT: codeword | length << 16 by slot (one bank each: no conflicts)
+    if (ENT && threadIdx.x < 11u) s_ent[threadIdx.x] = ent_word(threadIdx.x, 0u) | (ent_length(threadIdx.x) << 16);
     Smem S = setup_smem(smem, tab);
     grid_dep_wait();                   // from here on the control block and the length table are ready
     grid_dep_launch();
@@ -1086,8 +1088,8 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
                 uint32_t bits = 0;
 #pragma unroll
                 for (int i = 0; i < 16; i++)
-                    bits += ent_length(ent_slot((d[i] >> 8) & 0xFFu, anchor)) + ent_length(ent_slot(d[i] >> 24, anchor));
-                const uint32_t count = __reduce_add_sync(0xFFFFFFFFu, (bits + 15u) >> 4);
+                    bits += s_ent[ent_slot(__byte_perm(d[i], 0u, 0x4441), anchor)] + s_ent[ent_slot(d[i] >> 24, anchor)];
+                const uint32_t count = __reduce_add_sync(0xFFFFFFFFu, ((bits >> 16) + 15u) >> 4);     // (the low halves add up to less than 2^16)
                 gw[0] = anchor | (count << 8);
                 gw[1] = gw[2] = gw[3] = 0u;
             } else {
@@ -1200,10 +1202,11 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
                 uint32_t acc = 0, n = 0, pend = lane, pos = 32;
 #pragma unroll
                 for (int i = 0; i < 32; i++) {
-                    const uint32_t E = (i & 1) ? d[i >> 1] >> 24 : (d[i >> 1] >> 8) & 0xFFu;
+                    const uint32_t E = (i & 1) ? d[i >> 1] >> 24 : __byte_perm(d[i >> 1], 0u, 0x4441);
                     const uint32_t slot = ent_slot(E, anchor);
-                    acc |= ent_word(slot, E) << n;
-                    n += ent_length(slot);
+                    const uint32_t cw = s_ent[slot];
+                    acc |= ((cw & 0xFFFFu) | (slot == 10u ? E << 8 : 0u)) << n;
+                    n += cw >> 16;
                     if (i == 0) continue;
                     const bool more = n > 16u;             // the codeword runs past what the strand has taken
                     const uint32_t takers = __ballot_sync(0xFFFFFFFFu, more);
@@ -1916,7 +1919,7 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
                     for (int j = 0; j < 8; j++) ew[j] = 0u;
 #pragma unroll
                     for (int i = 0; i < 32; i++) {
-                        const bool more = ent_parse_length(buf) > avail;
+                        const bool more = ent_parse_length(ent_ones(buf)) > avail;
                         const uint32_t takers = __ballot_sync(0xFFFFFFFFu, more);
                         if (more) {
                             const uint32_t idx = pos + __popc(takers & lt_mask);
@@ -1926,8 +1929,9 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
                             avail += 16u;
                         }
                         pos += __popc(takers);
-                        const uint32_t len = ent_parse_length(buf);
-                        ew[i >> 2] |= ent_parse_value(buf, anchor) << (8 * (i & 3));
+                        const uint32_t ones = ent_ones(buf);
+                        const uint32_t len = ent_parse_length(ones);
+                        ew[i >> 2] |= ent_parse_value(buf, ones, anchor) << (8 * (i & 3));
                         buf >>= len;
                         avail -= len;
                     }
