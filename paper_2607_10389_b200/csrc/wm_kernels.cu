@@ -1821,6 +1821,13 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
          const Tables* __restrict__ tab)
 {
     extern __shared__ __align__(16) unsigned char smem[];
+    // ENT: what the low byte of a strand's bits says about the codeword there:
+    // length | (u & 0xFF) << 8 | escape << 16
+    __shared__ uint32_t s_parse[ENT ? 256 : 1];
+    if (ENT && threadIdx.x < 256u) {
+        const uint32_t s = ent_ones(threadIdx.x);
+        s_parse[threadIdx.x] = ent_parse_length(s) | (ent_parse_value(threadIdx.x, s, 0u) << 8) | (s == 8u ? 0x10000u : 0u);
+    }
     Smem S = setup_smem(smem, tab);
     grid_dep_wait();
     grid_dep_launch();
@@ -1919,7 +1926,7 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
                     for (int j = 0; j < 8; j++) ew[j] = 0u;
 #pragma unroll
                     for (int i = 0; i < 32; i++) {
-                        const bool more = ent_parse_length(ent_ones(buf)) > avail;
+                        const bool more = (s_parse[buf & 0xFFu] & 0xFFu) > avail;
                         const uint32_t takers = __ballot_sync(0xFFFFFFFFu, more);
                         if (more) {
                             const uint32_t idx = pos + __popc(takers & lt_mask);
@@ -1929,9 +1936,10 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
                             avail += 16u;
                         }
                         pos += __popc(takers);
-                        const uint32_t ones = ent_ones(buf);
-                        const uint32_t len = ent_parse_length(ones);
-                        ew[i >> 2] |= ent_parse_value(buf, ones, anchor) << (8 * (i & 3));
+                        const uint32_t cw = s_parse[buf & 0xFFu];
+                        const uint32_t len = cw & 0xFFu;
+                        const uint32_t E = (cw & 0x10000u) ? __byte_perm(buf, 0u, 0x4441) : (anchor + (cw >> 8)) & 0xFFu;
+                        ew[i >> 2] |= E << (8 * (i & 3));
                         buf >>= len;
                         avail -= len;
                     }
