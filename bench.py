@@ -371,6 +371,47 @@ def tail_schedule(wm, cfg, cur, shadow, wire, ws, dev, W, reps=8, super_mbs=(64,
     return out
 
 
+def entropy_option(wm, cfg, cur, shadow, wire, ws, dev, W_plain, peak, reps=20):
+    """The ENT option (entropy-coded exponents): ratio and call times beside the default format's."""
+    import torch
+    N, C = cfg.nbytes, cfg.chunk_bytes
+    nc = wm.num_chunks(N, C)
+    crc = torch.zeros(nc, dtype=torch.int32, device=dev)
+    crc_d = torch.zeros(nc, dtype=torch.int32, device=dev)
+    res_e, res_d = wm.new_result(dev), wm.new_result(dev)
+    wm.entropy_enable(True)
+    try:
+        wm.wm_encode(cur, C, None, crc, wire, ws, res_e)
+        r = wm.read_result(res_e)
+        if not r.ok:
+            raise SystemExit("entropy option: encode failed")
+        W = r.wire_len
+        wm.wm_decode_verify(wire, W, shadow, C, crc_d, ws, res_d)
+        if not (wm.read_result(res_d).ok and torch.equal(shadow, cur) and torch.equal(crc, crc_d)):
+            raise SystemExit("entropy option: round trip failed")
+        out = {"wire_bytes": W, "ratio": W / N, "ratio_default_format": W_plain / N}
+        for name, fn in (("encode", lambda: wm.wm_encode(cur, C, None, crc, wire, ws, res_e)),
+                         ("decode_verify", lambda: wm.wm_decode_verify(wire, W, shadow, C, crc_d, ws, res_d))):
+            for _ in range(3):
+                fn()
+            torch.cuda.synchronize()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            for _ in range(reps):
+                fn()
+            b.record()
+            torch.cuda.synchronize()
+            ms = a.elapsed_time(b) / reps
+            out[name + "_ms"] = ms
+            out[name + "_raw_gbs"] = N / (ms * 1e-3) / 1e9
+            out[name + "_frac_of_hbm_peak"] = (N + W) / (ms * 1e-3) / 1e9 / peak
+    finally:
+        wm.entropy_enable(False)
+    out["note"] = ("wm_entropy_enable(1): fixed prefix code of the exponents, strands interleaved in reader order; "
+                   "whole calls back to back; bound by integer instruction issue (one codeword per lane and step)")
+    return out
+
+
 def run_reference(args):
     """Reference arm: the CPU oracle timed on the host cores, a bounded sample per step."""
     rank, _, world = _dist()
@@ -632,6 +673,11 @@ def main():
     if not args.no_loop and cfg.kind == "kv":
         leaf = leaf_mode(wm, cfg, cur, wire, ws, dev, W, peak)
 
+    # the entropy-coded exponent option beside the default format
+    ent = None
+    if not args.no_loop and cfg.kind == "kv" and not args.zero_tiles:
+        ent = entropy_option(wm, cfg, cur, shadow, wire, ws, dev, W, peak)
+
     # verification placement: super-chunks on three streams against the whole cache stage by stage
     tail = None
     if not args.no_loop and args.workload in ("engine", "engine_256m"):
@@ -718,7 +764,7 @@ def main():
                        "wire_bytes": W, "ratio": W / N, "dirty_chunks": n_rewritten, "n_chunks": nc,
                        "l2": "inputs larger than L2 (no flush needed)", "parallelism": "replicas only",
                        "zero_tiles": bool(args.zero_tiles)},
-            "calls": per_call, "roofline": roofline, "precopy_loop": loop, "leaf_mode": leaf, "tail_schedule": tail,
+            "calls": per_call, "roofline": roofline, "precopy_loop": loop, "leaf_mode": leaf, "entropy_option": ent, "tail_schedule": tail,
             "cpu_baseline": base, "e2e": e2e,
             "gpu_launches": gpu_launches, "clocks": clocks,
         }

@@ -64,13 +64,13 @@ def check_meta_against_oracle(job, m, hdr, off, ln, crc, present):
     assert acc == int(hdr[48:52].view(np.uint32)[0])
 
 
-def check_chunks_against_oracle(job, cache, chunks, off, ln, crc, tab):
+def check_chunks_against_oracle(job, cache, chunks, off, ln, crc, tab, entropy=False):
     """Each sampled chunk, encoded alone by the oracle, gives the bytes found in the wire image."""
     tpc = job.chunk // TILE
     for c in chunks:
         lo, hi = c * job.chunk, min((c + 1) * job.chunk, job.n)
         raw = cache[lo:hi].cpu().numpy()
-        w1, crc1, r1 = oracle.encode(raw, job.chunk)
+        w1, crc1, r1 = oracle.encode(raw, job.chunk, entropy=entropy)
         assert r1.status == 0
         assert int(crc1[0]) == int(crc[c]) == oracle.crc32c(raw), f"chunk {c}: crc"
         me = oracle.meta_end(hi - lo, job.chunk)
@@ -115,6 +115,41 @@ def test_engine_cache_full_move_sampled_against_oracle():
     rd = wm.read_result(job.res_d)
     assert rd.ok and rd.cache_crc == r.cache_crc and rd.n_present == job.nc
     assert torch.equal(shadow, cur) and torch.equal(crc_dst, crc_b)
+
+
+def test_engine_cache_with_entropy_coded_exponents_sampled_against_oracle():
+    """The ENT option at full size: sampled chunks byte for byte, metadata, round trip, one flipped bit."""
+    cfg = inputs.CONFIGS["engine"]
+    cur = inputs.make_cache(cfg, "cuda")
+    job = Job(cfg.nbytes, cfg.chunk_bytes)
+    crc_b = torch.zeros(job.nc, dtype=torch.int32, device="cuda")
+    wm.entropy_enable(True)
+    try:
+        wm.wm_encode(cur, job.chunk, None, crc_b, job.wire, job.ws, job.res_e)
+        r = wm.read_result(job.res_e)
+        assert r.ok and r.n_present == job.nc
+        m, hdr, off, ln, crc, tab = job.meta()
+        assert int(hdr[6:8].view(np.uint16)[0]) == 4 and ((tab & 0x8000) != 0).all()
+        present = np.ones(job.nc, dtype=np.uint64)
+        check_meta_against_oracle(job, m, hdr, off, ln, crc, present)
+        assert 0.68 < r.wire_len / job.n < 0.72        # bit-plane packing: 0.757
+        check_chunks_against_oracle(job, cur, sample_chunks(job.nc, 6, 2), off, ln, crc, tab, entropy=True)
+        shadow = torch.zeros(job.n, dtype=torch.uint8, device="cuda")
+        crc_dst = torch.zeros(job.nc, dtype=torch.int32, device="cuda")
+        wm.wm_decode_verify(job.wire, r.wire_len, shadow, job.chunk, crc_dst, job.ws, job.res_d)
+        rd = wm.read_result(job.res_d)
+        assert rd.ok and rd.cache_crc == r.cache_crc and torch.equal(shadow, cur) and torch.equal(crc_dst, crc_b)
+        # one bit inside a stream of a tile in the middle of the image
+        c = job.nc // 2
+        at = job.meta_end + int(off[c]) + 9000
+        job.wire[at] ^= 0x10
+        crc_dst.fill_(7)
+        wm.wm_decode_verify(job.wire, r.wire_len, shadow, job.chunk, crc_dst, job.ws, job.res_d)
+        rd = wm.read_result(job.res_d)
+        assert rd.status_name in ("ERR_CHUNK_CRC", "ERR_DESC") and rd.first_bad_chunk == c and rd.n_bad_chunks == 1
+        assert bool((crc_dst == 7).all())
+    finally:
+        wm.entropy_enable(False)
 
 
 def test_random_cache_takes_the_raw_path_and_a_flipped_bit_is_rejected():
