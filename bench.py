@@ -465,6 +465,7 @@ def main():
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-loop", action="store_true", help="skip the pre-copy step loop")
     ap.add_argument("--zero-tiles", action="store_true", help="encoder option: all-zero tiles as table entries")
+    ap.add_argument("--entropy", action="store_true", help="codec option: entropy-coded exponents (ENT tiles) in every call")
     ap.add_argument("--profile", action="store_true",
                     help="profiler capture mode: round-trip check, warm-up and timed steps only")
     args = ap.parse_args()
@@ -492,6 +493,7 @@ def main():
     barrier, max_over_ranks = group.barrier, group.max_over_ranks
 
     wm.zero_tiles_enable(args.zero_tiles)
+    wm.entropy_enable(args.entropy)
     cfg, cur, prev, n_rewritten = make_workload(args.workload, dev)
     N, C = cfg.nbytes, cfg.chunk_bytes
     nc = wm.num_chunks(N, C)
@@ -675,7 +677,7 @@ def main():
 
     # the entropy-coded exponent option beside the default format
     ent = None
-    if not args.no_loop and cfg.kind == "kv" and not args.zero_tiles:
+    if not args.no_loop and cfg.kind == "kv" and not args.zero_tiles and not args.entropy:
         ent = entropy_option(wm, cfg, cur, shadow, wire, ws, dev, W, peak)
 
     # verification placement: super-chunks on three streams against the whole cache stage by stage
@@ -763,7 +765,7 @@ def main():
             "config": {"workload": args.workload, "nbytes": N, "chunk_bytes": C, "shape": list(cfg.shape),
                        "wire_bytes": W, "ratio": W / N, "dirty_chunks": n_rewritten, "n_chunks": nc,
                        "l2": "inputs larger than L2 (no flush needed)", "parallelism": "replicas only",
-                       "zero_tiles": bool(args.zero_tiles)},
+                       "zero_tiles": bool(args.zero_tiles), "entropy": bool(args.entropy)},
             "calls": per_call, "roofline": roofline, "precopy_loop": loop, "leaf_mode": leaf, "entropy_option": ent, "tail_schedule": tail,
             "cpu_baseline": base, "e2e": e2e,
             "gpu_launches": gpu_launches, "clocks": clocks,
