@@ -195,3 +195,40 @@ def test_ent_leaves(wm):
     dcrc = torch.zeros(nc, dtype=torch.int32, device="cuda")
     wm.wm_decode_verify_leaves(wire, r.wire_len, wm.make_leaf_table(dst), n, chunk, dcrc, ws, res)
     assert wm.read_result(res).status == 0 and all(torch.equal(x, y) for x, y in zip(leaves, dst))
+
+
+def test_gpu_reads_images_that_combine_both_options(wm):
+    """The GPU encoder ignores the zero-tile option while the entropy option is on, but the format
+    allows both in one image (the oracle writes it) and the GPU decoder reads it."""
+    n, chunk = 10 * TILE, 2 * TILE
+    a = _mixed_cache(n, 23)
+    a[6 * TILE:8 * TILE] = 0
+    w, crc, res = oracle.encode(a, chunk, zero_tiles=True, entropy=True)
+    assert struct.unpack_from("<H", w, 6)[0] == 6
+    out, dcrc, r = _run_decode(wm, w, n, chunk)
+    assert r.status == 0 and np.array_equal(out, a) and np.array_equal(dcrc, crc)
+    # the GPU encoder with both switches on writes the entropy image without zero entries
+    wm.zero_tiles_enable(True)
+    try:
+        wire, crc2, r2, _ = _run_encode(wm, a, chunk)
+    finally:
+        wm.zero_tiles_enable(False)
+    want, _, _ = oracle.encode(a, chunk, entropy=True)
+    assert r2.status == 0 and np.array_equal(wire[: r2.wire_len].cpu().numpy(), want)
+
+
+def test_ent_repeatable_under_load(wm):
+    """Placement is decided by whichever team gets there first; the bytes must not depend on it."""
+    import torch
+    from paper_2607_10389_b200 import inputs
+    cfg = inputs.CONFIGS["engine_small"]
+    a = inputs.make_cache(cfg).numpy().view(np.uint8).reshape(-1)
+    first = None
+    for _ in range(25):
+        wire, crc, r, _ = _run_encode(wm, a, cfg.chunk_bytes)
+        got = wire[: r.wire_len].clone()
+        if first is None:
+            first = got
+        assert r.status == 0 and torch.equal(got, first)
+        out, _, rd = _run_decode(wm, got.cpu().numpy(), a.size, cfg.chunk_bytes)
+        assert rd.status == 0 and np.array_equal(out, a)
