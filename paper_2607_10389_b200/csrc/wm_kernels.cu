@@ -912,7 +912,9 @@ __device__ __forceinline__ uint32_t ent_parse_value(uint32_t buf, uint32_t s, ui
 // tile, so it runs at the pace of the warp that has the most to do.
 // Template switches: MASKED (a dirty mask was given), LEAVES (the cache is a table of tensors;
 // tickets are claimed one step further ahead so that a tile's address can be looked up on the
-// way), ZEROS (the zero-tile option).
+// way), ZEROS (the zero-tile option), ENT (the entropy option: the measuring step adds up codeword
+// lengths instead of taking exponent ranges, the packing step writes the share's interleaved
+// stream of halfwords instead of bit planes).
 // Packed data goes from registers to the wire image directly: in every region of a PACK tile
 // a lane owns an aligned unit at a lane-strided place, so each warp store is one contiguous
 // sector-aligned run.  Claiming a tile before the previous offset is known means that, if the
@@ -1815,6 +1817,9 @@ __device__ __forceinline__ void unpack_group_planes(const PlaneWords& pw, uint32
 // the pace of its slowest one.)  LEAVES: the decoded tiles go to a table of tensors.
 // MODE 0: unpack, store, checksum (the normal call).  Strict calls run the kernel twice: MODE 1
 // unpacks and checksums without storing anything; MODE 2, after the verdict, unpacks and stores.
+// ENT: the image holds ENT tiles instead of PACK tiles; a warp reads its share's stream of
+// halfwords in phase 1 (the need test, the ballot and the fetch of every step) and leaves the
+// exponent bytes where the plane words would be.
 template <int TEAMS, bool LEAVES, int MODE, bool ENT = false>
 __global__ void __launch_bounds__(TEAMS * 256, 1)
 k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restrict__ dst, Ws ws,
