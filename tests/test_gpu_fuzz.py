@@ -1,0 +1,92 @@
+"""Seeded random geometries, masks, data recipes and codec options: the GPU's wire image, checksums
+and result record against the oracle's, then the round trip.  Tolerance 0."""
+import numpy as np
+import pytest
+
+import oracle
+
+pytestmark = pytest.mark.gpu
+TILE = 16384
+
+
+def _data(rng, n):
+    kind = rng.integers(0, 5)
+    if kind == 0:                                             # Gaussian at a random scale
+        v = (rng.normal(size=(n + 1) // 2) * float(2.0 ** rng.integers(-30, 30))).astype(np.float32)
+        a = (v.view(np.uint32) >> 16).astype("<u2").view(np.uint8)[:n].copy()
+    elif kind == 1:                                           # random bytes (raw tiles, NaN and Inf patterns)
+        a = rng.integers(0, 256, n, dtype=np.uint8)
+    elif kind == 2:                                           # per-tile mixture, some tiles zero or constant
+        a = np.empty(n, dtype=np.uint8)
+        for o in range(0, n, TILE):
+            m = min(TILE, n - o)
+            k = rng.integers(0, 4)
+            if k == 0:
+                a[o:o + m] = 0
+            elif k == 1:
+                a[o:o + m] = np.resize(np.array([0x80, 0x3F], dtype=np.uint8), m)
+            elif k == 2:
+                a[o:o + m] = rng.integers(0, 256, m, dtype=np.uint8)
+            else:
+                v = (rng.normal(size=(m + 1) // 2) * 3.0).astype(np.float32)
+                a[o:o + m] = (v.view(np.uint32) >> 16).astype("<u2").view(np.uint8)[:m]
+    elif kind == 3:                                           # wide exponent spread inside groups
+        e = rng.integers(0, 256, (n + 1) // 2).astype(np.uint32)
+        m = rng.integers(0, 128, (n + 1) // 2).astype(np.uint32)
+        s = rng.integers(0, 2, (n + 1) // 2).astype(np.uint32)
+        a = ((s << 15) | (e << 7) | m).astype("<u2").view(np.uint8)[:n].copy()
+    else:                                                     # narrow exponent spread: widths 0..3
+        e = (100 + rng.integers(0, int(rng.integers(1, 9)), (n + 1) // 2)).astype(np.uint32)
+        m = rng.integers(0, 128, (n + 1) // 2).astype(np.uint32)
+        a = ((e << 7) | m).astype("<u2").view(np.uint8)[:n].copy()
+    return a
+
+
+@pytest.mark.parametrize("seed", range(48))
+def test_random_case_matches_the_oracle(seed):
+    import torch
+    from paper_2607_10389_b200 import binding as wm
+    rng = np.random.default_rng(1000 + seed)
+    chunk = int(rng.choice([1, 2, 3, 4, 8])) * TILE
+    n = int(rng.integers(1, 40 * TILE))
+    if rng.integers(0, 4) == 0:
+        n = max(TILE, n // TILE * TILE)                       # no ragged tail
+    option = ["default", "zero", "entropy"][seed % 3]
+    a = _data(rng, n)
+    nc = oracle.num_chunks(n, chunk)
+    masked = bool(rng.integers(0, 2))
+    dirty = (rng.integers(0, 3, nc) > 0).astype(np.uint8) if masked else None
+    crc_in = oracle.checksum(a, chunk)
+    stale = crc_in.copy()
+    want, want_crc, want_res = oracle.encode(a, chunk, dirty=dirty, crc_in=stale, zero_tiles=option == "zero",
+                                             entropy=option == "entropy")
+    wm.zero_tiles_enable(option == "zero")
+    wm.entropy_enable(option == "entropy")
+    try:
+        ws = wm.new_workspace(n, chunk)
+        wire = torch.full((wm.wire_bound(n, chunk),), 0xC3, dtype=torch.uint8, device="cuda")
+        crc = torch.from_numpy(stale.view(np.int32).copy()).cuda()
+        res = wm.new_result()
+        d = None if dirty is None else torch.from_numpy(dirty).cuda()
+        wm.wm_encode(torch.from_numpy(a).cuda(), chunk, d, crc, wire, ws, res)
+        r = wm.read_result(res)
+        assert (r.status, r.wire_len, r.payload_bytes, r.n_present, r.cache_crc) == (
+            want_res.status, want_res.wire_len, want_res.payload_bytes, want_res.n_present, want_res.cache_crc)
+        assert np.array_equal(wire[: r.wire_len].cpu().numpy(), want)
+        assert np.array_equal(crc.cpu().numpy().view(np.uint32), want_crc)
+        # decode over a destination that holds the absent chunks already
+        base = a.copy()
+        if dirty is not None:
+            for c in range(nc):
+                if dirty[c]:
+                    base[c * chunk:(c + 1) * chunk] = 0x77
+        dst = torch.from_numpy(base).cuda()
+        dcrc = torch.from_numpy(stale.view(np.int32).copy()).cuda()
+        strict = bool(rng.integers(0, 2))
+        (wm.wm_decode_verify_strict if strict else wm.wm_decode_verify)(wire, r.wire_len, dst, chunk, dcrc, ws, res)
+        rd = wm.read_result(res)
+        assert rd.status == 0 and np.array_equal(dst.cpu().numpy(), a)
+        assert np.array_equal(dcrc.cpu().numpy().view(np.uint32), want_crc)
+    finally:
+        wm.zero_tiles_enable(False)
+        wm.entropy_enable(False)
