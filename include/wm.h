@@ -124,14 +124,16 @@ wm_status wm_dirty_diff(const void* cache, const void* prev, uint64_t nbytes, ui
  *
  *   header[64] | chunk_dir[16*n_chunks] | tile_tab[2*n_tiles] | zero pad to 32 | payload
  *   header: 0 "WMV1" | 4 u16 version=1 | 6 u16 flags (bit0: a dirty mask was given; bit1:
- *           the ZERO tile option, see wm_zero_tiles_enable) |
+ *           the ZERO tile option, see wm_zero_tiles_enable; bit2: ENT tiles instead of PACK
+ *           tiles, see wm_entropy_enable) |
  *           8 u64 nbytes | 16 u32 chunk_bytes | 20 u32 tile_bytes=16384 | 24 u32 n_chunks |
  *           28 u32 n_present | 32 u64 payload_bytes | 40 u64 wire_len | 48 u32 cache_crc |
  *           52 u32 meta_crc (CRC32C of the metadata with this field as zero) | 56 zero[8]
  *   chunk_dir[c]: u64 payload_off | u32 enc_len | u32 crc
  *   tile_tab[t] (u16): 0 tile of an absent chunk | 1 ZERO tile: a full tile whose bytes are
- *           all zero, no payload (only in images with flags bit1) | 258..511 PACK tile of 32*value bytes |
- *           512 RAW full tile | 0xFFFF RAW partial tail tile (nbytes mod 16384 bytes)
+ *           all zero, no payload (only in images with flags bit1) | 258..511 PACK tile of 32*value bytes
+ *           (only without flags bit2) | 512 RAW full tile | 0x8000 | n, n = 259..511: ENT tile of
+ *           32*n bytes (only with flags bit2) | 0xFFFF RAW partial tail tile (nbytes mod 16384 bytes)
  *   payload: encoded tiles of present chunks in ascending order, no padding
  *   PACK tile (32 groups of 256 elements): desc[32] u16 (base | w<<8 | chk<<12,
  *           chk = (base&15) ^ (base>>4) ^ w ^ 5) | SM[8192] | Epack_0 .. Epack_31.
