@@ -950,7 +950,11 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
     __shared__ uint32_t s_scanner;
     __shared__ uint32_t s_tmem;
     __shared__ uint32_t s_ent[16];     // ENT: codeword | length << 16 by slot (one bank each: no conflicts)
-    if (ENT && threadIdx.x < 11u) s_ent[threadIdx.x] = ent_word(threadIdx.x, 0u) | (ent_length(threadIdx.x) << 16);
+    __shared__ uint32_t s_len[16];     // ENT: length by slot
+    if (ENT && threadIdx.x < 11u) {
+        s_ent[threadIdx.x] = (threadIdx.x == 10u ? 0xFFFFu : ent_word(threadIdx.x, 0u)) | (ent_length(threadIdx.x) << 16);
+        s_len[threadIdx.x] = ent_length(threadIdx.x);
+    }
     Smem S = setup_smem(smem, tab);
     grid_dep_wait();                   // from here on the control block and the length table are ready
     grid_dep_launch();
@@ -1090,8 +1094,8 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
                 uint32_t bits = 0;
 #pragma unroll
                 for (int i = 0; i < 16; i++)
-                    bits += s_ent[ent_slot(__byte_perm(d[i], 0u, 0x4441), anchor)] + s_ent[ent_slot(d[i] >> 24, anchor)];
-                const uint32_t count = __reduce_add_sync(0xFFFFFFFFu, ((bits >> 16) + 15u) >> 4);     // (the low halves add up to less than 2^16)
+                    bits += s_len[ent_slot(__byte_perm(d[i], 0u, 0x4441), anchor)] + s_len[ent_slot(d[i] >> 24, anchor)];
+                const uint32_t count = __reduce_add_sync(0xFFFFFFFFu, (bits + 15u) >> 4);
                 gw[0] = anchor | (count << 8);
                 gw[1] = gw[2] = gw[3] = 0u;
             } else {
@@ -1205,9 +1209,9 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
 #pragma unroll
                 for (int i = 0; i < 32; i++) {
                     const uint32_t E = (i & 1) ? d[i >> 1] >> 24 : __byte_perm(d[i >> 1], 0u, 0x4441);
-                    const uint32_t slot = ent_slot(E, anchor);
-                    const uint32_t cw = s_ent[slot];
-                    acc |= ((cw & 0xFFFFu) | (slot == 10u ? E << 8 : 0u)) << n;
+                    const uint32_t cw = s_ent[ent_slot(E, anchor)];
+                    // (the table's escape entry is 0xFFFF: the AND lets the exponent through there only)
+                    acc |= (cw & ((E << 8) | 0xFFu)) << n;
                     n += cw >> 16;
                     if (i == 0) continue;
                     const bool more = n > 16u;             // the codeword runs past what the strand has taken
@@ -1926,7 +1930,7 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
                     const uint32_t st = stage_s + 8256u + 2u * before;
                     const uint32_t lt_mask = (1u << lane) - 1u;
                     uint32_t buf = 0, avail = 0, pos = 0, ew[8];
-                    bool over = false;
+                    const uint32_t last = mine - 1u;           // (mine >= 128)
 #pragma unroll
                     for (int j = 0; j < 8; j++) ew[j] = 0u;
 #pragma unroll
@@ -1934,21 +1938,21 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
                         const bool more = (s_parse[buf & 0xFFu] & 0xFFu) > avail;
                         const uint32_t takers = __ballot_sync(0xFFFFFFFFu, more);
                         if (more) {
-                            const uint32_t idx = pos + __popc(takers & lt_mask);
-                            uint32_t hw = 0;
-                            if (idx < mine) hw = lds_now_u16(st + 2u * idx); else over = true;
-                            buf |= hw << avail;
+                            // (an index past the stream's end is only clamped here: the stream then
+                            // fails the count check below, because every index is below the final pos)
+                            const uint32_t idx = min(pos + __popc(takers & lt_mask), last);
+                            buf |= lds_now_u16(st + 2u * idx) << avail;
                             avail += 16u;
                         }
                         pos += __popc(takers);
                         const uint32_t cw = s_parse[buf & 0xFFu];
                         const uint32_t len = cw & 0xFFu;
-                        const uint32_t E = (cw & 0x10000u) ? __byte_perm(buf, 0u, 0x4441) : (anchor + (cw >> 8)) & 0xFFu;
-                        ew[i >> 2] |= E << (8 * (i & 3));
+                        const uint32_t E = (cw & 0x10000u) ? buf >> 8 : anchor + (cw >> 8);      // (its low byte)
+                        ew[i >> 2] = __byte_perm(ew[i >> 2], E, (i & 3) == 0 ? 0x3214 : (i & 3) == 1 ? 0x3240 : (i & 3) == 2 ? 0x3410 : 0x4210);
                         buf >>= len;
                         avail -= len;
                     }
-                    if (__any_sync(0xFFFFFFFFu, over || buf != 0u) || pos != mine) verdict = 1;
+                    if (__any_sync(0xFFFFFFFFu, buf != 0u) || pos != mine) verdict = 1;
 #pragma unroll
                     for (int j = 0; j < 4; j++) {
                         sm[j] = j == 0 ? lds_now_v2<0>(sm_s) : j == 1 ? lds_now_v2<256>(sm_s) : j == 2 ? lds_now_v2<512>(sm_s) : lds_now_v2<768>(sm_s);
