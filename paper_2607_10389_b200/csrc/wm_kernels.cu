@@ -1830,12 +1830,14 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
          const Tables* __restrict__ tab)
 {
     extern __shared__ __align__(16) unsigned char smem[];
-    // ENT: what the low byte of a strand's bits says about the codeword there:
-    // length | (u & 0xFF) << 8 | escape << 16
-    __shared__ uint32_t s_parse[ENT ? 256 : 1];
+    // ENT: what the low byte of a strand's bits says about the codeword there: its length (16: the
+    // escape) and u as a byte.  Two byte tables: the index needs no scaling and a look-up gives a
+    // clean value.
+    __shared__ unsigned char s_plen[ENT ? 256 : 4], s_pu[ENT ? 256 : 4];
     if (ENT && threadIdx.x < 256u) {
         const uint32_t s = ent_ones(threadIdx.x);
-        s_parse[threadIdx.x] = ent_parse_length(s) | (ent_parse_value(threadIdx.x, s, 0u) << 8) | (s == 8u ? 0x10000u : 0u);
+        s_plen[threadIdx.x] = (unsigned char)ent_parse_length(s);
+        s_pu[threadIdx.x] = (unsigned char)(s == 8u ? 0u : ent_parse_value(threadIdx.x, s, 0u));
     }
     Smem S = setup_smem(smem, tab);
     grid_dep_wait();
@@ -1935,7 +1937,7 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
                     for (int j = 0; j < 8; j++) ew[j] = 0u;
 #pragma unroll
                     for (int i = 0; i < 32; i++) {
-                        const bool more = (s_parse[buf & 0xFFu] & 0xFFu) > avail;
+                        const bool more = s_plen[buf & 0xFFu] > avail;
                         const uint32_t takers = __ballot_sync(0xFFFFFFFFu, more);
                         if (more) {
                             // (an index past the stream's end is only clamped here: the stream then
@@ -1945,9 +1947,9 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
                             avail += 16u;
                         }
                         pos += __popc(takers);
-                        const uint32_t cw = s_parse[buf & 0xFFu];
-                        const uint32_t len = cw & 0xFFu;
-                        const uint32_t E = (cw & 0x10000u) ? buf >> 8 : anchor + (cw >> 8);      // (its low byte)
+                        const uint32_t low = buf & 0xFFu;
+                        const uint32_t len = s_plen[low];
+                        const uint32_t E = len == 16u ? buf >> 8 : anchor + s_pu[low];      // (its low byte)
                         ew[i >> 2] = __byte_perm(ew[i >> 2], E, (i & 3) == 0 ? 0x3214 : (i & 3) == 1 ? 0x3240 : (i & 3) == 2 ? 0x3410 : 0x4210);
                         buf >>= len;
                         avail -= len;
