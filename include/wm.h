@@ -276,6 +276,29 @@ wm_status wm_decode_verify_leaves(const void* wire, uint64_t wire_len, const wm_
                                   void* workspace, uint64_t workspace_bytes, wm_result* result, void* stream);
 
 /*
+ * wm_encode_opt / wm_decode_verify_opt - the codec calls with their options as an argument.
+ * The switches above are process-wide defaults for the plain calls; these two take the options
+ * per call and read nothing process-wide, so calls with different options can be issued from
+ * different threads and streams of one process.  Exactly one of (cache, leaves) and of (dst,
+ * dst_leaves) is non-NULL: the flat form or the leaf form (n_leaves is ignored in the flat form).
+ *   options  WM_OPT_ZERO_TILES (encode: the zero-tile option; ignored together with WM_OPT_ENTROPY)
+ *            WM_OPT_ENTROPY    (encode: write ENT tiles; decode: expect an image with ENT tiles)
+ *            WM_OPT_STRICT     (decode only: store nothing before every check has passed)
+ *            any other bit: WM_ERR_ARG, nothing is launched
+ * Everything else (arguments, layouts, statuses, what the result record holds) is as in
+ * wm_encode / wm_encode_leaves and wm_decode_verify / wm_decode_verify_leaves / _strict.
+ */
+#define WM_OPT_ZERO_TILES 1u
+#define WM_OPT_ENTROPY 2u
+#define WM_OPT_STRICT 4u
+wm_status wm_encode_opt(const void* cache, const wm_leaf* leaves, uint32_t n_leaves, uint64_t nbytes, uint32_t chunk_bytes,
+                        const uint8_t* dirty, uint32_t* crc_inout, void* wire, uint64_t wire_cap, void* workspace,
+                        uint64_t workspace_bytes, uint32_t options, wm_result* result, void* stream);
+wm_status wm_decode_verify_opt(const void* wire, uint64_t wire_len, void* dst, const wm_leaf* dst_leaves, uint32_t n_leaves,
+                               uint64_t nbytes, uint32_t chunk_bytes, uint32_t* dst_crc_inout, void* workspace,
+                               uint64_t workspace_bytes, uint32_t options, wm_result* result, void* stream);
+
+/*
  * wm_checksum_noalloc - wm_checksum for callers that cannot allocate device memory.
  * The paper has no counterpart to this call; it exists for hosts that may not call cudaMalloc
  * at the point where they need a checksum: code running inside a stream capture or under an

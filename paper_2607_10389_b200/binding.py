@@ -24,7 +24,7 @@ RESULT_BYTES = 40
 EXPORTS = ("wm_num_chunks", "wm_num_tiles", "wm_meta_bytes", "wm_wire_bound", "wm_workspace_bytes",
            "wm_checksum", "wm_dirty_diff", "wm_encode", "wm_decode_verify", "wm_last_launch_count",
            "wm_timing_enable", "wm_timing_read_ms", "wm_checksum_noalloc", "wm_encode_leaves",
-           "wm_decode_verify_leaves", "wm_zero_tiles_enable", "wm_decode_verify_strict", "wm_checksum_poly", "wm_entropy_enable")
+           "wm_decode_verify_leaves", "wm_zero_tiles_enable", "wm_decode_verify_strict", "wm_checksum_poly", "wm_entropy_enable", "wm_encode_opt", "wm_decode_verify_opt")
 
 
 class WmError(RuntimeError):
@@ -68,6 +68,10 @@ def load_library() -> ctypes.CDLL:
     lib.wm_decode_verify.argtypes = [vp, u64, vp, u64, u32, vp, vp, u64, vp, vp]
     lib.wm_decode_verify_strict.restype = ctypes.c_int
     lib.wm_decode_verify_strict.argtypes = [vp, u64, vp, u64, u32, vp, vp, u64, vp, vp]
+    lib.wm_encode_opt.restype = ctypes.c_int
+    lib.wm_encode_opt.argtypes = [vp, vp, u32, u64, u32, vp, vp, vp, u64, vp, u64, u32, vp, vp]
+    lib.wm_decode_verify_opt.restype = ctypes.c_int
+    lib.wm_decode_verify_opt.argtypes = [vp, u64, vp, vp, u32, u64, u32, vp, vp, u64, u32, vp, vp]
     lib.wm_encode_leaves.restype = ctypes.c_int
     lib.wm_encode_leaves.argtypes = [vp, u32, u64, u32, vp, vp, vp, u64, vp, u64, vp, vp]
     lib.wm_decode_verify_leaves.restype = ctypes.c_int
@@ -268,6 +272,40 @@ def wm_decode_verify_strict(wire: torch.Tensor, wire_len: int, dst: torch.Tensor
     _check(lib().wm_decode_verify_strict(wire.data_ptr(), int(wire_len), dst.data_ptr(), nbytes, chunk_bytes,
                                          dst_crc_inout.data_ptr(), workspace.data_ptr(), workspace.numel(),
                                          result.data_ptr(), _stream(stream)), "wm_decode_verify_strict")
+
+
+OPT_ZERO_TILES, OPT_ENTROPY, OPT_STRICT = 1, 2, 4
+
+
+def wm_encode_opt(cache, chunk_bytes: int, dirty, crc_inout: torch.Tensor, wire: torch.Tensor, workspace: torch.Tensor,
+                  result: torch.Tensor, options: int, stream=None, leaf_table=None, nbytes=None) -> None:
+    """wm_encode / wm_encode_leaves with the options given per call (OPT_ZERO_TILES, OPT_ENTROPY).
+    Flat form: `cache` is a tensor; leaf form: `cache` is None, `leaf_table` and `nbytes` are given."""
+    _dev_u8(wire, "wire")
+    if leaf_table is None:
+        _dev_u8(cache, "cache")
+        n, cp, lp, nl = cache.numel() * cache.element_size(), cache.data_ptr(), None, 0
+    else:
+        n, cp, lp, nl = int(nbytes), None, leaf_table.data_ptr(), leaf_table.shape[0]
+    _check(lib().wm_encode_opt(cp, lp, nl, n, chunk_bytes, None if dirty is None else dirty.data_ptr(), crc_inout.data_ptr(),
+                               wire.data_ptr(), wire.numel(), workspace.data_ptr(), workspace.numel(), int(options),
+                               result.data_ptr(), _stream(stream)), "wm_encode_opt")
+
+
+def wm_decode_verify_opt(wire: torch.Tensor, wire_len: int, dst, chunk_bytes: int, dst_crc_inout: torch.Tensor,
+                         workspace: torch.Tensor, result: torch.Tensor, options: int, stream=None, leaf_table=None,
+                         nbytes=None) -> None:
+    """The decode calls with the options given per call (OPT_ENTROPY: the image holds ENT tiles;
+    OPT_STRICT: nothing is stored before the verdict)."""
+    _dev_u8(wire, "wire")
+    if leaf_table is None:
+        _dev_u8(dst, "dst")
+        n, dp, lp, nl = dst.numel() * dst.element_size(), dst.data_ptr(), None, 0
+    else:
+        n, dp, lp, nl = int(nbytes), None, leaf_table.data_ptr(), leaf_table.shape[0]
+    _check(lib().wm_decode_verify_opt(wire.data_ptr(), int(wire_len), dp, lp, nl, n, chunk_bytes, dst_crc_inout.data_ptr(),
+                                      workspace.data_ptr(), workspace.numel(), int(options), result.data_ptr(),
+                                      _stream(stream)), "wm_decode_verify_opt")
 
 
 def make_leaf_table(tensors, device="cuda") -> torch.Tensor:

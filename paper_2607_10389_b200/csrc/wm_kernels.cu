@@ -2510,11 +2510,19 @@ wm_status wm_dirty_diff(const void* cache, const void* prev, uint64_t nbytes, ui
 }
 
 // Both forms of the encode call: a flat cache (leaves == nullptr) or a table of leaves.
+// The options the plain calls use: the process-wide switches.
+static uint32_t default_options()
+{
+    return (g_zero_tiles ? WM_OPT_ZERO_TILES : 0u) | (g_entropy ? WM_OPT_ENTROPY : 0u);
+}
+
 static wm_status encode_any(const void* cache, const wm_leaf* leaves, uint32_t n_leaves, uint64_t nbytes, uint32_t chunk_bytes,
                             const uint8_t* dirty, uint32_t* crc_inout, void* wire, uint64_t wire_cap, void* workspace,
-                            uint64_t workspace_bytes, wm_result* result, void* stream)
+                            uint64_t workspace_bytes, wm_result* result, void* stream, uint32_t options)
 {
     Geo g;
+    if (options & ~(WM_OPT_ZERO_TILES | WM_OPT_ENTROPY)) return WM_ERR_ARG;
+    const bool opt_ent = (options & WM_OPT_ENTROPY) != 0, opt_zero = (options & WM_OPT_ZERO_TILES) != 0;
     if (!crc_inout || !wire || !workspace || !result || !make_geo(nbytes, chunk_bytes, g)) return WM_ERR_ARG;
     if (leaves ? (n_leaves == 0 || n_leaves > kMaxLeaves) : (!cache || !aligned16(cache))) return WM_ERR_ARG;
     if (!aligned16(wire) || !aligned16(workspace) || workspace_bytes < ws_layout(g).total || wire_cap < g.meta_end)
@@ -2538,7 +2546,7 @@ static wm_status encode_any(const void* cache, const wm_leaf* leaves, uint32_t n
     {
         MainKernelTimer timer(ds, 2, s);
         // the entropy option takes precedence over the zero-tile option
-        const int variant = (dirty ? 1 : 0) | (leaves ? 2 : 0) | (g_entropy ? 8 : g_zero_tiles ? 4 : 0);
+        const int variant = (dirty ? 1 : 0) | (leaves ? 2 : 0) | (opt_ent ? 8 : opt_zero ? 4 : 0);
         auto go = [&](auto kernel) { launch_after(kernel, grid, kTeams * 256, kDynSmem, s, c, g, dirty, w, wire_cap, ws, ds->tables); };
         switch (variant) {
             case 0: go(k_encode<kTeams, false, false, false>); break;
@@ -2556,7 +2564,7 @@ static wm_status encode_any(const void* cache, const wm_leaf* leaves, uint32_t n
         }
     }
     launch_after(k_encode_finish, (g.n_chunks + g.finish_cb - 1) / g.finish_cb, 1024, 0, s, c, g, dirty, crc_inout, w, ws, ds->tables,
-                 chunk_powers(g), g_entropy ? 4u : g_zero_tiles ? 2u : 0u);
+                 chunk_powers(g), opt_ent ? 4u : opt_zero ? 2u : 0u);
     launch_after(k_meta_crc, (g.n_meta_slices + 3) / 4, 1024, kDynSmem, s, w, g, ws, ds->tables, result);
     g_launches = leaves ? 5 : 4;
     return launch_status();
@@ -2567,7 +2575,8 @@ wm_status wm_encode(const void* cache, uint64_t nbytes, uint32_t chunk_bytes, co
                     wm_result* result, void* stream)
 {
     if (!cache) return WM_ERR_ARG;
-    return encode_any(cache, nullptr, 0, nbytes, chunk_bytes, dirty, crc_inout, wire, wire_cap, workspace, workspace_bytes, result, stream);
+    return encode_any(cache, nullptr, 0, nbytes, chunk_bytes, dirty, crc_inout, wire, wire_cap, workspace, workspace_bytes, result, stream,
+                      default_options());
 }
 
 wm_status wm_encode_leaves(const wm_leaf* leaves, uint32_t n_leaves, uint64_t nbytes, uint32_t chunk_bytes, const uint8_t* dirty,
@@ -2575,16 +2584,19 @@ wm_status wm_encode_leaves(const wm_leaf* leaves, uint32_t n_leaves, uint64_t nb
                            wm_result* result, void* stream)
 {
     if (!leaves) return WM_ERR_ARG;
-    return encode_any(nullptr, leaves, n_leaves, nbytes, chunk_bytes, dirty, crc_inout, wire, wire_cap, workspace, workspace_bytes, result, stream);
+    return encode_any(nullptr, leaves, n_leaves, nbytes, chunk_bytes, dirty, crc_inout, wire, wire_cap, workspace, workspace_bytes, result, stream,
+                      default_options());
 }
 
 // Both forms of the decode call: a flat shadow buffer (leaves == nullptr) or a table of leaves.
 // strict: nothing is stored until every check has passed (two passes over the wire image).
 static wm_status decode_any(const void* wire, uint64_t wire_len, void* dst, const wm_leaf* leaves, uint32_t n_leaves, uint64_t nbytes,
                             uint32_t chunk_bytes, uint32_t* dst_crc_inout, void* workspace, uint64_t workspace_bytes,
-                            wm_result* result, void* stream, bool strict)
+                            wm_result* result, void* stream, uint32_t options)
 {
     Geo g;
+    if (options & ~(WM_OPT_ZERO_TILES | WM_OPT_ENTROPY | WM_OPT_STRICT)) return WM_ERR_ARG;
+    const bool strict = (options & WM_OPT_STRICT) != 0;
     if (!wire || !dst_crc_inout || !workspace || !result || !make_geo(nbytes, chunk_bytes, g)) return WM_ERR_ARG;
     if (leaves ? (n_leaves == 0 || n_leaves > kMaxLeaves) : (!dst || !aligned16(dst))) return WM_ERR_ARG;
     if (!aligned16(wire) || !aligned16(workspace) || workspace_bytes < ws_layout(g).total) return WM_ERR_ARG;
@@ -2602,7 +2614,7 @@ static wm_status decode_any(const void* wire, uint64_t wire_len, void* dst, cons
     }
     // a wire shorter than the metadata is rejected by the header check before anything else is read
     const uint32_t meta_blocks = (g.n_meta_slices + 3) / 4;
-    const bool ent = g_entropy;      // the option says which kind of image the call expects
+    const bool ent = (options & WM_OPT_ENTROPY) != 0;      // the option says which kind of image the call expects
     launch_after(k_decode_check, meta_blocks + (g.n_chunks + 31) / 32, 1024, 0, s, w, wire_len, g, ws, ds->tables, result, meta_blocks,
                  ent ? 1u : 0u);
     const uint32_t need = (g.n_tiles + kTeamsPlain - 1) / kTeamsPlain;
@@ -2637,7 +2649,7 @@ wm_status wm_decode_verify(const void* wire, uint64_t wire_len, void* dst, uint6
 {
     if (!dst) return WM_ERR_ARG;
     return decode_any(wire, wire_len, dst, nullptr, 0, nbytes, chunk_bytes, dst_crc_inout, workspace, workspace_bytes, result, stream,
-                      false);
+                      default_options());
 }
 
 wm_status wm_decode_verify_strict(const void* wire, uint64_t wire_len, void* dst, uint64_t nbytes, uint32_t chunk_bytes,
@@ -2646,7 +2658,7 @@ wm_status wm_decode_verify_strict(const void* wire, uint64_t wire_len, void* dst
 {
     if (!dst) return WM_ERR_ARG;
     return decode_any(wire, wire_len, dst, nullptr, 0, nbytes, chunk_bytes, dst_crc_inout, workspace, workspace_bytes, result, stream,
-                      true);
+                      default_options() | WM_OPT_STRICT);
 }
 
 wm_status wm_decode_verify_leaves(const void* wire, uint64_t wire_len, const wm_leaf* dst_leaves, uint32_t n_leaves, uint64_t nbytes,
@@ -2655,7 +2667,27 @@ wm_status wm_decode_verify_leaves(const void* wire, uint64_t wire_len, const wm_
 {
     if (!dst_leaves) return WM_ERR_ARG;
     return decode_any(wire, wire_len, nullptr, dst_leaves, n_leaves, nbytes, chunk_bytes, dst_crc_inout, workspace, workspace_bytes, result,
-                      stream, false);
+                      stream, default_options());
+}
+
+// The calls with their options as an argument (nothing process-wide is read): a cache as one
+// buffer (leaves == NULL) or as a table of leaves (cache / dst == NULL).
+wm_status wm_encode_opt(const void* cache, const wm_leaf* leaves, uint32_t n_leaves, uint64_t nbytes, uint32_t chunk_bytes,
+                        const uint8_t* dirty, uint32_t* crc_inout, void* wire, uint64_t wire_cap, void* workspace,
+                        uint64_t workspace_bytes, uint32_t options, wm_result* result, void* stream)
+{
+    if ((cache != nullptr) == (leaves != nullptr)) return WM_ERR_ARG;
+    return encode_any(cache, leaves, n_leaves, nbytes, chunk_bytes, dirty, crc_inout, wire, wire_cap, workspace, workspace_bytes, result, stream,
+                      options);
+}
+
+wm_status wm_decode_verify_opt(const void* wire, uint64_t wire_len, void* dst, const wm_leaf* dst_leaves, uint32_t n_leaves,
+                               uint64_t nbytes, uint32_t chunk_bytes, uint32_t* dst_crc_inout, void* workspace,
+                               uint64_t workspace_bytes, uint32_t options, wm_result* result, void* stream)
+{
+    if ((dst != nullptr) == (dst_leaves != nullptr)) return WM_ERR_ARG;
+    return decode_any(wire, wire_len, dst, dst_leaves, n_leaves, nbytes, chunk_bytes, dst_crc_inout, workspace, workspace_bytes, result, stream,
+                      options);
 }
 
 }  // extern "C"

@@ -78,10 +78,12 @@ class TailSchedule:
     """Buffers, streams and events for moving one cache geometry super-chunk by super-chunk."""
 
     def __init__(self, nbytes: int, chunk_bytes: int, super_bytes: int = 64 << 20, device="cuda", strict=False,
-                 ahead: int = 2):
+                 ahead: int = 2, entropy: bool = False):
         self.nbytes, self.chunk_bytes, self.super_bytes = int(nbytes), int(chunk_bytes), int(super_bytes)
         self.parts = plan_parts(self.nbytes, self.chunk_bytes, self.super_bytes)
         self.strict = strict
+        self.enc_options = wm.OPT_ENTROPY if entropy else 0
+        self.dec_options = self.enc_options | (wm.OPT_STRICT if strict else 0)
         total_wire = self.parts[-1].wire_offset + self.parts[-1].wire_cap
         self.wire_send = torch.empty(total_wire, dtype=torch.uint8, device=device)
         self.wire_recv = torch.empty(total_wire, dtype=torch.uint8, device=device)
@@ -114,7 +116,6 @@ class TailSchedule:
         """Move `src` into `dst` part by part.  `src_crc` receives the source's chunk CRCs, `dst_crc`
         is updated for every part that verified.  `tamper(part, received_image)` may alter a part's
         received bytes before they are decoded (tests use it to damage one part on the wire)."""
-        decode = wm.wm_decode_verify_strict if self.strict else wm.wm_decode_verify
         src, dst = src.reshape(-1).view(torch.uint8), dst.reshape(-1).view(torch.uint8)
         if src.numel() != self.nbytes or dst.numel() != self.nbytes:
             raise wm.WmError("cache size differs from the schedule's geometry")
@@ -129,9 +130,9 @@ class TailSchedule:
         for i in range(n + self.ahead):
             if i < n:
                 p = self.parts[i]
-                wm.wm_encode(src[p.offset: p.offset + p.nbytes], C, None,
-                             src_crc[p.first_chunk: p.first_chunk + p.n_chunks], self._send[i],
-                             self.ws_enc, self._res_enc[i], stream=self.s_enc)
+                wm.wm_encode_opt(src[p.offset: p.offset + p.nbytes], C, None,
+                                 src_crc[p.first_chunk: p.first_chunk + p.n_chunks], self._send[i],
+                                 self.ws_enc, self._res_enc[i], self.enc_options, stream=self.s_enc)
                 launches += wm.last_launch_count()
                 with torch.cuda.stream(self.s_enc):
                     self._host_enc[i].copy_(self._res_enc[i], non_blocking=True)
@@ -152,9 +153,9 @@ class TailSchedule:
                         tamper(p, self._recv[j][:length])
             self.ev_wire[j].record(self.s_wire)
             self.s_dec.wait_event(self.ev_wire[j])
-            decode(self._recv[j], length, dst[p.offset: p.offset + p.nbytes], C,
-                   dst_crc[p.first_chunk: p.first_chunk + p.n_chunks], self.ws_dec, self._res_dec[j],
-                   stream=self.s_dec)
+            wm.wm_decode_verify_opt(self._recv[j], length, dst[p.offset: p.offset + p.nbytes], C,
+                                    dst_crc[p.first_chunk: p.first_chunk + p.n_chunks], self.ws_dec, self._res_dec[j],
+                                    self.dec_options, stream=self.s_dec)
             launches += wm.last_launch_count()
         self.ev_end.record(self.s_dec)
         cur.wait_stream(self.s_dec)

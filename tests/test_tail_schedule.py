@@ -35,14 +35,14 @@ def _cache(n, seed):
 
 
 @pytest.mark.gpu
-@pytest.mark.parametrize("strict", [False, True])
-def test_every_part_is_the_oracles_image_of_its_range(strict):
+@pytest.mark.parametrize("strict,entropy", [(False, False), (True, False), (False, True), (True, True)])
+def test_every_part_is_the_oracles_image_of_its_range(strict, entropy):
     import torch
     from paper_2607_10389_b200 import tail_schedule as ts
     chunk, sup = 4 * TILE, 12 * TILE
     n = 3 * sup + 5 * TILE + 321                         # three full parts and a ragged one
     a = _cache(n, 11)
-    sched = ts.TailSchedule(n, chunk, sup, strict=strict)
+    sched = ts.TailSchedule(n, chunk, sup, strict=strict, entropy=entropy)
     assert len(sched.parts) == 4
     nc = oracle.num_chunks(n, chunk)
     src = torch.from_numpy(a).cuda()
@@ -57,7 +57,7 @@ def test_every_part_is_the_oracles_image_of_its_range(strict):
     assert np.array_equal(dst_crc.cpu().numpy().view(np.uint32), want_crc)
     total = 0
     for p, re, rd in zip(sched.parts, rep.encode, rep.decode):
-        wire, crc, res = oracle.encode(a[p.offset: p.offset + p.nbytes], chunk)
+        wire, crc, res = oracle.encode(a[p.offset: p.offset + p.nbytes], chunk, entropy=entropy)
         assert re.wire_len == wire.size == res.wire_len and re.cache_crc == res.cache_crc == rd.cache_crc
         got = sched.wire_recv[p.wire_offset: p.wire_offset + re.wire_len].cpu().numpy()
         assert np.array_equal(got, wire)
