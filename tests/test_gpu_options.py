@@ -71,3 +71,45 @@ def test_options_leaf_form_and_bad_arguments():
         wm.wm_encode_opt(leaves[0], chunk, None, crc, wire, ws, res, wm.OPT_STRICT)          # decode-only option
     with pytest.raises(wm.WmError, match="ERR_ARG"):
         wm.wm_decode_verify_opt(wire, r.wire_len, leaves[0], chunk, crc, ws, res, 16)
+
+
+def test_two_host_threads_with_different_options():
+    """Two threads of one process, each with its own stream, geometry, workspace and options, issue
+    calls at the same time; both get the oracle's images (the per-thread geometry caches and the
+    per-call options keep them apart)."""
+    import threading
+    import torch
+    from paper_2607_10389_b200 import binding as wm
+    jobs = [(11 * TILE + 5, 2 * TILE, wm.OPT_ENTROPY, {"entropy": True}), (16 * TILE, 4 * TILE, 0, {})]
+    errors = []
+
+    def work(k):
+        try:
+            n, chunk, opt, kw = jobs[k]
+            a = _cache(n, 40 + k)
+            want, want_crc, _ = oracle.encode(a, chunk, **kw)
+            stream = torch.cuda.Stream()
+            with torch.cuda.stream(stream):
+                src = torch.from_numpy(a).cuda()
+                nc = wm.num_chunks(n, chunk)
+                ws = wm.new_workspace(n, chunk)
+                wire = torch.empty(wm.wire_bound(n, chunk), dtype=torch.uint8, device="cuda")
+                crc = torch.zeros(nc, dtype=torch.int32, device="cuda")
+                res = wm.new_result()
+                dst = torch.zeros(n, dtype=torch.uint8, device="cuda")
+                for _ in range(40):
+                    wm.wm_encode_opt(src, chunk, None, crc, wire, ws, res, opt, stream=stream)
+                    wm.wm_decode_verify_opt(wire, want.size, dst, chunk, crc, ws, res, opt, stream=stream)
+                stream.synchronize()
+                r = wm.read_result(res)
+                assert r.status == 0 and np.array_equal(wire[: want.size].cpu().numpy(), want)
+                assert np.array_equal(dst.cpu().numpy(), a) and np.array_equal(crc.cpu().numpy().view(np.uint32), want_crc)
+        except BaseException as e:      # noqa: BLE001 - reported by the main thread
+            errors.append(repr(e))
+
+    threads = [threading.Thread(target=work, args=(k,)) for k in range(2)]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    assert not errors, errors
