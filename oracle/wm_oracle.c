@@ -423,6 +423,11 @@ static uint32_t encode_full_tile(const uint8_t* src, uint8_t* out, uint32_t* ent
         uint32_t any = 0;
         for (uint32_t i = 0; i < WMO_TILE; i++) any |= src[i];
         if (!any) { *entry = 1u; return 0; }
+        /* the same option: a tile whose 8192 elements all hold one (non-zero) value is entry 2 and
+         * 32 bytes of payload, the value first (little-endian u16), then 30 zero bytes */
+        uint32_t v0 = get16(src), same = 1;
+        for (uint32_t e = 1; e < 8192u; e++) if (get16(src + 2u * e) != v0) { same = 0; break; }
+        if (same) { memset(out, 0, 32); put16(out, v0); *entry = 2u; return 32u; }
     }
     /* option: entropy-coded exponents; the tile is an ENT tile when that is shorter than raw */
     if (options & WMO_OPT_ENTROPY) {
@@ -492,6 +497,8 @@ static uint32_t encode_full_tile(const uint8_t* src, uint8_t* out, uint32_t* ent
  *           40 u64 wire_len 48 u32 cache_crc     52 u32 meta_crc   56 8 zero bytes
  *   chunk_dir[c]: u64 payload_off | u32 enc_len | u32 crc
  *   tile_tab[t] : 0 absent | 1 ZERO full tile (all bytes zero, no payload) |
+ *                 2 CONST full tile (all 8192 elements equal and not zero; payload = the
+ *                 value, u16, and 30 zero bytes; entries 1 and 2 only with flags bit1) |
  *                 258..511 PACK of 32*value bytes | 512 RAW full tile |
  *                 0x8000 | n, n = 259..511: ENT of 32 n bytes | 0xFFFF RAW partial tail tile
  *   payload: encoded tiles of present chunks in ascending order, no padding.
@@ -710,6 +717,7 @@ int wmo_decode_verify_opt(const uint8_t* wire, uint64_t wire_len, uint8_t* dst, 
                 any = 1;
                 if (tlen < WMO_TILE) { if (e != 0xFFFFu) ok = 0; sum += tlen; }
                 else if (e == 1u && zero_ok) sum += 0;     /* ZERO tile: full tiles only, no payload */
+                else if (e == 2u && zero_ok) sum += 32u;   /* CONST tile: the value in 32 bytes of payload */
                 else if (e == 512u || (!ent_on && e >= 258u && e <= 511u)) sum += 32u * (uint64_t)e;
                 else if (ent_on && e >= (0x8000u | 259u) && e <= (0x8000u | 511u)) sum += 32u * (uint64_t)(e & 0x7FFFu);
                 else ok = 0;
@@ -735,7 +743,7 @@ int wmo_decode_verify_opt(const uint8_t* wire, uint64_t wire_len, uint8_t* dst, 
             for (uint64_t i = 0; i < ntc; i++) {
                 uint32_t e = get16(tab + 2u * (t0 + i));
                 if (e == 0) break;
-                uint64_t tlen = (e == 0xFFFFu) ? clen - i * WMO_TILE : (e == 1u) ? 0 : 32u * (uint64_t)(e & 0x7FFFu);
+                uint64_t tlen = (e == 0xFFFFu) ? clen - i * WMO_TILE : (e == 1u) ? 0 : (e == 2u) ? 32u : 32u * (uint64_t)(e & 0x7FFFu);
                 if (e != 0xFFFFu && (e & 0x8000u)) {
                     /* ENT tile: the header against the entry -> STRUCT, then every stream must be used up exactly -> DESC */
                     int tile_status = WMO_OK;
@@ -778,8 +786,9 @@ int wmo_decode_verify_opt(const uint8_t* wire, uint64_t wire_len, uint8_t* dst, 
             uint8_t* out = dst + c * (uint64_t)chunk_bytes;
             for (uint64_t i = 0; i < ntc; i++) {
                 uint32_t e = get16(tab + 2u * (t0 + i));
-                uint64_t tlen = (e == 0xFFFFu) ? clen - i * WMO_TILE : (e == 1u) ? 0 : 32u * (uint64_t)(e & 0x7FFFu);
+                uint64_t tlen = (e == 0xFFFFu) ? clen - i * WMO_TILE : (e == 1u) ? 0 : (e == 2u) ? 32u : 32u * (uint64_t)(e & 0x7FFFu);
                 if (e == 1u) memset(out + i * WMO_TILE, 0, WMO_TILE);
+                else if (e == 2u) { for (uint32_t k = 0; k < 8192u; k++) memcpy(out + i * WMO_TILE + 2u * k, payload + off, 2); }
                 else if (e != 0xFFFFu && (e & 0x8000u)) decode_ent_tile(payload + off, out + i * WMO_TILE);
                 else if (e == 512u || e == 0xFFFFu) memcpy(out + i * WMO_TILE, payload + off, tlen);
                 else decode_pack_tile(payload + off, out + i * WMO_TILE);

@@ -430,6 +430,49 @@ def test_only_all_zero_bytes_make_a_zero_tile(word):
     assert r.status == 0 and np.array_equal(out, tile.view(np.uint8))
 
 
+def test_constant_tiles_have_entry_two_and_the_value_as_payload():
+    """Same option: a tile whose elements all hold one non-zero value (-Inf as a mask fill, 1.0)
+    ships as entry 2 and 32 bytes: the value, then zeros.  Written out by hand here."""
+    a = _rand_tile(3)
+    minus_inf = np.full(8192, 0xFF80, dtype="<u2").view(np.uint8)
+    one = np.full(8192, 0x3F80, dtype="<u2").view(np.uint8)
+    z = np.zeros(TILE, dtype=np.uint8)
+    cache = np.concatenate([minus_inf, a, one, z])
+    wire, crc, res = oracle.encode(cache, 2 * TILE, zero_tiles=True)
+    wa, _, ra = oracle.encode(a, TILE)
+    ea = wa[96:ra.wire_len]
+    assert _tab(wire, 2, 4).tolist() == [2, int(_tab(wa, 1, 1)[0]), 2, 1]
+    me = oracle.meta_end(4 * TILE, 2 * TILE)
+    want = np.concatenate([np.array([0x80, 0xFF] + [0] * 30, np.uint8), ea, np.array([0x80, 0x3F] + [0] * 30, np.uint8)])
+    assert np.array_equal(wire[me:], want) and res.payload_bytes == want.size
+    assert [d[:2] for d in _dir(wire, 2)] == [(0, 32 + ea.size), (32 + ea.size, 32)]
+    assert struct.unpack_from("<H", wire, 6)[0] == 2
+    out, dcrc, r = oracle.decode_verify(wire, cache.size, 2 * TILE, dst=np.full(cache.size, 0xEE, np.uint8))
+    assert r.status == 0 and np.array_equal(out, cache) and np.array_equal(dcrc, crc)
+    # one element off: an ordinary tile again; and without the option nothing changes
+    c2 = cache.copy()
+    c2[100] ^= 1
+    w2, _, _ = oracle.encode(c2, 2 * TILE, zero_tiles=True)
+    assert _tab(w2, 2, 4)[0] >= 258
+    w3, _, _ = oracle.encode(cache, 2 * TILE)
+    assert min(_tab(w3, 2, 4).tolist()) >= 258
+    # entry 2 in an image that does not declare the option, a damaged value, a CONST entry on a ragged tile
+    bad = wire.copy()
+    bad[6] = 0
+    assert oracle.decode_verify(_refresh_meta_crc(bad, cache.size, 2 * TILE), cache.size, 2 * TILE)[2].status_name == "ERR_STRUCT"
+    bad = wire.copy()
+    bad[me] ^= 1
+    r = oracle.decode_verify(bad, cache.size, 2 * TILE)[2]
+    assert r.status_name == "ERR_CHUNK_CRC" and r.first_bad_chunk == 0
+    n = TILE + 64
+    rag = np.full(n // 2, 0x3F80, dtype="<u2").view(np.uint8)
+    wr, _, _ = oracle.encode(rag, 2 * TILE, zero_tiles=True)
+    assert _tab(wr, 1, 2).tolist() == [2, 0xFFFF]
+    wr = wr.copy()
+    struct.pack_into("<H", wr, 64 + 16 + 2, 2)
+    assert oracle.decode_verify(_refresh_meta_crc(wr, n, 2 * TILE), n, 2 * TILE)[2].status_name == "ERR_STRUCT"
+
+
 def _refresh_meta_crc(wire, nbytes, chunk):
     me = oracle.meta_end(nbytes, chunk)
     w = wire.copy()
