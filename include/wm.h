@@ -131,7 +131,9 @@ wm_status wm_dirty_diff(const void* cache, const void* prev, uint64_t nbytes, ui
  *           52 u32 meta_crc (CRC32C of the metadata with this field as zero) | 56 zero[8]
  *   chunk_dir[c]: u64 payload_off | u32 enc_len | u32 crc
  *   tile_tab[t] (u16): 0 tile of an absent chunk | 1 ZERO tile: a full tile whose bytes are
- *           all zero, no payload (only in images with flags bit1) | 258..511 PACK tile of 32*value bytes
+ *           all zero, no payload (only in images with flags bit1) | 2 CONST tile: a full tile whose 8192
+ *           elements all hold one non-zero value; payload = that value (u16) and 30 zero bytes
+ *           (only in images with flags bit1) | 258..511 PACK tile of 32*value bytes
  *           (only without flags bit2) | 512 RAW full tile | 0x8000 | n, n = 259..511: ENT tile of
  *           32*n bytes (only with flags bit2) | 0xFFFF RAW partial tail tile (nbytes mod 16384 bytes)
  *   payload: encoded tiles of present chunks in ascending order, no padding
@@ -210,9 +212,11 @@ wm_status wm_decode_verify_strict(const void* wire, uint64_t wire_len, void* dst
  * (Section 3.3).  Read here as zero-filled memory: with the option on, a full tile of a
  * present chunk whose 16384 bytes are all zero gets tile_tab entry 1 and no payload bytes
  * (without it such a tile packs to 8256 bytes), and header flags bit1 is set.  Only the
- * all-zero byte pattern qualifies (minus zero and denormals are data).  The decoder accepts
- * entry 1 in images that declare the option and writes zeros, which it checksums like any
- * decoded tile.  Process-wide switch, off by default (the detection costs the encoder about
+ * all-zero byte pattern qualifies for entry 1 (minus zero and denormals are data).  A full tile
+ * whose 8192 elements all hold one other value (a mask fill such as -Inf, say) gets entry 2 and
+ * 32 bytes of payload: the value, little-endian, and 30 zero bytes.  The decoder accepts
+ * entries 1 and 2 in images that declare the option, writes the zeros or the value, and
+ * checksums them like any decoded tile.  Process-wide switch, off by default (the detection costs the encoder about
  * 3 % on caches without such tiles); applies to wm_encode and wm_encode_leaves.
  */
 void wm_zero_tiles_enable(int on);

@@ -927,7 +927,9 @@ __device__ __forceinline__ uint32_t ent_parse_value(uint32_t buf, uint32_t s, ui
 constexpr uint32_t kQPresent = 1u << 31, kQFirst = 1u << 30, kQTile = (1u << 30) - 1u, kQNone = kQTile;
 // Marks in a team's width table: on a warp's first entry, all 2 KiB of the warp's rows are zero;
 // as the sum of the widths, the tile is all zero.
-constexpr uint32_t kWarpAllZero = 0x8000u, kSumZeroTile = 0xFFFFu;
+// kWarpConst: all 1024 elements of the warp's rows hold one value (its sign-mantissa byte rides in
+// bits 16-23 of the entry, the exponent is the base); kSumConstTile: the tile holds one value.
+constexpr uint32_t kWarpAllZero = 0x8000u, kWarpConst = 0x4000u, kSumZeroTile = 0xFFFFu, kSumConstTile = 0xFFFEu;
 
 template <bool MASKED>
 __device__ __forceinline__ uint32_t describe_tile(const Geo& g, const uint8_t* __restrict__ dirty, uint32_t t)
@@ -1119,11 +1121,15 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
             }
             // Option ZEROS.  Unused memory: when all four groups have exponent 0 throughout (rare in live data)
             // look at the words themselves; a warp whose 2 KiB are all zero marks its first entry.
-            if (ZEROS && (gw[0] | gw[1] | gw[2] | gw[3]) == 0u) {
-                uint32_t any = 0;
+            // The same for any one value (a mask fill, say): all four groups have one exponent and width
+            // 0; then every word must equal the warp's first, and that word's two halves each other.
+            if (ZEROS && gw[0] < 256u && gw[1] == gw[0] && gw[2] == gw[0] && gw[3] == gw[0]) {
+                const uint32_t first = __shfl_sync(0xFFFFFFFFu, d[0], 0);
+                uint32_t diff = (first >> 16) ^ (first & 0xFFFFu);
 #pragma unroll
-                for (int i = 0; i < 16; i++) any |= d[i];
-                if (!__any_sync(0xFFFFFFFFu, any != 0u)) gw[0] = kWarpAllZero;
+                for (int i = 0; i < 16; i++) diff |= d[i] ^ first;
+                if (!__any_sync(0xFFFFFFFFu, diff != 0u))
+                    gw[0] |= kWarpConst | ((first & 0xFFu) << 16) | (first == 0u ? kWarpAllZero : 0u);
             }
             // one lane leaves the warp's results; the warp that arrives last turns the 32 widths
             // into offsets and publishes the tile's length
@@ -1142,12 +1148,16 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
                 // (ENT: every warp's first entry carries its stream's halfwords, the other three are zero)
                 const uint32_t total = __reduce_add_sync(0xFFFFFFFFu, ENT ? wt >> 8 : (wt >> 8) & 15u);
                 // unused memory (every warp's first entry carries the mark): no payload
-                const bool zero_tile = ZEROS && __all_sync(0xFFFFFFFFu, (lane & 3u) != 0u || (wt & kWarpAllZero) != 0u);
+                // (one value throughout: every warp's first entry carries the mark and they are all alike;
+                // a tile of zeros has no payload, any other value 32 bytes)
+                const uint32_t wt0 = __shfl_sync(0xFFFFFFFFu, wt, 0);
+                const bool const_tile = ZEROS && __all_sync(0xFFFFFFFFu, (lane & 3u) != 0u || ((wt & kWarpConst) != 0u && wt == wt0));
+                const bool zero_tile = const_tile && (wt0 & kWarpAllZero) != 0u;
                 if (lane == 0) {
-                    tc->ssum[slY] = zero_tile ? kSumZeroTile : total;
+                    tc->ssum[slY] = zero_tile ? kSumZeroTile : const_tile ? kSumConstTile : total;
                     tc->wsum[slY] = 0;
                     if (ENT) publish_len(tYn, ent_tile_bytes(total) < kTile ? ent_tile_bytes(total) : kTile);
-                    else publish_len(tYn, zero_tile ? 0u : total <= 253u ? 8256u + 32u * total : kTile);
+                    else publish_len(tYn, zero_tile ? 0u : const_tile ? 32u : total <= 253u ? 8256u + 32u * total : kTile);
                 }
             }
 #ifndef WM_AB_NOTMEM
@@ -1174,7 +1184,8 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
             const bool packs = ENT ? ent_tile_bytes(Ssum) < kTile : Ssum <= 253u;
             // (a tile of all-zero bytes, marked in ssum, is its table entry and nothing else)
             const uint32_t enc_len = ENT ? (packs ? ent_tile_bytes(Ssum) : kTile)
-                                         : packs ? 8256u + 32u * Ssum : (ZEROS && Ssum == kSumZeroTile) ? 0u : kTile;
+                                         : packs ? 8256u + 32u * Ssum : (ZEROS && Ssum == kSumZeroTile) ? 0u
+                                         : (ZEROS && Ssum == kSumConstTile) ? 32u : kTile;
             unsigned char* const dst = payload + exclX;
             if (exclX + enc_len > room) {
                 trouble |= 1u;
@@ -1265,6 +1276,9 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
 #else
                 if (d[5] == 0x12345678u) stg_u8(dst + lane, d[1]);
 #endif
+            } else if (ZEROS && Ssum == kSumConstTile) {
+                // the value (any word's low half, rotated back), then 30 zero bytes
+                if (warp == 5 && lane < 8u) st_stream_u32(dst + 4u * lane, lane == 0u ? __funnelshift_r(d[0], d[0], 1) & 0xFFFFu : 0u);
             } else if (enc_len) {
                 unsigned char* q = dst + warp * 2048u + lane * 4u;
 #pragma unroll
@@ -1296,8 +1310,8 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
                         entry = nb < kTile ? 0x8000u | (nb / 32u) : 512u;
                         enc_len = nb < kTile ? nb : kTile;
                     } else {
-                        entry = Ssum <= 253u ? 258u + Ssum : (ZEROS && Ssum == kSumZeroTile) ? 1u : 512u;
-                        enc_len = (ZEROS && entry == 1u) ? 0u : 32u * entry;
+                        entry = Ssum <= 253u ? 258u + Ssum : (ZEROS && Ssum == kSumZeroTile) ? 1u : (ZEROS && Ssum == kSumConstTile) ? 2u : 512u;
+                        enc_len = (ZEROS && entry <= 2u) ? 32u * (entry - 1u) : 32u * entry;
                     }
                 } else {
                     entry = 0xFFFFu;
@@ -1629,6 +1643,7 @@ k_decode_check(const unsigned char* __restrict__ wire, uint64_t wire_len, Geo g,
                         l_any = true;
                         if (tl < kTile) { if (e != 0xFFFFu) l_ok = false; len = (uint32_t)tl; }
                         else if (e == 1u && zero_ok) len = 0;       // a tile of zeros: no payload
+                        else if (e == 2u && zero_ok) len = 32;      // a tile of one value: the value
                         else if (e == 512u || (!expect_ent && e >= 258u && e <= 511u)) len = 32u * e;
                         else if (expect_ent && e >= (0x8000u | 259u) && e <= (0x8000u | 511u)) len = 32u * (e & 0x7FFFu);   // ENT tile
                         else l_ok = false;
@@ -2010,10 +2025,13 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
                 }
 #endif
             }
-        } else if (e == 1u) {
-            // a tile of zeros: nothing was shipped; from here on it goes the way of a raw tile
+        } else if (e == 1u || e == 2u) {
+            // a tile of zeros (nothing was shipped) or of one value (the first two bytes of its 32):
+            // from here on it goes the way of a raw tile
+            uint32_t v = 0;
+            if (e == 2u) v = __ldg(reinterpret_cast<const unsigned short*>(payload + tc->slot[it & 3u].src)) * 0x10001u;
 #pragma unroll
-            for (int i = 0; i < 16; i++) w[i] = 0u;
+            for (int i = 0; i < 16; i++) w[i] = v;
         }
         team_bar(team);                      // stage free; the slots the leader filled last step visible;
                                              // the previous tile's digest parts complete

@@ -321,3 +321,66 @@ def test_zero_tiles_match_the_oracle(layout):
     out, dcrc, rd = g.decode(wire_dev, r.wire_len, dst=old, dst_crc=want_crc)
     assert same_result(rd, want_r) and rd.ok
     assert np.array_equal(out, want_out) and np.array_equal(out, a) and np.array_equal(dcrc, want_dcrc)
+
+
+@pytest.mark.parametrize("layout", ["mixed", "near_misses", "masked"])
+def test_constant_tiles_match_the_oracle(layout):
+    """The zero-tile option also ships a tile of one non-zero value (a mask fill) as entry 2 and
+    32 bytes; tiles that are constant only per warp, per half-word or but for one element are data."""
+    from gpu_util import Gpu, same_result, to_dev
+    from paper_2607_10389_b200 import binding as wm
+    rng = np.random.default_rng(12)
+    chunk = 4 * TILE
+    nt = 14
+    n = nt * TILE + 300
+    a = (rng.normal(size=(n + 1) // 2).astype(np.float32).view(np.uint32) >> 16).astype("<u2").view(np.uint8)[:n].copy()
+    v = a.view("<u2") if n % 2 == 0 else a[:n - 1].view("<u2")
+
+    def fill(t, value):
+        v[t * 8192:(t + 1) * 8192] = value
+
+    fill(1, 0xFF80)                       # -Inf
+    fill(2, 0x3F80)                       # 1.0
+    fill(5, 0x0001)                       # a denormal: exponent 0, not the zero tile
+    fill(6, 0x8000)                       # minus zero: constant, not zero
+    fill(9, 0)                            # zeros: entry 1 as before
+    fill(12, 0x7FC0)                      # NaN
+    if layout == "near_misses":
+        fill(3, 0x3F80); v[3 * 8192 + 8191] = 0x3F81                   # one element off at the very end
+        fill(4, 0x3F80); v[4 * 8192:4 * 8192 + 1024] = 0x3F00         # constant per warp, two values
+        fill(7, 0x4000); v[7 * 8192 + 1::2] = 0x4001                  # the two halves of every word differ
+        fill(8, 0x3F80); v[8 * 8192 + 4096] = 0xBF80                  # one sign flipped
+        fill(10, 0x0000); v[10 * 8192 + 77] = 0x0080                  # zeros but one
+    nc = (n + chunk - 1) // chunk
+    dirty = (np.arange(nc) % 2 == 0).astype(np.uint8) if layout == "masked" else None
+    crc_in = np.full(nc, 0xCAFE, dtype=np.uint32)
+    want_wire, want_crc, want = oracle.encode(a, chunk, dirty=dirty, crc_in=crc_in, zero_tiles=True)
+    tab = want_wire[64 + 16 * nc: 64 + 16 * nc + 2 * (nt + 1)].view("<u2")
+    if layout == "mixed":
+        assert [int(tab[t]) for t in (1, 2, 5, 6, 9, 12)] == [2, 2, 2, 2, 1, 2]
+    if layout == "near_misses":
+        assert all(int(tab[t]) >= 258 for t in (3, 4, 7, 8, 10))
+    g = Gpu(n, chunk)
+    wm.zero_tiles_enable(True)
+    try:
+        wire, crc, r, wire_dev = g.encode(to_dev(a), dirty=dirty, crc_in=crc_in)
+    finally:
+        wm.zero_tiles_enable(False)
+    assert same_result(r, want)
+    assert np.array_equal(wire[: r.wire_len], want_wire) and np.array_equal(crc, want_crc)
+    old = np.full(n, 0x5A, dtype=np.uint8)
+    if dirty is not None:
+        for c in np.nonzero(dirty == 0)[0]:
+            old[c * chunk:(c + 1) * chunk] = a[c * chunk:(c + 1) * chunk]
+    want_out, want_dcrc, want_r = oracle.decode_verify(want_wire, n, chunk, dst=old, dst_crc=want_crc)
+    out, dcrc, rd = g.decode(wire_dev, r.wire_len, dst=old, dst_crc=want_crc)
+    assert same_result(rd, want_r) and rd.ok and np.array_equal(out, a) and np.array_equal(dcrc, want_dcrc)
+    # a damaged value is caught by the chunk checksum; entry 2 without the option's flag is refused
+    bad = want_wire.copy()
+    me = oracle.meta_end(n, chunk)
+    first_const = 32 * int(tab[0])                     # tile 0 is an ordinary packed tile; tile 1's value follows it
+    if dirty is None:
+        bad[me + first_const] ^= 0x40                  # tile 1's value (tile 0 comes first in the payload)
+        want_bad = oracle.decode_verify(bad, n, chunk, dst=old, dst_crc=want_crc)[2]
+        _, _, rb = g.decode(to_dev(bad), bad.size, dst=old, dst_crc=want_crc)
+        assert same_result(rb, want_bad) and want_bad.status_name == "ERR_CHUNK_CRC"
