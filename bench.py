@@ -160,8 +160,18 @@ def cpu_baseline(cur_host, prev_host, chunk_bytes, target_s=10.0):
         list(pool.map(work, range(cores)))
     dtp = time.perf_counter() - t
     total = cores * per_thread * chunk_bytes
+    # courtesy strong baseline for the checksum step alone: the CPU's own CRC32C instruction
+    hw_gbs = None
+    import oracle
+    hw = oracle.hw_crc_library()
+    if hw is not None:
+        nh = min(cur_host.size, 256 * chunk_bytes)
+        t = time.perf_counter()
+        for o in range(0, nh, chunk_bytes):
+            hw.hw_crc32c_u64(cur_host[o:o + chunk_bytes].ctypes.data, min(chunk_bytes, nh - o))
+        hw_gbs = nh / (time.perf_counter() - t) / 1e9
     return {"value": total / dtp / 1e9, "unit": "GB/s", "cores": cores, "kind": "oracle",
-            "single_core_gbs": single,
+            "single_core_gbs": single, "checksum_only_sse42_single_core_gbs": hw_gbs,
             "sample": f"{cores} threads, each one pass of checksum+diff+encode+decode_verify over {per_thread} chunks "
                       f"({per_thread * chunk_bytes} bytes) of the workload's first {n_chunks} chunks, {dtp:.1f} s; "
                       f"single core: {n1} bytes in {dt1:.1f} s"}

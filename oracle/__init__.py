@@ -20,6 +20,7 @@ from .wm_oracle import (  # noqa: F401
     encode,
     encode_leaves,
     flatten_leaves,
+    hw_crc_library,
     meta_end,
     num_chunks,
     num_tiles,

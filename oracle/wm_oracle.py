@@ -109,6 +109,37 @@ def _result(r: _CResult) -> Result:
                   r.payload_bytes, r.cache_crc)
 
 
+_hw = None
+
+
+def hw_crc_library():
+    """The SSE4.2 `crc32` instruction behind two C functions (hw_crc32c: a byte per instruction,
+    hw_crc32c_u64: eight), compiled on first use; None where the host CPU lacks the instruction.
+    A second opinion for the pins and a strong CPU baseline; the oracle itself never uses it."""
+    global _hw
+    if _hw is None:
+        try:
+            has = "sse4_2" in open("/proc/cpuinfo").read()
+        except OSError:
+            has = False
+        if not has:
+            _hw = False
+        else:
+            os.makedirs(_OUT_DIR, exist_ok=True)
+            so = os.path.join(_OUT_DIR, "libhwcrc.so")
+            src = os.path.join(os.path.dirname(_SRC), "hwcrc.c")
+            if not os.path.exists(so) or os.path.getmtime(so) < os.path.getmtime(src):
+                tmp = so + f".{os.getpid()}.tmp"
+                subprocess.check_call(["gcc", "-O2", "-msse4.2", "-shared", "-fPIC", "-o", tmp, src])
+                os.replace(tmp, so)
+            lib = ctypes.CDLL(so)
+            for name in ("hw_crc32c", "hw_crc32c_u64"):
+                getattr(lib, name).restype = ctypes.c_uint32
+                getattr(lib, name).argtypes = [ctypes.c_void_p, ctypes.c_uint64]
+            _hw = lib
+    return _hw or None
+
+
 def crc_bitwise(data, poly: int = POLY_CRC32C) -> int:
     b = _bytes_view(np.frombuffer(data, dtype=np.uint8) if isinstance(data, (bytes, bytearray)) else data)
     return int(_load().wmo_crc_bitwise(_ptr(b), b.size, poly))
