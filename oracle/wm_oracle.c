@@ -256,7 +256,8 @@ static int plane_widths(uint32_t w, uint32_t p[3])
 /* ------------------------------------------------- ENT tiles (option) ---
  * Entropy-coded exponents (the variant of the codec the paper measured codes the exponent
  * plane with an entropy coder; Section 6.4).  An image that sets header flags bit 2 stores a
- * full tile either as an ENT tile or raw; the sign-mantissa plane is the one of a PACK tile.
+ * full tile as an ENT tile, a PACK tile or raw, whichever is shortest; the sign-mantissa plane
+ * of an ENT tile is the one of a PACK tile.
  *
  * A tile is eight shares of 16 rows (row = 128 bytes = 64 elements).  Share s has 32 strands;
  * strand l holds the 32 elements at 32-bit word l of the share's rows, row after row, low half
@@ -278,7 +279,7 @@ static int plane_widths(uint32_t w, uint32_t p[3])
  *
  *   ENT tile:  anchor[8] u8 | count[8] u16 (halfwords in each share's stream) | 40 zero bytes
  *              SM[8192] as in a PACK tile | the eight streams | zero fill to a multiple of 32
- *   entry = 0x8000 | length / 32, used iff the length is below 16384; else the tile is raw.
+ *   entry = 0x8000 | length / 32 (the length is below 16384 whenever the form is used).
  */
 static const int      ent_sym[10]  = {0, 1, -1, -2, 2, -3, -4, -5, 3, -6};
 static const uint32_t ent_len[10]  = {2, 2, 2, 4, 4, 4, 5, 6, 7, 8};
@@ -414,6 +415,7 @@ static int decode_ent_tile(const uint8_t* in, uint8_t* dst)
 
 #define WMO_OPT_ZERO_TILES 1   /* encoder options */
 #define WMO_OPT_ENTROPY 2
+#define WMO_OPT_ENT_ONLY 4
 
 static uint32_t encode_full_tile(const uint8_t* src, uint8_t* out, uint32_t* entry, int options)
 {
@@ -429,13 +431,20 @@ static uint32_t encode_full_tile(const uint8_t* src, uint8_t* out, uint32_t* ent
         for (uint32_t e = 1; e < 8192u; e++) if (get16(src + 2u * e) != v0) { same = 0; break; }
         if (same) { memset(out, 0, 32); put16(out, v0); *entry = 2u; return 32u; }
     }
-    /* option: entropy-coded exponents; the tile is an ENT tile when that is shorter than raw */
+    /* option: entropy-coded exponents.  The tile is stored in the shortest of the three forms
+     * (ENT, PACK, raw); on equal lengths PACK goes before ENT and a coded form before raw, so
+     * an image with the option is never longer than one without.  (WMO_OPT_ENT_ONLY, a switch
+     * of this oracle alone, leaves PACK out: the tests use it to pin the ENT coder by itself.) */
+    static uint8_t ent_buf[2 * WMO_TILE];
+    uint32_t ent_len = WMO_TILE;
     if (options & WMO_OPT_ENTROPY) {
-        uint32_t len = encode_ent_tile(src, out);
-        if (len < WMO_TILE) { *entry = 0x8000u | (len / 32u); return len; }
-        memcpy(out, src, WMO_TILE);
-        *entry = 512u;
-        return WMO_TILE;
+        ent_len = encode_ent_tile(src, ent_buf);
+        if (options & WMO_OPT_ENT_ONLY) {
+            if (ent_len < WMO_TILE) { memcpy(out, ent_buf, ent_len); *entry = 0x8000u | (ent_len / 32u); return ent_len; }
+            memcpy(out, src, WMO_TILE);
+            *entry = 512u;
+            return WMO_TILE;
+        }
     }
     for (uint32_t g = 0; g < WMO_GROUPS_PER_TILE; g++) {
         uint32_t mn = 255, mx = 0;
@@ -448,6 +457,10 @@ static uint32_t encode_full_tile(const uint8_t* src, uint8_t* out, uint32_t* ent
         uint32_t range = mx - mn, bits = 0;
         while (range) { bits++; range >>= 1; }
         base[g] = mn; w[g] = bits; S += bits;
+    }
+    {
+        uint32_t pack_len = S <= 253u ? 8256u + 32u * S : WMO_TILE;
+        if (ent_len < pack_len) { memcpy(out, ent_buf, ent_len); *entry = 0x8000u | (ent_len / 32u); return ent_len; }
     }
     if (S > 253u) {
         memcpy(out, src, WMO_TILE);
@@ -491,7 +504,7 @@ static uint32_t encode_full_tile(const uint8_t* src, uint8_t* out, uint32_t* ent
  *   multiple of 32 (= meta_end) | payload
  *
  *   header:  0 "WMV1"   4 u16 version=1   6 u16 flags (bit0: a dirty mask was given;
- *            bit1: ZERO tile option; bit2: ENT tiles instead of PACK tiles)
+ *            bit1: ZERO tile option; bit2: ENT tiles may occur)
  *            8 u64 nbytes   16 u32 chunk_bytes   20 u32 tile_bytes=16384
  *           24 u32 n_chunks 28 u32 n_present     32 u64 payload_bytes
  *           40 u64 wire_len 48 u32 cache_crc     52 u32 meta_crc   56 8 zero bytes
@@ -512,7 +525,7 @@ static uint32_t encode_full_tile(const uint8_t* src, uint8_t* out, uint32_t* ent
  */
 #define WMO_FLAG_MASKED 1u       /* header flags: a dirty mask was given             */
 #define WMO_FLAG_ZERO_TILES 2u   /* header flags: all-zero tiles are table entries   */
-#define WMO_FLAG_ENTROPY 4u      /* header flags: ENT tiles instead of PACK tiles    */
+#define WMO_FLAG_ENTROPY 4u      /* header flags: ENT tiles may occur                */
 
 int wmo_encode_opt(const uint8_t* cache, uint64_t nbytes, uint32_t chunk_bytes, const uint8_t* dirty,
                    uint32_t* crc_inout, uint8_t* wire, uint64_t wire_cap, int options, wmo_result* res);
@@ -524,7 +537,7 @@ int wmo_encode(const uint8_t* cache, uint64_t nbytes, uint32_t chunk_bytes, cons
 }
 
 /* options: WMO_OPT_ZERO_TILES (tile table entry 1; header flags bit 1), WMO_OPT_ENTROPY (ENT tiles
- * instead of PACK tiles; header flags bit 2). */
+ * where they are shorter than PACK tiles; header flags bit 2). */
 int wmo_encode_opt(const uint8_t* cache, uint64_t nbytes, uint32_t chunk_bytes, const uint8_t* dirty,
                    uint32_t* crc_inout, uint8_t* wire, uint64_t wire_cap, int options, wmo_result* res)
 {
@@ -680,7 +693,7 @@ int wmo_decode_verify_opt(const uint8_t* wire, uint64_t wire_len, uint8_t* dst, 
     }
     uint64_t payload_bytes = get64(wire + 32);
     int zero_ok = (get16(wire + 6) & 2u) != 0;      /* entry 1 is legal only in an image that declares the option */
-    int ent_on = (get16(wire + 6) & 4u) != 0;       /* ENT entries only with the flag, PACK entries only without */
+    int ent_on = (get16(wire + 6) & 4u) != 0;       /* ENT entries only in an image that declares the option */
     uint32_t n_present_hdr = get32(wire + 28);
     uint32_t cache_crc_hdr = get32(wire + 48);
     res->wire_len = wire_len; res->payload_bytes = payload_bytes;
@@ -718,7 +731,7 @@ int wmo_decode_verify_opt(const uint8_t* wire, uint64_t wire_len, uint8_t* dst, 
                 if (tlen < WMO_TILE) { if (e != 0xFFFFu) ok = 0; sum += tlen; }
                 else if (e == 1u && zero_ok) sum += 0;     /* ZERO tile: full tiles only, no payload */
                 else if (e == 2u && zero_ok) sum += 32u;   /* CONST tile: the value in 32 bytes of payload */
-                else if (e == 512u || (!ent_on && e >= 258u && e <= 511u)) sum += 32u * (uint64_t)e;
+                else if (e >= 258u && e <= 512u) sum += 32u * (uint64_t)e;
                 else if (ent_on && e >= (0x8000u | 259u) && e <= (0x8000u | 511u)) sum += 32u * (uint64_t)(e & 0x7FFFu);
                 else ok = 0;
             }

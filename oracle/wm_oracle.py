@@ -204,10 +204,12 @@ def dirty_diff(cache, prev, chunk_bytes: int):
 
 
 def encode(cache, chunk_bytes: int, dirty=None, crc_in=None, wire_cap: int | None = None, zero_tiles: bool = False,
-           entropy: bool = False):
+           entropy: bool = False, ent_only: bool = False):
     """Return (wire u8[wire_len or wire_cap], crc u32[n_chunks], Result).  ``zero_tiles``: the
     option that ships a full tile of all-zero bytes as a table entry without payload.
-    ``entropy``: the option that codes the exponents with the fixed prefix code (ENT tiles)."""
+    ``entropy``: the option that codes the exponents with the fixed prefix code (ENT tiles) where
+    that is shorter than the bit planes.  ``ent_only`` (this oracle alone, for pinning the ENT coder):
+    with ``entropy``, never choose a PACK tile."""
     b = _bytes_view(cache)
     nc = num_chunks(b.size, chunk_bytes)
     cap = wire_bound(b.size, chunk_bytes) if wire_cap is None else int(wire_cap)
@@ -216,7 +218,7 @@ def encode(cache, chunk_bytes: int, dirty=None, crc_in=None, wire_cap: int | Non
     d = None if dirty is None else np.ascontiguousarray(dirty, dtype=np.uint8)
     res = _CResult()
     st = _load().wmo_encode_opt(_ptr(b), b.size, chunk_bytes, None if d is None else _ptr(d), _ptr(crc),
-                                _ptr(wire), cap, (1 if zero_tiles else 0) | (2 if entropy else 0), ctypes.byref(res))
+                                _ptr(wire), cap, (1 if zero_tiles else 0) | (2 if entropy else 0) | (4 if ent_only else 0), ctypes.byref(res))
     _check(st, "encode")
     r = _result(res)
     if r.status == 0:

@@ -23,7 +23,8 @@ def _tile_of(value_u16):
 
 
 def _encode_one_tile(v):
-    wire, crc, res = oracle.encode(v.view(np.uint8), TILE, entropy=True)
+    # (ent_only: these hand-built tiles are so regular that the bit planes would win the choice)
+    wire, crc, res = oracle.encode(v.view(np.uint8), TILE, entropy=True, ent_only=True)
     assert res.status == 0 and oracle.meta_end(TILE, TILE) == META1
     flags = struct.unpack_from("<H", wire, 6)[0]
     entry = struct.unpack_from("<H", wire, 64 + 16)[0]
@@ -117,8 +118,18 @@ def test_sizes_follow_the_code_lengths_and_respect_shannon():
         L[u == k] = len(w)
     halfwords = -(-L.sum(axis=3) // 16)
     want_len = (8256 + 2 * halfwords.sum(axis=(1, 2)) + 31) // 32 * 32
-    assert np.array_equal(entries.astype(np.int64), np.where(want_len < TILE, 0x8000 | (want_len // 32), 512))
-    assert res.wire_len == me + int(np.minimum(want_len, TILE).sum())
+    # the bit-plane form of the same tiles: 32 groups of 256 elements in memory order
+    G = ((v >> 7) & 0xFF).astype(np.int64).reshape(n_tiles, 32, 256)
+    rng_ = G.max(axis=2) - G.min(axis=2)
+    S = np.where(rng_ > 0, np.floor(np.log2(np.maximum(rng_, 1))).astype(np.int64) + 1, 0).sum(axis=1)
+    pack_len = np.where(S <= 253, 8256 + 32 * S, TILE)
+    best = np.minimum(np.minimum(want_len, pack_len), TILE)
+    want_entry = np.where(want_len < pack_len, 0x8000 | (want_len // 32), np.where(S <= 253, 258 + S, 512))
+    assert np.array_equal(entries.astype(np.int64), want_entry)
+    assert res.wire_len == me + int(best.sum())
+    assert (entries & 0x8000).any()                           # the Gaussian tiles do take the ENT form
+    only, _, res_only = oracle.encode(v.view(np.uint8), 2 * TILE, entropy=True, ent_only=True)
+    assert res_only.wire_len == me + int(np.minimum(want_len, TILE).sum())
     # no uniquely decodable code beats the empirical entropy of what it codes
     for t in range(n_tiles):
         for s in range(8):
@@ -204,14 +215,16 @@ def test_damaged_ent_tiles_are_refused_with_the_right_status():
         w[me + 8256 + k] ^= 1 << (k % 8)
         seen.add(oracle.decode_verify(w, n, chunk)[2].status_name)
     assert seen <= {"ERR_DESC", "ERR_CHUNK_CRC"} and "ERR_CHUNK_CRC" in seen
-    # an ENT entry in an image that does not declare the option, and a PACK entry in one that does
+    # an ENT entry in an image that does not declare the option
     w = wire.copy()
     w[6] = 0
     assert oracle.decode_verify(_reseal(w, n, chunk), n, chunk)[2].status_name == "ERR_STRUCT"
+    # a PACK tile is at home in an image that declares the option (the encoder picks the shorter form)
     wp, _, _ = oracle.encode(a, chunk)
     wp = wp.copy()
     wp[6] = 4
-    assert oracle.decode_verify(_reseal(wp, n, chunk), n, chunk)[2].status_name == "ERR_STRUCT"
+    out_p, _, r_p = oracle.decode_verify(_reseal(wp, n, chunk), n, chunk)
+    assert r_p.status == 0 and np.array_equal(out_p, a)
     # flags above 7 are no format this decoder knows
     w = wire.copy()
     w[6] = 12
@@ -247,3 +260,32 @@ def test_every_codeword_bit_by_bit():
     assert not others.any()
     out, _, r = oracle.decode_verify(wire, TILE, TILE)
     assert r.status == 0 and np.array_equal(out.view("<u2"), v)
+
+
+def test_the_option_never_makes_an_image_longer():
+    """Per tile the shortest of ENT, PACK and raw is stored (PACK on a tie): regular data, where
+    the bit planes cost next to nothing, keeps its PACK tiles; an image with the option is never
+    longer than one without."""
+    const = _tile_of(0x3F80)                                              # one exponent: PACK at 8256 bytes
+    narrow = ((np.arange(8192) % 2 + 126) << 7).astype("<u2")             # two exponents everywhere: width 1
+    gauss = _gauss(8192, 77)
+    noise = np.random.default_rng(5).integers(0, 65536, 8192).astype("<u2")
+    v = np.concatenate([const, narrow, gauss, noise])
+    w_opt, _, r_opt = oracle.encode(v.view(np.uint8), 4 * TILE, entropy=True)
+    w_def, _, r_def = oracle.encode(v.view(np.uint8), 4 * TILE)
+    e_opt = w_opt[64 + 16: 64 + 16 + 8].view("<u2")
+    e_def = w_def[64 + 16: 64 + 16 + 8].view("<u2")
+    assert list(e_opt[:2]) == list(e_def[:2]) == [258, 258 + 32]          # PACK kept
+    assert e_opt[2] & 0x8000 and 258 <= e_def[2] < 512                    # ENT wins on the Gaussian tile
+    assert e_opt[3] == e_def[3] == 512                                    # noise stays raw
+    assert r_opt.wire_len < r_def.wire_len
+    out, _, r = oracle.decode_verify(w_opt, v.size * 2, 4 * TILE)
+    assert r.status == 0 and np.array_equal(out, v.view(np.uint8))
+    for seed in range(6):
+        x = _gauss(8192 * 3, 100 + seed, float(2.0 ** (seed - 3)))
+        x[:8192] = (x[:8192] & 0x807F) | (120 << 7)                        # a tile with one exponent
+        a_, _, ra = oracle.encode(x.view(np.uint8), TILE, entropy=True)
+        b_, _, rb = oracle.encode(x.view(np.uint8), TILE)
+        ea, eb = a_[64 + 48: 64 + 48 + 6].view("<u2"), b_[64 + 48: 64 + 48 + 6].view("<u2")
+        la = np.where(ea & 0x8000, 32 * (ea & 0x7FFF).astype(np.int64), 32 * ea.astype(np.int64))
+        assert (la <= 32 * eb.astype(np.int64)).all() and ra.wire_len <= rb.wire_len
