@@ -68,7 +68,8 @@ struct Ctrl {                 // first 256 bytes of the workspace
     unsigned long long payload_total;
     uint32_t hdr_n_present, hdr_cache_crc;
     uint32_t cache_acc;       // XOR of the chunks' terms of the whole-cache CRC
-    uint32_t pad[41];
+    uint32_t has_pack;        // decode of an image with the entropy option: it holds PACK tiles too
+    uint32_t pad[40];
 };
 static_assert(sizeof(Ctrl) == 256, "control block is 256 bytes");
 
@@ -769,7 +770,9 @@ struct EncTeamCtl {
                             // long after its last read)
     uint32_t wdig[8][8];    // per warp: its contribution to the tile digest
     uint32_t wsum[8];       // sum of widths so far | warps arrived << 16 (the last warp publishes)
-    uint32_t ssum[8];       // sum of the 32 widths of the slot's tile (set by that last warp)
+    uint32_t ssum[8];       // sum of the 32 widths of the slot's tile (set by that last warp), or a mark:
+                            // zero tile, constant tile, kSumEnt | halfwords for a tile stored in ENT form
+    uint32_t etab[8][8];    // entropy option, per warp: anchor | halfwords of its stream << 8
     uint32_t next[2];       // ticket claimed in this step (>= n_tiles: none left), by step parity
     uint32_t pad[2];
     unsigned long long excl[2];   // offset of the tile packed in the next step, by step parity
@@ -930,6 +933,8 @@ constexpr uint32_t kQPresent = 1u << 31, kQFirst = 1u << 30, kQTile = (1u << 30)
 // kWarpConst: all 1024 elements of the warp's rows hold one value (its sign-mantissa byte rides in
 // bits 16-23 of the entry, the exponent is the base); kSumConstTile: the tile holds one value.
 constexpr uint32_t kWarpAllZero = 0x8000u, kWarpConst = 0x4000u, kSumZeroTile = 0xFFFFu, kSumConstTile = 0xFFFEu;
+// The tile is stored in ENT form (shorter than its bit planes and than raw); low half: halfwords.
+constexpr uint32_t kSumEnt = 0x10000u;
 
 template <bool MASKED>
 __device__ __forceinline__ uint32_t describe_tile(const Geo& g, const uint8_t* __restrict__ dirty, uint32_t t)
@@ -1086,6 +1091,7 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
 #pragma unroll
             for (int i = 0; i < 16; i++) d[i] = __funnelshift_l(d[i], d[i], 1);
             uint32_t gw[4];               // per group: base | width << 8
+            uint32_t ent_w = 0;           // entropy option: anchor | halfwords << 8 of this warp's share
             if (ENT) {
                 // the share's anchor (rounded mean of its 1024 exponents: bytes 1 and 3 of a rotated
                 // word) and the halfwords its 32 strands need
@@ -1098,9 +1104,9 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
                 for (int i = 0; i < 16; i++)
                     bits += s_len[ent_slot(__byte_perm(d[i], 0u, 0x4441), anchor)] + s_len[ent_slot(d[i] >> 24, anchor)];
                 const uint32_t count = __reduce_add_sync(0xFFFFFFFFu, (bits + 15u) >> 4);
-                gw[0] = anchor | (count << 8);
-                gw[1] = gw[2] = gw[3] = 0u;
-            } else {
+                ent_w = anchor | (count << 8);
+            }
+            {
 #ifdef WM_AB_NOMINMAX
             gw[0] = gw[1] = gw[2] = gw[3] = 100u | (4u << 8);
 #else
@@ -1137,6 +1143,7 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
             if (lane == 0) {
                 tc->wdig[slY][warp] = v;
                 *reinterpret_cast<uint4*>(&tc->wtab[slY][4 * warp]) = make_uint4(gw[0], gw[1], gw[2], gw[3]);
+                if (ENT) tc->etab[slY][warp] = ent_w;
                 __threadfence_block();
                 last = (atomicAdd(&tc->wsum[slY], 1u) == 7u) ? 1u : 0u;
             }
@@ -1145,8 +1152,12 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
                 // (kept short: this warp is the one the team's length waits for; the groups'
                 // places inside the tile are worked out by each warp when it packs)
                 const uint32_t wt = *reinterpret_cast<volatile uint32_t*>(&tc->wtab[slY][lane]);
-                // (ENT: every warp's first entry carries its stream's halfwords, the other three are zero)
-                const uint32_t total = __reduce_add_sync(0xFFFFFFFFu, ENT ? wt >> 8 : (wt >> 8) & 15u);
+                const uint32_t total = __reduce_add_sync(0xFFFFFFFFu, (wt >> 8) & 15u);
+                // entropy option: the ENT form is taken when it is shorter than the planes and than raw
+                uint32_t halfwords = 0;
+                if (ENT) halfwords = __reduce_add_sync(0xFFFFFFFFu, lane < 8u ? *reinterpret_cast<volatile uint32_t*>(&tc->etab[slY][lane]) >> 8 : 0u);
+                const uint32_t plane_len = total <= 253u ? 8256u + 32u * total : kTile;
+                const bool ent_tile = ENT && ent_tile_bytes(halfwords) < plane_len;
                 // unused memory (every warp's first entry carries the mark): no payload
                 // (one value throughout: every warp's first entry carries the mark and they are all alike;
                 // a tile of zeros has no payload, any other value 32 bytes)
@@ -1154,10 +1165,9 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
                 const bool const_tile = ZEROS && __all_sync(0xFFFFFFFFu, (lane & 3u) != 0u || ((wt & kWarpConst) != 0u && wt == wt0));
                 const bool zero_tile = const_tile && (wt0 & kWarpAllZero) != 0u;
                 if (lane == 0) {
-                    tc->ssum[slY] = zero_tile ? kSumZeroTile : const_tile ? kSumConstTile : total;
+                    tc->ssum[slY] = zero_tile ? kSumZeroTile : const_tile ? kSumConstTile : ent_tile ? kSumEnt | halfwords : total;
                     tc->wsum[slY] = 0;
-                    if (ENT) publish_len(tYn, ent_tile_bytes(total) < kTile ? ent_tile_bytes(total) : kTile);
-                    else publish_len(tYn, zero_tile ? 0u : const_tile ? 32u : total <= 253u ? 8256u + 32u * total : kTile);
+                    publish_len(tYn, zero_tile ? 0u : const_tile ? 32u : ent_tile ? ent_tile_bytes(halfwords) : plane_len);
                 }
             }
 #ifndef WM_AB_NOTMEM
@@ -1180,20 +1190,22 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
 #ifndef WM_AB_NOTMEM
             tmem_load16(tmem_warp + 16u * ((step + 1u) & 3u), d);
 #endif
-            const uint32_t Ssum = tc->ssum[sl];
-            const bool packs = ENT ? ent_tile_bytes(Ssum) < kTile : Ssum <= 253u;
+            const uint32_t Smark = tc->ssum[sl];
+            const bool ent_form = ENT && (Smark & kSumEnt) != 0u;
+            const uint32_t Ssum = ent_form ? Smark & 0xFFFFu : Smark;       // halfwords, or the sum of the widths
+            const bool packs = !ent_form && Ssum <= 253u;
             // (a tile of all-zero bytes, marked in ssum, is its table entry and nothing else)
-            const uint32_t enc_len = ENT ? (packs ? ent_tile_bytes(Ssum) : kTile)
+            const uint32_t enc_len = ent_form ? ent_tile_bytes(Ssum)
                                          : packs ? 8256u + 32u * Ssum : (ZEROS && Ssum == kSumZeroTile) ? 0u
                                          : (ZEROS && Ssum == kSumConstTile) ? 32u : kTile;
             unsigned char* const dst = payload + exclX;
             if (exclX + enc_len > room) {
                 trouble |= 1u;
-            } else if (ENT && packs) {
+            } else if (ent_form) {
                 // header: anchors, stream lengths, 40 zero bytes; zero fill behind the last stream
                 if (warp == 5) {
                     if (lane < 8u) {
-                        const uint32_t wt = tc->wtab[sl][4u * lane];
+                        const uint32_t wt = tc->etab[sl][lane];
                         stg_u8(dst + lane, wt & 0xFFu);
                         stg_u16(dst + 8u + 2u * lane, wt >> 8);
                     } else if (lane < 18u) {
@@ -1209,9 +1221,8 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
                     stg_v2(sm_dst + 256 * j, (sa & 0xFEFEFEFEu) | (ya & 0x01010101u), (sb & 0xFEFEFEFEu) | (yb & 0x01010101u));
                 }
                 // this share's stream: it starts behind the streams of the warps before it
-                const uint32_t wall = tc->wtab[sl][lane] >> 8;
-                const uint32_t before = __reduce_add_sync(0xFFFFFFFFu, lane < 4u * warp ? wall : 0u);
-                const uint32_t anchor = tc->wtab[sl][4u * warp] & 0xFFu;
+                const uint32_t before = __reduce_add_sync(0xFFFFFFFFu, lane < warp ? tc->etab[sl][lane] >> 8 : 0u);
+                const uint32_t anchor = tc->etab[sl][warp] & 0xFFu;
                 unsigned char* const hw_dst = dst + 8256u + 2u * before;
                 const uint32_t lt_mask = (1u << lane) - 1u;
                 // acc: the strand's bits from the start of the halfword it took last (number `pend` of
@@ -1305,10 +1316,9 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
             if (qX >= kQPresent) {
                 if (tXn < g.n_full_tiles) {
                     const uint32_t Ssum = tc->ssum[sl];
-                    if (ENT) {
-                        const uint32_t nb = ent_tile_bytes(Ssum);
-                        entry = nb < kTile ? 0x8000u | (nb / 32u) : 512u;
-                        enc_len = nb < kTile ? nb : kTile;
+                    if (ENT && (Ssum & kSumEnt)) {
+                        enc_len = ent_tile_bytes(Ssum & 0xFFFFu);
+                        entry = 0x8000u | (enc_len / 32u);
                     } else {
                         entry = Ssum <= 253u ? 258u + Ssum : (ZEROS && Ssum == kSumZeroTile) ? 1u : (ZEROS && Ssum == kSumConstTile) ? 2u : 512u;
                         enc_len = (ZEROS && entry <= 2u) ? 32u * (entry - 1u) : 32u * entry;
@@ -1634,7 +1644,7 @@ k_decode_check(const unsigned char* __restrict__ wire, uint64_t wire_len, Geo g,
             for (uint32_t i0 = 0; i0 < ntc; i0 += 32) {
                 const uint32_t i = i0 + lane;
                 uint32_t len = 0;
-                bool l_ok = true, l_any = false, l_all = true;
+                bool l_ok = true, l_any = false, l_all = true, l_packs = false;
                 if (i < ntc) {
                     const uint32_t e = tab16[t0 + i];
                     const uint64_t tl = clen - (uint64_t)i * kTile;
@@ -1644,7 +1654,7 @@ k_decode_check(const unsigned char* __restrict__ wire, uint64_t wire_len, Geo g,
                         if (tl < kTile) { if (e != 0xFFFFu) l_ok = false; len = (uint32_t)tl; }
                         else if (e == 1u && zero_ok) len = 0;       // a tile of zeros: no payload
                         else if (e == 2u && zero_ok) len = 32;      // a tile of one value: the value
-                        else if (e == 512u || (!expect_ent && e >= 258u && e <= 511u)) len = 32u * e;
+                        else if (e >= 258u && e <= 512u) { len = 32u * e; l_packs = e < 512u; }
                         else if (expect_ent && e >= (0x8000u | 259u) && e <= (0x8000u | 511u)) len = 32u * (e & 0x7FFFu);   // ENT tile
                         else l_ok = false;
                     }
@@ -1657,6 +1667,7 @@ k_decode_check(const unsigned char* __restrict__ wire, uint64_t wire_len, Geo g,
                 }
                 if (i < ntc) ws.rel[t0 + i] = (uint32_t)(carry + incl - len);
                 carry += __shfl_sync(0xFFFFFFFFu, incl, 31);
+                if (expect_ent && __any_sync(0xFFFFFFFFu, l_packs) && lane == 0) atomicOr(&ws.ctrl->has_pack, 1u);
                 ok = ok && __all_sync(0xFFFFFFFFu, l_ok);
                 any = any || __any_sync(0xFFFFFFFFu, l_any);
                 all = all && __all_sync(0xFFFFFFFFu, l_all);
@@ -1836,10 +1847,12 @@ __device__ __forceinline__ void unpack_group_planes(const PlaneWords& pw, uint32
 // the pace of its slowest one.)  LEAVES: the decoded tiles go to a table of tensors.
 // MODE 0: unpack, store, checksum (the normal call).  Strict calls run the kernel twice: MODE 1
 // unpacks and checksums without storing anything; MODE 2, after the verdict, unpacks and stores.
-// ENT: the image holds ENT tiles instead of PACK tiles; a warp reads its share's stream of
-// halfwords in phase 1 (the need test, the ballot and the fetch of every step) and leaves the
-// exponent bytes where the plane words would be.
-template <int TEAMS, bool LEAVES, int MODE, bool ENT = false>
+// ENT 1 / 2: the image was written with the entropy option and holds ENT tiles only (1) or ENT
+// and PACK tiles (2; the check kernel noted which).  A call launches both, and the one that does
+// not apply returns at once: the kernel with a single kind of coded tile is the faster one.  A
+// warp reads its share's stream of halfwords in phase 1 (the need test, the ballot and the fetch
+// of every step) and leaves the exponent bytes where the plane words would be.
+template <int TEAMS, bool LEAVES, int MODE, int ENT = 0>
 __global__ void __launch_bounds__(TEAMS * 256, 1)
 k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restrict__ dst, Ws ws,
          const Tables* __restrict__ tab)
@@ -1849,7 +1862,7 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
     // escape) and u as a byte.  Two byte tables: the index needs no scaling and a look-up gives a
     // clean value.
     __shared__ unsigned char s_plen[ENT ? 256 : 4], s_pu[ENT ? 256 : 4];
-    if (ENT && threadIdx.x < 256u) {
+    if (ENT != 0 && threadIdx.x < 256u) {
         const uint32_t s = ent_ones(threadIdx.x);
         s_plen[threadIdx.x] = (unsigned char)ent_parse_length(s);
         s_pu[threadIdx.x] = (unsigned char)(s == 8u ? 0u : ent_parse_value(threadIdx.x, s, 0u));
@@ -1858,6 +1871,7 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
     grid_dep_wait();
     grid_dep_launch();
     if (ld_volatile_u32(&ws.ctrl->gate)) return;
+    if (ENT != 0 && (ENT == 1) == (ld_volatile_u32(&ws.ctrl->has_pack) != 0u)) return;      // the other kernel's image
     const uint32_t team = threadIdx.x / kTeamThreads, tt = threadIdx.x % kTeamThreads;
     const uint32_t warp = tt / 32, lane = tt % 32;
     unsigned char* stage = nullptr;
@@ -1887,8 +1901,10 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
         }
     };
     // staged tiles: full RAW and PACK tiles (everything except absent tiles and the ragged tail)
-    // (ENT images: raw tiles and ENT tiles, entry 0x8000 | length / 32)
-    auto is_staged = [](uint32_t e) { return ENT ? (e == 512u || (e > 0x8000u && e != 0xFFFFu)) : (e >= 258u && e <= 512u); };
+    // (images with the entropy option hold ENT tiles too: entry 0x8000 | length / 32)
+    auto is_ent_entry = [](uint32_t e) { return ENT != 0 && e > 0x8000u && e != 0xFFFFu; };
+    auto is_pack_entry = [](uint32_t e) { return ENT != 1 && e >= 258u && e < 512u; };
+    auto is_staged = [&](uint32_t e) { return e == 512u || is_pack_entry(e) || is_ent_entry(e); };
     auto start_copy = [&](const DecSlot& sl) {   // leader only
         const uint32_t e = sl.entry & 0xFFFFu;
         if (sl.t < g.n_tiles && is_staged(e)) bulk_load(stage, payload + sl.src, 32u * (e & 0x7FFFu), &tc->mbar, 0);
@@ -1917,7 +1933,8 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
         // leaf mode: where this tile goes (asked for now, needed when the stores begin)
         unsigned char* const o_leaf = LEAVES ? ws.tptr[t] : nullptr;
         const uint32_t p = it & 1u;
-        const bool is_pack = ENT ? (e > 0x8000u && e != 0xFFFFu) : (e >= 258u && e < 512u);     // a coded tile
+        const bool is_ent = is_ent_entry(e);
+        const bool is_pack = is_ent || is_pack_entry(e);            // a coded tile (in either form)
         bool decoded = true;
         uint32_t w[kWordsPerLane];
         uint32_t desc = 0;
@@ -1930,7 +1947,7 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
             phase ^= 1u;
             if (!is_pack) {
                 read_staged_words(stage, warp, lane, w);
-            } else if (ENT) {
+            } else if (is_ent) {
                 // ENT tile.  Header: the eight stream lengths against the entry (structure); then this
                 // warp reads its share's stream the way the format interleaves it: at step i every
                 // strand whose codeword i is not complete in the bits it holds takes the stream's next
@@ -1984,7 +2001,7 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
                         atomicOr(&ws.cflag[chunk_of(g, t)], CF_BAD4);
                     }
                 }
-            } else {
+            } else if (ENT != 1) {
 #ifdef WM_AB_D_NOP1
                 desc = 100u | (4u << 8);
                 for (int j = 0; j < 4; j++) { sm[j] = make_uint2(lane, it); pw[j].a = t; pw[j].b = e; }
@@ -2077,7 +2094,7 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
                     const uint32_t dg = __shfl_sync(0xFFFFFFFFu, desc, j);
                     const uint32_t base = dg & 0xFFu, wd = (dg >> 8) & 15u;
                     uint32_t ea = base * 0x01010101u, eb = ea;
-                    if (ENT) { ea = pw[j].a; eb = pw[j].b; }       // the exponent bytes are already there
+                    if (ENT == 1 || (ENT == 2 && is_ent)) { ea = pw[j].a; eb = pw[j].b; }     // the exponent bytes are already there
                     else if (wd == 4u) unpack_group_planes<4>(pw[j], base, ea, eb);       // by far the most frequent width
                     else switch (wd) {     // uniform across the warp
                         case 1: unpack_group_planes<1>(pw[j], base, ea, eb); break;
@@ -2275,7 +2292,9 @@ static const DeviceState* device_state()
                              (const void*)k_encode<kTeams, false, false, true>,  (const void*)k_encode<kTeams, true, false, true>,
                              (const void*)k_encode<kTeams, false, true, true>,   (const void*)k_encode<kTeams, true, true, true>,
                              (const void*)k_encode<kTeams, false, false, false, true>, (const void*)k_encode<kTeams, true, false, false, true>,
-                             (const void*)k_encode<kTeams, false, true, false, true>,  (const void*)k_encode<kTeams, true, true, false, true>};
+                             (const void*)k_encode<kTeams, false, true, false, true>,  (const void*)k_encode<kTeams, true, true, false, true>,
+                             (const void*)k_encode<kTeams, false, false, true, true>,  (const void*)k_encode<kTeams, true, false, true, true>,
+                             (const void*)k_encode<kTeams, false, true, true, true>,   (const void*)k_encode<kTeams, true, true, true, true>};
         for (const void* f : enc)
             if (cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, big) != cudaSuccess) return nullptr;
     }
@@ -2283,9 +2302,12 @@ static const DeviceState* device_state()
         const void* dec[] = {(const void*)k_decode<kTeamsPlain, false, 0>, (const void*)k_decode<kTeamsPlain, true, 0>,
                              (const void*)k_decode<kTeamsPlain, false, 1>, (const void*)k_decode<kTeamsPlain, true, 1>,
                              (const void*)k_decode<kTeamsPlain, false, 2>, (const void*)k_decode<kTeamsPlain, true, 2>,
-                             (const void*)k_decode<kTeamsPlain, false, 0, true>, (const void*)k_decode<kTeamsPlain, true, 0, true>,
-                             (const void*)k_decode<kTeamsPlain, false, 1, true>, (const void*)k_decode<kTeamsPlain, true, 1, true>,
-                             (const void*)k_decode<kTeamsPlain, false, 2, true>, (const void*)k_decode<kTeamsPlain, true, 2, true>};
+                             (const void*)k_decode<kTeamsPlain, false, 0, 1>, (const void*)k_decode<kTeamsPlain, true, 0, 1>,
+                             (const void*)k_decode<kTeamsPlain, false, 1, 1>, (const void*)k_decode<kTeamsPlain, true, 1, 1>,
+                             (const void*)k_decode<kTeamsPlain, false, 2, 1>, (const void*)k_decode<kTeamsPlain, true, 2, 1>,
+                             (const void*)k_decode<kTeamsPlain, false, 0, 2>, (const void*)k_decode<kTeamsPlain, true, 0, 2>,
+                             (const void*)k_decode<kTeamsPlain, false, 1, 2>, (const void*)k_decode<kTeamsPlain, true, 1, 2>,
+                             (const void*)k_decode<kTeamsPlain, false, 2, 2>, (const void*)k_decode<kTeamsPlain, true, 2, 2>};
         for (const void* f : dec)
             if (cudaFuncSetAttribute(f, cudaFuncAttributeMaxDynamicSharedMemorySize, big) != cudaSuccess) return nullptr;
     }
@@ -2563,8 +2585,7 @@ static wm_status encode_any(const void* cache, const wm_leaf* leaves, uint32_t n
     const uint32_t grid = need < (uint32_t)ds->sm_count ? need : (uint32_t)ds->sm_count;
     {
         MainKernelTimer timer(ds, 2, s);
-        // the entropy option takes precedence over the zero-tile option
-        const int variant = (dirty ? 1 : 0) | (leaves ? 2 : 0) | (opt_ent ? 8 : opt_zero ? 4 : 0);
+        const int variant = (dirty ? 1 : 0) | (leaves ? 2 : 0) | (opt_zero ? 4 : 0) | (opt_ent ? 8 : 0);
         auto go = [&](auto kernel) { launch_after(kernel, grid, kTeams * 256, kDynSmem, s, c, g, dirty, w, wire_cap, ws, ds->tables); };
         switch (variant) {
             case 0: go(k_encode<kTeams, false, false, false>); break;
@@ -2578,11 +2599,15 @@ static wm_status encode_any(const void* cache, const wm_leaf* leaves, uint32_t n
             case 8: go(k_encode<kTeams, false, false, false, true>); break;
             case 9: go(k_encode<kTeams, true, false, false, true>); break;
             case 10: go(k_encode<kTeams, false, true, false, true>); break;
-            default: go(k_encode<kTeams, true, true, false, true>); break;
+            case 11: go(k_encode<kTeams, true, true, false, true>); break;
+            case 12: go(k_encode<kTeams, false, false, true, true>); break;
+            case 13: go(k_encode<kTeams, true, false, true, true>); break;
+            case 14: go(k_encode<kTeams, false, true, true, true>); break;
+            default: go(k_encode<kTeams, true, true, true, true>); break;
         }
     }
     launch_after(k_encode_finish, (g.n_chunks + g.finish_cb - 1) / g.finish_cb, 1024, 0, s, c, g, dirty, crc_inout, w, ws, ds->tables,
-                 chunk_powers(g), opt_ent ? 4u : opt_zero ? 2u : 0u);
+                 chunk_powers(g), (opt_ent ? 4u : 0u) | (opt_zero ? 2u : 0u));
     launch_after(k_meta_crc, (g.n_meta_slices + 3) / 4, 1024, kDynSmem, s, w, g, ws, ds->tables, result);
     g_launches = leaves ? 5 : 4;
     return launch_status();
@@ -2643,9 +2668,9 @@ static wm_status decode_any(const void* wire, uint64_t wire_len, void* dst, cons
     };
     {
         MainKernelTimer timer(ds, 3, s);
-        if (ent) {
-            if (strict) pass(k_decode<kTeamsPlain, false, 1, true>, k_decode<kTeamsPlain, true, 1, true>);
-            else pass(k_decode<kTeamsPlain, false, 0, true>, k_decode<kTeamsPlain, true, 0, true>);
+        if (ent) {       // one of the two applies (ENT tiles only, or ENT and PACK tiles); the other returns at once
+            if (strict) { pass(k_decode<kTeamsPlain, false, 1, 1>, k_decode<kTeamsPlain, true, 1, 1>); pass(k_decode<kTeamsPlain, false, 1, 2>, k_decode<kTeamsPlain, true, 1, 2>); }
+            else { pass(k_decode<kTeamsPlain, false, 0, 1>, k_decode<kTeamsPlain, true, 0, 1>); pass(k_decode<kTeamsPlain, false, 0, 2>, k_decode<kTeamsPlain, true, 0, 2>); }
         } else {
             if (strict) pass(k_decode<kTeamsPlain, false, 1>, k_decode<kTeamsPlain, true, 1>);
             else pass(k_decode<kTeamsPlain, false, 0>, k_decode<kTeamsPlain, true, 0>);
@@ -2654,10 +2679,10 @@ static wm_status decode_any(const void* wire, uint64_t wire_len, void* dst, cons
     launch_after(k_decode_finish, (g.n_chunks + g.finish_cb - 1) / g.finish_cb, 1024, 0, s, w, wire_len, g, d, dst_crc_inout, ws, ds->tables,
                  result, chunk_powers(g), strict ? 1u : 0u);
     if (strict) {
-        if (ent) pass(k_decode<kTeamsPlain, false, 2, true>, k_decode<kTeamsPlain, true, 2, true>);
+        if (ent) { pass(k_decode<kTeamsPlain, false, 2, 1>, k_decode<kTeamsPlain, true, 2, 1>); pass(k_decode<kTeamsPlain, false, 2, 2>, k_decode<kTeamsPlain, true, 2, 2>); }
         else pass(k_decode<kTeamsPlain, false, 2>, k_decode<kTeamsPlain, true, 2>);
     }
-    g_launches = (leaves ? 5 : 4) + (strict ? 1 : 0);
+    g_launches = (leaves ? 5 : 4) + (strict ? 1 : 0) + (ent ? (strict ? 2 : 1) : 0);
     return launch_status();
 }
 

@@ -197,24 +197,57 @@ def test_ent_leaves(wm):
     assert wm.read_result(res).status == 0 and all(torch.equal(x, y) for x, y in zip(leaves, dst))
 
 
-def test_gpu_reads_images_that_combine_both_options(wm):
-    """The GPU encoder ignores the zero-tile option while the entropy option is on, but the format
-    allows both in one image (the oracle writes it) and the GPU decoder reads it."""
+def test_both_options_in_one_image(wm):
+    """Zero and constant tiles as table entries, the rest in the shortest of ENT, PACK and raw."""
     n, chunk = 10 * TILE, 2 * TILE
     a = _mixed_cache(n, 23)
     a[6 * TILE:8 * TILE] = 0
+    a[8 * TILE:9 * TILE].view("<u2")[:] = 0xFF80
     w, crc, res = oracle.encode(a, chunk, zero_tiles=True, entropy=True)
     assert struct.unpack_from("<H", w, 6)[0] == 6
+    entries = w[64 + 16 * 5: 64 + 16 * 5 + 20].view("<u2")
+    assert list(entries[6:9]) == [1, 1, 2] and entries[0] & 0x8000 and entries[1] == 512
     out, dcrc, r = _run_decode(wm, w, n, chunk)
     assert r.status == 0 and np.array_equal(out, a) and np.array_equal(dcrc, crc)
-    # the GPU encoder with both switches on writes the entropy image without zero entries
     wm.zero_tiles_enable(True)
     try:
         wire, crc2, r2, _ = _run_encode(wm, a, chunk)
     finally:
         wm.zero_tiles_enable(False)
-    want, _, _ = oracle.encode(a, chunk, entropy=True)
-    assert r2.status == 0 and np.array_equal(wire[: r2.wire_len].cpu().numpy(), want)
+    assert r2.status == 0 and np.array_equal(wire[: r2.wire_len].cpu().numpy(), w) and np.array_equal(crc2, crc)
+
+
+def test_regular_tiles_keep_their_bit_planes(wm):
+    """The option never lengthens an image: tiles whose bit planes are shorter than their ENT form
+    (one exponent, two exponents, narrow ranges) stay PACK tiles inside an image with the option."""
+    rng = np.random.default_rng(8)
+    tiles = [np.full(8192, 0x3F80, dtype="<u2"),
+             ((np.arange(8192) % 2 + 126) << 7).astype("<u2"),
+             _gauss(8192, 51),
+             ((rng.integers(100, 104, 8192) << 7) | rng.integers(0, 128, 8192)).astype("<u2"),
+             rng.integers(0, 65536, 8192).astype("<u2"),
+             _gauss(8192, 52, 1e-3)]
+    a = np.concatenate(tiles).view(np.uint8)
+    n, chunk = a.size, 2 * TILE
+    want, want_crc, want_res = oracle.encode(a, chunk, entropy=True)
+    plain, _, plain_res = oracle.encode(a, chunk)
+    entries = want[64 + 16 * 3: 64 + 16 * 3 + 12].view("<u2")
+    assert [int(e) & 0x8000 != 0 for e in entries] == [False, False, True, False, False, True]
+    assert want_res.wire_len < plain_res.wire_len
+    wire, crc, r, _ = _run_encode(wm, a, chunk)
+    got = wire[: r.wire_len].cpu().numpy()
+    assert r.status == 0 and np.array_equal(got, want) and np.array_equal(crc, want_crc)
+    for strict in (False, True):
+        out, dcrc, rd = _run_decode(wm, got, n, chunk, strict=strict)
+        assert rd.status == 0 and np.array_equal(out, a) and np.array_equal(dcrc, want_crc)
+    # a damaged descriptor of a PACK tile inside such an image is found like in any other image
+    me = oracle.meta_end(n, chunk)
+    bad = want.copy()
+    bad[me + 1] ^= 0x10
+    want_bad = oracle.decode_verify(bad, n, chunk, expect_entropy=True)[2]
+    _, _, rb = _run_decode(wm, bad, n, chunk)
+    assert (rb.status, rb.first_bad_chunk, rb.n_bad_chunks) == (want_bad.status, want_bad.first_bad_chunk, want_bad.n_bad_chunks)
+    assert want_bad.status_name == "ERR_DESC"
 
 
 def test_ent_repeatable_under_load(wm):

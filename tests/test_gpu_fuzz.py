@@ -51,17 +51,17 @@ def test_random_case_matches_the_oracle(seed):
     n = int(rng.integers(1, 40 * TILE))
     if rng.integers(0, 4) == 0:
         n = max(TILE, n // TILE * TILE)                       # no ragged tail
-    option = ["default", "zero", "entropy"][seed % 3]
+    option = ["default", "zero", "entropy", "zero+entropy"][seed % 4]
     a = _data(rng, n)
     nc = oracle.num_chunks(n, chunk)
     masked = bool(rng.integers(0, 2))
     dirty = (rng.integers(0, 3, nc) > 0).astype(np.uint8) if masked else None
     crc_in = oracle.checksum(a, chunk)
     stale = crc_in.copy()
-    want, want_crc, want_res = oracle.encode(a, chunk, dirty=dirty, crc_in=stale, zero_tiles=option == "zero",
-                                             entropy=option == "entropy")
-    wm.zero_tiles_enable(option == "zero")
-    wm.entropy_enable(option == "entropy")
+    want, want_crc, want_res = oracle.encode(a, chunk, dirty=dirty, crc_in=stale, zero_tiles="zero" in option,
+                                             entropy="entropy" in option)
+    wm.zero_tiles_enable("zero" in option)
+    wm.entropy_enable("entropy" in option)
     try:
         ws = wm.new_workspace(n, chunk)
         wire = torch.full((wm.wire_bound(n, chunk),), 0xC3, dtype=torch.uint8, device="cuda")

@@ -16,7 +16,8 @@ def _cache(n, seed):
     return a
 
 
-@pytest.mark.parametrize("options,kw", [(0, {}), (1, {"zero_tiles": True}), (2, {"entropy": True}), (3, {"entropy": True})])
+@pytest.mark.parametrize("options,kw", [(0, {}), (1, {"zero_tiles": True}), (2, {"entropy": True}),
+                                        (3, {"entropy": True, "zero_tiles": True})])
 def test_options_per_call_match_the_oracle(options, kw):
     import torch
     from paper_2607_10389_b200 import binding as wm
