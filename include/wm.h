@@ -124,8 +124,8 @@ wm_status wm_dirty_diff(const void* cache, const void* prev, uint64_t nbytes, ui
  *
  *   header[64] | chunk_dir[16*n_chunks] | tile_tab[2*n_tiles] | zero pad to 32 | payload
  *   header: 0 "WMV1" | 4 u16 version=1 | 6 u16 flags (bit0: a dirty mask was given; bit1:
- *           the ZERO tile option, see wm_zero_tiles_enable; bit2: ENT tiles instead of PACK
- *           tiles, see wm_entropy_enable) |
+ *           the ZERO tile option, see wm_zero_tiles_enable; bit2: ENT tiles may occur, see
+ *           wm_entropy_enable) |
  *           8 u64 nbytes | 16 u32 chunk_bytes | 20 u32 tile_bytes=16384 | 24 u32 n_chunks |
  *           28 u32 n_present | 32 u64 payload_bytes | 40 u64 wire_len | 48 u32 cache_crc |
  *           52 u32 meta_crc (CRC32C of the metadata with this field as zero) | 56 zero[8]
@@ -134,7 +134,7 @@ wm_status wm_dirty_diff(const void* cache, const void* prev, uint64_t nbytes, ui
  *           all zero, no payload (only in images with flags bit1) | 2 CONST tile: a full tile whose 8192
  *           elements all hold one non-zero value; payload = that value (u16) and 30 zero bytes
  *           (only in images with flags bit1) | 258..511 PACK tile of 32*value bytes
- *           (only without flags bit2) | 512 RAW full tile | 0x8000 | n, n = 259..511: ENT tile of
+ *           | 512 RAW full tile | 0x8000 | n, n = 259..511: ENT tile of
  *           32*n bytes (only with flags bit2) | 0xFFFF RAW partial tail tile (nbytes mod 16384 bytes)
  *   payload: encoded tiles of present chunks in ascending order, no padding
  *   PACK tile (32 groups of 256 elements): desc[32] u16 (base | w<<8 | chk<<12,
@@ -222,16 +222,18 @@ wm_status wm_decode_verify_strict(const void* wire, uint64_t wire_len, void* dst
 void wm_zero_tiles_enable(int on);
 
 /*
- * wm_entropy_enable - codec option: entropy-coded exponents (ENT tiles instead of PACK tiles).
+ * wm_entropy_enable - codec option: entropy-coded exponents (ENT tiles beside PACK tiles).
  * Paper: the codec it measured entropy-codes the exponent plane inside the verified envelope
  * (Section 6.4); the bit-plane packing of the default format stops at a fixed number of bits
- * per group.  With the option on, wm_encode / wm_encode_leaves store a full tile of a present
- * chunk as an ENT tile or raw, and set header flags bit 2; the wm_decode_verify family then
- * expects such images.  A decode call whose option differs from the image's flag returns
- * WM_ERR_FORMAT.  While this option is on, the zero-tile option is ignored.  Process-wide, off
- * by default; set it on both ends of a move before the calls are issued.
+ * per group.  With the option on, wm_encode / wm_encode_leaves store every full tile of a present
+ * chunk in the shortest of three forms, an ENT tile, a PACK tile or raw (PACK on a tie, a coded
+ * form before raw), and set header flags bit 2: such an image is never longer than one without
+ * the option.  The wm_decode_verify family then expects such images; a decode call whose option
+ * differs from the image's flag returns WM_ERR_FORMAT.  The zero-tile option combines with this
+ * one.  Process-wide, off by default; set it on both ends of a move before the calls are issued
+ * (or use the calls that take their options as an argument).
  *
- * ENT tile (entry 0x8000 | length / 32 in the tile table, length < 16384, else the tile is raw):
+ * ENT tile (entry 0x8000 | length / 32 in the tile table; the length is below 16384):
  *   a tile is eight shares of 16 rows (row = 128 bytes); share s has 32 strands, strand l = the 32
  *   elements at 32-bit word l of the share's rows, row after row, low half first.
  *   anchor_s = (sum of the share's 1024 exponents + 512) >> 10.  u = E - anchor_s is coded
