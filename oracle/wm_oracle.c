@@ -27,7 +27,10 @@
  * a hardware CRC instruction, zlib's combine identity and brute force.  The
  * encoder's byte layout is new, so no outside implementation exists for it:
  * "parity unpinned" against the outside world; it is pinned by hand-built
- * tiles, a size law recomputed independently, and the round trip.
+ * tiles, a size law recomputed independently, and the round trip.  The same
+ * holds for the ENT tiles of the entropy option ("parity unpinned" against the
+ * outside world): hand-derived streams, Kraft equality, Shannon's bound, the
+ * size law and the choice among the three forms recomputed independently.
  */
 #include <stdint.h>
 #include <stdlib.h>
