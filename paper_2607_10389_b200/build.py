@@ -7,7 +7,7 @@ import sys
 
 HERE = os.path.dirname(os.path.abspath(__file__))
 SRC = [os.path.join(HERE, "csrc", "wm_kernels.cu")]
-DEPS = [os.path.join(HERE, "csrc", f) for f in ("wm_kernels.cu", "wm_device.cuh", "wm_tables.h")] + [
+DEPS = [os.path.join(HERE, "csrc", f) for f in sorted(os.listdir(os.path.join(HERE, "csrc")))] + [
     os.path.join(os.path.dirname(HERE), "include", "wm.h")]
 OUT = os.path.join(HERE, "libwm.so")
 

@@ -1,0 +1,692 @@
+// wm_decode_verify: the gate (k_decode_check), the unpack + checksum kernel with its variants
+// (leaves, strict passes, entropy option) and the verdict (k_decode_finish).
+// Part of the one translation unit wm_kernels.cu (included there, in this order).
+#pragma once
+
+namespace wm {
+
+// ------------------------------------------------------------------ wm_decode_verify
+
+__global__ void k_decode_init(Ws ws)
+{
+    grid_dep_launch();
+    if (blockIdx.x == 0 && threadIdx.x < sizeof(Ctrl) / 4) {
+        uint32_t v = 0;
+        const uint32_t i = threadIdx.x;
+        if (i == offsetof(Ctrl, bad3_first) / 4 || i == offsetof(Ctrl, bad4_first) / 4 ||
+            i == offsetof(Ctrl, bad5_first) / 4 || i == offsetof(Ctrl, bad6_first) / 4 ||
+            i == offsetof(Ctrl, bad4_key) / 4 || i == offsetof(Ctrl, bad4_key) / 4 + 1)
+            v = 0xFFFFFFFFu;
+        reinterpret_cast<uint32_t*>(ws.ctrl)[i] = v;
+    }
+}
+
+__device__ __forceinline__ void fill_result(wm_result* result, const Ctrl* ctrl, uint64_t wire_len, int status,
+                                            uint32_t first, uint32_t count)
+{
+    wm_result r;
+    memset(&r, 0, sizeof r);
+    r.status = status;
+    r.first_bad_chunk = first;
+    r.n_bad_chunks = count;
+    r.n_present = ctrl->hdr_n_present;
+    r.payload_bytes = ctrl->payload_total;
+    r.wire_len = wire_len;
+    r.cache_crc = ctrl->hdr_cache_crc;
+    *result = r;
+}
+
+// Decode steps 1-3 in one kernel.  The first blocks digest the metadata slices (four teams
+// each), the others check the structure chunk by chunk (one warp per chunk: tile entries
+// against the chunk's length and enc_len; also each tile's offset inside its chunk's payload).
+// Neither part follows anything it reads: every index comes from the call's geometry, so the
+// structure pass is safe on damaged metadata and can run beside the CRC.  The last block to
+// finish decides in the specified order: metadata CRC first (WM_ERR_META_CRC), then the
+// structure (WM_ERR_STRUCT: per-chunk findings, payload offsets as the running sum of enc_len,
+// totals against the header).  A header that does not match the call stops every block at
+// once (WM_ERR_FORMAT).  A failure sets the gate that keeps the later kernels out.
+__global__ void __launch_bounds__(1024)
+k_decode_check(const unsigned char* __restrict__ wire, uint64_t wire_len, Geo g, Ws ws,
+               const Tables* __restrict__ tab, wm_result* result, uint32_t meta_blocks, uint32_t expect_ent)
+{
+    __shared__ uint32_t sG[1024];
+    __shared__ uint32_t sHT[1024];
+    __shared__ uint32_t s_dig[1024];
+    __shared__ uint32_t s_wdig[4][8];
+    __shared__ unsigned long long s_warp[32];
+    __shared__ unsigned long long s_carry;
+    __shared__ uint32_t s_first, s_count;
+    __shared__ bool s_last;
+    __shared__ int s_format_bad;
+    const uint32_t lane = threadIdx.x % 32, wblk = threadIdx.x / 32;
+    sHT[threadIdx.x] = (&tab->HT[0][0])[threadIdx.x];
+    load_small_chain_tables(sG, tab);
+    grid_dep_wait();
+    grid_dep_launch();
+    if (ld_volatile_u32(&ws.ctrl->gate)) return;        // leaf mode: the destination table was rejected
+    if (threadIdx.x == 0) s_format_bad = header_matches(wire, wire_len, g, expect_ent) ? 0 : 1;
+    __syncthreads();
+    if (s_format_bad) {
+        if (blockIdx.x == 0 && threadIdx.x == 0) {
+            ws.ctrl->gate = (uint32_t)WM_ERR_FORMAT;
+            wm_result r;
+            memset(&r, 0, sizeof r);
+            r.status = WM_ERR_FORMAT;
+            *result = r;
+        }
+        return;
+    }
+    const unsigned char* dir = wire + 64;
+    const bool zero_ok = ((reinterpret_cast<const uint32_t*>(wire)[1] >> 17) & 1u) != 0u;   // the image declares the option
+    if (blockIdx.x < meta_blocks) {
+        const uint32_t team = threadIdx.x / kTeamThreads, tt = threadIdx.x % kTeamThreads;
+        const uint32_t s = blockIdx.x * 4 + team;
+        if (s < g.n_meta_slices) meta_slice_parts(wire, g, s, sG, tab, s_wdig[team], tt / 32, lane);
+        __syncthreads();
+        if (tt == 0 && s < g.n_meta_slices) ws.mdig[s] = xor8(s_wdig[team]);
+    } else {
+        const uint16_t* tab16 = reinterpret_cast<const uint16_t*>(wire + 64 + 16ull * g.n_chunks);
+        const uint32_t c = (blockIdx.x - meta_blocks) * 32u + wblk;
+        if (c < g.n_chunks) {
+            const uint64_t clen = chunk_len_dev(g, c);
+            const uint32_t t0 = c * g.tiles_per_chunk;
+            const uint32_t ntc = (uint32_t)((clen + kTile - 1) / kTile);
+            const uint32_t elen = *reinterpret_cast<const uint32_t*>(dir + 16ull * c + 8);
+            unsigned long long carry = 0;
+            bool ok = true, any = false, all = true;
+            for (uint32_t i0 = 0; i0 < ntc; i0 += 32) {
+                const uint32_t i = i0 + lane;
+                uint32_t len = 0;
+                bool l_ok = true, l_any = false, l_all = true, l_packs = false;
+                if (i < ntc) {
+                    const uint32_t e = tab16[t0 + i];
+                    const uint64_t tl = clen - (uint64_t)i * kTile;
+                    if (e == 0) l_all = false;
+                    else {
+                        l_any = true;
+                        if (tl < kTile) { if (e != 0xFFFFu) l_ok = false; len = (uint32_t)tl; }
+                        else if (e == 1u && zero_ok) len = 0;       // a tile of zeros: no payload
+                        else if (e == 2u && zero_ok) len = 32;      // a tile of one value: the value
+                        else if (e >= 258u && e <= 512u) { len = 32u * e; l_packs = e < 512u; }
+                        else if (expect_ent && e >= (0x8000u | 259u) && e <= (0x8000u | 511u)) len = 32u * (e & 0x7FFFu);   // ENT tile
+                        else l_ok = false;
+                    }
+                }
+                uint32_t incl = len;
+#pragma unroll
+                for (int d = 1; d < 32; d <<= 1) {
+                    uint32_t o = __shfl_up_sync(0xFFFFFFFFu, incl, d);
+                    if (lane >= (uint32_t)d) incl += o;
+                }
+                if (i < ntc) ws.rel[t0 + i] = (uint32_t)(carry + incl - len);
+                carry += __shfl_sync(0xFFFFFFFFu, incl, 31);
+                if (expect_ent && __any_sync(0xFFFFFFFFu, l_packs) && lane == 0) atomicOr(&ws.ctrl->has_pack, 1u);
+                ok = ok && __all_sync(0xFFFFFFFFu, l_ok);
+                any = any || __any_sync(0xFFFFFFFFu, l_any);
+                all = all && __all_sync(0xFFFFFFFFu, l_all);
+            }
+            if (any && !all) ok = false;
+            if (carry != elen) ok = false;
+            if (lane == 0) {
+                ws.cflag[c] = (any ? CF_PRESENT : 0u) | (ok ? 0u : CF_BAD3);
+                if (!ok) { atomicMin(&ws.ctrl->bad3_first, c); atomicAdd(&ws.ctrl->bad3_count, 1u); }
+                if (any) atomicAdd(&ws.ctrl->n_present, 1u);
+            }
+        }
+    }
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        s_carry = 0; s_first = 0xFFFFFFFFu; s_count = 0;
+        __threadfence();
+        s_last = atomicAdd(&ws.ctrl->done_b, 1u) == gridDim.x - 1;
+    }
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+
+    // ---- the last block: metadata CRC first
+    const uint32_t crc = fold_meta_digests(g, ws, sHT, s_dig);
+    if (threadIdx.x == 0) {
+        const uint32_t* h = reinterpret_cast<const uint32_t*>(wire);
+        ws.ctrl->hdr_n_present = h[7];
+        ws.ctrl->hdr_cache_crc = h[12];
+        ws.ctrl->payload_total = h[8] | ((unsigned long long)h[9] << 32);
+        s_format_bad = 0;
+        if (crc != h[13]) {
+            s_format_bad = 1;
+            ws.ctrl->gate = (uint32_t)WM_ERR_META_CRC;
+            wm_result r;
+            memset(&r, 0, sizeof r);
+            r.status = WM_ERR_META_CRC;
+            r.n_present = h[7];
+            r.payload_bytes = ws.ctrl->payload_total;
+            r.wire_len = wire_len;
+            r.cache_crc = h[12];
+            *result = r;
+        }
+    }
+    __syncthreads();
+    if (s_format_bad) return;
+
+    // ---- then the structure across chunks
+    for (uint32_t base = 0; base < g.n_chunks; base += 1024) {
+        const uint32_t cc = base + threadIdx.x;
+        unsigned long long len = 0, po = 0;
+        if (cc < g.n_chunks) {
+            po = *reinterpret_cast<const unsigned long long*>(dir + 16ull * cc);
+            len = *reinterpret_cast<const uint32_t*>(dir + 16ull * cc + 8);
+        }
+        unsigned long long incl = len;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            unsigned long long o = __shfl_up_sync(0xFFFFFFFFu, incl, d);
+            if (lane >= (uint32_t)d) incl += o;
+        }
+        if (lane == 31) s_warp[wblk] = incl;
+        __syncthreads();
+        unsigned long long before = s_carry;
+        for (uint32_t w2 = 0; w2 < wblk; w2++) before += s_warp[w2];
+        if (cc < g.n_chunks && po != before + incl - len) {
+            // a chunk already counted by the per-chunk pass must not be counted twice
+            const uint32_t fl = ld_volatile_u32(&ws.cflag[cc]);
+            if (!(fl & CF_BAD3)) {
+                ws.cflag[cc] = fl | CF_BAD3;
+                atomicMin(&s_first, cc);
+                atomicAdd(&s_count, 1u);
+            }
+        }
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            unsigned long long tot = 0;
+            for (int w2 = 0; w2 < 32; w2++) tot += s_warp[w2];
+            s_carry += tot;
+        }
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) {
+        uint32_t first = min(s_first, ld_volatile_u32(&ws.ctrl->bad3_first));
+        uint32_t count = s_count + ld_volatile_u32(&ws.ctrl->bad3_count);
+        if (count == 0 && (s_carry != ws.ctrl->payload_total ||
+                           ld_volatile_u32(&ws.ctrl->n_present) != ws.ctrl->hdr_n_present)) {
+            first = 0; count = 1;
+        }
+        if (count) {
+            ws.ctrl->gate = (uint32_t)WM_ERR_STRUCT;
+            fill_result(result, ws.ctrl, wire_len, WM_ERR_STRUCT, first, count);
+        }
+    }
+}
+
+struct DecSlot {                 // what the team's first thread prepares for a tile ahead of its turn
+    uint32_t t;                  // tile (>= n_tiles: none left)
+    uint32_t entry;              // tile table entry | (first tile of its chunk) << 16
+    unsigned long long src;      // offset of the encoded tile inside the payload
+};
+struct DecTeamCtl {
+    uint32_t wdig[2][8];
+    DecSlot slot[4];             // ring: slot i & 3 belongs to the team's i-th tile
+    unsigned long long mbar;     // completion of the bulk copy into the team's stage
+    unsigned long long pad;
+};
+static_assert(sizeof(DecTeamCtl) % 16 == 0, "team control block keeps 16-byte alignment");
+
+// The plane words of one group as stored (aligned per-lane units, see pack_group_planes):
+// a = the 4-bit plane's word or the low half of an 8-bit plane; b = the 2-bit plane's 16 bits
+// in the low half and the 1-bit plane's byte in bits 16-23, or the high half of an 8-bit plane.
+struct PlaneWords { uint32_t a, b; };
+
+// rec: shared-window address of the group's planes; l4 / l2 / l1: 4, 2, 1 times the lane number
+__device__ __forceinline__ PlaneWords read_group_planes(uint32_t rec, uint32_t wd, uint32_t l4, uint32_t l2, uint32_t l1)
+{
+    PlaneWords pw;
+    pw.a = 0; pw.b = 0;
+    if (wd == 8u) {
+        const uint2 v = lds_now_v2<0>(rec + 2u * l4);
+        pw.a = v.x; pw.b = v.y;
+        return pw;
+    }
+    if (wd & 4u) { pw.a = lds_now<0>(rec + l4); rec += 128u; }
+    if (wd & 2u) { pw.b = lds_now_u16(rec + l2); rec += 64u; }
+    if (wd & 1u) { pw.b |= lds_now_u8(rec + l1) << 16; }
+    return pw;
+}
+
+// Inverse of pack_group_planes: the lane's eight exponent bytes (two words, coded order).
+template <int W>
+__device__ __forceinline__ void unpack_group_planes(const PlaneWords& pw, uint32_t base, uint32_t& ea, uint32_t& eb)
+{
+    uint32_t da = 0, db = 0;
+    if (W == 8) { da = pw.a; db = pw.b; }
+    else {
+        int sh = 0;
+        if (W & 4) {
+            const uint32_t t = __byte_perm(pw.a, 0, 0x1100), u = __byte_perm(pw.a, 0, 0x3322);
+            da = (t & 0x000F000Fu) | ((t >> 4) & 0x0F000F00u);
+            db = (u & 0x000F000Fu) | ((u >> 4) & 0x0F000F00u);
+            sh = 4;
+        }
+        if (W & 2) {        // byte -> four 2-bit fields, one per byte
+            uint32_t xa = pw.b & 0xFFu, xb = (pw.b >> 8) & 0xFFu;
+            xa = (xa * 0x1001u) & 0x000F000Fu; xa = (xa * 0x41u) & 0x03030303u;
+            xb = (xb * 0x1001u) & 0x000F000Fu; xb = (xb * 0x41u) & 0x03030303u;
+            da |= xa << sh; db |= xb << sh;
+            sh += 2;
+        }
+        if (W & 1) {        // nibble -> four bits, one per byte
+            const uint32_t xa = (((pw.b >> 16) & 0xFu) * 0x00204081u) & 0x01010101u;
+            const uint32_t xb = (((pw.b >> 20) & 0xFu) * 0x00204081u) & 0x01010101u;
+            da |= xa << sh; db |= xb << sh;
+        }
+    }
+    const uint32_t b4 = base * 0x01010101u;
+    if (base + ((1u << W) - 1u) <= 255u) {        // no byte can wrap: plain add
+        ea = da + b4; eb = db + b4;
+    } else {                                      // per byte (base + d) & 0xFF
+        ea = ((da & 0x7F7F7F7Fu) + (b4 & 0x7F7F7F7Fu)) ^ ((da ^ b4) & 0x80808080u);
+        eb = ((db & 0x7F7F7F7Fu) + (b4 & 0x7F7F7F7Fu)) ^ ((db ^ b4) & 0x80808080u);
+    }
+}
+
+// Unpack + checksum of the decoded bytes.  Tiles are claimed by ticket.  The team owns one
+// 16 KiB stage in shared memory; the encoded tile arrives there by one bulk copy (TMA) that is
+// started a tile ahead, each lane takes what it needs (descriptors, its 8 sign-mantissa bytes
+// and its plane words per group: at most 16 words) into registers, and the stage is handed to
+// the next copy while the team unpacks, stores and checksums.  One team barrier per tile.
+// Tiles are prepared ahead of their turn, one dependent step per tile so that nobody sits
+// waiting for an answer from L2: claim a ticket (three tiles ahead, warp 3), look up that
+// tile's table entry and offsets (two ahead, warp 0), start its copy (one ahead, warp 2); warp 1
+// folds and stores the previous tile's digest.  (Spread over warps because the team runs at
+// the pace of its slowest one.)  LEAVES: the decoded tiles go to a table of tensors.
+// MODE 0: unpack, store, checksum (the normal call).  Strict calls run the kernel twice: MODE 1
+// unpacks and checksums without storing anything; MODE 2, after the verdict, unpacks and stores.
+// ENT 1 / 2: the image was written with the entropy option and holds ENT tiles only (1) or ENT
+// and PACK tiles (2; the check kernel noted which).  A call launches both, and the one that does
+// not apply returns at once: the kernel with a single kind of coded tile is the faster one.  A
+// warp reads its share's stream of halfwords in phase 1 (the need test, the ballot and the fetch
+// of every step) and leaves the exponent bytes where the plane words would be.
+template <int TEAMS, bool LEAVES, int MODE, int ENT = 0>
+__global__ void __launch_bounds__(TEAMS * 256, 1)
+k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restrict__ dst, Ws ws,
+         const Tables* __restrict__ tab)
+{
+    extern __shared__ __align__(16) unsigned char smem[];
+    // ENT: what the low byte of a strand's bits says about the codeword there: its length (16: the
+    // escape) and u as a byte.  Two byte tables: the index needs no scaling and a look-up gives a
+    // clean value.
+    __shared__ unsigned char s_plen[ENT ? 256 : 4], s_pu[ENT ? 256 : 4];
+    if (ENT != 0 && threadIdx.x < 256u) {
+        const uint32_t s = ent_ones(threadIdx.x);
+        s_plen[threadIdx.x] = (unsigned char)ent_parse_length(s);
+        s_pu[threadIdx.x] = (unsigned char)(s == 8u ? 0u : ent_parse_value(threadIdx.x, s, 0u));
+    }
+    Smem S = setup_smem(smem, tab);
+    grid_dep_wait();
+    grid_dep_launch();
+    if (ld_volatile_u32(&ws.ctrl->gate)) return;
+    if (ENT != 0 && (ENT == 1) == (ld_volatile_u32(&ws.ctrl->has_pack) != 0u)) return;      // the other kernel's image
+    const uint32_t team = threadIdx.x / kTeamThreads, tt = threadIdx.x % kTeamThreads;
+    const uint32_t warp = tt / 32, lane = tt % 32;
+    unsigned char* stage = nullptr;
+    for (int i = 0; i < TEAMS; i++) {          // every thread carves the same blocks in the same order
+        unsigned char* p = S.take(kTile);
+        if ((uint32_t)i == team) stage = p;
+    }
+    DecTeamCtl* tc = reinterpret_cast<DecTeamCtl*>(S.take(TEAMS * sizeof(DecTeamCtl)));
+    if (!S.ok) { if (threadIdx.x == 0) atomicOr(&ws.ctrl->err, 4u); return; }
+    tc += team;
+    const unsigned char* const dir = wire + 64;
+    const uint16_t* const tab16 = reinterpret_cast<const uint16_t*>(wire + 64 + 16ull * g.n_chunks);
+    const unsigned char* const payload = wire + g.meta_end;
+    const bool leader = (tt == 0);
+    constexpr uint32_t kNone = 0xFFFFFFFFu;
+    const uint32_t stage_s = (uint32_t)__cvta_generic_to_shared(stage);
+    const uint32_t sm_s = stage_s + 64u + 1024u * warp + 8u * lane;     // this lane's sign-mantissa bytes, group 4 warp
+
+    // a tile's entry word and payload offset (blocking: prologue only)
+    auto lookup = [&](uint32_t t, DecSlot* sl) {
+        sl->t = t;
+        sl->entry = 0; sl->src = 0;
+        if (t < g.n_tiles) {
+            const uint32_t e = tab16[t];
+            sl->entry = e | (first_in_chunk(g, t) ? 0x10000u : 0u);
+            if (e) sl->src = *reinterpret_cast<const unsigned long long*>(dir + 16ull * chunk_of(g, t)) + ws.rel[t];
+        }
+    };
+    // staged tiles: full RAW and PACK tiles (everything except absent tiles and the ragged tail)
+    // (images with the entropy option hold ENT tiles too: entry 0x8000 | length / 32)
+    auto is_ent_entry = [](uint32_t e) { return ENT != 0 && e > 0x8000u && e != 0xFFFFu; };
+    auto is_pack_entry = [](uint32_t e) { return ENT != 1 && e >= 258u && e < 512u; };
+    auto is_staged = [&](uint32_t e) { return e == 512u || is_pack_entry(e) || is_ent_entry(e); };
+    auto start_copy = [&](const DecSlot& sl) {   // leader only
+        const uint32_t e = sl.entry & 0xFFFFu;
+        if (sl.t < g.n_tiles && is_staged(e)) bulk_load(stage, payload + sl.src, 32u * (e & 0x7FFFu), &tc->mbar, 0);
+    };
+
+    if (leader) {
+        mbar_init(&tc->mbar, 1);
+        lookup(atomicAdd(&ws.ctrl->ticket, 1u), &tc->slot[0]);
+        lookup(atomicAdd(&ws.ctrl->ticket, 1u), &tc->slot[1]);
+        tc->slot[2].t = atomicAdd(&ws.ctrl->ticket, 1u);      // its look-ups happen in the first step
+        start_copy(tc->slot[0]);
+    }
+    team_bar(team);
+    uint32_t phase = 0;
+    uint32_t trouble = 0;              // sticky: a copy never arrived
+    uint32_t t_done = kNone;           // tile whose digest parts wait in wdig[(it - 1) & 1]
+    for (uint32_t it = 0;; it++) {
+        const uint32_t t = tc->slot[it & 3u].t;
+        if (t >= g.n_tiles) {
+            team_bar(team);
+            if (tt == 32u && t_done != kNone) ws.dig[t_done] = xor8(tc->wdig[(it & 1u) ^ 1u]);
+            break;
+        }
+        const uint32_t ew = tc->slot[it & 3u].entry;
+        const uint32_t e = ew & 0xFFFFu;
+        // leaf mode: where this tile goes (asked for now, needed when the stores begin)
+        unsigned char* const o_leaf = LEAVES ? ws.tptr[t] : nullptr;
+        const uint32_t p = it & 1u;
+        const bool is_ent = is_ent_entry(e);
+        const bool is_pack = is_ent || is_pack_entry(e);            // a coded tile (in either form)
+        bool decoded = true;
+        uint32_t w[kWordsPerLane];
+        uint32_t desc = 0;
+        uint2 sm[4];
+        PlaneWords pw[4];
+
+        // ---- phase 1: everything this lane needs from the stage goes into registers
+        if (is_staged(e)) {
+            if (!mbar_wait(&tc->mbar, phase)) trouble = 1u;
+            phase ^= 1u;
+            if (!is_pack) {
+                read_staged_words(stage, warp, lane, w);
+            } else if (is_ent) {
+                // ENT tile.  Header: the eight stream lengths against the entry (structure); then this
+                // warp reads its share's stream the way the format interleaves it: at step i every
+                // strand whose codeword i is not complete in the bits it holds takes the stream's next
+                // halfword, strands in ascending order.  The stream must be used up exactly and the
+                // bits left in every strand must be zero (descriptor error otherwise).
+                const uint32_t cnt = lane < 8u ? lds_now_u16(stage_s + 8u + 2u * lane) : 0u;
+                const bool cnt_bad = lane < 8u && (cnt < 128u || cnt > 1024u);
+                const uint32_t total = __reduce_add_sync(0xFFFFFFFFu, cnt);
+                const uint32_t before = __reduce_add_sync(0xFFFFFFFFu, lane < warp ? cnt : 0u);
+                const uint32_t mine = __shfl_sync(0xFFFFFFFFu, cnt, warp);
+                int verdict = (__any_sync(0xFFFFFFFFu, cnt_bad) || ent_tile_bytes(total) != 32u * (e & 0x7FFFu)) ? 2 : 0;
+                if (!verdict) {
+                    const uint32_t anchor = lds_now_u8(stage_s + warp);
+                    const uint32_t st = stage_s + 8256u + 2u * before;
+                    const uint32_t lt_mask = (1u << lane) - 1u;
+                    uint32_t buf = 0, avail = 0, pos = 0, ew[8];
+                    const uint32_t last = mine - 1u;           // (mine >= 128)
+#pragma unroll
+                    for (int j = 0; j < 8; j++) ew[j] = 0u;
+#pragma unroll
+                    for (int i = 0; i < 32; i++) {
+                        const bool more = s_plen[buf & 0xFFu] > avail;
+                        const uint32_t takers = __ballot_sync(0xFFFFFFFFu, more);
+                        if (more) {
+                            // (an index past the stream's end is only clamped here: the stream then
+                            // fails the count check below, because every index is below the final pos)
+                            const uint32_t idx = min(pos + __popc(takers & lt_mask), last);
+                            buf |= lds_now_u16(st + 2u * idx) << avail;
+                            avail += 16u;
+                        }
+                        pos += __popc(takers);
+                        const uint32_t low = buf & 0xFFu;
+                        const uint32_t len = s_plen[low];
+                        const uint32_t E = len == 16u ? buf >> 8 : anchor + s_pu[low];      // (its low byte)
+                        ew[i >> 2] = __byte_perm(ew[i >> 2], E, (i & 3) == 0 ? 0x3214 : (i & 3) == 1 ? 0x3240 : (i & 3) == 2 ? 0x3410 : 0x4210);
+                        buf >>= len;
+                        avail -= len;
+                    }
+                    if (__any_sync(0xFFFFFFFFu, buf != 0u) || pos != mine) verdict = 1;
+#pragma unroll
+                    for (int j = 0; j < 4; j++) {
+                        sm[j] = j == 0 ? lds_now_v2<0>(sm_s) : j == 1 ? lds_now_v2<256>(sm_s) : j == 2 ? lds_now_v2<512>(sm_s) : lds_now_v2<768>(sm_s);
+                        pw[j].a = ew[2 * j];
+                        pw[j].b = ew[2 * j + 1];
+                    }
+                }
+                if (verdict) {               // (a stream that does not fit is this warp's finding alone)
+                    decoded = false;
+                    if (lane == 0) {
+                        atomicMin(&ws.ctrl->bad4_key, (unsigned long long)t * 2ull + (verdict == 2 ? 1ull : 0ull));
+                        atomicOr(&ws.cflag[chunk_of(g, t)], CF_BAD4);
+                    }
+                }
+            } else if (ENT != 1) {
+#ifdef WM_AB_D_NOP1
+                desc = 100u | (4u << 8);
+                for (int j = 0; j < 4; j++) { sm[j] = make_uint2(lane, it); pw[j].a = t; pw[j].b = e; }
+#else
+                desc = lds_now_u16(stage_s + 2u * lane);
+                const uint32_t wv = (desc >> 8) & 15u;
+                const uint32_t base_l = desc & 0xFFu, chk = desc >> 12;
+                const bool bad = wv > 8u || chk != (((base_l & 15u) ^ (base_l >> 4) ^ wv ^ 5u) & 15u);
+                const bool anybad = __any_sync(0xFFFFFFFFu, bad);
+                // sum of all 32 widths, and of the widths of the groups before this warp's four
+                const uint32_t Ssum = __reduce_add_sync(0xFFFFFFFFu, wv);
+                const uint32_t before = __reduce_add_sync(0xFFFFFFFFu, lane < 4u * warp ? wv : 0u);
+                const int verdict = anybad ? 1 : (258u + Ssum != e ? 2 : 0);
+                if (verdict) {               // every warp reaches the same verdict
+                    decoded = false;
+                    if (leader) {
+                        atomicMin(&ws.ctrl->bad4_key, (unsigned long long)t * 2ull + (verdict == 2 ? 1ull : 0ull));
+                        atomicOr(&ws.cflag[chunk_of(g, t)], CF_BAD4);
+                    }
+                } else {
+                    // lanes 0..3 end up with the descriptors of the warp's four groups, each with its
+                    // group's offset in the plane area in the high half
+                    const uint32_t own = __shfl_sync(0xFFFFFFFFu, desc, 4 * warp + (lane & 3u)) & 0xFFFFu;
+                    const uint32_t wo = (own >> 8) & 15u;
+                    uint32_t off = before;                          // running offset over the four groups
+                    const uint32_t w0 = __shfl_sync(0xFFFFFFFFu, wo, 0), w1 = __shfl_sync(0xFFFFFFFFu, wo, 1),
+                                   w2 = __shfl_sync(0xFFFFFFFFu, wo, 2);
+                    if ((lane & 3u) >= 1u) off += w0;
+                    if ((lane & 3u) >= 2u) off += w1;
+                    if ((lane & 3u) == 3u) off += w2;
+                    desc = own | (off << 16);
+#pragma unroll
+                    for (int j = 0; j < 4; j++) {
+                        const uint32_t dg = __shfl_sync(0xFFFFFFFFu, desc, j);
+                        sm[j] = j == 0 ? lds_now_v2<0>(sm_s) : j == 1 ? lds_now_v2<256>(sm_s) : j == 2 ? lds_now_v2<512>(sm_s) : lds_now_v2<768>(sm_s);
+                        pw[j] = read_group_planes(stage_s + 8256u + 32u * (dg >> 16), (dg >> 8) & 15u, 4u * lane, 2u * lane, lane);
+                    }
+                }
+#endif
+            }
+        } else if (e == 1u || e == 2u) {
+            // a tile of zeros (nothing was shipped) or of one value (the first two bytes of its 32):
+            // from here on it goes the way of a raw tile
+            uint32_t v = 0;
+            if (e == 2u) v = __ldg(reinterpret_cast<const unsigned short*>(payload + tc->slot[it & 3u].src)) * 0x10001u;
+#pragma unroll
+            for (int i = 0; i < 16; i++) w[i] = v;
+        }
+        team_bar(team);                      // stage free; the slots the leader filled last step visible;
+                                             // the previous tile's digest parts complete
+        // The leader: next tile's copy; the previous tile's digest; look-ups for the tile two
+        // ahead and the ticket of the tile three ahead (answers taken at the end of the step).
+        uint32_t l_e = 0, l_rel = 0, l_tk = kNone;
+        unsigned long long l_po = 0;
+        // (spread over three warps: the team waits for whichever warp has the most to do)
+        if (tt == 64u) start_copy(tc->slot[(it + 1u) & 3u]);
+        if (tt == 32u && t_done != kNone) ws.dig[t_done] = xor8(tc->wdig[p ^ 1u]);
+        uint32_t t_look = kNone;           // warps 0 and 3: the tile claimed a step ago (two tiles ahead)
+        if (leader) {                      // its table entry and offsets
+            t_look = tc->slot[(it + 2u) & 3u].t;
+            if (t_look < g.n_tiles) {
+                l_e = tab16[t_look];
+                l_rel = __ldcg(ws.rel + t_look);
+                l_po = *reinterpret_cast<const unsigned long long*>(dir + 16ull * chunk_of(g, t_look));
+            }
+        }
+        if (tt == 96u) {                   // the ticket of the tile three ahead
+            t_look = tc->slot[(it + 2u) & 3u].t;
+            if (t_look < g.n_tiles) l_tk = atomicAdd(&ws.ctrl->ticket, 1u);
+        }
+
+        // ---- phase 2: unpack, store, checksum
+        bool have_digest = false;
+        if (e != 0) {
+            unsigned char* o = LEAVES ? o_leaf : dst + (uint64_t)t * kTile;
+            bool fold = (ew >> 16) != 0;
+            if (e == 0xFFFFu) {
+                const unsigned char* src = payload + tc->slot[it & 3u].src;
+                const uint32_t len = g.tail_len;
+                if (MODE != 1) for (uint32_t i = tt; i < len; i += kTeamThreads) o[i] = src[i];
+                if (MODE != 2) load_tile_words_guarded(src, len, fold, warp, lane, w);
+                fold = false;
+            } else if (is_pack && decoded) {
+#ifdef WM_AB_D_NOUNPACK
+#pragma unroll
+                for (int j = 0; j < 4; j++) { w[4 * j] = sm[j].x; w[4 * j + 1] = sm[j].y; w[4 * j + 2] = pw[j].a; w[4 * j + 3] = pw[j].b; }
+#else
+#pragma unroll
+                for (int j = 0; j < 4; j++) {
+                    const uint32_t dg = __shfl_sync(0xFFFFFFFFu, desc, j);
+                    const uint32_t base = dg & 0xFFu, wd = (dg >> 8) & 15u;
+                    uint32_t ea = base * 0x01010101u, eb = ea;
+                    if (ENT == 1 || (ENT == 2 && is_ent)) { ea = pw[j].a; eb = pw[j].b; }     // the exponent bytes are already there
+                    else if (wd == 4u) unpack_group_planes<4>(pw[j], base, ea, eb);       // by far the most frequent width
+                    else switch (wd) {     // uniform across the warp
+                        case 1: unpack_group_planes<1>(pw[j], base, ea, eb); break;
+                        case 2: unpack_group_planes<2>(pw[j], base, ea, eb); break;
+                        case 3: unpack_group_planes<3>(pw[j], base, ea, eb); break;
+                        case 5: unpack_group_planes<5>(pw[j], base, ea, eb); break;
+                        case 6: unpack_group_planes<6>(pw[j], base, ea, eb); break;
+                        case 7: unpack_group_planes<7>(pw[j], base, ea, eb); break;
+                        case 8: unpack_group_planes<8>(pw[j], base, ea, eb); break;
+                        default: break;
+                    }
+                    // A word rotated left by one bit reads [E | m << 1 | sign of the other half] in
+                    // each half: swap bit 0 inside the byte pairs of the sign-mantissa words, put
+                    // the exponent bytes beside them, rotate back.
+                    const uint32_t xa = __byte_perm(sm[j].x, sm[j].x, 0x2301), xb = __byte_perm(sm[j].y, sm[j].y, 0x2301);
+                    const uint32_t sa = (sm[j].x & 0xFEFEFEFEu) | (xa & 0x01010101u), sb = (sm[j].y & 0xFEFEFEFEu) | (xb & 0x01010101u);
+                    const uint32_t r0 = __byte_perm(sa, ea, 0x5140), r1 = __byte_perm(sa, ea, 0x7362);
+                    const uint32_t r2 = __byte_perm(sb, eb, 0x5140), r3 = __byte_perm(sb, eb, 0x7362);
+                    w[4 * j] = __funnelshift_r(r0, r0, 1);
+                    w[4 * j + 1] = __funnelshift_r(r1, r1, 1);
+                    w[4 * j + 2] = __funnelshift_r(r2, r2, 1);
+                    w[4 * j + 3] = __funnelshift_r(r3, r3, 1);
+                }
+#endif
+            }
+            if (decoded) {
+#ifndef WM_AB_D_NOSTORE
+                if (MODE != 1 && e != 0xFFFFu) {
+                    unsigned char* q = o + warp * 2048u + lane * 4u;
+#pragma unroll
+                    for (int i = 0; i < 16; i++) st_stream_u32(q + i * 128, w[i]);
+                }
+#else
+                if (w[7] == 0x12345678u && e != 0xFFFFu) st_stream_u32(o + lane * 4u, w[2] ^ w[9] ^ w[12] ^ w[15] ^ w[0] ^ w[5]);
+#endif
+                if (MODE != 2) {
+#ifdef WM_AB_D_NOCRC
+                    const uint32_t v = w[3] ^ w[6] ^ w[8] ^ w[13] ^ w[1] ^ w[4] ^ w[10] ^ w[11] ^ w[14];
+#else
+                    const uint32_t v = tile_digest_part(S, w, fold, warp, lane);
+#endif
+                    if (lane == 0) tc->wdig[p][warp] = v;
+                    have_digest = true;
+                }
+            }
+        }
+        t_done = have_digest ? t : kNone;
+        if (leader && t_look < g.n_tiles) {
+            DecSlot* s2 = &tc->slot[(it + 2u) & 3u];
+            s2->entry = l_e | (first_in_chunk(g, t_look) ? 0x10000u : 0u);
+            s2->src = l_po + l_rel;
+        }
+        if (tt == 96u) tc->slot[(it + 3u) & 3u].t = l_tk;      // (none once the tickets have run out)
+    }
+    if (trouble && lane == 0) atomicOr(&ws.ctrl->err, 2u);
+}
+
+// Steps 5..8: chunk CRCs of the decoded bytes against the directory, stale check, cache CRC;
+// the last block to finish decides the status and, on success only, updates dst_crc_inout.
+__global__ void __launch_bounds__(1024)
+k_decode_finish(const unsigned char* __restrict__ wire, uint64_t wire_len, Geo g,
+                const unsigned char* __restrict__ dst, uint32_t* __restrict__ dst_crc, Ws ws,
+                const Tables* __restrict__ tab, wm_result* result, const __grid_constant__ ChunkPowers cp, uint32_t strict)
+{
+    __shared__ uint32_t sHT[1024];
+    __shared__ uint32_t sT0[256];
+    __shared__ FinishStage stage;
+    __shared__ uint32_t s_acc;
+    __shared__ bool s_last;
+    __shared__ int s_status;
+    load_ht_t0(sHT, sT0, tab);
+    grid_dep_wait();
+    if (ld_volatile_u32(&ws.ctrl->gate)) return;
+    const uint32_t c0 = blockIdx.x * g.finish_cb;
+    stage_chunk_digests(g, stage, ws.dig, c0);
+    const unsigned char* dir = wire + 64;
+    const uint32_t c = c0 + threadIdx.x;
+    const bool step4_failed = ld_volatile_u32(reinterpret_cast<const uint32_t*>(&ws.ctrl->bad4_key)) != 0xFFFFFFFFu ||
+                              ld_volatile_u32(reinterpret_cast<const uint32_t*>(&ws.ctrl->bad4_key) + 1) != 0xFFFFFFFFu;
+    uint32_t term = 0;
+    if (threadIdx.x < g.finish_cb && c < g.n_chunks) {
+        const uint32_t fl = ws.cflag[c];
+        const uint32_t want = *reinterpret_cast<const uint32_t*>(dir + 16ull * c + 12);
+        if (step4_failed) {
+            if (fl & CF_BAD4) { atomicMin(&ws.ctrl->bad4_first, c); atomicAdd(&ws.ctrl->bad4_count, 1u); }
+        } else if (fl & CF_PRESENT) {
+            // (a chunk shorter than four bytes is checksummed byte by byte: from dst, or, in a strict
+            // call, where nothing has been stored yet, from its raw copy in the wire image)
+            const unsigned char* tiny = chunk_first_byte(g, ws, dst, c);
+            if (strict && chunk_len_dev(g, c) < 4)
+                tiny = wire + g.meta_end + *reinterpret_cast<const unsigned long long*>(dir + 16ull * c);
+            const uint32_t got = chunk_crc_staged(g, sHT, sT0, stage, ws.dig, tiny, c, threadIdx.x);
+            if (got != want) { atomicMin(&ws.ctrl->bad5_first, c); atomicAdd(&ws.ctrl->bad5_count, 1u); }
+        } else {
+            if (dst_crc[c] != want) { atomicMin(&ws.ctrl->bad6_first, c); atomicAdd(&ws.ctrl->bad6_count, 1u); }
+        }
+        term = cache_crc_term(g, cp, want, c);
+    }
+    accumulate_cache_crc(ws.ctrl, term, &s_acc);
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        __threadfence();
+        s_last = atomicAdd(&ws.ctrl->done_a, 1u) == gridDim.x - 1;
+    }
+    __syncthreads();
+    if (!s_last) return;
+    __threadfence();
+    if (threadIdx.x == 0) {
+        const uint32_t cache_crc = ld_volatile_u32(&ws.ctrl->cache_acc);
+        int status = WM_OK;
+        uint32_t first = 0, count = 0;
+        const unsigned long long key = *reinterpret_cast<volatile unsigned long long*>(&ws.ctrl->bad4_key);
+        const uint32_t err = ld_volatile_u32(&ws.ctrl->err);
+        if (err) {                     // the kernels themselves failed: nothing can be said about the image
+            status = (err & 4u) ? WM_ERR_CUDA : WM_ERR_TIMEOUT;
+        } else if (key != ~0ull) {
+            status = (key & 1ull) ? WM_ERR_STRUCT : WM_ERR_DESC;
+            first = ld_volatile_u32(&ws.ctrl->bad4_first); count = ld_volatile_u32(&ws.ctrl->bad4_count);
+        } else if (ld_volatile_u32(&ws.ctrl->bad5_count)) {
+            status = WM_ERR_CHUNK_CRC;
+            first = ld_volatile_u32(&ws.ctrl->bad5_first); count = ld_volatile_u32(&ws.ctrl->bad5_count);
+        } else if (ld_volatile_u32(&ws.ctrl->bad6_count)) {
+            status = WM_ERR_STALE;
+            first = ld_volatile_u32(&ws.ctrl->bad6_first); count = ld_volatile_u32(&ws.ctrl->bad6_count);
+        } else if (cache_crc != ws.ctrl->hdr_cache_crc) {
+            status = WM_ERR_CACHE_CRC;
+        }
+        fill_result(result, ws.ctrl, wire_len, status, first, count);
+        s_status = status;
+        if (strict) {                  // the storing pass follows: it starts from ticket 0 and stays out after a failure
+            ws.ctrl->ticket = 0;
+            if (status != WM_OK) ws.ctrl->gate = (uint32_t)status;
+        }
+    }
+    __syncthreads();
+    if (s_status == WM_OK) {
+        for (uint32_t i = threadIdx.x; i < g.n_chunks; i += blockDim.x)
+            if (ws.cflag[i] & CF_PRESENT) dst_crc[i] = *reinterpret_cast<const uint32_t*>(dir + 16ull * i + 12);
+    }
+}
+
+}  // namespace wm
