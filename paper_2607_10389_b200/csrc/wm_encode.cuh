@@ -320,9 +320,9 @@ __device__ __forceinline__ uint32_t ent_parse_value(uint32_t buf, uint32_t s, ui
 // tile, so it runs at the pace of the warp that has the most to do.
 // Template switches: MASKED (a dirty mask was given), LEAVES (the cache is a table of tensors;
 // tickets are claimed one step further ahead so that a tile's address can be looked up on the
-// way), ZEROS (the zero-tile option), ENT (the entropy option: the measuring step adds up codeword
-// lengths instead of taking exponent ranges, the packing step writes the share's interleaved
-// stream of halfwords instead of bit planes).
+// way), ZEROS (the zero / constant tile option), ENT (the entropy option: the measuring step also
+// adds up codeword lengths, the tile takes the shorter of the two coded forms, and for the ENT
+// form the packing step writes the share's interleaved stream of halfwords instead of bit planes).
 // Packed data goes from registers to the wire image directly: in every region of a PACK tile
 // a lane owns an aligned unit at a lane-strided place, so each warp store is one contiguous
 // sector-aligned run.  Claiming a tile before the previous offset is known means that, if the
