@@ -125,7 +125,7 @@ def oracle_step(sample_cur, sample_prev, chunk_bytes):
     return int(dirty.sum())
 
 
-def cpu_baseline(cur_host, prev_host, chunk_bytes, target_s=10.0):
+def cpu_baseline(cur_host, prev_host, chunk_bytes, target_s=20.0):
     """Time the oracle, as it stands, on a bounded sample of the workload: once on one core, then
     on every core the process may use (one independent slice of the sample per thread: chunks are
     independent, and the oracle's C code runs outside the interpreter lock)."""
