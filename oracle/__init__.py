@@ -10,6 +10,7 @@ from .wm_oracle import (  # noqa: F401
     build,
     checksum,
     checksum_poly,
+    checksum_xxh64,
     crc32c,
     crc_bitwise,
     crc_combine,
@@ -25,5 +26,6 @@ from .wm_oracle import (  # noqa: F401
     num_chunks,
     num_tiles,
     wire_bound,
+    xxh64,
     STATUS,
 )

@@ -210,6 +210,57 @@ static uint32_t get16(const uint8_t* p) { return (uint32_t)p[0] | ((uint32_t)p[1
 static uint32_t get32(const uint8_t* p) { uint32_t v = 0; for (int i = 0; i < 4; i++) v |= (uint32_t)p[i] << (8 * i); return v; }
 static uint64_t get64(const uint8_t* p) { uint64_t v = 0; for (int i = 0; i < 8; i++) v |= (uint64_t)p[i] << (8 * i); return v; }
 
+/* ---------------------------------------------------------------- XXH64 ---
+ * The 64-bit xxHash of a byte string (the published algorithm, all arithmetic modulo 2^64,
+ * input read little-endian), as an alternative chunk checksum.  Four accumulators take the
+ * input in 32-byte stripes, lane k getting bytes [8k, 8k+8) of every stripe; they are merged,
+ * the length is added, the tail goes in 8, 4 and 1 bytes at a time, and an avalanche ends it.
+ */
+#define XP1 0x9E3779B185EBCA87ull
+#define XP2 0xC2B2AE3D27D4EB4Full
+#define XP3 0x165667B19E3779F9ull
+#define XP4 0x85EBCA77C2B2AE63ull
+#define XP5 0x27D4EB2F165667C5ull
+
+static uint64_t xrotl(uint64_t v, int r) { return (v << r) | (v >> (64 - r)); }
+static uint64_t xround(uint64_t acc, uint64_t in) { return xrotl(acc + in * XP2, 31) * XP1; }
+static uint64_t xmerge(uint64_t h, uint64_t v) { return (h ^ xround(0, v)) * XP1 + XP4; }
+
+uint64_t wmo_xxh64(const uint8_t* p, uint64_t n, uint64_t seed)
+{
+    const uint8_t* end = p + n;
+    uint64_t h;
+    if (n >= 32) {
+        uint64_t v1 = seed + XP1 + XP2, v2 = seed + XP2, v3 = seed, v4 = seed - XP1;
+        while ((uint64_t)(end - p) >= 32) {
+            v1 = xround(v1, get64(p));
+            v2 = xround(v2, get64(p + 8));
+            v3 = xround(v3, get64(p + 16));
+            v4 = xround(v4, get64(p + 24));
+            p += 32;
+        }
+        h = xrotl(v1, 1) + xrotl(v2, 7) + xrotl(v3, 12) + xrotl(v4, 18);
+        h = xmerge(h, v1); h = xmerge(h, v2); h = xmerge(h, v3); h = xmerge(h, v4);
+    } else {
+        h = seed + XP5;
+    }
+    h += n;
+    while ((uint64_t)(end - p) >= 8) { h = xrotl(h ^ xround(0, get64(p)), 27) * XP1 + XP4; p += 8; }
+    if ((uint64_t)(end - p) >= 4) { h = xrotl(h ^ ((uint64_t)get32(p) * XP1), 23) * XP2 + XP3; p += 4; }
+    while (p < end) { h = xrotl(h ^ ((uint64_t)*p * XP5), 11) * XP1; p++; }
+    h ^= h >> 33; h *= XP2; h ^= h >> 29; h *= XP3; h ^= h >> 32;
+    return h;
+}
+
+/* XXH64 of every chunk, as wmo_checksum does for the CRC. */
+int wmo_checksum_xxh64(const uint8_t* cache, uint64_t nbytes, uint32_t chunk_bytes, uint64_t seed, uint64_t* out)
+{
+    if (!cache || !out || !args_ok(nbytes, chunk_bytes)) return WMO_ERR_ARG;
+    uint64_t nc = wmo_num_chunks(nbytes, chunk_bytes);
+    for (uint64_t c = 0; c < nc; c++) out[c] = wmo_xxh64(cache + c * chunk_bytes, chunk_len(nbytes, chunk_bytes, c), seed);
+    return WMO_OK;
+}
+
 /* Position of element e (0..255, memory order) inside its group's coded order.
  * The group's 512 bytes are four rows of 128 bytes; element e sits in row
  * r = e / 64 at 32-bit word l = (e % 64) / 2, half h = e % 2.  Coded order takes

@@ -79,6 +79,10 @@ def _load():
         getattr(lib, name).argtypes = [u64, u32]
     lib.wmo_num_tiles.restype = u64
     lib.wmo_num_tiles.argtypes = [u64]
+    lib.wmo_xxh64.restype = ctypes.c_uint64
+    lib.wmo_xxh64.argtypes = [u8p, u64, u64]
+    lib.wmo_checksum_xxh64.restype = ctypes.c_int
+    lib.wmo_checksum_xxh64.argtypes = [u8p, u64, u32, u64, ctypes.c_void_p]
     lib.wmo_checksum.restype = ctypes.c_int
     lib.wmo_checksum.argtypes = [u8p, u64, u32, u32p]
     lib.wmo_dirty_diff.restype = ctypes.c_int
@@ -96,6 +100,8 @@ def _load():
 
 
 def _bytes_view(a) -> np.ndarray:
+    if isinstance(a, (bytes, bytearray, memoryview)):
+        return np.frombuffer(bytes(a), dtype=np.uint8)
     a = np.ascontiguousarray(a)
     return a.view(np.uint8).reshape(-1)
 
@@ -179,6 +185,20 @@ def checksum(cache, chunk_bytes: int) -> np.ndarray:
     b = _bytes_view(cache)
     out = np.zeros(num_chunks(b.size, chunk_bytes), dtype=np.uint32)
     _check(_load().wmo_checksum(_ptr(b), b.size, chunk_bytes, _ptr(out)), "checksum")
+    return out
+
+
+def xxh64(data, seed: int = 0) -> int:
+    """XXH64 of a byte string (the published algorithm, written out in the C file)."""
+    b = _bytes_view(data)
+    return int(_load().wmo_xxh64(_ptr(b), b.size, seed & 0xFFFFFFFFFFFFFFFF))
+
+
+def checksum_xxh64(cache, chunk_bytes: int, seed: int = 0) -> np.ndarray:
+    """XXH64 of every chunk (u64[n_chunks])."""
+    b = _bytes_view(cache)
+    out = np.zeros(num_chunks(b.size, chunk_bytes), dtype=np.uint64)
+    _check(_load().wmo_checksum_xxh64(_ptr(b), b.size, chunk_bytes, seed & 0xFFFFFFFFFFFFFFFF, out.ctypes.data), "checksum_xxh64")
     return out
 
 
