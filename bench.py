@@ -659,6 +659,21 @@ def main():
     zm = a.elapsed_time(b) / reps
     per_call["checksum_zlib_polynomial"] = {"call_ms": zm, "reps": reps,
                                             "call_frac_of_hbm_peak": (N + 4 * nc) / (zm * 1e-3) / 1e9 / peak}
+    # XXH64 of every chunk (a serial chain per chunk: four threads of work each)
+    h64 = torch.zeros(nc, dtype=torch.int64, device=dev)
+    for _ in range(3):
+        wm.wm_checksum_xxh64(cur, C, 0, h64)
+    torch.cuda.synchronize()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()
+    for _ in range(reps):
+        wm.wm_checksum_xxh64(cur, C, 0, h64)
+    b.record()
+    torch.cuda.synchronize()
+    xm = a.elapsed_time(b) / reps
+    per_call["checksum_xxh64"] = {"call_ms": xm, "reps": reps, "call_frac_of_hbm_peak": N / (xm * 1e-3) / 1e9 / peak,
+                                  "note": "bound by the latency of XXH64's serial chain (two dependent 64-bit "
+                                          "multiplications per 8 bytes, four chains per chunk), not by memory"}
     # dirty diff: bytes it actually has to read (clean chunks in full on both sides)
     per_call["dirty_diff"]["note"] = f"{n_rewritten} of {nc} chunks dirty; clean chunks are read in full on both sides"
 

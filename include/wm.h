@@ -102,6 +102,20 @@ wm_status wm_checksum_poly(const void* cache, uint64_t nbytes, uint32_t chunk_by
                            uint32_t* crc_out, void* workspace, uint64_t workspace_bytes, void* stream);
 
 /*
+ * wm_checksum_xxh64 - the 64-bit xxHash (XXH64) of every chunk, a checksum option beside the CRC.
+ * Paper: the verification plane fingerprints chunks (Section 6.5); a non-cryptographic 64-bit hash
+ * is the usual alternative where 32 bits are felt to be too few.  The values are those of the
+ * published algorithm (seed 0, empty input: 0xEF46DB3751D8E999; "123456789": 0x8CB841DB40E6AE83).
+ *   cache     [dev] nbytes bytes, 16-byte aligned, read only
+ *   seed      the hash's seed, the same for every chunk
+ *   hash_out  [dev] u64[n_chunks]; hash_out[c] = XXH64(cache[c*chunk_bytes, min((c+1)*chunk_bytes, nbytes)), seed)
+ * No workspace.  Unlike a CRC, hashes of pieces cannot be combined, so there is no whole-cache
+ * value and wm_encode / wm_decode_verify do not use this hash.  WM_ERR_ARG on a bad geometry.
+ */
+wm_status wm_checksum_xxh64(const void* cache, uint64_t nbytes, uint32_t chunk_bytes, uint64_t seed,
+                            uint64_t* hash_out, void* stream);
+
+/*
  * wm_dirty_diff - which chunks changed since the previous snapshot.
  * Paper: live pre-copy (Appendix G: round 0 ships every chunk, each later round the dirty
  * ones) and the measured dirty fraction per generation step (Section 3.3).  The compare is

@@ -24,7 +24,7 @@ RESULT_BYTES = 40
 EXPORTS = ("wm_num_chunks", "wm_num_tiles", "wm_meta_bytes", "wm_wire_bound", "wm_workspace_bytes",
            "wm_checksum", "wm_dirty_diff", "wm_encode", "wm_decode_verify", "wm_last_launch_count",
            "wm_timing_enable", "wm_timing_read_ms", "wm_checksum_noalloc", "wm_encode_leaves",
-           "wm_decode_verify_leaves", "wm_zero_tiles_enable", "wm_decode_verify_strict", "wm_checksum_poly", "wm_entropy_enable", "wm_encode_opt", "wm_decode_verify_opt")
+           "wm_decode_verify_leaves", "wm_zero_tiles_enable", "wm_decode_verify_strict", "wm_checksum_poly", "wm_entropy_enable", "wm_encode_opt", "wm_decode_verify_opt", "wm_checksum_xxh64")
 
 
 class WmError(RuntimeError):
@@ -58,6 +58,8 @@ def load_library() -> ctypes.CDLL:
     lib.wm_checksum.argtypes = [vp, u64, u32, vp, vp, u64, vp]
     lib.wm_checksum_poly.restype = ctypes.c_int
     lib.wm_checksum_poly.argtypes = [vp, u64, u32, ctypes.c_int, vp, vp, u64, vp]
+    lib.wm_checksum_xxh64.restype = ctypes.c_int
+    lib.wm_checksum_xxh64.argtypes = [vp, u64, u32, u64, vp, vp]
     lib.wm_checksum_noalloc.restype = ctypes.c_int
     lib.wm_checksum_noalloc.argtypes = [vp, u64, u32, vp, vp]
     lib.wm_dirty_diff.restype = ctypes.c_int
@@ -211,6 +213,14 @@ def wm_checksum_poly(cache: torch.Tensor, chunk_bytes: int, polynomial: int, crc
     nbytes = cache.numel() * cache.element_size()
     _check(lib().wm_checksum_poly(cache.data_ptr(), nbytes, chunk_bytes, int(polynomial), crc_out.data_ptr(),
                                   workspace.data_ptr(), workspace.numel(), _stream(stream)), "wm_checksum_poly")
+
+
+def wm_checksum_xxh64(cache: torch.Tensor, chunk_bytes: int, seed: int, hash_out: torch.Tensor, stream=None) -> None:
+    """XXH64 of every chunk into an int64 / uint64 tensor of n_chunks entries."""
+    _dev_u8(cache, "cache")
+    nbytes = cache.numel() * cache.element_size()
+    _check(lib().wm_checksum_xxh64(cache.data_ptr(), nbytes, chunk_bytes, int(seed) & 0xFFFFFFFFFFFFFFFF, hash_out.data_ptr(),
+                                   _stream(stream)), "wm_checksum_xxh64")
 
 
 NOALLOC_MAX_BYTES = 4 << 30

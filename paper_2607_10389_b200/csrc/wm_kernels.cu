@@ -26,6 +26,7 @@
 #include "wm_encode.cuh"
 #include "wm_meta.cuh"
 #include "wm_decode.cuh"
+#include "wm_xxh64.cuh"
 
 namespace wm {
 
@@ -247,6 +248,21 @@ wm_status wm_checksum_poly(const void* cache, uint64_t nbytes, uint32_t chunk_by
     }
     launch_after(k_checksum_finish, (g.n_chunks + g.finish_cb - 1) / g.finish_cb, 1024, 0, s, c, g, ws, tab, crc_out);
     g_launches = 2;
+    return launch_status();
+}
+
+// XXH64 of every chunk: one kernel, no workspace, no tables.
+wm_status wm_checksum_xxh64(const void* cache, uint64_t nbytes, uint32_t chunk_bytes, uint64_t seed, uint64_t* hash_out,
+                            void* stream)
+{
+    Geo g;
+    if (!cache || !hash_out || !make_geo(nbytes, chunk_bytes, g) || !aligned16(cache)) return WM_ERR_ARG;
+    if (!device_state()) return WM_ERR_CUDA;
+    const uint32_t threads = 4u * g.n_chunks;
+    k_xxh64<<<(threads + 31u) / 32u, 32, 0, static_cast<cudaStream_t>(stream)>>>(
+        static_cast<const unsigned char*>(cache), nbytes, chunk_bytes, g.n_chunks, seed,
+        reinterpret_cast<unsigned long long*>(hash_out));
+    g_launches = 1;
     return launch_status();
 }
 
