@@ -6,8 +6,10 @@
 // (digests of pieces cannot be combined, unlike a CRC).  So a chunk offers four threads of work
 // and the parallelism is across chunks: thread 4c + k owns accumulator k of chunk c, a warp
 // holds eight chunks, and one warp load fetches eight full 32-byte sectors.  What bounds the
-// kernel is the latency of that chain (two dependent 64-bit multiplications per 8 bytes), so the
-// loads run two batches of 32 stripes ahead of it, in registers.
+// kernel with large chunks is the latency of that chain, so the loads run two batches of 32
+// stripes ahead of it, in registers, and the product in * P2 is taken as a value arrives (off
+// the chain: only the add, the rotate and the multiplication by P1 depend on the accumulator).
+// With many small chunks (64 KiB) there are enough chains and the kernel runs at the memory rate.
 #pragma once
 
 namespace wm {
@@ -49,19 +51,19 @@ k_xxh64(const unsigned char* __restrict__ cache, uint64_t nbytes, uint32_t chunk
     uint64_t s = 0;
     if (stripes >= (uint64_t)kXBatch) {
 #pragma unroll
-        for (int i = 0; i < kXBatch; i++) a[i] = __ldcs(p + 4u * i);
+        for (int i = 0; i < kXBatch; i++) a[i] = __ldcs(p + 4u * i) * kXP2;
         // two batches per turn: while one is folded into the accumulator the other is on its way
         while (s + 2u * kXBatch <= stripes) {
 #pragma unroll
-            for (int i = 0; i < kXBatch; i++) b[i] = __ldcs(p + 4u * (s + kXBatch + i));
+            for (int i = 0; i < kXBatch; i++) b[i] = __ldcs(p + 4u * (s + kXBatch + i)) * kXP2;
 #pragma unroll
-            for (int i = 0; i < kXBatch; i++) v = x_round(v, a[i]);
+            for (int i = 0; i < kXBatch; i++) v = x_rotl(v + a[i], 31) * kXP1;
             s += kXBatch;
             if (s + 2u * kXBatch <= stripes) {
 #pragma unroll
-                for (int i = 0; i < kXBatch; i++) a[i] = __ldcs(p + 4u * (s + kXBatch + i));
+                for (int i = 0; i < kXBatch; i++) a[i] = __ldcs(p + 4u * (s + kXBatch + i)) * kXP2;
 #pragma unroll
-                for (int i = 0; i < kXBatch; i++) v = x_round(v, b[i]);
+                for (int i = 0; i < kXBatch; i++) v = x_rotl(v + b[i], 31) * kXP1;
                 s += kXBatch;
             } else {
 #pragma unroll
@@ -70,7 +72,7 @@ k_xxh64(const unsigned char* __restrict__ cache, uint64_t nbytes, uint32_t chunk
         }
         // a[] holds the batch that starts at s
 #pragma unroll
-        for (int i = 0; i < kXBatch; i++) v = x_round(v, a[i]);
+        for (int i = 0; i < kXBatch; i++) v = x_rotl(v + a[i], 31) * kXP1;
         s += kXBatch;
     }
     for (; s < stripes; s++) v = x_round(v, __ldcs(p + 4u * s));
