@@ -11,6 +11,7 @@
 #include <cstdint>
 #include <cstdio>
 #include <cstring>
+#include <atomic>
 #include <mutex>
 
 #include <cuda_runtime.h>
@@ -48,19 +49,22 @@ struct DeviceState {
     bool ready = false;
     cudaEvent_t ev[4][2] = {};   // optional timing of the four main kernels
 };
-static bool g_timing = false;
-static bool g_zero_tiles = false;   // wm_zero_tiles_enable
-static bool g_entropy = false;      // wm_entropy_enable
+// Process-wide switches: read by calls on any thread, so they are atomics (a call sees the value at
+// the moment it is issued; calls that must not depend on them take their options as an argument).
+static std::atomic<bool> g_timing{false};
+static std::atomic<bool> g_zero_tiles{false};   // wm_zero_tiles_enable
+static std::atomic<bool> g_entropy{false};      // wm_entropy_enable
 
 struct MainKernelTimer {        // records events around a main kernel when timing is enabled
-    const DeviceState* ds; int kind; cudaStream_t s;
+    const DeviceState* ds; int kind; cudaStream_t s; bool on;
     MainKernelTimer(const DeviceState* d, int k, cudaStream_t st) : ds(d), kind(k), s(st)
     {
-        if (g_timing) cudaEventRecord(ds->ev[kind][0], s);
+        on = g_timing.load(std::memory_order_relaxed);
+        if (on) cudaEventRecord(ds->ev[kind][0], s);
     }
     ~MainKernelTimer()
     {
-        if (g_timing) cudaEventRecord(ds->ev[kind][1], s);
+        if (on) cudaEventRecord(ds->ev[kind][1], s);
     }
 };
 static DeviceState g_dev[64];
