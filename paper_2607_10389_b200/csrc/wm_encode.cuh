@@ -362,10 +362,10 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
     __shared__ uint32_t s_scanner;
     __shared__ uint32_t s_tmem;
     __shared__ uint32_t s_ent[16];     // ENT: codeword | length << 16 by slot (one bank each: no conflicts)
-    __shared__ uint32_t s_len[16];     // ENT: length by slot
+    __shared__ unsigned char s_len8[16];   // ENT: length by slot (bytes: the index needs no scaling)
     if (ENT && threadIdx.x < 11u) {
         s_ent[threadIdx.x] = (threadIdx.x == 10u ? 0xFFFFu : ent_word(threadIdx.x, 0u)) | (ent_length(threadIdx.x) << 16);
-        s_len[threadIdx.x] = ent_length(threadIdx.x);
+        s_len8[threadIdx.x] = (unsigned char)ent_length(threadIdx.x);
     }
     Smem S = setup_smem(smem, tab);
     grid_dep_wait();                   // from here on the control block and the length table are ready
@@ -502,12 +502,12 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
                 // word) and the halfwords its 32 strands need
                 uint32_t acc = 0;
 #pragma unroll
-                for (int i = 0; i < 16; i++) acc += (d[i] >> 8) & 0x00FF00FFu;
-                const uint32_t anchor = (__reduce_add_sync(0xFFFFFFFFu, (acc & 0xFFFFu) + (acc >> 16)) + 512u) >> 10;
+                for (int i = 0; i < 16; i++) acc = __dp4a(d[i], 0x01000100u, acc);       // bytes 1 and 3
+                const uint32_t anchor = (__reduce_add_sync(0xFFFFFFFFu, acc) + 512u) >> 10;
                 uint32_t bits = 0;
 #pragma unroll
                 for (int i = 0; i < 16; i++)
-                    bits += s_len[ent_slot(__byte_perm(d[i], 0u, 0x4441), anchor)] + s_len[ent_slot(d[i] >> 24, anchor)];
+                    bits += s_len8[ent_slot(__byte_perm(d[i], 0u, 0x4441), anchor)] + s_len8[ent_slot(d[i] >> 24, anchor)];
                 const uint32_t count = __reduce_add_sync(0xFFFFFFFFu, (bits + 15u) >> 4);
                 ent_w = anchor | (count << 8);
             }
