@@ -12,8 +12,8 @@ __global__ void k_diff_init(Ws ws)
     if (threadIdx.x == 0 && blockIdx.x == 0) { ws.ctrl->ticket = 0; ws.ctrl->n_present = 0; }
 }
 
-// One block per chunk at a time (ticketed); the chunk is scanned in 32 KiB steps and dropped
-// at the first step that shows a difference.
+// One block per chunk at a time (ticketed); the chunk is scanned in 16 KiB half-steps, two of
+// them in flight, and dropped at the first one that shows a difference.
 __global__ void __launch_bounds__(256)
 k_diff(const unsigned char* __restrict__ cache, const unsigned char* __restrict__ prev, Geo g, Ws ws,
        uint8_t* __restrict__ dirty_out)
@@ -32,23 +32,36 @@ k_diff(const unsigned char* __restrict__ cache, const unsigned char* __restrict_
         const uint64_t clen = chunk_len_dev(g, c);
         const uint64_t vec_len = clen & ~(uint64_t)15;
         int any = 0;
-        for (uint64_t o = 0; o < vec_len; o += kStep) {
-            uint4 a[8], b[8];
+        // two half-steps in flight: the loads of the next one are issued before this one is judged,
+        // so the block-wide vote never finds the memory pipe empty
+        uint4 a[2][4], b[2][4];
+        auto fetch = [&](uint64_t o, int slot) {
 #pragma unroll
-            for (int k = 0; k < 8; k++) {
-                uint64_t p = o + ((uint64_t)k * 256 + threadIdx.x) * 16;
+            for (int k = 0; k < 4; k++) {
+                const uint64_t p = o + ((uint64_t)k * 256 + threadIdx.x) * 16;
                 if (p < vec_len) {
-                    a[k] = __ldcs(reinterpret_cast<const uint4*>(cache + base + p));
-                    b[k] = __ldcs(reinterpret_cast<const uint4*>(prev + base + p));
+                    a[slot][k] = __ldcs(reinterpret_cast<const uint4*>(cache + base + p));
+                    b[slot][k] = __ldcs(reinterpret_cast<const uint4*>(prev + base + p));
                 } else {
-                    a[k] = make_uint4(0, 0, 0, 0); b[k] = a[k];
+                    a[slot][k] = make_uint4(0, 0, 0, 0); b[slot][k] = a[slot][k];
                 }
             }
+        };
+        auto differs = [&](int slot) {
             uint32_t d = 0;
 #pragma unroll
-            for (int k = 0; k < 8; k++)
-                d |= (a[k].x ^ b[k].x) | (a[k].y ^ b[k].y) | (a[k].z ^ b[k].z) | (a[k].w ^ b[k].w);
-            any = __syncthreads_or(d != 0);
+            for (int k = 0; k < 4; k++)
+                d |= (a[slot][k].x ^ b[slot][k].x) | (a[slot][k].y ^ b[slot][k].y) | (a[slot][k].z ^ b[slot][k].z) | (a[slot][k].w ^ b[slot][k].w);
+            return d != 0;
+        };
+        constexpr uint32_t kHalf = kStep / 2;
+        if (vec_len) fetch(0, 0);
+        for (uint64_t o = 0; o < vec_len; o += 2 * kHalf) {
+            if (o + kHalf < vec_len) fetch(o + kHalf, 1);
+            any = __syncthreads_or(differs(0));
+            if (any || o + kHalf >= vec_len) break;
+            if (o + 2 * kHalf < vec_len) fetch(o + 2 * kHalf, 0);
+            any = __syncthreads_or(differs(1));
             if (any) break;
         }
         if (!any && vec_len < clen) {             // ragged tail of the last chunk, < 16 bytes
