@@ -726,7 +726,7 @@ def main():
     # leaf mode: the same cache held as one key and one value tensor per layer, encoded and
     # decoded in place, beside the flatten and rehydrate copies that this makes unnecessary
     leaf = None
-    if not args.no_loop and cfg.kind == "kv":
+    if not args.no_loop and cfg.kind in ("kv", "llm"):
         leaf = leaf_mode(wm, cfg, cur, wire, ws, dev, W, peak)
 
     # the entropy-coded exponent option beside the default format
