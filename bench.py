@@ -578,34 +578,6 @@ def main():
     gpu_launches = launches["n"]
     value = group.aggregate_gbs(N, ms_step)
 
-    # the same step captured once in a CUDA graph and replayed (the calls never allocate or
-    # synchronise): what is left of the host's launch work, which matters for small caches
-    graph_ms = None
-    if not args.profile:
-        try:
-            gs = torch.cuda.Stream()
-            with torch.cuda.stream(gs):
-                torch.cuda.synchronize()
-                graph = torch.cuda.CUDAGraph()
-                with torch.cuda.graph(graph, stream=gs):
-                    step()
-            for _ in range(3):
-                graph.replay()
-            torch.cuda.synchronize()
-            ga, gb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            ga.record()
-            for _ in range(min(args.steps, 50)):
-                graph.replay()
-            gb.record()
-            torch.cuda.synchronize()
-            graph_ms = ga.elapsed_time(gb) / min(args.steps, 50)
-            if not wm.read_result(res_d).ok:
-                raise SystemExit("graph replay: decode failed")
-            del graph
-        except RuntimeError as e:      # capture is an extra: report why it was not measured
-            graph_ms = None
-            print("graph replay not measured:", e, file=sys.stderr)
-    launches["n"] = gpu_launches
 
     if args.profile:
         if rank == 0:
@@ -803,6 +775,34 @@ def main():
         e2e = {"value": group.aggregate_gbs(N, e_ms), "unit": "GB/s", "h2d_bytes_per_step": N,
                "d2h_bytes_per_step": W + 80, "steps": e_steps, "ms_per_step": e_ms,
                "note": "two buffer sets, two streams: step k's copy-out overlaps step k+1's copy-in and compute"}
+
+    # the same step captured once in a CUDA graph and replayed (the calls never allocate or
+    # synchronise): what is left of the host's launch work, which matters for small caches
+    graph_ms = None
+    try:
+        gs = torch.cuda.Stream()
+        with torch.cuda.stream(gs):
+            torch.cuda.synchronize()
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=gs):
+                step()
+        for _ in range(3):
+            graph.replay()
+        torch.cuda.synchronize()
+        ga, gb = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        ga.record()
+        for _ in range(min(args.steps, 50)):
+            graph.replay()
+        gb.record()
+        torch.cuda.synchronize()
+        graph_ms = ga.elapsed_time(gb) / min(args.steps, 50)
+        if not wm.read_result(res_d).ok:
+            raise SystemExit("graph replay: decode failed")
+        del graph
+    except RuntimeError as e:      # capture is an extra: report why it was not measured
+        graph_ms = None
+        print("graph replay not measured:", e, file=sys.stderr)
+    launches["n"] = gpu_launches
 
     base = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
