@@ -289,3 +289,48 @@ def test_the_option_never_makes_an_image_longer():
         ea, eb = a_[64 + 48: 64 + 48 + 6].view("<u2"), b_[64 + 48: 64 + 48 + 6].view("<u2")
         la = np.where(ea & 0x8000, 32 * (ea & 0x7FFF).astype(np.int64), 32 * ea.astype(np.int64))
         assert (la <= 32 * eb.astype(np.int64)).all() and ra.wire_len <= rb.wire_len
+
+
+def _golden():
+    import os
+    ex = {}
+    for line in open(os.path.join(os.path.dirname(__file__), "golden", "ent_worked_examples.txt")):
+        if line.startswith("#") or not line.strip():
+            continue
+        name, key, *rest = line.split()
+        ex.setdefault(name, {}).setdefault(key, []).append(rest)
+    return ex
+
+
+def test_golden_worked_examples():
+    """The fixtures were written down from the format statement before looking at the coder's output."""
+    ex = _golden()
+    for name, spec in ex.items():
+        v = _tile_of(0x3F80)
+        if name == "one_odd":
+            e = spec["element"][0]
+            v[int(e[0])] = int(e[2], 16)
+        if name == "escapes":
+            for i in range(32):
+                v[64 * (i // 2) + i % 2] = 147 << 7
+        wire, flags, entry, t = _encode_one_tile(v)
+        if "anchors" in spec:
+            assert list(t[0:8]) == [int(x) for x in spec["anchors"][0]], name
+        if "counts" in spec:
+            assert list(t[8:24].view("<u2")) == [int(x) for x in spec["counts"][0]], name
+        if "entry" in spec:
+            assert entry == int(spec["entry"][0][0], 16), name
+        for sh in spec.get("share", []):
+            share = int(sh[0])
+            counts = t[8:24].view("<u2")
+            start = int(counts[:share].sum())
+            stream = t[8256 + 2 * start: 8256 + 2 * (start + int(counts[share]))].view("<u2")
+            seen = np.zeros(stream.size, dtype=bool)
+            for item in sh[2:]:
+                rng_, val = item.split(":")
+                lo, hi = (rng_.split("-") + [rng_])[:2]
+                for i in range(int(lo), int(hi) + 1):
+                    assert int(stream[i]) == int(val, 16), (name, i)
+                    seen[i] = True
+            if name != "escapes":
+                assert not stream[~seen].any(), name
