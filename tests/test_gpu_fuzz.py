@@ -90,3 +90,51 @@ def test_random_case_matches_the_oracle(seed):
     finally:
         wm.zero_tiles_enable(False)
         wm.entropy_enable(False)
+
+
+@pytest.mark.parametrize("seed", range(16))
+def test_random_leaf_tables_match_the_flat_image(seed):
+    """The cache cut into leaves at random tile boundaries (the last leaf may be ragged), every
+    option set, with and without a mask: the image is the oracle's image of the concatenation and
+    the decode lands in a second, differently cut set of leaves."""
+    import torch
+    from paper_2607_10389_b200 import binding as wm
+    rng = np.random.default_rng(3000 + seed)
+    chunk = int(rng.choice([1, 2, 4])) * TILE
+    nt = int(rng.integers(3, 48))
+    n = nt * TILE + int(rng.integers(0, 2)) * int(rng.integers(1, TILE))
+    a = _data(rng, n)
+    opt = seed % 4
+    nc = oracle.num_chunks(n, chunk)
+    dirty = (rng.integers(0, 3, nc) > 0).astype(np.uint8) if seed % 2 else None
+    stale = oracle.checksum(a, chunk)
+    want, want_crc, want_res = oracle.encode(a, chunk, dirty=dirty, crc_in=stale, zero_tiles=bool(opt & 1), entropy=bool(opt & 2))
+
+    def cut(k):
+        edges = sorted(set(int(x) for x in rng.integers(1, nt, k))) if nt > 1 else []
+        bounds = [0] + [e * TILE for e in edges] + [n]
+        return [(bounds[i], bounds[i + 1]) for i in range(len(bounds) - 1) if bounds[i + 1] > bounds[i]]
+
+    src = [torch.from_numpy(a[lo:hi].copy()).cuda() for lo, hi in cut(int(rng.integers(1, 9)))]
+    ws = wm.new_workspace(n, chunk)
+    wire = torch.full((wm.wire_bound(n, chunk),), 0x3C, dtype=torch.uint8, device="cuda")
+    crc = torch.from_numpy(stale.view(np.int32).copy()).cuda()
+    res = wm.new_result()
+    d = None if dirty is None else torch.from_numpy(dirty).cuda()
+    wm.wm_encode_opt(None, chunk, d, crc, wire, ws, res, opt, leaf_table=wm.make_leaf_table(src), nbytes=n)
+    r = wm.read_result(res)
+    assert r.status == 0 and r.wire_len == want_res.wire_len
+    assert np.array_equal(wire[: r.wire_len].cpu().numpy(), want) and np.array_equal(crc.cpu().numpy().view(np.uint32), want_crc)
+    base = a.copy()
+    if dirty is not None:
+        for c in range(nc):
+            if dirty[c]:
+                base[c * chunk:(c + 1) * chunk] = 0x77
+    spans = cut(int(rng.integers(1, 9)))
+    dst = [torch.from_numpy(base[lo:hi].copy()).cuda() for lo, hi in spans]
+    dcrc = torch.from_numpy(stale.view(np.int32).copy()).cuda()
+    wm.wm_decode_verify_opt(wire, r.wire_len, None, chunk, dcrc, ws, res, (opt & 2) | (wm.OPT_STRICT if seed % 3 == 0 else 0),
+                            leaf_table=wm.make_leaf_table(dst), nbytes=n)
+    assert wm.read_result(res).status == 0
+    for (lo, hi), t in zip(spans, dst):
+        assert np.array_equal(t.cpu().numpy(), a[lo:hi])
