@@ -138,3 +138,54 @@ def test_random_leaf_tables_match_the_flat_image(seed):
     assert wm.read_result(res).status == 0
     for (lo, hi), t in zip(spans, dst):
         assert np.array_equal(t.cpu().numpy(), a[lo:hi])
+
+
+@pytest.mark.parametrize("seed", range(12))
+def test_buffers_at_odd_sixteen_byte_offsets(seed):
+    """The ABI asks for 16-byte alignment and nothing more: cache, previous snapshot, wire image,
+    destination and workspace each start 16, 48, 80 ... bytes into their allocations."""
+    import torch
+    from paper_2607_10389_b200 import binding as wm
+    rng = np.random.default_rng(4000 + seed)
+    chunk = int(rng.choice([1, 2, 4])) * TILE
+    n = int(rng.integers(1, 30 * TILE))
+    a = _data(rng, n)
+    b = a.copy()
+    for _ in range(int(rng.integers(0, 4))):
+        b[int(rng.integers(0, n))] ^= 0x10
+    opt = seed % 4
+    nc = oracle.num_chunks(n, chunk)
+
+    def at_offset(nbytes, fill=None):
+        off = 16 * int(rng.integers(1, 16)) | 16
+        t = torch.empty(nbytes + off + 64, dtype=torch.uint8, device="cuda")
+        v = t[off: off + nbytes]
+        assert v.data_ptr() % 16 == 0 and v.data_ptr() % 32 != 0
+        if fill is not None:
+            v.copy_(torch.from_numpy(fill))
+        return v
+
+    cur, prev = at_offset(n, a), at_offset(n, b)
+    ws = at_offset(wm.workspace_bytes(n, chunk))
+    wire = at_offset(wm.wire_bound(n, chunk))
+    dst = at_offset(n)
+    crc = torch.zeros(nc, dtype=torch.int32, device="cuda")
+    res = wm.new_result()
+    wm.wm_checksum(cur, chunk, crc, ws)
+    assert np.array_equal(crc.cpu().numpy().view(np.uint32), oracle.checksum(a, chunk))
+    dirty = torch.zeros(nc, dtype=torch.uint8, device="cuda")
+    idx = torch.zeros(nc, dtype=torch.int32, device="cuda")
+    nd = torch.zeros(1, dtype=torch.int32, device="cuda")
+    wm.wm_dirty_diff(cur, prev, chunk, dirty, idx, nd, ws)
+    want_dirty, want_idx = oracle.dirty_diff(a, b, chunk)
+    assert np.array_equal(dirty.cpu().numpy(), want_dirty) and int(nd.item()) == len(want_idx)
+    want, want_crc, want_res = oracle.encode(a, chunk, zero_tiles=bool(opt & 1), entropy=bool(opt & 2))
+    wm.wm_encode_opt(cur, chunk, None, crc, wire, ws, res, opt)
+    r = wm.read_result(res)
+    assert r.status == 0 and np.array_equal(wire[: r.wire_len].cpu().numpy(), want)
+    dcrc = torch.zeros(nc, dtype=torch.int32, device="cuda")
+    wm.wm_decode_verify_opt(wire, r.wire_len, dst, chunk, dcrc, ws, res, opt & 2)
+    assert wm.read_result(res).status == 0 and np.array_equal(dst.cpu().numpy(), a)
+    h = torch.zeros(nc, dtype=torch.int64, device="cuda")
+    wm.wm_checksum_xxh64(cur, chunk, seed, h)
+    assert np.array_equal(h.cpu().numpy().view(np.uint64), oracle.checksum_xxh64(a, chunk, seed))
