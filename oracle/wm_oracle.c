@@ -76,10 +76,12 @@ uint32_t wmo_crc_bitwise(const uint8_t* p, uint64_t n, uint32_t poly)
     return crc ^ 0xFFFFFFFFu;
 }
 
-/* Same function through the classic one-byte table (built from the bit loop). */
+/* Same function through the classic one-byte table (built from the bit loop).  The functions
+ * of this file keep no state between calls and may be called from several threads at once (the
+ * tests run chunk ranges on a thread pool); the table is the one thing shared, and it is built
+ * when the library is loaded, before any caller exists. */
 static uint32_t g_tab[256];
-static int g_tab_ready = 0;
-static void build_tab(void)
+__attribute__((constructor)) static void build_tab(void)
 {
     for (uint32_t b = 0; b < 256; b++) {
         uint32_t v = b;
@@ -87,12 +89,10 @@ static void build_tab(void)
             v = (v >> 1) ^ ((v & 1u) ? WMO_POLY_CRC32C : 0u);
         g_tab[b] = v;
     }
-    g_tab_ready = 1;
 }
 
 uint32_t wmo_crc32c(const uint8_t* p, uint64_t n)
 {
-    if (!g_tab_ready) build_tab();
     uint32_t crc = 0xFFFFFFFFu;
     for (uint64_t i = 0; i < n; i++)
         crc = g_tab[(crc ^ p[i]) & 0xFFu] ^ (crc >> 8);
@@ -380,7 +380,7 @@ static uint32_t encode_ent_tile(const uint8_t* src, uint8_t* out)
         uint32_t anchor = (sum + 512u) >> 10;
         out[s] = (uint8_t)anchor;
         /* every strand as a bit string, and the bits used up to and including codeword i */
-        static uint8_t bit[32][32 * 16 + 16];
+        uint8_t bit[32][32 * 16 + 16];
         uint32_t upto[32][32];
         memset(bit, 0, sizeof bit);
         for (uint32_t l = 0; l < 32; l++) {
@@ -489,7 +489,7 @@ static uint32_t encode_full_tile(const uint8_t* src, uint8_t* out, uint32_t* ent
      * (ENT, PACK, raw); on equal lengths PACK goes before ENT and a coded form before raw, so
      * an image with the option is never longer than one without.  (WMO_OPT_ENT_ONLY, a switch
      * of this oracle alone, leaves PACK out: the tests use it to pin the ENT coder by itself.) */
-    static uint8_t ent_buf[2 * WMO_TILE];
+    uint8_t ent_buf[2 * WMO_TILE];
     uint32_t ent_len = WMO_TILE;
     if (options & WMO_OPT_ENTROPY) {
         ent_len = encode_ent_tile(src, ent_buf);

@@ -1,16 +1,19 @@
 """Parity at the full workload sizes, in the launch configuration the benchmark times.
 
-The oracle cannot run a multi-gigabyte cache in seconds, so these tests compare what it can
-compute one by one (sampled chunks: CRC, encoded payload bytes, tile table entries; the whole
-metadata block, which is small) and properties that hold at any size (directory offsets are the
-running sum of lengths, the decoded shadow equals the cache byte for byte, a flipped bit is
-rejected and nothing is installed).
+The engine cache and the incompressible cache are compared with the oracle completely: every
+chunk's CRC, every tile table entry and every payload byte of the wire image (the oracle runs the
+chunk runs on a thread pool, see oracle_pool.py), the metadata block recomputed with the oracle's
+CRC, and the dirty mask against the oracle's byte compare.  The 16 GiB cache is compared on
+sampled chunks (the oracle would need minutes for all of it) plus properties that hold at any
+size: directory offsets are the running sum of lengths, the decoded shadow equals the cache byte
+for byte, a flipped bit is rejected and nothing is installed.
 """
 import numpy as np
 import pytest
 import torch
 
 import oracle
+import oracle_pool
 from paper_2607_10389_b200 import binding as wm
 from paper_2607_10389_b200 import inputs
 
@@ -84,13 +87,23 @@ def check_chunks_against_oracle(job, cache, chunks, off, ln, crc, tab, entropy=F
         assert np.array_equal(tab[c * tpc: c * tpc + nt1], tab1), f"chunk {c}: tile table"
 
 
-def sample_chunks(nc, k, seed):
-    rng = np.random.default_rng(seed)
-    s = {0, 1, nc - 2, nc - 1} | set(int(x) for x in rng.integers(0, nc, k))
-    return sorted(c for c in s if 0 <= c < nc)
+def check_whole_image_against_oracle(job, cache, off, ln, crc, tab, present=None, **options):
+    """Every present chunk of the image, byte for byte: CRC, encoded length, tile table entries and
+    payload against the oracle's encoding of the same bytes; absent chunks have no tiles and no bytes."""
+    host = cache.cpu().numpy()
+    wire = job.wire.cpu().numpy()
+    ocrc, olen, otab, opay = oracle_pool.encode_runs(host, job.chunk, present=present, **options)
+    on = np.ones(job.nc, bool) if present is None else np.asarray(present).astype(bool)
+    assert np.array_equal(tab, otab), "tile table"
+    assert np.array_equal(ln, olen), "encoded lengths"
+    assert np.array_equal(crc[on], ocrc[on]), "chunk CRCs"
+    bad = [c for c in np.nonzero(on)[0]
+           if not np.array_equal(wire[job.meta_end + int(off[c]): job.meta_end + int(off[c]) + int(ln[c])], opay[c])]
+    assert not bad, f"payload bytes differ in chunks {bad[:8]} ({len(bad)} in all)"
+    return ocrc
 
 
-def test_engine_cache_full_move_sampled_against_oracle():
+def test_engine_cache_full_move_whole_image_against_oracle():
     cfg = inputs.CONFIGS["engine"]
     cur = inputs.make_cache(cfg, "cuda")
     job = Job(cfg.nbytes, cfg.chunk_bytes)
@@ -107,7 +120,7 @@ def test_engine_cache_full_move_sampled_against_oracle():
     check_meta_against_oracle(job, m, hdr, off, ln, crc, present)
     assert r.wire_len == int(hdr[40:48].view(np.uint64)[0]) and r.cache_crc == int(hdr[48:52].view(np.uint32)[0])
     assert 0.70 < r.wire_len / job.n < 0.80        # the exponent plane carries the saving
-    check_chunks_against_oracle(job, cur, sample_chunks(job.nc, 10, 1), off, ln, crc, tab)
+    check_whole_image_against_oracle(job, cur, off, ln, crc, tab)
 
     shadow = torch.zeros(job.n, dtype=torch.uint8, device="cuda")
     crc_dst = torch.zeros(job.nc, dtype=torch.int32, device="cuda")
@@ -117,8 +130,8 @@ def test_engine_cache_full_move_sampled_against_oracle():
     assert torch.equal(shadow, cur) and torch.equal(crc_dst, crc_b)
 
 
-def test_engine_cache_with_entropy_coded_exponents_sampled_against_oracle():
-    """The ENT option at full size: sampled chunks byte for byte, metadata, round trip, one flipped bit."""
+def test_engine_cache_with_entropy_coded_exponents_whole_image_against_oracle():
+    """The ENT option at full size: the whole image byte for byte, metadata, round trip, one flipped bit."""
     cfg = inputs.CONFIGS["engine"]
     cur = inputs.make_cache(cfg, "cuda")
     job = Job(cfg.nbytes, cfg.chunk_bytes)
@@ -133,7 +146,7 @@ def test_engine_cache_with_entropy_coded_exponents_sampled_against_oracle():
         present = np.ones(job.nc, dtype=np.uint64)
         check_meta_against_oracle(job, m, hdr, off, ln, crc, present)
         assert 0.68 < r.wire_len / job.n < 0.72        # bit-plane packing: 0.757
-        check_chunks_against_oracle(job, cur, sample_chunks(job.nc, 6, 2), off, ln, crc, tab, entropy=True)
+        check_whole_image_against_oracle(job, cur, off, ln, crc, tab, entropy=True)
         shadow = torch.zeros(job.n, dtype=torch.uint8, device="cuda")
         crc_dst = torch.zeros(job.nc, dtype=torch.int32, device="cuda")
         wm.wm_decode_verify(job.wire, r.wire_len, shadow, job.chunk, crc_dst, job.ws, job.res_d)
@@ -166,7 +179,7 @@ def test_random_cache_takes_the_raw_path_and_a_flipped_bit_is_rejected():
     assert r.payload_bytes == job.n and r.wire_len == job.meta_end + job.n
     assert (ln == job.chunk).all()
     check_meta_against_oracle(job, m, hdr, off, ln, dcrc, np.ones(job.nc, dtype=np.uint64))
-    check_chunks_against_oracle(job, cur, sample_chunks(job.nc, 4, 2), off, ln, dcrc, tab)
+    check_whole_image_against_oracle(job, cur, off, ln, dcrc, tab)
 
     shadow = torch.zeros(job.n, dtype=torch.uint8, device="cuda")
     crc_dst = torch.zeros(job.nc, dtype=torch.int32, device="cuda")
@@ -262,16 +275,16 @@ def test_precopy_step_loop_on_two_streams():
             assert torch.equal(dirty.cpu(), mask)
             assert torch.equal(idx[:nd].cpu().long(), torch.nonzero(mask).flatten())
             if k in oracle_steps:
+                # the mask and the index list against the oracle's byte compare of the two snapshots,
+                # then the whole masked image against the oracle's
+                o_dirty, o_idx = oracle_pool.dirty_diff(cur.cpu().numpy(), prev.cpu().numpy(), job.chunk)
+                assert np.array_equal(dirty.cpu().numpy(), o_dirty)
+                assert np.array_equal(idx[:nd].cpu().numpy().view(np.uint32), o_idx)
                 job.wire = wire
                 m, hdr, off, ln, crc, tab = job.meta()
                 present = mask.numpy().astype(np.uint64)
                 check_meta_against_oracle(job, m, hdr, off, ln, crc, present)
-                some = [int(c) for c in torch.nonzero(mask).flatten()[[0, nd // 2, nd - 1]]]
-                check_chunks_against_oracle(job, cur, some, off, ln, crc, tab)
-                absent = [int(c) for c in torch.nonzero(mask == 0).flatten()[:2]]
-                tpc = job.chunk // TILE
-                for c in absent:
-                    assert (tab[c * tpc:(c + 1) * tpc] == 0).all()
+                check_whole_image_against_oracle(job, cur, off, ln, crc, tab, present=mask.numpy())
             encoded = torch.cuda.Event()
             encoded.record(src)
         if pending is not None:
