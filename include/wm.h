@@ -47,7 +47,7 @@ typedef enum {
     WM_ERR_CHUNK_CRC = -7,  /* decode: a decoded chunk does not have the source's CRC    */
     WM_ERR_STALE = -8,      /* decode: a chunk not shipped differs at the destination    */
     WM_ERR_CACHE_CRC = -9,  /* decode: directory CRCs do not combine to the cache CRC    */
-    WM_ERR_TIMEOUT = -10,   /* a bounded device-side wait ran out                        */
+    WM_ERR_TIMEOUT = -10,   /* a bounded device-side wait ran out (see wm_wait_budget_ms) */
     WM_ERR_CUDA = -11       /* CUDA runtime error on launch                              */
 } wm_status;
 
@@ -72,6 +72,46 @@ uint64_t wm_meta_bytes(uint64_t nbytes, uint32_t chunk_bytes);
 uint64_t wm_wire_bound(uint64_t nbytes, uint32_t chunk_bytes);
 /* Scratch the calls below need for this geometry (one size fits all four). */
 uint64_t wm_workspace_bytes(uint64_t nbytes, uint32_t chunk_bytes);
+
+/*
+ * wm_wait_budget_ms - upper bound of every device-side wait, in milliseconds.
+ * Paper: fail-closed behaviour (Section 4.1: a move either completes verified or installs nothing).
+ * The kernels wait in three places: for a bulk copy into shared memory, for the placement
+ * scanner (encode: a tile's offset), and the scanner for the tiles' lengths.  Each wait is bounded
+ * by time on the GPU's own clock, not by a number of polls, so a kernel that shares the GPU with
+ * other work and is descheduled for a while is not mistaken for a failure, and a real failure
+ * never turns into a hang: when the budget has passed the kernel gives up, withdraws the
+ * remaining work, returns, and the call reports WM_ERR_TIMEOUT (the CUDA context stays usable and
+ * the next call on the same workspace starts clean).  Default 2000 ms; process-wide, read by each
+ * call when it is issued; 0 is taken as 1.
+ */
+void wm_wait_budget_ms(uint32_t ms);
+
+/*
+ * wm_workspace_status - device-side outcome of the last call that used this workspace.
+ * wm_encode and the wm_decode_verify family report through their result record; wm_checksum,
+ * wm_checksum_poly and wm_dirty_diff have none.  Their only device-side failure is a wait that
+ * ran out (or, WM_ERR_CUDA, a kernel that did not get its shared memory); then the checksum calls
+ * fill crc_out with zeros instead of delivering digests of data that never arrived, and this call
+ * says why.  wm_dirty_diff has no device-side wait and always leaves WM_OK here.
+ * Synchronous: copies one word from the workspace on `stream` and waits for the stream.
+ *   workspace [dev] a workspace a call was issued with on `stream`; NULL: the built-in scratch
+ *             of wm_checksum_noalloc on the current device
+ * Returns WM_OK, WM_ERR_TIMEOUT, WM_ERR_CUDA (also when the copy itself fails), or, after a codec
+ * call, what its result record says of WM_ERR_CAPACITY / WM_ERR_ARG.
+ */
+wm_status wm_workspace_status(const void* workspace, void* stream);
+
+/*
+ * wm_inject_stall - test hook for the give-up paths (the paper has no counterpart).
+ * While on, calls issued by this process leave out what their bounded waits wait for: the encode
+ * kernel's scanner returns at once (no tile ever gets its offset), the checksum and decode kernels
+ * do not start their bulk copies.  Every wait then runs out after wm_wait_budget_ms and the call
+ * ends in WM_ERR_TIMEOUT without a fault or a hang, which is what tests need to see the timeout
+ * handling run (set a budget of a few tens of milliseconds first).  Off by default; never turn
+ * it on in production.
+ */
+void wm_inject_stall(int on);
 
 /*
  * wm_checksum - CRC32C of every chunk of the flat cache.
@@ -184,15 +224,18 @@ wm_status wm_encode(const void* cache, uint64_t nbytes, uint32_t chunk_bytes, co
  *   1 header fields equal the call's arguments and wire_len        WM_ERR_FORMAT
  *   2 meta_crc                                                     WM_ERR_META_CRC
  *   3 directory and tile table are consistent                      WM_ERR_STRUCT
- *   4 PACK tiles in tile order: descriptors valid (WM_ERR_DESC), then 258 + sum w equals the
- *     tile entry (WM_ERR_STRUCT); the status is that of the lowest failing tile
+ *   4 coded tiles in tile order; the status is that of the lowest failing tile.  PACK tile:
+ *     descriptors valid (WM_ERR_DESC), then 258 + sum w equals the tile entry (WM_ERR_STRUCT).
+ *     ENT tile (images with flags bit2): the eight stream counts within 128..1024 and adding up
+ *     to the entry (WM_ERR_STRUCT), then every stream used up exactly by its 1024 codewords and
+ *     the fill bits of every strand zero (WM_ERR_DESC)
  *   5 CRC32C of every decoded chunk equals its directory CRC       WM_ERR_CHUNK_CRC
  *   6 absent chunk: dst_crc_inout[c] equals its directory CRC      WM_ERR_STALE
  *   7 the directory CRCs combine to header.cache_crc               WM_ERR_CACHE_CRC
  *   8 only then dst_crc_inout[c] <- crc for present chunks, status WM_OK
- * A bounded device-side wait that ran out (a bulk copy that never arrived) gives WM_ERR_TIMEOUT
- * ahead of steps 4..7: the kernels failed, nothing can be said about the image, nothing is
- * installed.
+ * A bounded device-side wait that ran out (a bulk copy that did not arrive within
+ * wm_wait_budget_ms) gives WM_ERR_TIMEOUT ahead of steps 4..7: the kernels failed, nothing can be
+ * said about the image, nothing is installed.
  *   dst           [dev] nbytes bytes, 16-byte aligned: the SHADOW slot.  Present chunks are
  *                 written, absent chunks are left as they are.  On any failure its content is
  *                 unspecified (never written outside [dst, dst+nbytes)) and dst_crc_inout is
@@ -205,8 +248,8 @@ wm_status wm_decode_verify(const void* wire, uint64_t wire_len, void* dst, uint6
 
 /*
  * wm_decode_verify_strict - verify first, write afterwards.
- * Paper: "the destination is bit-identical to the source, or nothing is installed" (Section 1;
- * Section 4.1: a torn state can never be installed).  wm_decode_verify gives that guarantee
+ * Paper: the all-or-nothing guarantee of a move (Section 1; Section 4.1: a torn state can never
+ * be installed).  wm_decode_verify gives that guarantee
  * through the caller's shadow buffer; this call gives it for a buffer that is decoded into in
  * place (the live cache of a pre-copy round): a first pass unpacks and checksums the image
  * without storing a byte, the verdict is taken with all of wm_decode_verify's checks, and only
@@ -301,9 +344,16 @@ wm_status wm_decode_verify_leaves(const void* wire, uint64_t wire_len, const wm_
  * per call and read nothing process-wide, so calls with different options can be issued from
  * different threads and streams of one process.  Exactly one of (cache, leaves) and of (dst,
  * dst_leaves) is non-NULL: the flat form or the leaf form (n_leaves is ignored in the flat form).
- *   options  WM_OPT_ZERO_TILES (encode: the zero-tile option; ignored together with WM_OPT_ENTROPY)
+ *   options  WM_OPT_ZERO_TILES (encode: the zero-tile option; it combines with WM_OPT_ENTROPY)
  *            WM_OPT_ENTROPY    (encode: write ENT tiles; decode: expect an image with ENT tiles)
  *            WM_OPT_STRICT     (decode only: store nothing before every check has passed)
+ *            WM_OPT_BLOCKS(n)  (n = 2..255 for encode, 1..255 for decode; 0 or absent: one block per SM):
+ *                              the main kernel runs on at most n thread blocks, each of which
+ *                              takes a whole SM.  For callers that share the GPU with other work
+ *                              (a generating session during pre-copy, Appendix G; the two
+ *                              streams of a pre-copy loop): the mover then leaves the other SMs
+ *                              alone.  Tiles are claimed by ticket, so the image and every result
+ *                              are the same for every n; only the time changes.
  *            any other bit: WM_ERR_ARG, nothing is launched
  * Everything else (arguments, layouts, statuses, what the result record holds) is as in
  * wm_encode / wm_encode_leaves and wm_decode_verify / wm_decode_verify_leaves / _strict.
@@ -311,6 +361,8 @@ wm_status wm_decode_verify_leaves(const void* wire, uint64_t wire_len, const wm_
 #define WM_OPT_ZERO_TILES 1u
 #define WM_OPT_ENTROPY 2u
 #define WM_OPT_STRICT 4u
+#define WM_OPT_BLOCKS_MASK 0xFF00u
+#define WM_OPT_BLOCKS(n) (((uint32_t)(n) & 0xFFu) << 8)
 wm_status wm_encode_opt(const void* cache, const wm_leaf* leaves, uint32_t n_leaves, uint64_t nbytes, uint32_t chunk_bytes,
                         const uint8_t* dirty, uint32_t* crc_inout, void* wire, uint64_t wire_cap, void* workspace,
                         uint64_t workspace_bytes, uint32_t options, wm_result* result, void* stream);

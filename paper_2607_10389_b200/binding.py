@@ -24,7 +24,9 @@ RESULT_BYTES = 40
 EXPORTS = ("wm_num_chunks", "wm_num_tiles", "wm_meta_bytes", "wm_wire_bound", "wm_workspace_bytes",
            "wm_checksum", "wm_dirty_diff", "wm_encode", "wm_decode_verify", "wm_last_launch_count",
            "wm_timing_enable", "wm_timing_read_ms", "wm_checksum_noalloc", "wm_encode_leaves",
-           "wm_decode_verify_leaves", "wm_zero_tiles_enable", "wm_decode_verify_strict", "wm_checksum_poly", "wm_entropy_enable", "wm_encode_opt", "wm_decode_verify_opt", "wm_checksum_xxh64")
+           "wm_decode_verify_leaves", "wm_zero_tiles_enable", "wm_decode_verify_strict", "wm_checksum_poly", "wm_entropy_enable",
+           "wm_encode_opt", "wm_decode_verify_opt", "wm_checksum_xxh64", "wm_wait_budget_ms", "wm_workspace_status",
+           "wm_inject_stall")
 
 
 class WmError(RuntimeError):
@@ -52,6 +54,12 @@ def load_library() -> ctypes.CDLL:
     lib.wm_zero_tiles_enable.argtypes = [ctypes.c_int]
     lib.wm_entropy_enable.restype = None
     lib.wm_entropy_enable.argtypes = [ctypes.c_int]
+    lib.wm_wait_budget_ms.restype = None
+    lib.wm_wait_budget_ms.argtypes = [u32]
+    lib.wm_inject_stall.restype = None
+    lib.wm_inject_stall.argtypes = [ctypes.c_int]
+    lib.wm_workspace_status.restype = ctypes.c_int
+    lib.wm_workspace_status.argtypes = [vp, vp]
     lib.wm_timing_read_ms.restype = ctypes.c_int
     lib.wm_timing_read_ms.argtypes = [ctypes.c_int, ctypes.POINTER(ctypes.c_float)]
     lib.wm_checksum.restype = ctypes.c_int
@@ -158,6 +166,23 @@ def entropy_enable(on: bool) -> None:
     """Codec option: entropy-coded exponents (ENT tiles).  Applies to the encode calls (what they
     write) and to the decode calls (what they expect) of this process."""
     lib().wm_entropy_enable(1 if on else 0)
+
+
+def wait_budget_ms(ms: int) -> None:
+    """Upper bound of every device-side wait of the calls issued from now on (default 2000 ms)."""
+    lib().wm_wait_budget_ms(int(ms))
+
+
+def inject_stall(on: bool) -> None:
+    """Test hook: calls issued while it is on leave out what their bounded waits wait for, so the
+    waits run out after the budget and the calls end in ERR_TIMEOUT."""
+    lib().wm_inject_stall(1 if on else 0)
+
+
+def workspace_status(workspace, stream=None) -> int:
+    """Device-side outcome (a wm_status) of the last call that used `workspace` on the stream;
+    None stands for the built-in scratch of wm_checksum_noalloc.  Synchronises the stream."""
+    return int(lib().wm_workspace_status(None if workspace is None else workspace.data_ptr(), _stream(stream)))
 
 
 def timing_read_ms(kind: int) -> float:
@@ -285,6 +310,12 @@ def wm_decode_verify_strict(wire: torch.Tensor, wire_len: int, dst: torch.Tensor
 
 
 OPT_ZERO_TILES, OPT_ENTROPY, OPT_STRICT = 1, 2, 4
+
+
+def opt_blocks(n: int) -> int:
+    """Option bits that cap the main kernel at n thread blocks (each takes one SM); 0: no cap."""
+    return (int(n) & 0xFF) << 8
+
 
 
 def wm_encode_opt(cache, chunk_bytes: int, dirty, crc_inout: torch.Tensor, wire: torch.Tensor, workspace: torch.Tensor,

@@ -36,14 +36,16 @@ k_tile_digests(const unsigned char* __restrict__ cache, Geo g, Ws ws, const Tabl
     const uint64_t stride = (uint64_t)gridDim.x * TEAMS;
     const uint64_t pol = l2_policy_evict_first();
     auto full = [&](uint64_t tile) { return tile < g.n_tiles && g.nbytes - tile * kTile >= kTile; };
-    auto start_copy = [&](uint64_t tile) {     // thread 0 only
-        if (full(tile)) bulk_load(stage, cache + tile * kTile, kTile, &tc->mbar, pol);
+    auto start_copy = [&](uint64_t tile) {     // one thread of the team
+        if (full(tile) && !(g.inject & kInjectNoCopy)) bulk_load(stage, cache + tile * kTile, kTile, &tc->mbar, pol);
     };
 
     uint64_t t = (uint64_t)blockIdx.x * TEAMS + team;
     if (tt == 64u) { mbar_init(&tc->mbar, 1); start_copy(t); }
     team_bar(team);
     uint32_t phase = 0, par = 0;
+    bool trouble = false;                        // sticky: a copy did not arrive within the budget
+    uint32_t lost = 0;                           // the stage's phase that never completed
     uint64_t t_done = ~0ull;                     // tile whose digest parts wait in wdig[par ^ 1]
     // One team barrier per tile.  The single-lane chores sit on different warps (the team waits
     // for whichever warp has the most to do): warp 2 starts the next copy, warp 1 folds and
@@ -53,7 +55,9 @@ k_tile_digests(const unsigned char* __restrict__ cache, Geo g, Ws ws, const Tabl
         uint32_t d[kWordsPerLane];
         bool fold = first;
         if (full(t)) {
-            if (!mbar_wait(&tc->mbar, phase) && lane == 0) atomicOr(&ws.ctrl->err, 2u);
+            // (after one wait has run out the thread waits for no other copy: the call has failed,
+            // what is left is to get out quickly)
+            if (!trouble && !mbar_wait(&tc->mbar, phase, g.wait_ns)) { trouble = true; lost = phase; if (lane == 0) atomicOr(&ws.ctrl->err, 2u); }
             phase ^= 1u;
             read_staged_words(stage, warp, lane, d);
         } else {
@@ -61,7 +65,7 @@ k_tile_digests(const unsigned char* __restrict__ cache, Geo g, Ws ws, const Tabl
             fold = false;
         }
         team_bar(team);                          // stage free; the previous tile's digest parts complete
-        if (tt == 64u) start_copy(t + stride);
+        if (tt == 64u && !trouble) start_copy(t + stride);
         if (tt == 32u && t_done != ~0ull) ws.dig[t_done] = xor8(tc->wdig[par ^ 1u]);
         const uint32_t v = tile_digest_part(S, d, fold, warp, lane);
         if (lane == 0) tc->wdig[par][warp] = v;
@@ -70,6 +74,9 @@ k_tile_digests(const unsigned char* __restrict__ cache, Geo g, Ws ws, const Tabl
     }
     team_bar(team);
     if (tt == 32u && t_done != ~0ull) ws.dig[t_done] = xor8(tc->wdig[par ^ 1u]);
+    // a thread that gave up gives the copy it stopped waiting for one more budget to land before
+    // the block, and with it the stage, goes away
+    if (trouble && !(g.inject & kInjectNoCopy)) mbar_wait(&tc->mbar, lost, g.wait_ns);
 }
 
 __global__ void __launch_bounds__(1024)
@@ -84,8 +91,12 @@ k_checksum_finish(const unsigned char* __restrict__ cache, Geo g, Ws ws, const T
     const uint32_t c0 = blockIdx.x * g.finish_cb;
     stage_chunk_digests(g, stage, ws.dig, c0);
     const uint32_t c = c0 + threadIdx.x;
+    // Fail closed: when the digest kernel reported trouble (a wait that ran out, no room for its
+    // stages) some digests are not those of the cache.  The vector is then zero-filled and the
+    // control block keeps the reason for wm_workspace_status.
+    const bool failed = ld_volatile_u32(&ws.ctrl->err) != 0u;
     if (threadIdx.x < g.finish_cb && c < g.n_chunks)
-        crc_out[c] = chunk_crc_staged(g, sHT, sT0, stage, ws.dig, cache + (uint64_t)c * g.chunk_bytes, c, threadIdx.x);
+        crc_out[c] = failed ? 0u : chunk_crc_staged(g, sHT, sT0, stage, ws.dig, cache + (uint64_t)c * g.chunk_bytes, c, threadIdx.x);
 }
 
 }  // namespace wm

@@ -360,7 +360,7 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
     auto is_staged = [&](uint32_t e) { return e == 512u || is_pack_entry(e) || is_ent_entry(e); };
     auto start_copy = [&](const DecSlot& sl) {   // leader only
         const uint32_t e = sl.entry & 0xFFFFu;
-        if (sl.t < g.n_tiles && is_staged(e)) bulk_load(stage, payload + sl.src, 32u * (e & 0x7FFFu), &tc->mbar, 0);
+        if (sl.t < g.n_tiles && is_staged(e) && !(g.inject & kInjectNoCopy)) bulk_load(stage, payload + sl.src, 32u * (e & 0x7FFFu), &tc->mbar, 0);
     };
 
     if (leader) {
@@ -372,7 +372,8 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
     }
     team_bar(team);
     uint32_t phase = 0;
-    uint32_t trouble = 0;              // sticky: a copy never arrived
+    uint32_t trouble = 0;              // sticky: a copy did not arrive within the budget
+    uint32_t lost = 0;                 // the stage's phase that never completed
     uint32_t t_done = kNone;           // tile whose digest parts wait in wdig[(it - 1) & 1]
     for (uint32_t it = 0;; it++) {
         const uint32_t t = tc->slot[it & 3u].t;
@@ -396,7 +397,13 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
 
         // ---- phase 1: everything this lane needs from the stage goes into registers
         if (is_staged(e)) {
-            if (!mbar_wait(&tc->mbar, phase)) trouble = 1u;
+            // (after one wait has run out the thread waits for no other copy and the team starts none:
+            // the call has failed, the tickets are withdrawn, what is left is to get out quickly)
+            if (!trouble && !mbar_wait(&tc->mbar, phase, g.wait_ns)) {
+                trouble = 1u;
+                lost = phase;
+                if (lane == 0) { atomicOr(&ws.ctrl->err, 2u); atomicMax(&ws.ctrl->ticket, 0x7FFF0000u); }
+            }
             phase ^= 1u;
             if (!is_pack) {
                 read_staged_words(stage, warp, lane, w);
@@ -510,7 +517,7 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
         uint32_t l_e = 0, l_rel = 0, l_tk = kNone;
         unsigned long long l_po = 0;
         // (spread over three warps: the team waits for whichever warp has the most to do)
-        if (tt == 64u) start_copy(tc->slot[(it + 1u) & 3u]);
+        if (tt == 64u && !trouble) start_copy(tc->slot[(it + 1u) & 3u]);
         if (tt == 32u && t_done != kNone) ws.dig[t_done] = xor8(tc->wdig[p ^ 1u]);
         uint32_t t_look = kNone;           // warps 0 and 3: the tile claimed a step ago (two tiles ahead)
         if (leader) {                      // its table entry and offsets
@@ -602,7 +609,9 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
         }
         if (tt == 96u) tc->slot[(it + 3u) & 3u].t = l_tk;      // (none once the tickets have run out)
     }
-    if (trouble && lane == 0) atomicOr(&ws.ctrl->err, 2u);
+    // a thread that gave up gives the copy it stopped waiting for one more budget to land before
+    // the block, and with it the stage, goes away
+    if (trouble && !(g.inject & kInjectNoCopy)) mbar_wait(&tc->mbar, lost, g.wait_ns);
 }
 
 // Steps 5..8: chunk CRCs of the decoded bytes against the directory, stale check, cache CRC;

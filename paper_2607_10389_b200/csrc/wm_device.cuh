@@ -271,19 +271,34 @@ __device__ __forceinline__ void bulk_load(void* smem_dst, const void* gsrc, uint
                      ::"r"(d), "l"(gsrc), "r"(bytes), "r"(b) : "memory");
 }
 
-// Wait for the phase with the given parity to complete (bounded).  Returns false on timeout.
-// try_wait suspends the thread in hardware until the phase completes or the time hint runs
-// out, so a waiting warp does not burn issue slots that the other teams on the SM need.
-__device__ __forceinline__ bool mbar_wait(unsigned long long* bar, uint32_t parity)
+// Nanoseconds of the GPU's wall clock.  Every device-side wait is bounded by TIME against the
+// call's budget (Geo::wait_ns, two seconds unless the caller set another), not by a number of
+// polls: a block that shares the GPU with other work can be descheduled for a long time, and a
+// poll count says nothing about how long that was.
+__device__ __forceinline__ unsigned long long now_ns()
+{
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+
+// Wait for the phase with the given parity to complete, for at most `budget_ns`.  Returns false
+// when the time ran out.  try_wait suspends the thread in hardware until the phase completes or
+// the time hint runs out, so a waiting warp does not burn issue slots that the other teams on
+// the SM need; the clock is only read after a try has come back empty.
+__device__ __forceinline__ bool mbar_wait(unsigned long long* bar, uint32_t parity, unsigned long long budget_ns)
 {
     const uint32_t b = (uint32_t)__cvta_generic_to_shared(bar);
-    for (uint32_t i = 0; i < 4096u; i++) {
+    unsigned long long t0 = 0;
+    for (uint32_t i = 0;; i++) {
         uint32_t done;
         asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-                     : "=r"(done) : "r"(b), "r"(parity), "r"(500000u) : "memory");
+                     : "=r"(done) : "r"(b), "r"(parity), "r"(200000u) : "memory");
         if (done) return true;
+        const unsigned long long t = now_ns();
+        if (i == 0) t0 = t;
+        else if (t - t0 > budget_ns) return false;
     }
-    return false;
 }
 
 __device__ __forceinline__ uint64_t l2_policy_evict_first()

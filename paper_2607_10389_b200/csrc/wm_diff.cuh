@@ -9,7 +9,7 @@ namespace wm {
 __global__ void k_diff_init(Ws ws)
 {
     grid_dep_launch();
-    if (threadIdx.x == 0 && blockIdx.x == 0) { ws.ctrl->ticket = 0; ws.ctrl->n_present = 0; }
+    if (threadIdx.x == 0 && blockIdx.x == 0) { ws.ctrl->ticket = 0; ws.ctrl->n_present = 0; ws.ctrl->err = 0; }
 }
 
 // One block per chunk at a time (ticketed); the chunk is scanned in 16 KiB half-steps, two of

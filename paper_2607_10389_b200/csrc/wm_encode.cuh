@@ -20,7 +20,6 @@ __global__ void k_encode_init(Geo g, Ws ws, unsigned char* wire)
 }
 
 constexpr uint32_t kFlagA = 1u << 30, kFlagP = 2u << 30, kValMask = (1u << 30) - 1u;
-constexpr uint32_t kSpinLimit = 1u << 20;
 constexpr uint32_t kUnit = 32;              // placement words count in units of 32 bytes
 
 // Placement of the encoded tiles: a chained scan with one dedicated scanner warp.
@@ -38,8 +37,8 @@ constexpr uint32_t kUnit = 32;              // placement words count in units of
 // the bottleneck, and assigning tiles statically made every round wait for its slowest team.
 // The scanner is running by construction (it won the lock), tiles are claimed in ticket
 // order, and a team publishes the length of a claimed tile without waiting for anyone, so the
-// owners' waits depend only on running code; they are bounded all the same and end in
-// WM_ERR_TIMEOUT.
+// owners' waits depend only on running code; they are bounded all the same, by time (the call's
+// wait budget), and end in WM_ERR_TIMEOUT.
 __device__ __forceinline__ void st_relaxed_u32(uint32_t* p, uint32_t v)
 {
     asm volatile("st.relaxed.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
@@ -63,13 +62,20 @@ __device__ __forceinline__ uint32_t next_ticket(Ctrl* ctrl)
     return atomicAdd(&ctrl->ticket, 1u);
 }
 
-// Owner side: exclusive prefix (bytes) of tile t (one lane spins; bounded).
-__device__ __forceinline__ unsigned long long wait_prefix(const uint32_t* lbk, uint32_t t, Ctrl* ctrl)
+// Owner side: exclusive prefix (bytes) of tile t (one lane spins, for at most `budget_ns`; the
+// poison flag and the clock are looked at every 64 polls).
+__device__ __forceinline__ unsigned long long wait_prefix(const uint32_t* lbk, uint32_t t, Ctrl* ctrl, unsigned long long budget_ns)
 {
-    for (uint32_t polls = 0; polls < kSpinLimit; polls++) {
+    unsigned long long t0 = 0;
+    for (uint32_t polls = 0;; polls++) {
         const uint32_t v = ld_relaxed_u32(lbk + t);
         if ((v >> 30) == 2u) return (unsigned long long)(v & kValMask) * kUnit;
-        if ((polls & 1023u) == 1023u && ld_volatile_u32(&ctrl->poison)) break;
+        if ((polls & 63u) == 63u) {
+            if (ld_volatile_u32(&ctrl->poison)) break;
+            const unsigned long long now = now_ns();
+            if (t0 == 0) t0 = now;
+            else if (now - t0 > budget_ns) break;
+        }
     }
     atomicOr(&ctrl->err, 2u);
     raise_poison(ctrl);
@@ -80,18 +86,14 @@ __device__ __forceinline__ unsigned long long wait_prefix(const uint32_t* lbk, u
 // coalesced asynchronous 16-byte copies (one round trip to L2, no registers held meanwhile);
 // lane l then owns entries 16 l .. 16 l + 15 of the window.
 constexpr int kScanPerLane = 16;
-__device__ void scan_tile_lengths(uint32_t* lbk, uint32_t n_tiles, uint32_t lane, Ctrl* ctrl, uint32_t* win)
+__device__ void scan_tile_lengths(uint32_t* lbk, uint32_t n_tiles, uint32_t lane, Ctrl* ctrl, uint32_t* win,
+                                  unsigned long long budget_ns)
 {
     uint64_t f = 0;                 // first unresolved entry
     uint64_t base = 0;              // units before f
-    uint32_t spins = 0;
-#ifdef WM_DEBUG_COUNTERS
-    uint32_t dbg_iters = 0, dbg_empty = 0;
-#endif
+    uint32_t spins = 0;             // polls in a row that resolved nothing
+    unsigned long long t0 = 0;      // the clock when that run of empty polls was first timed
     while (f < n_tiles) {
-#ifdef WM_DEBUG_COUNTERS
-        dbg_iters++;
-#endif
         const uint64_t w0 = f & ~3ull;                    // 16-byte aligned window start
         const uint32_t skip = (uint32_t)(f - w0);         // entries before f (already resolved)
 #pragma unroll
@@ -147,21 +149,24 @@ __device__ void scan_tile_lengths(uint32_t* lbk, uint32_t n_tiles, uint32_t lane
         const uint32_t k = k_all > skip ? k_all - skip : 0u;
         base += __shfl_sync(0xFFFFFFFFu, incl, 31);
         f += k;
-#ifdef WM_DEBUG_COUNTERS
-        if (k == 0) dbg_empty++;
-#endif
         if (k == 0) {
-            if (++spins > kSpinLimit || ((spins & 1023u) == 1023u && ld_volatile_u32(&ctrl->poison))) {
-                if (lane == 0) { atomicOr(&ctrl->err, 2u); raise_poison(ctrl); }
-                return;
+            // nothing new: the owners are behind.  Every 64 such polls in a row the scanner looks at the
+            // poison flag and at the clock; it gives up when no length has come in for the whole budget.
+            if ((++spins & 63u) == 0u) {
+                bool stop = ld_volatile_u32(&ctrl->poison) != 0u;
+                const unsigned long long now = now_ns();
+                if (t0 == 0) t0 = now;
+                else if (now - t0 > budget_ns) stop = true;
+                if (__any_sync(0xFFFFFFFFu, stop)) {
+                    if (lane == 0) { atomicOr(&ctrl->err, 2u); raise_poison(ctrl); }
+                    return;
+                }
             }
         } else {
             spins = 0;
+            t0 = 0;
         }
     }
-#ifdef WM_DEBUG_COUNTERS
-    if (lane == 0) { ctrl->pad[0] = dbg_iters; ctrl->pad[1] = dbg_empty; }
-#endif
 }
 
 __device__ __forceinline__ uint32_t desc_of(uint32_t base, uint32_t w)
@@ -375,7 +380,8 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
     __syncthreads();
     if (s_scanner) {
         uint32_t* win = reinterpret_cast<uint32_t*>(S.take(2048));      // 512 entries
-        if (threadIdx.x < 32 && win) scan_tile_lengths(ws.lbk, g.n_tiles, threadIdx.x, ws.ctrl, win);
+        // (test hook: with the scanner left out no offset is ever handed out, and the owners' waits run out)
+        if (threadIdx.x < 32 && win && !(g.inject & kInjectNoScanner)) scan_tile_lengths(ws.lbk, g.n_tiles, threadIdx.x, ws.ctrl, win, g.wait_ns);
         return;
     }
     const uint32_t team = threadIdx.x / kTeamThreads, tt = threadIdx.x % kTeamThreads;
@@ -455,11 +461,18 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
     qY = tc->next[0];
     if (leader) start_copy(qY, LEAVES ? tc->nptr[0] : tile_src(qY & kQTile));
 
-    uint32_t trouble = 0;              // sticky: 1 the image does not fit, 2 a copy never arrived
+    uint32_t trouble = 0;              // sticky: 1 the image does not fit, 2 a copy did not arrive within the budget
+    uint32_t lost = 0;                 // the stage's phase that never completed
     while (((qX & qV & qW & qY) & kQTile) != kQNone) {
         const bool hotY = is_hot(qY);
         if (hotY) {
-            if (!mbar_wait(&tc->mbar, phase)) trouble |= 2u;
+            // (after one wait has run out the thread waits for no other copy and the team starts none:
+            // the call has failed, the tickets are withdrawn, what is left is to get out quickly)
+            if (!(trouble & 2u) && !mbar_wait(&tc->mbar, phase, g.wait_ns)) {
+                trouble |= 2u;
+                lost = phase;
+                if (lane == 0) { atomicOr(&ws.ctrl->err, 2u); raise_poison(ws.ctrl); }
+            }
             phase ^= 1u;
 #pragma unroll
             for (int i = 0; i < 16; i++) d[i] = my_words[i * 32];
@@ -474,7 +487,7 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
         // of the tile to pack in the next step (warp 3).  Warp 1 notes what is left about X.
         uint32_t pv = 0, tk = 0xFFFFFFFFu;
         const unsigned char* pA = nullptr;
-        if (tt == 64u) start_copy(qN, LEAVES ? tc->nptr[par ^ 1u] : tile_src(qN & kQTile));
+        if (tt == 64u && !(trouble & 2u)) start_copy(qN, LEAVES ? tc->nptr[par ^ 1u] : tile_src(qN & kQTile));
         if (tt == 96u && is_tile(qV)) pv = ld_relaxed_u32(ws.lbk + (qV & kQTile));
         if (leader) {
             if (claiming) tk = next_ticket(ws.ctrl);
@@ -749,12 +762,9 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
             }
         }
         if (tt == 96u) {
-#ifdef WM_DEBUG_COUNTERS
-            atomicAdd(&ws.ctrl->pad[(pv >> 30) == 2u ? 3 : 2], 1u);
-#endif
             unsigned long long e = 0;
             if (is_tile(qV))
-                e = (pv >> 30) == 2u ? (unsigned long long)(pv & kValMask) * kUnit : wait_prefix(ws.lbk, qV & kQTile, ws.ctrl);
+                e = (pv >> 30) == 2u ? (unsigned long long)(pv & kValMask) * kUnit : wait_prefix(ws.lbk, qV & kQTile, ws.ctrl, g.wait_ns);
             tc->excl[par] = e;
         }
         qX = qV; qV = qW; qW = qY; qY = qN;
@@ -762,10 +772,10 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
         par ^= 1u;
         step++;
     }
-    if (trouble && lane == 0) {
-        atomicOr(&ws.ctrl->err, trouble);
-        if (trouble & 2u) raise_poison(ws.ctrl);
-    }
+    if ((trouble & 1u) && lane == 0) atomicOr(&ws.ctrl->err, 1u);
+    // a thread that gave up gives the copy it stopped waiting for one more budget to land before
+    // the block, and with it the stage, goes away
+    if (trouble & 2u) mbar_wait(&tc->mbar, lost, g.wait_ns);
     // every warp is done with its tensor memory: hand it back before the block exits
     tmem_fence_before_sync();
     __syncthreads();

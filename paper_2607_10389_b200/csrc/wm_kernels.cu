@@ -29,6 +29,13 @@
 #include "wm_decode.cuh"
 #include "wm_xxh64.cuh"
 
+// Scratch and tables of wm_checksum_noalloc live in the library image itself: two file-scope
+// __device__ arrays that every GPU loading the library carries until the process exits.  In host
+// code their names are host-side stand-ins, not device addresses, so the addresses are asked for
+// with cudaGetSymbolAddress (with the device in question current) and only those go to kernels.
+static __device__ __align__(256) unsigned char g_na_scratch[WM_NOALLOC_SCRATCH_BYTES];
+static __device__ __align__(256) unsigned char g_na_tables[sizeof(wm::Tables)];
+
 namespace wm {
 
 // ------------------------------------------------------------------ host side
@@ -177,6 +184,24 @@ void wm_timing_enable(int on) { g_timing = on != 0; }
 void wm_zero_tiles_enable(int on) { g_zero_tiles = on != 0; }
 void wm_entropy_enable(int on) { g_entropy = on != 0; }
 
+void wm_wait_budget_ms(uint32_t ms) { g_wait_ns = (uint64_t)(ms ? ms : 1u) * 1000000ull; }
+void wm_inject_stall(int on) { g_inject = on ? (kInjectNoScanner | kInjectNoCopy) : 0u; }
+
+wm_status wm_workspace_status(const void* workspace, void* stream)
+{
+    const Ctrl* ctrl = static_cast<const Ctrl*>(workspace);
+    if (!ctrl) {                       // the built-in scratch of wm_checksum_noalloc on the current device
+        void* p = nullptr;
+        if (cudaGetSymbolAddress(&p, g_na_scratch) != cudaSuccess || !p) return WM_ERR_CUDA;
+        ctrl = static_cast<const Ctrl*>(p);
+    }
+    uint32_t err = 0;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (cudaMemcpyAsync(&err, &ctrl->err, sizeof err, cudaMemcpyDeviceToHost, s) != cudaSuccess) return WM_ERR_CUDA;
+    if (cudaStreamSynchronize(s) != cudaSuccess) return WM_ERR_CUDA;
+    return (err & 8u) ? WM_ERR_ARG : (err & 4u) ? WM_ERR_CUDA : (err & 2u) ? WM_ERR_TIMEOUT : (err & 1u) ? WM_ERR_CAPACITY : WM_OK;
+}
+
 int wm_timing_read_ms(int kind, float* ms)
 {
     const DeviceState* ds = device_state();
@@ -198,6 +223,8 @@ wm_status wm_checksum(const void* cache, uint64_t nbytes, uint32_t chunk_bytes, 
     const unsigned char* c = static_cast<const unsigned char*>(cache);
     const uint32_t need = (g.n_tiles + kTeamsPlain - 1) / kTeamsPlain;
     const uint32_t grid = need < (uint32_t)ds->sm_count ? need : (uint32_t)ds->sm_count;
+    // the control block starts at zero: the error word in it is this call's outcome (wm_workspace_status)
+    if (cudaMemsetAsync(ws.ctrl, 0, sizeof(Ctrl), s) != cudaSuccess) return WM_ERR_CUDA;
     {
         MainKernelTimer timer(ds, 0, s);
         k_tile_digests<kTeamsPlain><<<grid, kTeamsPlain * 256, kDynSmem, s>>>(c, g, ws, ds->tables);
@@ -246,6 +273,8 @@ wm_status wm_checksum_poly(const void* cache, uint64_t nbytes, uint32_t chunk_by
     const unsigned char* c = static_cast<const unsigned char*>(cache);
     const uint32_t need = (g.n_tiles + kTeamsPlain - 1) / kTeamsPlain;
     const uint32_t grid = need < (uint32_t)ds->sm_count ? need : (uint32_t)ds->sm_count;
+    // the control block starts at zero: the error word in it is this call's outcome (wm_workspace_status)
+    if (cudaMemsetAsync(ws.ctrl, 0, sizeof(Ctrl), s) != cudaSuccess) return WM_ERR_CUDA;
     {
         MainKernelTimer timer(ds, 0, s);
         k_tile_digests<kTeamsPlain><<<grid, kTeamsPlain * 256, kDynSmem, s>>>(c, g, ws, tab);
@@ -271,13 +300,7 @@ wm_status wm_checksum_xxh64(const void* cache, uint64_t nbytes, uint32_t chunk_b
 }
 
 // ---- wm_checksum_noalloc: the checksum call for callers that must not allocate -------------
-//
-// Scratch and tables live in the library image itself: two file-scope __device__ arrays that
-// every GPU loading the library carries until the process exits.  In host code their names
-// are host-side stand-ins, not device addresses, so the addresses are asked for once per
-// device with cudaGetSymbolAddress (with that device current) and only those go to kernels.
-static __device__ __align__(256) unsigned char g_na_scratch[WM_NOALLOC_SCRATCH_BYTES];
-static __device__ __align__(256) unsigned char g_na_tables[sizeof(wm::Tables)];
+// (scratch and tables: the two file-scope __device__ arrays declared at the top of this file)
 
 namespace wm {
 struct NoAllocState {
@@ -374,7 +397,9 @@ static wm_status encode_any(const void* cache, const wm_leaf* leaves, uint32_t n
                             uint64_t workspace_bytes, wm_result* result, void* stream, uint32_t options)
 {
     Geo g;
-    if (options & ~(WM_OPT_ZERO_TILES | WM_OPT_ENTROPY)) return WM_ERR_ARG;
+    if (options & ~(WM_OPT_ZERO_TILES | WM_OPT_ENTROPY | WM_OPT_BLOCKS_MASK)) return WM_ERR_ARG;
+    const uint32_t block_cap = (options & WM_OPT_BLOCKS_MASK) >> 8;       // 0: every SM
+    if (block_cap == 1u) return WM_ERR_ARG;                               // one block scans, at least one encodes
     const bool opt_ent = (options & WM_OPT_ENTROPY) != 0, opt_zero = (options & WM_OPT_ZERO_TILES) != 0;
     if (!crc_inout || !wire || !workspace || !result || !make_geo(nbytes, chunk_bytes, g)) return WM_ERR_ARG;
     if (leaves ? (n_leaves == 0 || n_leaves > kMaxLeaves) : (!cache || !aligned16(cache))) return WM_ERR_ARG;
@@ -394,8 +419,11 @@ static wm_status encode_any(const void* cache, const wm_leaf* leaves, uint32_t n
         launch_after(k_leaf_map, map_blocks ? map_blocks : 1, 1024, 0, s, leaves, n_leaves, g, ws, result, 0);
     }
     // one block per SM: one of them scans, the others encode
+    // (tiles are claimed by ticket, so any number of blocks gives the same image; a caller that
+    // shares the GPU with other work caps it)
     const uint32_t need = (g.n_tiles + kTeams - 1) / kTeams + 1;
-    const uint32_t grid = need < (uint32_t)ds->sm_count ? need : (uint32_t)ds->sm_count;
+    uint32_t grid = need < (uint32_t)ds->sm_count ? need : (uint32_t)ds->sm_count;
+    if (block_cap && grid > block_cap) grid = block_cap;
     {
         MainKernelTimer timer(ds, 2, s);
         const int variant = (dirty ? 1 : 0) | (leaves ? 2 : 0) | (opt_zero ? 4 : 0) | (opt_ent ? 8 : 0);
@@ -451,7 +479,8 @@ static wm_status decode_any(const void* wire, uint64_t wire_len, void* dst, cons
                             wm_result* result, void* stream, uint32_t options)
 {
     Geo g;
-    if (options & ~(WM_OPT_ZERO_TILES | WM_OPT_ENTROPY | WM_OPT_STRICT)) return WM_ERR_ARG;
+    if (options & ~(WM_OPT_ZERO_TILES | WM_OPT_ENTROPY | WM_OPT_STRICT | WM_OPT_BLOCKS_MASK)) return WM_ERR_ARG;
+    const uint32_t block_cap = (options & WM_OPT_BLOCKS_MASK) >> 8;       // 0: every SM
     const bool strict = (options & WM_OPT_STRICT) != 0;
     if (!wire || !dst_crc_inout || !workspace || !result || !make_geo(nbytes, chunk_bytes, g)) return WM_ERR_ARG;
     if (leaves ? (n_leaves == 0 || n_leaves > kMaxLeaves) : (!dst || !aligned16(dst))) return WM_ERR_ARG;
@@ -474,7 +503,8 @@ static wm_status decode_any(const void* wire, uint64_t wire_len, void* dst, cons
     launch_after(k_decode_check, meta_blocks + (g.n_chunks + 31) / 32, 1024, 0, s, w, wire_len, g, ws, ds->tables, result, meta_blocks,
                  ent ? 1u : 0u);
     const uint32_t need = (g.n_tiles + kTeamsPlain - 1) / kTeamsPlain;
-    const uint32_t grid = need < (uint32_t)ds->sm_count ? need : (uint32_t)ds->sm_count;
+    uint32_t grid = need < (uint32_t)ds->sm_count ? need : (uint32_t)ds->sm_count;
+    if (block_cap && grid > block_cap) grid = block_cap;
     auto pass = [&](auto flat_kernel, auto leaf_kernel) {
         if (leaves) launch_after(leaf_kernel, grid, kTeamsPlain * 256, kDynSmem, s, w, g, d, ws, ds->tables);
         else launch_after(flat_kernel, grid, kTeamsPlain * 256, kDynSmem, s, w, g, d, ws, ds->tables);

@@ -24,7 +24,13 @@ struct Geo {
     uint32_t n_full_tiles;    // tiles of exactly 16384 bytes
     uint32_t finish_cb;       // chunks handled by one block of the finish kernels
     uint32_t poly;            // reflected CRC polynomial of the k_* powers (CRC32C except in wm_checksum_poly)
+    uint32_t inject;          // test hook (wm_inject_stall): kInject* bits, 0 in normal operation
+    uint64_t wait_ns;         // budget of every device-side wait (wm_wait_budget_ms)
 };
+// Geo::inject.  What a bounded wait waits for is left out, so that the wait runs out and the
+// give-up path can be tested without a fault: the scanner warp returns at once (encode), the bulk
+// copies into the stages are not issued (checksum, decode).
+constexpr uint32_t kInjectNoScanner = 1u, kInjectNoCopy = 2u;
 
 // Powers of k_chunk = x^(8 chunk_bytes), by 7-bit digit of the exponent: k_chunk^e is the product
 // of d0[e & 127], d1[(e >> 7) & 127], d2[(e >> 14) & 127] and, beyond 2^21 chunks, of the
@@ -39,7 +45,7 @@ struct ChunkPowers {
 struct Ctrl {                 // first 256 bytes of the workspace
     uint32_t ticket;
     uint32_t poison;
-    uint32_t err;             // bit0 capacity, bit1 timeout
+    uint32_t err;             // bit0 capacity, bit1 timeout, bit2 shared memory carve failed, bit3 leaf table refused
     uint32_t done_a;
     uint32_t done_b;
     uint32_t n_present;
@@ -115,7 +121,20 @@ constexpr uint64_t kMaxCodecBytes = 32ull << 30;
 constexpr uint32_t kFinishDigests = 8192;    // tile digests a finish block stages in shared memory
 constexpr uint32_t kFinishChunks = 128;      // at most this many chunks per finish block
 
+// Process-wide settings every call reads when it is issued (atomics: calls come from any thread).
+static std::atomic<uint64_t> g_wait_ns{2000ull * 1000ull * 1000ull};    // wm_wait_budget_ms
+static std::atomic<uint32_t> g_inject{0};                               // wm_inject_stall
+
+static bool make_geo_fixed(uint64_t nbytes, uint32_t chunk_bytes, Geo& g);
 static bool make_geo(uint64_t nbytes, uint32_t chunk_bytes, Geo& g)
+{
+    if (!make_geo_fixed(nbytes, chunk_bytes, g)) return false;
+    g.wait_ns = g_wait_ns.load(std::memory_order_relaxed);
+    g.inject = g_inject.load(std::memory_order_relaxed);
+    return true;
+}
+
+static bool make_geo_fixed(uint64_t nbytes, uint32_t chunk_bytes, Geo& g)
 {
     if (nbytes == 0 || chunk_bytes == 0 || chunk_bytes % kTile != 0 || chunk_bytes > (1u << 30)) return false;
     uint64_t nt = (nbytes + kTile - 1) / kTile;
@@ -125,6 +144,8 @@ static bool make_geo(uint64_t nbytes, uint32_t chunk_bytes, Geo& g)
     static thread_local bool have_last = false;
     if (have_last && last.nbytes == nbytes && last.chunk_bytes == chunk_bytes) { g = last; return true; }
     have_last = false;
+    g.inject = 0;
+    g.wait_ns = 0;
     g.nbytes = nbytes;
     g.chunk_bytes = chunk_bytes;
     g.tiles_per_chunk = chunk_bytes / kTile;

@@ -1,0 +1,58 @@
+"""Grid independence: tiles are claimed by ticket, so the wire image, the CRC vector and every
+result are the same whatever number of thread blocks the main kernels run on.  WM_OPT_BLOCKS caps
+that number for callers that share the GPU; here it also serves to prove the independence
+(1 encoding block beside the scanner, a handful, half the machine, all of it, more than exist)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2607_10389_b200 import binding as wm
+from paper_2607_10389_b200 import inputs
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("options,kw", [(0, {}), (wm.OPT_ENTROPY, {"entropy": True}),
+                                        (wm.OPT_ZERO_TILES | wm.OPT_ENTROPY, {"entropy": True, "zero_tiles": True})])
+def test_same_bytes_at_every_block_count(options, kw):
+    cfg = inputs.CONFIGS["engine_small"]
+    host = inputs.make_cache(cfg)[: cfg.nbytes - 1234].contiguous()
+    host[5 * 65536: 5 * 65536 + 3 * 16384] = 0
+    chunk = 65536
+    cur = host.cuda()
+    n = cur.numel()
+    nc = wm.num_chunks(n, chunk)
+    rng = np.random.default_rng(11)
+    for mask in (None, (rng.random(nc) < 0.75).astype(np.uint8)):
+        crc_in = rng.integers(0, 2**32, nc, dtype=np.uint64).astype(np.uint32)
+        want_wire, want_crc, want = oracle.encode(host.numpy(), chunk, dirty=mask, crc_in=crc_in, **kw)
+        d = None if mask is None else torch.from_numpy(mask).cuda()
+        ws, res = wm.new_workspace(n, chunk), wm.new_result()
+        wire = torch.zeros(wm.wire_bound(n, chunk), dtype=torch.uint8, device="cuda")
+        for blocks in (0, 2, 3, 37, 74, 148, 255):
+            crc = torch.from_numpy(crc_in.view(np.int32).copy()).cuda()
+            wire.fill_(0xEE)
+            wm.wm_encode_opt(cur, chunk, d, crc, wire, ws, res, options | wm.opt_blocks(blocks))
+            r = wm.read_result(res)
+            assert r.ok and (r.wire_len, r.cache_crc, r.n_present) == (want.wire_len, want.cache_crc, want.n_present), blocks
+            assert np.array_equal(wire[: r.wire_len].cpu().numpy(), want_wire), blocks
+            assert np.array_equal(crc.cpu().numpy().view(np.uint32), want_crc), blocks
+        for blocks in (0, 1, 2, 37, 74, 255):
+            dst = host.cuda() if mask is not None else torch.zeros(n, dtype=torch.uint8, device="cuda")
+            dst_crc = torch.from_numpy(want_crc.view(np.int32).copy()).cuda() if mask is not None else \
+                torch.zeros(nc, dtype=torch.int32, device="cuda")
+            wm.wm_decode_verify_opt(wire, r.wire_len, dst, chunk, dst_crc, ws, res,
+                                    (options & wm.OPT_ENTROPY) | wm.opt_blocks(blocks))
+            rd = wm.read_result(res)
+            assert rd.ok and torch.equal(dst, cur), blocks
+            assert np.array_equal(dst_crc.cpu().numpy().view(np.uint32), want_crc), blocks
+
+
+def test_a_block_cap_of_one_is_refused_for_encode():
+    cur = torch.zeros(65536, dtype=torch.uint8, device="cuda")
+    ws, res = wm.new_workspace(65536, 65536), wm.new_result()
+    wire = torch.zeros(wm.wire_bound(65536, 65536), dtype=torch.uint8, device="cuda")
+    crc = torch.zeros(1, dtype=torch.int32, device="cuda")
+    with pytest.raises(wm.WmError, match="ERR_ARG"):
+        wm.wm_encode_opt(cur, 65536, None, crc, wire, ws, res, wm.opt_blocks(1))
