@@ -44,8 +44,6 @@ k_tile_digests(const unsigned char* __restrict__ cache, Geo g, Ws ws, const Tabl
     if (tt == 64u) { mbar_init(&tc->mbar, 1); start_copy(t); }
     team_bar(team);
     uint32_t phase = 0, par = 0;
-    bool trouble = false;                        // sticky: a copy did not arrive within the budget
-    uint32_t lost = 0;                           // the stage's phase that never completed
     uint64_t t_done = ~0ull;                     // tile whose digest parts wait in wdig[par ^ 1]
     // One team barrier per tile.  The single-lane chores sit on different warps (the team waits
     // for whichever warp has the most to do): warp 2 starts the next copy, warp 1 folds and
@@ -55,9 +53,7 @@ k_tile_digests(const unsigned char* __restrict__ cache, Geo g, Ws ws, const Tabl
         uint32_t d[kWordsPerLane];
         bool fold = first;
         if (full(t)) {
-            // (after one wait has run out the thread waits for no other copy: the call has failed,
-            // what is left is to get out quickly)
-            if (!trouble && !mbar_wait(&tc->mbar, phase, g.wait_ns)) { trouble = true; lost = phase; if (lane == 0) atomicOr(&ws.ctrl->err, 2u); }
+            wait_for_copy<false>(&tc->mbar, phase, g.wait_ns, ws.ctrl, (g.inject & kInjectNoCopy) != 0u);
             phase ^= 1u;
             read_staged_words(stage, warp, lane, d);
         } else {
@@ -65,7 +61,7 @@ k_tile_digests(const unsigned char* __restrict__ cache, Geo g, Ws ws, const Tabl
             fold = false;
         }
         team_bar(team);                          // stage free; the previous tile's digest parts complete
-        if (tt == 64u && !trouble) start_copy(t + stride);
+        if (tt == 64u) start_copy(t + stride);
         if (tt == 32u && t_done != ~0ull) ws.dig[t_done] = xor8(tc->wdig[par ^ 1u]);
         const uint32_t v = tile_digest_part(S, d, fold, warp, lane);
         if (lane == 0) tc->wdig[par][warp] = v;
@@ -74,9 +70,6 @@ k_tile_digests(const unsigned char* __restrict__ cache, Geo g, Ws ws, const Tabl
     }
     team_bar(team);
     if (tt == 32u && t_done != ~0ull) ws.dig[t_done] = xor8(tc->wdig[par ^ 1u]);
-    // a thread that gave up gives the copy it stopped waiting for one more budget to land before
-    // the block, and with it the stage, goes away
-    if (trouble && !(g.inject & kInjectNoCopy)) mbar_wait(&tc->mbar, lost, g.wait_ns);
 }
 
 __global__ void __launch_bounds__(1024)

@@ -308,7 +308,7 @@ __device__ __forceinline__ void unpack_group_planes(const PlaneWords& pw, uint32
 template <int TEAMS, bool LEAVES, int MODE, int ENT = 0>
 __global__ void __launch_bounds__(TEAMS * 256, 1)
 k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restrict__ dst, Ws ws,
-         const Tables* __restrict__ tab)
+         const Tables* __restrict__ tab, LeafView lv)
 {
     extern __shared__ __align__(16) unsigned char smem[];
     // ENT: what the low byte of a strand's bits says about the codeword there: its length (16: the
@@ -372,8 +372,6 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
     }
     team_bar(team);
     uint32_t phase = 0;
-    uint32_t trouble = 0;              // sticky: a copy did not arrive within the budget
-    uint32_t lost = 0;                 // the stage's phase that never completed
     uint32_t t_done = kNone;           // tile whose digest parts wait in wdig[(it - 1) & 1]
     for (uint32_t it = 0;; it++) {
         const uint32_t t = tc->slot[it & 3u].t;
@@ -385,7 +383,7 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
         const uint32_t ew = tc->slot[it & 3u].entry;
         const uint32_t e = ew & 0xFFFFu;
         // leaf mode: where this tile goes (asked for now, needed when the stores begin)
-        unsigned char* const o_leaf = LEAVES ? ws.tptr[t] : nullptr;
+        const unsigned long long o_leaf = LEAVES ? ws.tptr[t] : 0ull;
         const uint32_t p = it & 1u;
         const bool is_ent = is_ent_entry(e);
         const bool is_pack = is_ent || is_pack_entry(e);            // a coded tile (in either form)
@@ -397,13 +395,7 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
 
         // ---- phase 1: everything this lane needs from the stage goes into registers
         if (is_staged(e)) {
-            // (after one wait has run out the thread waits for no other copy and the team starts none:
-            // the call has failed, the tickets are withdrawn, what is left is to get out quickly)
-            if (!trouble && !mbar_wait(&tc->mbar, phase, g.wait_ns)) {
-                trouble = 1u;
-                lost = phase;
-                if (lane == 0) { atomicOr(&ws.ctrl->err, 2u); atomicMax(&ws.ctrl->ticket, 0x7FFF0000u); }
-            }
+            wait_for_copy<ENT == 0>(&tc->mbar, phase, g.wait_ns, ws.ctrl, (g.inject & kInjectNoCopy) != 0u);
             phase ^= 1u;
             if (!is_pack) {
                 read_staged_words(stage, warp, lane, w);
@@ -462,10 +454,6 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
                     }
                 }
             } else if (ENT != 1) {
-#ifdef WM_AB_D_NOP1
-                desc = 100u | (4u << 8);
-                for (int j = 0; j < 4; j++) { sm[j] = make_uint2(lane, it); pw[j].a = t; pw[j].b = e; }
-#else
                 desc = lds_now_u16(stage_s + 2u * lane);
                 const uint32_t wv = (desc >> 8) & 15u;
                 const uint32_t base_l = desc & 0xFFu, chk = desc >> 12;
@@ -500,7 +488,6 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
                         pw[j] = read_group_planes(stage_s + 8256u + 32u * (dg >> 16), (dg >> 8) & 15u, 4u * lane, 2u * lane, lane);
                     }
                 }
-#endif
             }
         } else if (e == 1u || e == 2u) {
             // a tile of zeros (nothing was shipped) or of one value (the first two bytes of its 32):
@@ -517,7 +504,10 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
         uint32_t l_e = 0, l_rel = 0, l_tk = kNone;
         unsigned long long l_po = 0;
         // (spread over three warps: the team waits for whichever warp has the most to do)
-        if (tt == 64u && !trouble) start_copy(tc->slot[(it + 1u) & 3u]);
+        // (leaf mode, rare: a tile that is scattered through the leaf table keeps the stage a little
+        // longer, see below; the next copy starts when it is done with it)
+        const bool keeps_stage = LEAVES && MODE != 1 && (o_leaf >> 63) != 0ull && e != 0u && e != 0xFFFFu;
+        if (tt == 64u && !keeps_stage) start_copy(tc->slot[(it + 1u) & 3u]);
         if (tt == 32u && t_done != kNone) ws.dig[t_done] = xor8(tc->wdig[p ^ 1u]);
         uint32_t t_look = kNone;           // warps 0 and 3: the tile claimed a step ago (two tiles ahead)
         if (leader) {                      // its table entry and offsets
@@ -536,19 +526,47 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
         // ---- phase 2: unpack, store, checksum
         bool have_digest = false;
         if (e != 0) {
-            unsigned char* o = LEAVES ? o_leaf : dst + (uint64_t)t * kTile;
+            // (leaf mode: a walked tile, bit 63 of its descriptor, is stored byte by byte through the table)
+            const bool walked = LEAVES && (o_leaf >> 63) != 0ull;
+            unsigned char* o = LEAVES ? reinterpret_cast<unsigned char*>(o_leaf) : dst + (uint64_t)t * kTile;
             bool fold = (ew >> 16) != 0;
             if (e == 0xFFFFu) {
                 const unsigned char* src = payload + tc->slot[it & 3u].src;
                 const uint32_t len = g.tail_len;
-                if (MODE != 1) for (uint32_t i = tt; i < len; i += kTeamThreads) o[i] = src[i];
+                if (MODE != 1) {
+                    if (LEAVES) {               // (the ragged tile is always a walked one)
+                        uint32_t k = (uint32_t)o_leaf;
+                        for (uint32_t i = tt; i < len; i += kTeamThreads) *leaf_byte_addr(lv, k, (unsigned long long)t * kTile + i) = src[i];
+                    } else {
+                        for (uint32_t i = tt; i < len; i += kTeamThreads) o[i] = src[i];
+                    }
+                }
                 if (MODE != 2) load_tile_words_guarded(src, len, fold, warp, lane, w);
                 fold = false;
-            } else if (is_pack && decoded) {
-#ifdef WM_AB_D_NOUNPACK
-#pragma unroll
-                for (int j = 0; j < 4; j++) { w[4 * j] = sm[j].x; w[4 * j + 1] = sm[j].y; w[4 * j + 2] = pw[j].a; w[4 * j + 3] = pw[j].b; }
-#else
+            }
+            // where the decoded words go: word i of this lane to byte 128 i of its warp's 2 KiB.  Leaf
+            // mode has two more ways besides the plain 32-bit store: a tile that starts off a four-byte
+            // boundary takes halfword or byte stores, a walked tile goes into the stage first (free:
+            // the next copy was held back) and from there byte by byte to wherever the table says.
+            unsigned char* const q = o + warp * 2048u + lane * 4u;
+            uint32_t* const sw = reinterpret_cast<uint32_t*>(stage) + warp * 512u + lane;
+            const uint32_t how = !LEAVES ? 0u : walked ? 3u : (uint32_t)(o_leaf & 3ull) == 0u ? 0u : (o_leaf & 1ull) ? 2u : 1u;
+            // (the rest of the step once per way of storing, so that the choice is made once per tile)
+            auto rest_of_step = [&](auto how_c) {
+            constexpr uint32_t HOW = decltype(how_c)::value;
+            auto put = [&](int i, uint32_t v) {
+                if (HOW == 0u) st_stream_u32(q + i * 128, v);
+                else if (HOW == 1u) { stg_u16(q + i * 128, v); stg_u16(q + i * 128 + 2, v >> 16); }
+                else if (HOW == 2u) { stg_u8(q + i * 128, v); stg_u16(q + i * 128 + 1, v >> 8); stg_u8(q + i * 128 + 3, v >> 24); }
+                else sw[i * 32] = v;
+            };
+            if (is_pack && decoded) {
+                // A coded tile goes group by group: four words are rebuilt, stored, and fed to the
+                // checksum chain (which walks the lane's sixteen words in order anyway) before the next
+                // group is touched, so only four decoded words are alive at a time and the chain's
+                // table look-ups overlap the next group's arithmetic.
+                const uint32_t fold_mask = (fold && warp == 0u && lane == 0u) ? 0xFFFFFFFFu : 0u;
+                uint32_t st = 0, last = 0;
 #pragma unroll
                 for (int j = 0; j < 4; j++) {
                     const uint32_t dg = __shfl_sync(0xFFFFFFFFu, desc, j);
@@ -573,33 +591,46 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
                     const uint32_t sa = (sm[j].x & 0xFEFEFEFEu) | (xa & 0x01010101u), sb = (sm[j].y & 0xFEFEFEFEu) | (xb & 0x01010101u);
                     const uint32_t r0 = __byte_perm(sa, ea, 0x5140), r1 = __byte_perm(sa, ea, 0x7362);
                     const uint32_t r2 = __byte_perm(sb, eb, 0x5140), r3 = __byte_perm(sb, eb, 0x7362);
-                    w[4 * j] = __funnelshift_r(r0, r0, 1);
-                    w[4 * j + 1] = __funnelshift_r(r1, r1, 1);
-                    w[4 * j + 2] = __funnelshift_r(r2, r2, 1);
-                    w[4 * j + 3] = __funnelshift_r(r3, r3, 1);
+                    const uint32_t w0 = __funnelshift_r(r0, r0, 1), w1 = __funnelshift_r(r1, r1, 1);
+                    const uint32_t w2 = __funnelshift_r(r2, r2, 1), w3 = __funnelshift_r(r3, r3, 1);
+                    if (MODE != 1) { put(4 * j, w0); put(4 * j + 1, w1); put(4 * j + 2, w2); put(4 * j + 3, w3); }
+                    if (MODE != 2) {
+                        st = chain_step(S, st ^ w0 ^ (j == 0 ? fold_mask : 0u));
+                        st = chain_step(S, st ^ w1);
+                        st = chain_step(S, st ^ w2);
+                        if (j < 3) st = chain_step(S, st ^ w3); else last = st ^ w3;
+                    }
                 }
-#endif
-            }
-            if (decoded) {
-#ifndef WM_AB_D_NOSTORE
-                if (MODE != 1 && e != 0xFFFFu) {
-                    unsigned char* q = o + warp * 2048u + lane * 4u;
-#pragma unroll
-                    for (int i = 0; i < 16; i++) st_stream_u32(q + i * 128, w[i]);
-                }
-#else
-                if (w[7] == 0x12345678u && e != 0xFFFFu) st_stream_u32(o + lane * 4u, w[2] ^ w[9] ^ w[12] ^ w[15] ^ w[0] ^ w[5]);
-#endif
                 if (MODE != 2) {
-#ifdef WM_AB_D_NOCRC
-                    const uint32_t v = w[3] ^ w[6] ^ w[8] ^ w[13] ^ w[1] ^ w[4] ^ w[10] ^ w[11] ^ w[14];
-#else
+                    const uint32_t v = warp_place(S, __reduce_xor_sync(0xFFFFFFFFu, lane_finish(S, last)), warp, lane);
+                    if (lane == 0) tc->wdig[p][warp] = v;
+                    have_digest = true;
+                }
+            } else if (decoded) {
+                // raw, zero and constant tiles and the ragged tail: the sixteen words are there already
+                if (MODE != 1 && e != 0xFFFFu) {
+#pragma unroll
+                    for (int i = 0; i < 16; i++) put(i, w[i]);
+                }
+                if (MODE != 2) {
                     const uint32_t v = tile_digest_part(S, w, fold, warp, lane);
-#endif
                     if (lane == 0) tc->wdig[p][warp] = v;
                     have_digest = true;
                 }
             }
+            };
+            if (!LEAVES || how == 0u) rest_of_step(std::integral_constant<uint32_t, 0u>());
+            else if (how == 1u) rest_of_step(std::integral_constant<uint32_t, 1u>());
+            else if (how == 2u) rest_of_step(std::integral_constant<uint32_t, 2u>());
+            else rest_of_step(std::integral_constant<uint32_t, 3u>());
+        }
+        if (keeps_stage) {
+            // (every thread of the team comes here, whatever its warp made of the tile: a warp that
+            // refused its part left that part of the stage as it was, and the call fails anyway)
+            team_bar(team);
+            stage_to_walked_tile(lv, (uint32_t)o_leaf, (unsigned long long)t * kTile, kTile, stage, tt);
+            team_bar(team);
+            if (tt == 64u) start_copy(tc->slot[(it + 1u) & 3u]);
         }
         t_done = have_digest ? t : kNone;
         if (leader && t_look < g.n_tiles) {
@@ -609,9 +640,6 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
         }
         if (tt == 96u) tc->slot[(it + 3u) & 3u].t = l_tk;      // (none once the tickets have run out)
     }
-    // a thread that gave up gives the copy it stopped waiting for one more budget to land before
-    // the block, and with it the stage, goes away
-    if (trouble && !(g.inject & kInjectNoCopy)) mbar_wait(&tc->mbar, lost, g.wait_ns);
 }
 
 // Steps 5..8: chunk CRCs of the decoded bytes against the directory, stale check, cache CRC;
@@ -619,7 +647,8 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
 __global__ void __launch_bounds__(1024)
 k_decode_finish(const unsigned char* __restrict__ wire, uint64_t wire_len, Geo g,
                 const unsigned char* __restrict__ dst, uint32_t* __restrict__ dst_crc, Ws ws,
-                const Tables* __restrict__ tab, wm_result* result, const __grid_constant__ ChunkPowers cp, uint32_t strict)
+                const Tables* __restrict__ tab, wm_result* result, const __grid_constant__ ChunkPowers cp, uint32_t strict,
+                LeafView lv)
 {
     __shared__ uint32_t sHT[1024];
     __shared__ uint32_t sT0[256];
@@ -645,10 +674,13 @@ k_decode_finish(const unsigned char* __restrict__ wire, uint64_t wire_len, Geo g
         } else if (fl & CF_PRESENT) {
             // (a chunk shorter than four bytes is checksummed byte by byte: from dst, or, in a strict
             // call, where nothing has been stored yet, from its raw copy in the wire image)
-            const unsigned char* tiny = chunk_first_byte(g, ws, dst, c);
+            const unsigned char* tiny = chunk_first_byte(g, dst, c);
             if (strict && chunk_len_dev(g, c) < 4)
                 tiny = wire + g.meta_end + *reinterpret_cast<const unsigned long long*>(dir + 16ull * c);
-            const uint32_t got = chunk_crc_staged(g, sHT, sT0, stage, ws.dig, tiny, c, threadIdx.x);
+            // (leaf mode, not strict: the tiny chunk's bytes are read back through the table)
+            const uint32_t got = (!tiny && chunk_len_dev(g, c) < 4)
+                                     ? tiny_chunk_crc_leaves(sT0, lv, (unsigned long long)c * g.chunk_bytes, (uint32_t)chunk_len_dev(g, c))
+                                     : chunk_crc_staged(g, sHT, sT0, stage, ws.dig, tiny, c, threadIdx.x);
             if (got != want) { atomicMin(&ws.ctrl->bad5_first, c); atomicAdd(&ws.ctrl->bad5_count, 1u); }
         } else {
             if (dst_crc[c] != want) { atomicMin(&ws.ctrl->bad6_first, c); atomicAdd(&ws.ctrl->bad6_count, 1u); }

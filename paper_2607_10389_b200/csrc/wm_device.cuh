@@ -25,10 +25,12 @@ namespace wm {
 constexpr uint32_t kTile = 16384;
 constexpr uint32_t kTeamThreads = 256;
 constexpr uint32_t kWordsPerLane = 16;
-// Dynamic shared memory every table-using kernel asks for: the 144 KiB image plus 79 KiB
+// Dynamic shared memory every table-using kernel asks for: the 144 KiB image plus 81 KiB
 // that the 64 KiB alignment splits into a part below and a part above the image (with the
-// window starting at 1 KiB: 63 KiB below, 16 KiB above).  227 KiB is the per-block maximum.
-constexpr uint32_t kDynSmem = kImgBytes + 0x10000 + 0x3C00;
+// window starting at 1 KiB: 63 KiB below, 18 KiB above; a stage of the leaf-mode kernels is
+// 16 bytes longer than a tile, and one of the four has to fit above).  227 KiB is the per-block
+// maximum for static and dynamic shared memory together; the kernels' static part is below 1 KiB.
+constexpr uint32_t kDynSmem = kImgBytes + 0x10000 + 0x4400;
 
 struct Smem {
     uint32_t L01, L23, LNK;      // shared-window address of A01 / A23 / NK, or'ed with lane*4
@@ -271,36 +273,30 @@ __device__ __forceinline__ void bulk_load(void* smem_dst, const void* gsrc, uint
                      ::"r"(d), "l"(gsrc), "r"(bytes), "r"(b) : "memory");
 }
 
-// Nanoseconds of the GPU's wall clock.  Every device-side wait is bounded by TIME against the
-// call's budget (Geo::wait_ns, two seconds unless the caller set another), not by a number of
-// polls: a block that shares the GPU with other work can be descheduled for a long time, and a
-// poll count says nothing about how long that was.
-__device__ __forceinline__ unsigned long long now_ns()
+// The low 32 bits of the GPU's wall clock in nanoseconds (they wrap every 4.29 s).  Every
+// device-side wait is bounded by TIME against the call's budget (Geo::wait_ns, two seconds unless
+// the caller set another, never more than four), not by a number of polls: a block that shares
+// the GPU with other work can be descheduled for a long time, and a poll count says nothing about
+// how long that was.  Differences of two readings are taken modulo 2^32, which is exact for
+// spans below the wrap.
+__device__ __forceinline__ uint32_t now_ns()
 {
-    unsigned long long t;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    uint32_t t;
+    asm volatile("mov.u32 %0, %%globaltimer_lo;" : "=r"(t));
     return t;
 }
 
 // Wait for the phase with the given parity to complete, for at most `budget_ns`.  Returns false
 // when the time ran out.  try_wait suspends the thread in hardware until the phase completes or
 // the time hint runs out, so a waiting warp does not burn issue slots that the other teams on
-// the SM need; the clock is only read after a try has come back empty.
-__device__ __forceinline__ bool mbar_wait(unsigned long long* bar, uint32_t parity, unsigned long long budget_ns)
+// the SM need.  (The waiting loop itself, wait_for_copy, follows the control block's definition.)
+__device__ __forceinline__ uint32_t mbar_try(uint32_t bar_s, uint32_t parity)
 {
-    const uint32_t b = (uint32_t)__cvta_generic_to_shared(bar);
-    unsigned long long t0 = 0;
-    for (uint32_t i = 0;; i++) {
-        uint32_t done;
-        asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-                     : "=r"(done) : "r"(b), "r"(parity), "r"(200000u) : "memory");
-        if (done) return true;
-        const unsigned long long t = now_ns();
-        if (i == 0) t0 = t;
-        else if (t - t0 > budget_ns) return false;
-    }
+    uint32_t done;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(done) : "r"(bar_s), "r"(parity), "r"(200000u) : "memory");
+    return done;
 }
-
 __device__ __forceinline__ uint64_t l2_policy_evict_first()
 {
     uint64_t pol;

@@ -50,13 +50,6 @@ __device__ __forceinline__ uint32_t ld_relaxed_u32(const uint32_t* p)
     return v;
 }
 
-// Give up: waits end early once the flag is up, and the ticket counter jumps past every tile,
-// so that nobody claims another one (claiming itself never has to look at the flag).
-__device__ __forceinline__ void raise_poison(Ctrl* ctrl)
-{
-    atomicExch(&ctrl->poison, 1u);
-    atomicMax(&ctrl->ticket, 0x7FFF0000u);
-}
 __device__ __forceinline__ uint32_t next_ticket(Ctrl* ctrl)
 {
     return atomicAdd(&ctrl->ticket, 1u);
@@ -64,21 +57,15 @@ __device__ __forceinline__ uint32_t next_ticket(Ctrl* ctrl)
 
 // Owner side: exclusive prefix (bytes) of tile t (one lane spins, for at most `budget_ns`; the
 // poison flag and the clock are looked at every 64 polls).
-__device__ __forceinline__ unsigned long long wait_prefix(const uint32_t* lbk, uint32_t t, Ctrl* ctrl, unsigned long long budget_ns)
+__device__ __forceinline__ unsigned long long wait_prefix(const uint32_t* lbk, uint32_t t, Ctrl* ctrl, uint32_t budget_ns)
 {
-    unsigned long long t0 = 0;
+    const uint32_t t0 = now_ns();
     for (uint32_t polls = 0;; polls++) {
         const uint32_t v = ld_relaxed_u32(lbk + t);
         if ((v >> 30) == 2u) return (unsigned long long)(v & kValMask) * kUnit;
-        if ((polls & 63u) == 63u) {
-            if (ld_volatile_u32(&ctrl->poison)) break;
-            const unsigned long long now = now_ns();
-            if (t0 == 0) t0 = now;
-            else if (now - t0 > budget_ns) break;
-        }
+        if ((polls & 63u) == 63u && (ld_volatile_u32(&ctrl->poison) || now_ns() - t0 > budget_ns)) break;
     }
-    atomicOr(&ctrl->err, 2u);
-    raise_poison(ctrl);
+    give_up(ctrl);
     return 0;
 }
 
@@ -87,12 +74,12 @@ __device__ __forceinline__ unsigned long long wait_prefix(const uint32_t* lbk, u
 // lane l then owns entries 16 l .. 16 l + 15 of the window.
 constexpr int kScanPerLane = 16;
 __device__ void scan_tile_lengths(uint32_t* lbk, uint32_t n_tiles, uint32_t lane, Ctrl* ctrl, uint32_t* win,
-                                  unsigned long long budget_ns)
+                                  uint32_t budget_ns)
 {
     uint64_t f = 0;                 // first unresolved entry
     uint64_t base = 0;              // units before f
     uint32_t spins = 0;             // polls in a row that resolved nothing
-    unsigned long long t0 = 0;      // the clock when that run of empty polls was first timed
+    uint32_t t0 = 0;                // the clock when that run of empty polls began
     while (f < n_tiles) {
         const uint64_t w0 = f & ~3ull;                    // 16-byte aligned window start
         const uint32_t skip = (uint32_t)(f - w0);         // entries before f (already resolved)
@@ -152,19 +139,16 @@ __device__ void scan_tile_lengths(uint32_t* lbk, uint32_t n_tiles, uint32_t lane
         if (k == 0) {
             // nothing new: the owners are behind.  Every 64 such polls in a row the scanner looks at the
             // poison flag and at the clock; it gives up when no length has come in for the whole budget.
+            if (spins == 0u) t0 = now_ns();
             if ((++spins & 63u) == 0u) {
-                bool stop = ld_volatile_u32(&ctrl->poison) != 0u;
-                const unsigned long long now = now_ns();
-                if (t0 == 0) t0 = now;
-                else if (now - t0 > budget_ns) stop = true;
+                const bool stop = ld_volatile_u32(&ctrl->poison) != 0u || now_ns() - t0 > budget_ns;
                 if (__any_sync(0xFFFFFFFFu, stop)) {
-                    if (lane == 0) { atomicOr(&ctrl->err, 2u); raise_poison(ctrl); }
+                    if (lane == 0) give_up(ctrl);
                     return;
                 }
             }
         } else {
             spins = 0;
-            t0 = 0;
         }
     }
 }
@@ -188,7 +172,7 @@ struct EncTeamCtl {
     unsigned long long excl[2];   // offset of the tile packed in the next step, by step parity
     unsigned long long mbar;      // completion of the bulk copy into the team's stage
     unsigned long long pad2;
-    const unsigned char* nptr[2]; // leaf mode: where the tile in next[] lives, by step parity
+    unsigned long long nptr[2];   // leaf mode: descriptor (k_leaf_map) of the tile in next[], by step parity
 };
 static_assert(sizeof(EncTeamCtl) % 16 == 0, "team control block keeps 16-byte alignment");
 
@@ -334,10 +318,13 @@ __device__ __forceinline__ uint32_t ent_parse_value(uint32_t buf, uint32_t s, ui
 // scanner is late, this team waits while that tile's length is not out yet; with three steps
 // of slack that is rare, and it only delays: the teams that hold earlier tiles never depend
 // on this one.
-// A tile as a team passes it round: its number in the low 30 bits, kQFirst when it is the first
-// tile of its chunk, kQPresent when its chunk is encoded; kQNone: no tile.  (The codec takes
-// caches of at most 2^21 tiles, so a number never reaches the flag bits.)
-constexpr uint32_t kQPresent = 1u << 31, kQFirst = 1u << 30, kQTile = (1u << 30) - 1u, kQNone = kQTile;
+// A tile as a team passes it round: its number in the low 22 bits, kQFirst when it is the first
+// tile of its chunk, kQPresent when its chunk is encoded; kQNone: no tile.  Leaf mode adds
+// kQWalked when the tile is read through the leaf table instead of by a bulk copy, and for the
+// others, in bits 22-25, how many bytes above a 16-byte boundary the tile starts.  (The codec
+// takes caches of at most 2^21 tiles, so a number never reaches kQNone or the other fields.)
+constexpr uint32_t kQPresent = 1u << 31, kQFirst = 1u << 30, kQWalked = 1u << 29, kQTile = (1u << 22) - 1u, kQNone = kQTile;
+constexpr uint32_t kQOffShift = 22;
 // Marks in a team's width table: on a warp's first entry, all 2 KiB of the warp's rows are zero;
 // as the sum of the widths, the tile is all zero.
 // kWarpConst: all 1024 elements of the warp's rows hold one value (its sign-mantissa byte rides in
@@ -359,7 +346,7 @@ __device__ __forceinline__ uint32_t describe_tile(const Geo& g, const uint8_t* _
 template <int TEAMS, bool MASKED, bool LEAVES, bool ZEROS, bool ENT = false>
 __global__ void __launch_bounds__(TEAMS * 256, 1)
 k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restrict__ dirty,
-         unsigned char* __restrict__ wire, uint64_t wire_cap, Ws ws, const Tables* __restrict__ tab)
+         unsigned char* __restrict__ wire, uint64_t wire_cap, Ws ws, const Tables* __restrict__ tab, LeafView lv)
 {
     extern __shared__ __align__(16) unsigned char smem[];
     // The first block to get here becomes the scanner: one warp of it, alone on its SM (a warp
@@ -387,8 +374,11 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
     const uint32_t team = threadIdx.x / kTeamThreads, tt = threadIdx.x % kTeamThreads;
     const uint32_t warp = tt / 32, lane = tt % 32;
     unsigned char* stage = nullptr;
+    // (leaf mode: a tile may start off a 16-byte boundary; its copy then starts at the boundary
+    // below and is 16 bytes longer, so the stage is too)
+    constexpr uint32_t kStage = LEAVES ? kTile + 16u : kTile;
     for (int i = 0; i < TEAMS; i++) {          // every thread carves the same blocks in the same order
-        unsigned char* p = S.take(kTile);
+        unsigned char* p = S.take(kStage);
         if ((uint32_t)i == team) stage = p;
     }
     EncTeamCtl* tc = reinterpret_cast<EncTeamCtl*>(S.take(TEAMS * sizeof(EncTeamCtl)));
@@ -417,13 +407,24 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
 
     auto is_tile = [](uint32_t q) { return (q & kQTile) != kQNone; };
     auto is_hot = [&](uint32_t q) { return q >= kQPresent && (q & kQTile) < g.n_full_tiles; };   // present and full
+    auto is_walked = [](uint32_t q) { return LEAVES && (q & kQWalked) != 0u; };
     auto publish_len = [&](uint32_t t, uint32_t len) { st_relaxed_u32(ws.lbk + t, kFlagA | (len / kUnit)); };
-    // where tile t lives: the flat cache, or (leaf mode) the table that k_leaf_map filled
-    auto tile_src = [&](uint32_t t) -> const unsigned char* {
-        return LEAVES ? ws.tptr[t] : cache + (uint64_t)t * kTile;
+    // where tile t lives: its address in the flat cache, or (leaf mode) the descriptor that k_leaf_map wrote
+    auto tile_src = [&](uint32_t t) -> unsigned long long {
+        return LEAVES ? ws.tptr[t] : reinterpret_cast<unsigned long long>(cache + (uint64_t)t * kTile);
     };
-    auto start_copy = [&](uint32_t q, const unsigned char* src) {   // thread 0 of the team, after the barrier that frees the stage
-        if (is_hot(q)) bulk_load(stage, src, kTile, &tc->mbar, pol_once);
+    // One thread of the team, after the barrier that frees the stage.  Leaf mode: a tile may start
+    // off a 16-byte boundary; the copy then starts at the boundary below and takes 16 bytes more
+    // (k_leaf_map saw to it that they belong to the leaf); the readers shift by the remainder.
+    auto start_copy = [&](uint32_t q, unsigned long long src) {
+        if (!is_hot(q) || is_walked(q)) return;
+        const unsigned long long a = LEAVES ? src & ~15ull : src;
+        bulk_load(stage, reinterpret_cast<const void*>(a), (LEAVES && a != src) ? kTile + 16u : kTile, &tc->mbar, pol_once);
+    };
+    // leaf mode, handing a claimed tile on: its word carries the walked mark or the start's remainder
+    auto with_mark = [](uint32_t q, unsigned long long desc) {
+        if (!LEAVES || (q & kQTile) == kQNone) return q;
+        return (desc >> 63) ? q | kQWalked : q | (((uint32_t)desc & 15u) << kQOffShift);
     };
 
     // Tiles in flight, oldest first: X (packed in this step), V, W (waiting for their offsets),
@@ -452,8 +453,10 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
         tc->excl[0] = 0ull;
         tc->excl[1] = 0ull;
         if (LEAVES) {
-            tc->nptr[0] = is_tile(q0) ? tile_src(q0 & kQTile) : nullptr;
-            tc->nptr[1] = is_tile(q1) ? tile_src(q1 & kQTile) : nullptr;
+            tc->nptr[0] = is_tile(q0) ? tile_src(q0 & kQTile) : 0ull;
+            tc->nptr[1] = is_tile(q1) ? tile_src(q1 & kQTile) : 0ull;
+            tc->next[0] = with_mark(q0, tc->nptr[0]);
+            tc->next[1] = with_mark(q1, tc->nptr[1]);
             if (claiming) { qA = describe_tile<MASKED>(g, dirty, next_ticket(ws.ctrl)); claiming = is_tile(qA); }
         }
     }
@@ -461,21 +464,34 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
     qY = tc->next[0];
     if (leader) start_copy(qY, LEAVES ? tc->nptr[0] : tile_src(qY & kQTile));
 
-    uint32_t trouble = 0;              // sticky: 1 the image does not fit, 2 a copy did not arrive within the budget
-    uint32_t lost = 0;                 // the stage's phase that never completed
+    uint32_t trouble = 0;              // sticky: the image does not fit
     while (((qX & qV & qW & qY) & kQTile) != kQNone) {
         const bool hotY = is_hot(qY);
+        if (LEAVES && is_tile(qY) && qY >= kQPresent && (is_walked(qY) || !hotY)) {
+            // leaf mode, rare: a tile that crosses leaves (no copy was started for it) or the ragged last
+            // tile is gathered into the stage byte by byte; from there it goes the ordinary way
+            const uint32_t tY = qY & kQTile;
+            walked_tile_to_stage(lv, (uint32_t)ws.tptr[tY], (unsigned long long)tY * kTile, hotY ? kTile : tile_left(g, tY), stage, tt);
+            team_bar(team);
+        }
         if (hotY) {
-            // (after one wait has run out the thread waits for no other copy and the team starts none:
-            // the call has failed, the tickets are withdrawn, what is left is to get out quickly)
-            if (!(trouble & 2u) && !mbar_wait(&tc->mbar, phase, g.wait_ns)) {
-                trouble |= 2u;
-                lost = phase;
-                if (lane == 0) { atomicOr(&ws.ctrl->err, 2u); raise_poison(ws.ctrl); }
+            if (!is_walked(qY)) {
+                wait_for_copy<!ENT>(&tc->mbar, phase, g.wait_ns, ws.ctrl);
+                phase ^= 1u;
             }
-            phase ^= 1u;
+            // leaf mode: a tile that was copied from the 16-byte boundary below it starts that many
+            // bytes into the stage (0 for a walked tile): whole words from a quarter of that on, each
+            // put together from two neighbours when the remainder is no multiple of four
+            const uint32_t off = LEAVES ? (qY >> kQOffShift) & 15u : 0u;
+            const uint32_t sh = (off & 3u) * 8u;
+            const uint32_t* const p = my_words + (off >> 2);
+            if (LEAVES && sh) {
 #pragma unroll
-            for (int i = 0; i < 16; i++) d[i] = my_words[i * 32];
+                for (int i = 0; i < 16; i++) d[i] = __funnelshift_r(p[i * 32], p[i * 32 + 1], sh);
+            } else {
+#pragma unroll
+                for (int i = 0; i < 16; i++) d[i] = p[i * 32];
+            }
         }
         team_bar(team);                   // stage free; what the leader left at the end of the last step is visible
         const uint32_t qN = tc->next[par ^ 1u];
@@ -486,8 +502,8 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
         // step: the ticket of the tile to measure two steps on (warp 0, the leader) and the offset
         // of the tile to pack in the next step (warp 3).  Warp 1 notes what is left about X.
         uint32_t pv = 0, tk = 0xFFFFFFFFu;
-        const unsigned char* pA = nullptr;
-        if (tt == 64u && !(trouble & 2u)) start_copy(qN, LEAVES ? tc->nptr[par ^ 1u] : tile_src(qN & kQTile));
+        unsigned long long pA = 0;
+        if (tt == 64u) start_copy(qN, LEAVES ? tc->nptr[par ^ 1u] : tile_src(qN & kQTile));
         if (tt == 96u && is_tile(qV)) pv = ld_relaxed_u32(ws.lbk + (qV & kQTile));
         if (leader) {
             if (claiming) tk = next_ticket(ws.ctrl);
@@ -596,7 +612,8 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
             const bool present = qY >= kQPresent;
             if (tt == 0) publish_len(tYn, present ? tile_left(g, tYn) : 0u);
             if (present) {
-                load_tile_words_guarded(tile_src(tYn), tile_left(g, tYn), (qY & kQFirst) != 0, warp, lane, d);
+                // (leaf mode: the tile's bytes were gathered into the stage above)
+                load_tile_words_guarded(LEAVES ? stage : cache + (uint64_t)tYn * kTile, tile_left(g, tYn), (qY & kQFirst) != 0, warp, lane, d);
                 const uint32_t v = tile_digest_part(S, d, false, warp, lane);
                 if (lane == 0) tc->wdig[slY][warp] = v;
             }
@@ -719,9 +736,14 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
             if (exclX + enc_len > room) {
                 trouble |= 1u;
             } else {
-                const unsigned char* src = tile_src(tXn);
                 unsigned char* dst = payload + exclX;
-                for (uint32_t i = tt; i < enc_len; i += kTeamThreads) dst[i] = src[i];
+                if (LEAVES) {
+                    uint32_t k = (uint32_t)ws.tptr[tXn];               // (the ragged tile is always a walked one)
+                    for (uint32_t i = tt; i < enc_len; i += kTeamThreads) dst[i] = *leaf_byte_addr(lv, k, (unsigned long long)tXn * kTile + i);
+                } else {
+                    const unsigned char* src = cache + (uint64_t)tXn * kTile;
+                    for (uint32_t i = tt; i < enc_len; i += kTeamThreads) dst[i] = src[i];
+                }
             }
         }
 
@@ -753,8 +775,8 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
         if (leader) {
             uint32_t qn2 = kQNone;
             if (claiming) { qn2 = describe_tile<MASKED>(g, dirty, tk); claiming = is_tile(qn2); }
-            if (LEAVES) {              // hand over the tile whose address arrived during this step
-                tc->next[par] = qA;
+            if (LEAVES) {              // hand over the tile whose descriptor arrived during this step
+                tc->next[par] = with_mark(qA, pA);
                 tc->nptr[par] = pA;
                 qA = qn2;
             } else {
@@ -773,9 +795,6 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
         step++;
     }
     if ((trouble & 1u) && lane == 0) atomicOr(&ws.ctrl->err, 1u);
-    // a thread that gave up gives the copy it stopped waiting for one more budget to land before
-    // the block, and with it the stage, goes away
-    if (trouble & 2u) mbar_wait(&tc->mbar, lost, g.wait_ns);
     // every warp is done with its tensor memory: hand it back before the block exits
     tmem_fence_before_sync();
     __syncthreads();
@@ -787,7 +806,7 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
 __global__ void __launch_bounds__(1024)
 k_encode_finish(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restrict__ dirty,
                 uint32_t* __restrict__ crc_inout, unsigned char* __restrict__ wire, Ws ws,
-                const Tables* __restrict__ tab, const __grid_constant__ ChunkPowers cp, uint32_t option_flags)
+                const Tables* __restrict__ tab, const __grid_constant__ ChunkPowers cp, uint32_t option_flags, LeafView lv)
 {
     __shared__ uint32_t sHT[1024];
     __shared__ uint32_t sT0[256];
@@ -810,7 +829,9 @@ k_encode_finish(const unsigned char* __restrict__ cache, Geo g, const uint8_t* _
         present = (!dirty || dirty[c]) ? 1u : 0u;
         uint32_t crc;
         if (present) {
-            crc = chunk_crc_staged(g, sHT, sT0, stage, ws.dig, chunk_first_byte(g, ws, cache, c), c, threadIdx.x);
+            // (leaf mode: a last chunk shorter than four bytes is checksummed byte by byte through the table)
+            if (!cache && chunk_len_dev(g, c) < 4) crc = tiny_chunk_crc_leaves(sT0, lv, (unsigned long long)c * g.chunk_bytes, (uint32_t)chunk_len_dev(g, c));
+            else crc = chunk_crc_staged(g, sHT, sT0, stage, ws.dig, chunk_first_byte(g, cache, c), c, threadIdx.x);
             crc_inout[c] = crc;
         } else {
             crc = crc_inout[c];

@@ -13,6 +13,7 @@
 #include <cstring>
 #include <atomic>
 #include <mutex>
+#include <type_traits>
 
 #include <cuda_runtime.h>
 
@@ -184,7 +185,7 @@ void wm_timing_enable(int on) { g_timing = on != 0; }
 void wm_zero_tiles_enable(int on) { g_zero_tiles = on != 0; }
 void wm_entropy_enable(int on) { g_entropy = on != 0; }
 
-void wm_wait_budget_ms(uint32_t ms) { g_wait_ns = (uint64_t)(ms ? ms : 1u) * 1000000ull; }
+void wm_wait_budget_ms(uint32_t ms) { g_wait_ns = (ms == 0u ? 1u : ms > 4000u ? 4000u : ms) * 1000000u; }
 void wm_inject_stall(int on) { g_inject = on ? (kInjectNoScanner | kInjectNoCopy) : 0u; }
 
 wm_status wm_workspace_status(const void* workspace, void* stream)
@@ -412,6 +413,7 @@ static wm_status encode_any(const void* cache, const wm_leaf* leaves, uint32_t n
     Ws ws = ws_carve(workspace, g);
     const unsigned char* c = static_cast<const unsigned char*>(cache);
     unsigned char* w = static_cast<unsigned char*>(wire);
+    const LeafView lv = {leaves, ws.lstart, leaves ? n_leaves : 0u};
     const uint32_t init_blocks = (g.n_tiles + 1023) / 1024 < 1024 ? (g.n_tiles + 1023) / 1024 : 1024;
     k_encode_init<<<init_blocks ? init_blocks : 1, 1024, 0, s>>>(g, ws, w);
     if (leaves) {
@@ -427,7 +429,7 @@ static wm_status encode_any(const void* cache, const wm_leaf* leaves, uint32_t n
     {
         MainKernelTimer timer(ds, 2, s);
         const int variant = (dirty ? 1 : 0) | (leaves ? 2 : 0) | (opt_zero ? 4 : 0) | (opt_ent ? 8 : 0);
-        auto go = [&](auto kernel) { launch_after(kernel, grid, kTeams * 256, kDynSmem, s, c, g, dirty, w, wire_cap, ws, ds->tables); };
+        auto go = [&](auto kernel) { launch_after(kernel, grid, kTeams * 256, kDynSmem, s, c, g, dirty, w, wire_cap, ws, ds->tables, lv); };
         switch (variant) {
             case 0: go(k_encode<kTeams, false, false, false>); break;
             case 1: go(k_encode<kTeams, true, false, false>); break;
@@ -448,7 +450,7 @@ static wm_status encode_any(const void* cache, const wm_leaf* leaves, uint32_t n
         }
     }
     launch_after(k_encode_finish, (g.n_chunks + g.finish_cb - 1) / g.finish_cb, 1024, 0, s, c, g, dirty, crc_inout, w, ws, ds->tables,
-                 chunk_powers(g), (opt_ent ? 4u : 0u) | (opt_zero ? 2u : 0u));
+                 chunk_powers(g), (opt_ent ? 4u : 0u) | (opt_zero ? 2u : 0u), lv);
     launch_after(k_meta_crc, (g.n_meta_slices + 3) / 4, 1024, kDynSmem, s, w, g, ws, ds->tables, result);
     g_launches = leaves ? 5 : 4;
     return launch_status();
@@ -492,6 +494,7 @@ static wm_status decode_any(const void* wire, uint64_t wire_len, void* dst, cons
     Ws ws = ws_carve(workspace, g);
     const unsigned char* w = static_cast<const unsigned char*>(wire);
     unsigned char* d = static_cast<unsigned char*>(dst);
+    const LeafView lv = {leaves, ws.lstart, leaves ? n_leaves : 0u};
     k_decode_init<<<1, 64, 0, s>>>(ws);
     if (leaves) {
         const uint32_t map_blocks = (g.n_tiles + 4095) / 4096 < 64 ? (g.n_tiles + 4095) / 4096 : 64;
@@ -506,8 +509,8 @@ static wm_status decode_any(const void* wire, uint64_t wire_len, void* dst, cons
     uint32_t grid = need < (uint32_t)ds->sm_count ? need : (uint32_t)ds->sm_count;
     if (block_cap && grid > block_cap) grid = block_cap;
     auto pass = [&](auto flat_kernel, auto leaf_kernel) {
-        if (leaves) launch_after(leaf_kernel, grid, kTeamsPlain * 256, kDynSmem, s, w, g, d, ws, ds->tables);
-        else launch_after(flat_kernel, grid, kTeamsPlain * 256, kDynSmem, s, w, g, d, ws, ds->tables);
+        if (leaves) launch_after(leaf_kernel, grid, kTeamsPlain * 256, kDynSmem, s, w, g, d, ws, ds->tables, lv);
+        else launch_after(flat_kernel, grid, kTeamsPlain * 256, kDynSmem, s, w, g, d, ws, ds->tables, lv);
     };
     {
         MainKernelTimer timer(ds, 3, s);
@@ -520,7 +523,7 @@ static wm_status decode_any(const void* wire, uint64_t wire_len, void* dst, cons
         }
     }
     launch_after(k_decode_finish, (g.n_chunks + g.finish_cb - 1) / g.finish_cb, 1024, 0, s, w, wire_len, g, d, dst_crc_inout, ws, ds->tables,
-                 result, chunk_powers(g), strict ? 1u : 0u);
+                 result, chunk_powers(g), strict ? 1u : 0u, lv);
     if (strict) {
         if (ent) { pass(k_decode<kTeamsPlain, false, 2, 1>, k_decode<kTeamsPlain, true, 2, 1>); pass(k_decode<kTeamsPlain, false, 2, 2>, k_decode<kTeamsPlain, true, 2, 2>); }
         else pass(k_decode<kTeamsPlain, false, 2>, k_decode<kTeamsPlain, true, 2>);

@@ -25,7 +25,7 @@ struct Geo {
     uint32_t finish_cb;       // chunks handled by one block of the finish kernels
     uint32_t poly;            // reflected CRC polynomial of the k_* powers (CRC32C except in wm_checksum_poly)
     uint32_t inject;          // test hook (wm_inject_stall): kInject* bits, 0 in normal operation
-    uint64_t wait_ns;         // budget of every device-side wait (wm_wait_budget_ms)
+    uint32_t wait_ns;         // budget of every device-side wait (wm_wait_budget_ms; at most 4 s, see now_ns)
 };
 // Geo::inject.  What a bounded wait waits for is left out, so that the wait runs out and the
 // give-up path can be tested without a fault: the scanner warp returns at once (encode), the bulk
@@ -64,6 +64,55 @@ struct Ctrl {                 // first 256 bytes of the workspace
 };
 static_assert(sizeof(Ctrl) == 256, "control block is 256 bytes");
 
+// Give up: the call has failed.  The error word says why (bit 1: a wait ran out), waits end early
+// once the poison flag is up, and the ticket counter jumps past every tile, so that nobody claims
+// another one (claiming itself never has to look at a flag).
+__device__ __forceinline__ void give_up(Ctrl* ctrl)
+{
+    atomicOr(&ctrl->err, 2u);
+    atomicExch(&ctrl->poison, 1u);
+    atomicMax(&ctrl->ticket, 0x7FFF0000u);
+}
+
+// Wait for a bulk copy into a stage: the phase of `bar` with the given parity, for at most
+// `budget_ns`.  A copy is started a whole step before it is needed, so the first try nearly
+// always succeeds, and everything else happens only after a try has come back empty: the clock is
+// read, and when the budget has passed the thread gives up for the whole call, then gives the
+// copy one more budget to land (so that the block, and with it the stage, does not go away under
+// a copy still in flight) and returns false.  A thread that comes here after the call has been
+// given up makes its one try and no more.  `no_second`: test hook, no copy is in flight.
+// What follows a first try that came back empty.
+__device__ __forceinline__ bool wait_for_copy_rest(uint32_t b, uint32_t parity, uint32_t budget_ns, Ctrl* ctrl, bool no_second)
+{
+    if (*reinterpret_cast<volatile uint32_t*>(&ctrl->err) & 2u) return false;
+    uint32_t t0 = now_ns();
+    do {
+        if (mbar_try(b, parity)) return true;
+    } while (now_ns() - t0 <= budget_ns);
+    give_up(ctrl);
+    if (no_second) return false;
+    t0 = now_ns();
+    do {
+        if (mbar_try(b, parity)) break;
+    } while (now_ns() - t0 <= budget_ns);
+    return false;
+}
+__device__ __noinline__ bool wait_for_copy_rest_call(uint32_t b, uint32_t parity, uint32_t budget_ns, Ctrl* ctrl, bool no_second)
+{
+    return wait_for_copy_rest(b, parity, budget_ns, ctrl, no_second);
+}
+// OUT_OF_LINE: the rest is a call.  Which form is faster differs from kernel to kernel (it decides
+// how the compiler lays out the hot loop around it); each kernel takes the one measured better.
+template <bool OUT_OF_LINE>
+__device__ __forceinline__ bool wait_for_copy(unsigned long long* bar, uint32_t parity, uint32_t budget_ns, Ctrl* ctrl,
+                                              bool no_second = false)
+{
+    const uint32_t b = (uint32_t)__cvta_generic_to_shared(bar);
+    if (mbar_try(b, parity)) return true;
+    return OUT_OF_LINE ? wait_for_copy_rest_call(b, parity, budget_ns, ctrl, no_second)
+                       : wait_for_copy_rest(b, parity, budget_ns, ctrl, no_second);
+}
+
 struct Ws {
     Ctrl* ctrl;
     uint32_t* lbk;               // [n_tiles] placement look-back words
@@ -72,15 +121,17 @@ struct Ws {
     uint32_t* cflag;             // [n_chunks] bit0 present, bit1..: failed step 3/4/5/6
     uint32_t* ccrc;              // [n_chunks]
     uint32_t* mdig;              // [n_meta_slices]
-    unsigned char** tptr;        // [n_tiles] leaf mode: where each tile of the logical cache lives
+    unsigned long long* tptr;    // [n_tiles] leaf mode: where each tile of the logical cache lives (see k_leaf_map)
+    unsigned long long* lstart;  // [kMaxLeaves + 1] leaf mode: logical offset at which each leaf starts
 };
+constexpr uint32_t kMaxLeaves = 4096;
 
 constexpr uint32_t CF_PRESENT = 1, CF_BAD3 = 2, CF_BAD4 = 4, CF_BAD5 = 8, CF_BAD6 = 16;
 
 static inline uint64_t align16(uint64_t v) { return (v + 15) & ~(uint64_t)15; }
 
 struct WsLayout {
-    uint64_t state, dig, rel, cflag, ccrc, mdig, tptr, total;
+    uint64_t state, dig, rel, cflag, ccrc, mdig, tptr, lstart, total;
 };
 
 static WsLayout ws_layout(const Geo& g)
@@ -94,6 +145,7 @@ static WsLayout ws_layout(const Geo& g)
     L.ccrc = o;  o = align16(o + 4ull * g.n_chunks);
     L.mdig = o;  o = align16(o + 4ull * g.n_meta_slices);
     L.tptr = o;  o = align16(o + 8ull * g.n_tiles);
+    L.lstart = o; o = align16(o + 8ull * (kMaxLeaves + 1));
     L.total = o;
     return L;
 }
@@ -110,7 +162,8 @@ static Ws ws_carve(void* base, const Geo& g)
     w.cflag = reinterpret_cast<uint32_t*>(b + L.cflag);
     w.ccrc = reinterpret_cast<uint32_t*>(b + L.ccrc);
     w.mdig = reinterpret_cast<uint32_t*>(b + L.mdig);
-    w.tptr = reinterpret_cast<unsigned char**>(b + L.tptr);
+    w.tptr = reinterpret_cast<unsigned long long*>(b + L.tptr);
+    w.lstart = reinterpret_cast<unsigned long long*>(b + L.lstart);
     return w;
 }
 
@@ -122,7 +175,7 @@ constexpr uint32_t kFinishDigests = 8192;    // tile digests a finish block stag
 constexpr uint32_t kFinishChunks = 128;      // at most this many chunks per finish block
 
 // Process-wide settings every call reads when it is issued (atomics: calls come from any thread).
-static std::atomic<uint64_t> g_wait_ns{2000ull * 1000ull * 1000ull};    // wm_wait_budget_ms
+static std::atomic<uint32_t> g_wait_ns{2000u * 1000u * 1000u};         // wm_wait_budget_ms
 static std::atomic<uint32_t> g_inject{0};                               // wm_inject_stall
 
 static bool make_geo_fixed(uint64_t nbytes, uint32_t chunk_bytes, Geo& g);
@@ -223,12 +276,11 @@ __device__ __forceinline__ uint32_t xor8(const uint32_t* p)
     return p[0] ^ p[1] ^ p[2] ^ p[3] ^ p[4] ^ p[5] ^ p[6] ^ p[7];
 }
 
-// First byte of chunk c: in the flat buffer, or (leaf mode, flat == nullptr) where the chunk's
-// first tile lives.  Only chunks shorter than four bytes are ever read through it.
-__device__ __forceinline__ const unsigned char* chunk_first_byte(const Geo& g, const Ws& ws, const unsigned char* flat, uint32_t c)
+// First byte of chunk c in the flat buffer (nullptr in leaf mode, where the finish kernels walk
+// the leaf table instead).  Only chunks shorter than four bytes are ever read through it.
+__device__ __forceinline__ const unsigned char* chunk_first_byte(const Geo& g, const unsigned char* flat, uint32_t c)
 {
-    if (flat) return flat + (uint64_t)c * g.chunk_bytes;
-    return chunk_len_dev(g, c) < 4 ? ws.tptr[(uint64_t)c * g.tiles_per_chunk] : nullptr;
+    return flat ? flat + (uint64_t)c * g.chunk_bytes : nullptr;
 }
 
 // CRC32C of chunk c from its tiles' digests (Horner over tiles; the all-ones init was folded

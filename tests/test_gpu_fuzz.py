@@ -92,11 +92,12 @@ def test_random_case_matches_the_oracle(seed):
         wm.entropy_enable(False)
 
 
-@pytest.mark.parametrize("seed", range(16))
+@pytest.mark.parametrize("seed", range(32))
 def test_random_leaf_tables_match_the_flat_image(seed):
-    """The cache cut into leaves at random tile boundaries (the last leaf may be ragged), every
-    option set, with and without a mask: the image is the oracle's image of the concatenation and
-    the decode lands in a second, differently cut set of leaves."""
+    """The cache cut into leaves at random places (tile boundaries, 16-, 4-, 2-byte and odd
+    offsets, runs of tiny leaves), every option set, with and without a mask: the image is the
+    oracle's image of the concatenation and the decode lands in a second, differently cut set of
+    leaves."""
     import torch
     from paper_2607_10389_b200 import binding as wm
     rng = np.random.default_rng(3000 + seed)
@@ -111,8 +112,16 @@ def test_random_leaf_tables_match_the_flat_image(seed):
     want, want_crc, want_res = oracle.encode(a, chunk, dirty=dirty, crc_in=stale, zero_tiles=bool(opt & 1), entropy=bool(opt & 2))
 
     def cut(k):
-        edges = sorted(set(int(x) for x in rng.integers(1, nt, k))) if nt > 1 else []
-        bounds = [0] + [e * TILE for e in edges] + [n]
+        # granularity of the cut positions: whole tiles (as an engine's large tensors), or any
+        # multiple of 16 / 4 / 2 / 1 bytes; now and then a run of tiny leaves (scalar flags)
+        gran = int(rng.choice([TILE, 16, 4, 2, 1]))
+        edges = set(int(x) * gran for x in rng.integers(1, max(2, n // gran), k))
+        if rng.integers(0, 2):
+            o = int(rng.integers(1, n - 200))
+            for size in rng.choice([1, 2, 4, 8, 64], int(rng.integers(1, 12))):
+                o += int(size)
+                edges.add(o)
+        bounds = [0] + sorted(e for e in edges if 0 < e < n) + [n]
         return [(bounds[i], bounds[i + 1]) for i in range(len(bounds) - 1) if bounds[i + 1] > bounds[i]]
 
     src = [torch.from_numpy(a[lo:hi].copy()).cuda() for lo, hi in cut(int(rng.integers(1, 9)))]

@@ -37,12 +37,17 @@ def test_oracle_leaf_calls_are_the_flat_calls_on_the_concatenation():
 gpu = pytest.mark.gpu
 
 
-def _setup(nbytes, chunk, cuts, seed):
+def _setup(nbytes, chunk, cuts, seed, byte_cuts=False):
     import torch
     from paper_2607_10389_b200 import binding as wm
     g = torch.Generator(device="cuda").manual_seed(seed)
     flat = torch.randn(((nbytes + 1) // 2,), generator=g, device="cuda").to(torch.bfloat16).view(torch.uint8)[:nbytes].contiguous()
-    sizes = split_sizes(nbytes, cuts)
+    if byte_cuts:
+        edges = [0] + list(cuts) + [nbytes]
+        sizes = [b - a for a, b in zip(edges[:-1], edges[1:])]
+    else:
+        sizes = split_sizes(nbytes, cuts)
+    assert all(n > 0 for n in sizes) and sum(sizes) == nbytes
     leaves, o = [], 0
     for n in sizes:                      # separate allocations, as an engine's tensors are
         leaves.append(flat[o:o + n].clone())
@@ -50,15 +55,44 @@ def _setup(nbytes, chunk, cuts, seed):
     return torch, wm, flat, leaves
 
 
+def _flags(start, sizes):
+    """Cut positions of a run of small leaves that starts at byte `start`."""
+    out, o = [], start
+    for n in sizes:
+        out.append(o)
+        o += n
+    out.append(o)
+    return out
+
+
+LEAF_CASES = [
+    # leaves that are whole tiles (every tile moves by an aligned bulk copy)
+    (5 * 65536 + 3 * TILE + 1000, 65536, [t * TILE for t in (1, 2, 9, 17)]),       # ragged last leaf, chunks straddle leaves
+    (40 * TILE, 8 * TILE, [t * TILE for t in (8, 16, 24, 32)]),                    # leaves on chunk boundaries
+    (64 * TILE, 65536, [t * TILE for t in range(1, 64)]),                          # one tile per leaf
+    (3 * TILE + 2, 65536, []),                                                     # a single leaf
+    # leaves of any size: the tile grid falls anywhere inside them
+    (23 * TILE + 200, 65536, [3 * TILE + 16, 11 * TILE + 4096 + 32]),              # 16-byte remainders
+    (23 * TILE + 200, 65536, [3 * TILE + 8, 11 * TILE + 4096 + 12]),               # 8 and 4-byte remainders
+    (23 * TILE + 200, 65536, [3 * TILE + 2, 11 * TILE + 4096 + 6]),                # even remainders
+    (23 * TILE + 201, 65536, [3 * TILE + 1, 11 * TILE + 4096 + 7]),                # odd remainders
+    # scalar flags between tensors: runs of tiny leaves, a tile that crosses many of them
+    (30 * TILE, 4 * TILE, _flags(5 * TILE + 100, [8, 8, 1, 2, 64, 4]) + _flags(17 * TILE - 20, [8] * 6)),
+    (12 * TILE + 77, 2 * TILE, _flags(16, [1] * 40) + [7 * TILE - 1, 7 * TILE + 1]),
+    (6 * TILE, 65536, list(range(1, 200))),                                        # 199 one-byte leaves, then one large one
+    # a last chunk shorter than four bytes, spread over three one-byte leaves
+    (2 * 65536 + 3, 65536, [65536 + 5, 2 * 65536, 2 * 65536 + 1, 2 * 65536 + 2]),
+    # a leaf whose size is no multiple of 16 and ends exactly on the tile grid (its last tile is walked)
+    (9 * TILE, 65536, [8, 5 * TILE]),
+]
+
+
 @gpu
-@pytest.mark.parametrize("nbytes,chunk,cuts", [
-    (5 * 65536 + 3 * TILE + 1000, 65536, [1, 2, 9, 17]),       # ragged last leaf, chunks straddle leaves
-    (40 * TILE, 8 * TILE, [8, 16, 24, 32]),                    # leaves on chunk boundaries
-    (64 * TILE, 65536, list(range(1, 64))),                    # one tile per leaf
-    (3 * TILE + 2, 65536, []),                                 # a single leaf
-])
-def test_leaf_encode_and_decode_match_the_oracle(nbytes, chunk, cuts):
-    torch, wm, flat, leaves = _setup(nbytes, chunk, cuts, seed=nbytes % 1000)
+@pytest.mark.parametrize("nbytes,chunk,cuts", LEAF_CASES)
+@pytest.mark.parametrize("options", [0, 3])
+def test_leaf_encode_and_decode_match_the_oracle(nbytes, chunk, cuts, options):
+    torch, wm, flat, leaves = _setup(nbytes, chunk, cuts, seed=nbytes % 1000, byte_cuts=True)
+    kw = {"zero_tiles": True, "entropy": True} if options else {}
     nc = wm.num_chunks(nbytes, chunk)
     ws = wm.new_workspace(nbytes, chunk)
     cap = wm.wire_bound(nbytes, chunk)
@@ -66,12 +100,12 @@ def test_leaf_encode_and_decode_match_the_oracle(nbytes, chunk, cuts):
     table = wm.make_leaf_table(leaves)
     for dirty_np in (None, (np.arange(nc) % 3 != 1).astype(np.uint8)):
         crc_in = (np.arange(nc, dtype=np.uint64) * 2654435761 % (1 << 32)).astype(np.uint32)
-        want_wire, want_crc, want = oracle.encode_leaves([x.cpu().numpy() for x in leaves], chunk, dirty=dirty_np,
-                                                          crc_in=crc_in.astype(np.uint32))
+        want_wire, want_crc, want = oracle.encode(oracle.flatten_leaves([x.cpu().numpy() for x in leaves]), chunk, dirty=dirty_np,
+                                                  crc_in=crc_in.astype(np.uint32), **kw)
         wire = torch.full((cap + 64,), 0xA5, dtype=torch.uint8, device="cuda")
         crc = torch.from_numpy(crc_in.astype(np.uint32).view(np.int32).copy()).cuda()
         dirty = None if dirty_np is None else torch.from_numpy(dirty_np).cuda()
-        wm.wm_encode_leaves(table, nbytes, chunk, dirty, crc, wire, ws, res, wire_cap=cap)
+        wm.wm_encode_opt(None, chunk, dirty, crc, wire[:cap], ws, res, options, leaf_table=table, nbytes=nbytes)
         r = wm.read_result(res)
         assert (r.status, r.wire_len, r.n_present, r.cache_crc) == (want.status, want.wire_len, want.n_present, want.cache_crc)
         got = wire.cpu().numpy()
@@ -80,28 +114,37 @@ def test_leaf_encode_and_decode_match_the_oracle(nbytes, chunk, cuts):
         # the flat call gives the same image
         wire2 = torch.zeros(cap, dtype=torch.uint8, device="cuda")
         crc2 = torch.from_numpy(crc_in.astype(np.uint32).view(np.int32).copy()).cuda()
-        wm.wm_encode(flat, chunk, dirty, crc2, wire2, ws, res)
+        wm.wm_encode_opt(flat, chunk, dirty, crc2, wire2, ws, res, options)
         assert torch.equal(wire2[: r.wire_len], wire[: r.wire_len])
 
-        # decode into fresh leaves that hold the old content of the absent chunks
+        # decode into fresh leaves that hold the old content of the absent chunks; canary bytes
+        # behind every destination leaf must stay as they are
         old = flat.clone()
         if dirty_np is not None:
             for c in np.nonzero(dirty_np)[0]:
                 old[c * chunk: min((c + 1) * chunk, nbytes)] = 0x11
-        dst_leaves, o = [], 0
+        dst_store, dst_leaves, o = [], [], 0
         for x in leaves:
-            dst_leaves.append(old[o:o + x.numel()].clone())
+            buf = torch.full((x.numel() + 32,), 0xC3, dtype=torch.uint8, device="cuda")
+            buf[: x.numel()] = old[o:o + x.numel()]
+            dst_store.append(buf)
+            dst_leaves.append(buf[: x.numel()])
             o += x.numel()
         dtable = wm.make_leaf_table(dst_leaves)
-        dcrc = crc.clone()
-        wm.wm_decode_verify_leaves(wire, r.wire_len, dtable, nbytes, chunk, dcrc, ws, res)
-        rd = wm.read_result(res)
-        assert rd.ok and rd.cache_crc == want.cache_crc
-        assert all(torch.equal(a, b) for a, b in zip(dst_leaves, leaves))
-        # one flipped payload bit is caught on the way into the leaves
+        for strict in (0, wm.OPT_STRICT):
+            dcrc = crc.clone()
+            wm.wm_decode_verify_opt(wire, r.wire_len, None, chunk, dcrc, ws, res, (options & 2) | strict, leaf_table=dtable, nbytes=nbytes)
+            rd = wm.read_result(res)
+            assert rd.ok and rd.cache_crc == want.cache_crc
+            assert all(torch.equal(a, b) for a, b in zip(dst_leaves, leaves))
+            assert all(bool((b[-32:] == 0xC3).all()) for b in dst_store), "wrote past the end of a leaf"
+        # one flipped payload bit on the way into the leaves: the oracle's verdict on the same image
         wire[r.wire_len - 5] ^= 4
-        wm.wm_decode_verify_leaves(wire, r.wire_len, dtable, nbytes, chunk, dcrc, ws, res)
-        assert wm.read_result(res).status_name == "ERR_CHUNK_CRC"
+        wm.wm_decode_verify_opt(wire, r.wire_len, None, chunk, dcrc, ws, res, options & 2, leaf_table=dtable, nbytes=nbytes)
+        _, _, o_res = oracle.decode_verify(wire[: r.wire_len].cpu().numpy(), nbytes, chunk, dst=old.cpu().numpy(),
+                                           dst_crc=crc.cpu().numpy().view(np.uint32), expect_entropy=bool(options & 2))
+        rd = wm.read_result(res)
+        assert (rd.status, rd.first_bad_chunk, rd.n_bad_chunks) == (o_res.status, o_res.first_bad_chunk, o_res.n_bad_chunks)
 
 
 @gpu
@@ -118,13 +161,16 @@ def test_leaf_table_that_breaks_the_rules_is_rejected():
     r = wm.read_result(res)
     assert r.ok
     bad_tables = []
-    t = good.clone(); t[0, 1] -= 16; t[1, 1] += 16; bad_tables.append(t)          # a middle leaf that is not whole tiles
     t = good.clone(); t[2, 1] += TILE; bad_tables.append(t)                        # sizes do not add up
     t = good.clone(); t[1, 0] += 4; bad_tables.append(t)                           # misaligned leaf
     t = good.clone(); t[1, 1] = 0; bad_tables.append(t)                            # empty leaf
+    t = good.clone(); t[1, 0] = 0; bad_tables.append(t)                            # null leaf
+    # two sizes that wrap around 2^64 to the right total: -16384 and what is left + 16384
+    t = good.clone(); t[0, 1] = -TILE; t[1, 1] = int(good[0, 1]) + int(good[1, 1]) + TILE; bad_tables.append(t)
     for t in bad_tables:
         wm.wm_encode_leaves(t, nbytes, chunk, None, crc, wire, ws, res)
         assert wm.read_result(res).status_name == "ERR_ARG"
+        assert wm.workspace_status(ws) == -1
     # decode: a bad destination table is refused before anything is written
     wm.wm_encode_leaves(good, nbytes, chunk, None, crc, wire, ws, res)
     dst = [torch.full_like(x, 0x33) for x in leaves]
@@ -132,7 +178,7 @@ def test_leaf_table_that_breaks_the_rules_is_rejected():
         dt = wm.make_leaf_table(dst)
         dt[:, 1] = t[:, 1]
         if not torch.equal(t[:, 0], good[:, 0]):
-            dt[1, 0] += 4
+            dt[1, 0] = 0 if int(t[1, 0]) == 0 else dt[1, 0] + 4
         dcrc = torch.zeros(nc, dtype=torch.int32, device="cuda")
         wm.wm_decode_verify_leaves(wire, r.wire_len, dt, nbytes, chunk, dcrc, ws, res)
         assert wm.read_result(res).status_name == "ERR_ARG"
