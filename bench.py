@@ -326,6 +326,67 @@ def leaf_mode(wm, cfg, cur, wire, ws, dev, W, peak, reps=20):
     return out
 
 
+def leaf_mode_paper_table(wm, inputs_mod, cfg, cur, dev, peak, reps=20):
+    """The leaf calls on a table shaped like the paper's movable set: 450 leaves (420 tensors of
+    seeded random sizes and 30 flags of 2 to 64 bytes in between) adding up to 1,670,124,960 bytes,
+    filled with the first bytes of the workload's cache.  Most tiles then begin off a 16-byte
+    boundary inside their leaf and some cross leaves; beside it the flat calls on the same bytes."""
+    import torch
+    N, C = inputs_mod.PAPER_CACHE_BYTES, cfg.chunk_bytes
+    if cur.numel() < N:
+        return None
+    sizes = inputs_mod.paper_leaf_sizes()
+    nc = wm.num_chunks(N, C)
+    src, o = [], 0
+    for n in sizes:
+        src.append(cur[o:o + n].clone())
+        o += n
+    dst = [torch.empty_like(x) for x in src]
+    ts, td = wm.make_leaf_table(src, dev), wm.make_leaf_table(dst, dev)
+    ws = wm.new_workspace(N, C, dev)
+    wire = torch.empty(wm.wire_bound(N, C), dtype=torch.uint8, device=dev)
+    wire_flat = torch.empty_like(wire)
+    flat_dst = torch.empty(N, dtype=torch.uint8, device=dev)
+    crc = torch.zeros(nc, dtype=torch.int32, device=dev)
+    crc_d = torch.zeros(nc, dtype=torch.int32, device=dev)
+    res_e, res_d = wm.new_result(dev), wm.new_result(dev)
+    wm.wm_encode_leaves(ts, N, C, None, crc, wire, ws, res_e)
+    r = wm.read_result(res_e)
+    wm.wm_encode(cur[:N], C, None, crc_d, wire_flat, ws, res_d)
+    rf = wm.read_result(res_d)
+    if not (r.ok and rf.ok and r.wire_len == rf.wire_len and torch.equal(wire[: r.wire_len], wire_flat[: r.wire_len])):
+        raise SystemExit("leaf mode (paper table): the image differs from the flat call's")
+    W = r.wire_len
+    wm.wm_decode_verify_leaves(wire, W, td, N, C, crc_d, ws, res_d)
+    if not (wm.read_result(res_d).ok and all(torch.equal(a, b) for a, b in zip(src, dst))):
+        raise SystemExit("leaf mode (paper table): round trip failed")
+    calls = (("encode_leaves", lambda: wm.wm_encode_leaves(ts, N, C, None, crc, wire, ws, res_e)),
+             ("decode_verify_leaves", lambda: wm.wm_decode_verify_leaves(wire, W, td, N, C, crc_d, ws, res_d)),
+             ("encode_flat", lambda: wm.wm_encode(cur[:N], C, None, crc, wire_flat, ws, res_e)),
+             ("decode_verify_flat", lambda: wm.wm_decode_verify(wire_flat, W, flat_dst, C, crc_d, ws, res_d)))
+    edges, o = [], 0
+    for n in sizes[:-1]:
+        o += n
+        edges.append(o)
+    out = {"leaves": len(sizes), "nbytes": N, "wire_bytes": W,
+           "tiles_that_cross_leaves": len({e // 16384 for e in edges if e % 16384}),
+           "leaf_starts_off_16_bytes": sum(1 for e in edges if e % 16)}
+    for name, fn in calls:
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(reps):
+            fn()
+        b.record()
+        torch.cuda.synchronize()
+        out[name + "_ms"] = a.elapsed_time(b) / reps
+    out["encode_frac_of_hbm_peak"] = (N + W) / (out["encode_leaves_ms"] * 1e-3) / 1e9 / peak
+    out["decode_frac_of_hbm_peak"] = (N + W) / (out["decode_verify_leaves_ms"] * 1e-3) / 1e9 / peak
+    return out
+
+
 def tail_schedule(wm, cfg, cur, shadow, wire, ws, dev, W, reps=8, super_mbs=(64, 128, 256)):
     """Verification placement: the move cut into super-chunks on three streams (encode, a device-to-device
     copy standing in for the wire, decode + verify), against the same three stages run one after the
@@ -700,6 +761,8 @@ def main():
     leaf = None
     if not args.no_loop and cfg.kind in ("kv", "llm"):
         leaf = leaf_mode(wm, cfg, cur, wire, ws, dev, W, peak)
+        if leaf is not None and args.workload == "engine":
+            leaf["paper_table"] = leaf_mode_paper_table(wm, inputs_mod, cfg, cur, dev, peak)
 
     # the entropy-coded exponent option beside the default format
     ent = None

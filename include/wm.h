@@ -319,10 +319,17 @@ void wm_entropy_enable(int on);
  * byte for byte what wm_encode produces from the flattened buffer, and either decode call
  * accepts it.
  *   leaves    [dev] n_leaves entries (1..4096), read on the stream.  Every ptr is 16-byte
- *             aligned device memory; every nbytes is positive and, for all leaves but the
- *             last, a multiple of 16384; the sizes add up to nbytes.  A table that breaks
- *             these rules gives result->status WM_ERR_ARG and nothing is read or written
- *             through it.
+ *             aligned device memory; every nbytes is positive (any value: a two-byte flag
+ *             between two tensors is fine) and the sizes add up to nbytes.  A table that
+ *             breaks these rules gives result->status WM_ERR_ARG and nothing is read or
+ *             written through it.
+ * The 16 KiB tile grid lies over the concatenation, so a tile may begin anywhere inside a leaf.
+ * A tile that lies inside one leaf moves by the same bulk copy as in the flat calls (from the
+ * 16-byte boundary below its first byte, the kernel shifts by the remainder; decoded tiles whose
+ * destination is not four-byte aligned take halfword or byte stores, which is slower: put odd-sized
+ * leaves last where the order is yours to choose).  A tile that crosses a leaf boundary, at most
+ * two per leaf, is read and written byte by byte through the table.  No byte outside the leaves
+ * is ever read or written.
  * Everything else is as in wm_encode / wm_decode_verify.
  */
 typedef struct {

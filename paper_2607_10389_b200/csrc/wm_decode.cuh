@@ -308,7 +308,7 @@ __device__ __forceinline__ void unpack_group_planes(const PlaneWords& pw, uint32
 template <int TEAMS, bool LEAVES, int MODE, int ENT = 0>
 __global__ void __launch_bounds__(TEAMS * 256, 1)
 k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restrict__ dst, Ws ws,
-         const Tables* __restrict__ tab, LeafView lv)
+         const Tables* __restrict__ tab)
 {
     extern __shared__ __align__(16) unsigned char smem[];
     // ENT: what the low byte of a strand's bits says about the codeword there: its length (16: the
@@ -504,10 +504,7 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
         uint32_t l_e = 0, l_rel = 0, l_tk = kNone;
         unsigned long long l_po = 0;
         // (spread over three warps: the team waits for whichever warp has the most to do)
-        // (leaf mode, rare: a tile that is scattered through the leaf table keeps the stage a little
-        // longer, see below; the next copy starts when it is done with it)
-        const bool keeps_stage = LEAVES && MODE != 1 && (o_leaf >> 63) != 0ull && e != 0u && e != 0xFFFFu;
-        if (tt == 64u && !keeps_stage) start_copy(tc->slot[(it + 1u) & 3u]);
+        if (tt == 64u) start_copy(tc->slot[(it + 1u) & 3u]);
         if (tt == 32u && t_done != kNone) ws.dig[t_done] = xor8(tc->wdig[p ^ 1u]);
         uint32_t t_look = kNone;           // warps 0 and 3: the tile claimed a step ago (two tiles ahead)
         if (leader) {                      // its table entry and offsets
@@ -526,39 +523,28 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
         // ---- phase 2: unpack, store, checksum
         bool have_digest = false;
         if (e != 0) {
-            // (leaf mode: a walked tile, bit 63 of its descriptor, is stored byte by byte through the table)
-            const bool walked = LEAVES && (o_leaf >> 63) != 0ull;
             unsigned char* o = LEAVES ? reinterpret_cast<unsigned char*>(o_leaf) : dst + (uint64_t)t * kTile;
             bool fold = (ew >> 16) != 0;
             if (e == 0xFFFFu) {
                 const unsigned char* src = payload + tc->slot[it & 3u].src;
                 const uint32_t len = g.tail_len;
-                if (MODE != 1) {
-                    if (LEAVES) {               // (the ragged tile is always a walked one)
-                        uint32_t k = (uint32_t)o_leaf;
-                        for (uint32_t i = tt; i < len; i += kTeamThreads) *leaf_byte_addr(lv, k, (unsigned long long)t * kTile + i) = src[i];
-                    } else {
-                        for (uint32_t i = tt; i < len; i += kTeamThreads) o[i] = src[i];
-                    }
-                }
+                // (leaf mode: the ragged tile has a slot of its own in the side buffer)
+                if (MODE != 1) for (uint32_t i = tt; i < len; i += kTeamThreads) o[i] = src[i];
                 if (MODE != 2) load_tile_words_guarded(src, len, fold, warp, lane, w);
                 fold = false;
             }
-            // where the decoded words go: word i of this lane to byte 128 i of its warp's 2 KiB.  Leaf
-            // mode has two more ways besides the plain 32-bit store: a tile that starts off a four-byte
-            // boundary takes halfword or byte stores, a walked tile goes into the stage first (free:
-            // the next copy was held back) and from there byte by byte to wherever the table says.
+            // where the decoded words go: word i of this lane to byte 128 i of its warp's 2 KiB.  In leaf
+            // mode a tile may start off a four-byte boundary inside its leaf; it then takes halfword
+            // or byte stores instead of the plain 32-bit one.
             unsigned char* const q = o + warp * 2048u + lane * 4u;
-            uint32_t* const sw = reinterpret_cast<uint32_t*>(stage) + warp * 512u + lane;
-            const uint32_t how = !LEAVES ? 0u : walked ? 3u : (uint32_t)(o_leaf & 3ull) == 0u ? 0u : (o_leaf & 1ull) ? 2u : 1u;
+            const uint32_t how = !LEAVES ? 0u : (uint32_t)(o_leaf & 3ull) == 0u ? 0u : (o_leaf & 1ull) ? 2u : 1u;
             // (the rest of the step once per way of storing, so that the choice is made once per tile)
             auto rest_of_step = [&](auto how_c) {
             constexpr uint32_t HOW = decltype(how_c)::value;
             auto put = [&](int i, uint32_t v) {
                 if (HOW == 0u) st_stream_u32(q + i * 128, v);
                 else if (HOW == 1u) { stg_u16(q + i * 128, v); stg_u16(q + i * 128 + 2, v >> 16); }
-                else if (HOW == 2u) { stg_u8(q + i * 128, v); stg_u16(q + i * 128 + 1, v >> 8); stg_u8(q + i * 128 + 3, v >> 24); }
-                else sw[i * 32] = v;
+                else { stg_u8(q + i * 128, v); stg_u16(q + i * 128 + 1, v >> 8); stg_u8(q + i * 128 + 3, v >> 24); }
             };
             if (is_pack && decoded) {
                 // A coded tile goes group by group: four words are rebuilt, stored, and fed to the
@@ -621,16 +607,7 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
             };
             if (!LEAVES || how == 0u) rest_of_step(std::integral_constant<uint32_t, 0u>());
             else if (how == 1u) rest_of_step(std::integral_constant<uint32_t, 1u>());
-            else if (how == 2u) rest_of_step(std::integral_constant<uint32_t, 2u>());
-            else rest_of_step(std::integral_constant<uint32_t, 3u>());
-        }
-        if (keeps_stage) {
-            // (every thread of the team comes here, whatever its warp made of the tile: a warp that
-            // refused its part left that part of the stage as it was, and the call fails anyway)
-            team_bar(team);
-            stage_to_walked_tile(lv, (uint32_t)o_leaf, (unsigned long long)t * kTile, kTile, stage, tt);
-            team_bar(team);
-            if (tt == 64u) start_copy(tc->slot[(it + 1u) & 3u]);
+            else rest_of_step(std::integral_constant<uint32_t, 2u>());
         }
         t_done = have_digest ? t : kNone;
         if (leader && t_look < g.n_tiles) {
@@ -647,8 +624,7 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
 __global__ void __launch_bounds__(1024)
 k_decode_finish(const unsigned char* __restrict__ wire, uint64_t wire_len, Geo g,
                 const unsigned char* __restrict__ dst, uint32_t* __restrict__ dst_crc, Ws ws,
-                const Tables* __restrict__ tab, wm_result* result, const __grid_constant__ ChunkPowers cp, uint32_t strict,
-                LeafView lv)
+                const Tables* __restrict__ tab, wm_result* result, const __grid_constant__ ChunkPowers cp, uint32_t strict)
 {
     __shared__ uint32_t sHT[1024];
     __shared__ uint32_t sT0[256];
@@ -674,13 +650,10 @@ k_decode_finish(const unsigned char* __restrict__ wire, uint64_t wire_len, Geo g
         } else if (fl & CF_PRESENT) {
             // (a chunk shorter than four bytes is checksummed byte by byte: from dst, or, in a strict
             // call, where nothing has been stored yet, from its raw copy in the wire image)
-            const unsigned char* tiny = chunk_first_byte(g, dst, c);
+            const unsigned char* tiny = chunk_first_byte(g, ws, dst, c);
             if (strict && chunk_len_dev(g, c) < 4)
                 tiny = wire + g.meta_end + *reinterpret_cast<const unsigned long long*>(dir + 16ull * c);
-            // (leaf mode, not strict: the tiny chunk's bytes are read back through the table)
-            const uint32_t got = (!tiny && chunk_len_dev(g, c) < 4)
-                                     ? tiny_chunk_crc_leaves(sT0, lv, (unsigned long long)c * g.chunk_bytes, (uint32_t)chunk_len_dev(g, c))
-                                     : chunk_crc_staged(g, sHT, sT0, stage, ws.dig, tiny, c, threadIdx.x);
+            const uint32_t got = chunk_crc_staged(g, sHT, sT0, stage, ws.dig, tiny, c, threadIdx.x);
             if (got != want) { atomicMin(&ws.ctrl->bad5_first, c); atomicAdd(&ws.ctrl->bad5_count, 1u); }
         } else {
             if (dst_crc[c] != want) { atomicMin(&ws.ctrl->bad6_first, c); atomicAdd(&ws.ctrl->bad6_count, 1u); }

@@ -319,11 +319,10 @@ __device__ __forceinline__ uint32_t ent_parse_value(uint32_t buf, uint32_t s, ui
 // of slack that is rare, and it only delays: the teams that hold earlier tiles never depend
 // on this one.
 // A tile as a team passes it round: its number in the low 22 bits, kQFirst when it is the first
-// tile of its chunk, kQPresent when its chunk is encoded; kQNone: no tile.  Leaf mode adds
-// kQWalked when the tile is read through the leaf table instead of by a bulk copy, and for the
-// others, in bits 22-25, how many bytes above a 16-byte boundary the tile starts.  (The codec
-// takes caches of at most 2^21 tiles, so a number never reaches kQNone or the other fields.)
-constexpr uint32_t kQPresent = 1u << 31, kQFirst = 1u << 30, kQWalked = 1u << 29, kQTile = (1u << 22) - 1u, kQNone = kQTile;
+// tile of its chunk, kQPresent when its chunk is encoded; kQNone: no tile.  Leaf mode adds, in
+// bits 22-25, how many bytes above a 16-byte boundary the tile starts.  (The codec takes caches
+// of at most 2^21 tiles, so a number never reaches kQNone or the other fields.)
+constexpr uint32_t kQPresent = 1u << 31, kQFirst = 1u << 30, kQTile = (1u << 22) - 1u, kQNone = kQTile;
 constexpr uint32_t kQOffShift = 22;
 // Marks in a team's width table: on a warp's first entry, all 2 KiB of the warp's rows are zero;
 // as the sum of the widths, the tile is all zero.
@@ -346,7 +345,7 @@ __device__ __forceinline__ uint32_t describe_tile(const Geo& g, const uint8_t* _
 template <int TEAMS, bool MASKED, bool LEAVES, bool ZEROS, bool ENT = false>
 __global__ void __launch_bounds__(TEAMS * 256, 1)
 k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restrict__ dirty,
-         unsigned char* __restrict__ wire, uint64_t wire_cap, Ws ws, const Tables* __restrict__ tab, LeafView lv)
+         unsigned char* __restrict__ wire, uint64_t wire_cap, Ws ws, const Tables* __restrict__ tab)
 {
     extern __shared__ __align__(16) unsigned char smem[];
     // The first block to get here becomes the scanner: one warp of it, alone on its SM (a warp
@@ -407,9 +406,8 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
 
     auto is_tile = [](uint32_t q) { return (q & kQTile) != kQNone; };
     auto is_hot = [&](uint32_t q) { return q >= kQPresent && (q & kQTile) < g.n_full_tiles; };   // present and full
-    auto is_walked = [](uint32_t q) { return LEAVES && (q & kQWalked) != 0u; };
     auto publish_len = [&](uint32_t t, uint32_t len) { st_relaxed_u32(ws.lbk + t, kFlagA | (len / kUnit)); };
-    // where tile t lives: its address in the flat cache, or (leaf mode) the descriptor that k_leaf_map wrote
+    // where tile t lives: its address in the flat cache, or (leaf mode) the address that k_leaf_map wrote
     auto tile_src = [&](uint32_t t) -> unsigned long long {
         return LEAVES ? ws.tptr[t] : reinterpret_cast<unsigned long long>(cache + (uint64_t)t * kTile);
     };
@@ -417,14 +415,13 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
     // off a 16-byte boundary; the copy then starts at the boundary below and takes 16 bytes more
     // (k_leaf_map saw to it that they belong to the leaf); the readers shift by the remainder.
     auto start_copy = [&](uint32_t q, unsigned long long src) {
-        if (!is_hot(q) || is_walked(q)) return;
+        if (!is_hot(q)) return;
         const unsigned long long a = LEAVES ? src & ~15ull : src;
         bulk_load(stage, reinterpret_cast<const void*>(a), (LEAVES && a != src) ? kTile + 16u : kTile, &tc->mbar, pol_once);
     };
-    // leaf mode, handing a claimed tile on: its word carries the walked mark or the start's remainder
-    auto with_mark = [](uint32_t q, unsigned long long desc) {
-        if (!LEAVES || (q & kQTile) == kQNone) return q;
-        return (desc >> 63) ? q | kQWalked : q | (((uint32_t)desc & 15u) << kQOffShift);
+    // leaf mode, handing a claimed tile on: its word carries the start's remainder
+    auto with_mark = [](uint32_t q, unsigned long long addr) {
+        return (!LEAVES || (q & kQTile) == kQNone) ? q : q | (((uint32_t)addr & 15u) << kQOffShift);
     };
 
     // Tiles in flight, oldest first: X (packed in this step), V, W (waiting for their offsets),
@@ -467,21 +464,12 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
     uint32_t trouble = 0;              // sticky: the image does not fit
     while (((qX & qV & qW & qY) & kQTile) != kQNone) {
         const bool hotY = is_hot(qY);
-        if (LEAVES && is_tile(qY) && qY >= kQPresent && (is_walked(qY) || !hotY)) {
-            // leaf mode, rare: a tile that crosses leaves (no copy was started for it) or the ragged last
-            // tile is gathered into the stage byte by byte; from there it goes the ordinary way
-            const uint32_t tY = qY & kQTile;
-            walked_tile_to_stage(lv, (uint32_t)ws.tptr[tY], (unsigned long long)tY * kTile, hotY ? kTile : tile_left(g, tY), stage, tt);
-            team_bar(team);
-        }
         if (hotY) {
-            if (!is_walked(qY)) {
-                wait_for_copy<!ENT>(&tc->mbar, phase, g.wait_ns, ws.ctrl);
-                phase ^= 1u;
-            }
+            wait_for_copy<!ENT>(&tc->mbar, phase, g.wait_ns, ws.ctrl);
+            phase ^= 1u;
             // leaf mode: a tile that was copied from the 16-byte boundary below it starts that many
-            // bytes into the stage (0 for a walked tile): whole words from a quarter of that on, each
-            // put together from two neighbours when the remainder is no multiple of four
+            // bytes into the stage: whole words from a quarter of that on, each put together from two
+            // neighbours when the remainder is no multiple of four
             const uint32_t off = LEAVES ? (qY >> kQOffShift) & 15u : 0u;
             const uint32_t sh = (off & 3u) * 8u;
             const uint32_t* const p = my_words + (off >> 2);
@@ -612,8 +600,8 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
             const bool present = qY >= kQPresent;
             if (tt == 0) publish_len(tYn, present ? tile_left(g, tYn) : 0u);
             if (present) {
-                // (leaf mode: the tile's bytes were gathered into the stage above)
-                load_tile_words_guarded(LEAVES ? stage : cache + (uint64_t)tYn * kTile, tile_left(g, tYn), (qY & kQFirst) != 0, warp, lane, d);
+                // (leaf mode: the ragged tile has a slot of its own in the side buffer)
+                load_tile_words_guarded(reinterpret_cast<const unsigned char*>(tile_src(tYn)), tile_left(g, tYn), (qY & kQFirst) != 0, warp, lane, d);
                 const uint32_t v = tile_digest_part(S, d, false, warp, lane);
                 if (lane == 0) tc->wdig[slY][warp] = v;
             }
@@ -736,14 +724,9 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
             if (exclX + enc_len > room) {
                 trouble |= 1u;
             } else {
+                const unsigned char* src = reinterpret_cast<const unsigned char*>(tile_src(tXn));
                 unsigned char* dst = payload + exclX;
-                if (LEAVES) {
-                    uint32_t k = (uint32_t)ws.tptr[tXn];               // (the ragged tile is always a walked one)
-                    for (uint32_t i = tt; i < enc_len; i += kTeamThreads) dst[i] = *leaf_byte_addr(lv, k, (unsigned long long)tXn * kTile + i);
-                } else {
-                    const unsigned char* src = cache + (uint64_t)tXn * kTile;
-                    for (uint32_t i = tt; i < enc_len; i += kTeamThreads) dst[i] = src[i];
-                }
+                for (uint32_t i = tt; i < enc_len; i += kTeamThreads) dst[i] = src[i];
             }
         }
 
@@ -806,7 +789,7 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
 __global__ void __launch_bounds__(1024)
 k_encode_finish(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restrict__ dirty,
                 uint32_t* __restrict__ crc_inout, unsigned char* __restrict__ wire, Ws ws,
-                const Tables* __restrict__ tab, const __grid_constant__ ChunkPowers cp, uint32_t option_flags, LeafView lv)
+                const Tables* __restrict__ tab, const __grid_constant__ ChunkPowers cp, uint32_t option_flags)
 {
     __shared__ uint32_t sHT[1024];
     __shared__ uint32_t sT0[256];
@@ -829,9 +812,7 @@ k_encode_finish(const unsigned char* __restrict__ cache, Geo g, const uint8_t* _
         present = (!dirty || dirty[c]) ? 1u : 0u;
         uint32_t crc;
         if (present) {
-            // (leaf mode: a last chunk shorter than four bytes is checksummed byte by byte through the table)
-            if (!cache && chunk_len_dev(g, c) < 4) crc = tiny_chunk_crc_leaves(sT0, lv, (unsigned long long)c * g.chunk_bytes, (uint32_t)chunk_len_dev(g, c));
-            else crc = chunk_crc_staged(g, sHT, sT0, stage, ws.dig, chunk_first_byte(g, cache, c), c, threadIdx.x);
+            crc = chunk_crc_staged(g, sHT, sT0, stage, ws.dig, chunk_first_byte(g, ws, cache, c), c, threadIdx.x);
             crc_inout[c] = crc;
         } else {
             crc = crc_inout[c];

@@ -413,12 +413,12 @@ static wm_status encode_any(const void* cache, const wm_leaf* leaves, uint32_t n
     Ws ws = ws_carve(workspace, g);
     const unsigned char* c = static_cast<const unsigned char*>(cache);
     unsigned char* w = static_cast<unsigned char*>(wire);
-    const LeafView lv = {leaves, ws.lstart, leaves ? n_leaves : 0u};
     const uint32_t init_blocks = (g.n_tiles + 1023) / 1024 < 1024 ? (g.n_tiles + 1023) / 1024 : 1024;
     k_encode_init<<<init_blocks ? init_blocks : 1, 1024, 0, s>>>(g, ws, w);
     if (leaves) {
         const uint32_t map_blocks = (g.n_tiles + 4095) / 4096 < 64 ? (g.n_tiles + 4095) / 4096 : 64;
         launch_after(k_leaf_map, map_blocks ? map_blocks : 1, 1024, 0, s, leaves, n_leaves, g, ws, result, 0);
+        launch_after(k_leaf_gather, 1024, 256, 0, s, leaves, n_leaves, g, ws);
     }
     // one block per SM: one of them scans, the others encode
     // (tiles are claimed by ticket, so any number of blocks gives the same image; a caller that
@@ -429,7 +429,7 @@ static wm_status encode_any(const void* cache, const wm_leaf* leaves, uint32_t n
     {
         MainKernelTimer timer(ds, 2, s);
         const int variant = (dirty ? 1 : 0) | (leaves ? 2 : 0) | (opt_zero ? 4 : 0) | (opt_ent ? 8 : 0);
-        auto go = [&](auto kernel) { launch_after(kernel, grid, kTeams * 256, kDynSmem, s, c, g, dirty, w, wire_cap, ws, ds->tables, lv); };
+        auto go = [&](auto kernel) { launch_after(kernel, grid, kTeams * 256, kDynSmem, s, c, g, dirty, w, wire_cap, ws, ds->tables); };
         switch (variant) {
             case 0: go(k_encode<kTeams, false, false, false>); break;
             case 1: go(k_encode<kTeams, true, false, false>); break;
@@ -450,9 +450,9 @@ static wm_status encode_any(const void* cache, const wm_leaf* leaves, uint32_t n
         }
     }
     launch_after(k_encode_finish, (g.n_chunks + g.finish_cb - 1) / g.finish_cb, 1024, 0, s, c, g, dirty, crc_inout, w, ws, ds->tables,
-                 chunk_powers(g), (opt_ent ? 4u : 0u) | (opt_zero ? 2u : 0u), lv);
+                 chunk_powers(g), (opt_ent ? 4u : 0u) | (opt_zero ? 2u : 0u));
     launch_after(k_meta_crc, (g.n_meta_slices + 3) / 4, 1024, kDynSmem, s, w, g, ws, ds->tables, result);
-    g_launches = leaves ? 5 : 4;
+    g_launches = leaves ? 6 : 4;
     return launch_status();
 }
 
@@ -494,7 +494,6 @@ static wm_status decode_any(const void* wire, uint64_t wire_len, void* dst, cons
     Ws ws = ws_carve(workspace, g);
     const unsigned char* w = static_cast<const unsigned char*>(wire);
     unsigned char* d = static_cast<unsigned char*>(dst);
-    const LeafView lv = {leaves, ws.lstart, leaves ? n_leaves : 0u};
     k_decode_init<<<1, 64, 0, s>>>(ws);
     if (leaves) {
         const uint32_t map_blocks = (g.n_tiles + 4095) / 4096 < 64 ? (g.n_tiles + 4095) / 4096 : 64;
@@ -509,8 +508,8 @@ static wm_status decode_any(const void* wire, uint64_t wire_len, void* dst, cons
     uint32_t grid = need < (uint32_t)ds->sm_count ? need : (uint32_t)ds->sm_count;
     if (block_cap && grid > block_cap) grid = block_cap;
     auto pass = [&](auto flat_kernel, auto leaf_kernel) {
-        if (leaves) launch_after(leaf_kernel, grid, kTeamsPlain * 256, kDynSmem, s, w, g, d, ws, ds->tables, lv);
-        else launch_after(flat_kernel, grid, kTeamsPlain * 256, kDynSmem, s, w, g, d, ws, ds->tables, lv);
+        if (leaves) launch_after(leaf_kernel, grid, kTeamsPlain * 256, kDynSmem, s, w, g, d, ws, ds->tables);
+        else launch_after(flat_kernel, grid, kTeamsPlain * 256, kDynSmem, s, w, g, d, ws, ds->tables);
     };
     {
         MainKernelTimer timer(ds, 3, s);
@@ -522,13 +521,17 @@ static wm_status decode_any(const void* wire, uint64_t wire_len, void* dst, cons
             else pass(k_decode<kTeamsPlain, false, 0>, k_decode<kTeamsPlain, true, 0>);
         }
     }
+    // leaf mode: the tiles that crossed leaf boundaries were decoded into the side buffer; they
+    // go to their leaves behind the kernel that stores
+    if (leaves && !strict) launch_after(k_leaf_scatter, 1024, 256, 0, s, leaves, n_leaves, g, ws);
     launch_after(k_decode_finish, (g.n_chunks + g.finish_cb - 1) / g.finish_cb, 1024, 0, s, w, wire_len, g, d, dst_crc_inout, ws, ds->tables,
-                 result, chunk_powers(g), strict ? 1u : 0u, lv);
+                 result, chunk_powers(g), strict ? 1u : 0u);
     if (strict) {
         if (ent) { pass(k_decode<kTeamsPlain, false, 2, 1>, k_decode<kTeamsPlain, true, 2, 1>); pass(k_decode<kTeamsPlain, false, 2, 2>, k_decode<kTeamsPlain, true, 2, 2>); }
         else pass(k_decode<kTeamsPlain, false, 2>, k_decode<kTeamsPlain, true, 2>);
+        if (leaves) launch_after(k_leaf_scatter, 1024, 256, 0, s, leaves, n_leaves, g, ws);
     }
-    g_launches = (leaves ? 5 : 4) + (strict ? 1 : 0) + (ent ? (strict ? 2 : 1) : 0);
+    g_launches = (leaves ? 6 : 4) + (strict ? 1 : 0) + (ent ? (strict ? 2 : 1) : 0);
     return launch_status();
 }
 

@@ -60,7 +60,8 @@ struct Ctrl {                 // first 256 bytes of the workspace
     uint32_t hdr_n_present, hdr_cache_crc;
     uint32_t cache_acc;       // XOR of the chunks' terms of the whole-cache CRC
     uint32_t has_pack;        // decode of an image with the entropy option: it holds PACK tiles too
-    uint32_t pad[40];
+    uint32_t n_walked;        // leaf mode: tiles that go through the side buffer (see k_leaf_map)
+    uint32_t pad[39];
 };
 static_assert(sizeof(Ctrl) == 256, "control block is 256 bytes");
 
@@ -121,17 +122,20 @@ struct Ws {
     uint32_t* cflag;             // [n_chunks] bit0 present, bit1..: failed step 3/4/5/6
     uint32_t* ccrc;              // [n_chunks]
     uint32_t* mdig;              // [n_meta_slices]
-    unsigned long long* tptr;    // [n_tiles] leaf mode: where each tile of the logical cache lives (see k_leaf_map)
+    unsigned long long* tptr;    // [n_tiles] leaf mode: the address of each tile of the logical cache (see k_leaf_map)
     unsigned long long* lstart;  // [kMaxLeaves + 1] leaf mode: logical offset at which each leaf starts
+    uint32_t* wlist;             // [kMaxWalked] leaf mode: the tiles that go through the side buffer
+    unsigned char* side;         // [min(n_tiles, kMaxWalked)][16384] leaf mode: their slots
 };
 constexpr uint32_t kMaxLeaves = 4096;
+constexpr uint32_t kMaxWalked = 2048;        // 32 MiB of side buffer at most
 
 constexpr uint32_t CF_PRESENT = 1, CF_BAD3 = 2, CF_BAD4 = 4, CF_BAD5 = 8, CF_BAD6 = 16;
 
 static inline uint64_t align16(uint64_t v) { return (v + 15) & ~(uint64_t)15; }
 
 struct WsLayout {
-    uint64_t state, dig, rel, cflag, ccrc, mdig, tptr, lstart, total;
+    uint64_t state, dig, rel, cflag, ccrc, mdig, tptr, lstart, wlist, side, total;
 };
 
 static WsLayout ws_layout(const Geo& g)
@@ -146,6 +150,8 @@ static WsLayout ws_layout(const Geo& g)
     L.mdig = o;  o = align16(o + 4ull * g.n_meta_slices);
     L.tptr = o;  o = align16(o + 8ull * g.n_tiles);
     L.lstart = o; o = align16(o + 8ull * (kMaxLeaves + 1));
+    L.wlist = o; o = align16(o + 4ull * kMaxWalked);
+    L.side = o; o = align16(o + (uint64_t)kTile * (g.n_tiles < kMaxWalked ? g.n_tiles : kMaxWalked));
     L.total = o;
     return L;
 }
@@ -164,6 +170,8 @@ static Ws ws_carve(void* base, const Geo& g)
     w.mdig = reinterpret_cast<uint32_t*>(b + L.mdig);
     w.tptr = reinterpret_cast<unsigned long long*>(b + L.tptr);
     w.lstart = reinterpret_cast<unsigned long long*>(b + L.lstart);
+    w.wlist = reinterpret_cast<uint32_t*>(b + L.wlist);
+    w.side = b + L.side;
     return w;
 }
 
@@ -276,11 +284,13 @@ __device__ __forceinline__ uint32_t xor8(const uint32_t* p)
     return p[0] ^ p[1] ^ p[2] ^ p[3] ^ p[4] ^ p[5] ^ p[6] ^ p[7];
 }
 
-// First byte of chunk c in the flat buffer (nullptr in leaf mode, where the finish kernels walk
-// the leaf table instead).  Only chunks shorter than four bytes are ever read through it.
-__device__ __forceinline__ const unsigned char* chunk_first_byte(const Geo& g, const unsigned char* flat, uint32_t c)
+// First byte of chunk c: in the flat buffer, or (leaf mode, flat == nullptr) where the chunk's
+// first tile is (for the only chunk ever asked for, the ragged last one, that is its slot in the
+// side buffer).  Only chunks shorter than four bytes are read through it.
+__device__ __forceinline__ const unsigned char* chunk_first_byte(const Geo& g, const Ws& ws, const unsigned char* flat, uint32_t c)
 {
-    return flat ? flat + (uint64_t)c * g.chunk_bytes : nullptr;
+    if (flat) return flat + (uint64_t)c * g.chunk_bytes;
+    return chunk_len_dev(g, c) < 4 ? reinterpret_cast<const unsigned char*>(ws.tptr[(uint64_t)c * g.tiles_per_chunk]) : nullptr;
 }
 
 // CRC32C of chunk c from its tiles' digests (Horner over tiles; the all-ones init was folded

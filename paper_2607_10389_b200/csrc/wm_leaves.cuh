@@ -11,20 +11,22 @@ namespace wm {
 // 16 KiB tile grid is laid over that concatenation, so a tile may begin anywhere inside a leaf
 // and may run across leaf boundaries (a scalar flag between two tensors, say).  k_leaf_map
 // writes, per leaf, the logical offset at which it starts (ws.lstart, n + 1 entries) and, per
-// tile, a 64-bit descriptor (ws.tptr):
-//   bit 63 clear: the address of the tile's first byte.  All 16384 bytes sit in one leaf, and so
-//       does the 16-byte aligned block around them, so the tile can be moved by a bulk copy from
-//       the address rounded down to 16 (the main kernels shift the words by the remainder).
-//   bit 63 set:   a "walked" tile; the low 32 bits are the leaf that holds its first byte.  The
-//       tile crosses a leaf boundary, or is the ragged last tile, or ends within 16 bytes of the
-//       end of a leaf whose size is not a multiple of 16 (the aligned block would reach past
-//       the leaf).  Such tiles are read and written byte by byte through the leaf table; there
-//       are at most two per leaf.
+// tile, the address the main kernels use for it (ws.tptr):
+//   - a tile whose 16384 bytes sit in one leaf, together with the 16-byte aligned block around
+//     them: the address of its first byte inside the leaf.  It moves by a bulk copy from the
+//     address rounded down to 16; the main kernels shift the words by the remainder.
+//   - any other tile (it crosses a leaf boundary, or is the ragged last tile, or ends within 16
+//     bytes of the end of a leaf whose size is no multiple of 16: the aligned block would reach
+//     past the leaf) is a "walked" tile: it gets a 16 KiB slot in the workspace's side buffer and
+//     its address is the slot's.  k_leaf_gather fills the slots from the leaves before the encode
+//     kernel runs, k_leaf_scatter empties them into the leaves after the decode kernel has run,
+//     both run by run, byte by byte, so the main kernels see ordinary aligned tiles and carry no
+//     code for the exception.  There are at most two walked tiles per leaf; ws.wlist keeps their
+//     numbers, ctrl->n_walked their count.
 // Rules (a table that breaks one raises error bit 8; in decode mode it also closes the gate and
 // writes the result record; nothing is read or written through a rejected table): 1..4096
 // leaves, every pointer 16-byte aligned, every size positive and at most nbytes (so the sum
-// cannot wrap), the sizes add up to nbytes.
-constexpr unsigned long long kTileWalked = 1ull << 63;
+// cannot wrap), the sizes add up to nbytes, at most kMaxWalked walked tiles.
 
 __global__ void __launch_bounds__(1024)
 k_leaf_map(const wm_leaf* __restrict__ leaves, uint32_t n, Geo g, Ws ws, wm_result* result, int decode)
@@ -73,21 +75,23 @@ k_leaf_map(const wm_leaf* __restrict__ leaves, uint32_t n, Geo g, Ws ws, wm_resu
     __syncthreads();
     if (threadIdx.x == 0) s_start[n] = g.nbytes;
     __syncthreads();
-    if (s_bad) {
-        if (blockIdx.x == 0 && threadIdx.x == 0) {
-            atomicOr(&ws.ctrl->err, 8u);
-            if (decode) {
-                ws.ctrl->gate = (uint32_t)WM_ERR_ARG;
-                wm_result r;
-                memset(&r, 0, sizeof r);
-                r.status = WM_ERR_ARG;
-                *result = r;
-            }
+    auto refuse = [&]() {
+        atomicOr(&ws.ctrl->err, 8u);
+        if (decode) {
+            ws.ctrl->gate = (uint32_t)WM_ERR_ARG;
+            wm_result r;
+            memset(&r, 0, sizeof r);
+            r.status = WM_ERR_ARG;
+            *result = r;
         }
+    };
+    if (s_bad) {
+        if (blockIdx.x == 0 && threadIdx.x == 0) refuse();
         return;
     }
     if (blockIdx.x == 0)
         for (uint32_t i = threadIdx.x; i <= n; i += blockDim.x) ws.lstart[i] = s_start[i];
+    const uint32_t n_slots = g.n_tiles < kMaxWalked ? g.n_tiles : kMaxWalked;
     for (uint32_t t = blockIdx.x * blockDim.x + threadIdx.x; t < g.n_tiles; t += gridDim.x * blockDim.x) {
         const unsigned long long L0 = (unsigned long long)t * kTile;
         uint32_t lo = 0, hi = n;                       // the leaf with start[lo] <= L0 < start[lo + 1]
@@ -101,63 +105,80 @@ k_leaf_map(const wm_leaf* __restrict__ leaves, uint32_t n, Geo g, Ws ws, wm_resu
         const unsigned long long r = addr & 15ull;
         // whole, inside this leaf, and so is the aligned block that a shifted copy reads
         const bool direct = L0 + kTile <= g.nbytes && in_leaf + kTile + (r ? 16ull - r : 0ull) <= leaf_len;
-        ws.tptr[t] = direct ? addr : (kTileWalked | lo);
+        if (direct) {
+            ws.tptr[t] = addr;
+        } else {
+            const uint32_t slot = atomicAdd(&ws.ctrl->n_walked, 1u);
+            if (slot < n_slots) {
+                ws.wlist[slot] = t;
+                ws.tptr[t] = reinterpret_cast<unsigned long long>(ws.side + (size_t)slot * kTile);
+            } else {
+                ws.tptr[t] = 0ull;
+                if (slot == n_slots) refuse();         // too many tiles cut by leaf boundaries for the side buffer
+            }
+        }
     }
 }
 
-// ---- walked tiles: byte-exact access through the leaf table (rare, kept out of line) ----
-
-struct LeafView {
-    const wm_leaf* leaves;                 // [n] the caller's table
-    const unsigned long long* lstart;      // [n + 1] logical offsets (k_leaf_map)
-    uint32_t n;
-};
-
-// The address of logical byte L, walking forward from leaf k (k is moved along; L < nbytes).
-__device__ __forceinline__ unsigned char* leaf_byte_addr(const LeafView& lv, uint32_t& k, unsigned long long L)
+// The runs of consecutive bytes a walked tile is made of (one per leaf it touches), handed to
+// `f(leaf_bytes, tile_offset, run_length)`; every thread of the block goes through the same runs.
+template <typename F>
+__device__ __forceinline__ void for_each_run(const wm_leaf* __restrict__ leaves, const unsigned long long* __restrict__ lstart,
+                                             uint32_t n, const Geo& g, uint32_t t, F f)
 {
-    while (k + 1 < lv.n && L >= lv.lstart[k + 1]) k++;
-    return const_cast<unsigned char*>(static_cast<const unsigned char*>(lv.leaves[k].ptr)) + (L - lv.lstart[k]);
-}
-
-// A walked tile of `len` (1..16384) real bytes gathered into the team's stage in shared memory,
-// byte for byte (thread tt of the team's 256 takes bytes 64 tt .. 64 tt + 63); bytes beyond `len`
-// are set to zero.  `k0`: the leaf of the tile's first byte, `L0`: the tile's logical offset.  The
-// caller puts a team barrier behind it.
-__device__ __noinline__ void walked_tile_to_stage(LeafView lv, uint32_t k0, unsigned long long L0, uint32_t len,
-                                                  unsigned char* stage, uint32_t tt)
-{
-    uint32_t k = k0;
-    for (uint32_t w = 0; w < 16u; w++) {
-        const uint32_t at = 64u * tt + 4u * w;
-        uint32_t word = 0;
-        for (uint32_t j = 0; j < 4u; j++)
-            if (at + j < len) word |= (uint32_t)*leaf_byte_addr(lv, k, L0 + at + j) << (8u * j);
-        reinterpret_cast<uint32_t*>(stage)[at / 4u] = word;
+    const unsigned long long L0 = (unsigned long long)t * kTile;
+    const uint32_t len = (uint32_t)min((unsigned long long)kTile, g.nbytes - L0);
+    uint32_t lo = 0, hi = n;
+    while (hi - lo > 1) {
+        const uint32_t mid = (lo + hi) / 2;
+        if (lstart[mid] <= L0) lo = mid; else hi = mid;
+    }
+    uint32_t done = 0;
+    for (uint32_t k = lo; done < len && k < n; k++) {
+        const unsigned long long at = L0 + done;                       // first byte of the run (lstart[k] <= at < lstart[k + 1])
+        const uint32_t run = (uint32_t)min((unsigned long long)(len - done), lstart[k + 1] - at);
+        f(const_cast<unsigned char*>(static_cast<const unsigned char*>(leaves[k].ptr)) + (at - lstart[k]), done, run);
+        done += run;
     }
 }
 
-// The reverse: a decoded tile standing in the team's stage scattered to where the leaf table says
-// (thread tt takes bytes 64 tt .. 64 tt + 63; bytes beyond `len` are not part of the cache).
-__device__ __noinline__ void stage_to_walked_tile(LeafView lv, uint32_t k0, unsigned long long L0, uint32_t len,
-                                                  const unsigned char* stage, uint32_t tt)
+// Encode: every walked tile copied from the leaves into its slot (one block per tile at a time).
+__global__ void __launch_bounds__(256)
+k_leaf_gather(const wm_leaf* __restrict__ leaves, uint32_t n, Geo g, Ws ws)
 {
-    uint32_t k = k0;
-    for (uint32_t w = 0; w < 16u; w++) {
-        const uint32_t at = 64u * tt + 4u * w;
-        const uint32_t word = reinterpret_cast<const uint32_t*>(stage)[at / 4u];
-        for (uint32_t j = 0; j < 4u; j++)
-            if (at + j < len) *leaf_byte_addr(lv, k, L0 + at + j) = (unsigned char)(word >> (8u * j));
+    grid_dep_wait();
+    grid_dep_launch();
+    if (ld_volatile_u32(&ws.ctrl->err) & 8u) return;
+    const uint32_t n_walked = ld_volatile_u32(&ws.ctrl->n_walked);
+    for (uint32_t s = blockIdx.x; s < n_walked; s += gridDim.x) {
+        unsigned char* slot = ws.side + (size_t)s * kTile;
+        for_each_run(leaves, ws.lstart, n, g, ws.wlist[s], [&](const unsigned char* src, uint32_t off, uint32_t run) {
+#pragma unroll 16
+            for (uint32_t i = threadIdx.x; i < run; i += blockDim.x) slot[off + i] = src[i];
+        });
     }
 }
 
-// The cache's last chunk when it is shorter than four bytes (its CRC is taken byte by byte).
-__device__ __noinline__ uint32_t tiny_chunk_crc_leaves(const uint32_t* T0, LeafView lv, unsigned long long L0, uint32_t len)
+// Decode: every walked tile copied from its slot into the leaves.  Runs behind the decode kernel
+// that stores; stays out when the gate is closed (nothing was decoded, the slots hold nothing).
+__global__ void __launch_bounds__(256)
+k_leaf_scatter(const wm_leaf* __restrict__ leaves, uint32_t n, Geo g, Ws ws)
 {
-    // (every leaf holds at least one byte, so the last `len` bytes sit in the last `len` leaves)
-    uint32_t crc = 0xFFFFFFFFu, k = lv.n > len ? lv.n - len : 0u;
-    for (uint32_t i = 0; i < len; i++) crc = T0[(crc ^ *leaf_byte_addr(lv, k, L0 + i)) & 0xFF] ^ (crc >> 8);
-    return ~crc;
+    grid_dep_wait();
+    grid_dep_launch();
+    if (ld_volatile_u32(&ws.ctrl->gate)) return;
+    const uint16_t* tab16 = nullptr;
+    const uint32_t n_walked = ld_volatile_u32(&ws.ctrl->n_walked);
+    for (uint32_t s = blockIdx.x; s < n_walked; s += gridDim.x) {
+        const uint32_t t = ws.wlist[s];
+        if (!(ld_volatile_u32(&ws.cflag[chunk_of(g, t)]) & CF_PRESENT)) continue;     // a tile of an absent chunk was not decoded
+        const unsigned char* slot = ws.side + (size_t)s * kTile;
+        for_each_run(leaves, ws.lstart, n, g, t, [&](unsigned char* dst, uint32_t off, uint32_t run) {
+#pragma unroll 16
+            for (uint32_t i = threadIdx.x; i < run; i += blockDim.x) dst[i] = slot[off + i];
+        });
+    }
+    (void)tab16;
 }
 
 }  // namespace wm

@@ -189,3 +189,28 @@ def before_append(cache_u8: torch.Tensor, cfg: CacheConfig, appended: int):
         hi = (blk * tokens + filled) * row
         mask[lo // cfg.chunk_bytes:(hi - 1) // cfg.chunk_bytes + 1] = 1
     return prev, mask
+
+
+PAPER_CACHE_BYTES = 1_670_124_960      # the movable set of the paper's engine (Section 6.3)
+
+
+def paper_leaf_sizes(seed: int = 9, tensors: int = 420, flags: int = 30, total: int = PAPER_CACHE_BYTES):
+    """Sizes (bytes) of a leaf table shaped like the paper's movable set (Section 3.1, Section 5:
+    420 tensors, 450 manifest leaves with the scalar control flags; Section 6.3: 1,670,124,960
+    bytes in all).  The tensors get seeded random sizes (multiples of 256 bytes, a factor of four
+    between the smallest and the largest), the flags 2 to 64 bytes each, one flag after every
+    fourteenth tensor; the last tensor takes what is left, so the sizes add up to `total`."""
+    g = torch.Generator().manual_seed(seed)
+    flag_sizes = [int(x) for x in (2 ** torch.randint(1, 7, (flags,), generator=g))]
+    weights = 1.0 + 3.0 * torch.rand(tensors, generator=g)
+    room = total - sum(flag_sizes)
+    sizes = [int(room * float(w / weights.sum())) // 256 * 256 for w in weights]
+    sizes[-1] = room - sum(sizes[:-1])
+    assert min(sizes) > 0
+    out, every = [], tensors // flags
+    for i, n in enumerate(sizes):
+        out.append(n)
+        if (i + 1) % every == 0 and flag_sizes:
+            out.append(flag_sizes.pop())
+    assert sum(out) == total and len(out) == tensors + flags
+    return out

@@ -338,3 +338,49 @@ def test_engine_cache_as_sixty_leaves_gives_the_flat_image():
     wm.wm_decode_verify_leaves(wire_leaf, r_leaf.wire_len, dtable, job.n, job.chunk, crc_dst, job.ws, job.res_d)
     assert wm.read_result(job.res_d).ok and torch.equal(crc_dst, crc_flat)
     assert all(torch.equal(a, b) for a, b in zip(dst, leaves))
+
+
+def test_paper_shaped_leaf_table_gives_the_flat_image_and_scatters_back():
+    """450 leaves adding up to 1,670,124,960 bytes: 420 tensors of seeded random sizes with 30
+    flags of 2 to 64 bytes between them (the shape of the paper's movable set).  After the first
+    flag the tile grid no longer falls on 16-byte boundaries of the leaves, and some tiles cross
+    leaves.  The leaf-mode image must be the flat call's byte for byte (which the whole-image test
+    ties to the oracle; here chunks around every flag are also compared with the oracle directly),
+    and the decode must put every byte back where it came from and touch nothing else."""
+    cfg = inputs.CONFIGS["engine"]
+    n = inputs.PAPER_CACHE_BYTES
+    cur = inputs.make_cache(cfg, "cuda")[:n]
+    sizes = inputs.paper_leaf_sizes()
+    job = Job(n, cfg.chunk_bytes)
+    leaves, o = [], 0
+    for k in sizes:
+        leaves.append(cur[o:o + k].clone())
+        o += k
+    table = wm.make_leaf_table(leaves)
+    crc_flat = torch.zeros(job.nc, dtype=torch.int32, device="cuda")
+    crc_leaf = torch.zeros(job.nc, dtype=torch.int32, device="cuda")
+    wm.wm_encode(cur, job.chunk, None, crc_flat, job.wire, job.ws, job.res_e)
+    r_flat = wm.read_result(job.res_e)
+    wire_leaf = torch.empty_like(job.wire)
+    wm.wm_encode_leaves(table, n, job.chunk, None, crc_leaf, wire_leaf, job.ws, job.res_e)
+    r_leaf = wm.read_result(job.res_e)
+    assert r_flat.ok and r_leaf.ok
+    assert (r_leaf.wire_len, r_leaf.cache_crc, r_leaf.n_present) == (r_flat.wire_len, r_flat.cache_crc, r_flat.n_present)
+    assert torch.equal(wire_leaf[: r_leaf.wire_len], job.wire[: r_flat.wire_len]) and torch.equal(crc_leaf, crc_flat)
+    # the chunks that hold a flag, and the last (ragged) chunk, against the oracle
+    m, hdr, off, ln, crc, tab = job.meta()
+    flag_chunks, o = set(), 0
+    for k in sizes:
+        if k <= 64:
+            flag_chunks.add(o // job.chunk)
+        o += k
+    check_chunks_against_oracle(job, cur, sorted(flag_chunks)[:12] + [job.nc - 1], off, ln, crc, tab)
+    # decode into fresh leaves with guard bytes behind each
+    store = [torch.full((x.numel() + 16,), 0xC3, dtype=torch.uint8, device="cuda") for x in leaves]
+    dst = [b[: x.numel()] for b, x in zip(store, leaves)]
+    dtable = wm.make_leaf_table(dst)
+    crc_dst = torch.zeros(job.nc, dtype=torch.int32, device="cuda")
+    wm.wm_decode_verify_leaves(wire_leaf, r_leaf.wire_len, dtable, n, job.chunk, crc_dst, job.ws, job.res_d)
+    assert wm.read_result(job.res_d).ok and torch.equal(crc_dst, crc_flat)
+    assert all(torch.equal(a, b) for a, b in zip(dst, leaves))
+    assert all(bool((b[-16:] == 0xC3).all()) for b in store), "wrote past the end of a leaf"

@@ -185,6 +185,37 @@ def test_leaf_table_that_breaks_the_rules_is_rejected():
         assert all((x == 0x33).all() for x in dst) and not dcrc.any()
 
 
+@gpu
+def test_a_table_that_cuts_more_tiles_than_the_side_buffer_holds_is_refused():
+    """Tiles that cross leaf boundaries go through a side buffer of 2048 slots; 3000 leaves of one
+    tile and 16 bytes each cut 2999 tiles, which is refused as an argument error (the same cache as
+    1500 leaves of twice that size is accepted)."""
+    import torch
+    from paper_2607_10389_b200 import binding as wm
+    k = 3000
+    leaf = TILE + 16
+    nbytes, chunk = k * leaf, 4 * TILE
+    flat = torch.randint(0, 256, (nbytes,), dtype=torch.uint8, device="cuda")
+    nc = wm.num_chunks(nbytes, chunk)
+    ws, res = wm.new_workspace(nbytes, chunk), wm.new_result()
+    wire = torch.zeros(wm.wire_bound(nbytes, chunk), dtype=torch.uint8, device="cuda")
+    crc = torch.zeros(nc, dtype=torch.int32, device="cuda")
+    many = wm.make_leaf_table([flat[i * leaf:(i + 1) * leaf] for i in range(k)])
+    wm.wm_encode_leaves(many, nbytes, chunk, None, crc, wire, ws, res)
+    assert wm.read_result(res).status_name == "ERR_ARG"
+    fewer = wm.make_leaf_table([flat[i * 2 * leaf:(i + 1) * 2 * leaf] for i in range(k // 2)])
+    wm.wm_encode_leaves(fewer, nbytes, chunk, None, crc, wire, ws, res)
+    r = wm.read_result(res)
+    wire2 = torch.zeros_like(wire)
+    wm.wm_encode(flat, chunk, None, crc, wire2, ws, res)
+    assert r.ok and torch.equal(wire[: r.wire_len], wire2[: r.wire_len])
+    dst = torch.zeros_like(flat)
+    dmany = wm.make_leaf_table([dst[i * leaf:(i + 1) * leaf] for i in range(k)])
+    dcrc = torch.zeros_like(crc)
+    wm.wm_decode_verify_leaves(wire, r.wire_len, dmany, nbytes, chunk, dcrc, ws, res)
+    assert wm.read_result(res).status_name == "ERR_ARG" and not bool(dst.any()) and not bool(dcrc.any())
+
+
 def test_append_only_workload_dirties_only_the_chunks_that_hold_the_new_tokens():
     from paper_2607_10389_b200 import inputs
     cfg = inputs.CONFIGS["llm_append_small"]
