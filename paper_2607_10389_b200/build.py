@@ -25,8 +25,6 @@ def build(force: bool = False, verbose: bool = False) -> str:
     nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
     cmd = [nvcc, "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
            "-diag-suppress", "177", "-shared", "-Xcompiler", "-fPIC", "-o", OUT + ".tmp"] + SRC
-    for d in os.environ.get("WM_DEFINES", "").split():
-        cmd.insert(1, "-D" + d)
     if verbose:
         cmd.insert(1, "-Xptxas")
         cmd.insert(2, "-v")

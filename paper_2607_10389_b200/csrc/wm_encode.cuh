@@ -502,11 +502,7 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
         const uint32_t slY = (sl + 3u) & 7u;
         const uint32_t tYn = qY & kQTile;
         if (hotY) {
-#ifdef WM_AB_NOCRC
-            const uint32_t v = d[3];
-#else
             const uint32_t v = tile_digest_part(S, d, (qY & kQFirst) != 0, warp, lane);
-#endif
             // From here on the words are kept rotated left by one bit: each half then reads
             // [E | mantissa | a sign bit], E in its high byte (the two sign bits of a word
             // land in each other's half; the packing step puts them right).
@@ -529,9 +525,6 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
                 ent_w = anchor | (count << 8);
             }
             {
-#ifdef WM_AB_NOMINMAX
-            gw[0] = gw[1] = gw[2] = gw[3] = 100u | (4u << 8);
-#else
 #pragma unroll
             for (int j = 0; j < 4; j++) {
                 const uint32_t a0 = d[4 * j], a1 = d[4 * j + 1], a2 = d[4 * j + 2], a3 = d[4 * j + 3];
@@ -545,7 +538,6 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
                 const uint32_t emax = (__reduce_max_sync(0xFFFFFFFFu, mx) >> 8) & 0xFFu;
                 gw[j] = emin | ((32u - __clz(emax - emin)) << 8);
             }
-#endif
             }
             // Option ZEROS.  Unused memory: when all four groups have exponent 0 throughout (rare in live data)
             // look at the words themselves; a warp whose 2 KiB are all zero marks its first entry.
@@ -592,9 +584,7 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
                     publish_len(tYn, zero_tile ? 0u : const_tile ? 32u : ent_tile ? ent_tile_bytes(halfwords) : plane_len);
                 }
             }
-#ifndef WM_AB_NOTMEM
             tmem_store16(tmem_warp + 16u * (step & 3u), d);
-#endif
         } else if (is_tile(qY)) {
             // rare: a tile of an absent chunk (length 0) or the ragged last tile (stored raw)
             const bool present = qY >= kQPresent;
@@ -610,9 +600,7 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
         // ---- X: its words back from tensor memory, packed straight into the wire image
         const uint32_t tXn = qX & kQTile;
         if (is_hot(qX)) {
-#ifndef WM_AB_NOTMEM
             tmem_load16(tmem_warp + 16u * ((step + 1u) & 3u), d);
-#endif
             const uint32_t Smark = tc->ssum[sl];
             const bool ent_form = ENT && (Smark & kSumEnt) != 0u;
             const uint32_t Ssum = ent_form ? Smark & 0xFFFFu : Smark;       // halfwords, or the sum of the widths
@@ -671,7 +659,6 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
                 }
                 stg_u16(hw_dst + 2u * pend, acc & 0xFFFFu);
             } else if (packs) {
-#ifndef WM_AB_NOPACK
                 if (warp == 5) {           // (any one warp: not one that has a single-lane chore)
                     const uint32_t wt = tc->wtab[sl][lane];
                     stg_u16(dst + 2 * lane, desc_of(wt & 0xFFu, (wt >> 8) & 15u));
@@ -707,9 +694,6 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
                         default: break;
                     }
                 }
-#else
-                if (d[5] == 0x12345678u) stg_u8(dst + lane, d[1]);
-#endif
             } else if (ZEROS && Ssum == kSumConstTile) {
                 // the value (any word's low half, rotated back), then 30 zero bytes
                 if (warp == 5 && lane < 8u) st_stream_u32(dst + 4u * lane, lane == 0u ? __funnelshift_r(d[0], d[0], 1) & 0xFFFFu : 0u);

@@ -41,14 +41,8 @@ namespace wm {
 
 // ------------------------------------------------------------------ host side
 
-#ifndef WM_TEAMS
-#define WM_TEAMS 4
-#endif
-constexpr int kTeams = WM_TEAMS;            // encode: teams per block (plus the scanner warp)
-#ifndef WM_TEAMS_PLAIN
-#define WM_TEAMS_PLAIN 4
-#endif
-constexpr int kTeamsPlain = WM_TEAMS_PLAIN;  // checksum / decode: teams per block
+constexpr int kTeams = 4;        // encode: teams per block (plus the scanner warp)
+constexpr int kTeamsPlain = 4;   // checksum / decode: teams per block
 
 struct DeviceState {
     Tables* tables = nullptr;
