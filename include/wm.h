@@ -380,10 +380,9 @@ wm_status wm_decode_verify_opt(const void* wire, uint64_t wire_len, void* dst, c
 /*
  * wm_checksum_noalloc - wm_checksum for callers that cannot allocate device memory.
  * The paper has no counterpart to this call; it exists for hosts that may not call cudaMalloc
- * at the point where they need a checksum: code running inside a stream capture or under an
- * allocator that has been frozen for the life of a serving process, plug-ins that are handed
- * a stream and buffers but no allocation rights, and start-up or recovery paths that must not
- * touch the device heap.  Same result as wm_checksum, bit for bit, but the scratch memory and
+ * at the point where they need a checksum: code running under an allocator that has been
+ * frozen for the life of a serving process, plug-ins that are handed a stream and buffers but
+ * no allocation rights, and start-up or recovery paths that must not touch the device heap.  Same result as wm_checksum, bit for bit, but the scratch memory and
  * the constant tables sit in arrays built into the library image (about 1.2 MiB that every
  * GPU loading the library keeps until the process exits), so the call takes no workspace.
  *   - Limit: nbytes <= WM_NOALLOC_MAX_BYTES (4 GiB); larger inputs return WM_ERR_ARG and

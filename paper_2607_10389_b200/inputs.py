@@ -191,6 +191,40 @@ def before_append(cache_u8: torch.Tensor, cfg: CacheConfig, appended: int):
     return prev, mask
 
 
+def append_schedule(cfg: CacheConfig, steps: int, fill_to: float = 0.727):
+    """Token counts of an append-only run (Section 3.3: the window of the text model fills from
+    0.249 towards 0.727 while no step rewrites anything): `steps` appends that take the window
+    from cfg.fill to `fill_to` in equal parts, with one step in the middle that appends nothing
+    (an all-clean step).  Returns a list of (first_token, count)."""
+    first, last = filled_tokens(cfg), int(round(fill_to * cfg.shape[3]))
+    real = steps - 1
+    edges = [first + (last - first) * i // real for i in range(real + 1)]
+    out = [(edges[i], edges[i + 1] - edges[i]) for i in range(real)]
+    out.insert(real // 2, (edges[real // 2], 0))
+    return out
+
+
+def append_tokens(cache_u8: torch.Tensor, cfg: CacheConfig, first: int, count: int, seed: int) -> torch.Tensor:
+    """Append `count` tokens at position `first` of every (layer, key/value, head) row block, in
+    place, with fresh draws; nothing else is touched.  Returns the chunks that hold them (u8[n_chunks])."""
+    layers, two, heads, tokens, dim = cfg.shape
+    nc = (cfg.nbytes + cfg.chunk_bytes - 1) // cfg.chunk_bytes
+    mask = torch.zeros(nc, dtype=torch.uint8)
+    if count == 0:
+        return mask
+    g = _gen(seed, cache_u8.device)
+    view = cache_u8.view(torch.bfloat16).view(cfg.shape)
+    fresh = torch.randn((layers, two, heads, count, dim), generator=g, device=cache_u8.device)
+    fresh = torch.where(fresh == 0, torch.ones_like(fresh), fresh)       # (a token written is never all zero bits)
+    view[:, :, :, first:first + count] = fresh.to(torch.bfloat16)
+    row = dim * 2
+    for blk in range(layers * two * heads):
+        lo = (blk * tokens + first) * row
+        hi = (blk * tokens + first + count) * row
+        mask[lo // cfg.chunk_bytes:(hi - 1) // cfg.chunk_bytes + 1] = 1
+    return mask
+
+
 PAPER_CACHE_BYTES = 1_670_124_960      # the movable set of the paper's engine (Section 6.3)
 
 

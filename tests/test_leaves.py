@@ -264,3 +264,61 @@ def test_append_only_step_with_zero_tiles_matches_the_oracle():
             assert wm.read_result(res).ok and torch.equal(dst, cur)
     finally:
         wm.zero_tiles_enable(False)
+
+
+def test_append_only_schedule_fills_the_window_and_has_an_all_clean_step():
+    """The window fills from 0.249 to 0.727 over a run of appends (Section 3.3); every step dirties
+    exactly the chunks that hold its new tokens, the step that appends nothing is all clean and its
+    image is metadata only."""
+    from paper_2607_10389_b200 import inputs
+    cfg = inputs.CONFIGS["llm_append_small"]
+    cur = inputs.make_cache(cfg, "cpu")
+    sched = inputs.append_schedule(cfg, 6)
+    assert sched[0][0] == inputs.filled_tokens(cfg) and sum(c for _, c in sched) == round(0.727 * cfg.shape[3]) - sched[0][0]
+    assert [c for _, c in sched].count(0) == 1
+    crc = oracle.checksum(cur.numpy(), cfg.chunk_bytes)
+    for k, (first, count) in enumerate(sched):
+        prev = cur.clone()
+        mask = inputs.append_tokens(cur, cfg, first, count, seed=40 + k)
+        d, _ = oracle.dirty_diff(cur.numpy(), prev.numpy(), cfg.chunk_bytes)
+        assert np.array_equal(d, mask.numpy())
+        wire, crc, res = oracle.encode(cur.numpy(), cfg.chunk_bytes, dirty=d, crc_in=crc, zero_tiles=True)
+        if count == 0:
+            assert res.n_present == 0 and res.payload_bytes == 0 and res.wire_len == oracle.meta_end(cfg.nbytes, cfg.chunk_bytes)
+        else:
+            assert 0 < res.n_present <= d.size // 2
+        out, _, r = oracle.decode_verify(wire, cfg.nbytes, cfg.chunk_bytes, dst=prev.numpy(), dst_crc=oracle.checksum(prev.numpy(), cfg.chunk_bytes))
+        assert r.status == 0 and np.array_equal(out, cur.numpy())
+
+
+@gpu
+def test_append_only_schedule_on_the_gpu_matches_the_oracle_step_by_step():
+    import torch
+    from paper_2607_10389_b200 import binding as wm
+    from paper_2607_10389_b200 import inputs
+    cfg = inputs.CONFIGS["llm_append_small"]
+    cur = inputs.make_cache(cfg, "cuda")
+    n, chunk = cfg.nbytes, cfg.chunk_bytes
+    nc = wm.num_chunks(n, chunk)
+    ws, res = wm.new_workspace(n, chunk), wm.new_result()
+    wire = torch.zeros(wm.wire_bound(n, chunk), dtype=torch.uint8, device="cuda")
+    dirty = torch.zeros(nc, dtype=torch.uint8, device="cuda")
+    nd = torch.zeros(1, dtype=torch.int32, device="cuda")
+    crc = torch.from_numpy(oracle.checksum(cur.cpu().numpy(), chunk).view(np.int32).copy()).cuda()
+    dst, dcrc = cur.clone(), crc.clone()
+    for k, (first, count) in enumerate(inputs.append_schedule(cfg, 6)):
+        prev = cur.clone()
+        mask = inputs.append_tokens(cur, cfg, first, count, seed=40 + k)
+        wm.wm_dirty_diff(cur, prev, chunk, dirty, None, nd, ws)
+        assert torch.equal(dirty.cpu(), mask) and int(nd.item()) == int(mask.sum())
+        want_wire, want_crc, want = oracle.encode(cur.cpu().numpy(), chunk, dirty=mask.numpy(),
+                                                  crc_in=crc.cpu().numpy().view(np.uint32), zero_tiles=True)
+        wm.wm_encode_opt(cur, chunk, dirty, crc, wire, ws, res, wm.OPT_ZERO_TILES)
+        r = wm.read_result(res)
+        assert (r.status, r.wire_len, r.n_present, r.cache_crc) == (want.status, want.wire_len, want.n_present, want.cache_crc)
+        assert np.array_equal(wire[: r.wire_len].cpu().numpy(), want_wire)
+        assert np.array_equal(crc.cpu().numpy().view(np.uint32), want_crc)
+        if count == 0:
+            assert r.payload_bytes == 0
+        wm.wm_decode_verify_opt(wire, r.wire_len, dst, chunk, dcrc, ws, res, 0)
+        assert wm.read_result(res).ok and torch.equal(dst, cur) and torch.equal(dcrc, crc)

@@ -159,6 +159,34 @@ def test_five_bit_group_planes_by_hand():
     assert ep.tolist() == want.tolist()
 
 
+@pytest.mark.parametrize("d,length,want_bytes", [
+    # One element differs from its group's base, memory element 201 of group 0: row 3, word 4, high
+    # half, so coded position k = 8*4 + 2*3 + 1 = 39.  Bytes worked out on paper from the format text:
+    # width 2 (d = 10b): one 2-bit plane; k = 39 sits at bits 78-79 = byte 9, bits 6-7
+    (0b10, 64, {9: 0x80}),
+    # width 3 (d = 101b): 2-bit plane takes bits 0-1 (01b), then the 1-bit plane (from byte 64) takes
+    # bit 2: bit 39 = byte 4, bit 7
+    (0b101, 96, {9: 0x40, 64 + 4: 0x80}),
+    # width 6 (d = 101101b): 4-bit plane takes 1101b into the high nibble of byte 19 (k odd), the
+    # 2-bit plane (from byte 128) takes 10b
+    (0b101101, 192, {19: 0xD0, 128 + 9: 0x80}),
+    # width 7 (d = 1011010b): 4-bit plane 1010b, 2-bit plane 01b, 1-bit plane (from byte 192) 1
+    (0b1011010, 224, {19: 0xA0, 128 + 9: 0x40, 192 + 4: 0x80}),
+])
+def test_two_and_three_plane_groups_by_hand(d, length, want_bytes):
+    E = np.full(8192, 60)
+    E[201] = 60 + d
+    wire, _, _ = oracle.encode(_bf16_tile(E), TILE)
+    ep = wire[96 + 64 + 8192:]
+    assert len(ep) == length
+    want = np.zeros(length, dtype=np.uint8)
+    for at, v in want_bytes.items():
+        want[at] = v
+    assert ep.tolist() == want.tolist()
+    desc = struct.unpack_from("<H", wire, 96)[0]
+    assert desc & 0xFF == 60 and (desc >> 8) & 15 == d.bit_length()
+
+
 def test_raw_fallback_never_expands_beyond_metadata():
     rng = np.random.default_rng(2)
     n, chunk = 8 * TILE, 4 * TILE
