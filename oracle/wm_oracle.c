@@ -430,15 +430,22 @@ static int ent_header_bad(const uint8_t* in, uint32_t entry)
     return ((8256u + 2u * total + 31u) / 32u) != (entry & 0x7FFFu);
 }
 
-/* Read the eight streams of an ENT tile whose header fits.  With dst != NULL the tile is
- * written there.  Returns 0 when every stream is used up exactly and the bits left over in every
- * strand's last halfword are zero, 1 otherwise. */
-static int decode_ent_tile(const uint8_t* in, uint8_t* dst)
+/* Read the eight streams of an ENT tile whose header fits (`entry`: its tile-table entry).  With
+ * dst != NULL the tile is written there.  Returns 0 when every byte of the tile is accounted for:
+ * every stream used up exactly, the bits left over in every strand's last halfword zero, every
+ * anchor the rounded mean of the exponents its share decodes to (what the encoder writes), the 40
+ * spare header bytes and the fill behind the last stream zero; 1 otherwise.  With these no bit of
+ * an ENT tile can change without the tile being refused or the decoded bytes changing. */
+static int decode_ent_tile(const uint8_t* in, uint8_t* dst, uint32_t entry)
 {
     const uint8_t* stream = in + 64 + 8192;
     int bad = 0;
+    uint32_t hw_total = 0;
+    for (uint32_t i = 24; i < 64; i++)
+        if (in[i]) bad = 1;
     for (uint32_t s = 0; s < 8; s++) {
-        uint32_t anchor = in[s], count = get16(in + 8 + 2u * s), pos = 0;
+        uint32_t anchor = in[s], count = get16(in + 8 + 2u * s), pos = 0, esum = 0;
+        hw_total += count;
         uint32_t buf[32] = {0}, avail[32] = {0};
         for (uint32_t i = 0; i < 32; i++)
             for (uint32_t l = 0; l < 32; l++) {
@@ -453,6 +460,7 @@ static int decode_ent_tile(const uint8_t* in, uint8_t* dst)
                 uint32_t len = ent_parse(buf[l], anchor, &E);
                 buf[l] >>= len;
                 avail[l] -= len;
+                esum += E;
                 if (dst) {
                     uint32_t e = ent_elem(s, l, i);
                     uint32_t SM = in[64u + 256u * (e / 256u) + coded_pos(e % 256u)];
@@ -462,8 +470,11 @@ static int decode_ent_tile(const uint8_t* in, uint8_t* dst)
         if (pos != count) bad = 1;
         for (uint32_t l = 0; l < 32; l++)
             if (buf[l]) bad = 1;                 /* the fill bits of a strand's last halfword are zero */
+        if (((esum + 512u) >> 10) != anchor) bad = 1;
         stream += 2u * count;
     }
+    for (uint32_t i = 8256u + 2u * hw_total; i < 32u * (entry & 0x7FFFu); i++)
+        if (in[i]) bad = 1;
     return bad;
 }
 
@@ -707,7 +718,9 @@ static void decode_pack_tile(const uint8_t* in, uint8_t* dst)
  *  4 every PACK tile, in tile order: descriptors (w <= 8, check nibble) -> DESC,
  *    then 258 + sum w equals the tile entry                         -> STRUCT;
  *    every ENT tile: stream counts in range and adding up to the entry -> STRUCT,
- *    then each stream used up exactly by its 1024 codewords, fill bits zero -> DESC
+ *    then each stream used up exactly by its 1024 codewords, fill bits zero, anchors the
+ *    rounded means of what they decode, spare header bytes and end fill zero -> DESC;
+ *    every CONST tile: the 30 bytes behind the value zero            -> DESC
  *    (status of the lowest failing tile; n_bad_chunks = chunks with a failing tile)
  *  5 decode; CRC32C of each decoded chunk equals its directory CRC  -> CHUNK_CRC
  *  6 absent chunk: dst_crc_inout[c] equals its directory CRC        -> STALE
@@ -815,11 +828,15 @@ int wmo_decode_verify_opt(const uint8_t* wire, uint64_t wire_len, uint8_t* dst, 
                     /* ENT tile: the header against the entry -> STRUCT, then every stream must be used up exactly -> DESC */
                     int tile_status = WMO_OK;
                     if (ent_header_bad(payload + off, e)) tile_status = WMO_ERR_STRUCT;
-                    else if (decode_ent_tile(payload + off, NULL)) tile_status = WMO_ERR_DESC;
+                    else if (decode_ent_tile(payload + off, NULL, e)) tile_status = WMO_ERR_DESC;
                     if (tile_status != WMO_OK) {
                         chunk_bad = 1;
                         if (status == WMO_OK) status = tile_status;
                     }
+                } else if (e == 2u) {
+                    /* CONST tile: the 30 bytes behind the value are zero -> DESC */
+                    for (uint32_t k = 2; k < 32; k++)
+                        if (payload[off + k]) { chunk_bad = 1; if (status == WMO_OK) status = WMO_ERR_DESC; break; }
                 } else if (e >= 258u && e <= 511u) {
                     const uint8_t* in = payload + off;
                     int tile_status = WMO_OK; uint32_t S = 0;
@@ -856,7 +873,7 @@ int wmo_decode_verify_opt(const uint8_t* wire, uint64_t wire_len, uint8_t* dst, 
                 uint64_t tlen = (e == 0xFFFFu) ? clen - i * WMO_TILE : (e == 1u) ? 0 : (e == 2u) ? 32u : 32u * (uint64_t)(e & 0x7FFFu);
                 if (e == 1u) memset(out + i * WMO_TILE, 0, WMO_TILE);
                 else if (e == 2u) { for (uint32_t k = 0; k < 8192u; k++) memcpy(out + i * WMO_TILE + 2u * k, payload + off, 2); }
-                else if (e != 0xFFFFu && (e & 0x8000u)) decode_ent_tile(payload + off, out + i * WMO_TILE);
+                else if (e != 0xFFFFu && (e & 0x8000u)) decode_ent_tile(payload + off, out + i * WMO_TILE, e);
                 else if (e == 512u || e == 0xFFFFu) memcpy(out + i * WMO_TILE, payload + off, tlen);
                 else decode_pack_tile(payload + off, out + i * WMO_TILE);
                 off += tlen;

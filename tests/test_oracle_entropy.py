@@ -334,3 +334,55 @@ def test_golden_worked_examples():
                     seen[i] = True
             if name != "escapes":
                 assert not stream[~seen].any(), name
+
+
+def test_no_bit_of_an_image_with_both_options_can_flip_unnoticed():
+    """Every single bit of a small image that holds an ENT tile, a CONST tile, a ZERO tile and a
+    ragged tail (zero-tile and entropy options together): flipped, the image is refused.  That
+    includes the bytes that carry no data: the spare bytes of an ENT tile's header, the fill behind
+    its last stream, the zeros behind a CONST tile's value; and the anchors, which must be the
+    rounded means of what their shares decode to."""
+    a = np.concatenate([_gauss(TILE // 2, 31).view(np.uint8), np.full(8192, 0xFF80, "<u2").view(np.uint8),
+                        np.zeros(TILE, np.uint8), _gauss(150, 32).view(np.uint8)])
+    n, chunk = a.size, 4 * TILE
+    wire, crc, res = oracle.encode(a, chunk, zero_tiles=True, entropy=True)
+    nt = oracle.num_tiles(n)
+    tab = wire[64 + 16: 64 + 16 + 2 * nt].view(np.uint16).tolist()
+    assert tab[0] & 0x8000 and tab[0] != 0xFFFF and tab[1:] == [2, 1, 0xFFFF]
+    out, _, r = oracle.decode_verify(wire, n, chunk, expect_entropy=True)
+    assert r.status == 0 and np.array_equal(out, a)
+    accepted = []
+    for bit in range(wire.size * 8):
+        w = wire.copy()
+        w[bit // 8] ^= 1 << (bit % 8)
+        if oracle.decode_verify(w, n, chunk, expect_entropy=True)[2].status == 0:
+            accepted.append(bit)
+    assert not accepted, f"{len(accepted)} flipped bits were accepted, first at byte {accepted[0] // 8}"
+
+
+def test_spare_bytes_and_anchors_of_coded_tiles_are_checked():
+    v = _gauss(TILE // 2, 33)
+    wire, _, res = oracle.encode(v.view(np.uint8), TILE, entropy=True)
+    me = oracle.meta_end(TILE, TILE)
+    for at in (me + 24, me + 63, res.wire_len - 1):          # spare header bytes; the last fill byte, if the tile has fill
+        if at == res.wire_len - 1:
+            counts = wire[me + 8: me + 24].view(np.uint16).astype(np.int64)
+            if 8256 + 2 * int(counts.sum()) == res.wire_len - me:
+                continue
+        w = wire.copy()
+        w[at] ^= 0x40
+        assert oracle.decode_verify(w, TILE, TILE)[2].status_name == "ERR_DESC", at
+    # an anchor that moves shifts everything its share decodes to, which the chunk CRC sees ...
+    w = wire.copy()
+    w[me + 3] += 1
+    assert oracle.decode_verify(w, TILE, TILE)[2].status_name == "ERR_CHUNK_CRC"
+    # ... unless every codeword of the share is an escape (the exponent itself): then only the rule
+    # that an anchor is the rounded mean of its share stands between a flipped anchor bit and OK
+    E = np.full(8192, 120)
+    E[3 * 1024: 4 * 1024] = np.tile([0, 255], 512)              # share 3: mean 127.5 -> anchor 128, all escapes
+    t = ((E << 7) | 0x15).astype("<u2")
+    wire, _, res = oracle.encode(t.view(np.uint8), TILE, entropy=True, ent_only=True)
+    assert wire[me + 3] == 128 and oracle.decode_verify(wire, TILE, TILE)[2].status == 0
+    w = wire.copy()
+    w[me + 3] ^= 4
+    assert oracle.decode_verify(w, TILE, TILE)[2].status_name == "ERR_DESC"
