@@ -327,6 +327,65 @@ def precopy_loop(wm, inputs, cfg, cur, prev, dst, wire_a, ws_a, dev, peak, steps
                     "and b for the destination's decode kernel (WM_OPT_BLOCKS)"}
 
 
+def append_loop(wm, inputs, cfg, cur, dst, wire, ws, dev, steps=8):
+    """The append-only run of the text-model cache: the window fills from cfg.fill to 0.727 in
+    `steps` appends, one of which appends nothing.  Per step wm_dirty_diff -> wm_encode of the dirty
+    chunks (zero-tile option) -> wm_decode_verify into the destination, on one stream, timed on
+    the device; the caches of all steps are generated beforehand."""
+    import torch
+    N, C = cfg.nbytes, cfg.chunk_bytes
+    nc = wm.num_chunks(N, C)
+    sched = inputs.append_schedule(cfg, steps)
+    states, masks = [cur], []
+    for k, (first, count) in enumerate(sched):
+        nxt = states[-1].clone()
+        masks.append(inputs.append_tokens(nxt, cfg, first, count, seed=7000 + k))
+        states.append(nxt)
+    crc_src = torch.zeros(nc, dtype=torch.int32, device=dev)
+    crc_dst = torch.zeros(nc, dtype=torch.int32, device=dev)
+    dirty = torch.zeros(nc, dtype=torch.uint8, device=dev)
+    n_dirty = torch.zeros(1, dtype=torch.int32, device=dev)
+    res_e, res_d = wm.new_result(dev), wm.new_result(dev)
+    wm.wm_encode_opt(cur, C, None, crc_src, wire, ws, res_e, wm.OPT_ZERO_TILES)
+    r = wm.read_result(res_e)
+    wm.wm_decode_verify_opt(wire, r.wire_len, dst, C, crc_dst, ws, res_d, 0)
+    if not (r.ok and wm.read_result(res_d).ok and torch.equal(dst, cur)):
+        raise SystemExit("append loop: levelling move failed")
+    out = []
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(2)]
+    for k in range(steps):
+        a, b = states[k + 1], states[k]
+        lens = None
+        for rep in range(2):                   # first time: lengths and checks; second time: timed, no host read inside
+            if rep == 1:
+                dst.copy_(b)
+                crc_src.copy_(crc_keep)
+                crc_dst.copy_(crc_keep)
+                torch.cuda.synchronize()
+                ev[0].record()
+            else:
+                crc_keep = crc_src.clone()
+            wm.wm_dirty_diff(a, b, C, dirty, None, n_dirty, ws)
+            wm.wm_encode_opt(a, C, dirty, crc_src, wire, ws, res_e, wm.OPT_ZERO_TILES)
+            if rep == 0:
+                rr = wm.read_result(res_e)
+                if not rr.ok or rr.n_present != int(masks[k].sum()):
+                    raise SystemExit(f"append loop: step {k}: encode failed or wrong dirty count")
+                lens = rr
+            wm.wm_decode_verify_opt(wire, lens.wire_len, dst, C, crc_dst, ws, res_d, 0)
+            if rep == 1:
+                ev[1].record()
+            torch.cuda.synchronize()
+            if not wm.read_result(res_d).ok or not torch.equal(dst, a):
+                raise SystemExit(f"append loop: step {k} did not arrive")
+        out.append({"fill_after": (sched[k][0] + sched[k][1]) / cfg.shape[3], "appended_tokens": sched[k][1],
+                    "dirty_fraction": lens.n_present / nc, "wire_bytes": lens.wire_len, "payload_bytes": lens.payload_bytes,
+                    "ms": ev[0].elapsed_time(ev[1])})
+    del states
+    return {"steps": out, "note": "one stream, device time of diff + encode(dirty chunks, zero-tile option) + decode-verify-install "
+                                  "per append; the step that appends nothing is all clean: its image is the metadata alone"}
+
+
 def leaf_mode(wm, cfg, cur, wire, ws, dev, W, peak, reps=20):
     """wm_encode_leaves / wm_decode_verify_leaves on layers x {key, value} separate tensors."""
     import torch
@@ -810,6 +869,11 @@ def main():
     if not args.no_loop and args.workload in ("engine", "engine_256m"):
         loop = precopy_loop(wm, inputs_mod, cfg, cur, prev, shadow, wire, ws, dev, peak)
 
+    # the append-only run of the text-model cache (window fill 0.249 -> 0.727, with an all-clean step)
+    append = None
+    if not args.no_loop and cfg.kind == "llm":
+        append = append_loop(wm, inputs_mod, cfg, cur, shadow, wire, ws, dev)
+
     # leaf mode: the same cache held as one key and one value tensor per layer, encoded and
     # decoded in place, beside the flatten and rehydrate copies that this makes unnecessary
     leaf = None
@@ -937,7 +1001,7 @@ def main():
                        "wire_bytes": W, "ratio": W / N, "dirty_chunks": n_rewritten, "n_chunks": nc,
                        "l2": "inputs larger than L2 (no flush needed)", "parallelism": "replicas only",
                        "zero_tiles": bool(args.zero_tiles), "entropy": bool(args.entropy)},
-            "calls": per_call, "roofline": roofline, "precopy_loop": loop, "leaf_mode": leaf, "entropy_option": ent, "tail_schedule": tail,
+            "calls": per_call, "roofline": roofline, "precopy_loop": loop, "append_loop": append, "leaf_mode": leaf, "entropy_option": ent, "tail_schedule": tail,
             "cpu_baseline": base, "e2e": e2e,
             "gpu_launches": gpu_launches, "clocks": clocks,
         }

@@ -227,8 +227,11 @@ wm_status wm_encode(const void* cache, uint64_t nbytes, uint32_t chunk_bytes, co
  *   4 coded tiles in tile order; the status is that of the lowest failing tile.  PACK tile:
  *     descriptors valid (WM_ERR_DESC), then 258 + sum w equals the tile entry (WM_ERR_STRUCT).
  *     ENT tile (images with flags bit2): the eight stream counts within 128..1024 and adding up
- *     to the entry (WM_ERR_STRUCT), then every stream used up exactly by its 1024 codewords and
- *     the fill bits of every strand zero (WM_ERR_DESC)
+ *     to the entry (WM_ERR_STRUCT), then every stream used up exactly by its 1024 codewords, the
+ *     fill bits of every strand zero, every anchor the rounded mean of the exponents its share
+ *     decodes to, the header's 40 spare bytes and the fill behind the last stream zero
+ *     (WM_ERR_DESC).  CONST tile (images with flags bit1): the 30 bytes behind the value zero
+ *     (WM_ERR_DESC).  No byte of a coded tile is left unaccounted for
  *   5 CRC32C of every decoded chunk equals its directory CRC       WM_ERR_CHUNK_CRC
  *   6 absent chunk: dst_crc_inout[c] equals its directory CRC      WM_ERR_STALE
  *   7 the directory CRCs combine to header.cache_crc               WM_ERR_CACHE_CRC
@@ -303,7 +306,9 @@ void wm_zero_tiles_enable(int on);
  *   Layout: anchor[8] u8 | count[8] u16 (halfwords per stream) | 40 zero bytes | SM[8192] as in
  *   a PACK tile | the eight streams | zero fill to a multiple of 32 bytes.
  * Decode checks (step 4): counts within 128..1024 and adding up to the entry (else WM_ERR_STRUCT);
- * every stream used up exactly and the fill bits of every strand zero (else WM_ERR_DESC).
+ * every stream used up exactly, the fill bits of every strand, the 40 spare header bytes and the
+ * fill behind the last stream zero, every anchor equal to the formula above applied to what its
+ * share decodes to (else WM_ERR_DESC).
  */
 void wm_entropy_enable(int on);
 

@@ -439,6 +439,19 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
                         avail -= len;
                     }
                     if (__any_sync(0xFFFFFFFFu, buf != 0u) || pos != mine) verdict = 1;
+                    // the anchor must be what the encoder writes: the rounded mean of the share's exponents
+                    // (otherwise the anchor of a share that holds escapes only could change unnoticed)
+                    uint32_t esum = 0;
+#pragma unroll
+                    for (int j = 0; j < 8; j++) esum = __dp4a(ew[j], 0x01010101u, esum);
+                    if (((__reduce_add_sync(0xFFFFFFFFu, esum) + 512u) >> 10) != anchor) verdict = 1;
+                    // the bytes that carry nothing are zero: the header's spare 40, the fill behind the last stream
+                    if (warp == 0u) {
+                        const uint32_t spare = (lane >= 6u && lane < 16u) ? lds_now<0>(stage_s + 4u * lane) : 0u;
+                        const uint32_t fill_at = 8256u + 2u * total + 2u * lane;
+                        const uint32_t fill = fill_at < 32u * (e & 0x7FFFu) ? lds_now_u16(stage_s + fill_at) : 0u;
+                        if (__any_sync(0xFFFFFFFFu, (spare | fill) != 0u)) verdict = 1;
+                    }
 #pragma unroll
                     for (int j = 0; j < 4; j++) {
                         sm[j] = j == 0 ? lds_now_v2<0>(sm_s) : j == 1 ? lds_now_v2<256>(sm_s) : j == 2 ? lds_now_v2<512>(sm_s) : lds_now_v2<768>(sm_s);
@@ -493,7 +506,19 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
             // a tile of zeros (nothing was shipped) or of one value (the first two bytes of its 32):
             // from here on it goes the way of a raw tile
             uint32_t v = 0;
-            if (e == 2u) v = __ldg(reinterpret_cast<const unsigned short*>(payload + tc->slot[it & 3u].src)) * 0x10001u;
+            if (e == 2u) {
+                // (the value's 32 bytes: the value itself, and 30 bytes that must be zero)
+                const uint32_t* cp = reinterpret_cast<const uint32_t*>(payload + tc->slot[it & 3u].src);
+                const uint32_t x = lane < 8u ? __ldg(cp + lane) : 0u;
+                v = (__shfl_sync(0xFFFFFFFFu, x, 0) & 0xFFFFu) * 0x10001u;
+                if (__any_sync(0xFFFFFFFFu, (lane == 0u ? x >> 16 : x) != 0u)) {       // every warp reaches the same verdict
+                    decoded = false;
+                    if (leader) {
+                        atomicMin(&ws.ctrl->bad4_key, (unsigned long long)t * 2ull);
+                        atomicOr(&ws.cflag[chunk_of(g, t)], CF_BAD4);
+                    }
+                }
+            }
 #pragma unroll
             for (int i = 0; i < 16; i++) w[i] = v;
         }

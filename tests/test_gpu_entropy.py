@@ -265,3 +265,40 @@ def test_ent_repeatable_under_load(wm):
         assert r.status == 0 and torch.equal(got, first)
         out, _, rd = _run_decode(wm, got.cpu().numpy(), a.size, cfg.chunk_bytes)
         assert rd.status == 0 and np.array_equal(out, a)
+
+
+def test_bits_that_carry_no_data_are_checked_like_the_oracle_checks_them(wm):
+    """An image with an ENT tile, a CONST tile, a ZERO tile and a ragged tail.  Every bit of the
+    metadata, of the ENT tile's header, of its last 64 bytes (the end fill), of the CONST tile's 32
+    bytes, and a sample of all the others is flipped in turn; each time the verdict (status, first
+    bad chunk, count) is the oracle's, and it is never OK."""
+    import torch
+    a = np.concatenate([_gauss(TILE // 2, 31).view(np.uint8), np.full(8192, 0xFF80, "<u2").view(np.uint8),
+                        np.zeros(TILE, np.uint8), _gauss(150, 32).view(np.uint8)])
+    n, chunk = a.size, 4 * TILE
+    want_wire, _, want = oracle.encode(a, chunk, zero_tiles=True, entropy=True)
+    opt = wm.OPT_ZERO_TILES | wm.OPT_ENTROPY
+    ws, res = wm.new_workspace(n, chunk), wm.new_result()
+    wire = torch.zeros(wm.wire_bound(n, chunk), dtype=torch.uint8, device="cuda")
+    crc = torch.zeros(1, dtype=torch.int32, device="cuda")
+    wm.wm_encode_opt(torch.from_numpy(a).cuda(), chunk, None, crc, wire, ws, res, opt)
+    r = wm.read_result(res)
+    assert r.ok and np.array_equal(wire[: r.wire_len].cpu().numpy(), want_wire)
+    me = oracle.meta_end(n, chunk)
+    ent_len = 32 * (int(want_wire[64 + 16: 64 + 18].view(np.uint16)[0]) & 0x7FFF)
+    bits = set(range(me * 8)) | set(range(me * 8, (me + 64) * 8)) | set(range((me + ent_len - 64) * 8, (me + ent_len + 32) * 8))
+    rng = np.random.default_rng(3)
+    bits |= set(int(b) for b in rng.integers(0, r.wire_len * 8, 1500))
+    dst = torch.zeros(n, dtype=torch.uint8, device="cuda")
+    dcrc = torch.zeros(1, dtype=torch.int32, device="cuda")
+    for bit in sorted(bits):
+        wire[bit // 8] ^= 1 << (bit % 8)
+        wm.wm_decode_verify_opt(wire, r.wire_len, dst, chunk, dcrc, ws, res, wm.OPT_ENTROPY)
+        rd = wm.read_result(res)
+        w = want_wire.copy()
+        w[bit // 8] ^= 1 << (bit % 8)
+        o = oracle.decode_verify(w, n, chunk, expect_entropy=True)[2]
+        assert rd.status != 0 and (rd.status, rd.first_bad_chunk, rd.n_bad_chunks) == (o.status, o.first_bad_chunk, o.n_bad_chunks), bit
+        wire[bit // 8] ^= 1 << (bit % 8)
+    wm.wm_decode_verify_opt(wire, r.wire_len, dst, chunk, dcrc, ws, res, wm.OPT_ENTROPY)
+    assert wm.read_result(res).ok and np.array_equal(dst.cpu().numpy(), a)
