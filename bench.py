@@ -650,6 +650,8 @@ def main():
     ap.add_argument("--no-loop", action="store_true", help="skip the pre-copy step loop")
     ap.add_argument("--zero-tiles", action="store_true", help="encoder option: all-zero tiles as table entries")
     ap.add_argument("--entropy", action="store_true", help="codec option: entropy-coded exponents (ENT tiles) in every call")
+    ap.add_argument("--variant", default="plain", choices=["plain", "masked", "leaves", "paper_leaves", "xxh64", "xxh64_64k"],
+                    help="with --profile: which calls make up a step (for profiler captures of the other kernel variants)")
     ap.add_argument("--profile", action="store_true",
                     help="profiler capture mode: round-trip check, warm-up and timed steps only")
     args = ap.parse_args()
@@ -731,6 +733,57 @@ def main():
     if int(n_dirty.item()) != n_rewritten:
         raise SystemExit("dirty count differs from the generated pattern")
     W = r.wire_len
+
+    if args.profile and args.variant != "plain":
+        # profiler captures of the other kernel variants: a step is the calls that run them
+        if args.variant == "masked":
+            # a pre-copy round: diff against the previous snapshot, encode the dirty chunks only,
+            # decode into a destination that holds the previous snapshot
+            crc_prev = torch.zeros(nc, dtype=torch.int32, device=dev)
+            wm.wm_checksum(prev, C, crc_prev, ws)
+            wm.wm_dirty_diff(cur, prev, C, dirty, dirty_idx, n_dirty, ws)
+            crc_m = crc_prev.clone()
+            wm.wm_encode(cur, C, dirty, crc_m, wire, ws, res_e)
+            wl = wm.read_result(res_e).wire_len
+
+            def step():
+                shadow.copy_(prev)
+                crc_m.copy_(crc_prev)
+                crc_dst.copy_(crc_prev)
+                wm.wm_dirty_diff(cur, prev, C, dirty, dirty_idx, n_dirty, ws)
+                wm.wm_encode(cur, C, dirty, crc_m, wire, ws, res_e)
+                wm.wm_decode_verify(wire, wl, shadow, C, crc_dst, ws, res_d)
+        elif args.variant in ("leaves", "paper_leaves"):
+            if args.variant == "leaves":
+                n_leaves = cfg.shape[0] * cfg.shape[1]
+                sizes, n_l = [N // n_leaves] * n_leaves, N
+            else:       # the paper-shaped table scaled to this cache: the same 450 sizes in proportion
+                full = inputs_mod.paper_leaf_sizes()
+                sizes = [max(2, s * N // inputs_mod.PAPER_CACHE_BYTES // 2 * 2) for s in full]
+                sizes[-1] += N - sum(sizes)
+                n_l = N
+            src_l, o = [], 0
+            for k in sizes:
+                src_l.append(cur[o:o + k].clone())
+                o += k
+            dst_l = [torch.empty_like(x) for x in src_l]
+            ts, td = wm.make_leaf_table(src_l, dev), wm.make_leaf_table(dst_l, dev)
+            wm.wm_encode_leaves(ts, n_l, C, None, crc_b, wire, ws, res_e)
+            wl = wm.read_result(res_e).wire_len
+
+            def step():
+                wm.wm_encode_leaves(ts, n_l, C, None, crc_b, wire, ws, res_e)
+                wm.wm_decode_verify_leaves(wire, wl, td, n_l, C, crc_dst, ws, res_d)
+        else:
+            xc = C if args.variant == "xxh64" else 65536
+            hashes = torch.zeros(wm.num_chunks(N, xc), dtype=torch.int64, device=dev)
+
+            def step():
+                wm.wm_checksum_xxh64(cur, xc, 0, hashes)
+        step()
+        torch.cuda.synchronize()
+        if not (wm.read_result(res_e).ok and wm.read_result(res_d).ok):
+            raise SystemExit("profile variant: a call failed")
 
     for _ in range(args.warmup):
         step()
