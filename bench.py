@@ -607,11 +607,12 @@ def run_reference(args):
     cfg = inputs.CONFIGS[name]
     sample_chunks = 16
     n = min(cfg.nbytes, sample_chunks * cfg.chunk_bytes)
-    # the sample is the head of a reduced cache of the same recipe (drawn on the CPU)
-    small = inputs.CONFIGS["engine_small"] if cfg.kind == "kv" else cfg
-    cur = inputs.make_cache(small, "cpu").numpy()
-    reps = -(-n // cur.size)
-    cur = np.tile(cur, reps)[:n].copy()
+    # the sample is the head of the workload's own cache: its first layers, drawn with the same
+    # generator on the same kind of device as the GPU arm draws them (torch is plumbing here: it
+    # makes the input, the timed work is the oracle's on the host cores)
+    import torch
+    draw_on = "cuda" if torch.cuda.is_available() else "cpu"
+    cur = inputs.make_cache(cfg, draw_on, head_bytes=n).cpu().numpy()[:n].copy()
     prev = cur.copy()
     nc = n // cfg.chunk_bytes
     mask = inputs.step_pattern(nc, 1, 0.75, seed=cfg.seed + 100).numpy()
@@ -625,7 +626,7 @@ def run_reference(args):
         oracle_step(cur, prev, cfg.chunk_bytes)
     dt = (time.perf_counter() - t) / args.steps
     v = n / dt / 1e9
-    sample = f"{n} bytes ({nc} chunks of {cfg.chunk_bytes}) of the {name} recipe per step, single thread"
+    sample = f"the first {n} bytes ({nc} chunks of {cfg.chunk_bytes}) of the {name} cache per step, single thread"
     print(json.dumps({
         "impl": "reference", "metric": METRIC,
         "value": v, "unit": "GB/s", "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,

@@ -68,9 +68,16 @@ def _gen(seed: int, device) -> torch.Generator:
     return g
 
 
-def make_cache(cfg: CacheConfig, device="cpu") -> torch.Tensor:
-    """Return the cache as a flat uint8 tensor of cfg.nbytes bytes on `device`."""
+def make_cache(cfg: CacheConfig, device="cpu", head_bytes: int | None = None) -> torch.Tensor:
+    """Return the cache as a flat uint8 tensor of cfg.nbytes bytes on `device`.  With `head_bytes`
+    only the leading layers that cover that many bytes are drawn (the same bytes the whole cache
+    begins with: layers are drawn one after the other from one generator)."""
     device = torch.device(device)
+    if head_bytes is not None and cfg.kind in ("kv", "gauss"):
+        per_layer = cfg.nbytes // cfg.shape[0]
+        keep = min(cfg.shape[0], -(-head_bytes // per_layer))
+        head = CacheConfig(cfg.name, (keep,) + tuple(cfg.shape[1:]), keep * per_layer, cfg.chunk_bytes, cfg.seed, cfg.kind, cfg.fill)
+        return make_cache(head, device)
     g = _gen(cfg.seed, device)
     if cfg.kind == "bytes":
         out = torch.empty(cfg.nbytes, dtype=torch.uint8, device=device)

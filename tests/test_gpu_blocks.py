@@ -56,3 +56,36 @@ def test_a_block_cap_of_one_is_refused_for_encode():
     crc = torch.zeros(1, dtype=torch.int32, device="cuda")
     with pytest.raises(wm.WmError, match="ERR_ARG"):
         wm.wm_encode_opt(cur, 65536, None, crc, wire, ws, res, wm.opt_blocks(1))
+
+
+def test_placement_is_repeatable_over_many_moves_and_block_counts():
+    """Which team gets which tile first changes from run to run and with the number of blocks; the
+    bytes must not.  400 moves of a 64 MiB cache, every option set, block counts drawn at random:
+    every image equals the first of its option set byte for byte, every round trip returns the
+    cache, and no call ends in a timeout."""
+    cfg = inputs.CONFIGS["engine_small"]
+    g = torch.Generator(device="cuda").manual_seed(77)
+    n, chunk = 64 << 20, 1 << 20
+    cur = (torch.randn(n // 2, generator=g, device="cuda") * 3).to(torch.bfloat16).view(torch.uint8)
+    cur[5 << 20: 6 << 20] = 0
+    nc = wm.num_chunks(n, chunk)
+    ws, res = wm.new_workspace(n, chunk), wm.new_result()
+    wire = torch.zeros(wm.wire_bound(n, chunk), dtype=torch.uint8, device="cuda")
+    crc = torch.zeros(nc, dtype=torch.int32, device="cuda")
+    dst = torch.zeros(n, dtype=torch.uint8, device="cuda")
+    dcrc = torch.zeros(nc, dtype=torch.int32, device="cuda")
+    rng = np.random.default_rng(5)
+    first = {}
+    for i in range(400):
+        opt = int(rng.integers(0, 4))
+        be, bd = int(rng.choice([0, 2, 5, 37, 74, 111, 148])), int(rng.choice([0, 1, 5, 37, 74, 111, 148]))
+        wm.wm_encode_opt(cur, chunk, None, crc, wire, ws, res, opt | wm.opt_blocks(be))
+        r = wm.read_result(res)
+        assert r.ok, (i, r.status_name)
+        img = wire[: r.wire_len]
+        if opt not in first:
+            first[opt] = (img.clone(), crc.clone())
+        assert torch.equal(img, first[opt][0]) and torch.equal(crc, first[opt][1]), (i, opt, be)
+        if i % 4 == 0:
+            wm.wm_decode_verify_opt(wire, r.wire_len, dst, chunk, dcrc, ws, res, (opt & wm.OPT_ENTROPY) | wm.opt_blocks(bd))
+            assert wm.read_result(res).ok and torch.equal(dst, cur) and torch.equal(dcrc, crc), (i, opt, bd)

@@ -269,7 +269,7 @@ def test_capacity_error_and_argument_errors(G):
         wm.wm_checksum(to_dev(a), 1000, torch.zeros(4, dtype=torch.int32, device="cuda"), g.ws)
 
 
-def test_repeatable_and_grid_independent_bytes(G):
+def test_repeatable_bytes(G):
     """The wire image is canonical: repeated runs give identical bytes."""
     cfg = inputs.CONFIGS["tiny8m"]
     a = inputs.make_cache(cfg).cuda()
