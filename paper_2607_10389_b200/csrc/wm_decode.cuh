@@ -130,7 +130,7 @@ k_decode_check(const unsigned char* __restrict__ wire, uint64_t wire_len, Geo g,
             if (lane == 0) {
                 ws.cflag[c] = (any ? CF_PRESENT : 0u) | (ok ? 0u : CF_BAD3);
                 if (!ok) { atomicMin(&ws.ctrl->bad3_first, c); atomicAdd(&ws.ctrl->bad3_count, 1u); }
-                if (any) atomicAdd(&ws.ctrl->n_present, 1u);
+                if (any) ws.plist[atomicAdd(&ws.ctrl->n_present, 1u)] = c;     // (the present chunks, in any order: k_decode claims their tiles only)
             }
         }
     }
@@ -340,6 +340,26 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
     const unsigned char* const payload = wire + g.meta_end;
     const bool leader = (tt == 0);
     constexpr uint32_t kNone = 0xFFFFFFFFu;
+    // The tile behind a ticket.  Without a mask tickets are tile numbers (one past the last tile:
+    // none left).  An image made with a dirty mask (header flags bit 0) holds the tiles of its
+    // present chunks only; k_decode_check listed those chunks (ws.plist, in any order: nothing here
+    // depends on the order of tiles), and ticket k is tile k mod tiles_per_chunk of the
+    // (k / tiles_per_chunk)-th listed chunk, so a sparse image costs nothing for what it leaves
+    // out.  Only the cache's last chunk can have fewer tiles: a ticket that falls behind its end
+    // has no tile, and the claimer draws the next one at once.
+    const bool masked = ((reinterpret_cast<const uint32_t*>(wire)[1] >> 16) & 1u) != 0u;
+    const uint32_t n_tickets = masked ? ld_volatile_u32(&ws.ctrl->n_present) * g.tiles_per_chunk : 0u;
+    auto claim = [&]() -> uint32_t {
+        uint32_t k = atomicAdd(&ws.ctrl->ticket, 1u);
+        if (!masked) return k;
+        while (k < n_tickets) {
+            const uint32_t j = chunk_of(g, k);
+            const uint32_t t = ws.plist[j] * g.tiles_per_chunk + (k - j * g.tiles_per_chunk);
+            if (t < g.n_tiles) return t;
+            k = atomicAdd(&ws.ctrl->ticket, 1u);
+        }
+        return kNone;
+    };
     const uint32_t stage_s = (uint32_t)__cvta_generic_to_shared(stage);
     const uint32_t sm_s = stage_s + 64u + 1024u * warp + 8u * lane;     // this lane's sign-mantissa bytes, group 4 warp
 
@@ -365,9 +385,9 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
 
     if (leader) {
         mbar_init(&tc->mbar, 1);
-        lookup(atomicAdd(&ws.ctrl->ticket, 1u), &tc->slot[0]);
-        lookup(atomicAdd(&ws.ctrl->ticket, 1u), &tc->slot[1]);
-        tc->slot[2].t = atomicAdd(&ws.ctrl->ticket, 1u);      // its look-ups happen in the first step
+        lookup(claim(), &tc->slot[0]);
+        lookup(claim(), &tc->slot[1]);
+        tc->slot[2].t = claim();      // its look-ups happen in the first step
         start_copy(tc->slot[0]);
     }
     team_bar(team);
@@ -542,7 +562,7 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
         }
         if (tt == 96u) {                   // the ticket of the tile three ahead
             t_look = tc->slot[(it + 2u) & 3u].t;
-            if (t_look < g.n_tiles) l_tk = atomicAdd(&ws.ctrl->ticket, 1u);
+            if (t_look < g.n_tiles) l_tk = claim();
         }
 
         // ---- phase 2: unpack, store, checksum

@@ -7,7 +7,13 @@ namespace wm {
 
 // ------------------------------------------------------------------ wm_encode
 
-__global__ void k_encode_init(Geo g, Ws ws, unsigned char* wire)
+// Clears the control block and the placement words, zero-fills the padding behind the tile
+// table.  With a dirty mask the main kernel claims the tiles of the present chunks only, so
+// here the table entries of all tiles start at 0 (absent) and the first block lists the present
+// chunks in ascending order (ws.plist, ballot + popc scan) and leaves the number of tiles to
+// claim in the control block.
+__global__ void __launch_bounds__(1024)
+k_encode_init(Geo g, Ws ws, unsigned char* wire, const uint8_t* __restrict__ dirty)
 {
     grid_dep_launch();
     const uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -17,6 +23,44 @@ __global__ void k_encode_init(Geo g, Ws ws, unsigned char* wire)
     // zero padding between the tile table and the payload
     const uint64_t tab_end = 64ull + 16ull * g.n_chunks + 2ull * g.n_tiles;
     if (i < g.meta_end - tab_end) wire[tab_end + i] = 0;
+    __syncthreads();                                   // the control block is cleared before anything is written into it
+    if (!dirty) {
+        if (i == 0) ws.ctrl->n_tickets = g.n_tiles;
+        return;
+    }
+    uint16_t* tile_tab = reinterpret_cast<uint16_t*>(wire + 64 + 16ull * g.n_chunks);
+    for (uint64_t t = i; t < g.n_tiles; t += stride) tile_tab[t] = 0;
+    if (blockIdx.x != 0) return;
+    __shared__ uint32_t s_warp[32];
+    __shared__ uint32_t s_carry;
+    const uint32_t lane = threadIdx.x % 32, warp = threadIdx.x / 32;
+    if (threadIdx.x == 0) s_carry = 0;
+    __syncthreads();
+    for (uint32_t base = 0; base < g.n_chunks; base += 1024) {
+        const uint32_t c = base + threadIdx.x;
+        const bool d = c < g.n_chunks && dirty[c] != 0;
+        const uint32_t bal = __ballot_sync(0xFFFFFFFFu, d);
+        if (lane == 0) s_warp[warp] = __popc(bal);
+        __syncthreads();
+        uint32_t before = s_carry;
+        for (uint32_t w2 = 0; w2 < warp; w2++) before += s_warp[w2];
+        if (d) ws.plist[before + __popc(bal & ((1u << lane) - 1u))] = c;
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            uint32_t tot = 0;
+            for (int w2 = 0; w2 < 32; w2++) tot += s_warp[w2];
+            s_carry += tot;
+        }
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) {
+        // every present chunk has tiles_per_chunk tiles, except the cache's last chunk
+        const uint32_t np = s_carry;
+        uint32_t nt = np * g.tiles_per_chunk;
+        if (np && dirty[g.n_chunks - 1]) nt -= g.tiles_per_chunk - (g.n_tiles - (g.n_chunks - 1) * g.tiles_per_chunk);
+        ws.ctrl->n_list = np;
+        ws.ctrl->n_tickets = nt;
+    }
 }
 
 constexpr uint32_t kFlagA = 1u << 30, kFlagP = 2u << 30, kValMask = (1u << 30) - 1u;
@@ -172,7 +216,8 @@ struct EncTeamCtl {
     unsigned long long excl[2];   // offset of the tile packed in the next step, by step parity
     unsigned long long mbar;      // completion of the bulk copy into the team's stage
     unsigned long long pad2;
-    unsigned long long nptr[2];   // leaf mode: descriptor (k_leaf_map) of the tile in next[], by step parity
+    unsigned long long nptr[2];   // leaf mode: address (k_leaf_map) of the tile in next[], by step parity
+    uint32_t kring[8];            // with a mask: the ticket of the tile in each ring slot (placement runs over tickets)
 };
 static_assert(sizeof(EncTeamCtl) % 16 == 0, "team control block keeps 16-byte alignment");
 
@@ -332,14 +377,21 @@ constexpr uint32_t kWarpAllZero = 0x8000u, kWarpConst = 0x4000u, kSumZeroTile = 
 // The tile is stored in ENT form (shorter than its bit planes and than raw); low half: halfwords.
 constexpr uint32_t kSumEnt = 0x10000u;
 
+// The tile behind ticket k.  Without a mask tickets are tile numbers.  With one, only the tiles of
+// present chunks are claimed: ticket k is tile k mod tiles_per_chunk of the (k / tiles_per_chunk)-th
+// present chunk (plist, ascending, written by k_encode_init), so placement runs over tickets and a
+// sparse mask costs nothing for what it leaves out.
 template <bool MASKED>
-__device__ __forceinline__ uint32_t describe_tile(const Geo& g, const uint8_t* __restrict__ dirty, uint32_t t)
+__device__ __forceinline__ uint32_t describe_tile(const Geo& g, const uint32_t* __restrict__ plist, uint32_t n_tickets, uint32_t k)
 {
-    if (t >= g.n_tiles) return kQNone;
-    uint32_t q = t;
-    if (first_in_chunk(g, t)) q |= kQFirst;
-    if (!MASKED || dirty[chunk_of(g, t)] != 0) q |= kQPresent;
-    return q;
+    if (k >= n_tickets) return kQNone;
+    uint32_t t = k;
+    bool first = first_in_chunk(g, k);
+    if (MASKED) {
+        const uint32_t j = chunk_of(g, k);
+        t = plist[j] * g.tiles_per_chunk + (k - j * g.tiles_per_chunk);
+    }
+    return t | kQPresent | (first ? kQFirst : 0u);
 }
 
 template <int TEAMS, bool MASKED, bool LEAVES, bool ZEROS, bool ENT = false>
@@ -367,7 +419,7 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
     if (s_scanner) {
         uint32_t* win = reinterpret_cast<uint32_t*>(S.take(2048));      // 512 entries
         // (test hook: with the scanner left out no offset is ever handed out, and the owners' waits run out)
-        if (threadIdx.x < 32 && win && !(g.inject & kInjectNoScanner)) scan_tile_lengths(ws.lbk, g.n_tiles, threadIdx.x, ws.ctrl, win, g.wait_ns);
+        if (threadIdx.x < 32 && win && !(g.inject & kInjectNoScanner)) scan_tile_lengths(ws.lbk, MASKED ? ld_volatile_u32(&ws.ctrl->n_tickets) : g.n_tiles, threadIdx.x, ws.ctrl, win, g.wait_ns);
         return;
     }
     const uint32_t team = threadIdx.x / kTeamThreads, tt = threadIdx.x % kTeamThreads;
@@ -406,7 +458,10 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
 
     auto is_tile = [](uint32_t q) { return (q & kQTile) != kQNone; };
     auto is_hot = [&](uint32_t q) { return q >= kQPresent && (q & kQTile) < g.n_full_tiles; };   // present and full
-    auto publish_len = [&](uint32_t t, uint32_t len) { st_relaxed_u32(ws.lbk + t, kFlagA | (len / kUnit)); };
+    // (the placement words are indexed by ticket: with a mask that is the ring slot's ticket, else the tile number)
+    const uint32_t n_tickets = MASKED ? ld_volatile_u32(&ws.ctrl->n_tickets) : g.n_tiles;
+    auto place_of = [&](uint32_t slot, uint32_t t) { return MASKED ? tc->kring[slot] : t; };
+    auto publish_len = [&](uint32_t slot, uint32_t t, uint32_t len) { st_relaxed_u32(ws.lbk + place_of(slot, t), kFlagA | (len / kUnit)); };
     // where tile t lives: its address in the flat cache, or (leaf mode) the address that k_leaf_map wrote
     auto tile_src = [&](uint32_t t) -> unsigned long long {
         return LEAVES ? ws.tptr[t] : reinterpret_cast<unsigned long long>(cache + (uint64_t)t * kTile);
@@ -439,12 +494,16 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
     // Leaf mode claims one step further ahead: a tile's address is looked up in the step between
     // its claim and its hand-over, so that the leader never waits for that answer either.
     uint32_t qA = kQNone;              // leader, leaf mode: claimed and described, address on its way
+    uint32_t kA = 0;                   // ... and its ticket
     if (leader) {
         for (int i = 0; i < 8; i++) tc->wsum[i] = 0;
         mbar_init(&tc->mbar, 1);
-        const uint32_t q0 = describe_tile<MASKED>(g, dirty, next_ticket(ws.ctrl));
-        const uint32_t q1 = is_tile(q0) ? describe_tile<MASKED>(g, dirty, next_ticket(ws.ctrl)) : kQNone;
+        const uint32_t k0 = next_ticket(ws.ctrl);
+        const uint32_t q0 = describe_tile<MASKED>(g, ws.plist, n_tickets, k0);
+        const uint32_t k1 = is_tile(q0) ? next_ticket(ws.ctrl) : 0xFFFFFFFFu;
+        const uint32_t q1 = is_tile(q0) ? describe_tile<MASKED>(g, ws.plist, n_tickets, k1) : kQNone;
         claiming = is_tile(q1);
+        if (MASKED) { tc->kring[3] = k0; tc->kring[4] = k1; }      // the slots in which they will be measured
         tc->next[0] = q0;
         tc->next[1] = q1;
         tc->excl[0] = 0ull;
@@ -454,7 +513,7 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
             tc->nptr[1] = is_tile(q1) ? tile_src(q1 & kQTile) : 0ull;
             tc->next[0] = with_mark(q0, tc->nptr[0]);
             tc->next[1] = with_mark(q1, tc->nptr[1]);
-            if (claiming) { qA = describe_tile<MASKED>(g, dirty, next_ticket(ws.ctrl)); claiming = is_tile(qA); }
+            if (claiming) { kA = next_ticket(ws.ctrl); qA = describe_tile<MASKED>(g, ws.plist, n_tickets, kA); claiming = is_tile(qA); }
         }
     }
     team_bar(team);
@@ -492,7 +551,7 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
         uint32_t pv = 0, tk = 0xFFFFFFFFu;
         unsigned long long pA = 0;
         if (tt == 64u) start_copy(qN, LEAVES ? tc->nptr[par ^ 1u] : tile_src(qN & kQTile));
-        if (tt == 96u && is_tile(qV)) pv = ld_relaxed_u32(ws.lbk + (qV & kQTile));
+        if (tt == 96u && is_tile(qV)) pv = ld_relaxed_u32(ws.lbk + place_of((sl + 1u) & 7u, qV & kQTile));
         if (leader) {
             if (claiming) tk = next_ticket(ws.ctrl);
             if (LEAVES && is_tile(qA)) pA = tile_src(qA & kQTile);
@@ -581,14 +640,14 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
                 if (lane == 0) {
                     tc->ssum[slY] = zero_tile ? kSumZeroTile : const_tile ? kSumConstTile : ent_tile ? kSumEnt | halfwords : total;
                     tc->wsum[slY] = 0;
-                    publish_len(tYn, zero_tile ? 0u : const_tile ? 32u : ent_tile ? ent_tile_bytes(halfwords) : plane_len);
+                    publish_len(slY, tYn, zero_tile ? 0u : const_tile ? 32u : ent_tile ? ent_tile_bytes(halfwords) : plane_len);
                 }
             }
             tmem_store16(tmem_warp + 16u * (step & 3u), d);
         } else if (is_tile(qY)) {
             // rare: a tile of an absent chunk (length 0) or the ragged last tile (stored raw)
             const bool present = qY >= kQPresent;
-            if (tt == 0) publish_len(tYn, present ? tile_left(g, tYn) : 0u);
+            if (tt == 0) publish_len(slY, tYn, present ? tile_left(g, tYn) : 0u);
             if (present) {
                 // (leaf mode: the ragged tile has a slot of its own in the side buffer)
                 load_tile_words_guarded(reinterpret_cast<const unsigned char*>(tile_src(tYn)), tile_left(g, tYn), (qY & kQFirst) != 0, warp, lane, d);
@@ -737,23 +796,27 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
             }
             tile_tab[tXn] = (uint16_t)entry;
             if (qX & kQFirst) *reinterpret_cast<unsigned long long*>(dir + 16ull * chunk_of(g, tXn)) = exclX;
-            if (tXn + 1 == g.n_tiles) ws.ctrl->payload_total = exclX + enc_len;
+            if (place_of(sl, tXn) + 1 == n_tickets) ws.ctrl->payload_total = exclX + enc_len;
         }
         if (leader) {
             uint32_t qn2 = kQNone;
-            if (claiming) { qn2 = describe_tile<MASKED>(g, dirty, tk); claiming = is_tile(qn2); }
-            if (LEAVES) {              // hand over the tile whose descriptor arrived during this step
+            if (claiming) { qn2 = describe_tile<MASKED>(g, ws.plist, n_tickets, tk); claiming = is_tile(qn2); }
+            // (the tile handed over now is measured two steps on, in ring slot sl + 5)
+            if (LEAVES) {              // hand over the tile whose address arrived during this step
                 tc->next[par] = with_mark(qA, pA);
                 tc->nptr[par] = pA;
+                if (MASKED) tc->kring[(sl + 5u) & 7u] = kA;
                 qA = qn2;
+                kA = tk;
             } else {
                 tc->next[par] = qn2;
+                if (MASKED) tc->kring[(sl + 5u) & 7u] = tk;
             }
         }
         if (tt == 96u) {
             unsigned long long e = 0;
             if (is_tile(qV))
-                e = (pv >> 30) == 2u ? (unsigned long long)(pv & kValMask) * kUnit : wait_prefix(ws.lbk, qV & kQTile, ws.ctrl, g.wait_ns);
+                e = (pv >> 30) == 2u ? (unsigned long long)(pv & kValMask) * kUnit : wait_prefix(ws.lbk, place_of((sl + 1u) & 7u, qV & kQTile), ws.ctrl, g.wait_ns);
             tc->excl[par] = e;
         }
         qX = qV; qV = qW; qW = qY; qY = qN;
@@ -801,9 +864,22 @@ k_encode_finish(const unsigned char* __restrict__ cache, Geo g, const uint8_t* _
         } else {
             crc = crc_inout[c];
         }
-        const unsigned long long po = *reinterpret_cast<const unsigned long long*>(dir + 16ull * c);
-        const unsigned long long nx = (c + 1 < g.n_chunks)
-                                          ? *reinterpret_cast<const unsigned long long*>(dir + 16ull * (c + 1)) : total;
+        // Where the chunk's payload starts: a present chunk's offset was written by the team that
+        // placed its first tile; an absent chunk (the main kernel never saw it) starts where the next
+        // present chunk does, or at the end of the payload.
+        const uint32_t n_list = dirty ? ld_volatile_u32(&ws.ctrl->n_list) : 0u;
+        auto starts_at = [&](uint32_t cc) -> unsigned long long {
+            if (cc >= g.n_chunks) return total;
+            if (!dirty || dirty[cc]) return *reinterpret_cast<const unsigned long long*>(dir + 16ull * cc);
+            uint32_t lo = 0, hi = n_list;              // the first listed chunk above cc
+            while (lo < hi) {
+                const uint32_t mid = (lo + hi) / 2;
+                if (ws.plist[mid] < cc) lo = mid + 1; else hi = mid;
+            }
+            return lo < n_list ? *reinterpret_cast<const unsigned long long*>(dir + 16ull * ws.plist[lo]) : total;
+        };
+        const unsigned long long po = starts_at(c), nx = starts_at(c + 1);
+        if (!present) *reinterpret_cast<unsigned long long*>(dir + 16ull * c) = po;
         *reinterpret_cast<uint32_t*>(dir + 16ull * c + 8) = (uint32_t)(nx - po);
         *reinterpret_cast<uint32_t*>(dir + 16ull * c + 12) = crc;
         term = cache_crc_term(g, cp, crc, c);

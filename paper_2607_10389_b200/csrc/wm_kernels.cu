@@ -408,7 +408,7 @@ static wm_status encode_any(const void* cache, const wm_leaf* leaves, uint32_t n
     const unsigned char* c = static_cast<const unsigned char*>(cache);
     unsigned char* w = static_cast<unsigned char*>(wire);
     const uint32_t init_blocks = (g.n_tiles + 1023) / 1024 < 1024 ? (g.n_tiles + 1023) / 1024 : 1024;
-    k_encode_init<<<init_blocks ? init_blocks : 1, 1024, 0, s>>>(g, ws, w);
+    k_encode_init<<<init_blocks ? init_blocks : 1, 1024, 0, s>>>(g, ws, w, dirty);
     if (leaves) {
         const uint32_t map_blocks = (g.n_tiles + 4095) / 4096 < 64 ? (g.n_tiles + 4095) / 4096 : 64;
         launch_after(k_leaf_map, map_blocks ? map_blocks : 1, 1024, 0, s, leaves, n_leaves, g, ws, result, 0);

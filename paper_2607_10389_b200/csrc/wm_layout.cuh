@@ -61,7 +61,9 @@ struct Ctrl {                 // first 256 bytes of the workspace
     uint32_t cache_acc;       // XOR of the chunks' terms of the whole-cache CRC
     uint32_t has_pack;        // decode of an image with the entropy option: it holds PACK tiles too
     uint32_t n_walked;        // leaf mode: tiles that go through the side buffer (see k_leaf_map)
-    uint32_t pad[39];
+    uint32_t n_list;          // masked images: present chunks listed in plist
+    uint32_t n_tickets;       // tiles the main kernel has to claim (masked: those of the listed chunks only)
+    uint32_t pad[37];
 };
 static_assert(sizeof(Ctrl) == 256, "control block is 256 bytes");
 
@@ -124,6 +126,7 @@ struct Ws {
     uint32_t* mdig;              // [n_meta_slices]
     unsigned long long* tptr;    // [n_tiles] leaf mode: the address of each tile of the logical cache (see k_leaf_map)
     unsigned long long* lstart;  // [kMaxLeaves + 1] leaf mode: logical offset at which each leaf starts
+    uint32_t* plist;             // [n_chunks] masked images: the present chunks (encode: ascending; decode: any order)
     uint32_t* wlist;             // [kMaxWalked] leaf mode: the tiles that go through the side buffer
     unsigned char* side;         // [min(n_tiles, kMaxWalked)][16384] leaf mode: their slots
 };
@@ -135,7 +138,7 @@ constexpr uint32_t CF_PRESENT = 1, CF_BAD3 = 2, CF_BAD4 = 4, CF_BAD5 = 8, CF_BAD
 static inline uint64_t align16(uint64_t v) { return (v + 15) & ~(uint64_t)15; }
 
 struct WsLayout {
-    uint64_t state, dig, rel, cflag, ccrc, mdig, tptr, lstart, wlist, side, total;
+    uint64_t state, dig, rel, cflag, ccrc, mdig, tptr, lstart, plist, wlist, side, total;
 };
 
 static WsLayout ws_layout(const Geo& g)
@@ -150,6 +153,7 @@ static WsLayout ws_layout(const Geo& g)
     L.mdig = o;  o = align16(o + 4ull * g.n_meta_slices);
     L.tptr = o;  o = align16(o + 8ull * g.n_tiles);
     L.lstart = o; o = align16(o + 8ull * (kMaxLeaves + 1));
+    L.plist = o; o = align16(o + 4ull * g.n_chunks);
     L.wlist = o; o = align16(o + 4ull * kMaxWalked);
     L.side = o; o = align16(o + (uint64_t)kTile * (g.n_tiles < kMaxWalked ? g.n_tiles : kMaxWalked));
     L.total = o;
@@ -170,6 +174,7 @@ static Ws ws_carve(void* base, const Geo& g)
     w.mdig = reinterpret_cast<uint32_t*>(b + L.mdig);
     w.tptr = reinterpret_cast<unsigned long long*>(b + L.tptr);
     w.lstart = reinterpret_cast<unsigned long long*>(b + L.lstart);
+    w.plist = reinterpret_cast<uint32_t*>(b + L.plist);
     w.wlist = reinterpret_cast<uint32_t*>(b + L.wlist);
     w.side = b + L.side;
     return w;
