@@ -226,11 +226,11 @@ wm_status wm_encode(const void* cache, uint64_t nbytes, uint32_t chunk_bytes, co
  *   3 directory and tile table are consistent                      WM_ERR_STRUCT
  *   4 coded tiles in tile order; the status is that of the lowest failing tile.  PACK tile:
  *     descriptors valid (WM_ERR_DESC), then 258 + sum w equals the tile entry (WM_ERR_STRUCT).
- *     ENT tile (images with flags bit2): the eight stream counts within 128..1024 and adding up
- *     to the entry (WM_ERR_STRUCT), then every stream used up exactly by its 1024 codewords, the
- *     fill bits of every strand zero, every anchor the rounded mean of the exponents its share
- *     decodes to, the header's 40 spare bytes and the fill behind the last stream zero
- *     (WM_ERR_DESC).  CONST tile (images with flags bit1): the 30 bytes behind the value zero
+ *     ENT tile (images with flags bit2): the eight word counts within 64..319 and adding up
+ *     to the entry (WM_ERR_STRUCT), then every share's strand lengths adding up to its word
+ *     count, every strand's 32 codewords taking exactly its length, the fill bits of every
+ *     stream's last word zero, every anchor the rounded mean of the exponents its share decodes
+ *     to, the header's 40 spare bytes and the fill behind the last stream zero (WM_ERR_DESC).  CONST tile (images with flags bit1): the 30 bytes behind the value zero
  *     (WM_ERR_DESC).  No byte of a coded tile is left unaccounted for
  *   5 CRC32C of every decoded chunk equals its directory CRC       WM_ERR_CHUNK_CRC
  *   6 absent chunk: dst_crc_inout[c] equals its directory CRC      WM_ERR_STALE
@@ -299,16 +299,21 @@ void wm_zero_tiles_enable(int on);
  *   anchor_s = (sum of the share's 1024 exponents + 512) >> 10.  u = E - anchor_s is coded
  *       u:    0   +1   -1   -2    +2    -3    -4     -5      +3       -6        other
  *       bits: 00  10   01   1100  1110  1101  11110  111110  1111110  11111110  11111111 + E (8 bits, low first)
- *   (in writing order; a strand is an LSB-first bit string, zero-filled to whole 16-bit halfwords).
- *   A share's strands are interleaved into one stream in the order a reader needs them: at step
- *   i = 0..31 every strand whose codeword i is not complete in the halfwords it has taken so far
- *   takes the stream's next halfword, strands in ascending order.
- *   Layout: anchor[8] u8 | count[8] u16 (halfwords per stream) | 40 zero bytes | SM[8192] as in
- *   a PACK tile | the eight streams | zero fill to a multiple of 32 bytes.
- * Decode checks (step 4): counts within 128..1024 and adding up to the entry (else WM_ERR_STRUCT);
- * every stream used up exactly, the fill bits of every strand, the 40 spare header bytes and the
- * fill behind the last stream zero, every anchor equal to the formula above applied to what its
- * share decodes to (else WM_ERR_DESC).
+ *   (in writing order).  A strand's bit string is its 32 codewords one after the other (64 to 512
+ *   bits).  A share's stream is its 32 strands' strings one after the other, strand 0 first,
+ *   without gaps, written LSB-first into 32-bit little-endian words and zero-filled to a whole
+ *   word.  Every strand's length minus 64 is stored in a byte, so that a reader can start on
+ *   all 32 strands of a share at once (lane l of a warp decodes strand l from the bit where the
+ *   lengths before it add up to); a tile with a strand longer than 319 bits is not stored in
+ *   this form.
+ *   Layout: anchor[8] u8 | words[8] u16 (32-bit words per stream) | 40 zero bytes | SM[8192] as in
+ *   a PACK tile | bits[8][32] u8 (strand lengths - 64) | the eight streams | zero fill to a
+ *   multiple of 32 bytes.
+ * Decode checks (step 4): word counts within 64..319 and adding up to the entry (else
+ * WM_ERR_STRUCT); a share's strand lengths adding up to its word count, every strand's 32
+ * codewords taking exactly its length, the fill bits of every stream's last word, the 40 spare
+ * header bytes and the fill behind the last stream zero, every anchor equal to the formula above
+ * applied to what its share decodes to (else WM_ERR_DESC).
  */
 void wm_entropy_enable(int on);
 

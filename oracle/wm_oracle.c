@@ -325,19 +325,23 @@ static int plane_widths(uint32_t w, uint32_t p[3])
  *      any other u: 11111111 followed by the eight bits of E itself, low bit first (16 bits)
  *   (as numbers, first bit = bit 0: 0, 1, 2, 3, 7, 11, 15, 31, 63, 127, 255 | E << 8).
  *
- * The 32 strands of a share are cut into 16-bit halfwords (the last one zero-filled) and
- * interleaved into one stream in the order a reader needs them: the reader walks i = 0..31;
- * at step i every strand whose codeword i is not complete in the halfwords it has taken so
- * far takes the next halfword of the stream, strands in ascending order; then every strand
- * consumes its codeword i.  (A codeword is at most 16 bits, so one halfword always suffices.)
+ * A strand's bit string is its 32 codewords one after the other (64 to 512 bits).  A share's
+ * stream is its 32 strands' strings one after the other, strand 0 first, with no gaps, written
+ * LSB-first into 32-bit little-endian words and zero-filled to a whole word.  The length of
+ * every strand, minus 64, is stored in one byte, so that a reader can start on all strands at
+ * once; a tile with a strand longer than 319 bits is not stored in this form.
  *
- *   ENT tile:  anchor[8] u8 | count[8] u16 (halfwords in each share's stream) | 40 zero bytes
- *              SM[8192] as in a PACK tile | the eight streams | zero fill to a multiple of 32
+ *   ENT tile:  anchor[8] u8 | words[8] u16 (32-bit words in each share's stream) | 40 zero bytes
+ *              SM[8192] as in a PACK tile | bits[8][32] u8 (strand lengths - 64) |
+ *              the eight streams | zero fill to a multiple of 32
  *   entry = 0x8000 | length / 32 (the length is below 16384 whenever the form is used).
  */
 static const int      ent_sym[10]  = {0, 1, -1, -2, 2, -3, -4, -5, 3, -6};
 static const uint32_t ent_len[10]  = {2, 2, 2, 4, 4, 4, 5, 6, 7, 8};
 static const uint32_t ent_bits[10] = {0, 1, 2, 3, 7, 11, 15, 31, 63, 127};
+
+#define WMO_ENT_FIXED (64u + 8192u + 256u)      /* header, sign-mantissa plane, strand lengths */
+#define WMO_ENT_MAX_STRAND 319u
 
 static uint32_t ent_elem(uint32_t share, uint32_t strand, uint32_t i)
 {
@@ -353,8 +357,19 @@ static void ent_codeword(uint32_t E, uint32_t anchor, uint32_t* bits, uint32_t* 
     *len = 16u;
 }
 
-/* Length and symbol of the codeword at the low end of `buf` (bits beyond the valid ones are
- * zero).  Returns the length; *E receives the exponent. */
+/* `n` bits (n <= 32) from bit `at` on of the LSB-first bit string `p` of `nbits` bits; bits
+ * beyond the end read as zero. */
+static uint32_t get_bits(const uint8_t* p, uint64_t nbits, uint64_t at, uint32_t n)
+{
+    uint64_t v = 0, first = at / 8u, nbytes = nbits / 8u;       /* (nbits is a whole number of bytes) */
+    for (uint32_t k = 0; k < 5; k++)
+        if (first + k < nbytes) v |= (uint64_t)p[first + k] << (8u * k);
+    v >>= at % 8u;
+    return (uint32_t)(n >= 32u ? v : v & ((1ull << n) - 1ull));
+}
+
+/* Length and symbol of the codeword at the low end of `buf` (16 bits suffice).  Returns the
+ * length; *E receives the exponent. */
 static uint32_t ent_parse(uint32_t buf, uint32_t anchor, uint32_t* E)
 {
     for (int k = 0; k < 10; k++)
@@ -367,99 +382,83 @@ static uint32_t ent_parse(uint32_t buf, uint32_t anchor, uint32_t* E)
 }
 
 /* Encode the exponents of one tile as ENT streams.  Returns the tile's length in bytes (a
- * multiple of 32; it may exceed the tile size, in which case the caller stores the tile raw
- * and `out` is not used).  `out` must hold 64 + 8192 + 8 * 32 * 64 + 32 bytes. */
+ * multiple of 32), or WMO_TILE when the form cannot hold the tile (a strand of more than 319 bits)
+ * or is not shorter than the tile itself; `out` is then not to be used.  `out` must hold
+ * 2 * WMO_TILE bytes. */
 static uint32_t encode_ent_tile(const uint8_t* src, uint8_t* out)
 {
-    uint32_t hw_total = 0;
-    memset(out, 0, 64);
-    uint8_t* stream = out + 64 + 8192;
+    memset(out, 0, 2 * WMO_TILE);
+    uint8_t* stream = out + WMO_ENT_FIXED;
+    uint32_t words_total = 0;
     for (uint32_t s = 0; s < 8; s++) {
         uint32_t sum = 0;
         for (uint32_t e = 0; e < 1024; e++) sum += (get16(src + 2u * (1024u * s + e)) >> 7) & 0xFFu;
         uint32_t anchor = (sum + 512u) >> 10;
         out[s] = (uint8_t)anchor;
-        /* every strand as a bit string, and the bits used up to and including codeword i */
-        uint8_t bit[32][32 * 16 + 16];
-        uint32_t upto[32][32];
-        memset(bit, 0, sizeof bit);
+        uint64_t at = 0;                         /* bits of the share's stream written so far */
+        uint8_t* sp = stream + 4u * words_total;
         for (uint32_t l = 0; l < 32; l++) {
-            uint32_t n = 0;
+            uint64_t start = at;
             for (uint32_t i = 0; i < 32; i++) {
                 uint32_t E = (get16(src + 2u * ent_elem(s, l, i)) >> 7) & 0xFFu, cw, len;
                 ent_codeword(E, anchor, &cw, &len);
-                for (uint32_t b = 0; b < len; b++) bit[l][n + b] = (uint8_t)((cw >> b) & 1u);
-                n += len;
-                upto[l][i] = n;
+                for (uint32_t b = 0; b < len; b++, at++)
+                    if ((cw >> b) & 1u) sp[at / 8u] |= (uint8_t)(1u << (at % 8u));
             }
+            if (at - start > WMO_ENT_MAX_STRAND) return WMO_TILE;
+            out[64u + 8192u + 32u * s + l] = (uint8_t)(at - start - 64u);
         }
-        uint32_t taken[32] = {0}, count = 0;
-        for (uint32_t i = 0; i < 32; i++)
-            for (uint32_t l = 0; l < 32; l++)
-                if (upto[l][i] > 16u * taken[l]) {
-                    uint32_t hw = 0;
-                    for (uint32_t b = 0; b < 16; b++) hw |= (uint32_t)bit[l][16u * taken[l] + b] << b;
-                    put16(stream + 2u * (hw_total + count), hw);
-                    taken[l]++;
-                    count++;
-                }
-        put16(out + 8 + 2u * s, count);
-        hw_total += count;
+        uint32_t words = (uint32_t)((at + 31u) / 32u);
+        put16(out + 8 + 2u * s, words);
+        words_total += words;
+        if (WMO_ENT_FIXED + 4u * words_total >= WMO_TILE) return WMO_TILE;
     }
-    uint32_t len = 8256u + 2u * hw_total;
-    while (len % 32u) out[len++] = 0;
+    uint32_t len = (WMO_ENT_FIXED + 4u * words_total + 31u) & ~31u;
     /* sign-mantissa plane: the PACK tile's */
     for (uint32_t g = 0; g < WMO_GROUPS_PER_TILE; g++)
         for (uint32_t e = 0; e < WMO_GROUP_ELEMS; e++) {
             uint32_t v = get16(src + 2u * (g * WMO_GROUP_ELEMS + e));
             out[64u + 256u * g + coded_pos(e)] = (uint8_t)(((v & 0x7Fu) << 1) | (v >> 15));
         }
-    return len;
+    return len < WMO_TILE ? len : WMO_TILE;
 }
 
-/* Header of an ENT tile against its table entry: every share's count within what 32 strands
- * of 32 codewords can need, and the length they add up to.  Returns 0 when it fits. */
+/* Header of an ENT tile against its table entry: every share's word count within what 32
+ * strands of 64 to 319 bits can need, and the length they add up to.  Returns 0 when it fits. */
 static int ent_header_bad(const uint8_t* in, uint32_t entry)
 {
     uint32_t total = 0;
     for (uint32_t s = 0; s < 8; s++) {
         uint32_t c = get16(in + 8 + 2u * s);
-        if (c < 128u || c > 1024u) return 1;
+        if (c < 64u || c > 319u) return 1;
         total += c;
     }
-    return ((8256u + 2u * total + 31u) / 32u) != (entry & 0x7FFFu);
+    return ((WMO_ENT_FIXED + 4u * total + 31u) / 32u) != (entry & 0x7FFFu);
 }
 
 /* Read the eight streams of an ENT tile whose header fits (`entry`: its tile-table entry).  With
  * dst != NULL the tile is written there.  Returns 0 when every byte of the tile is accounted for:
- * every stream used up exactly, the bits left over in every strand's last halfword zero, every
- * anchor the rounded mean of the exponents its share decodes to (what the encoder writes), the 40
- * spare header bytes and the fill behind the last stream zero; 1 otherwise.  With these no bit of
+ * the strand lengths of every share add up to its word count, every strand's 32 codewords take
+ * exactly its length, the fill bits of every stream's last word are zero, every anchor is the
+ * rounded mean of the exponents its share decodes to (what the encoder writes), the 40 spare
+ * header bytes and the fill behind the last stream are zero; 1 otherwise.  With these no bit of
  * an ENT tile can change without the tile being refused or the decoded bytes changing. */
 static int decode_ent_tile(const uint8_t* in, uint8_t* dst, uint32_t entry)
 {
-    const uint8_t* stream = in + 64 + 8192;
+    const uint8_t* stream = in + WMO_ENT_FIXED;
     int bad = 0;
-    uint32_t hw_total = 0;
+    uint32_t words_total = 0;
     for (uint32_t i = 24; i < 64; i++)
         if (in[i]) bad = 1;
     for (uint32_t s = 0; s < 8; s++) {
-        uint32_t anchor = in[s], count = get16(in + 8 + 2u * s), pos = 0, esum = 0;
-        hw_total += count;
-        uint32_t buf[32] = {0}, avail[32] = {0};
-        for (uint32_t i = 0; i < 32; i++)
-            for (uint32_t l = 0; l < 32; l++) {
-                uint32_t E;
-                if (ent_parse(buf[l], anchor, &E) > avail[l]) {
-                    uint32_t hw = 0;
-                    if (pos < count) hw = get16(stream + 2u * pos); else bad = 1;
-                    pos++;
-                    buf[l] |= hw << avail[l];
-                    avail[l] += 16u;
-                }
-                uint32_t len = ent_parse(buf[l], anchor, &E);
-                buf[l] >>= len;
-                avail[l] -= len;
+        uint32_t anchor = in[s], words = get16(in + 8 + 2u * s), esum = 0;
+        uint64_t nbits = 32ull * words, at = 0;
+        for (uint32_t l = 0; l < 32; l++) {
+            uint64_t want = 64u + in[64u + 8192u + 32u * s + l], start = at;
+            uint64_t p = at;
+            for (uint32_t i = 0; i < 32; i++) {
+                uint32_t E, len = ent_parse(get_bits(stream, nbits, p, 16), anchor, &E);
+                p += len;
                 esum += E;
                 if (dst) {
                     uint32_t e = ent_elem(s, l, i);
@@ -467,13 +466,17 @@ static int decode_ent_tile(const uint8_t* in, uint8_t* dst, uint32_t entry)
                     put16(dst + 2u * e, ((SM & 1u) << 15) | (E << 7) | (SM >> 1));
                 }
             }
-        if (pos != count) bad = 1;
-        for (uint32_t l = 0; l < 32; l++)
-            if (buf[l]) bad = 1;                 /* the fill bits of a strand's last halfword are zero */
+            if (p - start != want) bad = 1;      /* the codewords take exactly the length that is written down */
+            at = start + want;                   /* the next strand starts where the lengths say */
+        }
+        if ((at + 31u) / 32u != words) bad = 1;
+        for (uint64_t b = at; b < nbits; b++)    /* the fill bits of the stream's last word are zero */
+            if (get_bits(stream, nbits, b, 1)) bad = 1;
         if (((esum + 512u) >> 10) != anchor) bad = 1;
-        stream += 2u * count;
+        stream += 4u * words;
+        words_total += words;
     }
-    for (uint32_t i = 8256u + 2u * hw_total; i < 32u * (entry & 0x7FFFu); i++)
+    for (uint32_t i = WMO_ENT_FIXED + 4u * words_total; i < 32u * (entry & 0x7FFFu); i++)
         if (in[i]) bad = 1;
     return bad;
 }

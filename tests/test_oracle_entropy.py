@@ -41,12 +41,13 @@ def test_prefix_code_is_complete_and_prefix_free():
 
 def test_constant_tile_by_hand():
     """All elements 1.0 (0x3F80): every anchor is 127, every codeword is '00', a strand is 64 zero
-    bits = 4 halfwords, a share's stream 128 zero halfwords."""
+    bits (length byte 0), a share's stream 32 * 64 bits = 64 zero words; the tile is 64 + 8192 + 256
+    + 8 * 256 = 10560 bytes = 32 * 330."""
     wire, flags, entry, t = _encode_one_tile(_tile_of(0x3F80))
-    assert flags == 4 and entry == (0x8000 | 322) and t.size == 322 * 32 == 8256 + 8 * 128 * 2
-    want = np.zeros(322 * 32, dtype=np.uint8)
+    assert flags == 4 and entry == (0x8000 | 330) and t.size == 330 * 32
+    want = np.zeros(330 * 32, dtype=np.uint8)
     want[0:8] = 127
-    want[8:24] = np.full(8, 128, dtype="<u2").view(np.uint8)
+    want[8:24] = np.full(8, 64, dtype="<u2").view(np.uint8)
     assert np.array_equal(t, want)
     out, _, r = oracle.decode_verify(wire, TILE, TILE)
     assert r.status == 0 and np.array_equal(out.view("<u2"), _tile_of(0x3F80))
@@ -54,41 +55,74 @@ def test_constant_tile_by_hand():
 
 def test_one_different_element_lands_where_the_format_says():
     """Share 3, strand 5, element 7 of the strand is 2.0: u = +1, written '10' at bits 14-15 of the
-    strand's first halfword; with 2-bit codewords everywhere strand l takes its k-th halfword at
-    step 8 k, so that halfword is number 32 k + l of the share's stream."""
+    strand.  Every strand is 64 bits, so strand 5 starts at bit 320 of its share's stream: the set
+    bit is bit 334 = word 10, bit 14; share 3's stream starts at word 3 * 64."""
     v = _tile_of(0x3F80)
     elem = 64 * (16 * 3 + 7 // 2) + 2 * 5 + 7 % 2
     v[elem] = 0x4000
     wire, flags, entry, t = _encode_one_tile(v)
-    assert entry == (0x8000 | 322)
-    streams = t[8256:].view("<u2")
-    want = np.zeros(1024, dtype="<u2")
-    want[3 * 128 + 0 * 32 + 5] = 1 << 14
-    assert np.array_equal(streams[:1024], want)
-    sm = t[64:8256]
-    assert not sm.any()                                     # sign and mantissa bits are all zero
+    assert entry == (0x8000 | 330)
+    assert not t[8256:8512].any()                           # every strand is 64 bits long
+    streams = t[8512:].view("<u4")
+    want = np.zeros(512, dtype="<u4")
+    want[3 * 64 + 10] = 1 << 14
+    assert np.array_equal(streams[:512], want)
+    assert not t[64:8256].any()                             # sign and mantissa bits are all zero
     out, _, r = oracle.decode_verify(wire, TILE, TILE)
     assert r.status == 0 and np.array_equal(out.view("<u2"), v)
 
 
-def test_a_strand_of_escapes_is_interleaved_as_the_reader_needs_it():
-    """Share 0, strand 0 holds 2^20 (E = 147), everything else 1.0 (E = 127): the share's mean is
-    127.6, anchor 128.  Strand 0 is 32 escapes of 16 bits (0xFF, then E), one halfword per step;
-    the other strands code u = -1 as '01', one halfword per 8 steps."""
+def _escapes_example():
+    """Share 0: the first ten elements of strand 0 are 2^20 (E = 147), strand 1 is 0.5 throughout
+    (E = 126), everything else 1.0 (E = 127)."""
+    v = _tile_of(0x3F80)
+    for i in range(10):
+        v[64 * (i // 2) + i % 2] = 147 << 7
+    for i in range(32):
+        v[64 * (i // 2) + 2 + i % 2] = 126 << 7
+    return v
+
+
+def test_strands_follow_one_another_bit_by_bit():
+    """The share's exponents add up to 982 * 127 + 10 * 147 + 32 * 126 = 130216, anchor (130216 + 512)
+    >> 10 = 127.  Strand 0 is ten escapes (11111111 then E = 147, low bit first: halfword 0x93FF)
+    and 22 codewords '00': 204 bits, length byte 140.  Strand 1 starts at bit 204 (word 6, bit 12)
+    and codes u = -1 as '01' 32 times: 64 bits of 1010...10 from the high end, byte 0xAA.  The
+    share has 204 + 31 * 64 = 2188 bits = 69 words; the tile 8512 + 4 * (69 + 7 * 64) = 10580 bytes,
+    rounded up to 10592 = 32 * 331."""
+    v = _escapes_example()
+    wire, flags, entry, t = _encode_one_tile(v)
+    assert list(t[0:8]) == [127] * 8
+    assert list(t[8:24].view("<u2")) == [69] + [64] * 7
+    assert entry == (0x8000 | 331)
+    lens = t[8256:8512]
+    assert lens[0] == 140 and not lens[1:].any()
+    s = t[8512:].view("<u4")
+    want = np.zeros(s.size, dtype="<u4")
+    want[0:5] = 0x93FF93FF
+    want[6], want[7], want[8] = 0xAAAAA000, 0xAAAAAAAA, 0x00000AAA
+    assert np.array_equal(s, want)
+    out, _, r = oracle.decode_verify(wire, TILE, TILE)
+    assert r.status == 0 and np.array_equal(out.view("<u2"), v)
+
+
+def test_a_strand_too_long_for_its_length_byte_keeps_the_tile_out_of_the_form():
+    """A strand of 32 escapes would be 512 bits; the length byte ends at 319.  Such a tile is stored
+    in one of the other forms (here raw under ent_only, PACK otherwise), and 319 bits still fit."""
     v = _tile_of(0x3F80)
     for i in range(32):
         v[64 * (i // 2) + i % 2] = 147 << 7
     wire, flags, entry, t = _encode_one_tile(v)
-    assert t[0] == 128 and list(t[1:8]) == [127] * 7
-    counts = t[8:24].view("<u2")
-    assert list(counts) == [32 + 31 * 4] + [128] * 7
-    s = t[8256:].view("<u2")
-    esc, m1 = 0xFF | (147 << 8), 0xAAAA                     # '01' eight times, LSB first
-    assert s[0] == esc and np.all(s[1:32] == m1)            # step 0: every strand, in order
-    assert np.all(s[32:39] == esc)                          # steps 1..7: strand 0 alone
-    assert s[39] == esc and np.all(s[40:71] == m1)          # step 8: strand 0, then the others' second halfword
-    assert np.all(s[71:78] == esc)                          # steps 9..15
-    assert np.all(s[156:156 + 128 * 7] == 0)                # shares 1..7: all '00'
+    assert entry == 512
+    w2, _, _ = oracle.encode(v.view(np.uint8), TILE, entropy=True)
+    assert 258 <= struct.unpack_from("<H", w2, 64 + 16)[0] < 512
+    # 18 escapes, one 5-bit codeword (u = -4) and 13 codewords of 2 bits: 288 + 5 + 26 = 319 bits
+    v = _tile_of(0x3F80)
+    for i in range(18):
+        v[64 * (i // 2) + i % 2] = 147 << 7
+    v[64 * 9] = 123 << 7
+    wire, flags, entry, t = _encode_one_tile(v)
+    assert entry & 0x8000 and t[8256] == 255
     out, _, r = oracle.decode_verify(wire, TILE, TILE)
     assert r.status == 0 and np.array_equal(out.view("<u2"), v)
 
@@ -116,8 +150,10 @@ def test_sizes_follow_the_code_lengths_and_respect_shannon():
     L = np.full(u.shape, 16)
     for k, w in CODE.items():
         L[u == k] = len(w)
-    halfwords = -(-L.sum(axis=3) // 16)
-    want_len = (8256 + 2 * halfwords.sum(axis=(1, 2)) + 31) // 32 * 32
+    strand_bits = L.sum(axis=3)                                           # [tile, share, strand]
+    words = -(-strand_bits.sum(axis=2) // 32)
+    want_len = (8512 + 4 * words.sum(axis=1) + 31) // 32 * 32
+    want_len = np.where(strand_bits.max(axis=(1, 2)) > 319, TILE, want_len)  # a strand the length byte cannot hold
     # the bit-plane form of the same tiles: 32 groups of 256 elements in memory order
     G = ((v >> 7) & 0xFF).astype(np.int64).reshape(n_tiles, 32, 256)
     rng_ = G.max(axis=2) - G.min(axis=2)
@@ -239,9 +275,9 @@ def test_default_images_are_unchanged_by_the_option():
 
 def test_every_codeword_bit_by_bit():
     """Share 0, strand 0 starts with one element for each coded u (in the table's order), all else
-    is E = 127.  The strand's bit string is the codewords as the format lists them; where its six
-    halfwords sit in the stream follows from when it runs out of bits (steps 0, 5, 8, 12, 20, 28)
-    against the other strands' steps 0, 8, 16, 24."""
+    is E = 127.  The strand's bit string is the codewords as the format lists them, 44 bits, then 22
+    times '00': 88 bits, length byte 24; it is the head of the share's stream, the other strands
+    (64 zero bits each) follow: 88 + 31 * 64 = 2072 bits = 65 words."""
     us = [0, 1, -1, -2, 2, -3, -4, -5, 3, -6]
     v = _tile_of(0x3F80)
     for i, u in enumerate(us):
@@ -251,13 +287,10 @@ def test_every_codeword_bit_by_bit():
     bits = "".join(CODE[u] for u in us) + "00" * 22
     assert len(bits) == 88
     bits += "0" * 8
-    hw = [sum(int(bits[16 * k + b]) << b for b in range(16)) for k in range(6)]
-    s = t[8256:].view("<u2")
-    assert struct.unpack_from("<H", t, 8)[0] == 6 + 31 * 4
-    where = [0, 32, 33, 65, 97, 129]
-    assert [int(s[i]) for i in where] == hw
-    others = np.delete(s[:130], where)
-    assert not others.any()
+    words = [sum(int(bits[32 * k + b]) << b for b in range(32)) for k in range(3)]
+    s = t[8512:].view("<u4")
+    assert struct.unpack_from("<H", t, 8)[0] == 65 and t[8256] == 24 and not t[8257:8512].any()
+    assert [int(x) for x in s[:3]] == words and not s[3:].any()
     out, _, r = oracle.decode_verify(wire, TILE, TILE)
     assert r.status == 0 and np.array_equal(out.view("<u2"), v)
 
@@ -311,8 +344,7 @@ def test_golden_worked_examples():
             e = spec["element"][0]
             v[int(e[0])] = int(e[2], 16)
         if name == "escapes":
-            for i in range(32):
-                v[64 * (i // 2) + i % 2] = 147 << 7
+            v = _escapes_example()
         wire, flags, entry, t = _encode_one_tile(v)
         if "anchors" in spec:
             assert list(t[0:8]) == [int(x) for x in spec["anchors"][0]], name
@@ -320,20 +352,27 @@ def test_golden_worked_examples():
             assert list(t[8:24].view("<u2")) == [int(x) for x in spec["counts"][0]], name
         if "entry" in spec:
             assert entry == int(spec["entry"][0][0], 16), name
+        lens = np.zeros(256, dtype=np.int64)
+        for item in spec.get("lengths", [[]])[0]:
+            at, val = item.split(":")
+            lens[int(at)] = int(val)
+        assert list(t[8256:8512]) == list(lens), name
+        counts = t[8:24].view("<u2")
         for sh in spec.get("share", []):
             share = int(sh[0])
-            counts = t[8:24].view("<u2")
             start = int(counts[:share].sum())
-            stream = t[8256 + 2 * start: 8256 + 2 * (start + int(counts[share]))].view("<u2")
-            seen = np.zeros(stream.size, dtype=bool)
+            stream = t[8512 + 4 * start: 8512 + 4 * (start + int(counts[share]))].view("<u4")
+            want = np.zeros(stream.size, dtype=np.int64)
             for item in sh[2:]:
                 rng_, val = item.split(":")
                 lo, hi = (rng_.split("-") + [rng_])[:2]
-                for i in range(int(lo), int(hi) + 1):
-                    assert int(stream[i]) == int(val, 16), (name, i)
-                    seen[i] = True
-            if name != "escapes":
-                assert not stream[~seen].any(), name
+                want[int(lo): int(hi) + 1] = int(val, 16)
+            assert [int(x) for x in stream] == list(want), name
+        listed = {int(sh[0]) for sh in spec.get("share", [])}
+        for share in range(8):
+            if share not in listed:
+                start = int(counts[:share].sum())
+                assert not t[8512 + 4 * start: 8512 + 4 * (start + int(counts[share]))].any(), (name, share)
 
 
 def test_no_bit_of_an_image_with_both_options_can_flip_unnoticed():
@@ -364,25 +403,28 @@ def test_spare_bytes_and_anchors_of_coded_tiles_are_checked():
     v = _gauss(TILE // 2, 33)
     wire, _, res = oracle.encode(v.view(np.uint8), TILE, entropy=True)
     me = oracle.meta_end(TILE, TILE)
-    for at in (me + 24, me + 63, res.wire_len - 1):          # spare header bytes; the last fill byte, if the tile has fill
-        if at == res.wire_len - 1:
-            counts = wire[me + 8: me + 24].view(np.uint16).astype(np.int64)
-            if 8256 + 2 * int(counts.sum()) == res.wire_len - me:
-                continue
+    words = int(wire[me + 8: me + 24].view(np.uint16).astype(np.int64).sum())
+    spots = [me + 24, me + 63]                               # spare header bytes
+    if 8512 + 4 * words < res.wire_len - me:
+        spots.append(res.wire_len - 1)                       # the last fill byte, when the tile has fill
+    for at in spots:
         w = wire.copy()
         w[at] ^= 0x40
         assert oracle.decode_verify(w, TILE, TILE)[2].status_name == "ERR_DESC", at
-    # an anchor that moves shifts everything its share decodes to, which the chunk CRC sees ...
+    # an anchor that moves shifts everything its share decodes to, which the chunk CRC sees
     w = wire.copy()
     w[me + 3] += 1
     assert oracle.decode_verify(w, TILE, TILE)[2].status_name == "ERR_CHUNK_CRC"
-    # ... unless every codeword of the share is an escape (the exponent itself): then only the rule
-    # that an anchor is the rounded mean of its share stands between a flipped anchor bit and OK
-    E = np.full(8192, 120)
-    E[3 * 1024: 4 * 1024] = np.tile([0, 255], 512)              # share 3: mean 127.5 -> anchor 128, all escapes
-    t = ((E << 7) | 0x15).astype("<u2")
-    wire, _, res = oracle.encode(t.view(np.uint8), TILE, entropy=True, ent_only=True)
-    assert wire[me + 3] == 128 and oracle.decode_verify(wire, TILE, TILE)[2].status == 0
+    # ... but the same exponents can be written with another anchor: E = 127 everywhere is '00' under
+    # anchor 127 and '10' (u = +1) under anchor 126.  Such an image decodes to the right bytes; it is
+    # refused because an anchor must be the rounded mean of what its share decodes to.
+    wire, _, res = oracle.encode(_tile_of(0x3F80).view(np.uint8), TILE, entropy=True, ent_only=True)
+    assert oracle.decode_verify(wire, TILE, TILE)[2].status == 0
     w = wire.copy()
-    w[me + 3] ^= 4
+    w[me + 0] = 126
+    w[me + 8512: me + 8512 + 256] = 0x55                     # '10' is the number 1 in a 2-bit field
+    assert oracle.decode_verify(w, TILE, TILE)[2].status_name == "ERR_DESC"
+    # a strand length that does not match its codewords
+    w = wire.copy()
+    w[me + 8256 + 7] = 2
     assert oracle.decode_verify(w, TILE, TILE)[2].status_name == "ERR_DESC"
