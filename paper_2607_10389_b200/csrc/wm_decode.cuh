@@ -314,11 +314,10 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
     // ENT: what the low byte of a strand's bits says about the codeword there: its length (16: the
     // escape) and u as a byte.  Two byte tables: the index needs no scaling and a look-up gives a
     // clean value.
-    __shared__ unsigned char s_plen[ENT ? 256 : 4], s_pu[ENT ? 256 : 4];
+    __shared__ unsigned short s_ptab[ENT ? 256 : 2];       // length | u << 8 (length 16: the escape)
     if (ENT != 0 && threadIdx.x < 256u) {
         const uint32_t s = ent_ones(threadIdx.x);
-        s_plen[threadIdx.x] = (unsigned char)ent_parse_length(s);
-        s_pu[threadIdx.x] = (unsigned char)(s == 8u ? 0u : ent_parse_value(threadIdx.x, s, 0u));
+        s_ptab[threadIdx.x] = (unsigned short)(ent_parse_length(s) | (s == 8u ? 0u : (ent_parse_value(threadIdx.x, s, 0u) & 0xFFu) << 8));
     }
     Smem S = setup_smem(smem, tab);
     grid_dep_wait();
@@ -420,45 +419,58 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
             if (!is_pack) {
                 read_staged_words(stage, warp, lane, w);
             } else if (is_ent) {
-                // ENT tile.  Header: the eight stream lengths against the entry (structure); then this
-                // warp reads its share's stream the way the format interleaves it: at step i every
-                // strand whose codeword i is not complete in the bits it holds takes the stream's next
-                // halfword, strands in ascending order.  The stream must be used up exactly and the
-                // bits left in every strand must be zero (descriptor error otherwise).
+                // ENT tile.  Header: the eight word counts against the entry (structure).  Then lane l
+                // reads strand l of this warp's share: the strands lie one behind the other in the
+                // share's stream and their lengths are written down, so a prefix sum over the lanes
+                // gives every lane the bit where its strand starts, and from there it reads its 32
+                // codewords through a 64-bit window that is refilled a word at a time before every
+                // second codeword.  No lane waits for another.
                 const uint32_t cnt = lane < 8u ? lds_now_u16(stage_s + 8u + 2u * lane) : 0u;
-                const bool cnt_bad = lane < 8u && (cnt < 128u || cnt > 1024u);
+                const bool cnt_bad = lane < 8u && (cnt < 64u || cnt > 319u);
                 const uint32_t total = __reduce_add_sync(0xFFFFFFFFu, cnt);
                 const uint32_t before = __reduce_add_sync(0xFFFFFFFFu, lane < warp ? cnt : 0u);
                 const uint32_t mine = __shfl_sync(0xFFFFFFFFu, cnt, warp);
                 int verdict = (__any_sync(0xFFFFFFFFu, cnt_bad) || ent_tile_bytes(total) != 32u * (e & 0x7FFFu)) ? 2 : 0;
+                const uint32_t nb = 64u + lds_now_u8(stage_s + 8256u + 32u * warp + lane);      // this strand's bits
+                uint32_t incl = nb;
+#pragma unroll
+                for (int d = 1; d < 32; d <<= 1) {
+                    const uint32_t o = __shfl_up_sync(0xFFFFFFFFu, incl, d);
+                    if (lane >= (uint32_t)d) incl += o;
+                }
+                const uint32_t share_bits = __shfl_sync(0xFFFFFFFFu, incl, 31);
+                if (!verdict && ((share_bits + 31u) >> 5) != mine) verdict = 1;
                 if (!verdict) {
                     const uint32_t anchor = lds_now_u8(stage_s + warp);
-                    const uint32_t st = stage_s + 8256u + 2u * before;
-                    const uint32_t lt_mask = (1u << lane) - 1u;
-                    uint32_t buf = 0, avail = 0, pos = 0, ew[8];
-                    const uint32_t last = mine - 1u;           // (mine >= 128)
+                    const uint32_t st = stage_s + 8512u + 4u * before;
+                    const uint32_t start = incl - nb, wi = start >> 5, sh = start & 31u;
+                    // (a strand that runs past its length only fails the check below: no word beyond
+                    // the share's last two is ever read)
+                    unsigned long long buf = (((unsigned long long)lds_now<4>(st + 4u * wi) << 32) | lds_now<0>(st + 4u * wi)) >> sh;
+                    uint32_t avail = 64u - sh, next = wi + 2u, ew[8];
 #pragma unroll
                     for (int j = 0; j < 8; j++) ew[j] = 0u;
 #pragma unroll
                     for (int i = 0; i < 32; i++) {
-                        const bool more = s_plen[buf & 0xFFu] > avail;
-                        const uint32_t takers = __ballot_sync(0xFFFFFFFFu, more);
-                        if (more) {
-                            // (an index past the stream's end is only clamped here: the stream then
-                            // fails the count check below, because every index is below the final pos)
-                            const uint32_t idx = min(pos + __popc(takers & lt_mask), last);
-                            buf |= lds_now_u16(st + 2u * idx) << avail;
-                            avail += 16u;
+                        if ((i & 1) == 0 && avail <= 32u) {
+                            buf |= (unsigned long long)lds_now<0>(st + 4u * min(next, mine + 1u)) << avail;
+                            avail += 32u;
+                            next++;
                         }
-                        pos += __popc(takers);
-                        const uint32_t low = buf & 0xFFu;
-                        const uint32_t len = s_plen[low];
-                        const uint32_t E = len == 16u ? buf >> 8 : anchor + s_pu[low];      // (its low byte)
+                        const uint32_t lo32 = (uint32_t)buf;
+                        const uint32_t tv = s_ptab[lo32 & 0xFFu];
+                        const uint32_t len = tv & 31u;
+                        const uint32_t E = len == 16u ? lo32 >> 8 : anchor + (tv >> 8);      // (its low byte)
                         ew[i >> 2] = __byte_perm(ew[i >> 2], E, (i & 3) == 0 ? 0x3214 : (i & 3) == 1 ? 0x3240 : (i & 3) == 2 ? 0x3410 : 0x4210);
                         buf >>= len;
                         avail -= len;
                     }
-                    if (__any_sync(0xFFFFFFFFu, buf != 0u) || pos != mine) verdict = 1;
+                    // the 32 codewords took exactly the strand's length; behind the last strand the
+                    // stream's last word is zero
+                    const uint32_t used = 32u * (next - wi) - sh - avail;
+                    const uint32_t fill = 32u * mine - share_bits;
+                    const bool fill_bad = lane == 31u && ((uint32_t)buf & ((1u << fill) - 1u)) != 0u;
+                    if (__any_sync(0xFFFFFFFFu, used != nb || fill_bad)) verdict = 1;
                     // the anchor must be what the encoder writes: the rounded mean of the share's exponents
                     // (otherwise the anchor of a share that holds escapes only could change unnoticed)
                     uint32_t esum = 0;
@@ -468,9 +480,9 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
                     // the bytes that carry nothing are zero: the header's spare 40, the fill behind the last stream
                     if (warp == 0u) {
                         const uint32_t spare = (lane >= 6u && lane < 16u) ? lds_now<0>(stage_s + 4u * lane) : 0u;
-                        const uint32_t fill_at = 8256u + 2u * total + 2u * lane;
-                        const uint32_t fill = fill_at < 32u * (e & 0x7FFFu) ? lds_now_u16(stage_s + fill_at) : 0u;
-                        if (__any_sync(0xFFFFFFFFu, (spare | fill) != 0u)) verdict = 1;
+                        const uint32_t fill_at = 8512u + 4u * total + 4u * lane;
+                        const uint32_t end_fill = fill_at < 32u * (e & 0x7FFFu) ? lds_now<0>(stage_s + fill_at) : 0u;
+                        if (__any_sync(0xFFFFFFFFu, (spare | end_fill) != 0u)) verdict = 1;
                     }
 #pragma unroll
                     for (int j = 0; j < 4; j++) {

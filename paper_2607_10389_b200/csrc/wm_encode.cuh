@@ -209,8 +209,8 @@ struct EncTeamCtl {
     uint32_t wdig[8][8];    // per warp: its contribution to the tile digest
     uint32_t wsum[8];       // sum of widths so far | warps arrived << 16 (the last warp publishes)
     uint32_t ssum[8];       // sum of the 32 widths of the slot's tile (set by that last warp), or a mark:
-                            // zero tile, constant tile, kSumEnt | halfwords for a tile stored in ENT form
-    uint32_t etab[8][8];    // entropy option, per warp: anchor | halfwords of its stream << 8
+                            // zero tile, constant tile, kSumEnt | words of the streams for a tile stored in ENT form
+    uint32_t etab[8][8];    // entropy option, per warp: anchor | words of its stream << 8 (0xFFFF: a strand too long for the form)
     uint32_t next[2];       // ticket claimed in this step (>= n_tiles: none left), by step parity
     uint32_t pad[2];
     unsigned long long excl[2];   // offset of the tile packed in the next step, by step parity
@@ -218,6 +218,8 @@ struct EncTeamCtl {
     unsigned long long pad2;
     unsigned long long nptr[2];   // leaf mode: address (k_leaf_map) of the tile in next[], by step parity
     uint32_t kring[8];            // with a mask: the ticket of the tile in each ring slot (placement runs over tickets)
+    unsigned char sbits[4][256];  // entropy option: every strand's bit length - 64, from the measuring step to the
+                                  // packing step three steps on (slot: step mod 4, as in tensor memory)
 };
 static_assert(sizeof(EncTeamCtl) % 16 == 0, "team control block keeps 16-byte alignment");
 
@@ -284,10 +286,10 @@ __device__ __forceinline__ void pack_group_planes(uint32_t e4a, uint32_t e4b, ui
 // ---- ENT tiles: entropy-coded exponents (an encoder option; header flags bit 2) --------------
 // A warp's 2 KiB of a tile (16 rows) is one share; lane l's 32 elements (its 16 words, low half
 // first) are strand l.  Every exponent is coded as u = E - anchor with a fixed prefix code, the
-// anchor being the rounded mean of the share's exponents; a strand is an LSB-first bit string
-// cut into halfwords, and the 32 strands of a share are interleaved in the order a reader
-// needs them: at step i every strand whose codeword i is not complete in what it has taken so
-// far takes the stream's next halfword, strands in ascending order.
+// anchor being the rounded mean of the share's exponents; a strand is the LSB-first bit string of
+// its 32 codewords, and the 32 strands of a share lie one behind the other in the share's
+// stream, their lengths written down in a byte each, so that every lane of the reading warp
+// finds the start of its strand with one prefix sum and nobody waits for anybody.
 //   u        -6  -5  -4  -3  -2  -1   0   1   2   3   other
 //   length    8   6   5   4   4   2   2   2   4   7   16 (eight ones, then E itself)
 //   bits    127  31  15  11   3   2   0   1   7  63   255 | E << 8        (first bit = bit 0)
@@ -312,11 +314,12 @@ __device__ __forceinline__ uint32_t ent_word(uint32_t slot, uint32_t E)
     const uint32_t w = ent_lut(0x0B0F1F7Fu, 0x01000203u, 0x00FF3F07u, slot);       // 127 31 15 11 | 3 2 0 1 | 7 63 255
     return w | (slot == 10u ? E << 8 : 0u);
 }
-// Bytes of an ENT tile whose eight streams hold `halfwords` halfwords in all (a multiple of 32;
-// 16384 or more means that the tile is stored raw instead).
-__device__ __forceinline__ uint32_t ent_tile_bytes(uint32_t halfwords)
+// Bytes of an ENT tile whose eight streams hold `words` 32-bit words in all (a multiple of 32;
+// 16384 or more means that the tile takes another form): header, sign-mantissa plane, strand
+// lengths, streams.
+__device__ __forceinline__ uint32_t ent_tile_bytes(uint32_t words)
 {
-    return (8256u + 2u * halfwords + 31u) & ~31u;
+    return (8512u + 4u * words + 31u) & ~31u;
 }
 // Decoder side.  A codeword is s ones and a zero (s < 8; eight ones: the escape), followed for
 // s = 0 and s = 2 by one more bit x:  s = 0: u = -x;  1: +1;  2: -2 - x;  3: +2;  4..7: -4, -5, +3, -6.
@@ -356,7 +359,7 @@ __device__ __forceinline__ uint32_t ent_parse_value(uint32_t buf, uint32_t s, ui
 // tickets are claimed one step further ahead so that a tile's address can be looked up on the
 // way), ZEROS (the zero / constant tile option), ENT (the entropy option: the measuring step also
 // adds up codeword lengths, the tile takes the shorter of the two coded forms, and for the ENT
-// form the packing step writes the share's interleaved stream of halfwords instead of bit planes).
+// form the packing step writes the strands' lengths and the share's stream of words instead of bit planes).
 // Packed data goes from registers to the wire image directly: in every region of a PACK tile
 // a lane owns an aligned unit at a lane-strided place, so each warp store is one contiguous
 // sector-aligned run.  Claiming a tile before the previous offset is known means that, if the
@@ -374,7 +377,7 @@ constexpr uint32_t kQOffShift = 22;
 // kWarpConst: all 1024 elements of the warp's rows hold one value (its sign-mantissa byte rides in
 // bits 16-23 of the entry, the exponent is the base); kSumConstTile: the tile holds one value.
 constexpr uint32_t kWarpAllZero = 0x8000u, kWarpConst = 0x4000u, kSumZeroTile = 0xFFFFu, kSumConstTile = 0xFFFEu;
-// The tile is stored in ENT form (shorter than its bit planes and than raw); low half: halfwords.
+// The tile is stored in ENT form (shorter than its bit planes and than raw); low half: words of its streams.
 constexpr uint32_t kSumEnt = 0x10000u;
 
 // The tile behind ticket k.  Without a mask tickets are tile numbers.  With one, only the tiles of
@@ -568,10 +571,10 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
 #pragma unroll
             for (int i = 0; i < 16; i++) d[i] = __funnelshift_l(d[i], d[i], 1);
             uint32_t gw[4];               // per group: base | width << 8
-            uint32_t ent_w = 0;           // entropy option: anchor | halfwords << 8 of this warp's share
+            uint32_t ent_w = 0;           // entropy option: anchor | words << 8 of this warp's share
             if (ENT) {
                 // the share's anchor (rounded mean of its 1024 exponents: bytes 1 and 3 of a rotated
-                // word) and the halfwords its 32 strands need
+                // word), every strand's length in bits and the words the share's stream needs
                 uint32_t acc = 0;
 #pragma unroll
                 for (int i = 0; i < 16; i++) acc = __dp4a(d[i], 0x01000100u, acc);       // bytes 1 and 3
@@ -580,8 +583,12 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
 #pragma unroll
                 for (int i = 0; i < 16; i++)
                     bits += s_len8[ent_slot(__byte_perm(d[i], 0u, 0x4441), anchor)] + s_len8[ent_slot(d[i] >> 24, anchor)];
-                const uint32_t count = __reduce_add_sync(0xFFFFFFFFu, (bits + 15u) >> 4);
-                ent_w = anchor | (count << 8);
+                // (a strand the length byte cannot hold, above 319 bits, keeps the tile out of the form:
+                // the count is then so large that the form is never the shortest)
+                const uint32_t share_bits = __reduce_add_sync(0xFFFFFFFFu, bits);
+                const bool too_long = __any_sync(0xFFFFFFFFu, bits > 319u);
+                tc->sbits[step & 3u][32u * warp + lane] = (unsigned char)(bits - 64u);
+                ent_w = anchor | ((too_long ? 0xFFFFu : (share_bits + 31u) >> 5) << 8);
             }
             {
 #pragma unroll
@@ -662,7 +669,7 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
             tmem_load16(tmem_warp + 16u * ((step + 1u) & 3u), d);
             const uint32_t Smark = tc->ssum[sl];
             const bool ent_form = ENT && (Smark & kSumEnt) != 0u;
-            const uint32_t Ssum = ent_form ? Smark & 0xFFFFu : Smark;       // halfwords, or the sum of the widths
+            const uint32_t Ssum = ent_form ? Smark & 0xFFFFu : Smark;       // words of the streams, or the sum of the widths
             const bool packs = !ent_form && Ssum <= 253u;
             // (a tile of all-zero bytes, marked in ssum, is its table entry and nothing else)
             const uint32_t enc_len = ent_form ? ent_tile_bytes(Ssum)
@@ -672,7 +679,7 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
             if (exclX + enc_len > room) {
                 trouble |= 1u;
             } else if (ent_form) {
-                // header: anchors, stream lengths, 40 zero bytes; zero fill behind the last stream
+                // header: anchors, word counts, 40 zero bytes; zero fill behind the last stream
                 if (warp == 5) {
                     if (lane < 8u) {
                         const uint32_t wt = tc->etab[sl][lane];
@@ -681,7 +688,7 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
                     } else if (lane < 18u) {
                         st_stream_u32(dst + 24u + 4u * (lane - 8u), 0u);
                     }
-                    if (2u * lane < enc_len - 8256u - 2u * Ssum) stg_u16(dst + 8256u + 2u * Ssum + 2u * lane, 0u);
+                    if (4u * lane < enc_len - 8512u - 4u * Ssum) st_stream_u32(dst + 8512u + 4u * Ssum + 4u * lane, 0u);
                 }
                 unsigned char* const sm_dst = dst + sm_off;
 #pragma unroll
@@ -690,33 +697,49 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
                     const uint32_t ya = __byte_perm(sa, sa, 0x2301), yb = __byte_perm(sb, sb, 0x2301);
                     stg_v2(sm_dst + 256 * j, (sa & 0xFEFEFEFEu) | (ya & 0x01010101u), (sb & 0xFEFEFEFEu) | (yb & 0x01010101u));
                 }
-                // this share's stream: it starts behind the streams of the warps before it
+                // This share's stream starts behind the streams of the warps before it; inside it the
+                // strands follow one another bit by bit, so lane l starts where the lengths of the
+                // lanes before it (measured three steps ago) add up to.
                 const uint32_t before = __reduce_add_sync(0xFFFFFFFFu, lane < warp ? tc->etab[sl][lane] >> 8 : 0u);
                 const uint32_t anchor = tc->etab[sl][warp] & 0xFFu;
-                unsigned char* const hw_dst = dst + 8256u + 2u * before;
-                const uint32_t lt_mask = (1u << lane) - 1u;
-                // acc: the strand's bits from the start of the halfword it took last (number `pend` of
-                // the stream) on; n of them are valid.  Step 0: every strand takes one halfword.
-                uint32_t acc = 0, n = 0, pend = lane, pos = 32;
+                const uint32_t nb8 = tc->sbits[(step + 1u) & 3u][32u * warp + lane];
+                stg_u8(dst + 8256u + 32u * warp + lane, nb8);
+                uint32_t incl = 64u + nb8;
+#pragma unroll
+                for (int k = 1; k < 32; k <<= 1) {
+                    const uint32_t o = __shfl_up_sync(0xFFFFFFFFu, incl, k);
+                    if (lane >= (uint32_t)k) incl += o;
+                }
+                const uint32_t start = incl - 64u - nb8;
+                unsigned char* const w_dst = dst + 8512u + 4u * before;
+                // acc: the stream's bits from the last word boundary on, n of them valid (the first n
+                // of the lane's first word belong to the lane before it).  Words go out as they fill
+                // up, except the lane's first one, which is held back until the lane before has handed
+                // over the bits it left in it.
+                unsigned long long acc = 0;
+                uint32_t n = start & 31u, wp = start >> 5, w_first = 0;
+                bool have_first = false;
 #pragma unroll
                 for (int i = 0; i < 32; i++) {
                     const uint32_t E = (i & 1) ? d[i >> 1] >> 24 : __byte_perm(d[i >> 1], 0u, 0x4441);
                     const uint32_t cw = s_ent[ent_slot(E, anchor)];
                     // (the table's escape entry is 0xFFFF: the AND lets the exponent through there only)
-                    acc |= (cw & ((E << 8) | 0xFFu)) << n;
+                    acc |= (unsigned long long)(cw & ((E << 8) | 0xFFu) & 0xFFFFu) << n;
                     n += cw >> 16;
-                    if (i == 0) continue;
-                    const bool more = n > 16u;             // the codeword runs past what the strand has taken
-                    const uint32_t takers = __ballot_sync(0xFFFFFFFFu, more);
-                    if (more) {
-                        stg_u16(hw_dst + 2u * pend, acc & 0xFFFFu);
-                        acc >>= 16;
-                        n -= 16u;
-                        pend = pos + __popc(takers & lt_mask);
+                    if ((i & 1) && n >= 32u) {             // (two codewords are 32 bits at most: one word per pair)
+                        const uint32_t word = (uint32_t)acc;
+                        if (have_first) st_stream_u32(w_dst + 4u * wp, word); else w_first = word;
+                        have_first = true;
+                        acc >>= 32;
+                        n -= 32u;
+                        wp++;
                     }
-                    pos += __popc(takers);
                 }
-                stg_u16(hw_dst + 2u * pend, acc & 0xFFFFu);
+                // (a strand is 64 bits at least, so every lane has crossed a word boundary by now)
+                const uint32_t tail = (uint32_t)acc;                   // n bits of the next word, 0 when n == 0
+                const uint32_t from_below = __shfl_up_sync(0xFFFFFFFFu, tail, 1);
+                st_stream_u32(w_dst + 4u * (start >> 5), w_first | (lane ? from_below : 0u));
+                if (lane == 31u && n) st_stream_u32(w_dst + 4u * wp, tail);
             } else if (packs) {
                 if (warp == 5) {           // (any one warp: not one that has a single-lane chore)
                     const uint32_t wt = tc->wtab[sl][lane];
