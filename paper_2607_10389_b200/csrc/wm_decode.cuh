@@ -303,8 +303,8 @@ __device__ __forceinline__ void unpack_group_planes(const PlaneWords& pw, uint32
 // ENT 1 / 2: the image was written with the entropy option and holds ENT tiles only (1) or ENT
 // and PACK tiles (2; the check kernel noted which).  A call launches both, and the one that does
 // not apply returns at once: the kernel with a single kind of coded tile is the faster one.  A
-// warp reads its share's stream of halfwords in phase 1 (the need test, the ballot and the fetch
-// of every step) and leaves the exponent bytes where the plane words would be.
+// warp reads its share's stream in phase 1, every lane its own strand, and leaves the exponent
+// bytes where the plane words would be.
 template <int TEAMS, bool LEAVES, int MODE, int ENT = 0>
 __global__ void __launch_bounds__(TEAMS * 256, 1)
 k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restrict__ dst, Ws ws,
@@ -446,30 +446,36 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
                     const uint32_t start = incl - nb, wi = start >> 5, sh = start & 31u;
                     // (a strand that runs past its length only fails the check below: no word beyond
                     // the share's last two is ever read)
-                    unsigned long long buf = (((unsigned long long)lds_now<4>(st + 4u * wi) << 32) | lds_now<0>(st + 4u * wi)) >> sh;
+                    // The window: lo holds the next 32 bits of the strand, hi what follows, `avail` of the
+                    // 64 are real.  (PTX shifts clamp at 32, which is what the edge cases need.)
+                    uint32_t lo = lds_now<0>(st + 4u * wi), hi = lds_now<4>(st + 4u * wi);
+                    lo = __funnelshift_r(lo, hi, sh);
+                    hi >>= sh;
                     uint32_t avail = 64u - sh, next = wi + 2u, ew[8];
 #pragma unroll
                     for (int j = 0; j < 8; j++) ew[j] = 0u;
 #pragma unroll
                     for (int i = 0; i < 32; i++) {
-                        if ((i & 1) == 0 && avail <= 32u) {
-                            buf |= (unsigned long long)lds_now<0>(st + 4u * min(next, mine + 1u)) << avail;
+                        if ((i & 1) == 0 && avail <= 32u) {      // (two codewords take 32 bits at most)
+                            const uint32_t w = lds_now<0>(st + 4u * min(next, mine + 1u));
+                            lo |= shl_clamp(w, avail);
+                            hi = shr_clamp(w, 32u - avail);
                             avail += 32u;
                             next++;
                         }
-                        const uint32_t lo32 = (uint32_t)buf;
-                        const uint32_t tv = s_ptab[lo32 & 0xFFu];
+                        const uint32_t tv = s_ptab[lo & 0xFFu];
                         const uint32_t len = tv & 31u;
-                        const uint32_t E = len == 16u ? lo32 >> 8 : anchor + (tv >> 8);      // (its low byte)
+                        const uint32_t E = len == 16u ? lo >> 8 : anchor + (tv >> 8);      // (its low byte)
                         ew[i >> 2] = __byte_perm(ew[i >> 2], E, (i & 3) == 0 ? 0x3214 : (i & 3) == 1 ? 0x3240 : (i & 3) == 2 ? 0x3410 : 0x4210);
-                        buf >>= len;
+                        lo = __funnelshift_r(lo, hi, len);
+                        hi >>= len;
                         avail -= len;
                     }
                     // the 32 codewords took exactly the strand's length; behind the last strand the
                     // stream's last word is zero
                     const uint32_t used = 32u * (next - wi) - sh - avail;
                     const uint32_t fill = 32u * mine - share_bits;
-                    const bool fill_bad = lane == 31u && ((uint32_t)buf & ((1u << fill) - 1u)) != 0u;
+                    const bool fill_bad = lane == 31u && (lo & ((1u << fill) - 1u)) != 0u;
                     if (__any_sync(0xFFFFFFFFu, used != nb || fill_bad)) verdict = 1;
                     // the anchor must be what the encoder writes: the rounded mean of the share's exponents
                     // (otherwise the anchor of a share that holds escapes only could change unnoticed)

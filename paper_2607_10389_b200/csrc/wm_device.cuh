@@ -232,6 +232,21 @@ __device__ __forceinline__ uint32_t ld_volatile_u32(const uint32_t* p)
     return v;
 }
 
+// Shifts whose amount may be 32 (the result is then 0, as the hardware's shifts define it; in C
+// a shift by the operand's width is undefined).
+__device__ __forceinline__ uint32_t shl_clamp(uint32_t v, uint32_t n)
+{
+    uint32_t r;
+    asm("shl.b32 %0, %1, %2;" : "=r"(r) : "r"(v), "r"(n));
+    return r;
+}
+__device__ __forceinline__ uint32_t shr_clamp(uint32_t v, uint32_t n)
+{
+    uint32_t r;
+    asm("shr.b32 %0, %1, %2;" : "=r"(r) : "r"(v), "r"(n));
+    return r;
+}
+
 __device__ __forceinline__ uint32_t min_u16x2(uint32_t a, uint32_t b)
 {
     uint32_t d;

@@ -634,10 +634,10 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
                 const uint32_t wt = *reinterpret_cast<volatile uint32_t*>(&tc->wtab[slY][lane]);
                 const uint32_t total = __reduce_add_sync(0xFFFFFFFFu, (wt >> 8) & 15u);
                 // entropy option: the ENT form is taken when it is shorter than the planes and than raw
-                uint32_t halfwords = 0;
-                if (ENT) halfwords = __reduce_add_sync(0xFFFFFFFFu, lane < 8u ? *reinterpret_cast<volatile uint32_t*>(&tc->etab[slY][lane]) >> 8 : 0u);
+                uint32_t ent_words = 0;
+                if (ENT) ent_words = __reduce_add_sync(0xFFFFFFFFu, lane < 8u ? *reinterpret_cast<volatile uint32_t*>(&tc->etab[slY][lane]) >> 8 : 0u);
                 const uint32_t plane_len = total <= 253u ? 8256u + 32u * total : kTile;
-                const bool ent_tile = ENT && ent_tile_bytes(halfwords) < plane_len;
+                const bool ent_tile = ENT && ent_tile_bytes(ent_words) < plane_len;
                 // unused memory (every warp's first entry carries the mark): no payload
                 // (one value throughout: every warp's first entry carries the mark and they are all alike;
                 // a tile of zeros has no payload, any other value 32 bytes)
@@ -645,9 +645,9 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
                 const bool const_tile = ZEROS && __all_sync(0xFFFFFFFFu, (lane & 3u) != 0u || ((wt & kWarpConst) != 0u && wt == wt0));
                 const bool zero_tile = const_tile && (wt0 & kWarpAllZero) != 0u;
                 if (lane == 0) {
-                    tc->ssum[slY] = zero_tile ? kSumZeroTile : const_tile ? kSumConstTile : ent_tile ? kSumEnt | halfwords : total;
+                    tc->ssum[slY] = zero_tile ? kSumZeroTile : const_tile ? kSumConstTile : ent_tile ? kSumEnt | ent_words : total;
                     tc->wsum[slY] = 0;
-                    publish_len(slY, tYn, zero_tile ? 0u : const_tile ? 32u : ent_tile ? ent_tile_bytes(halfwords) : plane_len);
+                    publish_len(slY, tYn, zero_tile ? 0u : const_tile ? 32u : ent_tile ? ent_tile_bytes(ent_words) : plane_len);
                 }
             }
             tmem_store16(tmem_warp + 16u * (step & 3u), d);
