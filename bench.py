@@ -591,8 +591,9 @@ def entropy_option(wm, cfg, cur, shadow, wire, ws, dev, W_plain, peak, reps=20):
             out[name + "_frac_of_hbm_peak"] = (N + W) / (ms * 1e-3) / 1e9 / peak
     finally:
         wm.entropy_enable(False)
-    out["note"] = ("wm_entropy_enable(1): fixed prefix code of the exponents, strands interleaved in reader order; "
-                   "whole calls back to back; bound by integer instruction issue (one codeword per lane and step)")
+    out["note"] = ("wm_entropy_enable(1): fixed prefix code of the exponents, a share's strands one behind the other with "
+                   "their lengths written down; whole calls back to back; bound by integer instruction issue (one "
+                   "table look-up per codeword and lane)")
     return out
 
 
