@@ -89,3 +89,54 @@ def test_placement_is_repeatable_over_many_moves_and_block_counts():
         if i % 4 == 0:
             wm.wm_decode_verify_opt(wire, r.wire_len, dst, chunk, dcrc, ws, res, (opt & wm.OPT_ENTROPY) | wm.opt_blocks(bd))
             assert wm.read_result(res).ok and torch.equal(dst, cur) and torch.equal(dcrc, crc), (i, opt, bd)
+
+
+@pytest.mark.parametrize("chunk_tiles", [1, 3, 4])
+@pytest.mark.parametrize("options,kw", [(0, {}), (wm.OPT_ENTROPY | wm.OPT_ZERO_TILES, {"entropy": True, "zero_tiles": True})])
+def test_sparse_and_degenerate_masks(chunk_tiles, options, kw):
+    """Masked calls claim only the tiles of present chunks.  The masks that stress that: nothing
+    present, everything present (with the mask flag), only the short last chunk, everything but
+    the last chunk, single chunks, every other chunk; chunk sizes of 1, 3 (no power of two) and
+    4 tiles on a cache whose last chunk and last tile are ragged.  Image, CRC vector and result
+    are the oracle's; the decode installs exactly the present chunks."""
+    TILE = 16384
+    chunk = chunk_tiles * TILE
+    cfg = inputs.CONFIGS["engine_small"]
+    host = inputs.make_cache(cfg)[: 41 * TILE + 777].contiguous()
+    host[7 * TILE: 9 * TILE] = 0
+    cur = host.cuda()
+    n = cur.numel()
+    nc = wm.num_chunks(n, chunk)
+    masks = {"none": np.zeros(nc, np.uint8), "all": np.ones(nc, np.uint8)}
+    m = np.zeros(nc, np.uint8); m[-1] = 1; masks["last only"] = m
+    m = np.ones(nc, np.uint8); m[-1] = 0; masks["all but last"] = m
+    m = np.zeros(nc, np.uint8); m[0] = 1; masks["first only"] = m
+    m = np.zeros(nc, np.uint8); m[nc // 2] = 1; masks["one in the middle"] = m
+    masks["every other"] = (np.arange(nc) % 2).astype(np.uint8)
+    masks["every other, and the last"] = ((np.arange(nc) % 2 == 0) | (np.arange(nc) == nc - 1)).astype(np.uint8)
+    rng = np.random.default_rng(1)
+    crc_in = rng.integers(0, 2**32, nc, dtype=np.uint64).astype(np.uint32)
+    ws, res = wm.new_workspace(n, chunk), wm.new_result()
+    wire = torch.zeros(wm.wire_bound(n, chunk), dtype=torch.uint8, device="cuda")
+    old = torch.full((n,), 0x3C, dtype=torch.uint8, device="cuda")
+    for name, mask in masks.items():
+        want_wire, want_crc, want = oracle.encode(host.numpy(), chunk, dirty=mask, crc_in=crc_in, **kw)
+        crc = torch.from_numpy(crc_in.view(np.int32).copy()).cuda()
+        wire.fill_(0xEE)
+        wm.wm_encode_opt(cur, chunk, torch.from_numpy(mask).cuda(), crc, wire, ws, res, options)
+        r = wm.read_result(res)
+        assert r.ok and (r.wire_len, r.cache_crc, r.n_present, r.payload_bytes) == \
+            (want.wire_len, want.cache_crc, want.n_present, want.payload_bytes), name
+        assert np.array_equal(wire[: r.wire_len].cpu().numpy(), want_wire), name
+        assert np.array_equal(crc.cpu().numpy().view(np.uint32), want_crc), name
+        dst = old.clone()
+        dcrc = torch.from_numpy(want_crc.view(np.int32).copy()).cuda()
+        wm.wm_decode_verify_opt(wire, r.wire_len, dst, chunk, dcrc, ws, res, options & wm.OPT_ENTROPY)
+        assert wm.read_result(res).ok, name
+        got = dst.cpu().numpy()
+        for c in range(nc):
+            lo, hi = c * chunk, min((c + 1) * chunk, n)
+            if mask[c]:
+                assert np.array_equal(got[lo:hi], host.numpy()[lo:hi]), (name, c)
+            else:
+                assert (got[lo:hi] == 0x3C).all(), (name, c)
