@@ -167,7 +167,6 @@ k_leaf_scatter(const wm_leaf* __restrict__ leaves, uint32_t n, Geo g, Ws ws)
     grid_dep_wait();
     grid_dep_launch();
     if (ld_volatile_u32(&ws.ctrl->gate)) return;
-    const uint16_t* tab16 = nullptr;
     const uint32_t n_walked = ld_volatile_u32(&ws.ctrl->n_walked);
     for (uint32_t s = blockIdx.x; s < n_walked; s += gridDim.x) {
         const uint32_t t = ws.wlist[s];
@@ -178,7 +177,6 @@ k_leaf_scatter(const wm_leaf* __restrict__ leaves, uint32_t n, Geo g, Ws ws)
             for (uint32_t i = threadIdx.x; i < run; i += blockDim.x) dst[i] = slot[off + i];
         });
     }
-    (void)tab16;
 }
 
 }  // namespace wm
