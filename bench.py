@@ -34,6 +34,8 @@ NCU_TRAFFIC_BYTES = {"engine": 1671779840 + 1208417280, "engine_256m": 262412800
 
 # the headline metric as the baseline file words it; a step is one pass of the whole path:
 # wm_checksum, wm_dirty_diff, wm_encode (full, fused with the checksum) and wm_decode_verify
+L2_BYTES = 126 * 1000 * 1000          # B200 L2
+L2_FLUSH_BYTES = 256 << 20
 METRIC = "raw-cache GB/s for checksum+encode and decode+verify, % HBM roofline, ratio"
 
 
@@ -55,20 +57,25 @@ class ClockSampler:
         self.samples, self._stop, self._thread = [], threading.Event(), None
         self.max_mhz = None
 
-    def _run(self):
+    def _open(self):
+        """NVML handle of the GPU (done before the timed region, so that even a region of a few
+        milliseconds gets its samples)."""
+        import pynvml as nv
+        nv.nvmlInit()
+        h = None
+        if self.uuid:
+            try:
+                h = nv.nvmlDeviceGetHandleByUUID(self.uuid)
+            except Exception:
+                h = None
+        if h is None:
+            h = nv.nvmlDeviceGetHandleByIndex(self.index)
+        self.max_mhz = nv.nvmlDeviceGetMaxClockInfo(h, nv.NVML_CLOCK_SM)
+        return nv, h
+
+    def _run(self, nv, h):
         try:
-            import pynvml as nv
-            nv.nvmlInit()
-            h = None
-            if self.uuid:
-                try:
-                    h = nv.nvmlDeviceGetHandleByUUID(self.uuid)
-                except Exception:
-                    h = None
-            if h is None:
-                h = nv.nvmlDeviceGetHandleByIndex(self.index)
-            self.max_mhz = nv.nvmlDeviceGetMaxClockInfo(h, nv.NVML_CLOCK_SM)
-            while not self._stop.is_set():
+            while True:
                 mhz = nv.nvmlDeviceGetClockInfo(h, nv.NVML_CLOCK_SM)
                 try:
                     reasons = nv.nvmlDeviceGetCurrentClocksEventReasons(h)
@@ -79,18 +86,25 @@ class ClockSampler:
                 except Exception:
                     watts = None
                 self.samples.append((mhz, reasons, watts))
-                time.sleep(self.period)
-        except Exception as e:  # NVML missing: report that instead of inventing clocks
+                if self._stop.wait(self.period):
+                    break
+        except Exception as e:
             self.samples.append(("error", str(e), None))
 
     def __enter__(self):
-        self._thread = threading.Thread(target=self._run, daemon=True)
+        try:
+            nv, h = self._open()
+        except Exception as e:  # NVML missing: report that instead of inventing clocks
+            self.samples.append(("error", str(e), None))
+            return self
+        self._thread = threading.Thread(target=self._run, args=(nv, h), daemon=True)
         self._thread.start()
         return self
 
     def __exit__(self, *a):
         self._stop.set()
-        self._thread.join(timeout=2)
+        if self._thread is not None:
+            self._thread.join(timeout=2)
 
     def summary(self):
         good = [s for s in self.samples if s[0] != "error"]
@@ -796,13 +810,28 @@ def main():
         gpu_uuid = "GPU-" + str(torch.cuda.get_device_properties(dev).uuid)
     except Exception:
         gpu_uuid = None
+    # A cache that fits in L2 would be timed out of the cache after its first step: there a buffer
+    # larger than L2 is written between the timed steps, each step in its own pair of events.
+    flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev) if N <= L2_BYTES else None
     with ClockSampler(local_rank, gpu_uuid) as clk:
-        ev0.record()
-        for _ in range(args.steps):
-            step()
-        ev1.record()
-        barrier()
-    ms_total = max_over_ranks(ev0.elapsed_time(ev1))
+        if flush is None:
+            ev0.record()
+            for _ in range(args.steps):
+                step()
+            ev1.record()
+            barrier()
+            ms_total = max_over_ranks(ev0.elapsed_time(ev1))
+        else:
+            pairs = []
+            for _ in range(args.steps):
+                flush.zero_()
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record()
+                step()
+                b.record()
+                pairs.append((a, b))
+            barrier()
+            ms_total = max_over_ranks(sum(a.elapsed_time(b) for a, b in pairs))
     ms_step = ms_total / args.steps
     gpu_launches = launches["n"]
     value = group.aggregate_gbs(N, ms_step)
@@ -1054,7 +1083,8 @@ def main():
             "dtype": "u8", "data": "synthetic",
             "config": {"workload": args.workload, "nbytes": N, "chunk_bytes": C, "shape": list(cfg.shape),
                        "wire_bytes": W, "ratio": W / N, "dirty_chunks": n_rewritten, "n_chunks": nc,
-                       "l2": "inputs larger than L2 (no flush needed)", "parallelism": "replicas only",
+                       "l2": "inputs larger than L2 (no flush needed)" if flush is None else
+                             "cache fits in L2: a 256 MiB buffer is written between the timed steps (each step in its own event pair)", "parallelism": "replicas only",
                        "zero_tiles": bool(args.zero_tiles), "entropy": bool(args.entropy)},
             "calls": per_call, "roofline": roofline, "precopy_loop": loop, "append_loop": append, "leaf_mode": leaf, "entropy_option": ent, "tail_schedule": tail,
             "cpu_baseline": base, "e2e": e2e,
