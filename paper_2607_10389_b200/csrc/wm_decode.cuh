@@ -37,14 +37,20 @@ __device__ __forceinline__ void fill_result(wm_result* result, const Ctrl* ctrl,
 }
 
 // Decode steps 1-3 in one kernel.  The first blocks digest the metadata slices (four teams
-// each), the others check the structure chunk by chunk (one warp per chunk: tile entries
-// against the chunk's length and enc_len; also each tile's offset inside its chunk's payload).
+// each), the others check the structure chunk by chunk (tile entries against the chunk's length
+// and enc_len; also each tile's offset inside its chunk's payload): one warp per chunk, or, when
+// a chunk has 16 tiles or fewer, as many whole chunks as fit the warp's 32 lanes side by side.
 // Neither part follows anything it reads: every index comes from the call's geometry, so the
 // structure pass is safe on damaged metadata and can run beside the CRC.  The last block to
 // finish decides in the specified order: metadata CRC first (WM_ERR_META_CRC), then the
 // structure (WM_ERR_STRUCT: per-chunk findings, payload offsets as the running sum of enc_len,
 // totals against the header).  A header that does not match the call stops every block at
 // once (WM_ERR_FORMAT).  A failure sets the gate that keeps the later kernels out.
+__host__ __device__ __forceinline__ uint32_t check_chunks_per_warp(uint32_t tiles_per_chunk)
+{
+    return tiles_per_chunk <= 16u ? 32u / tiles_per_chunk : 1u;
+}
+
 __global__ void __launch_bounds__(1024)
 k_decode_check(const unsigned char* __restrict__ wire, uint64_t wire_len, Geo g, Ws ws,
                const Tables* __restrict__ tab, wm_result* result, uint32_t meta_blocks, uint32_t expect_ent)
@@ -53,14 +59,12 @@ k_decode_check(const unsigned char* __restrict__ wire, uint64_t wire_len, Geo g,
     __shared__ uint32_t sHT[1024];
     __shared__ uint32_t s_dig[1024];
     __shared__ uint32_t s_wdig[4][8];
-    __shared__ unsigned long long s_warp[32];
-    __shared__ unsigned long long s_carry;
+    __shared__ unsigned long long s_part[33];
     __shared__ uint32_t s_first, s_count;
     __shared__ bool s_last;
     __shared__ int s_format_bad;
     const uint32_t lane = threadIdx.x % 32, wblk = threadIdx.x / 32;
-    sHT[threadIdx.x] = (&tab->HT[0][0])[threadIdx.x];
-    load_small_chain_tables(sG, tab);
+    if (blockIdx.x < meta_blocks) load_small_chain_tables(sG, tab);       // (the structure blocks need no tables)
     grid_dep_wait();
     grid_dep_launch();
     if (ld_volatile_u32(&ws.ctrl->gate)) return;        // leaf mode: the destination table was rejected
@@ -86,58 +90,101 @@ k_decode_check(const unsigned char* __restrict__ wire, uint64_t wire_len, Geo g,
         if (tt == 0 && s < g.n_meta_slices) ws.mdig[s] = xor8(s_wdig[team]);
     } else {
         const uint16_t* tab16 = reinterpret_cast<const uint16_t*>(wire + 64 + 16ull * g.n_chunks);
-        const uint32_t c = (blockIdx.x - meta_blocks) * 32u + wblk;
-        if (c < g.n_chunks) {
-            const uint64_t clen = chunk_len_dev(g, c);
-            const uint32_t t0 = c * g.tiles_per_chunk;
-            const uint32_t ntc = (uint32_t)((clen + kTile - 1) / kTile);
-            const uint32_t elen = *reinterpret_cast<const uint32_t*>(dir + 16ull * c + 8);
-            unsigned long long carry = 0;
-            bool ok = true, any = false, all = true;
-            for (uint32_t i0 = 0; i0 < ntc; i0 += 32) {
-                const uint32_t i = i0 + lane;
-                uint32_t len = 0;
-                bool l_ok = true, l_any = false, l_all = true, l_packs = false;
-                if (i < ntc) {
-                    const uint32_t e = tab16[t0 + i];
-                    const uint64_t tl = clen - (uint64_t)i * kTile;
-                    if (e == 0) l_all = false;
-                    else {
-                        l_any = true;
-                        if (tl < kTile) { if (e != 0xFFFFu) l_ok = false; len = (uint32_t)tl; }
-                        else if (e == 1u && zero_ok) len = 0;       // a tile of zeros: no payload
-                        else if (e == 2u && zero_ok) len = 32;      // a tile of one value: the value
-                        else if (e >= 258u && e <= 512u) { len = 32u * e; l_packs = e < 512u; }
-                        else if (expect_ent && e >= (0x8000u | 259u) && e <= (0x8000u | 511u)) len = 32u * (e & 0x7FFFu);   // ENT tile
-                        else l_ok = false;
-                    }
-                }
-                uint32_t incl = len;
-#pragma unroll
-                for (int d = 1; d < 32; d <<= 1) {
-                    uint32_t o = __shfl_up_sync(0xFFFFFFFFu, incl, d);
-                    if (lane >= (uint32_t)d) incl += o;
-                }
-                if (i < ntc) ws.rel[t0 + i] = (uint32_t)(carry + incl - len);
-                carry += __shfl_sync(0xFFFFFFFFu, incl, 31);
-                if (expect_ent && __any_sync(0xFFFFFFFFu, l_packs) && lane == 0) atomicOr(&ws.ctrl->has_pack, 1u);
-                ok = ok && __all_sync(0xFFFFFFFFu, l_ok);
-                any = any || __any_sync(0xFFFFFFFFu, l_any);
-                all = all && __all_sync(0xFFFFFFFFu, l_all);
+        // one tile entry: its payload length and what it says about its chunk
+        struct Entry { uint32_t len; bool ok, any, all, packs; };
+        auto read_entry = [&](uint32_t t, uint64_t left) {      // left: bytes of the chunk from this tile on
+            Entry r = {0u, true, false, true, false};
+            const uint32_t e = tab16[t];
+            if (e == 0) r.all = false;
+            else {
+                r.any = true;
+                if (left < kTile) { if (e != 0xFFFFu) r.ok = false; r.len = (uint32_t)left; }
+                else if (e == 1u && zero_ok) r.len = 0;       // a tile of zeros: no payload
+                else if (e == 2u && zero_ok) r.len = 32;      // a tile of one value: the value
+                else if (e >= 258u && e <= 512u) { r.len = 32u * e; r.packs = e < 512u; }
+                else if (expect_ent && e >= (0x8000u | 259u) && e <= (0x8000u | 511u)) r.len = 32u * (e & 0x7FFFu);   // ENT tile
+                else r.ok = false;
             }
-            if (any && !all) ok = false;
-            if (carry != elen) ok = false;
-            if (lane == 0) {
+            return r;
+        };
+        const uint32_t tpc = g.tiles_per_chunk, cpw = check_chunks_per_warp(tpc);
+        const uint32_t cw = ((blockIdx.x - meta_blocks) * 32u + wblk) * cpw;        // the warp's first chunk
+        bool present = false, bad = false;            // the verdict on chunk c, held by the lane that reports it
+        uint32_t c = cw;
+        if (cpw == 1u) {
+            if (c < g.n_chunks) {
+                const uint64_t clen = chunk_len_dev(g, c);
+                const uint32_t t0 = c * tpc;
+                const uint32_t ntc = (uint32_t)((clen + kTile - 1) / kTile);
+                const uint32_t elen = *reinterpret_cast<const uint32_t*>(dir + 16ull * c + 8);
+                unsigned long long carry = 0;
+                bool ok = true, any = false, all = true;
+                for (uint32_t i0 = 0; i0 < ntc; i0 += 32) {
+                    const uint32_t i = i0 + lane;
+                    Entry en = {0u, true, false, true, false};
+                    if (i < ntc) en = read_entry(t0 + i, clen - (uint64_t)i * kTile);
+                    uint32_t incl = en.len;
+#pragma unroll
+                    for (int d = 1; d < 32; d <<= 1) {
+                        uint32_t o = __shfl_up_sync(0xFFFFFFFFu, incl, d);
+                        if (lane >= (uint32_t)d) incl += o;
+                    }
+                    if (i < ntc) ws.rel[t0 + i] = (uint32_t)(carry + incl - en.len);
+                    carry += __shfl_sync(0xFFFFFFFFu, incl, 31);
+                    if (expect_ent && __any_sync(0xFFFFFFFFu, en.packs) && lane == 0) atomicOr(&ws.ctrl->has_pack, 1u);
+                    ok = ok && __all_sync(0xFFFFFFFFu, en.ok);
+                    any = any || __any_sync(0xFFFFFFFFu, en.any);
+                    all = all && __all_sync(0xFFFFFFFFu, en.all);
+                }
+                if (any && !all) ok = false;
+                if (carry != elen) ok = false;
+                present = any && lane == 0;
+                bad = !ok && lane == 0;
+                if (lane == 0) ws.cflag[c] = (any ? CF_PRESENT : 0u) | (ok ? 0u : CF_BAD3);
+            }
+        } else {
+            // lanes [k * tpc, (k + 1) * tpc) hold chunk cw + k; the lanes behind the last whole chunk idle
+            const uint32_t seg = lane / tpc, li = lane - seg * tpc;
+            c = cw + seg;
+            const bool active = seg < cpw && c < g.n_chunks;
+            const uint64_t clen = active ? chunk_len_dev(g, c) : 0ull;
+            const uint32_t ntc = (uint32_t)((clen + kTile - 1) / kTile);
+            const bool in = active && li < ntc;
+            Entry en = {0u, true, false, true, false};
+            if (in) en = read_entry(c * tpc + li, clen - (uint64_t)li * kTile);
+            uint32_t incl = en.len;
+#pragma unroll
+            for (int d = 1; d < 16; d <<= 1) {           // (a lane adds from inside its own chunk only)
+                const uint32_t o = __shfl_up_sync(0xFFFFFFFFu, incl, d);
+                if (li >= (uint32_t)d) incl += o;
+            }
+            if (in) ws.rel[c * tpc + li] = incl - en.len;
+            const uint32_t tot = __shfl_sync(0xFFFFFFFFu, incl, min(seg * tpc + tpc - 1u, 31u));      // (lanes behind the chunk's last tile add 0)
+            const uint32_t segmask = active ? ((1u << tpc) - 1u) << (seg * tpc) : 0u;
+            const bool ok_all = (__ballot_sync(0xFFFFFFFFu, en.ok) & segmask) == segmask;
+            const bool any = (__ballot_sync(0xFFFFFFFFu, en.any) & segmask) != 0u;
+            const bool all = (__ballot_sync(0xFFFFFFFFu, in && !en.all) & segmask) == 0u;
+            if (expect_ent && __any_sync(0xFFFFFFFFu, en.packs) && lane == 0) atomicOr(&ws.ctrl->has_pack, 1u);
+            if (active && li == 0) {
+                const uint32_t elen = *reinterpret_cast<const uint32_t*>(dir + 16ull * c + 8);
+                const bool ok = ok_all && !(any && !all) && tot == elen;
+                present = any;
+                bad = !ok;
                 ws.cflag[c] = (any ? CF_PRESENT : 0u) | (ok ? 0u : CF_BAD3);
-                if (!ok) { atomicMin(&ws.ctrl->bad3_first, c); atomicAdd(&ws.ctrl->bad3_count, 1u); }
-                if (any) ws.plist[atomicAdd(&ws.ctrl->n_present, 1u)] = c;     // (the present chunks, in any order: k_decode claims their tiles only)
             }
         }
+        // (the present chunks, in any order: k_decode claims their tiles only; one count per warp)
+        const uint32_t pres = __ballot_sync(0xFFFFFFFFu, present);
+        uint32_t slot0 = 0;
+        if (lane == 0 && pres) slot0 = atomicAdd(&ws.ctrl->n_present, (uint32_t)__popc(pres));
+        slot0 = __shfl_sync(0xFFFFFFFFu, slot0, 0);
+        if (present) ws.plist[slot0 + __popc(pres & ((1u << lane) - 1u))] = c;
+        if (bad) { atomicMin(&ws.ctrl->bad3_first, c); atomicAdd(&ws.ctrl->bad3_count, 1u); }
     }
     __threadfence();
     __syncthreads();
     if (threadIdx.x == 0) {
-        s_carry = 0; s_first = 0xFFFFFFFFu; s_count = 0;
+        s_first = 0xFFFFFFFFu; s_count = 0;
         __threadfence();
         s_last = atomicAdd(&ws.ctrl->done_b, 1u) == gridDim.x - 1;
     }
@@ -146,6 +193,7 @@ k_decode_check(const unsigned char* __restrict__ wire, uint64_t wire_len, Geo g,
     __threadfence();
 
     // ---- the last block: metadata CRC first
+    sHT[threadIdx.x] = (&tab->HT[0][0])[threadIdx.x];
     const uint32_t crc = fold_meta_digests(g, ws, sHT, s_dig);
     if (threadIdx.x == 0) {
         const uint32_t* h = reinterpret_cast<const uint32_t*>(wire);
@@ -169,25 +217,17 @@ k_decode_check(const unsigned char* __restrict__ wire, uint64_t wire_len, Geo g,
     __syncthreads();
     if (s_format_bad) return;
 
-    // ---- then the structure across chunks
-    for (uint32_t base = 0; base < g.n_chunks; base += 1024) {
-        const uint32_t cc = base + threadIdx.x;
-        unsigned long long len = 0, po = 0;
-        if (cc < g.n_chunks) {
-            po = *reinterpret_cast<const unsigned long long*>(dir + 16ull * cc);
-            len = *reinterpret_cast<const uint32_t*>(dir + 16ull * cc + 8);
-        }
-        unsigned long long incl = len;
-#pragma unroll
-        for (int d = 1; d < 32; d <<= 1) {
-            unsigned long long o = __shfl_up_sync(0xFFFFFFFFu, incl, d);
-            if (lane >= (uint32_t)d) incl += o;
-        }
-        if (lane == 31) s_warp[wblk] = incl;
-        __syncthreads();
-        unsigned long long before = s_carry;
-        for (uint32_t w2 = 0; w2 < wblk; w2++) before += s_warp[w2];
-        if (cc < g.n_chunks && po != before + incl - len) {
+    // ---- then the structure across chunks: every payload_off is the sum of the lengths before
+    // it (every thread a run of consecutive chunks, one prefix over the threads' sums)
+    const uint32_t per = (g.n_chunks + 1023u) / 1024u;
+    const uint32_t c0 = min(threadIdx.x * per, g.n_chunks), c1 = min(c0 + per, g.n_chunks);
+    unsigned long long mine = 0;
+    for (uint32_t cc = c0; cc < c1; cc++) mine += *reinterpret_cast<const uint32_t*>(dir + 16ull * cc + 8);
+    unsigned long long payload_sum;
+    unsigned long long run = block_prefix(mine, s_part, payload_sum);
+    for (uint32_t cc = c0; cc < c1; cc++) {
+        const unsigned long long po = *reinterpret_cast<const unsigned long long*>(dir + 16ull * cc);
+        if (po != run) {
             // a chunk already counted by the per-chunk pass must not be counted twice
             const uint32_t fl = ld_volatile_u32(&ws.cflag[cc]);
             if (!(fl & CF_BAD3)) {
@@ -196,18 +236,13 @@ k_decode_check(const unsigned char* __restrict__ wire, uint64_t wire_len, Geo g,
                 atomicAdd(&s_count, 1u);
             }
         }
-        __syncthreads();
-        if (threadIdx.x == 0) {
-            unsigned long long tot = 0;
-            for (int w2 = 0; w2 < 32; w2++) tot += s_warp[w2];
-            s_carry += tot;
-        }
-        __syncthreads();
+        run += *reinterpret_cast<const uint32_t*>(dir + 16ull * cc + 8);
     }
+    __syncthreads();
     if (threadIdx.x == 0) {
         uint32_t first = min(s_first, ld_volatile_u32(&ws.ctrl->bad3_first));
         uint32_t count = s_count + ld_volatile_u32(&ws.ctrl->bad3_count);
-        if (count == 0 && (s_carry != ws.ctrl->payload_total ||
+        if (count == 0 && (payload_sum != ws.ctrl->payload_total ||
                            ld_volatile_u32(&ws.ctrl->n_present) != ws.ctrl->hdr_n_present)) {
             first = 0; count = 1;
         }

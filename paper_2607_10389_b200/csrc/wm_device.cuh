@@ -401,4 +401,36 @@ __device__ __forceinline__ uint32_t crc_bytewise(const uint32_t* T0, const unsig
     return ~crc;
 }
 
+// Exclusive prefix of `v` over the threads of a 1024-thread block, in thread order, and the
+// block's total.  s_part: 33 values of shared memory.  Block-wide (two barriers); one use per
+// kernel, or a barrier between uses.  The kernels that scan a per-chunk array give every thread
+// a run of consecutive chunks, so one such prefix does for any number of chunks.
+template <typename T>
+__device__ __forceinline__ T block_prefix(T v, T* s_part, T& total)
+{
+    const uint32_t lane = threadIdx.x % 32, warp = threadIdx.x / 32;
+    T incl = v;
+#pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        const T o = __shfl_up_sync(0xFFFFFFFFu, incl, d);
+        if (lane >= (uint32_t)d) incl += o;
+    }
+    if (lane == 31) s_part[warp] = incl;
+    __syncthreads();
+    if (warp == 0) {
+        const T p = s_part[lane];
+        T pi = p;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const T o = __shfl_up_sync(0xFFFFFFFFu, pi, d);
+            if (lane >= (uint32_t)d) pi += o;
+        }
+        s_part[lane] = pi - p;
+        if (lane == 31) s_part[32] = pi;
+    }
+    __syncthreads();
+    total = s_part[32];
+    return s_part[warp] + incl - v;
+}
+
 }  // namespace wm

@@ -74,34 +74,23 @@ k_diff(const unsigned char* __restrict__ cache, const unsigned char* __restrict_
     }
 }
 
-// Ascending index list of dirty chunks and their count (one block, ballot + popc scan).
+// Ascending index list of dirty chunks and their count: one block, every thread a run of
+// consecutive chunks, one prefix over the threads' counts.
 __global__ void __launch_bounds__(1024)
 k_diff_compact(Geo g, const uint8_t* __restrict__ dirty, uint32_t* __restrict__ idx_out, uint32_t* __restrict__ n_out)
 {
-    __shared__ uint32_t s_warp[32];
-    __shared__ uint32_t s_carry;
-    const uint32_t lane = threadIdx.x % 32, warp = threadIdx.x / 32;
+    __shared__ uint32_t s_part[33];
     grid_dep_wait();
-    if (threadIdx.x == 0) s_carry = 0;
-    __syncthreads();
-    for (uint32_t base = 0; base < g.n_chunks; base += 1024) {
-        const uint32_t c = base + threadIdx.x;
-        const bool d = c < g.n_chunks && dirty[c] != 0;
-        const uint32_t bal = __ballot_sync(0xFFFFFFFFu, d);
-        if (lane == 0) s_warp[warp] = __popc(bal);
-        __syncthreads();
-        uint32_t before = s_carry;
-        for (uint32_t w2 = 0; w2 < warp; w2++) before += s_warp[w2];
-        if (d && idx_out) idx_out[before + __popc(bal & ((1u << lane) - 1u))] = c;
-        __syncthreads();
-        if (threadIdx.x == 0) {
-            uint32_t tot = 0;
-            for (int w2 = 0; w2 < 32; w2++) tot += s_warp[w2];
-            s_carry += tot;
-        }
-        __syncthreads();
-    }
-    if (threadIdx.x == 0) *n_out = s_carry;
+    const uint32_t per = (g.n_chunks + 1023u) / 1024u;
+    const uint32_t c0 = min(threadIdx.x * per, g.n_chunks), c1 = min(c0 + per, g.n_chunks);
+    uint32_t mine = 0;
+    for (uint32_t c = c0; c < c1; c++) mine += dirty[c] != 0 ? 1u : 0u;
+    uint32_t total;
+    uint32_t at = block_prefix(mine, s_part, total);
+    if (idx_out)
+        for (uint32_t c = c0; c < c1; c++)
+            if (dirty[c] != 0) idx_out[at++] = c;
+    if (threadIdx.x == 0) *n_out = total;
 }
 
 }  // namespace wm

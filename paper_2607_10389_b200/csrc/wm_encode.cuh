@@ -10,8 +10,8 @@ namespace wm {
 // Clears the control block and the placement words, zero-fills the padding behind the tile
 // table.  With a dirty mask the main kernel claims the tiles of the present chunks only, so
 // here the table entries of all tiles start at 0 (absent) and the first block lists the present
-// chunks in ascending order (ws.plist, ballot + popc scan) and leaves the number of tiles to
-// claim in the control block.
+// chunks in ascending order (ws.plist; every thread a run of consecutive chunks, one prefix over
+// the threads' counts) and leaves the number of tiles to claim in the control block.
 __global__ void __launch_bounds__(1024)
 k_encode_init(Geo g, Ws ws, unsigned char* wire, const uint8_t* __restrict__ dirty)
 {
@@ -31,31 +31,18 @@ k_encode_init(Geo g, Ws ws, unsigned char* wire, const uint8_t* __restrict__ dir
     uint16_t* tile_tab = reinterpret_cast<uint16_t*>(wire + 64 + 16ull * g.n_chunks);
     for (uint64_t t = i; t < g.n_tiles; t += stride) tile_tab[t] = 0;
     if (blockIdx.x != 0) return;
-    __shared__ uint32_t s_warp[32];
-    __shared__ uint32_t s_carry;
-    const uint32_t lane = threadIdx.x % 32, warp = threadIdx.x / 32;
-    if (threadIdx.x == 0) s_carry = 0;
-    __syncthreads();
-    for (uint32_t base = 0; base < g.n_chunks; base += 1024) {
-        const uint32_t c = base + threadIdx.x;
-        const bool d = c < g.n_chunks && dirty[c] != 0;
-        const uint32_t bal = __ballot_sync(0xFFFFFFFFu, d);
-        if (lane == 0) s_warp[warp] = __popc(bal);
-        __syncthreads();
-        uint32_t before = s_carry;
-        for (uint32_t w2 = 0; w2 < warp; w2++) before += s_warp[w2];
-        if (d) ws.plist[before + __popc(bal & ((1u << lane) - 1u))] = c;
-        __syncthreads();
-        if (threadIdx.x == 0) {
-            uint32_t tot = 0;
-            for (int w2 = 0; w2 < 32; w2++) tot += s_warp[w2];
-            s_carry += tot;
-        }
-        __syncthreads();
-    }
+    __shared__ uint32_t s_part[33];
+    const uint32_t per = (g.n_chunks + 1023u) / 1024u;
+    const uint32_t c0 = min(threadIdx.x * per, g.n_chunks), c1 = min(c0 + per, g.n_chunks);
+    uint32_t mine = 0;
+    for (uint32_t c = c0; c < c1; c++) mine += dirty[c] != 0 ? 1u : 0u;
+    uint32_t n_listed;
+    uint32_t at = block_prefix(mine, s_part, n_listed);
+    for (uint32_t c = c0; c < c1; c++)
+        if (dirty[c] != 0) ws.plist[at++] = c;
     if (threadIdx.x == 0) {
         // every present chunk has tiles_per_chunk tiles, except the cache's last chunk
-        const uint32_t np = s_carry;
+        const uint32_t np = n_listed;
         uint32_t nt = np * g.tiles_per_chunk;
         if (np && dirty[g.n_chunks - 1]) nt -= g.tiles_per_chunk - (g.n_tiles - (g.n_chunks - 1) * g.tiles_per_chunk);
         ws.ctrl->n_list = np;

@@ -495,8 +495,9 @@ static wm_status decode_any(const void* wire, uint64_t wire_len, void* dst, cons
     }
     // a wire shorter than the metadata is rejected by the header check before anything else is read
     const uint32_t meta_blocks = (g.n_meta_slices + 3) / 4;
+    const uint32_t chunks_per_block = 32u * check_chunks_per_warp(g.tiles_per_chunk);
     const bool ent = (options & WM_OPT_ENTROPY) != 0;      // the option says which kind of image the call expects
-    launch_after(k_decode_check, meta_blocks + (g.n_chunks + 31) / 32, 1024, 0, s, w, wire_len, g, ws, ds->tables, result, meta_blocks,
+    launch_after(k_decode_check, meta_blocks + (g.n_chunks + chunks_per_block - 1) / chunks_per_block, 1024, 0, s, w, wire_len, g, ws, ds->tables, result, meta_blocks,
                  ent ? 1u : 0u);
     const uint32_t need = (g.n_tiles + kTeamsPlain - 1) / kTeamsPlain;
     uint32_t grid = need < (uint32_t)ds->sm_count ? need : (uint32_t)ds->sm_count;
