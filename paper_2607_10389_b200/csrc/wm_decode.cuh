@@ -218,16 +218,32 @@ k_decode_check(const unsigned char* __restrict__ wire, uint64_t wire_len, Geo g,
     if (s_format_bad) return;
 
     // ---- then the structure across chunks: every payload_off is the sum of the lengths before
-    // it (every thread a run of consecutive chunks, one prefix over the threads' sums)
-    const uint32_t per = (g.n_chunks + 1023u) / 1024u;
-    const uint32_t c0 = min(threadIdx.x * per, g.n_chunks), c1 = min(c0 + per, g.n_chunks);
+    // it.  Every warp takes a run of consecutive chunks, 32 at a time (consecutive lanes read
+    // consecutive directory entries); one prefix over the warps' sums gives each run its start.
+    const uint32_t per_w = (g.n_chunks + 31u) / 32u;
+    const uint32_t w0 = min(wblk * per_w, g.n_chunks), w1 = min(w0 + per_w, g.n_chunks);
     unsigned long long mine = 0;
-    for (uint32_t cc = c0; cc < c1; cc++) mine += *reinterpret_cast<const uint32_t*>(dir + 16ull * cc + 8);
+    for (uint32_t cc = w0 + lane; cc < w1; cc += 32u) mine += *reinterpret_cast<const uint32_t*>(dir + 16ull * cc + 8);
+#pragma unroll
+    for (int d = 16; d >= 1; d >>= 1) mine += __shfl_xor_sync(0xFFFFFFFFu, mine, d);      // the warp's sum, in every lane
     unsigned long long payload_sum;
-    unsigned long long run = block_prefix(mine, s_part, payload_sum);
-    for (uint32_t cc = c0; cc < c1; cc++) {
-        const unsigned long long po = *reinterpret_cast<const unsigned long long*>(dir + 16ull * cc);
-        if (po != run) {
+    unsigned long long run = block_prefix(lane == 0 ? mine : 0ull, s_part, payload_sum);  // lane 0: where the warp's run starts
+    run = __shfl_sync(0xFFFFFFFFu, run, 0);
+    for (uint32_t base = w0; base < w1; base += 32u) {
+        const uint32_t cc = base + lane;
+        unsigned long long len = 0, po = 0;
+        if (cc < w1) {
+            const uint4 en = *reinterpret_cast<const uint4*>(dir + 16ull * cc);
+            po = en.x | ((unsigned long long)en.y << 32);
+            len = en.z;
+        }
+        unsigned long long incl = len;
+#pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const unsigned long long o = __shfl_up_sync(0xFFFFFFFFu, incl, d);
+            if (lane >= (uint32_t)d) incl += o;
+        }
+        if (cc < w1 && po != run + incl - len) {
             // a chunk already counted by the per-chunk pass must not be counted twice
             const uint32_t fl = ld_volatile_u32(&ws.cflag[cc]);
             if (!(fl & CF_BAD3)) {
@@ -236,7 +252,7 @@ k_decode_check(const unsigned char* __restrict__ wire, uint64_t wire_len, Geo g,
                 atomicAdd(&s_count, 1u);
             }
         }
-        run += *reinterpret_cast<const uint32_t*>(dir + 16ull * cc + 8);
+        run += __shfl_sync(0xFFFFFFFFu, incl, 31);
     }
     __syncthreads();
     if (threadIdx.x == 0) {
@@ -796,8 +812,23 @@ k_decode_finish(const unsigned char* __restrict__ wire, uint64_t wire_len, Geo g
     }
     __syncthreads();
     if (s_status == WM_OK) {
-        for (uint32_t i = threadIdx.x; i < g.n_chunks; i += blockDim.x)
-            if (ws.cflag[i] & CF_PRESENT) dst_crc[i] = *reinterpret_cast<const uint32_t*>(dir + 16ull * i + 12);
+        // (both loads of a chunk are issued before either is looked at, eight chunks at a time:
+        // a cache of many small chunks would otherwise pay two round trips to L2 per chunk, in a row)
+        for (uint32_t base = threadIdx.x; base < g.n_chunks; base += 8u * blockDim.x) {
+            uint32_t fl[8], want[8];
+#pragma unroll
+            for (int k = 0; k < 8; k++) {
+                const uint32_t i = base + k * blockDim.x;
+                fl[k] = 0;
+                if (i < g.n_chunks) {
+                    fl[k] = ws.cflag[i];
+                    want[k] = *reinterpret_cast<const uint32_t*>(dir + 16ull * i + 12);
+                }
+            }
+#pragma unroll
+            for (int k = 0; k < 8; k++)
+                if (fl[k] & CF_PRESENT) dst_crc[base + k * blockDim.x] = want[k];
+        }
     }
 }
 
