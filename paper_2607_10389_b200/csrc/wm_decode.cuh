@@ -44,7 +44,10 @@ __device__ __forceinline__ void fill_result(wm_result* result, const Ctrl* ctrl,
 // structure pass is safe on damaged metadata and can run beside the CRC.  The last block to
 // finish decides in the specified order: metadata CRC first (WM_ERR_META_CRC), then the
 // structure (WM_ERR_STRUCT: per-chunk findings, payload offsets as the running sum of enc_len,
-// totals against the header).  A header that does not match the call stops every block at
+// totals against the header).  The offsets are the running sum exactly when the first is 0 and
+// every other one is its predecessor's plus that one's enc_len, which the structure pass checks
+// chunk by chunk as it goes; only when that fails somewhere does the last block walk the whole
+// directory to find which chunks differ from the running sum (the specified count).  A header that does not match the call stops every block at
 // once (WM_ERR_FORMAT).  A failure sets the gate that keeps the later kernels out.
 __host__ __device__ __forceinline__ uint32_t check_chunks_per_warp(uint32_t tiles_per_chunk)
 {
@@ -107,6 +110,13 @@ k_decode_check(const unsigned char* __restrict__ wire, uint64_t wire_len, Geo g,
             }
             return r;
         };
+        // chunk cc's offset against its predecessor's (one lane per chunk)
+        auto offset_follows = [&](uint32_t cc) {
+            const unsigned long long po = *reinterpret_cast<const unsigned long long*>(dir + 16ull * cc);
+            if (cc == 0) return po == 0ull;
+            const uint4 pr = *reinterpret_cast<const uint4*>(dir + 16ull * (cc - 1u));
+            return po == (pr.x | ((unsigned long long)pr.y << 32)) + pr.z;
+        };
         const uint32_t tpc = g.tiles_per_chunk, cpw = check_chunks_per_warp(tpc);
         const uint32_t cw = ((blockIdx.x - meta_blocks) * 32u + wblk) * cpw;        // the warp's first chunk
         bool present = false, bad = false;            // the verdict on chunk c, held by the lane that reports it
@@ -140,7 +150,10 @@ k_decode_check(const unsigned char* __restrict__ wire, uint64_t wire_len, Geo g,
                 if (carry != elen) ok = false;
                 present = any && lane == 0;
                 bad = !ok && lane == 0;
-                if (lane == 0) ws.cflag[c] = (any ? CF_PRESENT : 0u) | (ok ? 0u : CF_BAD3);
+                if (lane == 0) {
+                    ws.cflag[c] = (any ? CF_PRESENT : 0u) | (ok ? 0u : CF_BAD3);
+                    if (!offset_follows(c)) ws.ctrl->off_bad = 1u;
+                }
             }
         } else {
             // lanes [k * tpc, (k + 1) * tpc) hold chunk cw + k; the lanes behind the last whole chunk idle
@@ -171,6 +184,7 @@ k_decode_check(const unsigned char* __restrict__ wire, uint64_t wire_len, Geo g,
                 present = any;
                 bad = !ok;
                 ws.cflag[c] = (any ? CF_PRESENT : 0u) | (ok ? 0u : CF_BAD3);
+                if (!offset_follows(c)) ws.ctrl->off_bad = 1u;
             }
         }
         // (the present chunks, in any order: k_decode claims their tiles only; one count per warp)
@@ -217,42 +231,53 @@ k_decode_check(const unsigned char* __restrict__ wire, uint64_t wire_len, Geo g,
     __syncthreads();
     if (s_format_bad) return;
 
-    // ---- then the structure across chunks: every payload_off is the sum of the lengths before
-    // it.  Every warp takes a run of consecutive chunks, 32 at a time (consecutive lanes read
+    // ---- then the structure across chunks.  Every offset followed from its predecessor: the
+    // offsets are the running sum, and the payload's length is the last chunk's end.  Otherwise
+    // the chunks whose payload_off is not the sum of the lengths before it are found and counted:
+    // every warp takes a run of consecutive chunks, 32 at a time (consecutive lanes read
     // consecutive directory entries); one prefix over the warps' sums gives each run its start.
-    const uint32_t per_w = (g.n_chunks + 31u) / 32u;
-    const uint32_t w0 = min(wblk * per_w, g.n_chunks), w1 = min(w0 + per_w, g.n_chunks);
-    unsigned long long mine = 0;
-    for (uint32_t cc = w0 + lane; cc < w1; cc += 32u) mine += *reinterpret_cast<const uint32_t*>(dir + 16ull * cc + 8);
-#pragma unroll
-    for (int d = 16; d >= 1; d >>= 1) mine += __shfl_xor_sync(0xFFFFFFFFu, mine, d);      // the warp's sum, in every lane
     unsigned long long payload_sum;
-    unsigned long long run = block_prefix(lane == 0 ? mine : 0ull, s_part, payload_sum);  // lane 0: where the warp's run starts
-    run = __shfl_sync(0xFFFFFFFFu, run, 0);
-    for (uint32_t base = w0; base < w1; base += 32u) {
-        const uint32_t cc = base + lane;
-        unsigned long long len = 0, po = 0;
-        if (cc < w1) {
-            const uint4 en = *reinterpret_cast<const uint4*>(dir + 16ull * cc);
-            po = en.x | ((unsigned long long)en.y << 32);
-            len = en.z;
-        }
-        unsigned long long incl = len;
+    if (!ld_volatile_u32(&ws.ctrl->off_bad)) {       // (block-uniform)
+        const uint4 en = *reinterpret_cast<const uint4*>(dir + 16ull * (g.n_chunks - 1u));
+        payload_sum = (en.x | ((unsigned long long)en.y << 32)) + en.z;
+    } else {
+        const uint32_t per_w = (g.n_chunks + 31u) / 32u;
+        const uint32_t w0 = min(wblk * per_w, g.n_chunks), w1 = min(w0 + per_w, g.n_chunks);
+        unsigned long long mine = 0;
+        for (uint32_t cc = w0 + lane; cc < w1; cc += 32u) mine += *reinterpret_cast<const uint32_t*>(dir + 16ull * cc + 8);
 #pragma unroll
-        for (int d = 1; d < 32; d <<= 1) {
-            const unsigned long long o = __shfl_up_sync(0xFFFFFFFFu, incl, d);
-            if (lane >= (uint32_t)d) incl += o;
-        }
-        if (cc < w1 && po != run + incl - len) {
-            // a chunk already counted by the per-chunk pass must not be counted twice
-            const uint32_t fl = ld_volatile_u32(&ws.cflag[cc]);
-            if (!(fl & CF_BAD3)) {
-                ws.cflag[cc] = fl | CF_BAD3;
-                atomicMin(&s_first, cc);
-                atomicAdd(&s_count, 1u);
+        for (int d = 16; d >= 1; d >>= 1) mine += __shfl_xor_sync(0xFFFFFFFFu, mine, d);      // the warp's sum, in every lane
+        unsigned long long run = block_prefix(lane == 0 ? mine : 0ull, s_part, payload_sum);  // lane 0: where the warp's run starts
+        run = __shfl_sync(0xFFFFFFFFu, run, 0);
+        for (uint32_t base = w0; base < w1; base += 128u) {
+            uint4 en[4];                   // (four rounds' entries asked for at once: one round trip to L2, not four)
+#pragma unroll
+            for (int k = 0; k < 4; k++) {
+                const uint32_t cc = base + 32u * k + lane;
+                en[k] = cc < w1 ? *reinterpret_cast<const uint4*>(dir + 16ull * cc) : make_uint4(0u, 0u, 0u, 0u);
+            }
+#pragma unroll
+            for (int k = 0; k < 4; k++) {
+                const uint32_t cc = base + 32u * k + lane;
+                const unsigned long long po = en[k].x | ((unsigned long long)en[k].y << 32), len = en[k].z;
+                unsigned long long incl = len;
+#pragma unroll
+                for (int d = 1; d < 32; d <<= 1) {
+                    const unsigned long long o = __shfl_up_sync(0xFFFFFFFFu, incl, d);
+                    if (lane >= (uint32_t)d) incl += o;
+                }
+                if (cc < w1 && po != run + incl - len) {
+                    // a chunk already counted by the per-chunk pass must not be counted twice
+                    const uint32_t fl = ld_volatile_u32(&ws.cflag[cc]);
+                    if (!(fl & CF_BAD3)) {
+                        ws.cflag[cc] = fl | CF_BAD3;
+                        atomicMin(&s_first, cc);
+                        atomicAdd(&s_count, 1u);
+                    }
+                }
+                run += __shfl_sync(0xFFFFFFFFu, incl, 31);
             }
         }
-        run += __shfl_sync(0xFFFFFFFFu, incl, 31);
     }
     __syncthreads();
     if (threadIdx.x == 0) {

@@ -63,7 +63,8 @@ struct Ctrl {                 // first 256 bytes of the workspace
     uint32_t n_walked;        // leaf mode: tiles that go through the side buffer (see k_leaf_map)
     uint32_t n_list;          // masked images: present chunks listed in plist
     uint32_t n_tickets;       // tiles the main kernel has to claim (masked: those of the listed chunks only)
-    uint32_t pad[37];
+    uint32_t off_bad;         // decode: some chunk's payload_off is not its predecessor's plus that one's enc_len
+    uint32_t pad[36];
 };
 static_assert(sizeof(Ctrl) == 256, "control block is 256 bytes");
 
