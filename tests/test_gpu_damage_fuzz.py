@@ -29,7 +29,7 @@ def _image(option, seed):
 def damage(wire, n, chunk, rng):
     w = wire.copy()
     me = oracle.meta_end(n, chunk)
-    kind = rng.integers(0, 6)
+    kind = rng.integers(0, 8)
     if kind == 0:                                   # a bit anywhere
         i = int(rng.integers(0, w.size)); w[i] ^= 1 << int(rng.integers(0, 8))
     elif kind == 1:                                 # a bit in the metadata
@@ -45,6 +45,17 @@ def damage(wire, n, chunk, rng):
         nc = oracle.num_chunks(n, chunk)
         t = int(rng.integers(0, oracle.num_tiles(n)))
         struct.pack_into("<H", w, 64 + 16 * nc + 2 * t, int(rng.choice([0, 1, 2, 258, 300, 512, 0x8000 | 300, 0x8000 | 511, 0xFFFF, 7])))
+        z = w[:me].copy(); z[52:56] = 0
+        w[52:56] = np.frombuffer(struct.pack("<I", oracle.crc32c(z)), dtype=np.uint8)
+    elif kind in (5, 6):                            # a directory field altered (an offset, or a length: every later
+        import struct                               # chunk is then off the running sum), metadata CRC made right again
+        c = int(rng.integers(0, oracle.num_chunks(n, chunk)))
+        if kind == 5:
+            po = struct.unpack_from("<Q", w, 64 + 16 * c)[0]
+            struct.pack_into("<Q", w, 64 + 16 * c, po + 32 * int(rng.integers(1, 5)))
+        else:
+            el = struct.unpack_from("<I", w, 64 + 16 * c + 8)[0]
+            struct.pack_into("<I", w, 64 + 16 * c + 8, max(0, el + 32 * int(rng.integers(-2, 3))))
         z = w[:me].copy(); z[52:56] = 0
         w[52:56] = np.frombuffer(struct.pack("<I", oracle.crc32c(z)), dtype=np.uint8)
     else:                                           # truncated or extended
