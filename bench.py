@@ -983,34 +983,41 @@ def main():
         host_cache.copy_(cur)
         host_wire = torch.empty(W, dtype=torch.uint8, pin_memory=True)
         host_res = torch.empty(80, dtype=torch.uint8, pin_memory=True)
-        e_steps = max(4, min(args.steps, 8))
-        # Two sets of device buffers and two streams: while the copy-out stream reads step k's wire
-        # image and result records back to the host, the work stream already copies step k+1's
-        # cache in and runs the path on it.  Every step still pays its own host->device copy of
-        # the whole cache and its own device->host copy of the image inside the timed region.
-        work, out = torch.cuda.Stream(), torch.cuda.Stream()
+        e_steps = max(4, min(args.steps, 24))
+        # Two sets of device buffers and three streams: copy-in, the path, copy-out.  While step k
+        # runs on one set, step k+1's cache is already coming in on the other and step k-1's wire
+        # image and result records are going out.  Every step still pays its own host->device copy
+        # of the whole cache and its own device->host copy of the image inside the timed region.
+        cin, work, out = torch.cuda.Stream(), torch.cuda.Stream(), torch.cuda.Stream()
         curs = [cur, torch.empty_like(cur)]
         wires = [wire, torch.empty_like(wire)]
         res_es = [res_e, wm.new_result(dev)]
         res_ds = [res_d, wm.new_result(dev)]
         host_wires = [host_wire, torch.empty(W, dtype=torch.uint8, pin_memory=True)]
         host_ress = [host_res, torch.empty(80, dtype=torch.uint8, pin_memory=True)]
-        done_out = [None, None]
+        done_out = [None, None]            # the set's last image has left the device
+        done_work = [None, None]           # the set's last pass over its cache has ended
 
         def e2e_step(i):
             b = i & 1
-            with torch.cuda.stream(work):
-                if done_out[b] is not None:
-                    work.wait_event(done_out[b])           # the set's last image has left the device
+            with torch.cuda.stream(cin):
+                if done_work[b] is not None:
+                    cin.wait_event(done_work[b])
                 curs[b].copy_(host_cache, non_blocking=True)
+                arrived = torch.cuda.Event()
+                arrived.record(cin)
+            with torch.cuda.stream(work):
+                work.wait_event(arrived)
+                if done_out[b] is not None:
+                    work.wait_event(done_out[b])
                 wm.wm_checksum(curs[b], C, crc_a, ws, stream=work)
                 wm.wm_dirty_diff(curs[b], prev, C, dirty, dirty_idx, n_dirty, ws, stream=work)
                 wm.wm_encode(curs[b], C, None, crc_b, wires[b], ws, res_es[b], stream=work)
                 wm.wm_decode_verify(wires[b], W, shadow, C, crc_dst, ws, res_ds[b], stream=work)
-                ready = torch.cuda.Event()
-                ready.record(work)
+                done_work[b] = torch.cuda.Event()
+                done_work[b].record(work)
             with torch.cuda.stream(out):
-                out.wait_event(ready)
+                out.wait_event(done_work[b])
                 host_wires[b].copy_(wires[b][:W], non_blocking=True)
                 host_ress[b][:40].copy_(res_es[b], non_blocking=True)
                 host_ress[b][40:].copy_(res_ds[b], non_blocking=True)
@@ -1021,10 +1028,10 @@ def main():
         e2e_step(0)
         e2e_step(1)
         barrier()
-        done_out = [None, None]
+        done_out, done_work = [None, None], [None, None]
         t0 = torch.cuda.Event(enable_timing=True)
         t1 = torch.cuda.Event(enable_timing=True)
-        t0.record(work)
+        t0.record(cin)
         for i in range(e_steps):
             e2e_step(i)
         with torch.cuda.stream(out):
@@ -1039,7 +1046,7 @@ def main():
         e_ms = max_over_ranks(t0.elapsed_time(t1)) / e_steps
         e2e = {"value": group.aggregate_gbs(N, e_ms), "unit": "GB/s", "h2d_bytes_per_step": N,
                "d2h_bytes_per_step": W + 80, "steps": e_steps, "ms_per_step": e_ms,
-               "note": "two buffer sets, two streams: step k's copy-out overlaps step k+1's copy-in and compute"}
+               "note": "two buffer sets, three streams: step k runs while step k+1's cache comes in and step k-1's image goes out"}
 
     # the same step captured once in a CUDA graph and replayed (the calls never allocate or
     # synchronise): what is left of the host's launch work, which matters for small caches
