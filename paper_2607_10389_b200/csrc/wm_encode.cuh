@@ -394,10 +394,11 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
     // that shares its scheduler with busy ones gets too few issue slots to keep up).
     __shared__ uint32_t s_scanner;
     __shared__ uint32_t s_tmem;
-    __shared__ uint32_t s_ent[16];     // ENT: codeword | length << 16 by slot (one bank each: no conflicts)
+    __shared__ uint2 s_ent[16];        // ENT, by slot: x = codeword | length << 16, y = 1 << length
     __shared__ unsigned char s_len8[16];   // ENT: length by slot (bytes: the index needs no scaling)
     if (ENT && threadIdx.x < 11u) {
-        s_ent[threadIdx.x] = (threadIdx.x == 10u ? 0xFFFFu : ent_word(threadIdx.x, 0u)) | (ent_length(threadIdx.x) << 16);
+        s_ent[threadIdx.x] = make_uint2((threadIdx.x == 10u ? 0xFFFFu : ent_word(threadIdx.x, 0u)) | (ent_length(threadIdx.x) << 16),
+                                        1u << ent_length(threadIdx.x));
         s_len8[threadIdx.x] = (unsigned char)ent_length(threadIdx.x);
     }
     Smem S = setup_smem(smem, tab);
@@ -700,20 +701,26 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
                 const uint32_t start = incl - 64u - nb8;
                 unsigned char* const w_dst = dst + 8512u + 4u * before;
                 // acc: the stream's bits from the last word boundary on, n of them valid (the first n
-                // of the lane's first word belong to the lane before it).  Words go out as they fill
-                // up, except the lane's first one, which is held back until the lane before has handed
-                // over the bits it left in it.
+                // of the lane's first word belong to the lane before it).  Two codewords are joined
+                // first (32 bits at most) and go in together; both shifts are multiplications by a
+                // power of two from the table or from n (one multiply-add each, on the pipe that has
+                // little else to do here, where the shifts and ORs would queue up with everything
+                // else).  Words go out as they fill up, except the lane's first one, which is held
+                // back until the lane before has handed over the bits it left in it.
                 unsigned long long acc = 0;
                 uint32_t n = start & 31u, wp = start >> 5, w_first = 0;
                 bool have_first = false;
 #pragma unroll
-                for (int i = 0; i < 32; i++) {
-                    const uint32_t E = (i & 1) ? d[i >> 1] >> 24 : __byte_perm(d[i >> 1], 0u, 0x4441);
-                    const uint32_t cw = s_ent[ent_slot(E, anchor)];
+                for (int i = 0; i < 16; i++) {
+                    const uint32_t E0 = __byte_perm(d[i], 0u, 0x4441), E1 = d[i] >> 24;
+                    const uint2 t0 = s_ent[ent_slot(E0, anchor)], t1 = s_ent[ent_slot(E1, anchor)];
                     // (the table's escape entry is 0xFFFF: the AND lets the exponent through there only)
-                    acc |= (unsigned long long)(cw & ((E << 8) | 0xFFu) & 0xFFFFu) << n;
-                    n += cw >> 16;
-                    if ((i & 1) && n >= 32u) {             // (two codewords are 32 bits at most: one word per pair)
+                    const uint32_t c0 = t0.x & __byte_perm(E0, 0xFFu, 0x4404) & 0xFFFFu;
+                    const uint32_t c1 = t1.x & __byte_perm(E1, 0xFFu, 0x4404) & 0xFFFFu;
+                    const uint32_t pair = c1 * t0.y + c0;
+                    asm("mad.wide.u32 %0, %1, %2, %0;" : "+l"(acc) : "r"(pair), "r"(1u << n));
+                    n += (t0.x >> 16) + (t1.x >> 16);
+                    if (n >= 32u) {                        // (two codewords are 32 bits at most: one word per pair)
                         const uint32_t word = (uint32_t)acc;
                         if (have_first) st_stream_u32(w_dst + 4u * wp, word); else w_first = word;
                         have_first = true;
