@@ -87,11 +87,11 @@ def test_altered_directory_gets_the_oracles_verdict(tpc, n_chunks):
     assert len(seen_counts) >= 3                        # single chunks and long runs of them both occurred
 
 
-def test_many_small_chunks_round_trip_and_mask():
-    """4 tiles per chunk, a few thousand chunks: lists of present chunks, offsets and the per-chunk
-    scans at a size where a thread owns several chunks."""
-    chunk = 4 * TILE
-    nc = 2600
+@pytest.mark.parametrize("tpc,nc", [(1, 2100), (3, 1100), (4, 2600)])
+def test_many_small_chunks_round_trip_and_mask(tpc, nc):
+    """A few tiles per chunk, a few thousand chunks: lists of present chunks, offsets and the
+    per-chunk scans at a size where a thread owns several chunks."""
+    chunk = tpc * TILE
     n = nc * chunk - 5000
     a = _cache(n, 77)
     rng = np.random.default_rng(5)
