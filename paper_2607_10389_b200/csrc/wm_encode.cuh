@@ -486,6 +486,11 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
     // its claim and its hand-over, so that the leader never waits for that answer either.
     uint32_t qA = kQNone;              // leader, leaf mode: claimed and described, address on its way
     uint32_t kA = 0;                   // ... and its ticket
+    // With a mask (flat cache) a ticket's tile is found through the list of present chunks.  That
+    // look-up too is started in the step after the claim and used at that step's end, so a ticket
+    // is handed over one step later than without a mask and the leader claims one step further ahead.
+    constexpr bool kLateList = MASKED && !LEAVES;
+    bool haveA = false;                // leader, kLateList: ticket kA is a tile and waits for its chunk number
     if (leader) {
         for (int i = 0; i < 8; i++) tc->wsum[i] = 0;
         mbar_init(&tc->mbar, 1);
@@ -506,6 +511,7 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
             tc->next[1] = with_mark(q1, tc->nptr[1]);
             if (claiming) { kA = next_ticket(ws.ctrl); qA = describe_tile<MASKED>(g, ws.plist, n_tickets, kA); claiming = is_tile(qA); }
         }
+        if (kLateList && claiming) { kA = next_ticket(ws.ctrl); claiming = haveA = kA < n_tickets; }
     }
     team_bar(team);
     qY = tc->next[0];
@@ -543,9 +549,11 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
         unsigned long long pA = 0;
         if (tt == 64u) start_copy(qN, LEAVES ? tc->nptr[par ^ 1u] : tile_src(qN & kQTile));
         if (tt == 96u && is_tile(qV)) pv = ld_relaxed_u32(ws.lbk + place_of((sl + 1u) & 7u, qV & kQTile));
+        uint32_t plA = 0;
         if (leader) {
             if (claiming) tk = next_ticket(ws.ctrl);
             if (LEAVES && is_tile(qA)) pA = tile_src(qA & kQTile);
+            if (kLateList && haveA) plA = __ldg(ws.plist + chunk_of(g, kA));
         }
 
         // ---- Y: digest, exponent ranges, length out, words parked
@@ -815,7 +823,18 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
             if (qX & kQFirst) *reinterpret_cast<unsigned long long*>(dir + 16ull * chunk_of(g, tXn)) = exclX;
             if (place_of(sl, tXn) + 1 == n_tickets) ws.ctrl->payload_total = exclX + enc_len;
         }
-        if (leader) {
+        if (leader && kLateList) {     // hand over the ticket whose chunk number arrived during this step
+            uint32_t qn = kQNone;
+            if (haveA) {
+                const uint32_t j = chunk_of(g, kA);
+                qn = (plA * g.tiles_per_chunk + (kA - j * g.tiles_per_chunk)) | kQPresent | (first_in_chunk(g, kA) ? kQFirst : 0u);
+            }
+            tc->next[par] = qn;
+            tc->kring[(sl + 5u) & 7u] = kA;
+            haveA = claiming && tk < n_tickets;
+            claiming = haveA;
+            kA = tk;
+        } else if (leader) {
             uint32_t qn2 = kQNone;
             if (claiming) { qn2 = describe_tile<MASKED>(g, ws.plist, n_tickets, tk); claiming = is_tile(qn2); }
             // (the tile handed over now is measured two steps on, in ring slot sl + 5)
