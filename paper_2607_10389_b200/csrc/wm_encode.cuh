@@ -194,7 +194,7 @@ struct EncTeamCtl {
                             // slots: one per tile in flight and spares, so that a slot is rewritten
                             // long after its last read)
     uint32_t wdig[8][8];    // per warp: its contribution to the tile digest
-    uint32_t wsum[8];       // sum of widths so far | warps arrived << 16 (the last warp publishes)
+    uint32_t spare8[8];
     uint32_t ssum[8];       // sum of the 32 widths of the slot's tile (set by that last warp), or a mark:
                             // zero tile, constant tile, kSumEnt | words of the streams for a tile stored in ENT form
     uint32_t etab[8][8];    // entropy option, per warp: anchor | words of its stream << 8 (0xFFFF: a strand too long for the form)
@@ -492,7 +492,6 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
     constexpr bool kLateList = MASKED && !LEAVES;
     bool haveA = false;                // leader, kLateList: ticket kA is a tile and waits for its chunk number
     if (leader) {
-        for (int i = 0; i < 8; i++) tc->wsum[i] = 0;
         mbar_init(&tc->mbar, 1);
         const uint32_t k0 = next_ticket(ws.ctrl);
         const uint32_t q0 = describe_tile<MASKED>(g, ws.plist, n_tickets, k0);
@@ -540,6 +539,31 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
         team_bar(team);                   // stage free; what the leader left at the end of the last step is visible
         const uint32_t qN = tc->next[par ^ 1u];
         const unsigned long long exclX = tc->excl[par ^ 1u];
+        // The tile measured in the last step (W now): its 32 widths are complete behind the barrier.
+        // One warp that has no other single-lane chore adds them up and publishes the tile's length
+        // (half a step later than the last-arriving warp could have, which the three steps of slack
+        // before the tile is packed absorb; but no warp waits for a counter in the measuring step
+        // and the sum is off the path of whichever warp was slowest there).
+        if (warp == 6u && is_hot(qW)) {
+            const uint32_t slW = (sl + 2u) & 7u;
+            const uint32_t wt = tc->wtab[slW][lane];
+            const uint32_t total = __reduce_add_sync(0xFFFFFFFFu, (wt >> 8) & 15u);
+            // entropy option: the ENT form is taken when it is shorter than the planes and than raw
+            uint32_t ent_words = 0;
+            if (ENT) ent_words = __reduce_add_sync(0xFFFFFFFFu, lane < 8u ? tc->etab[slW][lane] >> 8 : 0u);
+            const uint32_t plane_len = total <= 253u ? 8256u + 32u * total : kTile;
+            const bool ent_tile = ENT && ent_tile_bytes(ent_words) < plane_len;
+            // unused memory (every warp's first entry carries the mark): no payload
+            // (one value throughout: every warp's first entry carries the mark and they are all alike;
+            // a tile of zeros has no payload, any other value 32 bytes)
+            const uint32_t wt0 = __shfl_sync(0xFFFFFFFFu, wt, 0);
+            const bool const_tile = ZEROS && __all_sync(0xFFFFFFFFu, (lane & 3u) != 0u || ((wt & kWarpConst) != 0u && wt == wt0));
+            const bool zero_tile = const_tile && (wt0 & kWarpAllZero) != 0u;
+            if (lane == 0) {
+                tc->ssum[slW] = zero_tile ? kSumZeroTile : const_tile ? kSumConstTile : ent_tile ? kSumEnt | ent_words : total;
+                publish_len(slW, qW & kQTile, zero_tile ? 0u : const_tile ? 32u : ent_tile ? ent_tile_bytes(ent_words) : plane_len);
+            }
+        }
         // The team's single-lane chores are spread over its warps, because the team waits for
         // whichever warp has the most to do.  Warp 2 starts the copy of the next tile (it has the
         // whole step to arrive).  Two round trips to L2 are started now and used at the end of the
@@ -613,38 +637,12 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
                 if (!__any_sync(0xFFFFFFFFu, diff != 0u))
                     gw[0] |= kWarpConst | ((first & 0xFFu) << 16) | (first == 0u ? kWarpAllZero : 0u);
             }
-            // one lane leaves the warp's results; the warp that arrives last turns the 32 widths
-            // into offsets and publishes the tile's length
-            uint32_t last = 0;
+            // one lane leaves the warp's results; the tile's length is added up and published right
+            // after the next barrier, when all eight warps' widths are there (see the top of the step)
             if (lane == 0) {
                 tc->wdig[slY][warp] = v;
                 *reinterpret_cast<uint4*>(&tc->wtab[slY][4 * warp]) = make_uint4(gw[0], gw[1], gw[2], gw[3]);
                 if (ENT) tc->etab[slY][warp] = ent_w;
-                __threadfence_block();
-                last = (atomicAdd(&tc->wsum[slY], 1u) == 7u) ? 1u : 0u;
-            }
-            if (__shfl_sync(0xFFFFFFFFu, last, 0)) {
-                __threadfence_block();
-                // (kept short: this warp is the one the team's length waits for; the groups'
-                // places inside the tile are worked out by each warp when it packs)
-                const uint32_t wt = *reinterpret_cast<volatile uint32_t*>(&tc->wtab[slY][lane]);
-                const uint32_t total = __reduce_add_sync(0xFFFFFFFFu, (wt >> 8) & 15u);
-                // entropy option: the ENT form is taken when it is shorter than the planes and than raw
-                uint32_t ent_words = 0;
-                if (ENT) ent_words = __reduce_add_sync(0xFFFFFFFFu, lane < 8u ? *reinterpret_cast<volatile uint32_t*>(&tc->etab[slY][lane]) >> 8 : 0u);
-                const uint32_t plane_len = total <= 253u ? 8256u + 32u * total : kTile;
-                const bool ent_tile = ENT && ent_tile_bytes(ent_words) < plane_len;
-                // unused memory (every warp's first entry carries the mark): no payload
-                // (one value throughout: every warp's first entry carries the mark and they are all alike;
-                // a tile of zeros has no payload, any other value 32 bytes)
-                const uint32_t wt0 = __shfl_sync(0xFFFFFFFFu, wt, 0);
-                const bool const_tile = ZEROS && __all_sync(0xFFFFFFFFu, (lane & 3u) != 0u || ((wt & kWarpConst) != 0u && wt == wt0));
-                const bool zero_tile = const_tile && (wt0 & kWarpAllZero) != 0u;
-                if (lane == 0) {
-                    tc->ssum[slY] = zero_tile ? kSumZeroTile : const_tile ? kSumConstTile : ent_tile ? kSumEnt | ent_words : total;
-                    tc->wsum[slY] = 0;
-                    publish_len(slY, tYn, zero_tile ? 0u : const_tile ? 32u : ent_tile ? ent_tile_bytes(ent_words) : plane_len);
-                }
             }
             tmem_store16(tmem_warp + 16u * (step & 3u), d);
         } else if (is_tile(qY)) {
