@@ -340,13 +340,16 @@ __device__ __forceinline__ void tmem_free_all(uint32_t taddr)
 __device__ __forceinline__ void tmem_fence_before_sync() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tmem_fence_after_sync() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
-// 16 registers -> 16 columns of this thread's lane, and back (each waits for its completion).
+// 16 registers -> 16 columns of this thread's lane, and back.  A store is waited for when the
+// next one is issued (a step later) and once more before the memory is handed back: its data is
+// fetched three steps on, with three such waits in between, so nobody stands still for it.
+__device__ __forceinline__ void tmem_wait_stores() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_store16(uint32_t taddr, const uint32_t (&w)[16])
 {
+    tmem_wait_stores();
     asm volatile("tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};"
                  ::"r"(taddr), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3]), "r"(w[4]), "r"(w[5]), "r"(w[6]), "r"(w[7]),
                    "r"(w[8]), "r"(w[9]), "r"(w[10]), "r"(w[11]), "r"(w[12]), "r"(w[13]), "r"(w[14]), "r"(w[15]) : "memory");
-    asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory");
 }
 __device__ __forceinline__ void tmem_load16(uint32_t taddr, uint32_t (&w)[16])
 {

@@ -860,6 +860,7 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
     }
     if ((trouble & 1u) && lane == 0) atomicOr(&ws.ctrl->err, 1u);
     // every warp is done with its tensor memory: hand it back before the block exits
+    tmem_wait_stores();
     tmem_fence_before_sync();
     __syncthreads();
     if (threadIdx.x < 32) tmem_free_all(s_tmem);
