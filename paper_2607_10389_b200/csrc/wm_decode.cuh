@@ -304,6 +304,10 @@ struct DecTeamCtl {
     DecSlot slot[4];             // ring: slot i & 3 belongs to the team's i-th tile
     unsigned long long mbar;     // completion of the bulk copy into the team's stage
     unsigned long long pad;
+    // what the leader asks for about the tile two ahead arrives here (the 16 bytes around its table
+    // entry, around its offset inside its chunk, and its chunk's directory entry): answers that are
+    // a step under way and would otherwise hold registers of every thread for that long
+    uint4 in_tab, in_rel, in_dir;
 };
 static_assert(sizeof(DecTeamCtl) % 16 == 0, "team control block keeps 16-byte alignment");
 
@@ -640,8 +644,7 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
                                              // the previous tile's digest parts complete
         // The leader: next tile's copy; the previous tile's digest; look-ups for the tile two
         // ahead and the ticket of the tile three ahead (answers taken at the end of the step).
-        uint32_t l_e = 0, l_rel = 0, l_tk = kNone;
-        unsigned long long l_po = 0;
+        uint32_t l_tk = kNone;
         // (spread over three warps: the team waits for whichever warp has the most to do)
         if (tt == 64u) start_copy(tc->slot[(it + 1u) & 3u]);
         if (tt == 32u && t_done != kNone) ws.dig[t_done] = xor8(tc->wdig[p ^ 1u]);
@@ -649,9 +652,9 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
         if (leader) {                      // its table entry and offsets
             t_look = tc->slot[(it + 2u) & 3u].t;
             if (t_look < g.n_tiles) {
-                l_e = tab16[t_look];
-                l_rel = __ldcg(ws.rel + t_look);
-                l_po = *reinterpret_cast<const unsigned long long*>(dir + 16ull * chunk_of(g, t_look));
+                cp_async16(&tc->in_tab, tab16 + (t_look & ~7u));
+                cp_async16(&tc->in_rel, ws.rel + (t_look & ~3u));
+                cp_async16(&tc->in_dir, dir + 16ull * chunk_of(g, t_look));
             }
         }
         if (tt == 96u) {                   // the ticket of the tile three ahead
@@ -750,7 +753,11 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
         }
         t_done = have_digest ? t : kNone;
         if (leader && t_look < g.n_tiles) {
+            cp_async_wait_all();
             DecSlot* s2 = &tc->slot[(it + 2u) & 3u];
+            const uint32_t l_e = reinterpret_cast<const volatile unsigned short*>(&tc->in_tab)[t_look & 7u];
+            const uint32_t l_rel = reinterpret_cast<const volatile uint32_t*>(&tc->in_rel)[t_look & 3u];
+            const unsigned long long l_po = *reinterpret_cast<const volatile unsigned long long*>(&tc->in_dir);
             s2->entry = l_e | (first_in_chunk(g, t_look) ? 0x10000u : 0u);
             s2->src = l_po + l_rel;
         }

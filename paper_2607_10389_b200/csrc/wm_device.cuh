@@ -360,6 +360,14 @@ __device__ __forceinline__ void tmem_load16(uint32_t taddr, uint32_t (&w)[16])
     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
 
+// 16 bytes from global to shared memory without a register in between (both 16-byte aligned;
+// past L1).  A thread that has issued some waits for its own with cp_async_wait_all.
+__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gsrc)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"((uint32_t)__cvta_generic_to_shared(smem_dst)), "l"(gsrc) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
+
 // A staged tile's words for this lane: word `lane` of rows 16*warp .. 16*warp+15 (conflict free).
 __device__ __forceinline__ void read_staged_words(const unsigned char* stage, uint32_t warp, uint32_t lane,
                                                   uint32_t (&w)[16])
