@@ -414,9 +414,14 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
     DecTeamCtl* tc = reinterpret_cast<DecTeamCtl*>(S.take(TEAMS * sizeof(DecTeamCtl)));
     if (!S.ok) { if (threadIdx.x == 0) atomicOr(&ws.ctrl->err, 4u); return; }
     tc += team;
-    const unsigned char* const dir = wire + 64;
-    const uint16_t* const tab16 = reinterpret_cast<const uint16_t*>(wire + 64 + 16ull * g.n_chunks);
-    const unsigned char* const payload = wire + g.meta_end;
+    // The image's parts.  Each is needed by one thread of a team once per tile, so they are worked
+    // out from the kernel's arguments where they are used rather than kept in registers of every
+    // thread for the whole loop (`fresh` keeps the compiler from hoisting the sums back out: the
+    // kernel has no register to spare, and a value it spills costs every warp a trip to L2 per tile).
+    auto fresh = [](const unsigned char* p) { asm volatile("" : "+l"(p)); return p; };
+    auto dir_of = [&]() { return fresh(wire) + 64; };
+    auto tab16_of = [&]() { return reinterpret_cast<const uint16_t*>(fresh(wire) + 64 + 16ull * g.n_chunks); };
+    auto payload_of = [&]() { return fresh(wire) + g.meta_end; };
     const bool leader = (tt == 0);
     constexpr uint32_t kNone = 0xFFFFFFFFu;
     // The tile behind a ticket.  Without a mask tickets are tile numbers (one past the last tile:
@@ -447,9 +452,9 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
         sl->t = t;
         sl->entry = 0; sl->src = 0;
         if (t < g.n_tiles) {
-            const uint32_t e = tab16[t];
+            const uint32_t e = tab16_of()[t];
             sl->entry = e | (first_in_chunk(g, t) ? 0x10000u : 0u);
-            if (e) sl->src = *reinterpret_cast<const unsigned long long*>(dir + 16ull * chunk_of(g, t)) + ws.rel[t];
+            if (e) sl->src = *reinterpret_cast<const unsigned long long*>(dir_of() + 16ull * chunk_of(g, t)) + ws.rel[t];
         }
     };
     // staged tiles: full RAW and PACK tiles (everything except absent tiles and the ragged tail)
@@ -459,7 +464,7 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
     auto is_staged = [&](uint32_t e) { return e == 512u || is_pack_entry(e) || is_ent_entry(e); };
     auto start_copy = [&](const DecSlot& sl) {   // leader only
         const uint32_t e = sl.entry & 0xFFFFu;
-        if (sl.t < g.n_tiles && is_staged(e) && !(g.inject & kInjectNoCopy)) bulk_load(stage, payload + sl.src, 32u * (e & 0x7FFFu), &tc->mbar, 0);
+        if (sl.t < g.n_tiles && is_staged(e) && !(g.inject & kInjectNoCopy)) bulk_load(stage, payload_of() + sl.src, 32u * (e & 0x7FFFu), &tc->mbar, 0);
     };
 
     if (leader) {
@@ -626,7 +631,7 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
             uint32_t v = 0;
             if (e == 2u) {
                 // (the value's 32 bytes: the value itself, and 30 bytes that must be zero)
-                const uint32_t* cp = reinterpret_cast<const uint32_t*>(payload + tc->slot[it & 3u].src);
+                const uint32_t* cp = reinterpret_cast<const uint32_t*>(payload_of() + tc->slot[it & 3u].src);
                 const uint32_t x = lane < 8u ? __ldg(cp + lane) : 0u;
                 v = (__shfl_sync(0xFFFFFFFFu, x, 0) & 0xFFFFu) * 0x10001u;
                 if (__any_sync(0xFFFFFFFFu, (lane == 0u ? x >> 16 : x) != 0u)) {       // every warp reaches the same verdict
@@ -652,9 +657,9 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
         if (leader) {                      // its table entry and offsets
             t_look = tc->slot[(it + 2u) & 3u].t;
             if (t_look < g.n_tiles) {
-                cp_async16(&tc->in_tab, tab16 + (t_look & ~7u));
+                cp_async16(&tc->in_tab, tab16_of() + (t_look & ~7u));
                 cp_async16(&tc->in_rel, ws.rel + (t_look & ~3u));
-                cp_async16(&tc->in_dir, dir + 16ull * chunk_of(g, t_look));
+                cp_async16(&tc->in_dir, dir_of() + 16ull * chunk_of(g, t_look));
             }
         }
         if (tt == 96u) {                   // the ticket of the tile three ahead
@@ -668,7 +673,7 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
             unsigned char* o = LEAVES ? reinterpret_cast<unsigned char*>(o_leaf) : dst + (uint64_t)t * kTile;
             bool fold = (ew >> 16) != 0;
             if (e == 0xFFFFu) {
-                const unsigned char* src = payload + tc->slot[it & 3u].src;
+                const unsigned char* src = payload_of() + tc->slot[it & 3u].src;
                 const uint32_t len = g.tail_len;
                 // (leaf mode: the ragged tile has a slot of its own in the side buffer)
                 if (MODE != 1) for (uint32_t i = tt; i < len; i += kTeamThreads) o[i] = src[i];
