@@ -29,7 +29,7 @@ FALLBACK_HBM_GBS = 6650.0
 # DRAM bytes read + written per launch of the encode kernel, from single-pass ncu captures of this
 # benchmark (dram__bytes_read.sum + dram__bytes_write.sum; summaries under profiles/).  A workload
 # without a capture reports null.
-NCU_TRAFFIC_BYTES = {"engine": 1671779840 + 1208417280, "engine_256m": 262412800 + 145585000}
+NCU_TRAFFIC_BYTES = {"engine": 1671721728 + 1208218624, "engine_256m": 262455000 + 145051000}
 
 
 # the headline metric as the baseline file words it; a step is one pass of the whole path:
