@@ -591,32 +591,39 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
                 }
             } else if (ENT != 1) {
                 desc = lds_now_u16(stage_s + 2u * lane);
-                const uint32_t wv = (desc >> 8) & 15u;
-                const uint32_t base_l = desc & 0xFFu, chk = desc >> 12;
-                const bool bad = wv > 8u || chk != (((base_l & 15u) ^ (base_l >> 4) ^ wv ^ 5u) & 15u);
-                const bool anybad = __any_sync(0xFFFFFFFFu, bad);
-                // sum of all 32 widths, and of the widths of the groups before this warp's four
-                const uint32_t Ssum = __reduce_add_sync(0xFFFFFFFFu, wv);
-                const uint32_t before = __reduce_add_sync(0xFFFFFFFFu, lane < 4u * warp ? wv : 0u);
-                const int verdict = anybad ? 1 : (258u + Ssum != e ? 2 : 0);
-                if (verdict) {               // every warp reaches the same verdict
-                    decoded = false;
-                    if (leader) {
+                // Whether the descriptors are sound (step 4) is one warp's business, the one without
+                // a single-lane chore: its verdict goes to the control block and decides the call's
+                // status.  The other warps do not wait for it; they only have to stay inside the
+                // stage whatever they find, so a width the format does not have reads as 8 and an
+                // offset stops where a sound tile's last group can start.  What they unpack from an
+                // unsound tile is garbage in a destination that a failed call leaves unspecified.
+                if (warp == 7u) {
+                    const uint32_t wr = (desc >> 8) & 15u, base_l = desc & 0xFFu, chk = desc >> 12;
+                    const bool bad = wr > 8u || chk != (((base_l & 15u) ^ (base_l >> 4) ^ wr ^ 5u) & 15u);
+                    const bool anybad = __any_sync(0xFFFFFFFFu, bad);
+                    const uint32_t Ssum = __reduce_add_sync(0xFFFFFFFFu, wr);
+                    const int verdict = anybad ? 1 : (258u + Ssum != e ? 2 : 0);
+                    if (verdict && lane == 0) {
                         atomicMin(&ws.ctrl->bad4_key, (unsigned long long)t * 2ull + (verdict == 2 ? 1ull : 0ull));
                         atomicOr(&ws.cflag[chunk_of(g, t)], CF_BAD4);
                     }
-                } else {
+                }
+                // widths of the groups before this warp's four
+                const uint32_t wv = min((desc >> 8) & 15u, 8u);
+                const uint32_t before = __reduce_add_sync(0xFFFFFFFFu, lane < 4u * warp ? wv : 0u);
+                {
                     // lanes 0..3 end up with the descriptors of the warp's four groups, each with its
                     // group's offset in the plane area in the high half
                     const uint32_t own = __shfl_sync(0xFFFFFFFFu, desc, 4 * warp + (lane & 3u)) & 0xFFFFu;
-                    const uint32_t wo = (own >> 8) & 15u;
+                    const uint32_t wo = min((own >> 8) & 15u, 8u);
                     uint32_t off = before;                          // running offset over the four groups
                     const uint32_t w0 = __shfl_sync(0xFFFFFFFFu, wo, 0), w1 = __shfl_sync(0xFFFFFFFFu, wo, 1),
                                    w2 = __shfl_sync(0xFFFFFFFFu, wo, 2);
                     if ((lane & 3u) >= 1u) off += w0;
                     if ((lane & 3u) >= 2u) off += w1;
                     if ((lane & 3u) == 3u) off += w2;
-                    desc = own | (off << 16);
+                    off = min(off, 245u);                           // (8256 + 32 * 245 + 256 bytes of planes end inside the stage)
+                    desc = (own & 0xF0FFu) | (wo << 8) | (off << 16);
 #pragma unroll
                     for (int j = 0; j < 4; j++) {
                         const uint32_t dg = __shfl_sync(0xFFFFFFFFu, desc, j);

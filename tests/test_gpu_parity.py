@@ -231,6 +231,50 @@ def test_single_bit_flips_match_oracle_verdicts(G):
     assert (live.cpu().numpy() == 0x11).all()      # the live buffer is never the decoder's target
 
 
+def test_unsound_descriptors_keep_the_decoder_inside_its_stage(G):
+    """Descriptor blocks overwritten wholesale (all ones: width 15 in every group; widths 8 and
+    valid check bits throughout: a sum the tile cannot have; random bytes): the verdict is the
+    oracle's, nothing faults, the destination's checksums stay as they were and the next call on
+    the same workspace decodes the untouched image.  (Only one warp of a team judges the
+    descriptors; the others read whatever widths they find, clamped so that they stay in bounds.)"""
+    from gpu_util import same_result, to_dev
+    rng = np.random.default_rng(33)
+    n = 9 * TILE + 1000
+    v = (rng.normal(size=n // 2) * 3.0).astype(np.float32)
+    a = (v.view(np.uint32) >> 16).astype("<u2").view(np.uint8).copy()
+    chunk = 4 * TILE
+    g = G(n, chunk)
+    wire, crc, res, wire_dev = g.encode(to_dev(a))
+    want_wire = oracle.encode(a, chunk)[0]
+    assert np.array_equal(wire[: res.wire_len], want_wire)
+    me = oracle.meta_end(n, chunk)
+    tab = np.frombuffer(want_wire[64 + 16 * oracle.num_chunks(n, chunk): me].tobytes(), dtype="<u2")[: oracle.num_tiles(n)]
+    starts = me + np.concatenate([[0], np.cumsum([32 * int(e) if e < 0xFFFF else n % TILE for e in tab])[:-1]])
+    packed = [i for i, e in enumerate(tab) if 258 <= e < 512]
+    assert len(packed) >= 8
+
+    def desc_word(base, w):
+        return base | (w << 8) | ((((base & 15) ^ (base >> 4) ^ w ^ 5) & 15) << 12)
+
+    blocks = {
+        "all ones": np.full(64, 0xFF, np.uint8),
+        "width 8 everywhere, check bits right": np.array([desc_word(100, 8)] * 32, dtype="<u2").view(np.uint8),
+        "width 15 with matching check bits": np.array([desc_word(7, 15)] * 32, dtype="<u2").view(np.uint8),
+        "random": rng.integers(0, 256, 64, dtype=np.uint8),
+    }
+    for name, block in blocks.items():
+        for t in (packed[0], packed[len(packed) // 2], packed[-1]):
+            hw = want_wire.copy()
+            hw[starts[t]: starts[t] + 64] = block
+            want_r = oracle.decode_verify(hw, n, chunk)[2]
+            assert want_r.status_name in ("ERR_DESC", "ERR_STRUCT"), (name, t, want_r.status_name)
+            _, dcrc, r = g.decode(to_dev(np.concatenate([hw, np.zeros((-hw.size) % 16, np.uint8)])), res.wire_len)
+            assert same_result(r, want_r), (name, t, r, want_r)
+            assert not dcrc.any()
+    out, dcrc, r = g.decode(wire_dev, res.wire_len)
+    assert r.ok and np.array_equal(out, a) and np.array_equal(dcrc, crc)
+
+
 def test_truncation_extension_wrong_arguments(G):
     from gpu_util import same_result, to_dev
     rng = np.random.default_rng(5)
