@@ -194,8 +194,8 @@ struct EncTeamCtl {
                             // slots: one per tile in flight and spares, so that a slot is rewritten
                             // long after its last read)
     uint32_t wdig[8][8];    // per warp: its contribution to the tile digest
-    uint32_t spare8[8];
-    uint32_t ssum[8];       // sum of the 32 widths of the slot's tile (set by that last warp), or a mark:
+    uint32_t spare8[8];     // (unused)
+    uint32_t ssum[8];       // sum of the 32 widths of the slot's tile (set by the publishing warp), or a mark:
                             // zero tile, constant tile, kSumEnt | words of the streams for a tile stored in ENT form
     uint32_t etab[8][8];    // entropy option, per warp: anchor | words of its stream << 8 (0xFFFF: a strand too long for the form)
     uint32_t next[2];       // ticket claimed in this step (>= n_tiles: none left), by step parity
@@ -330,14 +330,14 @@ __device__ __forceinline__ uint32_t ent_parse_value(uint32_t buf, uint32_t s, ui
 // Single-pass fused checksum + encode.  Each team keeps four tiles in flight:
 //     X  measured three steps ago, packed and written to the wire image in this step
 //     V, W  measured two / one steps ago, waiting for their offsets
-//     Y  checksummed and measured in this step (its length is published at once)
+//     Y  checksummed and measured in this step (its length is published right after the next barrier)
 // The team owns one 16 KiB stage in shared memory that bulk copies (TMA) fill, one tile per
 // step, each copy started a whole step before its tile is needed.  A measured tile's words
 // (16 registers per lane) are parked in tensor memory until its offset is known, so a tile is
 // read from memory once and nothing waits in registers.  Per step:
-//     take Y's words from the stage | team barrier | start the copy of the next Y |
-//     digest + exponent ranges of Y, publish len(Y) | park Y | fetch X | pack X straight into
-//     the wire image
+//     take Y's words from the stage | team barrier | publish len(W), the tile measured a step
+//     ago | start the copy of the next Y | digest + exponent ranges of Y | park Y | fetch X |
+//     pack X straight into the wire image
 // Meanwhile two round trips to L2 are in flight whose answers are needed a step later: the
 // ticket of the tile to measure two steps on and the offset of the tile to pack next.  These and
 // the other single-lane chores of a step sit on different warps: the team passes one barrier per
