@@ -414,6 +414,17 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
     DecTeamCtl* tc = reinterpret_cast<DecTeamCtl*>(S.take(TEAMS * sizeof(DecTeamCtl)));
     if (!S.ok) { if (threadIdx.x == 0) atomicOr(&ws.ctrl->err, 4u); return; }
     tc += team;
+    // The team's control block by its 32-bit shared-window address.  What every thread does with it
+    // in the loop (its tile's slot, the copy's barrier, a warp's digest part) goes through that
+    // address; the single-thread chores make themselves a pointer from it where they stand.  A
+    // 64-bit pointer kept for the whole loop was the one value the kernel spilled, and it came
+    // back from L2 (the L1 is small beside 225 KiB of shared memory) in every warp, every tile.
+    const uint32_t tc_s = (uint32_t)__cvta_generic_to_shared(tc);
+    auto TC = [&]() {
+        uint32_t a = tc_s;
+        asm volatile("" : "+r"(a));
+        return static_cast<DecTeamCtl*>(__cvta_shared_to_generic((size_t)a));
+    };
     // The image's parts.  Each is needed by one thread of a team once per tile, so they are worked
     // out from the kernel's arguments where they are used rather than kept in registers of every
     // thread for the whole loop (`fresh` keeps the compiler from hoisting the sums back out: the
@@ -464,7 +475,7 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
     auto is_staged = [&](uint32_t e) { return e == 512u || is_pack_entry(e) || is_ent_entry(e); };
     auto start_copy = [&](const DecSlot& sl) {   // leader only
         const uint32_t e = sl.entry & 0xFFFFu;
-        if (sl.t < g.n_tiles && is_staged(e) && !(g.inject & kInjectNoCopy)) bulk_load(stage, payload_of() + sl.src, 32u * (e & 0x7FFFu), &tc->mbar, 0);
+        if (sl.t < g.n_tiles && is_staged(e) && !(g.inject & kInjectNoCopy)) bulk_load(stage, payload_of() + sl.src, 32u * (e & 0x7FFFu), &TC()->mbar, 0);
     };
 
     if (leader) {
@@ -478,13 +489,13 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
     uint32_t phase = 0;
     uint32_t t_done = kNone;           // tile whose digest parts wait in wdig[(it - 1) & 1]
     for (uint32_t it = 0;; it++) {
-        const uint32_t t = tc->slot[it & 3u].t;
+        const uint32_t t = lds_now<offsetof(DecTeamCtl, slot)>(tc_s + 16u * (it & 3u));
         if (t >= g.n_tiles) {
             team_bar(team);
-            if (tt == 32u && t_done != kNone) ws.dig[t_done] = xor8(tc->wdig[(it & 1u) ^ 1u]);
+            if (tt == 32u && t_done != kNone) ws.dig[t_done] = xor8(TC()->wdig[(it & 1u) ^ 1u]);
             break;
         }
-        const uint32_t ew = tc->slot[it & 3u].entry;
+        const uint32_t ew = lds_now<offsetof(DecTeamCtl, slot) + 4>(tc_s + 16u * (it & 3u));
         const uint32_t e = ew & 0xFFFFu;
         // leaf mode: where this tile goes (asked for now, needed when the stores begin)
         const unsigned long long o_leaf = LEAVES ? ws.tptr[t] : 0ull;
@@ -499,7 +510,7 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
 
         // ---- phase 1: everything this lane needs from the stage goes into registers
         if (is_staged(e)) {
-            wait_for_copy<ENT == 0>(&tc->mbar, phase, g.wait_ns, ws.ctrl, (g.inject & kInjectNoCopy) != 0u);
+            wait_for_copy_at<ENT == 0>(tc_s + (uint32_t)offsetof(DecTeamCtl, mbar), phase, g.wait_ns, ws.ctrl, (g.inject & kInjectNoCopy) != 0u);
             phase ^= 1u;
             if (!is_pack) {
                 read_staged_words(stage, warp, lane, w);
@@ -638,7 +649,7 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
             uint32_t v = 0;
             if (e == 2u) {
                 // (the value's 32 bytes: the value itself, and 30 bytes that must be zero)
-                const uint32_t* cp = reinterpret_cast<const uint32_t*>(payload_of() + tc->slot[it & 3u].src);
+                const uint32_t* cp = reinterpret_cast<const uint32_t*>(payload_of() + TC()->slot[it & 3u].src);
                 const uint32_t x = lane < 8u ? __ldg(cp + lane) : 0u;
                 v = (__shfl_sync(0xFFFFFFFFu, x, 0) & 0xFFFFu) * 0x10001u;
                 if (__any_sync(0xFFFFFFFFu, (lane == 0u ? x >> 16 : x) != 0u)) {       // every warp reaches the same verdict
@@ -658,19 +669,19 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
         // ahead and the ticket of the tile three ahead (answers taken at the end of the step).
         uint32_t l_tk = kNone;
         // (spread over three warps: the team waits for whichever warp has the most to do)
-        if (tt == 64u) start_copy(tc->slot[(it + 1u) & 3u]);
-        if (tt == 32u && t_done != kNone) ws.dig[t_done] = xor8(tc->wdig[p ^ 1u]);
+        if (tt == 64u) start_copy(TC()->slot[(it + 1u) & 3u]);
+        if (tt == 32u && t_done != kNone) ws.dig[t_done] = xor8(TC()->wdig[p ^ 1u]);
         uint32_t t_look = kNone;           // warps 0 and 3: the tile claimed a step ago (two tiles ahead)
         if (leader) {                      // its table entry and offsets
-            t_look = tc->slot[(it + 2u) & 3u].t;
+            t_look = TC()->slot[(it + 2u) & 3u].t;
             if (t_look < g.n_tiles) {
-                cp_async16(&tc->in_tab, tab16_of() + (t_look & ~7u));
-                cp_async16(&tc->in_rel, ws.rel + (t_look & ~3u));
-                cp_async16(&tc->in_dir, dir_of() + 16ull * chunk_of(g, t_look));
+                cp_async16(&TC()->in_tab, tab16_of() + (t_look & ~7u));
+                cp_async16(&TC()->in_rel, ws.rel + (t_look & ~3u));
+                cp_async16(&TC()->in_dir, dir_of() + 16ull * chunk_of(g, t_look));
             }
         }
         if (tt == 96u) {                   // the ticket of the tile three ahead
-            t_look = tc->slot[(it + 2u) & 3u].t;
+            t_look = TC()->slot[(it + 2u) & 3u].t;
             if (t_look < g.n_tiles) l_tk = claim();
         }
 
@@ -680,7 +691,7 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
             unsigned char* o = LEAVES ? reinterpret_cast<unsigned char*>(o_leaf) : dst + (uint64_t)t * kTile;
             bool fold = (ew >> 16) != 0;
             if (e == 0xFFFFu) {
-                const unsigned char* src = payload_of() + tc->slot[it & 3u].src;
+                const unsigned char* src = payload_of() + TC()->slot[it & 3u].src;
                 const uint32_t len = g.tail_len;
                 // (leaf mode: the ragged tile has a slot of its own in the side buffer)
                 if (MODE != 1) for (uint32_t i = tt; i < len; i += kTeamThreads) o[i] = src[i];
@@ -743,7 +754,7 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
                 }
                 if (MODE != 2) {
                     const uint32_t v = warp_place(S, __reduce_xor_sync(0xFFFFFFFFu, lane_finish(S, last)), warp, lane);
-                    if (lane == 0) tc->wdig[p][warp] = v;
+                    if (lane == 0) sts_now(tc_s + (uint32_t)offsetof(DecTeamCtl, wdig) + 32u * p + 4u * warp, v);
                     have_digest = true;
                 }
             } else if (decoded) {
@@ -754,7 +765,7 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
                 }
                 if (MODE != 2) {
                     const uint32_t v = tile_digest_part(S, w, fold, warp, lane);
-                    if (lane == 0) tc->wdig[p][warp] = v;
+                    if (lane == 0) sts_now(tc_s + (uint32_t)offsetof(DecTeamCtl, wdig) + 32u * p + 4u * warp, v);
                     have_digest = true;
                 }
             }
@@ -766,14 +777,14 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
         t_done = have_digest ? t : kNone;
         if (leader && t_look < g.n_tiles) {
             cp_async_wait_all();
-            DecSlot* s2 = &tc->slot[(it + 2u) & 3u];
-            const uint32_t l_e = reinterpret_cast<const volatile unsigned short*>(&tc->in_tab)[t_look & 7u];
-            const uint32_t l_rel = reinterpret_cast<const volatile uint32_t*>(&tc->in_rel)[t_look & 3u];
-            const unsigned long long l_po = *reinterpret_cast<const volatile unsigned long long*>(&tc->in_dir);
+            DecSlot* s2 = &TC()->slot[(it + 2u) & 3u];
+            const uint32_t l_e = reinterpret_cast<const volatile unsigned short*>(&TC()->in_tab)[t_look & 7u];
+            const uint32_t l_rel = reinterpret_cast<const volatile uint32_t*>(&TC()->in_rel)[t_look & 3u];
+            const unsigned long long l_po = *reinterpret_cast<const volatile unsigned long long*>(&TC()->in_dir);
             s2->entry = l_e | (first_in_chunk(g, t_look) ? 0x10000u : 0u);
             s2->src = l_po + l_rel;
         }
-        if (tt == 96u) tc->slot[(it + 3u) & 3u].t = l_tk;      // (none once the tickets have run out)
+        if (tt == 96u) TC()->slot[(it + 3u) & 3u].t = l_tk;      // (none once the tickets have run out)
     }
 }
 

@@ -115,6 +115,11 @@ __device__ __forceinline__ uint32_t lds_now_u8(uint32_t addr)
     return v;
 }
 
+__device__ __forceinline__ void sts_now(uint32_t addr, uint32_t v)
+{
+    asm volatile("st.shared.u32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");
+}
+
 // Programmatic dependent launch.  Every call enqueues a short chain of kernels; each kernel but
 // the first is launched with permission to start before its predecessor has finished.  It then
 // sets up what does not depend on the predecessor (tables into shared memory, allocations) and

@@ -108,13 +108,18 @@ __device__ __noinline__ bool wait_for_copy_rest_call(uint32_t b, uint32_t parity
 // OUT_OF_LINE: the rest is a call.  Which form is faster differs from kernel to kernel (it decides
 // how the compiler lays out the hot loop around it); each kernel takes the one measured better.
 template <bool OUT_OF_LINE>
-__device__ __forceinline__ bool wait_for_copy(unsigned long long* bar, uint32_t parity, uint32_t budget_ns, Ctrl* ctrl,
-                                              bool no_second = false)
+__device__ __forceinline__ bool wait_for_copy_at(uint32_t b, uint32_t parity, uint32_t budget_ns, Ctrl* ctrl,
+                                                 bool no_second = false)        // b: the barrier's shared-window address
 {
-    const uint32_t b = (uint32_t)__cvta_generic_to_shared(bar);
     if (mbar_try(b, parity)) return true;
     return OUT_OF_LINE ? wait_for_copy_rest_call(b, parity, budget_ns, ctrl, no_second)
                        : wait_for_copy_rest(b, parity, budget_ns, ctrl, no_second);
+}
+template <bool OUT_OF_LINE>
+__device__ __forceinline__ bool wait_for_copy(unsigned long long* bar, uint32_t parity, uint32_t budget_ns, Ctrl* ctrl,
+                                              bool no_second = false)
+{
+    return wait_for_copy_at<OUT_OF_LINE>((uint32_t)__cvta_generic_to_shared(bar), parity, budget_ns, ctrl, no_second);
 }
 
 struct Ws {
