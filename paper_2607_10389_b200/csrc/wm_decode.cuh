@@ -475,7 +475,7 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
     auto is_staged = [&](uint32_t e) { return e == 512u || is_pack_entry(e) || is_ent_entry(e); };
     auto start_copy = [&](const DecSlot& sl) {   // leader only
         const uint32_t e = sl.entry & 0xFFFFu;
-        if (sl.t < g.n_tiles && is_staged(e) && !(g.inject & kInjectNoCopy)) bulk_load(stage, payload_of() + sl.src, 32u * (e & 0x7FFFu), &TC()->mbar, 0);
+        if (sl.t < g.n_tiles && is_staged(e) && !(g.inject & kInjectNoCopy)) bulk_load_at(stage_s, payload_of() + sl.src, 32u * (e & 0x7FFFu), tc_s + (uint32_t)offsetof(DecTeamCtl, mbar), 0);
     };
 
     if (leader) {
@@ -513,7 +513,7 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
             wait_for_copy_at<ENT == 0>(tc_s + (uint32_t)offsetof(DecTeamCtl, mbar), phase, g.wait_ns, ws.ctrl, (g.inject & kInjectNoCopy) != 0u);
             phase ^= 1u;
             if (!is_pack) {
-                read_staged_words(stage, warp, lane, w);
+                read_staged_words_at(stage_s, warp, lane, w);
             } else if (is_ent) {
                 // ENT tile.  Header: the eight word counts against the entry (structure).  Then lane l
                 // reads strand l of this warp's share: the strands lie one behind the other in the

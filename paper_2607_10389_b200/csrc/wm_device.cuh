@@ -293,6 +293,18 @@ __device__ __forceinline__ void bulk_load(void* smem_dst, const void* gsrc, uint
                      ::"r"(d), "l"(gsrc), "r"(bytes), "r"(b) : "memory");
 }
 
+// The same with both shared-memory places given by their 32-bit shared-window addresses.
+__device__ __forceinline__ void bulk_load_at(uint32_t d, const void* gsrc, uint32_t bytes, uint32_t b, uint64_t policy)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(b), "r"(bytes) : "memory");
+    if (policy)
+        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;"
+                     ::"r"(d), "l"(gsrc), "r"(bytes), "r"(b), "l"(policy) : "memory");
+    else
+        asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                     ::"r"(d), "l"(gsrc), "r"(bytes), "r"(b) : "memory");
+}
+
 // The low 32 bits of the GPU's wall clock in nanoseconds (they wrap every 4.29 s).  Every
 // device-side wait is bounded by TIME against the call's budget (Geo::wait_ns, two seconds unless
 // the caller set another, never more than four), not by a number of polls: a block that shares
@@ -380,6 +392,16 @@ __device__ __forceinline__ void read_staged_words(const unsigned char* stage, ui
     const uint32_t* p = reinterpret_cast<const uint32_t*>(stage) + warp * 512u + lane;
 #pragma unroll
     for (int i = 0; i < 16; i++) w[i] = p[i * 32];
+}
+
+// (the stage given by its 32-bit shared-window address)
+__device__ __forceinline__ void read_staged_words_at(uint32_t stage_s, uint32_t warp, uint32_t lane, uint32_t (&w)[16])
+{
+    const uint32_t p = stage_s + 4u * (warp * 512u + lane);
+    w[0] = lds_now<0>(p);     w[1] = lds_now<128>(p);   w[2] = lds_now<256>(p);   w[3] = lds_now<384>(p);
+    w[4] = lds_now<512>(p);   w[5] = lds_now<640>(p);   w[6] = lds_now<768>(p);   w[7] = lds_now<896>(p);
+    w[8] = lds_now<1024>(p);  w[9] = lds_now<1152>(p);  w[10] = lds_now<1280>(p); w[11] = lds_now<1408>(p);
+    w[12] = lds_now<1536>(p); w[13] = lds_now<1664>(p); w[14] = lds_now<1792>(p); w[15] = lds_now<1920>(p);
 }
 
 // One 32-bit word of a tile of `len` (1..16384) real bytes that is right-aligned in a virtual
