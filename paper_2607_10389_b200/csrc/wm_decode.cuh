@@ -308,6 +308,8 @@ struct DecTeamCtl {
     // entry, around its offset inside its chunk, and its chunk's directory entry): answers that are
     // a step under way and would otherwise hold registers of every thread for that long
     uint4 in_tab, in_rel, in_dir;
+    uint4 in_ptr;                // leaf mode: the 16 bytes around the tile's address in the leaves
+    unsigned long long dstp[4];  // leaf mode, same ring as slot[]: where the tile goes
 };
 static_assert(sizeof(DecTeamCtl) % 16 == 0, "team control block keeps 16-byte alignment");
 
@@ -460,6 +462,7 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
 
     // a tile's entry word and payload offset (blocking: prologue only)
     auto lookup = [&](uint32_t t, DecSlot* sl) {
+        if (LEAVES && t < g.n_tiles) tc->dstp[sl - tc->slot] = ws.tptr[t];
         sl->t = t;
         sl->entry = 0; sl->src = 0;
         if (t < g.n_tiles) {
@@ -497,8 +500,6 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
         }
         const uint32_t ew = lds_now<offsetof(DecTeamCtl, slot) + 4>(tc_s + 16u * (it & 3u));
         const uint32_t e = ew & 0xFFFFu;
-        // leaf mode: where this tile goes (asked for now, needed when the stores begin)
-        const unsigned long long o_leaf = LEAVES ? ws.tptr[t] : 0ull;
         const uint32_t p = it & 1u;
         const bool is_ent = is_ent_entry(e);
         const bool is_pack = is_ent || is_pack_entry(e);            // a coded tile (in either form)
@@ -678,6 +679,7 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
                 cp_async16(&TC()->in_tab, tab16_of() + (t_look & ~7u));
                 cp_async16(&TC()->in_rel, ws.rel + (t_look & ~3u));
                 cp_async16(&TC()->in_dir, dir_of() + 16ull * chunk_of(g, t_look));
+                if (LEAVES) cp_async16(&TC()->in_ptr, ws.tptr + (t_look & ~1u));
             }
         }
         if (tt == 96u) {                   // the ticket of the tile three ahead
@@ -688,6 +690,11 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
         // ---- phase 2: unpack, store, checksum
         bool have_digest = false;
         if (e != 0) {
+            unsigned long long o_leaf = 0ull;
+            if (LEAVES) {
+                const uint2 v = lds_now_v2<offsetof(DecTeamCtl, dstp)>(tc_s + 8u * (it & 3u));
+                o_leaf = v.x | ((unsigned long long)v.y << 32);
+            }
             unsigned char* o = LEAVES ? reinterpret_cast<unsigned char*>(o_leaf) : dst + (uint64_t)t * kTile;
             bool fold = (ew >> 16) != 0;
             if (e == 0xFFFFu) {
@@ -783,6 +790,7 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
             const unsigned long long l_po = *reinterpret_cast<const volatile unsigned long long*>(&TC()->in_dir);
             s2->entry = l_e | (first_in_chunk(g, t_look) ? 0x10000u : 0u);
             s2->src = l_po + l_rel;
+            if (LEAVES) TC()->dstp[(it + 2u) & 3u] = reinterpret_cast<const volatile unsigned long long*>(&TC()->in_ptr)[t_look & 1u];
         }
         if (tt == 96u) TC()->slot[(it + 3u) & 3u].t = l_tk;      // (none once the tickets have run out)
     }
