@@ -115,6 +115,19 @@ __device__ __forceinline__ uint32_t lds_now_u8(uint32_t addr)
     return v;
 }
 
+// Look-ups in tables that do not change once they are set up (no volatile: the compiler may place them)
+__device__ __forceinline__ uint32_t lds_tab_u8(uint32_t addr)
+{
+    uint32_t v;
+    asm("ld.shared.u8 %0, [%1];" : "=r"(v) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ uint32_t lds_tab_u16(uint32_t addr)
+{
+    uint32_t v;
+    asm("{\n\t.reg .u16 t;\n\tld.shared.u16 t, [%1];\n\tcvt.u32.u16 %0, t;\n\t}" : "=r"(v) : "r"(addr));
+    return v;
+}
 __device__ __forceinline__ void sts_now(uint32_t addr, uint32_t v)
 {
     asm volatile("st.shared.u32 [%0], %1;" ::"r"(addr), "r"(v) : "memory");

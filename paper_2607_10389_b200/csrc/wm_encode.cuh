@@ -394,13 +394,6 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
     // that shares its scheduler with busy ones gets too few issue slots to keep up).
     __shared__ uint32_t s_scanner;
     __shared__ uint32_t s_tmem;
-    __shared__ uint2 s_ent[16];        // ENT, by slot: x = codeword | length << 16, y = 1 << length
-    __shared__ unsigned char s_len8[16];   // ENT: length by slot (bytes: the index needs no scaling)
-    if (ENT && threadIdx.x < 11u) {
-        s_ent[threadIdx.x] = make_uint2((threadIdx.x == 10u ? 0xFFFFu : ent_word(threadIdx.x, 0u)) | (ent_length(threadIdx.x) << 16),
-                                        1u << ent_length(threadIdx.x));
-        s_len8[threadIdx.x] = (unsigned char)ent_length(threadIdx.x);
-    }
     Smem S = setup_smem(smem, tab);
     grid_dep_wait();                   // from here on the control block and the length table are ready
     grid_dep_launch();
@@ -424,8 +417,21 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
         if ((uint32_t)i == team) stage = p;
     }
     EncTeamCtl* tc = reinterpret_cast<EncTeamCtl*>(S.take(TEAMS * sizeof(EncTeamCtl)));
+    // ENT: codeword length and codeword by k = E - anchor + 256 (1..511), so that a look-up is the
+    // exponent added to an address the share works out once (no slot arithmetic per element); the
+    // escape's codeword reads 0xFFFF (the packing step lets the exponent through its high byte)
+    unsigned char* const t_lenE = ENT ? S.take(512) : nullptr;
+    unsigned short* const t_cwE = ENT ? reinterpret_cast<unsigned short*>(S.take(1024)) : nullptr;
     if (!S.ok) { if (threadIdx.x == 0) atomicOr(&ws.ctrl->err, 4u); return; }
     tc += team;
+    if (ENT && threadIdx.x < 512u) {
+        const int u = (int)threadIdx.x - 256;
+        const uint32_t slot = (u >= -6 && u <= 3) ? (uint32_t)(u + 6) : 10u;
+        t_lenE[threadIdx.x] = (unsigned char)ent_length(slot);
+        t_cwE[threadIdx.x] = (unsigned short)(slot == 10u ? 0xFFFFu : ent_word(slot, 0u));
+    }
+    const uint32_t lenE_s = ENT ? (uint32_t)__cvta_generic_to_shared(t_lenE) + 256u : 0u;
+    const uint32_t cwE_s = ENT ? (uint32_t)__cvta_generic_to_shared(t_cwE) + 512u : 0u;
 
     // Tensor memory for the tiles in flight: allocated by the block's first warp, the address
     // goes round through shared memory.  Warp w of the block owns lanes 32 (w % 4) .. + 31 and
@@ -600,9 +606,10 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
                 for (int i = 0; i < 16; i++) acc = __dp4a(d[i], 0x01000100u, acc);       // bytes 1 and 3
                 const uint32_t anchor = (__reduce_add_sync(0xFFFFFFFFu, acc) + 512u) >> 10;
                 uint32_t bits = 0;
+                const uint32_t lb = lenE_s - anchor;
 #pragma unroll
                 for (int i = 0; i < 16; i++)
-                    bits += s_len8[ent_slot(__byte_perm(d[i], 0u, 0x4441), anchor)] + s_len8[ent_slot(d[i] >> 24, anchor)];
+                    bits += lds_tab_u8(lb + __byte_perm(d[i], 0u, 0x4441)) + lds_tab_u8(lb + (d[i] >> 24));
                 // (a strand the length byte cannot hold, above 319 bits, keeps the tile out of the form:
                 // the count is then so large that the form is never the shortest)
                 const uint32_t share_bits = __reduce_add_sync(0xFFFFFFFFu, bits);
@@ -716,16 +723,17 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
                 unsigned long long acc = 0;
                 uint32_t n = start & 31u, wp = start >> 5, w_first = 0;
                 bool have_first = false;
+                const uint32_t lb = lenE_s - anchor, cb = cwE_s - 2u * anchor;
 #pragma unroll
                 for (int i = 0; i < 16; i++) {
                     const uint32_t E0 = __byte_perm(d[i], 0u, 0x4441), E1 = d[i] >> 24;
-                    const uint2 t0 = s_ent[ent_slot(E0, anchor)], t1 = s_ent[ent_slot(E1, anchor)];
+                    const uint32_t len0 = lds_tab_u8(lb + E0), len1 = lds_tab_u8(lb + E1);
                     // (the table's escape entry is 0xFFFF: the AND lets the exponent through there only)
-                    const uint32_t c0 = t0.x & __byte_perm(E0, 0xFFu, 0x4404) & 0xFFFFu;
-                    const uint32_t c1 = t1.x & __byte_perm(E1, 0xFFu, 0x4404) & 0xFFFFu;
-                    const uint32_t pair = c1 * t0.y + c0;
+                    const uint32_t c0 = lds_tab_u16(cb + 2u * E0) & __byte_perm(E0, 0xFFu, 0x4404);
+                    const uint32_t c1 = lds_tab_u16(cb + 2u * E1) & __byte_perm(E1, 0xFFu, 0x4404);
+                    const uint32_t pair = c1 * (1u << len0) + c0;
                     asm("mad.wide.u32 %0, %1, %2, %0;" : "+l"(acc) : "r"(pair), "r"(1u << n));
-                    n += (t0.x >> 16) + (t1.x >> 16);
+                    n += len0 + len1;
                     if (n >= 32u) {                        // (two codewords are 32 bits at most: one word per pair)
                         const uint32_t word = (uint32_t)acc;
                         if (have_first) st_stream_u32(w_dst + 4u * wp, word); else w_first = word;
