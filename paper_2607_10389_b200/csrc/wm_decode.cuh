@@ -396,11 +396,14 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
     // ENT: what the low byte of a strand's bits says about the codeword there: its length (16: the
     // escape) and u as a byte.  Two byte tables: the index needs no scaling and a look-up gives a
     // clean value.
-    __shared__ unsigned short s_ptab[ENT ? 256 : 2];       // length | u << 8 (length 16: the escape)
+    // (256-byte aligned: the window's low byte OR'ed into the table's address is the look-up's address)
+    __shared__ __align__(256) unsigned char s_ptab[ENT ? 512 : 4];       // [0..255] length (16: the escape), [256..511] u
     if (ENT != 0 && threadIdx.x < 256u) {
         const uint32_t s = ent_ones(threadIdx.x);
-        s_ptab[threadIdx.x] = (unsigned short)(ent_parse_length(s) | (s == 8u ? 0u : (ent_parse_value(threadIdx.x, s, 0u) & 0xFFu) << 8));
+        s_ptab[threadIdx.x] = (unsigned char)ent_parse_length(s);
+        s_ptab[256u + threadIdx.x] = (unsigned char)(s == 8u ? 0u : ent_parse_value(threadIdx.x, s, 0u));
     }
+    const uint32_t ptab_s = (uint32_t)__cvta_generic_to_shared(s_ptab);
     Smem S = setup_smem(smem, tab);
     grid_dep_wait();
     grid_dep_launch();
@@ -560,9 +563,9 @@ k_decode(const unsigned char* __restrict__ wire, Geo g, unsigned char* __restric
                             avail += 32u;
                             next++;
                         }
-                        const uint32_t tv = s_ptab[lo & 0xFFu];
-                        const uint32_t len = tv & 31u;
-                        const uint32_t E = len == 16u ? lo >> 8 : anchor + (tv >> 8);      // (its low byte)
+                        const uint32_t at = (lo & 0xFFu) | ptab_s;
+                        const uint32_t len = lds_tab_u8(at);
+                        const uint32_t E = len == 16u ? lo >> 8 : anchor + lds_tab_u8(at + 256u);      // (its low byte)
                         ew[i >> 2] = __byte_perm(ew[i >> 2], E, (i & 3) == 0 ? 0x3214 : (i & 3) == 1 ? 0x3240 : (i & 3) == 2 ? 0x3410 : 0x4210);
                         lo = __funnelshift_r(lo, hi, len);
                         hi >>= len;
