@@ -806,9 +806,10 @@ k_encode(const unsigned char* __restrict__ cache, Geo g, const uint8_t* __restri
 
         // What is left to note about X is done by two other warps' first lanes (the leader's
         // warp is the one the team waits for): the digest by warp 1; the table entry, where its
-        // chunk starts and the total by warp 4.
+        // chunk starts and the total by warp 7 (not warp 4: warps w and w + 4 issue through the same
+        // scheduler, and warp 4 would share the end of the step with the leader's hand-over).
         if (tt == 32u && qX >= kQPresent && is_tile(qX)) ws.dig[tXn] = xor8(tc->wdig[sl]);
-        if (tt == 128u && is_tile(qX)) {
+        if (tt == 224u && is_tile(qX)) {
             uint32_t entry = 0, enc_len = 0;
             if (qX >= kQPresent) {
                 if (tXn < g.n_full_tiles) {
